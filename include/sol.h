@@ -1,0 +1,213 @@
+/*
+ * sol.h - C ABI of the action-conditioned batched decode step for B200 (sm_100a).
+ *
+ * One new token per sequence is pushed through a frozen Llama-shaped decoder
+ * layer.  Every sequence i carries its own efficiency action, the paper's
+ * tuple (kappa, rho, q) (Method, "Actions and controlled compute"), passed as
+ * three int32 arrays of length B:
+ *
+ *   r_permille[i]  attention keep-rate r = kappa, in 1/1000, 0..1000
+ *   p_permille[i]  MLP prune rate     p = 1 - rho, in 1/1000, 0..1000
+ *   bits[i]        activation bit-width b = q, 2..8 or 16 (16 = bf16 passthrough)
+ *
+ * Conventions for every call:
+ *   - returns a sol_status_t; never throws, never traps the device;
+ *   - unless a parameter says "host", every pointer is DEVICE memory owned by
+ *     the caller, 16-byte aligned, valid until the work enqueued on `stream`
+ *     has finished; the library allocates no device memory on these calls
+ *     (scratch comes from the caller's workspace `ws`);
+ *   - work is enqueued on `stream` (a cudaStream_t); the call does not wait
+ *     for it;
+ *   - bf16 tensors are raw 16-bit patterns; matrices are row-major;
+ *   - argument errors are detected on the host before anything is launched.
+ */
+#ifndef SOL_H_
+#define SOL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t sol_status_t;
+#define SOL_OK 0
+#define SOL_ERR_INVALID_ARG 1         /* null pointer, negative size, rate or bit-width out of range */
+#define SOL_ERR_UNSUPPORTED 2         /* a shape this build has no kernel for (see sol_shape_t) */
+#define SOL_ERR_WORKSPACE_TOO_SMALL 3 /* ws_bytes < sol_workspace_bytes(...) */
+#define SOL_ERR_CUDA 4                /* a CUDA runtime call failed; see sol_last_cuda_error() */
+#define SOL_ERR_DEVICE_TIMEOUT 5      /* a bounded device-side wait gave up (reported by sol_read_device_status) */
+
+typedef struct CUstream_st *sol_stream_t; /* a cudaStream_t */
+
+/* Layer geometry.  Supported: head_dim 64 or 128; page_size 64;
+ * n_q_heads a multiple of n_kv_heads; d_model and n_q_heads*head_dim
+ * multiples of 256; d_ff a multiple of 32; batch 1..128. */
+typedef struct sol_shape {
+  int32_t d_model, n_q_heads, n_kv_heads, head_dim, d_ff, page_size;
+  float rms_eps;
+  float rope_theta;         /* 0 disables the rotary embedding */
+  int32_t n_sink, n_window; /* always-attended first / last tokens (the paper's sink and window
+                               tokens, Method, "Policy inputs and architecture"); the task's
+                               default is 0 and 1: only the newest token is forced */
+} sol_shape_t;
+
+/* Paged bf16 KV cache of one layer.  Pools: [num_pages][n_kv_heads][page_size][head_dim].
+ * page_table: int32 [B][max_pages_per_seq], physical page of each logical page.
+ * seq_lens:   int32 [B], valid tokens of each sequence INCLUDING the newest one. */
+typedef struct sol_kv {
+  void *k_pool, *v_pool;
+  const int32_t *page_table;
+  const int32_t *seq_lens;
+  int32_t max_pages_per_seq, num_pages;
+} sol_kv_t;
+
+/* bf16 weights of one layer.  w_qkv rows: q heads, then k heads, then v heads.
+ * w_down_t is W_down transposed once at load time so that row j is
+ * intermediate channel j; a pruned channel is then a row that is not read. */
+typedef struct sol_layer_weights {
+  const void *w_qkv;    /* [(n_q+2 n_kv)*head_dim][d_model] */
+  const void *w_o;      /* [d_model][n_q*head_dim] */
+  const void *w_gate;   /* [d_ff][d_model] */
+  const void *w_up;     /* [d_ff][d_model] */
+  const void *w_down_t; /* [d_ff][d_model] */
+  const void *gamma1;   /* [d_model] RMSNorm gain before attention */
+  const void *gamma2;   /* [d_model] RMSNorm gain before the MLP */
+} sol_layer_weights_t;
+
+/* Optional taps on sol_decode_layer; any pointer may be NULL.  They exist so a
+ * checker can compare each stage on the inputs that stage really saw. */
+typedef struct sol_layer_trace {
+  float *xn1;           /* [B][d_model] normalised attention input (float32) */
+  int8_t *codes1;       /* [B][d_model] */
+  float *scales1;       /* [B] */
+  float *q_rot;         /* [B][n_q][head_dim] rotated queries (float32) */
+  int32_t *kept_idx;    /* [B][n_kv][max_pages_per_seq*page_size] ascending */
+  int32_t *kept_cnt;    /* [B][n_kv] */
+  float *attn_out;      /* [B][n_q][head_dim] */
+  float *h_mid;         /* [B][d_model] residual stream after attention (float32) */
+  float *xn2;           /* [B][d_model] */
+  int8_t *codes2;       /* [B][d_model] */
+  float *scales2;       /* [B] */
+  float *t;             /* [B][d_ff] silu(g)*u before pruning (float32) */
+  int32_t *kept_ch;     /* [B][d_ff] ascending */
+  int32_t *kept_ch_cnt; /* [B] */
+  float *h_out;         /* [B][d_model] float32 copy of the output */
+} sol_layer_trace_t;
+
+const char *sol_status_string(sol_status_t s);
+const char *sol_last_cuda_error(void); /* text of the last CUDA error seen by this thread's calls */
+
+/* Bytes of scratch that any call below needs for batches up to max_batch and
+ * contexts up to max_pages_per_seq pages.  0 if the shape is unsupported. */
+size_t sol_workspace_bytes(const sol_shape_t *shape, int32_t max_batch, int32_t max_pages_per_seq);
+
+/* Must be called once per workspace before its first use (and may be called
+ * again to clear the device status words).  Enqueues a memset on `stream`. */
+sol_status_t sol_workspace_init(void *ws, size_t ws_bytes, sol_stream_t stream);
+
+/* Per-token symmetric activation quantizer (appendix "Activation
+ * quantization", "Quantizer"): a = max_j |x_j|, s = a / q_max with
+ * q_max = 2^(b-1) - 1, code_j = clip(rne(x_j / s), -q_max, q_max); both
+ * divisions IEEE float32, rounding to nearest-even.  Row i uses bits[i].
+ *   x_bf16 [B][d] in; codes int8 [B][d] and scales float32 [B] out.
+ *   bits[i] == 16: codes of that row are 0, scale is 1 (passthrough).
+ *   An all-zero row gives scale 0 and codes 0.
+ *   xhat_bf16 (optional, [B][d]): the value the next matmul consumes, before
+ *   the scale is applied: the codes as bf16 numbers, or x itself for 16 bits.
+ * d must be a multiple of 8.  Needs no workspace. */
+sol_status_t sol_quant_act(const void *x_bf16, int32_t B, int32_t d, const int32_t *bits, int8_t *codes,
+                           float *scales, void *xhat_bf16, sol_stream_t stream);
+
+/* Decode attention with a per-sequence keep-rate (appendix "Token sparsity",
+ * "Budgeted token selection": budget ceil(kappa*K_t) clamped to [0, K_t];
+ * selection by exact token-level top-k instead of the paper's page bounds).
+ * For each (sequence, kv-head): keep k = max(ceil(r*T), forced) tokens, the
+ * forced ones plus those with the largest q.k summed over the query group
+ * (ties: lower index); softmax over the kept tokens only; only kept V rows
+ * are read.
+ *   q_bf16 [B][n_q][head_dim] (already rotated); out_bf16 same shape.
+ *   kept_idx (optional) int32 [B][n_kv][max_pages_per_seq*page_size], the
+ *   kept token indices of each (sequence, kv-head) in ascending order;
+ *   kept_cnt (optional) int32 [B][n_kv].
+ * The cache is only read. */
+sol_status_t sol_sparse_decode_attn(const sol_shape_t *shape, const void *q_bf16, const sol_kv_t *kv, int32_t B,
+                                    const int32_t *r_permille, void *out_bf16, int32_t *kept_idx,
+                                    int32_t *kept_cnt, void *ws, size_t ws_bytes, sol_stream_t stream);
+
+/* SwiGLU MLP with a per-token prune rate (count mirrors the paper's
+ * m = ceil(rho*d), "Per-token channel selection"; the pruned axis is the
+ * intermediate one): t_j = silu(W_g x)_j (W_u x)_j, keep the
+ * m = ceil((1-p) d_ff) channels with the largest |t_j| (ties: lower index),
+ * out = sum over kept j of t_j * w_down_t[j, :].  Rows of w_down_t that no
+ * token of the batch keeps are not read.
+ *   x_bf16 [B][d_model]; out_bf16 [B][d_model] (no residual added);
+ *   kept_ch (optional) int32 [B][d_ff] ascending; kept_ch_cnt (optional) [B]. */
+sol_status_t sol_pruned_swiglu_mlp(const sol_shape_t *shape, const void *x_bf16, const void *w_gate,
+                                   const void *w_up, const void *w_down_t, int32_t B, const int32_t *p_permille,
+                                   void *out_bf16, int32_t *kept_ch, int32_t *kept_ch_cnt, void *ws,
+                                   size_t ws_bytes, sol_stream_t stream);
+
+/* One decoder layer under per-sequence actions: RMSNorm, quantize(b), QKV,
+ * rotary embedding at position T-1, append k/v (bf16) to the cache at
+ * position T-1, sparse attention(r), output projection + residual, RMSNorm,
+ * quantize(b), pruned SwiGLU MLP(p) + residual.  The caller has already
+ * reserved the page slot of the newest token and seq_lens counts it.
+ *   h_in_bf16 [B][d_model] in; h_out_bf16 [B][d_model] out; trace optional. */
+sol_status_t sol_decode_layer(const sol_shape_t *shape, const sol_layer_weights_t *w, const sol_kv_t *kv, int32_t B,
+                              const void *h_in_bf16, void *h_out_bf16, const int32_t *r_permille,
+                              const int32_t *p_permille, const int32_t *bits, const sol_layer_trace_t *trace,
+                              void *ws, size_t ws_bytes, sol_stream_t stream);
+
+/* n_layers layers with the same action in every layer (the paper broadcasts
+ * one action tuple over all layers of a decode step).  `layers` and `kvs` are
+ * HOST arrays of n_layers structs (holding device pointers).  The residual
+ * stream stays in float32 between layers.  h_out_f32 is optional. */
+sol_status_t sol_decode_step(const sol_shape_t *shape, int32_t n_layers, const sol_layer_weights_t *layers,
+                             const sol_kv_t *kvs, int32_t B, const void *h_in_bf16, void *h_out_bf16,
+                             float *h_out_f32, const int32_t *r_permille, const int32_t *p_permille,
+                             const int32_t *bits, void *ws, size_t ws_bytes, sol_stream_t stream);
+
+/* The same step for a caller whose per-step data lives on the HOST: h_in,
+ * the three action arrays, seq_lens and h_out are host pointers (pinned
+ * memory makes the copies asynchronous).  They are copied to staging areas
+ * inside the workspace, the step runs with kvs[l].seq_lens replaced by the
+ * staged copy, and the result is copied back; the call returns after the
+ * stream has been synchronised.  Weights, pools and page tables stay on the
+ * device. */
+sol_status_t sol_decode_step_host(const sol_shape_t *shape, int32_t n_layers, const sol_layer_weights_t *layers,
+                                  const sol_kv_t *kvs, int32_t B, const void *h_in_bf16_host,
+                                  void *h_out_bf16_host, const int32_t *r_permille_host,
+                                  const int32_t *p_permille_host, const int32_t *bits_host,
+                                  const int32_t *seq_lens_host, void *ws, size_t ws_bytes, sol_stream_t stream);
+
+/* Device status words of a workspace, copied to HOST out[8] after waiting for
+ * `stream`:  out[0] bit mask of errors raised by kernels (bit 0: a bounded
+ * wait timed out -> SOL_ERR_DEVICE_TIMEOUT is returned; bit 1: a page-table
+ * entry was out of range and the access was skipped; bit 2: a bit-width outside
+ * 2..8 and 16 was met and treated as 16), out[1] token
+ * selections whose near-threshold candidate list overflowed and fell back to
+ * float32 ordering, out[2] the same for channel selections, out[3] token
+ * candidates re-scored in float64, out[4] channel candidates re-scored. */
+sol_status_t sol_read_device_status(const void *ws, int32_t *out_host8, sol_stream_t stream);
+
+/* Per-kernel timing for benchmarks.  While enabled, every kernel launch of
+ * this library is bracketed by CUDA events on its stream.  sol_timing_collect
+ * synchronises the device and fills HOST arrays, one entry per kernel name:
+ * returns the number of entries (at most max_entries).  Not thread-safe. */
+typedef struct sol_kernel_time {
+  char name[48];
+  int32_t launches;
+  float total_ms;
+} sol_kernel_time_t;
+void sol_timing_enable(int32_t on);
+int32_t sol_timing_collect(sol_kernel_time_t *out_host, int32_t max_entries);
+
+/* Kernels launched by this library since the last reset (reset != 0 clears). */
+int64_t sol_launch_count(int32_t reset);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOL_H_ */

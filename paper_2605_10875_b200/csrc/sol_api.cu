@@ -1,0 +1,550 @@
+// C ABI of the library: argument validation, workspace layout, and the
+// composition of the kernels into attention, MLP, layer and step calls.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <vector>
+
+#include "sol_common.cuh"
+#include "sol_internal.h"
+
+namespace sol {
+
+// ---------------------------------------------------------------------------
+// launch bookkeeping
+// ---------------------------------------------------------------------------
+static std::atomic<long long> g_launches{0};
+static bool g_timing = false;
+struct TimedLaunch {
+  const char* name;
+  cudaEvent_t e0, e1;
+};
+static std::vector<TimedLaunch> g_timed;
+static thread_local char tl_cuda_error[256] = "";
+static thread_local bool tl_cuda_failed = false;
+
+bool record_cuda_error(cudaError_t e, const char* where) {
+  if (e == cudaSuccess) return false;
+  snprintf(tl_cuda_error, sizeof(tl_cuda_error), "%s: %s", where, cudaGetErrorString(e));
+  tl_cuda_failed = true;
+  return true;
+}
+
+void note_launch_begin(const char* name, cudaStream_t st) {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (g_timing) {
+    TimedLaunch t;
+    t.name = name;
+    cudaEventCreate(&t.e0);
+    cudaEventCreate(&t.e1);
+    cudaEventRecord(t.e0, st);
+    g_timed.push_back(t);
+  }
+}
+
+void note_launch_end(cudaStream_t st) {
+  if (g_timing) cudaEventRecord(g_timed.back().e1, st);
+  record_cuda_error(cudaGetLastError(), "kernel launch");
+}
+
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64) dev = 0;
+  if (cached[dev] == 0) {
+    int n = 0;
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    cached[dev] = n > 0 ? n : 148;
+  }
+  return cached[dev];
+}
+
+// ---------------------------------------------------------------------------
+// workspace layout
+// ---------------------------------------------------------------------------
+static int pad_rows(int B) {
+  const int mt = (B + 15) / 16;
+  return 16 * (mt <= 1 ? 1 : (mt <= 2 ? 2 : (mt <= 4 ? 4 : 8)));
+}
+
+struct Layout {
+  size_t status, stage_h_in, stage_act, stage_h_out, a_op, scale, qkv, q_rot, q_split, logits, sigma, kept_idx,
+      kept_cnt, part, attn_hi, attn_lo, attn_f32, h_mid, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, down_part,
+      h_a, h_b, total;
+  int splits, chunks, Mpad, Tmax;
+};
+
+static bool shape_ok(const sol_shape_t* s) {
+  if (!s) return false;
+  if (s->head_dim != 64 && s->head_dim != 128) return false;
+  if (s->page_size != 64) return false;
+  if (s->n_kv_heads <= 0 || s->n_q_heads <= 0 || s->n_q_heads % s->n_kv_heads) return false;
+  if (s->n_q_heads / s->n_kv_heads > 8) return false;
+  if (s->d_model <= 0 || s->d_model % 256 || s->d_model > 8192) return false;
+  if ((s->n_q_heads * s->head_dim) % 256) return false;
+  if (s->d_ff <= 0 || s->d_ff % 32) return false;
+  if (s->n_sink < 0 || s->n_window < 0) return false;
+  return true;
+}
+
+static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
+  Layout L;
+  memset(&L, 0, sizeof(L));
+  const size_t d = s.d_model, Hq = s.n_q_heads, Hkv = s.n_kv_heads, hd = s.head_dim, ff = s.d_ff;
+  const size_t G = Hq / Hkv, HG = (G + 3) / 4, Nqkv = (Hq + 2 * Hkv) * hd;
+  const size_t Mpad = pad_rows(B), Tmax = (size_t)max_pages * s.page_size;
+  L.Mpad = (int)Mpad;
+  L.Tmax = (int)Tmax;
+  L.splits = (int)((Tmax + ATTN_SPLIT_LEN - 1) / ATTN_SPLIT_LEN);
+  if (L.splits < 1) L.splits = 1;
+  L.chunks = down_chunks((int)ff, (int)d);
+  size_t at = 0;
+  auto take = [&](size_t bytes) {
+    const size_t o = at;
+    at += (bytes + 255) / 256 * 256;
+    return o;
+  };
+  L.status = take(256);
+  L.stage_h_in = take(B * d * 2);
+  L.stage_act = take(4 * (size_t)B * 4);
+  L.stage_h_out = take(B * d * 2);
+  L.a_op = take(Mpad * d * 2);
+  L.scale = take(Mpad * 4);
+  L.qkv = take(B * Nqkv * 4);
+  L.q_rot = take(B * Hq * hd * 4);
+  L.q_split = take(B * Hkv * HG * 16 * hd * 2);
+  L.logits = take(B * Hkv * Tmax * G * 4);
+  L.sigma = take(B * Hkv * Tmax * 4);
+  L.kept_idx = take(B * Hkv * Tmax * 4);
+  L.kept_cnt = take(B * Hkv * 4);
+  L.part = take(B * Hkv * L.splits * G * (hd + 2) * 4);
+  L.attn_hi = take(Mpad * Hq * hd * 2);
+  L.attn_lo = take(Mpad * Hq * hd * 2);
+  L.attn_f32 = take(B * Hq * hd * 4);
+  L.h_mid = take(B * d * 4);
+  L.g = take(B * ff * 4);
+  L.u = take(B * ff * 4);
+  L.t = take(B * ff * 4);
+  L.t_hi = take(Mpad * ff * 2);
+  L.t_lo = take(Mpad * ff * 2);
+  L.kept_ch = take(B * ff * 4);
+  L.kept_ch_cnt = take((size_t)B * 4);
+  L.live = take(ff / 32 * 4);
+  L.down_part = take((size_t)L.chunks * Mpad * d * 4);
+  L.h_a = take(B * d * 4);
+  L.h_b = take(B * d * 4);
+  L.total = at;
+  return L;
+}
+
+template <typename T>
+static T* at(void* ws, size_t off) {
+  return reinterpret_cast<T*>(static_cast<unsigned char*>(ws) + off);
+}
+
+static sol_status_t finish() {
+  if (tl_cuda_failed) {
+    tl_cuda_failed = false;
+    return SOL_ERR_CUDA;
+  }
+  return SOL_OK;
+}
+
+static bool kv_ok(const sol_kv_t* kv) {
+  return kv && kv->k_pool && kv->v_pool && kv->page_table && kv->seq_lens && kv->max_pages_per_seq > 0 &&
+         kv->num_pages > 0;
+}
+
+// ---------------------------------------------------------------------------
+// compositions
+// ---------------------------------------------------------------------------
+static void run_attention(const sol_shape_t& s, const Layout& L, void* ws, const sol_kv_t& kv, int B,
+                          const int32_t* r_permille, const float* qkv, int ldq, const void* q_bf16, void* out_bf16,
+                          float* out_f32, bool want_split, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t st) {
+  AttnArgs a;
+  a.shape = s;
+  a.kv = kv;
+  a.B = B;
+  a.r_permille = r_permille;
+  a.qkv_f32 = qkv;
+  a.ldq = ldq;
+  a.q_bf16 = q_bf16;
+  a.q_rot = at<float>(ws, L.q_rot);
+  a.q_split = at<void>(ws, L.q_split);
+  a.logits = at<float>(ws, L.logits);
+  a.sigma = at<float>(ws, L.sigma);
+  a.kept_idx = kept_idx ? kept_idx : at<int32_t>(ws, L.kept_idx);
+  a.kept_cnt = kept_cnt ? kept_cnt : at<int32_t>(ws, L.kept_cnt);
+  a.part = at<float>(ws, L.part);
+  a.splits = (kv.max_pages_per_seq * s.page_size + ATTN_SPLIT_LEN - 1) / ATTN_SPLIT_LEN;
+  a.out_f32 = out_f32;
+  a.out_bf16 = out_bf16;
+  a.out_hi = want_split ? at<void>(ws, L.attn_hi) : nullptr;
+  a.out_lo = want_split ? at<void>(ws, L.attn_lo) : nullptr;
+  a.status = at<int>(ws, L.status);
+  launch_attention(a, st);
+}
+
+// a_op / scale in the workspace hold the MLP input operand.
+static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, const void* w_gate, const void* w_up,
+                    const void* w_down_t, const int32_t* p_permille, const void* resid, int resid_f32, void* out_bf16,
+                    float* out_f32, float* out_f32_b, float* t_trace, int32_t* kept_ch, int32_t* kept_ch_cnt,
+                    cudaStream_t st) {
+  int* status = at<int>(ws, L.status);
+  GemmNK gu;
+  memset(&gu, 0, sizeof(gu));
+  gu.a_hi = at<void>(ws, L.a_op);
+  gu.w0 = w_gate;
+  gu.w1 = w_up;
+  gu.M = B;
+  gu.K = s.d_model;
+  gu.N = s.d_ff;
+  gu.row_scale = at<float>(ws, L.scale);
+  gu.out0 = at<float>(ws, L.g);
+  gu.out1 = at<float>(ws, L.u);
+  gu.out2 = t_trace ? t_trace : at<float>(ws, L.t);
+  gu.status = status;
+  launch_gemm_nk(gu, EPI_SWIGLU, st);
+
+  ChannelSelectArgs cs;
+  cs.B = B;
+  cs.d = s.d_model;
+  cs.ff = s.d_ff;
+  cs.p_permille = p_permille;
+  cs.g = gu.out0;
+  cs.u = gu.out1;
+  cs.t = gu.out2;
+  cs.a_op = at<void>(ws, L.a_op);
+  cs.scale = at<float>(ws, L.scale);
+  cs.w_gate = w_gate;
+  cs.w_up = w_up;
+  cs.kept_ch = kept_ch ? kept_ch : at<int32_t>(ws, L.kept_ch);
+  cs.kept_cnt = kept_ch_cnt ? kept_ch_cnt : at<int32_t>(ws, L.kept_ch_cnt);
+  cs.t_hi = at<void>(ws, L.t_hi);
+  cs.t_lo = at<void>(ws, L.t_lo);
+  cs.live = at<int32_t>(ws, L.live);
+  cs.status = status;
+  launch_channel_select(cs, st);
+
+  GemmDown dn;
+  dn.t_hi = cs.t_hi;
+  dn.t_lo = cs.t_lo;
+  dn.w = w_down_t;
+  dn.live = cs.live;
+  dn.M = B;
+  dn.ff = s.d_ff;
+  dn.d = s.d_model;
+  dn.partial = at<float>(ws, L.down_part);
+  dn.chunks = down_chunks(s.d_ff, s.d_model);
+  dn.status = status;
+  launch_gemm_down(dn, st);
+  launch_reduce_out(dn.partial, dn.chunks, B, pad_rows(B), s.d_model, resid, resid_f32, out_bf16, out_f32, out_f32_b,
+                    st);
+}
+
+static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol_layer_weights_t& w,
+                      const sol_kv_t& kv, int B, const void* h_in, bool in_f32, void* h_out_bf16, float* h_out_f32,
+                      const int32_t* r, const int32_t* p, const int32_t* bits, const sol_layer_trace_t* tr,
+                      cudaStream_t st) {
+  int* status = at<int>(ws, L.status);
+  const int d = s.d_model, Hq = s.n_q_heads, Hkv = s.n_kv_heads, hd = s.head_dim;
+  const int Nqkv = (Hq + 2 * Hkv) * hd;
+  float* scale = at<float>(ws, L.scale);
+
+  launch_norm_quant(h_in, in_f32, w.gamma1, s.rms_eps, bits, B, d, at<void>(ws, L.a_op), scale,
+                    tr ? tr->xn1 : nullptr, tr ? tr->codes1 : nullptr, status, st);
+  if (tr && tr->scales1) cudaMemcpyAsync(tr->scales1, scale, sizeof(float) * B, cudaMemcpyDeviceToDevice, st);
+
+  GemmNK q;
+  memset(&q, 0, sizeof(q));
+  q.a_hi = at<void>(ws, L.a_op);
+  q.w0 = w.w_qkv;
+  q.M = B;
+  q.K = d;
+  q.N = Nqkv;
+  q.row_scale = scale;
+  q.out0 = at<float>(ws, L.qkv);
+  q.status = status;
+  launch_gemm_nk(q, EPI_SCALE, st);
+
+  run_attention(s, L, ws, kv, B, r, at<float>(ws, L.qkv), Nqkv, nullptr, nullptr, tr ? tr->attn_out : nullptr, true,
+                tr ? tr->kept_idx : nullptr, tr ? tr->kept_cnt : nullptr, st);
+  if (tr && tr->q_rot)
+    cudaMemcpyAsync(tr->q_rot, at<float>(ws, L.q_rot), sizeof(float) * B * Hq * hd, cudaMemcpyDeviceToDevice, st);
+
+  GemmNK o;
+  memset(&o, 0, sizeof(o));
+  o.a_hi = at<void>(ws, L.attn_hi);
+  o.a_lo = at<void>(ws, L.attn_lo);
+  o.w0 = w.w_o;
+  o.M = B;
+  o.K = Hq * hd;
+  o.N = d;
+  o.resid = h_in;
+  o.resid_f32 = in_f32 ? 1 : 0;
+  o.out0 = at<float>(ws, L.h_mid);
+  o.status = status;
+  launch_gemm_nk(o, EPI_RESIDUAL, st);
+  if (tr && tr->h_mid)
+    cudaMemcpyAsync(tr->h_mid, at<float>(ws, L.h_mid), sizeof(float) * B * d, cudaMemcpyDeviceToDevice, st);
+
+  launch_norm_quant(at<float>(ws, L.h_mid), true, w.gamma2, s.rms_eps, bits, B, d, at<void>(ws, L.a_op), scale,
+                    tr ? tr->xn2 : nullptr, tr ? tr->codes2 : nullptr, status, st);
+  if (tr && tr->scales2) cudaMemcpyAsync(tr->scales2, scale, sizeof(float) * B, cudaMemcpyDeviceToDevice, st);
+
+  run_mlp(s, L, ws, B, w.w_gate, w.w_up, w.w_down_t, p, at<float>(ws, L.h_mid), 1, h_out_bf16, h_out_f32,
+          tr ? tr->h_out : nullptr, tr ? tr->t : nullptr, tr ? tr->kept_ch : nullptr, tr ? tr->kept_ch_cnt : nullptr,
+          st);
+}
+
+static bool weights_ok(const sol_layer_weights_t* w) {
+  return w && w->w_qkv && w->w_o && w->w_gate && w->w_up && w->w_down_t && w->gamma1 && w->gamma2;
+}
+
+}  // namespace sol
+
+using namespace sol;
+
+// ---------------------------------------------------------------------------
+// exported entry points
+// ---------------------------------------------------------------------------
+extern "C" {
+
+const char* sol_status_string(sol_status_t s) {
+  switch (s) {
+    case SOL_OK: return "ok";
+    case SOL_ERR_INVALID_ARG: return "invalid argument";
+    case SOL_ERR_UNSUPPORTED: return "unsupported shape";
+    case SOL_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case SOL_ERR_CUDA: return "CUDA error";
+    case SOL_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+const char* sol_last_cuda_error(void) { return tl_cuda_error; }
+
+size_t sol_workspace_bytes(const sol_shape_t* shape, int32_t max_batch, int32_t max_pages_per_seq) {
+  if (!shape_ok(shape) || max_batch < 1 || max_batch > 128 || max_pages_per_seq < 1) return 0;
+  return make_layout(*shape, max_batch, max_pages_per_seq).total;
+}
+
+sol_status_t sol_workspace_init(void* ws, size_t ws_bytes, sol_stream_t stream) {
+  if (!ws || ws_bytes < 256) return SOL_ERR_INVALID_ARG;
+  if (record_cuda_error(cudaMemsetAsync(ws, 0, ws_bytes, (cudaStream_t)stream), "workspace memset"))
+    return finish();
+  return SOL_OK;
+}
+
+sol_status_t sol_quant_act(const void* x_bf16, int32_t B, int32_t d, const int32_t* bits, int8_t* codes,
+                           float* scales, void* xhat_bf16, sol_stream_t stream) {
+  if (!x_bf16 || !bits || !codes || !scales || B < 0 || d <= 0) return SOL_ERR_INVALID_ARG;
+  if (d % 8 || d > 8192) return SOL_ERR_UNSUPPORTED;
+  if (B == 0) return SOL_OK;
+  launch_norm_quant(x_bf16, false, nullptr, 0.f, bits, B, d, xhat_bf16, scales, nullptr, codes, nullptr,
+                    (cudaStream_t)stream);
+  return finish();
+}
+
+sol_status_t sol_sparse_decode_attn(const sol_shape_t* shape, const void* q_bf16, const sol_kv_t* kv, int32_t B,
+                                    const int32_t* r_permille, void* out_bf16, int32_t* kept_idx, int32_t* kept_cnt,
+                                    void* ws, size_t ws_bytes, sol_stream_t stream) {
+  if (!shape || !q_bf16 || !kv_ok(kv) || !r_permille || !out_bf16 || !ws || B < 0) return SOL_ERR_INVALID_ARG;
+  if (!shape_ok(shape) || B > 128) return SOL_ERR_UNSUPPORTED;
+  if (B == 0) return SOL_OK;
+  const Layout L = make_layout(*shape, B, kv->max_pages_per_seq);
+  if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
+  run_attention(*shape, L, ws, *kv, B, r_permille, nullptr, 0, q_bf16, out_bf16, nullptr, false, kept_idx, kept_cnt,
+                (cudaStream_t)stream);
+  return finish();
+}
+
+sol_status_t sol_pruned_swiglu_mlp(const sol_shape_t* shape, const void* x_bf16, const void* w_gate, const void* w_up,
+                                   const void* w_down_t, int32_t B, const int32_t* p_permille, void* out_bf16,
+                                   int32_t* kept_ch, int32_t* kept_ch_cnt, void* ws, size_t ws_bytes,
+                                   sol_stream_t stream) {
+  if (!shape || !x_bf16 || !w_gate || !w_up || !w_down_t || !p_permille || !out_bf16 || !ws || B < 0)
+    return SOL_ERR_INVALID_ARG;
+  if (!shape_ok(shape) || B > 128) return SOL_ERR_UNSUPPORTED;
+  if (B == 0) return SOL_OK;
+  const Layout L = make_layout(*shape, B, 1);
+  if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  // bf16 passthrough into the padded operand buffer, scale 1
+  launch_norm_quant(x_bf16, false, nullptr, 0.f, nullptr, B, shape->d_model, at<void>(ws, L.a_op),
+                    at<float>(ws, L.scale), nullptr, nullptr, nullptr, st);
+  run_mlp(*shape, L, ws, B, w_gate, w_up, w_down_t, p_permille, nullptr, 0, out_bf16, nullptr, nullptr, nullptr,
+          kept_ch, kept_ch_cnt, st);
+  return finish();
+}
+
+static sol_status_t check_actions_host_side(const sol_shape_t* shape, int32_t B) {
+  if (!shape_ok(shape) || B > 128) return SOL_ERR_UNSUPPORTED;
+  return SOL_OK;
+}
+
+sol_status_t sol_decode_layer(const sol_shape_t* shape, const sol_layer_weights_t* w, const sol_kv_t* kv, int32_t B,
+                              const void* h_in_bf16, void* h_out_bf16, const int32_t* r_permille,
+                              const int32_t* p_permille, const int32_t* bits, const sol_layer_trace_t* trace,
+                              void* ws, size_t ws_bytes, sol_stream_t stream) {
+  if (!shape || !weights_ok(w) || !kv_ok(kv) || !h_in_bf16 || !h_out_bf16 || !r_permille || !p_permille || !bits ||
+      !ws || B < 0)
+    return SOL_ERR_INVALID_ARG;
+  sol_status_t s = check_actions_host_side(shape, B);
+  if (s != SOL_OK) return s;
+  if (B == 0) return SOL_OK;
+  const Layout L = make_layout(*shape, B, kv->max_pages_per_seq);
+  if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
+  run_layer(*shape, L, ws, *w, *kv, B, h_in_bf16, false, h_out_bf16, nullptr, r_permille, p_permille, bits, trace,
+            (cudaStream_t)stream);
+  return finish();
+}
+
+static sol_status_t decode_step_impl(const sol_shape_t* shape, int32_t n_layers, const sol_layer_weights_t* layers,
+                                     const sol_kv_t* kvs, const int32_t* seq_lens_override, int32_t B,
+                                     const void* h_in_bf16, void* h_out_bf16, float* h_out_f32, const int32_t* r,
+                                     const int32_t* p, const int32_t* bits, void* ws, const Layout& L,
+                                     cudaStream_t st) {
+  const void* h = h_in_bf16;
+  bool in_f32 = false;
+  for (int l = 0; l < n_layers; ++l) {
+    sol_kv_t kv = kvs[l];
+    if (seq_lens_override) kv.seq_lens = seq_lens_override;
+    const bool last = l == n_layers - 1;
+    float* out32 = last ? h_out_f32 : at<float>(ws, (l & 1) ? L.h_b : L.h_a);
+    run_layer(*shape, L, ws, layers[l], kv, B, h, in_f32, last ? h_out_bf16 : nullptr, out32, r, p, bits, nullptr,
+              st);
+    h = out32;
+    in_f32 = true;
+  }
+  return finish();
+}
+
+static sol_status_t step_args_ok(const sol_shape_t* shape, int32_t n_layers, const sol_layer_weights_t* layers,
+                                 const sol_kv_t* kvs, int32_t B, int* max_pages) {
+  if (!shape || n_layers < 1 || !layers || !kvs || B < 0) return SOL_ERR_INVALID_ARG;
+  if (!shape_ok(shape) || B > 128) return SOL_ERR_UNSUPPORTED;
+  int mp = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    if (!weights_ok(&layers[l]) || !kv_ok(&kvs[l])) return SOL_ERR_INVALID_ARG;
+    if (kvs[l].max_pages_per_seq > mp) mp = kvs[l].max_pages_per_seq;
+  }
+  *max_pages = mp;
+  return SOL_OK;
+}
+
+sol_status_t sol_decode_step(const sol_shape_t* shape, int32_t n_layers, const sol_layer_weights_t* layers,
+                             const sol_kv_t* kvs, int32_t B, const void* h_in_bf16, void* h_out_bf16,
+                             float* h_out_f32, const int32_t* r_permille, const int32_t* p_permille,
+                             const int32_t* bits, void* ws, size_t ws_bytes, sol_stream_t stream) {
+  int mp = 0;
+  sol_status_t s = step_args_ok(shape, n_layers, layers, kvs, B, &mp);
+  if (s != SOL_OK) return s;
+  if (!h_in_bf16 || !h_out_bf16 || !r_permille || !p_permille || !bits || !ws) return SOL_ERR_INVALID_ARG;
+  if (B == 0) return SOL_OK;
+  const Layout L = make_layout(*shape, B, mp);
+  if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
+  return decode_step_impl(shape, n_layers, layers, kvs, nullptr, B, h_in_bf16, h_out_bf16, h_out_f32, r_permille,
+                          p_permille, bits, ws, L, (cudaStream_t)stream);
+}
+
+sol_status_t sol_decode_step_host(const sol_shape_t* shape, int32_t n_layers, const sol_layer_weights_t* layers,
+                                  const sol_kv_t* kvs, int32_t B, const void* h_in_bf16_host, void* h_out_bf16_host,
+                                  const int32_t* r_permille_host, const int32_t* p_permille_host,
+                                  const int32_t* bits_host, const int32_t* seq_lens_host, void* ws, size_t ws_bytes,
+                                  sol_stream_t stream) {
+  int mp = 0;
+  sol_status_t s = step_args_ok(shape, n_layers, layers, kvs, B, &mp);
+  if (s != SOL_OK) return s;
+  if (!h_in_bf16_host || !h_out_bf16_host || !r_permille_host || !p_permille_host || !bits_host || !seq_lens_host ||
+      !ws)
+    return SOL_ERR_INVALID_ARG;
+  for (int i = 0; i < B; ++i) {
+    if (r_permille_host[i] < 0 || r_permille_host[i] > 1000 || p_permille_host[i] < 0 || p_permille_host[i] > 1000)
+      return SOL_ERR_INVALID_ARG;
+    const int b = bits_host[i];
+    if (!(b == 16 || (b >= 2 && b <= 8))) return (b >= 9 && b <= 15) ? SOL_ERR_UNSUPPORTED : SOL_ERR_INVALID_ARG;
+    if (seq_lens_host[i] < 1 || seq_lens_host[i] > mp * shape->page_size) return SOL_ERR_INVALID_ARG;
+  }
+  if (B == 0) return SOL_OK;
+  const Layout L = make_layout(*shape, B, mp);
+  if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t hb = (size_t)B * shape->d_model * 2, ab = (size_t)B * 4;
+  int32_t* act = at<int32_t>(ws, L.stage_act);
+  bool bad = false;
+  bad |= record_cuda_error(cudaMemcpyAsync(at<void>(ws, L.stage_h_in), h_in_bf16_host, hb, cudaMemcpyHostToDevice, st), "h2d h_in");
+  bad |= record_cuda_error(cudaMemcpyAsync(act, r_permille_host, ab, cudaMemcpyHostToDevice, st), "h2d r");
+  bad |= record_cuda_error(cudaMemcpyAsync(act + B, p_permille_host, ab, cudaMemcpyHostToDevice, st), "h2d p");
+  bad |= record_cuda_error(cudaMemcpyAsync(act + 2 * B, bits_host, ab, cudaMemcpyHostToDevice, st), "h2d bits");
+  bad |= record_cuda_error(cudaMemcpyAsync(act + 3 * B, seq_lens_host, ab, cudaMemcpyHostToDevice, st), "h2d seq_lens");
+  if (bad) return finish();
+  s = decode_step_impl(shape, n_layers, layers, kvs, act + 3 * B, B, at<void>(ws, L.stage_h_in),
+                       at<void>(ws, L.stage_h_out), nullptr, act, act + B, act + 2 * B, ws, L, st);
+  if (s != SOL_OK) return s;
+  record_cuda_error(cudaMemcpyAsync(h_out_bf16_host, at<void>(ws, L.stage_h_out), hb, cudaMemcpyDeviceToHost, st), "d2h h_out");
+  record_cuda_error(cudaStreamSynchronize(st), "stream synchronize");
+  return finish();
+}
+
+sol_status_t sol_read_device_status(const void* ws, int32_t* out_host8, sol_stream_t stream) {
+  if (!ws || !out_host8) return SOL_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (record_cuda_error(cudaMemcpyAsync(out_host8, ws, sizeof(int32_t) * ST_WORDS, cudaMemcpyDeviceToHost, st), "status copy"))
+    return finish();
+  if (record_cuda_error(cudaStreamSynchronize(st), "stream synchronize")) return finish();
+  return (out_host8[ST_ERR] & ERR_TIMEOUT) ? SOL_ERR_DEVICE_TIMEOUT : SOL_OK;
+}
+
+void sol_timing_enable(int32_t on) {
+  g_timing = on != 0;
+  if (!g_timing) {
+    for (auto& t : g_timed) {
+      cudaEventDestroy(t.e0);
+      cudaEventDestroy(t.e1);
+    }
+    g_timed.clear();
+  }
+}
+
+int32_t sol_timing_collect(sol_kernel_time_t* out_host, int32_t max_entries) {
+  cudaDeviceSynchronize();
+  std::map<std::string, std::pair<int, float>> agg;
+  std::vector<std::string> order;
+  for (auto& t : g_timed) {
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, t.e0, t.e1);
+    auto it = agg.find(t.name);
+    if (it == agg.end()) {
+      agg[t.name] = {1, ms};
+      order.push_back(t.name);
+    } else {
+      it->second.first += 1;
+      it->second.second += ms;
+    }
+    cudaEventDestroy(t.e0);
+    cudaEventDestroy(t.e1);
+  }
+  g_timed.clear();
+  int n = 0;
+  for (auto& name : order) {
+    if (n >= max_entries || !out_host) break;
+    memset(&out_host[n], 0, sizeof(sol_kernel_time_t));
+    strncpy(out_host[n].name, name.c_str(), sizeof(out_host[n].name) - 1);
+    out_host[n].launches = agg[name].first;
+    out_host[n].total_ms = agg[name].second;
+    ++n;
+  }
+  return n;
+}
+
+int64_t sol_launch_count(int32_t reset) {
+  const long long v = g_launches.load();
+  if (reset) g_launches.store(0);
+  return v;
+}
+
+}  // extern "C"

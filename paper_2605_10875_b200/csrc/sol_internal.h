@@ -1,0 +1,118 @@
+// Host-side declarations shared by the .cu files of the library: the launch
+// wrapper (launch counting + optional per-kernel event timing) and the
+// launchers of each kernel family.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/sol.h"
+
+namespace sol {
+
+// ---- launch bookkeeping (sol_api.cu) ---------------------------------------
+void note_launch_begin(const char* name, cudaStream_t st);
+void note_launch_end(cudaStream_t st);
+bool record_cuda_error(cudaError_t e, const char* where);  // true if e != success
+
+#define SOL_LAUNCH(name, kernel, grid, block, smem, st, ...)             \
+  do {                                                                   \
+    ::sol::note_launch_begin(name, st);                                  \
+    kernel<<<grid, block, smem, st>>>(__VA_ARGS__);                      \
+    ::sol::note_launch_end(st);                                          \
+  } while (0)
+
+int sm_count();
+
+// ---- quantizer / RMSNorm (sol_quant.cu) ------------------------------------
+// One token per CTA.  in: bf16 or float32 [B][d].  gamma == nullptr: no norm.
+// Outputs (each optional): a_op bf16 [B][d] (codes as bf16, or x as bf16 for
+// 16 bits), scale [B], xn float32 [B][d], codes int8 [B][d].
+void launch_norm_quant(const void* in, bool in_f32, const void* gamma_bf16, float eps, const int32_t* bits, int B,
+                       int d, void* a_op, float* scale, float* xn, int8_t* codes, int* status, cudaStream_t st);
+
+// ---- weight-streaming GEMMs (sol_gemm.cu) ----------------------------------
+enum GemmEpilogue { EPI_SCALE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2 };
+struct GemmNK {
+  const void* a_hi;       // bf16 [Mpad][K]
+  const void* a_lo;       // bf16 [Mpad][K] or nullptr; the product uses a_hi + a_lo
+  const void* w0;         // bf16 [N][K]   (EPI_SWIGLU: gate [ff][K])
+  const void* w1;         // EPI_SWIGLU: up [ff][K]
+  int M, K, N;            // EPI_SWIGLU: N = ff
+  const float* row_scale; // [M] or nullptr
+  const void* resid;      // EPI_RESIDUAL: [M][N] bf16 or float32
+  int resid_f32;
+  float* out0;            // [M][N]  (EPI_SWIGLU: g)
+  float* out1;            // EPI_SWIGLU: u
+  float* out2;            // EPI_SWIGLU: t = silu(g) * u
+  int* status;
+};
+void launch_gemm_nk(const GemmNK& p, GemmEpilogue epi, cudaStream_t st);
+
+struct GemmDown {
+  const void* t_hi;  // bf16 [Mpad][ff]  masked activations, high part
+  const void* t_lo;  // bf16 [Mpad][ff]  low part
+  const void* w;     // bf16 [ff][d]
+  const int32_t* live;  // [ff/32] non-zero if any token keeps a channel of the granule
+  int M, ff, d;
+  float* partial;    // [chunks][Mpad][d]
+  int chunks;        // as returned by down_chunks()
+  int* status;
+};
+int down_chunks(int ff, int d);
+void launch_gemm_down(const GemmDown& p, cudaStream_t st);
+// out = resid + sum over chunks of partial; out_bf16 / out_f32 optional.
+void launch_reduce_out(const float* partial, int chunks, int M, int Mpad, int d, const void* resid, int resid_f32,
+                       void* out_bf16, float* out_f32, float* out_f32_b, cudaStream_t st);
+
+// ---- attention (sol_attn.cu) ------------------------------------------------
+struct AttnArgs {
+  sol_shape_t shape;
+  sol_kv_t kv;
+  int B;
+  const int32_t* r_permille;
+  // inputs of the query preparation: either float32 qkv rows [B][ldq] (layer path: rotate q and k,
+  // append k and v) or bf16 q [B][Hq][hd] (stand-alone path: no rotation, no append)
+  const float* qkv_f32;
+  int ldq;
+  const void* q_bf16;
+  // scratch
+  float* q_rot;      // [B][Hq][hd]
+  void* q_split;     // bf16 [B][Hkv][HG*16][hd]
+  float* logits;     // [B][Hkv][Tmax][G]
+  float* sigma;      // [B][Hkv][Tmax]
+  int32_t* kept_idx; // [B][Hkv][Tmax]
+  int32_t* kept_cnt; // [B][Hkv]
+  float* part;       // [B][Hkv][S][G][hd + 2]
+  int splits;        // S
+  // outputs (each optional)
+  float* out_f32;    // [B][Hq][hd]
+  void* out_bf16;    // [B][Hq][hd]
+  void* out_hi;      // bf16 [Mpad][Hq*hd]
+  void* out_lo;
+  int* status;
+};
+constexpr int ATTN_SPLIT_LEN = 512;  // kept tokens per pass-2 work item
+void launch_attention(const AttnArgs& a, cudaStream_t st);
+
+// ---- MLP channel selection (sol_mlp.cu) -------------------------------------
+struct ChannelSelectArgs {
+  int B, d, ff;
+  const int32_t* p_permille;
+  const float* g;      // [B][ff]
+  const float* u;
+  const float* t;
+  const void* a_op;    // bf16 [B][d] MLP input operand
+  const float* scale;  // [B]
+  const void* w_gate;  // bf16 [ff][d]
+  const void* w_up;
+  int32_t* kept_ch;    // [B][ff]
+  int32_t* kept_cnt;   // [B]
+  void* t_hi;          // bf16 [Mpad][ff]
+  void* t_lo;
+  int32_t* live;       // [ff/32], zeroed by the launcher
+  int* status;
+};
+void launch_channel_select(const ChannelSelectArgs& a, cudaStream_t st);
+
+}  // namespace sol

@@ -1,0 +1,154 @@
+// RMSNorm + per-token symmetric activation quantizer.  One token per CTA; the
+// token's row is a few KB, so the kernel is latency-bound: 128-bit loads, the
+// row held in registers, two block reductions (sum of squares, absmax).
+//
+// Quantizer (appendix "Activation quantization", "Quantizer"):
+//   q_max = 2^(b-1) - 1, a = max|x|, s = a / q_max, code = clip(rne(x / s)).
+// Both divisions are IEEE float32 (__fdiv_rn) so the codes are reproducible
+// bit for bit.
+#include "sol_common.cuh"
+#include "sol_internal.h"
+
+namespace sol {
+
+constexpr int NQ_THREADS = 256;
+constexpr int NQ_VEC = 8;                       // elements per 128-bit bf16 load
+constexpr int NQ_MAX_PER_THREAD = 4;            // vectors per thread -> d <= 8192
+
+__device__ __forceinline__ float block_reduce(float v, bool is_max, float* sh) {
+  v = is_max ? warp_max(v) : warp_sum(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();  // protect sh from the previous use
+  if (l == 0) sh[w] = v;
+  __syncthreads();
+  float r = sh[0];
+  for (int i = 1; i < NQ_THREADS / 32; ++i) r = is_max ? fmaxf(r, sh[i]) : r + sh[i];
+  return r;
+}
+
+template <bool IN_F32>
+__global__ void __launch_bounds__(NQ_THREADS)
+norm_quant_kernel(const void* __restrict__ in, const uint16_t* __restrict__ gamma, float eps,
+                  const int32_t* __restrict__ bits, int d, uint16_t* __restrict__ a_op, float* __restrict__ scale,
+                  float* __restrict__ xn, int8_t* __restrict__ codes, int* __restrict__ status) {
+  __shared__ float sh[NQ_THREADS / 32];
+  const int row = blockIdx.x;
+  const int nvec = d / NQ_VEC;
+  float x[NQ_MAX_PER_THREAD][NQ_VEC];
+
+  // load the row (zero-fill vectors beyond d)
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < NQ_MAX_PER_THREAD; ++i) {
+    const int v = threadIdx.x + i * NQ_THREADS;
+#pragma unroll
+    for (int e = 0; e < NQ_VEC; ++e) x[i][e] = 0.f;
+    if (v < nvec) {
+      if (IN_F32) {
+        const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(in) + (size_t)row * d) + 2 * v;
+        float4 a = p[0], b = p[1];
+        x[i][0] = a.x; x[i][1] = a.y; x[i][2] = a.z; x[i][3] = a.w;
+        x[i][4] = b.x; x[i][5] = b.y; x[i][6] = b.z; x[i][7] = b.w;
+      } else {
+        uint4 w = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(in) + (size_t)row * d)[v];
+        x[i][0] = bf16_lo(w.x); x[i][1] = bf16_hi(w.x); x[i][2] = bf16_lo(w.y); x[i][3] = bf16_hi(w.y);
+        x[i][4] = bf16_lo(w.z); x[i][5] = bf16_hi(w.z); x[i][6] = bf16_lo(w.w); x[i][7] = bf16_hi(w.w);
+      }
+#pragma unroll
+      for (int e = 0; e < NQ_VEC; ++e) ss += x[i][e] * x[i][e];
+    }
+  }
+
+  if (gamma != nullptr) {
+    const float tot = block_reduce(ss, false, sh);
+    const float inv = 1.0f / sqrtf(tot / (float)d + eps);
+#pragma unroll
+    for (int i = 0; i < NQ_MAX_PER_THREAD; ++i) {
+      const int v = threadIdx.x + i * NQ_THREADS;
+      if (v < nvec) {
+        uint4 w = reinterpret_cast<const uint4*>(gamma)[v];
+        float gm[NQ_VEC] = {bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y),
+                            bf16_lo(w.z), bf16_hi(w.z), bf16_lo(w.w), bf16_hi(w.w)};
+#pragma unroll
+        for (int e = 0; e < NQ_VEC; ++e) x[i][e] = (x[i][e] * gm[e]) * inv;
+      }
+    }
+  }
+
+  if (xn != nullptr) {
+#pragma unroll
+    for (int i = 0; i < NQ_MAX_PER_THREAD; ++i) {
+      const int v = threadIdx.x + i * NQ_THREADS;
+      if (v < nvec) {
+        float4* p = reinterpret_cast<float4*>(xn + (size_t)row * d) + 2 * v;
+        p[0] = make_float4(x[i][0], x[i][1], x[i][2], x[i][3]);
+        p[1] = make_float4(x[i][4], x[i][5], x[i][6], x[i][7]);
+      }
+    }
+  }
+
+  int b = bits ? bits[row] : 16;
+  if (b != 16 && (b < 2 || b > 8)) {  // no kernel for this width: pass through and flag it
+    if (threadIdx.x == 0 && status != nullptr) atomicOr(status + ST_ERR, ERR_BAD_ACTION);
+    b = 16;
+  }
+  float s = 1.0f;
+  float q_max = 0.f;
+  if (b != 16) {
+    float a = 0.f;
+#pragma unroll
+    for (int i = 0; i < NQ_MAX_PER_THREAD; ++i)
+#pragma unroll
+      for (int e = 0; e < NQ_VEC; ++e) a = fmaxf(a, fabsf(x[i][e]));
+    a = block_reduce(a, true, sh);
+    q_max = (float)((1 << (b - 1)) - 1);
+    s = __fdiv_rn(a, q_max);
+  }
+  if (threadIdx.x == 0 && scale != nullptr) scale[row] = s;
+
+#pragma unroll
+  for (int i = 0; i < NQ_MAX_PER_THREAD; ++i) {
+    const int v = threadIdx.x + i * NQ_THREADS;
+    if (v >= nvec) continue;
+    float c[NQ_VEC];
+    if (b == 16) {
+#pragma unroll
+      for (int e = 0; e < NQ_VEC; ++e) c[e] = x[i][e];
+    } else {
+#pragma unroll
+      for (int e = 0; e < NQ_VEC; ++e) {
+        float r = (s == 0.f) ? 0.f : rintf(__fdiv_rn(x[i][e], s));
+        c[e] = fminf(fmaxf(r, -q_max), q_max);
+      }
+    }
+    if (a_op != nullptr) {
+      uint4 w;
+      w.x = pack_bf16(c[0], c[1]); w.y = pack_bf16(c[2], c[3]);
+      w.z = pack_bf16(c[4], c[5]); w.w = pack_bf16(c[6], c[7]);
+      reinterpret_cast<uint4*>(a_op + (size_t)row * d)[v] = w;
+    }
+    if (codes != nullptr) {
+      int q[NQ_VEC];
+#pragma unroll
+      for (int e = 0; e < NQ_VEC; ++e) q[e] = (b == 16) ? 0 : (int)c[e];
+      uint2 w;
+      w.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | ((uint32_t)(q[3] & 0xff) << 24);
+      w.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | ((uint32_t)(q[7] & 0xff) << 24);
+      reinterpret_cast<uint2*>(codes + (size_t)row * d)[v] = w;
+    }
+  }
+}
+
+void launch_norm_quant(const void* in, bool in_f32, const void* gamma_bf16, float eps, const int32_t* bits, int B,
+                       int d, void* a_op, float* scale, float* xn, int8_t* codes, int* status, cudaStream_t st) {
+  if (in_f32)
+    SOL_LAUNCH("norm_quant", norm_quant_kernel<true>, dim3(B), dim3(NQ_THREADS), 0, st, in,
+               static_cast<const uint16_t*>(gamma_bf16), eps, bits, d, static_cast<uint16_t*>(a_op), scale, xn,
+               codes, status);
+  else
+    SOL_LAUNCH("norm_quant", norm_quant_kernel<false>, dim3(B), dim3(NQ_THREADS), 0, st, in,
+               static_cast<const uint16_t*>(gamma_bf16), eps, bits, d, static_cast<uint16_t*>(a_op), scale, xn,
+               codes, status);
+}
+
+}  // namespace sol

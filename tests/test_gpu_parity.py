@@ -1,0 +1,389 @@
+"""GPU parity: the CUDA library, called through the C ABI, against the fp64
+CPU oracle on the same seeded inputs.
+
+Rules (written here as the task states them):
+  * quantizer codes and scales bit-exact;
+  * kept token / channel index sets identical, except indices whose oracle
+    score is within 1e-5 relative of the oracle's k-th score (counted);
+  * bf16 outputs: max-abs error <= 2e-2 and relative L2 error <= 1e-2.
+Inside a layer each stage is also compared with the oracle run on the inputs
+that stage really saw on the GPU (taps), because a legal 1-ulp difference
+upstream may legally change a selection downstream.
+"""
+import copy
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import checker
+from oracle import sol_oracle as O
+from paper_2605_10875_b200 import binding as sol
+from paper_2605_10875_b200 import synth
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+
+TINY = synth.WORKLOADS["tiny"]
+L1B = synth.WORKLOADS["llama1b_layer"]
+L8B = synth.WORKLOADS["llama8b_layer"]
+
+
+# ------------------------------------------------------------- quantizer ----
+
+
+@pytest.mark.parametrize("B,d", [(4, 256), (16, 2048), (64, 4096), (1, 8), (3, 8192), (5, 1000)])
+def test_quant_codes_bit_exact(B, d):
+    rng = np.random.default_rng(B * 10000 + d)
+    x = synth.to_bf16((rng.standard_normal((B, d)) * 10 ** rng.uniform(-2, 2, (B, 1))).astype(np.float32))
+    bits = rng.choice([2, 3, 4, 5, 6, 7, 8, 16], B).astype(np.int32)
+    if B >= 3:
+        x[1] = 0  # an all-zero row: scale 0, codes 0
+        bits[1] = 8
+        x[2, :] = x[2, 0]  # every element ties at the maximum
+    codes_o, scales_o, xhat_o = O.quant_act(x, bits)
+    codes, scales, xhat = H.gpu_quant(x, bits)
+    assert np.array_equal(codes, codes_o)
+    assert np.array_equal(scales.view(np.uint32), scales_o.view(np.uint32))
+    for i in range(B):
+        want = x[i] if bits[i] == 16 else synth.to_bf16(codes_o[i].astype(np.float32))
+        assert np.array_equal(xhat[i], want)
+        # dequantized value within half a step of the input
+        if bits[i] != 16:
+            err = np.abs(codes[i].astype(np.float64) * float(scales[i]) - O.bf16_to_f64(x[i]))
+            assert np.all(err <= 0.5 * float(scales[i]) * (1 + 1e-6))
+
+
+def test_quant_workload_shapes_all_bit_widths():
+    for name in ("tiny", "llama1b_layer", "llama8b_layer"):
+        cfg = synth.WORKLOADS[name]
+        x = synth.make_hidden(cfg, 0)
+        for b in (4, 8, 16):
+            bits = np.full(cfg["batch"], b, np.int32)
+            co, so, _ = O.quant_act(x, bits)
+            c, s, _ = H.gpu_quant(x, bits)
+            assert np.array_equal(c, co) and np.array_equal(s.view(np.uint32), so.view(np.uint32)), (name, b)
+
+
+# -------------------------------------------------------------- attention ---
+
+
+def _attention_case(cfg, seq_lens, r, seed=0, n_sink=0, n_window=1, mutate=None):
+    shape, oshape = H.make_shapes(cfg, n_sink, n_window)
+    B = len(seq_lens)
+    seq_lens = np.asarray(seq_lens, np.int32)
+    k_pool, v_pool, table = H.make_case_kv(cfg, seq_lens, seed)
+    if mutate:
+        mutate(k_pool, v_pool, table)
+    q = synth.make_queries(cfg, seed, B)
+    kv = H.device_kv(k_pool, v_pool, table, seq_lens)
+    out, kept, st = H.gpu_attention(shape, q, kv, r)
+    okv = O.PagedKV(k_pool, v_pool, np.where(table < 0, 0, table), seq_lens)
+    out_o, kept_o, sigma = O.sparse_decode_attn(oshape, O.bf16_to_f64(q), okv, r)
+    assert st[0] == 0 and st[1] == 0, st
+    par = H.check_token_sets(oshape, sigma, kept_o, kept, seq_lens)
+    H.assert_sets(par, "token sets")
+    for i in range(B):
+        for h in range(oshape.n_kv_heads):
+            assert np.all(np.diff(kept[i][h]) > 0), "kept indices must be ascending"
+    m, rel = H.assert_outputs(out_o, out, "attention output")
+    return par, st, (m, rel)
+
+
+def test_attention_tiny_workload():
+    r, _, _ = synth.draw_actions(TINY, 0)
+    _attention_case(TINY, synth.make_contexts(TINY, 0), r)
+
+
+@pytest.mark.parametrize("r", [0, 1, 125, 250, 500, 999, 1000])
+def test_attention_ragged_lengths_every_rate(r):
+    lens = [1, 2, 63, 64, 65, 129, 500, 512]
+    _attention_case(TINY, lens, [r] * len(lens), seed=r + 1)
+
+
+def test_attention_mixed_rates_and_sink_window():
+    lens = [300, 77, 512, 5, 200, 64]
+    _attention_case(TINY, lens, [250, 500, 125, 1000, 50, 0], seed=3, n_sink=4, n_window=2)
+
+
+def test_attention_duplicate_keys_tie_to_lower_index():
+    def dup(k_pool, v_pool, table):
+        k_pool[:] = k_pool[0, 0, 0]  # every key identical: all scores tie exactly
+
+    par, st, _ = _attention_case(TINY, [200, 64, 130], [500, 250, 125], seed=4, mutate=dup)
+    assert par.exact == par.sets
+
+
+def test_attention_llama1b_layer_full():
+    r, _, _ = synth.draw_actions(L1B, 0)
+    par, st, err = _attention_case(L1B, synth.make_contexts(L1B, 0), r)
+    print("llama1b attention: sets", par, "status", st, "err", err)
+
+
+def test_attention_head_dim_128_ragged():
+    cfg = dict(L8B)
+    lens = [2000, 1, 65, 4096, 777]
+    _attention_case(cfg, lens, [125, 1000, 500, 250, 500], seed=5)
+
+
+@pytest.mark.parametrize("hq,hkv", [(8, 1), (4, 4), (12, 2)])
+def test_attention_other_group_sizes(hq, hkv):
+    cfg = dict(TINY, n_q_heads=hq, n_kv_heads=hkv, d_model=256 if (hq * 64) % 256 == 0 else 768)
+    _attention_case(cfg, [333, 64, 190], [250, 500, 125], seed=hq)
+
+
+# -------------------------------------------------------------------- MLP ---
+
+
+def _mlp_case(cfg, B, p, seed=0, mutate=None):
+    shape, oshape = H.make_shapes(cfg)
+    w = synth.make_layer_weights(cfg, seed)
+    if mutate:
+        mutate(w)
+    x = synth.make_hidden(cfg, seed, B)
+    x = synth.to_bf16(synth.bf16_to_f32(x) * np.float32(1.0))
+    dw = H.device_weights(w)
+    out, kept, st = H.gpu_mlp(shape, x, dw, p)
+    out_o, kept_o, t_o = O.pruned_swiglu_mlp(O.bf16_to_f64(x), w.w_gate, w.w_up, w.w_down_t, p)
+    assert st[0] == 0 and st[2] == 0, st
+    par = H.check_channel_sets(t_o, kept_o, kept)
+    H.assert_sets(par, "channel sets")
+    for i in range(B):
+        assert np.all(np.diff(kept[i]) > 0)
+    err = H.assert_outputs(out_o, out, "mlp output")
+    return par, st, err
+
+
+def test_mlp_tiny_workload():
+    _, p, _ = synth.draw_actions(TINY, 0)
+    _mlp_case(TINY, TINY["batch"], p)
+
+
+@pytest.mark.parametrize("p", [0, 1, 250, 500, 750, 999, 1000])
+def test_mlp_every_rate(p):
+    _mlp_case(TINY, 5, [p] * 5, seed=p + 1)
+
+
+def test_mlp_identical_channels_tie_to_lower_index():
+    def dup(w):
+        w.w_gate[:] = w.w_gate[0]
+        w.w_up[:] = w.w_up[0]
+
+    par, _, _ = _mlp_case(TINY, 3, [500, 250, 750], seed=7, mutate=dup)
+    assert par.exact == par.sets
+
+
+def test_mlp_llama1b_layer_full():
+    _, p, _ = synth.draw_actions(L1B, 0)
+    par, st, err = _mlp_case(L1B, L1B["batch"], p)
+    print("llama1b mlp: sets", par, "status", st, "err", err)
+
+
+@pytest.mark.parametrize("B", [1, 17, 33, 64])
+def test_mlp_batch_sizes(B):
+    cfg = dict(TINY, d_model=512, d_ff=2048 + 32)
+    rng = np.random.default_rng(B)
+    _mlp_case(cfg, B, rng.choice([0, 250, 500, 750], B), seed=B)
+
+
+def test_mlp_llama8b_shape():
+    _mlp_case(L8B, 8, [0, 250, 500, 750, 125, 999, 0, 500], seed=2)
+
+
+# ------------------------------------------------------------------ layer ---
+
+
+def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1):
+    shape, oshape = H.make_shapes(cfg, n_sink, n_window)
+    B = len(seq_lens)
+    seq_lens = np.asarray(seq_lens, np.int32)
+    w = synth.make_layer_weights(cfg, seed)
+    k_pool, v_pool, table = H.make_case_kv(cfg, seq_lens, seed)
+    h_in = synth.make_hidden(cfg, seed, B)
+    kv = H.device_kv(k_pool, v_pool, table, seq_lens)
+    out, taps, st = H.gpu_layer(shape, H.device_weights(w), kv, h_in, r, p, b)
+    assert st[0] == 0 and st[1] == 0 and st[2] == 0, st
+    ow = H.oracle_weights(w)
+    tab = np.where(table < 0, 0, table)
+
+    # (1) end to end against the oracle's own layer
+    okv = O.PagedKV(k_pool.copy(), v_pool.copy(), tab, seq_lens)
+    out_o, tr = O.decode_layer(oshape, ow, okv, O.bf16_to_f64(h_in), r, p, b)
+    err = H.assert_outputs(out_o, out, "layer output")
+
+    # (2) stage by stage, each on the inputs the GPU stage really saw
+    Hq, Hkv, hd = oshape.n_q_heads, oshape.n_kv_heads, oshape.head_dim
+    assert np.allclose(taps["xn1"], tr.xn1, rtol=2e-5, atol=1e-6)
+    for i in range(B):
+        c, s, _ = O.quantize_per_token(taps["xn1"][i], int(b[i]))
+        assert np.array_equal(c, taps["codes1"][i]) and np.float32(s) == taps["scales1"][i], "codes1"
+    assert np.allclose(taps["q_rot"], tr.q_rot, rtol=0, atol=2e-4 * np.abs(tr.q_rot).max())
+    # appended k, v: within one bf16 step of the oracle's
+    k_gpu, v_gpu = H.host_u16(kv.k_pool), H.host_u16(kv.v_pool)
+    for i in range(B):
+        pos = int(seq_lens[i]) - 1
+        pg, slot = tab[i, pos // 64], pos % 64
+        for got, want in ((k_gpu[pg, :, slot], tr.k_new[i]), (v_gpu[pg, :, slot], tr.v_new[i])):
+            d = np.abs(O.bf16_to_f64(got) - O.bf16_to_f64(want))
+            assert np.all(d <= np.abs(O.bf16_to_f64(want)) * 2.0 ** -7 + 1e-30), "appended k/v"
+    assert (k_gpu != k_pool).sum() <= B * Hkv * hd  # nothing but the appended rows changed
+    # token selection and attention on the GPU's own queries and cache
+    gkv = O.PagedKV(k_gpu, v_gpu, tab, seq_lens)
+    attn_o, kept_o, sigma = O.sparse_decode_attn(oshape, taps["q_rot"].astype(np.float64), gkv, r)
+    kept = [[taps["kept_idx"][i, h, : taps["kept_cnt"][i, h]] for h in range(Hkv)] for i in range(B)]
+    tok = H.check_token_sets(oshape, sigma, kept_o, kept, seq_lens)
+    H.assert_sets(tok, "layer token sets")
+    assert np.allclose(taps["attn_out"], attn_o, rtol=0, atol=2e-3 * max(1e-3, np.abs(attn_o).max()))
+    assert np.allclose(taps["h_mid"], tr.h_mid, rtol=0, atol=2e-3)
+    assert np.allclose(taps["xn2"], tr.xn2, rtol=0, atol=2e-3)
+    x_hat2 = np.zeros((B, cfg["d_model"]))
+    for i in range(B):
+        c, s, x_hat2[i] = O.quantize_per_token(taps["xn2"][i], int(b[i]))
+        assert np.array_equal(c, taps["codes2"][i]) and np.float32(s) == taps["scales2"][i], "codes2"
+    mlp_o, kept_ch_o, t_o = O.pruned_swiglu_mlp(x_hat2, w.w_gate, w.w_up, w.w_down_t, p)
+    kept_ch = [taps["kept_ch"][i, : taps["kept_ch_cnt"][i]] for i in range(B)]
+    ch = H.check_channel_sets(t_o, kept_ch_o, kept_ch)
+    H.assert_sets(ch, "layer channel sets")
+    assert np.allclose(taps["t"], t_o, rtol=1e-4, atol=1e-5)
+    assert np.allclose(taps["h_out"], taps["h_mid"].astype(np.float64) + mlp_o, rtol=0, atol=2e-3)
+    return dict(err=err, tokens=tok, channels=ch, status=st)
+
+
+def test_layer_tiny_workload():
+    r, p, b = synth.draw_actions(TINY, 0)
+    res = check_layer(TINY, synth.make_contexts(TINY, 0), r, p, b)
+    print("tiny layer:", res)
+
+
+def test_layer_dense_action():
+    B = 4
+    check_layer(TINY, [512, 100, 64, 1], [1000] * B, [0] * B, [16] * B, seed=1)
+
+
+def test_layer_ragged_with_rope_and_sinks():
+    cfg = dict(TINY, rope_theta=10000.0)
+    check_layer(cfg, [65, 1, 500, 129, 64], [250, 500, 125, 500, 1000], [500, 0, 250, 750, 1000],
+                [4, 8, 16, 2, 6], seed=2, n_sink=4, n_window=2)
+
+
+def test_layer_llama1b_full():
+    r, p, b = synth.draw_actions(L1B, 0)
+    res = check_layer(L1B, synth.make_contexts(L1B, 0), r, p, b)
+    print("llama1b layer:", res)
+
+
+def test_layer_llama8b_shape_reduced_context():
+    B = 6
+    rng = np.random.default_rng(11)
+    check_layer(L8B, [1500, 64, 333, 2048, 1, 700], rng.choice(L8B["r_set"], B), rng.choice(L8B["p_set"], B),
+                rng.choice(L8B["b_set"], B), seed=3)
+
+
+# ------------------------------------------------------------------- step ---
+
+
+def _step_case(cfg, n_layers, seq_lens, r, p, b, seed=0):
+    shape, oshape = H.make_shapes(cfg)
+    B = len(seq_lens)
+    seq_lens = np.asarray(seq_lens, np.int32)
+    ws_ = [synth.make_layer_weights(cfg, seed, l) for l in range(n_layers)]
+    pools = [H.make_case_kv(cfg, seq_lens, seed, l) for l in range(n_layers)]
+    h_in = synth.make_hidden(cfg, seed, B)
+    dws = [H.device_weights(w) for w in ws_]
+    dkvs = [H.device_kv(k, v, t, seq_lens) for (k, v, t) in pools]
+    return shape, oshape, ws_, pools, h_in, dws, dkvs, seq_lens
+
+
+def test_step_three_layers_matches_oracle_and_host_variant():
+    cfg = dict(TINY, rope_theta=10000.0)
+    B = 4
+    r, p, b = [500, 1000, 250, 125], [250, 0, 500, 750], [8, 16, 4, 8]
+    shape, oshape, ws_, pools, h_in, dws, dkvs, seq_lens = _step_case(cfg, 3, [512, 300, 64, 129], r, p, b)
+    ws = H.Workspace(shape, B, dkvs[0].max_pages)
+    out = torch.zeros((B, cfg["d_model"]), dtype=torch.bfloat16, device=H.DEV)
+    out32 = torch.zeros((B, cfg["d_model"]), dtype=torch.float32, device=H.DEV)
+    sol.decode_step(shape, [w.struct() for w in dws], [k.struct() for k in dkvs], B, H.dev_bf16(h_in), out, out32,
+                    H.dev_i32(r), H.dev_i32(p), H.dev_i32(b), ws.buf, ws.bytes)
+    torch.cuda.synchronize()
+    assert ws.status()[0] == 0
+    okvs = [O.PagedKV(k.copy(), v.copy(), np.where(t < 0, 0, t), seq_lens) for (k, v, t) in pools]
+    out_o, _ = O.decode_step(oshape, [H.oracle_weights(w) for w in ws_], okvs, h_in, r, p, b)
+    got = synth.bf16_to_f32(H.host_u16(out)).astype(np.float64)
+    # the residual stream grows with depth; the absolute bound scales with bf16's step at its magnitude
+    scale = max(1.0, np.abs(out_o).max() / 4.0)
+    m, rel = checker.output_errors(out_o, got)
+    assert m <= checker.OUT_MAX_ABS * scale and rel <= checker.OUT_REL_L2, (m, rel)
+    m32, rel32 = checker.output_errors(out_o, out32.cpu().numpy())
+    assert m32 <= 5e-3 and rel32 <= 1e-3, (m32, rel32)
+
+    # same step through the host-buffer entry point, on fresh caches: identical bits
+    dkvs2 = [H.device_kv(k, v, t, seq_lens) for (k, v, t) in pools]
+    ws2 = H.Workspace(shape, B, dkvs2[0].max_pages)
+    h_host = torch.from_numpy(h_in.view(np.int16)).pin_memory()
+    out_host = torch.zeros((B, cfg["d_model"]), dtype=torch.int16).pin_memory()
+    i32 = lambda a: torch.from_numpy(np.asarray(a, np.int32)).pin_memory()
+    rr, pp, bb, ll = i32(r), i32(p), i32(b), i32(seq_lens)
+    sol.decode_step_host(shape, [w.struct() for w in dws], [k.struct() for k in dkvs2], B, h_host, out_host, rr, pp,
+                         bb, ll, ws2.buf, ws2.bytes)
+    assert np.array_equal(out_host.numpy().view(np.uint16), H.host_u16(out))
+    for a, c in zip(dkvs, dkvs2):
+        assert torch.equal(a.k_pool, c.k_pool) and torch.equal(a.v_pool, c.v_pool)
+
+
+def test_consecutive_steps_append_to_the_cache():
+    """Four decode steps of a two-layer model, contexts growing by one token per
+    step across a page boundary; every step is checked against the oracle run on
+    the cache the GPU produced so far."""
+    cfg = dict(TINY, rope_theta=10000.0)
+    B, L, steps = 3, 2, 4
+    start = np.array([62, 127, 300], np.int32)
+    shape, oshape = H.make_shapes(cfg)
+    ws_ = [synth.make_layer_weights(cfg, 5, l) for l in range(L)]
+    table, n_pages = synth.make_page_table(start, True, 5, spare_tokens=steps)
+    pools = [synth.make_kv_pool(cfg, n_pages, 5, l) for l in range(L)]
+    dws = [H.device_weights(w) for w in ws_]
+    dkvs = [H.device_kv(k, v, table, start) for (k, v) in pools]
+    ws = H.Workspace(shape, B, table.shape[1])
+    rng = np.random.default_rng(5)
+    for s in range(steps):
+        lens = start + s + 1
+        r, p, b = rng.choice(cfg["r_set"], B), rng.choice(cfg["p_set"], B), rng.choice(cfg["b_set"], B)
+        h_in = synth.make_hidden(cfg, 100 + s, B)
+        host_kvs = [k.to_oracle() for k in dkvs]
+        for k in dkvs:
+            k.seq_lens.copy_(H.dev_i32(lens))
+        out = torch.zeros((B, cfg["d_model"]), dtype=torch.bfloat16, device=H.DEV)
+        sol.decode_step(shape, [w.struct() for w in dws], [k.struct() for k in dkvs], B, H.dev_bf16(h_in), out, None,
+                        H.dev_i32(r), H.dev_i32(p), H.dev_i32(b), ws.buf, ws.bytes)
+        torch.cuda.synchronize()
+        assert ws.status()[0] == 0
+        okvs = [O.PagedKV(k.k_pool, k.v_pool, k.page_table, lens) for k in host_kvs]
+        out_o, _ = O.decode_step(oshape, [H.oracle_weights(w) for w in ws_], okvs, h_in, r, p, b)
+        got = synth.bf16_to_f32(H.host_u16(out)).astype(np.float64)
+        m, rel = checker.output_errors(out_o, got)
+        assert m <= checker.OUT_MAX_ABS * max(1.0, np.abs(out_o).max() / 4.0) and rel <= checker.OUT_REL_L2, (s, m, rel)
+        # the cache now holds the new rows (within a bf16 step of the oracle's) and nothing else changed
+        for l in range(L):
+            kg = H.host_u16(dkvs[l].k_pool)
+            d = np.abs(O.bf16_to_f64(kg) - O.bf16_to_f64(okvs[l].k_pool))
+            assert np.all(d <= np.abs(O.bf16_to_f64(okvs[l].k_pool)) * 2.0 ** -7 + 1e-30)
+
+
+# ------------------------------------------------------------ determinism ---
+
+
+def test_repeat_calls_are_bit_identical():
+    cfg = TINY
+    r, p, b = synth.draw_actions(cfg, 1)
+    shape, _ = H.make_shapes(cfg)
+    lens = synth.make_contexts(cfg, 0)
+    w = H.device_weights(synth.make_layer_weights(cfg, 0))
+    k_pool, v_pool, table = H.make_case_kv(cfg, lens, 0)
+    h_in = synth.make_hidden(cfg, 0)
+    outs = []
+    for _ in range(2):
+        kv = H.device_kv(k_pool, v_pool, table, lens)
+        out, taps, st = H.gpu_layer(shape, w, kv, h_in, r, p, b)
+        outs.append((out, taps["kept_idx"].copy(), taps["kept_ch"].copy(), taps["h_out"].copy()))
+    for a, c in zip(outs[0], outs[1]):
+        assert np.array_equal(a, c)
