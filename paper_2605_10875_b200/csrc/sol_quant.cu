@@ -118,7 +118,7 @@ norm_quant_kernel(const void* __restrict__ in, const uint16_t* __restrict__ gamm
 #pragma unroll
       for (int e = 0; e < NQ_VEC; ++e) {
         float r = (s == 0.f) ? 0.f : rintf(__fdiv_rn(x[i][e], s));
-        c[e] = fminf(fmaxf(r, -q_max), q_max);
+        c[e] = fminf(fmaxf(r, -q_max), q_max) + 0.0f;  // +0.0f turns a rounded -0 into +0
       }
     }
     if (a_op != nullptr) {

@@ -51,7 +51,7 @@ def test_quant_codes_bit_exact(B, d):
         # dequantized value within half a step of the input
         if bits[i] != 16:
             err = np.abs(codes[i].astype(np.float64) * float(scales[i]) - O.bf16_to_f64(x[i]))
-            assert np.all(err <= 0.5 * float(scales[i]) * (1 + 1e-6))
+            assert np.all(err <= 0.5 * float(scales[i]) * (1 + 2e-5))  # float32 rounding of x/s
 
 
 def test_quant_workload_shapes_all_bit_widths():
@@ -194,9 +194,16 @@ def test_mlp_llama8b_shape():
 
 
 def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1):
+    """Runs one layer on the GPU with every tap, then checks each stage against
+    the oracle's stage applied to the inputs the GPU stage really saw, and the
+    whole layer against the oracle's own layer.  A float32-vs-float64 difference
+    of one ulp upstream may legally flip a quantizer code or a selection that
+    sits exactly on a boundary; when that happened the end-to-end comparison is
+    reported but not asserted (the chain of stage checks still covers it)."""
     shape, oshape = H.make_shapes(cfg, n_sink, n_window)
     B = len(seq_lens)
     seq_lens = np.asarray(seq_lens, np.int32)
+    d, Hq, Hkv, hd = cfg["d_model"], oshape.n_q_heads, oshape.n_kv_heads, oshape.head_dim
     w = synth.make_layer_weights(cfg, seed)
     k_pool, v_pool, table = H.make_case_kv(cfg, seq_lens, seed)
     h_in = synth.make_hidden(cfg, seed, B)
@@ -205,48 +212,73 @@ def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1):
     assert st[0] == 0 and st[1] == 0 and st[2] == 0, st
     ow = H.oracle_weights(w)
     tab = np.where(table < 0, 0, table)
+    h64 = O.bf16_to_f64(h_in)
 
-    # (1) end to end against the oracle's own layer
+    # the oracle's own layer
     okv = O.PagedKV(k_pool.copy(), v_pool.copy(), tab, seq_lens)
-    out_o, tr = O.decode_layer(oshape, ow, okv, O.bf16_to_f64(h_in), r, p, b)
-    err = H.assert_outputs(out_o, out, "layer output")
+    out_o, tr = O.decode_layer(oshape, ow, okv, h64, r, p, b)
 
-    # (2) stage by stage, each on the inputs the GPU stage really saw
-    Hq, Hkv, hd = oshape.n_q_heads, oshape.n_kv_heads, oshape.head_dim
+    # stage 1: RMSNorm (float32 on the GPU) and quantizer (bit-exact on the GPU's own normalised row)
     assert np.allclose(taps["xn1"], tr.xn1, rtol=2e-5, atol=1e-6)
+    x_hat1 = np.zeros((B, d))
     for i in range(B):
-        c, s, _ = O.quantize_per_token(taps["xn1"][i], int(b[i]))
+        c, s, x_hat1[i] = O.quantize_per_token(taps["xn1"][i], int(b[i]))
         assert np.array_equal(c, taps["codes1"][i]) and np.float32(s) == taps["scales1"][i], "codes1"
-    assert np.allclose(taps["q_rot"], tr.q_rot, rtol=0, atol=2e-4 * np.abs(tr.q_rot).max())
-    # appended k, v: within one bf16 step of the oracle's
+    # stage 2: QKV projection, rotary embedding, append
+    qkv = x_hat1 @ O.bf16_to_f64(w.w_qkv).T
+    q_ref = np.stack([O.rope_rotate(qkv[i, : Hq * hd].reshape(Hq, hd), int(seq_lens[i]) - 1, oshape.rope_theta)
+                      for i in range(B)])
+    assert np.allclose(taps["q_rot"], q_ref, rtol=0, atol=1e-5 * max(1.0, np.abs(q_ref).max())), "q_rot"
     k_gpu, v_gpu = H.host_u16(kv.k_pool), H.host_u16(kv.v_pool)
     for i in range(B):
         pos = int(seq_lens[i]) - 1
         pg, slot = tab[i, pos // 64], pos % 64
-        for got, want in ((k_gpu[pg, :, slot], tr.k_new[i]), (v_gpu[pg, :, slot], tr.v_new[i])):
-            d = np.abs(O.bf16_to_f64(got) - O.bf16_to_f64(want))
-            assert np.all(d <= np.abs(O.bf16_to_f64(want)) * 2.0 ** -7 + 1e-30), "appended k/v"
+        k_ref = O.rope_rotate(qkv[i, Hq * hd:(Hq + Hkv) * hd].reshape(Hkv, hd), pos, oshape.rope_theta)
+        v_ref = qkv[i, (Hq + Hkv) * hd:].reshape(Hkv, hd)
+        for got, want in ((k_gpu[pg, :, slot], k_ref), (v_gpu[pg, :, slot], v_ref)):
+            # the appended row is the bf16 nearest to the float32 value: within one bf16 step of the float64 one
+            assert np.all(np.abs(O.bf16_to_f64(got) - want) <= np.abs(want) * 2.0 ** -8 * 1.01 + 1e-6), "append"
     assert (k_gpu != k_pool).sum() <= B * Hkv * hd  # nothing but the appended rows changed
-    # token selection and attention on the GPU's own queries and cache
+    # stage 3: token selection and attention on the GPU's own queries and cache
     gkv = O.PagedKV(k_gpu, v_gpu, tab, seq_lens)
     attn_o, kept_o, sigma = O.sparse_decode_attn(oshape, taps["q_rot"].astype(np.float64), gkv, r)
     kept = [[taps["kept_idx"][i, h, : taps["kept_cnt"][i, h]] for h in range(Hkv)] for i in range(B)]
     tok = H.check_token_sets(oshape, sigma, kept_o, kept, seq_lens)
     H.assert_sets(tok, "layer token sets")
-    assert np.allclose(taps["attn_out"], attn_o, rtol=0, atol=2e-3 * max(1e-3, np.abs(attn_o).max()))
-    assert np.allclose(taps["h_mid"], tr.h_mid, rtol=0, atol=2e-3)
-    assert np.allclose(taps["xn2"], tr.xn2, rtol=0, atol=2e-3)
-    x_hat2 = np.zeros((B, cfg["d_model"]))
+    if tok.exact == tok.sets:
+        assert np.allclose(taps["attn_out"], attn_o, rtol=0, atol=1e-4 * max(1.0, np.abs(attn_o).max())), "attn_out"
+    # stage 4: output projection + residual on the GPU's own attention output
+    h_mid_ref = h64 + taps["attn_out"].astype(np.float64).reshape(B, Hq * hd) @ O.bf16_to_f64(w.w_o).T
+    assert np.allclose(taps["h_mid"], h_mid_ref, rtol=0, atol=1e-4), "h_mid"
+    # stage 5: second RMSNorm + quantizer
+    xn2_ref = np.stack([O.rmsnorm(taps["h_mid"][i].astype(np.float64), O.bf16_to_f64(w.gamma2), oshape.rms_eps)
+                        for i in range(B)])
+    assert np.allclose(taps["xn2"], xn2_ref, rtol=2e-5, atol=1e-6), "xn2"
+    x_hat2 = np.zeros((B, d))
     for i in range(B):
         c, s, x_hat2[i] = O.quantize_per_token(taps["xn2"][i], int(b[i]))
         assert np.array_equal(c, taps["codes2"][i]) and np.float32(s) == taps["scales2"][i], "codes2"
+    # stage 6: pruned MLP on the GPU's own quantized input
     mlp_o, kept_ch_o, t_o = O.pruned_swiglu_mlp(x_hat2, w.w_gate, w.w_up, w.w_down_t, p)
     kept_ch = [taps["kept_ch"][i, : taps["kept_ch_cnt"][i]] for i in range(B)]
     ch = H.check_channel_sets(t_o, kept_ch_o, kept_ch)
     H.assert_sets(ch, "layer channel sets")
-    assert np.allclose(taps["t"], t_o, rtol=1e-4, atol=1e-5)
-    assert np.allclose(taps["h_out"], taps["h_mid"].astype(np.float64) + mlp_o, rtol=0, atol=2e-3)
-    return dict(err=err, tokens=tok, channels=ch, status=st)
+    assert np.allclose(taps["t"], t_o, rtol=1e-4, atol=1e-5), "t"
+    if ch.exact == ch.sets:
+        assert np.allclose(taps["h_out"], taps["h_mid"].astype(np.float64) + mlp_o, rtol=0, atol=2e-4), "h_out"
+    # stage 7: the bf16 output is the float32 result rounded to nearest-even
+    assert np.array_equal(synth.to_bf16(taps["h_out"]), synth.to_bf16(out.astype(np.float32))), "bf16 rounding"
+
+    # end to end against the oracle's own layer
+    flips = int((taps["codes1"] != tr.codes1).sum() + (taps["codes2"] != tr.codes2).sum())
+    own_tok = H.check_token_sets(oshape, tr.extra["sigma"], tr.kept_tokens, kept, seq_lens)
+    own_ch = H.check_channel_sets(tr.t, tr.kept_channels, kept_ch)
+    diverged = flips > 0 or own_tok.exact != own_tok.sets or own_ch.exact != own_ch.sets
+    err = checker.output_errors(out_o, out)
+    if not diverged:
+        H.assert_outputs(out_o, out, "layer output")
+    return dict(err=err, code_flips=flips, tokens=tok, channels=ch, own_tokens=own_tok, own_channels=own_ch,
+                status=st, end_to_end_asserted=not diverged)
 
 
 def test_layer_tiny_workload():
@@ -309,10 +341,8 @@ def test_step_three_layers_matches_oracle_and_host_variant():
     okvs = [O.PagedKV(k.copy(), v.copy(), np.where(t < 0, 0, t), seq_lens) for (k, v, t) in pools]
     out_o, _ = O.decode_step(oshape, [H.oracle_weights(w) for w in ws_], okvs, h_in, r, p, b)
     got = synth.bf16_to_f32(H.host_u16(out)).astype(np.float64)
-    # the residual stream grows with depth; the absolute bound scales with bf16's step at its magnitude
-    scale = max(1.0, np.abs(out_o).max() / 4.0)
     m, rel = checker.output_errors(out_o, got)
-    assert m <= checker.OUT_MAX_ABS * scale and rel <= checker.OUT_REL_L2, (m, rel)
+    assert m <= checker.OUT_MAX_ABS and rel <= checker.OUT_REL_L2, (m, rel)
     m32, rel32 = checker.output_errors(out_o, out32.cpu().numpy())
     assert m32 <= 5e-3 and rel32 <= 1e-3, (m32, rel32)
 
@@ -361,7 +391,7 @@ def test_consecutive_steps_append_to_the_cache():
         out_o, _ = O.decode_step(oshape, [H.oracle_weights(w) for w in ws_], okvs, h_in, r, p, b)
         got = synth.bf16_to_f32(H.host_u16(out)).astype(np.float64)
         m, rel = checker.output_errors(out_o, got)
-        assert m <= checker.OUT_MAX_ABS * max(1.0, np.abs(out_o).max() / 4.0) and rel <= checker.OUT_REL_L2, (s, m, rel)
+        assert m <= checker.OUT_MAX_ABS and rel <= checker.OUT_REL_L2, (s, m, rel)
         # the cache now holds the new rows (within a bf16 step of the oracle's) and nothing else changed
         for l in range(L):
             kg = H.host_u16(dkvs[l].k_pool)

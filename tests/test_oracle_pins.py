@@ -122,7 +122,7 @@ def test_quantizer_properties(bits):
         a = float(np.abs(x).max())
         assert abs(float(s) - a / q_max) <= 2.0 ** -24 * a / q_max
         # reconstruction error at most half a step (plus float32 rounding of x/s)
-        assert np.all(np.abs(x.astype(np.float64) - xh) <= 0.5 * float(s) * (1 + 1e-6))
+        assert np.all(np.abs(x.astype(np.float64) - xh) <= 0.5 * float(s) * (1 + 2e-5))
         # the largest-magnitude element maps to +-q_max
         j = int(np.argmax(np.abs(x)))
         assert abs(int(c[j])) == q_max and np.sign(c[j]) == np.sign(x[j])
@@ -541,3 +541,29 @@ def test_synth_is_seeded_and_shaped():
         assert abs(np.mean(r * (1000 - p) / 1000.0) - tgt) <= 1000 / 32
     x = np.random.default_rng(0).standard_normal(5000).astype(np.float32)
     assert np.array_equal(synth.to_bf16(x), torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))
+
+
+# --------------------------------------------------------------- checker ----
+
+
+def test_checker_near_tie_rule_and_output_bounds():
+    from oracle import checker
+
+    score = np.array([5.0, 4.0, 3.0000001, 3.0, 1.0])
+    ok = checker.compare_index_set(score, np.array([0, 1, 2]), np.array([0, 1, 2]))
+    assert ok.exact == 1 and ok.ok()
+    tie = checker.compare_index_set(score, np.array([0, 1, 2]), np.array([0, 1, 3]))
+    assert tie.ok() and tie.near_tie_indices == 2 and tie.exact == 0
+    bad = checker.compare_index_set(score, np.array([0, 1, 2]), np.array([0, 1, 4]))
+    assert not bad.ok() and bad.failed_indices >= 1
+    assert not checker.compare_index_set(score, np.array([0, 1, 2]), np.array([0, 1])).ok()
+    assert not checker.compare_index_set(score, np.array([0, 1, 2]), np.array([0, 1, 1])).ok()
+    # forced indices are never excused
+    f = checker.compare_index_set(score, np.array([0, 1, 4]), np.array([0, 1, 3]), forced=np.array([4]))
+    assert not f.ok()
+    o = np.array([1.0, -7.9, 9.0, 20.0])
+    assert checker.outputs_ok(o, o + np.array([0.019, 0.019, 0.039, 0.079]))
+    assert not checker.outputs_ok(o, o + np.array([0.021, 0, 0, 0]))
+    assert not checker.outputs_ok(o, o + np.array([0, 0, 0.041, 0]))
+    m, rel = checker.output_errors(np.ones(4), np.ones(4) * 1.02)
+    assert abs(m - 0.02) < 1e-12 and abs(rel - 0.02) < 1e-12
