@@ -1,0 +1,489 @@
+#!/usr/bin/env python
+"""Benchmark of the action-conditioned decode step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A "step" is one pass of the whole hot path (every layer of the workload) over
+one batch of synthetic input.  Prints ONE JSON line (rank 0).  With N > 1
+(launched by torch.distributed.run) every rank runs an independent replica of
+the step on its own GPU: the path needs no exchange between sequences, so
+there is no collective in the data path; the ranks meet only at the barriers
+around the timed region and the slowest rank's time is reported.
+
+`--impl reference` times the CPU oracle on the host cores instead (a
+deliberately plain fp64 program; a reported baseline, not a target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_10875_b200 import synth  # noqa: E402
+
+METRIC = "action-conditioned decode steps/s"
+UNIT = "steps/s"
+HBM_SPEC_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+ROTATE = 4  # distinct copies of weights + cache, cycled so that no step finds its inputs in L2
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
+# the ncu capture summarised under profiles/, keyed by (workload, kernel); absent -> null.
+NCU_TRAFFIC_BYTES = {}
+
+
+def _plain(o):
+    return o.item() if hasattr(o, "item") else str(o)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------
+# algorithmic bytes
+# ----------------------------------------------------------------------------
+
+
+def kept_tokens(r_permille, T):
+    T = int(T)
+    return min(T, max(1, (int(r_permille) * T + 999) // 1000))
+
+
+def kernel_bytes(cfg, seq_lens, r, union_rows):
+    """Bytes each streaming kernel must move per launch (one layer)."""
+    d, hq, hkv, hd, ff = cfg["d_model"], cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"], cfg["d_ff"]
+    k_bytes = sum(hkv * int(T) * hd * 2 for T in seq_lens)
+    v_bytes = sum(hkv * kept_tokens(ri, T) * hd * 2 for ri, T in zip(r, seq_lens))
+    return {
+        "attn_score": k_bytes,
+        "attn_gather_v": v_bytes,
+        "gemm_qkv": (hq + 2 * hkv) * hd * d * 2,
+        "gemm_out_proj": d * hq * hd * 2,
+        "gemm_gate_up_swiglu": 2 * ff * d * 2,
+        "gemm_down_gathered": union_rows * d * 2,
+    }
+
+
+# ----------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+            self._period = period_s
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self._period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": int(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------
+# the GPU arm
+# ----------------------------------------------------------------------------
+
+
+class Replica:
+    """Device-resident state of one workload: ROTATE copies of weights and caches."""
+
+    def __init__(self, cfg, device, seed=0):
+        import torch
+
+        from paper_2605_10875_b200 import binding as sol
+
+        self.torch, self.sol, self.cfg, self.device = torch, sol, cfg, device
+        self.B, self.L = cfg["batch"], cfg["layers"]
+        self.seq_lens = synth.make_contexts(cfg, seed)
+        self.shape = sol.make_shape(cfg["d_model"], cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"], cfg["d_ff"],
+                                    64, synth.RMS_EPS, cfg.get("rope_theta", 0.0), 0, 1)
+        table, n_pages = synth.make_page_table(self.seq_lens, cfg.get("shuffle_pages", True), seed)
+        self.max_pages, self.n_pages = table.shape[1], n_pages
+        self.table = self._i32(np.where(table < 0, 0, table))
+        self.lens_dev = self._i32(self.seq_lens)
+        names = ("w_qkv", "w_o", "w_gate", "w_up", "w_down_t", "gamma1", "gamma2")
+        self.weights, self.kvs, self._keep = [], [], []
+        for l in range(self.L):
+            w = synth.make_layer_weights(cfg, seed, l)
+            base_w = [self._bf16(getattr(w, n)) for n in names]
+            k, v = synth.make_kv_pool(cfg, n_pages, seed, l)
+            base_kv = [self._bf16(k), self._bf16(v)]
+            per_copy_w, per_copy_kv = [], []
+            for c in range(ROTATE):
+                ws_ = base_w if c == 0 else [t.clone() for t in base_w]
+                kv_ = base_kv if c == 0 else [t.clone() for t in base_kv]
+                self._keep += ws_ + kv_
+                per_copy_w.append(sol.make_weights(*ws_))
+                per_copy_kv.append(sol.make_kv(kv_[0], kv_[1], self.table, self.lens_dev, self.max_pages, n_pages))
+            self.weights.append(per_copy_w)
+            self.kvs.append(per_copy_kv)
+        self.ws_bytes = sol.workspace_bytes(self.shape, self.B, self.max_pages)
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=device)
+        sol.workspace_init(self.ws, self.ws_bytes)
+        self.h_in = self._bf16(synth.make_hidden(cfg, seed))
+        self.h_out = torch.zeros((self.B, cfg["d_model"]), dtype=torch.bfloat16, device=device)
+        # pinned host buffers for the end-to-end path
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        self.h_in_host = pin(synth.make_hidden(cfg, seed).view(np.int16))
+        self.h_out_host = torch.zeros((self.B, cfg["d_model"]), dtype=torch.int16).pin_memory()
+        self.lens_host = pin(self.seq_lens.astype(np.int32))
+        torch.cuda.synchronize()
+
+    def _bf16(self, u16):
+        t = self.torch
+        return t.from_numpy(np.ascontiguousarray(u16).view(np.int16)).to(self.device).view(t.bfloat16)
+
+    def _i32(self, a):
+        return self.torch.from_numpy(np.ascontiguousarray(np.asarray(a, np.int32))).to(self.device)
+
+    def set_actions(self, r, p, b):
+        self.r_np, self.p_np, self.b_np = [np.asarray(x, np.int32) for x in (r, p, b)]
+        self.r, self.p, self.b = self._i32(r), self._i32(p), self._i32(b)
+        pin = lambda a: self.torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        self.r_host, self.p_host, self.b_host = pin(self.r_np), pin(self.p_np), pin(self.b_np)
+
+    def step(self, i):
+        c = i % ROTATE
+        self.sol.decode_step(self.shape, [w[c] for w in self.weights], [k[c] for k in self.kvs], self.B, self.h_in,
+                             self.h_out, None, self.r, self.p, self.b, self.ws, self.ws_bytes)
+
+    def step_host(self, i):
+        c = i % ROTATE
+        self.sol.decode_step_host(self.shape, [w[c] for w in self.weights], [k[c] for k in self.kvs], self.B,
+                                  self.h_in_host, self.h_out_host, self.r_host, self.p_host, self.b_host,
+                                  self.lens_host, self.ws, self.ws_bytes)
+
+    def union_rows(self):
+        """Rows of W_down that at least one token keeps, from one traced call of layer 0."""
+        t, sol = self.torch, self.sol
+        ff = self.cfg["d_ff"]
+        kept = t.full((self.B, ff), -1, dtype=t.int32, device=self.device)
+        cnt = t.zeros((self.B,), dtype=t.int32, device=self.device)
+        out = t.zeros_like(self.h_out)
+        sol.decode_layer(self.shape, self.weights[0][0], self.kvs[0][0], self.B, self.h_in, out, self.r, self.p,
+                         self.b, sol.make_trace(kept_ch=kept, kept_ch_cnt=cnt), self.ws, self.ws_bytes)
+        t.cuda.synchronize()
+        k, c = kept.cpu().numpy(), cnt.cpu().numpy()
+        rows = set()
+        for i in range(self.B):
+            rows.update(k[i, : c[i]].tolist())
+        return len(rows)
+
+    def required_bytes_per_step(self, union_rows):
+        kb = kernel_bytes(self.cfg, self.seq_lens, self.r_np, union_rows)
+        return self.L * sum(kb.values()), kb
+
+
+def timed_steps(rep, steps, warmup, barrier, fn):
+    """`steps` calls of fn(i) after `warmup`; device time by CUDA events, max over ranks."""
+    torch = rep.torch
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        fn(warmup + i)
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    return e0.elapsed_time(e1)  # ms
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_10875_b200 import binding as sol
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(device))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    sol.lib()
+    cfg = synth.WORKLOADS[args.workload]
+    rep = Replica(cfg, device, seed=0)
+    r, p, b = synth.draw_actions(cfg, 0)
+    rep.set_actions(r, p, b)
+    union = rep.union_rows()
+    req_bytes, kb = rep.required_bytes_per_step(union)
+    peak_gbs, peak_kind = measured_peaks()
+
+    # --- headline: K steps, inputs resident in HBM ---
+    sol.launch_count(reset=True)
+    with ClockSampler(local) as clocks:
+        ms = max_over_ranks(timed_steps(rep, args.steps, args.warmup, barrier, rep.step))
+    launches = sol.launch_count(reset=True) * args.steps // (args.steps + args.warmup)
+    status = sol.read_device_status(rep.ws)
+    ms_per_step = ms / args.steps
+    value = world * args.steps / (ms / 1e3)
+
+    # --- the same steps with per-kernel CUDA events, for the dominant kernel's roofline ---
+    prof_steps = min(args.steps, 200)
+    sol.timing_enable(True)
+    timed_steps(rep, prof_steps, 3, barrier, rep.step)
+    rows = sol.timing_collect()
+    sol.timing_enable(False)
+    per_kernel = {}
+    n_prof = prof_steps + 3
+    for name, n, tot in rows:
+        per_kernel[name] = {"launches_per_step": n // n_prof, "us_per_launch": 1e3 * tot / n,
+                            "us_per_step": 1e3 * tot / n_prof}
+    tot_us = sum(v["us_per_step"] for v in per_kernel.values())
+    for v in per_kernel.values():
+        v["share"] = round(v["us_per_step"] / tot_us, 4)
+        v["us_per_launch"] = round(v["us_per_launch"], 3)
+        v["us_per_step"] = round(v["us_per_step"], 3)
+    for name, nbytes in kb.items():
+        if name in per_kernel:
+            per_kernel[name]["bytes_per_launch"] = nbytes
+            per_kernel[name]["gbs"] = round(nbytes / per_kernel[name]["us_per_launch"] / 1e3, 1)
+    streaming = {k: v for k, v in per_kernel.items() if "bytes_per_launch" in v}
+    dom = max(streaming, key=lambda k: streaming[k]["us_per_step"])
+    achieved = streaming[dom]["gbs"]
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
+                "frac": round(achieved / peak_gbs, 4), "peak_kind": f"of {peak_kind}",
+                "bytes_per_launch": streaming[dom]["bytes_per_launch"],
+                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dom))}
+
+    # --- end to end: host buffers in, host buffers out, every step ---
+    e2e_steps = min(args.steps, 500)
+    ms_e2e = max_over_ranks(timed_steps(rep, e2e_steps, 3, barrier, rep.step_host))
+    hb = rep.B * cfg["d_model"] * 2
+    e2e = {"value": round(world * e2e_steps / (ms_e2e / 1e3), 2), "unit": UNIT, "steps": e2e_steps,
+           "h2d_bytes_per_step": hb + 4 * rep.B * 4, "d2h_bytes_per_step": hb}
+
+    # --- budget sweep: every sequence with the same action ---
+    sweep = []
+    if not args.no_sweep:
+        for (rr, pp, bb) in [(1000, 0, 16), (500, 0, 16), (250, 0, 16), (125, 0, 16), (1000, 500, 16),
+                             (1000, 0, 8), (1000, 0, 4), (125, 750, 4)]:
+            rep.set_actions(*synth.uniform_actions(rep.B, rr, pp, bb))
+            u = rep.union_rows()
+            byt, _ = rep.required_bytes_per_step(u)
+            n = min(args.steps, 300)
+            t_ms = max_over_ranks(timed_steps(rep, n, 5, barrier, rep.step)) / n
+            sweep.append({"r": rr / 1000, "p": pp / 1000, "b": bb, "us_per_step": round(1e3 * t_ms, 2),
+                          "required_mb": round(byt / 1e6, 1), "hbm_gbs": round(byt / t_ms / 1e6, 1),
+                          "frac_of_measured": round(byt / t_ms / 1e6 / peak_gbs, 4)})
+        rep.set_actions(r, p, b)
+
+    line = None
+    if rank == 0:
+        cpu = None if (world > 1 or args.no_cpu_baseline) else cpu_baseline(args.workload, budget_s=20.0)
+        hbm_gbs = req_bytes / ms_per_step / 1e6
+        line = {
+            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "layers": cfg["layers"], "batch": cfg["batch"],
+                       "context": int(np.max(rep.seq_lens)), "actions": "per-sequence uniform draw, seed 0",
+                       "l2": f"inputs larger than L2: {ROTATE} rotating copies of weights and KV cache",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "required_bytes_per_step": int(req_bytes),
+            "hbm_tbs": round(hbm_gbs / 1e3, 4),
+            "hbm_frac_of_measured_peak": round(hbm_gbs / peak_gbs, 4),
+            "hbm_frac_of_spec_8tbs": round(hbm_gbs / HBM_SPEC_GBS, 4),
+            "roofline": roofline, "kernels": per_kernel, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": int(launches), "clocks": clocks.summary(), "device_status": status,
+            "budget_sweep": sweep,
+        }
+        print(json.dumps(line, default=_plain), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return line
+
+
+# ----------------------------------------------------------------------------
+# the CPU oracle arm (baseline)
+# ----------------------------------------------------------------------------
+
+
+def _oracle_inputs(cfg, n_seq, seed=0):
+    """Inputs of the first n_seq sequences of the workload, one layer, as the oracle takes them."""
+    from oracle import sol_oracle as O
+
+    lens = synth.make_contexts(cfg, seed)[:n_seq]
+    table, n_pages = synth.make_page_table(lens, cfg.get("shuffle_pages", True), seed)
+    k, v = synth.make_kv_pool(cfg, n_pages, seed, 0)
+    w = synth.make_layer_weights(cfg, seed, 0)
+    ow = O.LayerWeights(w.w_qkv, w.w_o, w.w_gate, w.w_up, w.w_down_t, w.gamma1, w.gamma2)
+    shape = O.Shape(cfg["d_model"], cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"], cfg["d_ff"], 64,
+                    synth.RMS_EPS, cfg.get("rope_theta", 0.0), 0, 1)
+    kv = O.PagedKV(k, v, np.where(table < 0, 0, table), lens)
+    r, p, b = synth.draw_actions(cfg, seed)
+    h = O.bf16_to_f64(synth.make_hidden(cfg, seed)[:n_seq])
+    return O, shape, ow, kv, h, r[:n_seq], p[:n_seq], b[:n_seq]
+
+
+def _host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+
+        n = [int(i.get("num_threads", 1)) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return 1
+
+
+def cpu_baseline(workload, budget_s=20.0):
+    """Times the oracle, as it stands, on a bounded sample of the workload: one layer over the first
+    n sequences, n chosen so the work stays near `budget_s`; scaled to whole steps per second."""
+    cfg = synth.WORKLOADS[workload]
+    B, L = cfg["batch"], cfg["layers"]
+    O, shape, ow, kv, h, r, p, b = _oracle_inputs(cfg, 1)
+    t0 = time.perf_counter()
+    O.decode_layer(shape, ow, kv, h, r, p, b)
+    t1 = time.perf_counter() - t0
+    n = int(max(1, min(B, budget_s // max(t1, 1e-3))))
+    if n > 1:
+        O, shape, ow, kv, h, r, p, b = _oracle_inputs(cfg, n)
+        t0 = time.perf_counter()
+        O.decode_layer(shape, ow, kv, h, r, p, b)
+        t1 = time.perf_counter() - t0
+    step_s = t1 * (B / n) * L
+    return {"value": round(1.0 / step_s, 6), "unit": UNIT, "cores": _host_threads(), "kind": "oracle",
+            "sample": f"one layer over the first {n} of {B} sequences, timed once ({t1:.2f} s), "
+                      f"scaled by {B}/{n} sequences x {L} layers"}
+
+
+def run_reference(args):
+    """The oracle as the reference arm: every step is the bounded sample of cpu_baseline."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return None
+    cfg = synth.WORKLOADS[args.workload]
+    B, L = cfg["batch"], cfg["layers"]
+    O, shape, ow, kv, h, r, p, b = _oracle_inputs(cfg, 1)
+    t0 = time.perf_counter()
+    O.decode_layer(shape, ow, kv, h, r, p, b)
+    t1 = time.perf_counter() - t0
+    total = args.steps + args.warmup
+    n = int(max(1, min(B, (150.0 / total) // max(t1, 1e-3))))
+    steps = args.steps
+    if n == 1 and t1 * total > 300.0:
+        steps = max(1, int(300.0 / t1) - args.warmup)
+    O, shape, ow, kv, h, r, p, b = _oracle_inputs(cfg, n)
+    for _ in range(args.warmup):
+        O.decode_layer(shape, ow, kv, h, r, p, b)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        O.decode_layer(shape, ow, kv, h, r, p, b)
+    dt = (time.perf_counter() - t0) / steps
+    step_s = dt * (B / n) * L
+    value = round(1.0 / step_s, 6)
+    sample = (f"each step: one layer over the first {n} of {B} sequences ({dt:.2f} s), "
+              f"scaled by {B}/{n} sequences x {L} layers")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": steps, "warmup": args.warmup,
+            "ms_per_step": round(1e3 * step_s, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "layers": L, "batch": B, "context": int(np.max(kv.seq_lens)),
+                       "actions": "per-sequence uniform draw, seed 0"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": _host_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="llama1b_layer", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args)
+    else:
+        args.steps = 2000 if args.steps is None else args.steps
+        args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
