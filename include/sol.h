@@ -136,6 +136,31 @@ sol_status_t sol_sparse_decode_attn(const sol_shape_t *shape, const void *q_bf16
                                     const int32_t *r_permille, void *out_bf16, int32_t *kept_idx,
                                     int32_t *kept_cnt, void *ws, size_t ws_bytes, sol_stream_t stream);
 
+/* The same attention for callers that cannot provide a workspace (the paper has
+ * no counterpart: this entry exists for hosts that may not allocate).  A serving
+ * process that handed all of its device memory to a pool at start-up, a plugin
+ * inside a runtime that owns the allocator, or a loop that must never reach
+ * cudaMalloc / cudaFree can call this instead of sol_sparse_decode_attn: the
+ * scratch is a fixed array of SOL_STATIC_SCRATCH_BYTES inside the library
+ * image, present on every GPU that loads the library until the process exits.
+ * The call allocates nothing.
+ *   Inputs and outputs as sol_sparse_decode_attn; kept_idx / kept_cnt optional.
+ *   status_out (optional, DEVICE int32[8]) receives the status words of this
+ *   call (layout as sol_read_device_status) by a copy enqueued on `stream`.
+ *   Limit: B * n_kv * max_pages_per_seq * 64 * (4 G + 8) bytes plus small terms
+ *   must fit the array (for 4 query / 2 kv heads of 64: batch 4 with contexts
+ *   up to about 30 thousand tokens); a larger problem is refused with
+ *   SOL_ERR_WORKSPACE_TOO_SMALL before anything is launched.
+ *   The first call on each device looks up the array's device address (with
+ *   that device current); make that first call outside any stream capture.
+ *   All calls on a device share the one array and it keeps the previous call's
+ *   contents (the status words are cleared at the start of each call): two
+ *   calls whose GPU work can overlap (different streams or threads) race. */
+#define SOL_STATIC_SCRATCH_BYTES (4u << 20)
+sol_status_t sol_sparse_decode_attn_static(const sol_shape_t *shape, const void *q_bf16, const sol_kv_t *kv,
+                                           int32_t B, const int32_t *r_permille, void *out_bf16, int32_t *kept_idx,
+                                           int32_t *kept_cnt, int32_t *status_out, sol_stream_t stream);
+
 /* SwiGLU MLP with a per-token prune rate (count mirrors the paper's
  * m = ceil(rho*d), "Per-token channel selection"; the pruned axis is the
  * intermediate one): t_j = silu(W_g x)_j (W_u x)_j, keep the

@@ -23,7 +23,7 @@ SOL_ERR_DEVICE_TIMEOUT = 5
 
 EXPORTS = [
     "sol_status_string", "sol_last_cuda_error", "sol_workspace_bytes", "sol_workspace_init", "sol_quant_act",
-    "sol_sparse_decode_attn", "sol_pruned_swiglu_mlp", "sol_decode_layer", "sol_decode_step",
+    "sol_sparse_decode_attn", "sol_sparse_decode_attn_static", "sol_pruned_swiglu_mlp", "sol_decode_layer", "sol_decode_step",
     "sol_decode_step_host", "sol_read_device_status", "sol_timing_enable", "sol_timing_collect",
     "sol_launch_count",
 ]
@@ -86,6 +86,8 @@ def lib() -> C.CDLL:
         L.sol_quant_act.argtypes = [P, I, I, P, P, P, P, P]
         L.sol_sparse_decode_attn.restype = I
         L.sol_sparse_decode_attn.argtypes = [C.POINTER(SolShape), P, C.POINTER(SolKV), I, P, P, P, P, P, S, P]
+        L.sol_sparse_decode_attn_static.restype = I
+        L.sol_sparse_decode_attn_static.argtypes = [C.POINTER(SolShape), P, C.POINTER(SolKV), I, P, P, P, P, P, P]
         L.sol_pruned_swiglu_mlp.restype = I
         L.sol_pruned_swiglu_mlp.argtypes = [C.POINTER(SolShape), P, P, P, P, I, P, P, P, P, P, S, P]
         L.sol_decode_layer.restype = I
@@ -177,6 +179,22 @@ def sparse_decode_attn(shape, q_bf16, kv: SolKV, B: int, r_permille, out_bf16, k
                                      _ptr(kept_idx), _ptr(kept_cnt), _ptr(ws), ws_bytes, _stream(stream))
     if check:
         _check(s, "sol_sparse_decode_attn")
+    return s
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def sparse_decode_attn_static(shape, q_bf16, kv: SolKV, B: int, r_permille, out_bf16, kept_idx=None, kept_cnt=None,
+                              status_out=None, stream=None, check=True) -> int:
+    """sol_sparse_decode_attn for a caller with no workspace to give: the scratch is a fixed array
+    inside the library (STATIC_SCRATCH_BYTES per GPU), nothing is allocated.  Problems that do not
+    fit are refused with SOL_ERR_WORKSPACE_TOO_SMALL.  Calls share the array: do not overlap them."""
+    s = lib().sol_sparse_decode_attn_static(C.byref(shape), _ptr(q_bf16), C.byref(kv), B, _ptr(r_permille),
+                                            _ptr(out_bf16), _ptr(kept_idx), _ptr(kept_cnt), _ptr(status_out),
+                                            _stream(stream))
+    if check:
+        _check(s, "sol_sparse_decode_attn_static")
     return s
 
 

@@ -32,6 +32,12 @@ bool record_cuda_error(cudaError_t e, const char* where) {
   return true;
 }
 
+bool take_cuda_failure() {
+  const bool f = tl_cuda_failed;
+  tl_cuda_failed = false;
+  return f;
+}
+
 void note_launch_begin(const char* name, cudaStream_t st) {
   g_launches.fetch_add(1, std::memory_order_relaxed);
   if (g_timing) {

@@ -14,6 +14,7 @@ namespace sol {
 void note_launch_begin(const char* name, cudaStream_t st);
 void note_launch_end(cudaStream_t st);
 bool record_cuda_error(cudaError_t e, const char* where);  // true if e != success
+bool take_cuda_failure();  // true if a CUDA call of this thread failed since the last check; clears the mark
 
 #define SOL_LAUNCH(name, kernel, grid, block, smem, st, ...)             \
   do {                                                                   \

@@ -1,0 +1,133 @@
+// sol_sparse_decode_attn_static: the decode attention for callers that cannot
+// hand the library a workspace.
+//
+// Some hosts of this library never get to call cudaMalloc on the decode path:
+// a serving process whose memory pool was carved up at start-up and has
+// nothing left to lend, a plugin running inside another runtime that owns
+// the allocator, a latency-critical loop where an allocation (or the implicit
+// synchronisation a free can bring) is not allowed.  For them the scratch of
+// the attention call (split queries, logits, selection scores, kept lists,
+// split partials, status words) lives in one fixed array that is part of the
+// library image: SOL_STATIC_SCRATCH_BYTES of device memory on every GPU that
+// loads the library, held until the process exits.
+//
+// The array's name in host code is only a handle for the runtime, not a device
+// address, so the address is looked up once per device with
+// cudaGetSymbolAddress (with that device current) and that pointer is what
+// the kernels receive.
+#include <mutex>
+
+#include "sol_common.cuh"
+#include "sol_internal.h"
+
+namespace {
+
+constexpr size_t kScratchBytes = SOL_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_mu;
+unsigned char* g_scratch_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the array on the current device; resolved on the first call per device.
+sol_status_t scratch_of_current_device(unsigned char** out) {
+  int dev = 0;
+  if (sol::record_cuda_error(cudaGetDevice(&dev), "cudaGetDevice")) return SOL_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return SOL_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_mu);
+  if (g_scratch_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (sol::record_cuda_error(cudaGetSymbolAddress(&p, g_static_scratch), "cudaGetSymbolAddress")) return SOL_ERR_CUDA;
+    if (p == nullptr) return SOL_ERR_CUDA;
+    g_scratch_ptr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = g_scratch_ptr[dev];
+  return SOL_OK;
+}
+
+struct StaticLayout {
+  size_t status, q_rot, q_split, logits, sigma, kept_idx, kept_cnt, part, total;
+  int splits;
+};
+
+StaticLayout layout_for(const sol_shape_t& s, int B, int max_pages) {
+  StaticLayout L;
+  const size_t Hq = s.n_q_heads, Hkv = s.n_kv_heads, hd = s.head_dim, G = Hq / Hkv, HG = (G + 3) / 4;
+  const size_t Tmax = (size_t)max_pages * s.page_size;
+  L.splits = (int)((Tmax + sol::ATTN_SPLIT_LEN - 1) / sol::ATTN_SPLIT_LEN);
+  size_t at = 0;
+  auto take = [&](size_t bytes) {
+    const size_t o = at;
+    at += (bytes + 255) / 256 * 256;
+    return o;
+  };
+  L.status = take(256);
+  L.q_rot = take(B * Hq * hd * 4);
+  L.q_split = take(B * Hkv * HG * 16 * hd * 2);
+  L.logits = take(B * Hkv * Tmax * G * 4);
+  L.sigma = take(B * Hkv * Tmax * 4);
+  L.kept_idx = take(B * Hkv * Tmax * 4);
+  L.kept_cnt = take(B * Hkv * 4);
+  L.part = take(B * Hkv * (size_t)L.splits * G * (hd + 2) * 4);
+  L.total = at;
+  return L;
+}
+
+bool attention_shape_ok(const sol_shape_t* s) {
+  if (!s) return false;
+  if (s->head_dim != 64 && s->head_dim != 128) return false;
+  if (s->page_size != 64) return false;
+  if (s->n_kv_heads <= 0 || s->n_q_heads <= 0 || s->n_q_heads % s->n_kv_heads) return false;
+  if (s->n_q_heads / s->n_kv_heads > 8) return false;
+  return s->n_sink >= 0 && s->n_window >= 0;
+}
+
+}  // namespace
+
+extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, const void* q_bf16,
+                                                      const sol_kv_t* kv, int32_t B, const int32_t* r_permille,
+                                                      void* out_bf16, int32_t* kept_idx, int32_t* kept_cnt,
+                                                      int32_t* status_out, sol_stream_t stream) {
+  if (!shape || !q_bf16 || !kv || !kv->k_pool || !kv->v_pool || !kv->page_table || !kv->seq_lens ||
+      kv->max_pages_per_seq <= 0 || kv->num_pages <= 0 || !r_permille || !out_bf16 || B < 0)
+    return SOL_ERR_INVALID_ARG;
+  if (!attention_shape_ok(shape) || B > 128) return SOL_ERR_UNSUPPORTED;
+  if (B == 0) return SOL_OK;
+  const StaticLayout L = layout_for(*shape, B, kv->max_pages_per_seq);
+  if (L.total > kScratchBytes) return SOL_ERR_WORKSPACE_TOO_SMALL;  // the fixed scratch cannot hold this problem
+
+  unsigned char* base = nullptr;
+  const sol_status_t s = scratch_of_current_device(&base);
+  if (s != SOL_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  // the array keeps whatever the previous call left; only the status words must start at zero
+  if (sol::record_cuda_error(cudaMemsetAsync(base + L.status, 0, 256, st), "status memset")) return SOL_ERR_CUDA;
+
+  sol::AttnArgs a;
+  a.shape = *shape;
+  a.kv = *kv;
+  a.B = B;
+  a.r_permille = r_permille;
+  a.qkv_f32 = nullptr;
+  a.ldq = 0;
+  a.q_bf16 = q_bf16;
+  a.q_rot = reinterpret_cast<float*>(base + L.q_rot);
+  a.q_split = base + L.q_split;
+  a.logits = reinterpret_cast<float*>(base + L.logits);
+  a.sigma = reinterpret_cast<float*>(base + L.sigma);
+  a.kept_idx = kept_idx ? kept_idx : reinterpret_cast<int32_t*>(base + L.kept_idx);
+  a.kept_cnt = kept_cnt ? kept_cnt : reinterpret_cast<int32_t*>(base + L.kept_cnt);
+  a.part = reinterpret_cast<float*>(base + L.part);
+  a.splits = L.splits;
+  a.out_f32 = nullptr;
+  a.out_bf16 = out_bf16;
+  a.out_hi = nullptr;
+  a.out_lo = nullptr;
+  a.status = reinterpret_cast<int*>(base + L.status);
+  sol::launch_attention(a, st);
+  if (status_out != nullptr &&
+      sol::record_cuda_error(cudaMemcpyAsync(status_out, base + L.status, sizeof(int32_t) * sol::ST_WORDS,
+                                             cudaMemcpyDeviceToDevice, st), "status copy"))
+    return SOL_ERR_CUDA;
+  return sol::take_cuda_failure() ? SOL_ERR_CUDA : SOL_OK;
+}
