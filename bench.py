@@ -34,7 +34,7 @@ METRIC = "action-conditioned decode steps/s"
 UNIT = "steps/s"
 HBM_SPEC_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-ROTATE = 4  # distinct copies of weights + cache, cycled so that no step finds its inputs in L2
+ROTATE = 4  # distinct copies of weights + cache, cycled so that no step finds its inputs in L2 (--rotate)
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
 # the ncu capture summarised under profiles/, keyed by (workload, kernel); absent -> null.
@@ -472,9 +472,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--workload", default="llama1b_layer", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--rotate", type=int, default=ROTATE,
+                    help="distinct copies of weights and KV cache cycled through the steps (1 for a small profiler capture)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    globals()["ROTATE"] = max(1, args.rotate)
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup

@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -68,6 +69,26 @@ int sm_count() {
   return cached[dev];
 }
 
+void ensure_dynamic_smem(const void* kernel, int bytes) {
+  struct Entry { int dev; const void* fn; int bytes; };
+  static Entry table[256];
+  static int n = 0;
+  static std::mutex mu;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  std::lock_guard<std::mutex> lock(mu);
+  for (int i = 0; i < n; ++i) {
+    if (table[i].dev == dev && table[i].fn == kernel) {
+      if (table[i].bytes >= bytes) return;
+      record_cuda_error(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes), "smem attribute");
+      table[i].bytes = bytes;
+      return;
+    }
+  }
+  record_cuda_error(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes), "smem attribute");
+  if (n < 256) table[n++] = Entry{dev, kernel, bytes};
+}
+
 // ---------------------------------------------------------------------------
 // workspace layout
 // ---------------------------------------------------------------------------
@@ -78,7 +99,7 @@ static int pad_rows(int B) {
 
 struct Layout {
   size_t status, stage_h_in, stage_act, stage_h_out, a_op, scale, qkv, q_rot, q_split, logits, sigma, kept_idx,
-      kept_cnt, part, attn_hi, attn_lo, attn_f32, h_mid, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, down_part,
+      kept_cnt, part, work_items, work_ctr, attn_hi, attn_lo, attn_f32, h_mid, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, down_part,
       h_a, h_b, total;
   int splits, chunks, Mpad, Tmax;
 };
@@ -91,7 +112,7 @@ static bool shape_ok(const sol_shape_t* s) {
   if (s->n_q_heads / s->n_kv_heads > 8) return false;
   if (s->d_model <= 0 || s->d_model % 256 || s->d_model > 8192) return false;
   if ((s->n_q_heads * s->head_dim) % 256) return false;
-  if (s->d_ff <= 0 || s->d_ff % 32) return false;
+  if (s->d_ff <= 0 || s->d_ff % 32 || s->d_ff > 49152) return false;
   if (s->n_sink < 0 || s->n_window < 0) return false;
   return true;
 }
@@ -104,8 +125,7 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   const size_t Mpad = pad_rows(B), Tmax = (size_t)max_pages * s.page_size;
   L.Mpad = (int)Mpad;
   L.Tmax = (int)Tmax;
-  L.splits = (int)((Tmax + ATTN_SPLIT_LEN - 1) / ATTN_SPLIT_LEN);
-  if (L.splits < 1) L.splits = 1;
+  L.splits = attn_splits(s.head_dim, max_pages, s.page_size);
   L.chunks = down_chunks((int)ff, (int)d);
   size_t at = 0;
   auto take = [&](size_t bytes) {
@@ -127,6 +147,8 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   L.kept_idx = take(B * Hkv * Tmax * 4);
   L.kept_cnt = take(B * Hkv * 4);
   L.part = take(B * Hkv * L.splits * G * (hd + 2) * 4);
+  L.work_items = take(B * Hkv * (size_t)L.splits * 4);
+  L.work_ctr = take((2 + B * Hkv) * 4);
   L.attn_hi = take(Mpad * Hq * hd * 2);
   L.attn_lo = take(Mpad * Hq * hd * 2);
   L.attn_f32 = take(B * Hq * hd * 4);
@@ -185,7 +207,9 @@ static void run_attention(const sol_shape_t& s, const Layout& L, void* ws, const
   a.kept_idx = kept_idx ? kept_idx : at<int32_t>(ws, L.kept_idx);
   a.kept_cnt = kept_cnt ? kept_cnt : at<int32_t>(ws, L.kept_cnt);
   a.part = at<float>(ws, L.part);
-  a.splits = (kv.max_pages_per_seq * s.page_size + ATTN_SPLIT_LEN - 1) / ATTN_SPLIT_LEN;
+  a.splits = attn_splits(s.head_dim, kv.max_pages_per_seq, s.page_size);
+  a.work_items = at<int32_t>(ws, L.work_items);
+  a.work_ctr = at<int32_t>(ws, L.work_ctr);
   a.out_f32 = out_f32;
   a.out_bf16 = out_bf16;
   a.out_hi = want_split ? at<void>(ws, L.attn_hi) : nullptr;
@@ -334,7 +358,9 @@ const char* sol_status_string(sol_status_t s) {
 const char* sol_last_cuda_error(void) { return tl_cuda_error; }
 
 size_t sol_workspace_bytes(const sol_shape_t* shape, int32_t max_batch, int32_t max_pages_per_seq) {
-  if (!shape_ok(shape) || max_batch < 1 || max_batch > 128 || max_pages_per_seq < 1) return 0;
+  if (!shape_ok(shape) || max_batch < 1 || max_batch > 128 || max_pages_per_seq < 1 ||
+      max_pages_per_seq > MAX_PAGES_PER_SEQ)
+    return 0;
   return make_layout(*shape, max_batch, max_pages_per_seq).total;
 }
 
@@ -359,7 +385,7 @@ sol_status_t sol_sparse_decode_attn(const sol_shape_t* shape, const void* q_bf16
                                     const int32_t* r_permille, void* out_bf16, int32_t* kept_idx, int32_t* kept_cnt,
                                     void* ws, size_t ws_bytes, sol_stream_t stream) {
   if (!shape || !q_bf16 || !kv_ok(kv) || !r_permille || !out_bf16 || !ws || B < 0) return SOL_ERR_INVALID_ARG;
-  if (!shape_ok(shape) || B > 128) return SOL_ERR_UNSUPPORTED;
+  if (!shape_ok(shape) || B > 128 || kv->max_pages_per_seq > MAX_PAGES_PER_SEQ) return SOL_ERR_UNSUPPORTED;
   if (B == 0) return SOL_OK;
   const Layout L = make_layout(*shape, B, kv->max_pages_per_seq);
   if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
@@ -401,6 +427,7 @@ sol_status_t sol_decode_layer(const sol_shape_t* shape, const sol_layer_weights_
     return SOL_ERR_INVALID_ARG;
   sol_status_t s = check_actions_host_side(shape, B);
   if (s != SOL_OK) return s;
+  if (kv->max_pages_per_seq > MAX_PAGES_PER_SEQ) return SOL_ERR_UNSUPPORTED;
   if (B == 0) return SOL_OK;
   const Layout L = make_layout(*shape, B, kv->max_pages_per_seq);
   if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
@@ -438,6 +465,7 @@ static sol_status_t step_args_ok(const sol_shape_t* shape, int32_t n_layers, con
     if (!weights_ok(&layers[l]) || !kv_ok(&kvs[l])) return SOL_ERR_INVALID_ARG;
     if (kvs[l].max_pages_per_seq > mp) mp = kvs[l].max_pages_per_seq;
   }
+  if (mp > MAX_PAGES_PER_SEQ) return SOL_ERR_UNSUPPORTED;
   *max_pages = mp;
   return SOL_OK;
 }

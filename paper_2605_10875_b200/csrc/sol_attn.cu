@@ -39,83 +39,101 @@ struct PrepDev {
   const uint16_t* q_bf16;  // [B][Hq][hd] or nullptr
   float* q_rot;
   uint16_t* q_split;
+  int32_t* work_ctr;  // zeroed here: [0] items emitted, [1] next item, [2 + b*Hkv + kvh] finished items
   int* status;
 };
 
-__global__ void __launch_bounds__(256) attn_prep_kernel(const PrepDev p) {
+constexpr int PREP_THREADS = 128;
+
+// One CTA per (kv-head, sequence): the G query heads of the group, the new k row and the new v row.
+__global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p) {
   __shared__ float cs[64], sn[64];  // hd/2 <= 64
-  const int b = blockIdx.x;
+  const int kvh = blockIdx.x, b = blockIdx.y;
   const int Hq = p.sh.n_q_heads, Hkv = p.sh.n_kv_heads, hd = p.sh.head_dim, half = hd / 2;
   const int G = Hq / Hkv, HG = (G + 3) / 4;
+  const int tid = threadIdx.x;
   const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
   const int pos = T - 1;
   const bool layer = p.qkv != nullptr;
   const bool rope = layer && p.sh.rope_theta > 0.f;
-  if (threadIdx.x < half) {
+
+  if (tid == 0) {
+    p.work_ctr[2 + b * Hkv + kvh] = 0;
+    if (b == 0 && kvh == 0) {
+      p.work_ctr[0] = 0;
+      p.work_ctr[1] = 0;
+    }
+  }
+  if (tid < half) {
     float c = 1.f, s = 0.f;
     if (rope) {
-      const double inv = pow((double)p.sh.rope_theta, -2.0 * (double)threadIdx.x / (double)hd);
-      double sd, cd;
-      sincos((double)pos * inv, &sd, &cd);
-      c = (float)cd;
-      s = (float)sd;
+      // angle = pos * theta^(-2i/hd) in float64, reduced to [-pi, pi] before the float32 sine and cosine
+      const double inv = exp2(-2.0 * (double)tid / (double)hd * log2((double)p.sh.rope_theta));
+      const double a = (double)pos * inv;
+      const double k = rint(a * 0.15915494309189535);
+      const float r = (float)fma(-k, 6.283185307179586, a);
+      sincosf(r, &s, &c);
     }
-    cs[threadIdx.x] = c;
-    sn[threadIdx.x] = s;
+    cs[tid] = c;
+    sn[tid] = s;
   }
+  // zero the operand rows of this (sequence, kv-head): pad rows and the unused fourth slot stay zero
+  uint16_t* qs = p.q_split + (size_t)(b * Hkv + kvh) * HG * 16 * hd;
+  for (int i = tid * 8; i < HG * 16 * hd; i += PREP_THREADS * 8) *reinterpret_cast<uint4*>(qs + i) = make_uint4(0, 0, 0, 0);
   __syncthreads();
 
-  // zero the operand rows that carry no head (pad rows and the unused fourth slot)
-  uint16_t* qs = p.q_split + (size_t)b * Hkv * HG * 16 * hd;
-  for (int i = threadIdx.x; i < Hkv * HG * 16 * hd; i += blockDim.x) qs[i] = 0;
-  __syncthreads();
-
-  // queries
-  for (int i = threadIdx.x; i < Hq * hd; i += blockDim.x) {
-    const int h = i / hd, e = i % hd;
-    float q;
+  // queries of the group: element pair (f, f + half) of one head per iteration
+  for (int i = tid; i < G * half; i += PREP_THREADS) {
+    const int gi = i / half, f = i % half, h = kvh * G + gi;
+    float q0, q1;
     if (layer) {
       const float* src = p.qkv + (size_t)b * p.ldq + h * hd;
-      const int f = e < half ? e : e - half;
-      const float other = e < half ? -src[e + half] : src[e - half];
-      q = src[e] * cs[f] + other * sn[f];
+      const float x0 = src[f], x1 = src[f + half];
+      q0 = x0 * cs[f] + (-x1) * sn[f];
+      q1 = x1 * cs[f] + x0 * sn[f];
     } else {
-      q = bf2f(p.q_bf16[((size_t)b * Hq + h) * hd + e]);
+      const uint16_t* src = p.q_bf16 + ((size_t)b * Hq + h) * hd;
+      q0 = bf2f(src[f]);
+      q1 = bf2f(src[f + half]);
     }
-    p.q_rot[((size_t)b * Hq + h) * hd + e] = q;
-    const uint16_t hi = f2bf(q);
-    const float r1 = q - bf2f(hi);
-    const uint16_t mid = f2bf(r1);
-    const float r2 = r1 - bf2f(mid);
-    const uint16_t lo = f2bf(r2);
-    const int kvh = h / G, gi = h % G, hg = gi >> 2, t = gi & 3;
-    uint16_t* base = qs + ((size_t)(kvh * HG + hg) * 16) * hd + e;
-    base[(2 * t) * hd] = hi;
-    base[(2 * t + 1) * hd] = mid;
-    base[(8 + 2 * t) * hd] = lo;
+    float* qr = p.q_rot + ((size_t)b * Hq + h) * hd;
+    qr[f] = q0;
+    qr[f + half] = q1;
+    const int hg = gi >> 2, t = gi & 3;
+    uint16_t* base = qs + (size_t)(hg * 16) * hd;
+#pragma unroll
+    for (int w = 0; w < 2; ++w) {
+      const float q = w ? q1 : q0;
+      const int e = w ? f + half : f;
+      const uint16_t hi = f2bf(q);
+      const float r1 = q - bf2f(hi);
+      const uint16_t mid = f2bf(r1);
+      const float r2 = r1 - bf2f(mid);
+      base[(2 * t) * hd + e] = hi;
+      base[(2 * t + 1) * hd + e] = mid;
+      base[(8 + 2 * t) * hd + e] = f2bf(r2);
+    }
   }
 
-  if (!layer) return;
+  if (!layer || T <= 0) return;
   // new k (rotated) and v, rounded to bf16, written at position T-1
-  if (T <= 0) return;
   const int lp = pos / PAGE, slot = pos % PAGE;
   const int page = lp < p.kv.max_pages_per_seq ? p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + lp] : -1;
   if (page < 0 || page >= p.kv.num_pages) {
-    if (threadIdx.x == 0) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+    if (tid == 0) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
     return;
   }
   uint16_t* kp = static_cast<uint16_t*>(p.kv.k_pool);
   uint16_t* vp = static_cast<uint16_t*>(p.kv.v_pool);
-  for (int i = threadIdx.x; i < Hkv * hd; i += blockDim.x) {
-    const int h = i / hd, e = i % hd;
-    const float* ks = p.qkv + (size_t)b * p.ldq + (Hq + h) * hd;
-    const float* vs = p.qkv + (size_t)b * p.ldq + (Hq + Hkv + h) * hd;
-    const int f = e < half ? e : e - half;
-    const float other = e < half ? -ks[e + half] : ks[e - half];
-    const float k = ks[e] * cs[f] + other * sn[f];
-    const size_t dst = (((size_t)page * Hkv + h) * PAGE + slot) * hd + e;
-    kp[dst] = f2bf(k);
-    vp[dst] = f2bf(vs[e]);
+  const float* ks = p.qkv + (size_t)b * p.ldq + (Hq + kvh) * hd;
+  const float* vs = p.qkv + (size_t)b * p.ldq + (Hq + Hkv + kvh) * hd;
+  const size_t dst = (((size_t)page * Hkv + kvh) * PAGE + slot) * hd;
+  for (int f = tid; f < half; f += PREP_THREADS) {
+    const float x0 = ks[f], x1 = ks[f + half];
+    kp[dst + f] = f2bf(x0 * cs[f] + (-x1) * sn[f]);
+    kp[dst + f + half] = f2bf(x1 * cs[f] + x0 * sn[f]);
+    vp[dst + f] = f2bf(vs[f]);
+    vp[dst + f + half] = f2bf(vs[f + half]);
   }
 }
 
@@ -230,282 +248,417 @@ struct SelectDev {
   sol_shape_t sh;
   sol_kv_t kv;
   const int32_t* r_permille;
-  int Tmax;
+  int Tmax, S, split_len;
   const float* q_rot;
-  float* sigma;  // candidates are overwritten with +-inf once decided
+  const float* sigma;
   int32_t* kept_idx;
   int32_t* kept_cnt;
+  int32_t* work_items;
+  int32_t* work_ctr;
   int* status;
 };
 
+// One CTA per (sequence, kv-head).  The scores are copied to shared memory once; every later pass
+// (radix digits, window scan, compaction) reads them from there.  Decided candidates are marked by
+// overwriting the shared copy with +-inf.
 __global__ void __launch_bounds__(SEL_THREADS) token_select_kernel(const SelectDev p) {
+  extern __shared__ __align__(16) float sv[];  // [T] scores of this (sequence, kv-head)
   __shared__ SelectSmem sm;
   __shared__ double qsum[128];
 
   const int kvh = blockIdx.x, b = blockIdx.y;
   const int Hkv = p.sh.n_kv_heads, hd = p.sh.head_dim, G = p.sh.n_q_heads / Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bk = b * Hkv + kvh;
   const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
-  const size_t row = ((size_t)b * Hkv + kvh) * p.Tmax;
-  float* sig = p.sigma + row;
-  if (T <= 0) {
-    if (tid == 0) p.kept_cnt[b * Hkv + kvh] = 0;
-    return;
-  }
-  const int n_sink = min(max(p.sh.n_sink, 0), T);
-  const int n_win = min(max(p.sh.n_window, 0), T - n_sink);
-  const int nf = n_sink + n_win;
-  long long bud = ((long long)p.r_permille[b] * T + 999) / 1000;
-  if (bud > T) bud = T;
-  const int k = min(T, max((int)bud, nf));
-  auto forced = [&](int j) { return j < n_sink || j >= T - n_win; };
+  const size_t row = (size_t)bk * p.Tmax;
+  const float* sig = p.sigma + row;
 
-  // mode 0: keep all; 1: forced only; 2: kept iff sigma > thr (candidates already decided and
-  // overwritten with +-inf); 3: key threshold with index-ordered ties (float32 ordering)
-  float thr = 0.f;
-  uint32_t key_thr = 0;
-  int tie_need = 0;
-  int mode;
+  int total = 0;
+  if (T > 0) {
+    const int n_sink = min(max(p.sh.n_sink, 0), T);
+    const int n_win = min(max(p.sh.n_window, 0), T - n_sink);
+    const int nf = n_sink + n_win;
+    long long bud = ((long long)p.r_permille[b] * T + 999) / 1000;
+    if (bud > T) bud = T;
+    const int k = min(T, max((int)bud, nf));
+    auto forced = [&](int j) { return j < n_sink || j >= T - n_win; };
 
-  if (k >= T) {
-    mode = 0;
-  } else if (k <= nf) {
-    mode = 1;
-  } else {
-    key_thr = radix_select_kth(
-        [&](int j) { return forced(j) ? 0xffffffffu : float_key(sig[j] + 0.0f); }, T, k, tie_need, sm);
-    mode = 3;
+    // mode 0: keep all; 1: forced only; 2: kept iff score > thr (candidates already decided and
+    // overwritten with +-inf); 3: key threshold with index-ordered ties (float32 ordering)
+    float thr = 0.f;
+    uint32_t key_thr = 0;
+    int tie_need = 0;
+    int mode;
 
-    // ---- window around the threshold, re-scored in float64 ----
-    const float thr32 = key_to_float(key_thr);
-    float mx = 0.f;
-    for (int j = tid; j < T; j += SEL_THREADS)
-      if (!forced(j)) mx = fmaxf(mx, fabsf(sig[j]));
-    mx = warp_max(mx);
-    if (lane == 0) sm.f[warp] = mx;
-    if (tid < 4) sm.counts[tid] = 0;
-    __syncthreads();
-    mx = sm.f[0];
-    for (int i = 1; i < SEL_WARPS; ++i) mx = fmaxf(mx, sm.f[i]);
-    // 2^-16 of the largest score: far above the float32 accumulation error of a head_dim-long dot product
-    const float delta = mx * 1.52587890625e-05f;
-    const float hi = thr32 + delta, lo = thr32 - delta;
-    int n_in = 0;
-    for (int j = tid; j < T; j += SEL_THREADS) {
-      if (forced(j)) continue;
-      const float s = sig[j] + 0.0f;
-      if (s > hi) {
-        ++n_in;
-      } else if (s >= lo) {
-        const int slot = atomicAdd(&sm.counts[0], 1);
-        if (slot < SEL_CAND_CAP) sm.cand_idx[slot] = j;
-      }
-    }
-    if (n_in) atomicAdd(&sm.counts[1], n_in);
-    __syncthreads();
-    const int n_cand = sm.counts[0];
-    const int need = k - nf - sm.counts[1];
-    if (n_cand > SEL_CAND_CAP) {
-      if (tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
+    if (k >= T) {
+      mode = 0;
+    } else if (k <= nf) {
+      mode = 1;
     } else {
-      if (n_cand != need) {
-        if (tid == 0) atomicAdd(p.status + ST_TOK_REFINED, n_cand);
-        for (int e = tid; e < hd; e += SEL_THREADS) {
-          double a = 0.0;
-          for (int h = 0; h < G; ++h) a += (double)p.q_rot[((size_t)b * p.sh.n_q_heads + kvh * G + h) * hd + e];
-          qsum[e] = a;
-        }
-        __syncthreads();
-        const uint16_t* kp = static_cast<const uint16_t*>(p.kv.k_pool);
-        for (int c = warp; c < n_cand; c += SEL_WARPS) {
-          const int j = sm.cand_idx[c];
-          const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + j / PAGE];
-          double a = 0.0;
-          if (page >= 0 && page < p.kv.num_pages) {
-            const uint16_t* kr = kp + (((size_t)page * Hkv + kvh) * PAGE + (j % PAGE)) * hd;
-            for (int e = lane; e < hd; e += 32) a += qsum[e] * (double)bf2f(kr[e]);
-          }
-          a = warp_sum_d(a);
-          if (lane == 0) sm.cand_val[c] = a;
-        }
-        __syncthreads();
-        rank_candidates(n_cand, need, sm, [&](int c, bool keep) { sig[sm.cand_idx[c]] = keep ? INFINITY : -INFINITY; });
-      } else {
-        for (int c = tid; c < n_cand; c += SEL_THREADS) sig[sm.cand_idx[c]] = INFINITY;
+      float mx = 0.f;
+      for (int j = tid; j < T; j += SEL_THREADS) {
+        const float s = sig[j] + 0.0f;
+        sv[j] = s;
+        if (!forced(j)) mx = fmaxf(mx, fabsf(s));
       }
-      thr = hi;
-      mode = 2;
+      mx = warp_max(mx);
+      if (lane == 0) sm.f[warp] = mx;
+      if (tid < 4) sm.counts[tid] = 0;
       __syncthreads();
+      mx = sm.f[0];
+      for (int i = 1; i < SEL_WARPS; ++i) mx = fmaxf(mx, sm.f[i]);
+
+      key_thr = radix_select_kth([&](int j) { return forced(j) ? 0xffffffffu : float_key(sv[j]); }, T, k, tie_need, sm);
+      mode = 3;
+
+      // ---- window around the threshold, re-scored in float64 ----
+      const float thr32 = key_to_float(key_thr);
+      // 2^-16 of the largest score: far above the float32 accumulation error of a head_dim-long dot product
+      const float delta = mx * 1.52587890625e-05f;
+      const float hi = thr32 + delta, lo = thr32 - delta;
+      int n_in = 0;
+      for (int j = tid; j < T; j += SEL_THREADS) {
+        if (forced(j)) continue;
+        const float s = sv[j];
+        if (s > hi) {
+          ++n_in;
+        } else if (s >= lo) {
+          const int slot = atomicAdd(&sm.counts[0], 1);
+          if (slot < SEL_CAND_CAP) sm.cand_idx[slot] = j;
+        }
+      }
+      if (n_in) atomicAdd(&sm.counts[1], n_in);
+      __syncthreads();
+      const int n_cand = sm.counts[0];
+      const int need = k - nf - sm.counts[1];
+      if (n_cand > SEL_CAND_CAP) {
+        if (tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
+      } else {
+        if (n_cand != need) {
+          if (tid == 0) atomicAdd(p.status + ST_TOK_REFINED, n_cand);
+          for (int e = tid; e < hd; e += SEL_THREADS) {
+            double a = 0.0;
+            for (int h = 0; h < G; ++h) a += (double)p.q_rot[((size_t)b * p.sh.n_q_heads + kvh * G + h) * hd + e];
+            qsum[e] = a;
+          }
+          __syncthreads();
+          const uint16_t* kp = static_cast<const uint16_t*>(p.kv.k_pool);
+          for (int c = warp; c < n_cand; c += SEL_WARPS) {
+            const int j = sm.cand_idx[c];
+            const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + j / PAGE];
+            double a = 0.0;
+            if (page >= 0 && page < p.kv.num_pages) {
+              const uint16_t* kr = kp + (((size_t)page * Hkv + kvh) * PAGE + (j % PAGE)) * hd;
+              for (int e = lane; e < hd; e += 32) a += qsum[e] * (double)bf2f(kr[e]);
+            }
+            a = warp_sum_d(a);
+            if (lane == 0) sm.cand_val[c] = a;
+          }
+          __syncthreads();
+          rank_candidates(n_cand, need, sm, [&](int c, bool keep) { sv[sm.cand_idx[c]] = keep ? INFINITY : -INFINITY; });
+        } else {
+          for (int c = tid; c < n_cand; c += SEL_THREADS) sv[sm.cand_idx[c]] = INFINITY;
+        }
+        thr = hi;
+        mode = 2;
+        __syncthreads();
+      }
     }
+
+    auto klass = [&](int j) -> int {
+      if (mode == 0) return 2;
+      if (forced(j)) return 2;
+      if (mode == 1) return 0;
+      const float s = sv[j];
+      if (mode == 2) return s > thr ? 2 : 0;
+      const uint32_t key = float_key(s);
+      return key > key_thr ? 2 : (key == key_thr ? 1 : 0);
+    };
+    ordered_compact(klass, [](int, bool) {}, T, mode == 3 ? tie_need : 0, p.kept_idx + row, p.kept_cnt + bk, sm);
+    total = k;  // the compaction keeps exactly k indices
+  } else if (tid == 0) {
+    p.kept_cnt[bk] = 0;
   }
 
-  auto klass = [&](int j) -> int {
-    if (mode == 0) return 2;
-    if (forced(j)) return 2;
-    if (mode == 1) return 0;
-    const float s = sig[j] + 0.0f;
-    if (mode == 2) return s > thr ? 2 : 0;
-    const uint32_t key = float_key(s);
-    return key > key_thr ? 2 : (key == key_thr ? 1 : 0);
-  };
-  ordered_compact(klass, [](int, bool) {}, T, mode == 3 ? tie_need : 0, p.kept_idx + row,
-                  p.kept_cnt + (b * Hkv + kvh), sm);
+  // pass-2 work items of this (sequence, kv-head): one per split_len kept tokens, at least one so
+  // that the output is always written
+  const int ns = max(1, (total + p.split_len - 1) / p.split_len);
+  __syncthreads();
+  if (tid == 0) sm.pick[0] = atomicAdd(p.work_ctr, ns);
+  __syncthreads();
+  const int base = sm.pick[0];
+  for (int i = tid; i < ns; i += SEL_THREADS) p.work_items[base + i] = bk * p.S + i;
 }
 
 // ============================================================================
-// attn_gather (pass 2) and combine
+// attn_gather (pass 2) with the combine step folded in
 // ============================================================================
 struct GatherDev {
   sol_kv_t kv;
-  int Hkv, G, Tmax, S;
+  int Hq, Hkv, G, Tmax, S;
   const float* logits;
   const int32_t* kept_idx;
   const int32_t* kept_cnt;
+  const int32_t* work_items;
+  int32_t* work_ctr;
   float* part;  // [B][Hkv][S][G][HD + 2]
   float scale_log2;
-  int* status;
-};
-
-__device__ __forceinline__ void softmax_merge(float& m, float& l, float* acc, int n, float m2, float l2,
-                                              const float* acc2) {
-  const float mn = fmaxf(m, m2);
-  const float e1 = (m == -INFINITY) ? 0.f : exp2f(m - mn);
-  const float e2 = (m2 == -INFINITY) ? 0.f : exp2f(m2 - mn);
-  l = l * e1 + l2 * e2;
-  for (int i = 0; i < n; ++i) acc[i] = acc[i] * e1 + acc2[i] * e2;
-  m = mn;
-}
-
-constexpr int GA_WARPS = 4;
-
-template <int HD, int GMAX>
-__global__ void __launch_bounds__(GA_WARPS * 32) attn_gather_kernel(const GatherDev p) {
-  constexpr int LPT = HD / 8;       // lanes per token row (16 bytes each)
-  constexpr int TPW = 32 / LPT;     // tokens per warp iteration
-  __shared__ float sh_acc[GA_WARPS][GMAX][HD];
-  __shared__ float sh_ml[GA_WARPS][GMAX][2];
-  const int s = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int cnt = p.kept_cnt[b * p.Hkv + kvh];
-  const int n0 = s * ATTN_SPLIT_LEN, n1 = min(cnt, n0 + ATTN_SPLIT_LEN);
-  if (n0 >= n1) return;
-  const size_t row = ((size_t)b * p.Hkv + kvh) * p.Tmax;
-  const int grp = lane / LPT, sub = lane % LPT;
-  const uint16_t* vp = static_cast<const uint16_t*>(p.kv.v_pool);
-  const int G = p.G;
-
-  float m[GMAX], l[GMAX], acc[GMAX][8];
-#pragma unroll
-  for (int h = 0; h < GMAX; ++h) {
-    m[h] = -INFINITY;
-    l[h] = 0.f;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) acc[h][e] = 0.f;
-  }
-
-  for (int n = n0 + warp * TPW + grp; n < n1; n += GA_WARPS * TPW) {
-    const int j = p.kept_idx[row + n];
-    const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + j / PAGE];
-    if (page < 0 || page >= p.kv.num_pages) {
-      atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
-      continue;
-    }
-    const uint4 vw = *reinterpret_cast<const uint4*>(vp + (((size_t)page * p.Hkv + kvh) * PAGE + (j % PAGE)) * HD + sub * 8);
-    const float v[8] = {bf16_lo(vw.x), bf16_hi(vw.x), bf16_lo(vw.y), bf16_hi(vw.y),
-                        bf16_lo(vw.z), bf16_hi(vw.z), bf16_lo(vw.w), bf16_hi(vw.w)};
-    const float* lg = p.logits + (row + j) * G;
-#pragma unroll
-    for (int h = 0; h < GMAX; ++h) {
-      if (h < G) {
-        const float x = lg[h] * p.scale_log2;
-        const float mn = fmaxf(m[h], x);
-        const float corr = exp2f(m[h] - mn);  // m = -inf gives 0
-        const float pw = exp2f(x - mn);
-        l[h] = l[h] * corr + pw;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[h][e] = acc[h][e] * corr + pw * v[e];
-        m[h] = mn;
-      }
-    }
-  }
-
-  // merge the token groups of the warp (lanes with equal `sub` hold the same dims)
-#pragma unroll
-  for (int o = LPT; o < 32; o <<= 1) {
-#pragma unroll
-    for (int h = 0; h < GMAX; ++h) {
-      if (h < G) {
-        const float m2 = __shfl_xor_sync(0xffffffffu, m[h], o);
-        const float l2 = __shfl_xor_sync(0xffffffffu, l[h], o);
-        float a2[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) a2[e] = __shfl_xor_sync(0xffffffffu, acc[h][e], o);
-        softmax_merge(m[h], l[h], acc[h], 8, m2, l2, a2);
-      }
-    }
-  }
-  if (grp == 0) {
-#pragma unroll
-    for (int h = 0; h < GMAX; ++h) {
-      if (h < G) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) sh_acc[warp][h][sub * 8 + e] = acc[h][e];
-        if (sub == 0) {
-          sh_ml[warp][h][0] = m[h];
-          sh_ml[warp][h][1] = l[h];
-        }
-      }
-    }
-  }
-  __syncthreads();
-  // merge the warps and write the partial of this split
-  float* dst = p.part + (((size_t)(b * p.Hkv + kvh) * p.S + s) * G) * (HD + 2);
-  for (int i = threadIdx.x; i < G * HD; i += GA_WARPS * 32) {
-    const int h = i / HD, e = i % HD;
-    float mm = sh_ml[0][h][0], ll = sh_ml[0][h][1], a = sh_acc[0][h][e];
-    for (int w = 1; w < GA_WARPS; ++w) {
-      const float a2 = sh_acc[w][h][e];
-      softmax_merge(mm, ll, &a, 1, sh_ml[w][h][0], sh_ml[w][h][1], &a2);
-    }
-    dst[h * (HD + 2) + e] = a;
-    if (e == 0) {
-      dst[h * (HD + 2) + HD] = mm;
-      dst[h * (HD + 2) + HD + 1] = ll;
-    }
-  }
-}
-
-struct CombineDev {
-  int Hq, Hkv, G, hd, S;
-  const int32_t* kept_cnt;
-  const float* part;
   float* out_f32;
   uint16_t* out_bf16;
   uint16_t* out_hi;
   uint16_t* out_lo;
+  int* status;
 };
 
-__global__ void attn_combine_kernel(const CombineDev p) {
-  const int b = blockIdx.y, h = blockIdx.x;
-  const int kvh = h / p.G, gi = h % p.G;
-  const int cnt = p.kept_cnt[b * p.Hkv + kvh];
-  const int ns = (cnt + ATTN_SPLIT_LEN - 1) / ATTN_SPLIT_LEN;
-  const int e = threadIdx.x;
-  if (e >= p.hd) return;
-  float m = -INFINITY, l = 0.f, a = 0.f;
-  for (int s = 0; s < ns; ++s) {
-    const float* src = p.part + ((((size_t)(b * p.Hkv + kvh) * p.S + s) * p.G) + gi) * (p.hd + 2);
-    const float a2 = src[e];
-    softmax_merge(m, l, &a, 1, src[p.hd], src[p.hd + 1], &a2);
-  }
-  const float o = l > 0.f ? a / l : 0.f;
-  const size_t idx = ((size_t)b * p.Hq + h) * p.hd + e;
-  if (p.out_f32) p.out_f32[idx] = o;
-  if (p.out_bf16) p.out_bf16[idx] = f2bf(o);
-  if (p.out_hi) {
-    const uint16_t hi = f2bf(o);
-    p.out_hi[idx] = hi;
-    p.out_lo[idx] = f2bf(o - bf2f(hi));
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+// waits until at most n (0..3) of this thread's copy groups are still in flight
+__device__ __forceinline__ void cp_async_wait_dyn(int n) {
+  if (n <= 0) cp_async_wait<0>();
+  else if (n == 1) cp_async_wait<1>();
+  else if (n == 2) cp_async_wait<2>();
+  else cp_async_wait<3>();
+}
+
+constexpr int GA_WARPS = 4;
+constexpr int GA_THREADS = GA_WARPS * 32;
+
+template <int HD, int GMAX>
+struct GatherLayout {
+  static constexpr int SPLIT = HD == 64 ? 256 : 128;  // kept tokens per work item (attn_split_len)
+  static constexpr int TPW = SPLIT / GA_WARPS;        // tokens per warp
+  static constexpr int KSTEPS = TPW / 16;             // MMA k-steps per warp
+  static constexpr int ROW_STRIDE = HD * 2 + 16;      // bytes; +16 keeps ldmatrix rows on distinct banks
+  static constexpr int P_STRIDE = SPLIT + 8;          // bf16 elements; +8 spreads the heads over the banks
+  static constexpr int V_BYTES = SPLIT * ROW_STRIDE;
+  static constexpr int P_BYTES = 2 * GMAX * P_STRIDE * 2;
+  static constexpr int ROWIDX_BYTES = SPLIT * 4;
+  static constexpr int BYTES = V_BYTES + P_BYTES + ROWIDX_BYTES + 64;
+  static_assert(KSTEPS >= 1 && KSTEPS <= 4, "copy groups are waited on with at most 3 in flight");
+  static_assert(GA_WARPS * GMAX * (HD + 2) * 4 <= V_BYTES, "the merge scratch reuses the V tile");
+};
+
+// Persistent CTAs take (sequence, kv-head, split) items from the work list.  Per item each warp owns
+// a quarter of the kept tokens: it resolves their V row addresses, starts all row copies (cp.async,
+// one commit group per 16 tokens), turns the kept logits into softmax weights relative to the warp's
+// own maximum, and multiplies weights by rows on the tensor cores as the groups land: the weights
+// (bf16 high part in MMA rows 0..G-1, low part in rows 8..8+G-1) are the A operand, the V rows the
+// B operand.  The CTA that finishes the last item of a (sequence, kv-head) merges its partials.
+template <int HD, int GMAX>
+__global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev p) {
+  using L = GatherLayout<HD, GMAX>;
+  extern __shared__ __align__(128) unsigned char smem[];
+  unsigned char* vt = smem;
+  uint16_t* p_hi = reinterpret_cast<uint16_t*>(smem + L::V_BYTES);
+  uint16_t* p_lo = p_hi + GMAX * L::P_STRIDE;
+  uint32_t* rowidx = reinterpret_cast<uint32_t*>(smem + L::V_BYTES + L::P_BYTES);
+  int* flag = reinterpret_cast<int*>(smem + L::V_BYTES + L::P_BYTES + L::ROWIDX_BYTES);
+  float* sc_acc = reinterpret_cast<float*>(smem);                        // [GA_WARPS][GMAX][HD], after the MMAs
+  float* sc_ml = sc_acc + GA_WARPS * GMAX * HD;                          // [GA_WARPS][GMAX][2]
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int G = p.G, Hkv = p.Hkv;
+  const uint16_t* vp = static_cast<const uint16_t*>(p.kv.v_pool);
+  constexpr int CH = HD / 8;  // 16-byte chunks per row
+
+  for (;;) {
+    if (tid == 0) {
+      const int it = atomicAdd(p.work_ctr + 1, 1);
+      flag[0] = it < p.work_ctr[0] ? p.work_items[it] : -1;
+    }
+    __syncthreads();
+    const int item = flag[0];
+    if (item < 0) break;
+    const int bk = item / p.S, s = item % p.S;
+    const int b = bk / Hkv, kvh = bk % Hkv;
+    const int cnt = p.kept_cnt[bk];
+    const int n0 = s * L::SPLIT, n1 = min(cnt, n0 + L::SPLIT);
+    const size_t row = (size_t)bk * p.Tmax;
+    const int tok0 = warp * L::TPW;  // first token slot of this warp within the item
+
+    // ---- row addresses of this warp's tokens ----
+    int jj[L::TPW / 32];
+#pragma unroll
+    for (int i = 0; i < L::TPW / 32; ++i) {
+      const int slot = tok0 + lane + 32 * i;
+      const int n = n0 + slot;
+      uint32_t ridx = 0xffffffffu;
+      jj[i] = -1;
+      if (n < n1) {
+        const int j = p.kept_idx[row + n];
+        const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + j / PAGE];
+        if (page >= 0 && page < p.kv.num_pages) {
+          ridx = (uint32_t)((page * Hkv + kvh) * PAGE + (j % PAGE));
+          jj[i] = j;
+        } else {
+          atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+        }
+      }
+      rowidx[slot] = ridx;
+    }
+    __syncwarp();
+
+    // ---- start every row copy; rows of absent tokens are zero-filled ----
+#pragma unroll
+    for (int ks = 0; ks < L::KSTEPS; ++ks) {
+#pragma unroll
+      for (int i = 0; i < 16 * CH / 32; ++i) {
+        const int c = lane + 32 * i;
+        const int slot = tok0 + ks * 16 + c / CH, ch = c % CH;
+        const uint32_t ridx = rowidx[slot];
+        unsigned char* dst = vt + slot * L::ROW_STRIDE + ch * 16;
+        if (ridx != 0xffffffffu) cp_async16(smem_u32(dst), vp + (size_t)ridx * HD + ch * 8);
+        else *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+      }
+      cp_async_commit();
+    }
+
+    // ---- softmax weights relative to the warp's maximum ----
+    float x[L::TPW / 32][GMAX];
+    float mh[GMAX], lh[GMAX];
+#pragma unroll
+    for (int h = 0; h < GMAX; ++h) mh[h] = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < L::TPW / 32; ++i) {
+#pragma unroll
+      for (int h = 0; h < GMAX; ++h) {
+        x[i][h] = -INFINITY;
+        if (h < G && jj[i] >= 0) x[i][h] = p.logits[(row + jj[i]) * G + h] * p.scale_log2;
+        mh[h] = fmaxf(mh[h], x[i][h]);
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < GMAX; ++h) {
+      mh[h] = warp_max(mh[h]);
+      lh[h] = 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < L::TPW / 32; ++i) {
+      const int slot = tok0 + lane + 32 * i;
+#pragma unroll
+      for (int h = 0; h < GMAX; ++h) {
+        if (h < G) {
+          const float pw = x[i][h] == -INFINITY ? 0.f : exp2f(x[i][h] - mh[h]);
+          lh[h] += pw;
+          const uint16_t hi = f2bf(pw);
+          p_hi[h * L::P_STRIDE + slot] = hi;
+          p_lo[h * L::P_STRIDE + slot] = f2bf(pw - bf2f(hi));
+        }
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < GMAX; ++h) lh[h] = warp_sum(lh[h]);
+    __syncwarp();
+
+    // ---- weights x rows on the tensor cores, as the copy groups land ----
+    float acc[HD / 8][4];
+#pragma unroll
+    for (int nt = 0; nt < HD / 8; ++nt)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) acc[nt][r] = 0.f;
+    const int mi = lane >> 3, mr = lane & 7;  // ldmatrix: this lane addresses row mr of matrix mi
+#pragma unroll
+    for (int ks = 0; ks < L::KSTEPS; ++ks) {
+      cp_async_wait_dyn(L::KSTEPS - 1 - ks);
+      __syncwarp();
+      const int kb = tok0 + ks * 16;
+      uint32_t a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+      if (g < G) {
+        a0 = *reinterpret_cast<const uint32_t*>(p_hi + g * L::P_STRIDE + kb + 2 * t);
+        a1 = *reinterpret_cast<const uint32_t*>(p_lo + g * L::P_STRIDE + kb + 2 * t);
+        a2 = *reinterpret_cast<const uint32_t*>(p_hi + g * L::P_STRIDE + kb + 8 + 2 * t);
+        a3 = *reinterpret_cast<const uint32_t*>(p_lo + g * L::P_STRIDE + kb + 8 + 2 * t);
+      }
+      const uint32_t vrow = smem_u32(vt) + (kb + (mi & 1) * 8 + mr) * L::ROW_STRIDE;
+#pragma unroll
+      for (int pr = 0; pr < HD / 16; ++pr) {
+        uint32_t bfr[4];
+        ldsm_x4_trans(bfr, vrow + ((2 * pr + (mi >> 1)) * 8) * 2);
+        mma_bf16(acc[2 * pr], a0, a1, a2, a3, bfr[0], bfr[1]);
+        mma_bf16(acc[2 * pr + 1], a0, a1, a2, a3, bfr[2], bfr[3]);
+      }
+    }
+    __syncthreads();  // every warp is done with the V tile: its space becomes the merge scratch
+
+    if (g < G) {
+#pragma unroll
+      for (int nt = 0; nt < HD / 8; ++nt) {
+        float* d = sc_acc + ((size_t)(warp * GMAX + g) * HD) + nt * 8 + 2 * t;
+        d[0] = acc[nt][0] + acc[nt][2];
+        d[1] = acc[nt][1] + acc[nt][3];
+      }
+    }
+    if (lane == 0) {
+#pragma unroll
+      for (int h = 0; h < GMAX; ++h) {
+        sc_ml[(warp * GMAX + h) * 2] = mh[h];
+        sc_ml[(warp * GMAX + h) * 2 + 1] = lh[h];
+      }
+    }
+    __syncthreads();
+    float* dst = p.part + (((size_t)bk * p.S + s) * G) * (HD + 2);
+    for (int i = tid; i < G * HD; i += GA_THREADS) {
+      const int h = i / HD, e = i % HD;
+      float M = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < GA_WARPS; ++w) M = fmaxf(M, sc_ml[(w * GMAX + h) * 2]);
+      float a = 0.f, l = 0.f;
+#pragma unroll
+      for (int w = 0; w < GA_WARPS; ++w) {
+        const float mw = sc_ml[(w * GMAX + h) * 2];
+        const float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
+        a += sc_acc[(size_t)(w * GMAX + h) * HD + e] * f;
+        l += sc_ml[(w * GMAX + h) * 2 + 1] * f;
+      }
+      dst[h * (HD + 2) + e] = a;
+      if (e == 0) {
+        dst[h * (HD + 2) + HD] = M;
+        dst[h * (HD + 2) + HD + 1] = l;
+      }
+    }
+
+    // ---- the last item of this (sequence, kv-head) merges the partials ----
+    const int ns = max(1, (cnt + L::SPLIT - 1) / L::SPLIT);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) flag[1] = atomicAdd(p.work_ctr + 2 + bk, 1) == ns - 1 ? 1 : 0;
+    __syncthreads();
+    if (flag[1]) {
+      __threadfence();
+      const float* src0 = p.part + ((size_t)bk * p.S * G) * (HD + 2);
+      for (int i = tid; i < G * HD; i += GA_THREADS) {
+        const int h = i / HD, e = i % HD;
+        float m = -INFINITY, l = 0.f, a = 0.f;
+        for (int q = 0; q < ns; ++q) {
+          const float* src = src0 + ((size_t)q * G + h) * (HD + 2);
+          const float m2 = __ldcg(src + HD), l2 = __ldcg(src + HD + 1), a2 = __ldcg(src + e);
+          const float mn = fmaxf(m, m2);
+          const float e1 = (m == -INFINITY) ? 0.f : exp2f(m - mn);
+          const float e2 = (m2 == -INFINITY) ? 0.f : exp2f(m2 - mn);
+          l = l * e1 + l2 * e2;
+          a = a * e1 + a2 * e2;
+          m = mn;
+        }
+        const float o = l > 0.f ? a / l : 0.f;
+        const size_t idx = ((size_t)b * p.Hq + kvh * G + h) * HD + e;
+        if (p.out_f32) p.out_f32[idx] = o;
+        if (p.out_bf16) p.out_bf16[idx] = f2bf(o);
+        if (p.out_hi) {
+          const uint16_t hi = f2bf(o);
+          p.out_hi[idx] = hi;
+          p.out_lo[idx] = f2bf(o - bf2f(hi));
+        }
+      }
+    }
+    __syncthreads();  // the scratch and the flags are reused by the next item
   }
 }
 
@@ -516,12 +669,19 @@ template <int HD>
 static void launch_score(const ScoreDev& d, int HG, dim3 grid, cudaStream_t st) {
   const int smem = SC_WARPS * PAGE * HD * 2 + SC_WARPS * 8 + 32;
   if (HG == 1) {
-    cudaFuncSetAttribute(attn_score_kernel<HD, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_score_kernel<HD, 1>), smem);
     SOL_LAUNCH("attn_score", (attn_score_kernel<HD, 1>), grid, dim3(SC_WARPS * 32), smem, st, d);
   } else {
-    cudaFuncSetAttribute(attn_score_kernel<HD, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_score_kernel<HD, 2>), smem);
     SOL_LAUNCH("attn_score", (attn_score_kernel<HD, 2>), grid, dim3(SC_WARPS * 32), smem, st, d);
   }
+}
+
+template <int HD, int GMAX>
+static void launch_gather(const GatherDev& d, int grid, cudaStream_t st) {
+  using L = GatherLayout<HD, GMAX>;
+  ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_gather_kernel<HD, GMAX>), L::BYTES);
+  SOL_LAUNCH("attn_gather_v", (attn_gather_kernel<HD, GMAX>), dim3(grid), dim3(GA_THREADS), L::BYTES, st, d);
 }
 
 void launch_attention(const AttnArgs& a, cudaStream_t st) {
@@ -532,8 +692,8 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   PrepDev pd;
   pd.sh = sh; pd.kv = a.kv; pd.qkv = a.qkv_f32; pd.ldq = a.ldq;
   pd.q_bf16 = static_cast<const uint16_t*>(a.q_bf16);
-  pd.q_rot = a.q_rot; pd.q_split = static_cast<uint16_t*>(a.q_split); pd.status = a.status;
-  SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(a.B), dim3(256), 0, st, pd);
+  pd.q_rot = a.q_rot; pd.q_split = static_cast<uint16_t*>(a.q_split); pd.work_ctr = a.work_ctr; pd.status = a.status;
+  SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(Hkv, a.B), dim3(PREP_THREADS), 0, st, pd);
 
   ScoreDev sd;
   sd.kv = a.kv; sd.Hkv = Hkv; sd.G = G; sd.HG = HG; sd.Tmax = Tmax;
@@ -544,30 +704,34 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   else launch_score<128>(sd, HG, sgrid, st);
 
   SelectDev se;
-  se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.q_rot = a.q_rot;
-  se.sigma = a.sigma; se.kept_idx = a.kept_idx; se.kept_cnt = a.kept_cnt; se.status = a.status;
-  SOL_LAUNCH("token_select", token_select_kernel, dim3(Hkv, a.B), dim3(SEL_THREADS), 0, st, se);
-
-  GatherDev gd;
-  gd.kv = a.kv; gd.Hkv = Hkv; gd.G = G; gd.Tmax = Tmax; gd.S = a.splits;
-  gd.logits = a.logits; gd.kept_idx = a.kept_idx; gd.kept_cnt = a.kept_cnt; gd.part = a.part;
-  gd.scale_log2 = (float)(1.4426950408889634 / sqrt((double)hd));
-  gd.status = a.status;
-  dim3 ggrid(a.splits, Hkv, a.B);
-  if (hd == 64) {
-    if (G <= 4) SOL_LAUNCH("attn_gather_v", (attn_gather_kernel<64, 4>), ggrid, dim3(GA_WARPS * 32), 0, st, gd);
-    else SOL_LAUNCH("attn_gather_v", (attn_gather_kernel<64, 8>), ggrid, dim3(GA_WARPS * 32), 0, st, gd);
-  } else {
-    if (G <= 4) SOL_LAUNCH("attn_gather_v", (attn_gather_kernel<128, 4>), ggrid, dim3(GA_WARPS * 32), 0, st, gd);
-    else SOL_LAUNCH("attn_gather_v", (attn_gather_kernel<128, 8>), ggrid, dim3(GA_WARPS * 32), 0, st, gd);
+  se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.S = a.splits;
+  se.split_len = attn_split_len(hd); se.q_rot = a.q_rot;
+  se.sigma = a.sigma; se.kept_idx = a.kept_idx; se.kept_cnt = a.kept_cnt;
+  se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
+  {
+    const int smem = Tmax * 4;
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&token_select_kernel), smem);
+    SOL_LAUNCH("token_select", token_select_kernel, dim3(Hkv, a.B), dim3(SEL_THREADS), smem, st, se);
   }
 
-  CombineDev cd;
-  cd.Hq = Hq; cd.Hkv = Hkv; cd.G = G; cd.hd = hd; cd.S = a.splits;
-  cd.kept_cnt = a.kept_cnt; cd.part = a.part; cd.out_f32 = a.out_f32;
-  cd.out_bf16 = static_cast<uint16_t*>(a.out_bf16);
-  cd.out_hi = static_cast<uint16_t*>(a.out_hi); cd.out_lo = static_cast<uint16_t*>(a.out_lo);
-  SOL_LAUNCH("attn_combine", attn_combine_kernel, dim3(Hq, a.B), dim3(hd), 0, st, cd);
+  GatherDev gd;
+  gd.kv = a.kv; gd.Hq = Hq; gd.Hkv = Hkv; gd.G = G; gd.Tmax = Tmax; gd.S = a.splits;
+  gd.logits = a.logits; gd.kept_idx = a.kept_idx; gd.kept_cnt = a.kept_cnt;
+  gd.work_items = a.work_items; gd.work_ctr = a.work_ctr; gd.part = a.part;
+  gd.scale_log2 = (float)(1.4426950408889634 / sqrt((double)hd));
+  gd.out_f32 = a.out_f32;
+  gd.out_bf16 = static_cast<uint16_t*>(a.out_bf16);
+  gd.out_hi = static_cast<uint16_t*>(a.out_hi); gd.out_lo = static_cast<uint16_t*>(a.out_lo);
+  gd.status = a.status;
+  const long long items = (long long)a.B * Hkv * a.splits;
+  const int grid = (int)(items < (long long)sm_count() * 5 ? items : (long long)sm_count() * 5);
+  if (hd == 64) {
+    if (G <= 4) launch_gather<64, 4>(gd, grid, st);
+    else launch_gather<64, 8>(gd, grid, st);
+  } else {
+    if (G <= 4) launch_gather<128, 4>(gd, grid, st);
+    else launch_gather<128, 8>(gd, grid, st);
+  }
 }
 
 }  // namespace sol

@@ -218,11 +218,7 @@ static void launch_nk_mt(const NKDev& d, int grid, cudaStream_t st) {
   const char* name = EPI == EPI_SWIGLU ? "gemm_gate_up_swiglu" : (EPI == EPI_RESIDUAL ? "gemm_out_proj" : "gemm_qkv");
 #define SOL_NK_CASE(MTV)                                                                                      \
   case MTV: {                                                                                                 \
-    static bool attr_done = false;                                                                            \
-    if (!attr_done) {                                                                                         \
-      cudaFuncSetAttribute(gemm_nk_kernel<EPI, MTV>, cudaFuncAttributeMaxDynamicSharedMemorySize, NK_SMEM);   \
-      attr_done = true;                                                                                       \
-    }                                                                                                         \
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&gemm_nk_kernel<EPI, MTV>), NK_SMEM);                   \
     SOL_LAUNCH(name, (gemm_nk_kernel<EPI, MTV>), dim3(grid), dim3(NK_THREADS), NK_SMEM, st, d);               \
   } break;
   switch (d.MT) {
@@ -417,7 +413,7 @@ void launch_gemm_down(const GemmDown& p, cudaStream_t st) {
   dim3 grid(p.d / DN_NS, p.chunks);
 #define SOL_DN_CASE(MTV)                                                                                  \
   case MTV: {                                                                                             \
-    cudaFuncSetAttribute(gemm_down_kernel<MTV>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);       \
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&gemm_down_kernel<MTV>), smem);                     \
     SOL_LAUNCH("gemm_down_gathered", gemm_down_kernel<MTV>, grid, dim3(DN_THREADS), smem, st, d);         \
   } break;
   switch (mt) {

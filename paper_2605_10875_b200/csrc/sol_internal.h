@@ -24,6 +24,10 @@ bool take_cuda_failure();  // true if a CUDA call of this thread failed since th
   } while (0)
 
 int sm_count();
+// Raises a kernel's dynamic shared memory limit to at least `bytes` on the current device
+// (remembered per device and kernel, so repeated calls cost a table lookup).
+void ensure_dynamic_smem(const void* kernel, int bytes);
+constexpr int MAX_PAGES_PER_SEQ = 768;  // 49152 tokens: the selection kernel keeps one float per token in shared memory
 
 // ---- quantizer / RMSNorm (sol_quant.cu) ------------------------------------
 // One token per CTA.  in: bf16 or float32 [B][d].  gamma == nullptr: no norm.
@@ -85,7 +89,9 @@ struct AttnArgs {
   int32_t* kept_idx; // [B][Hkv][Tmax]
   int32_t* kept_cnt; // [B][Hkv]
   float* part;       // [B][Hkv][S][G][hd + 2]
-  int splits;        // S
+  int splits;        // S = ceil(Tmax / attn_split_len(hd))
+  int32_t* work_items;  // [B*Hkv*S] pass-2 work list, filled by the selection kernel
+  int32_t* work_ctr;    // [2 + B*Hkv]: items emitted, next item to take, finished items per (sequence, kv-head)
   // outputs (each optional)
   float* out_f32;    // [B][Hq][hd]
   void* out_bf16;    // [B][Hq][hd]
@@ -93,7 +99,13 @@ struct AttnArgs {
   void* out_lo;
   int* status;
 };
-constexpr int ATTN_SPLIT_LEN = 512;  // kept tokens per pass-2 work item
+// Kept tokens per pass-2 work item: 32 KB of V rows.
+inline int attn_split_len(int head_dim) { return head_dim == 64 ? 256 : 128; }
+inline int attn_splits(int head_dim, int max_pages, int page_size) {
+  const int len = attn_split_len(head_dim);
+  const int s = (max_pages * page_size + len - 1) / len;
+  return s < 1 ? 1 : s;
+}
 void launch_attention(const AttnArgs& a, cudaStream_t st);
 
 // ---- MLP channel selection (sol_mlp.cu) -------------------------------------

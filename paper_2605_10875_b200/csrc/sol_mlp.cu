@@ -36,6 +36,7 @@ struct ChanDev {
 };
 
 __global__ void __launch_bounds__(SEL_THREADS) channel_select_kernel(const ChanDev p) {
+  extern __shared__ __align__(16) float tv[];  // [ff] silu(g)*u of this token
   __shared__ SelectSmem sm;
   const int b = blockIdx.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -50,22 +51,32 @@ __global__ void __launch_bounds__(SEL_THREADS) channel_select_kernel(const ChanD
   // decided candidates are recorded in the list itself: cand_idx[c] = j or ~j (dropped)
   int n_cand = 0;
 
+  // one pass over global memory: t into shared memory, and (when a selection is needed) the largest |g|, |u|
+  const bool select = m < ff && m > 0;
+  float gmax = 0.f, umax = 0.f;
+  {
+    const float* gg = p.g + (size_t)b * ff;
+    const float* uu = p.u + (size_t)b * ff;
+    for (int j = tid * 4; j < ff; j += SEL_THREADS * 4) {
+      *reinterpret_cast<float4*>(tv + j) = *reinterpret_cast<const float4*>(tt + j);
+      if (select) {
+        const float4 g4 = *reinterpret_cast<const float4*>(gg + j), u4 = *reinterpret_cast<const float4*>(uu + j);
+        gmax = fmaxf(fmaxf(gmax, fmaxf(fabsf(g4.x), fabsf(g4.y))), fmaxf(fabsf(g4.z), fabsf(g4.w)));
+        umax = fmaxf(fmaxf(umax, fmaxf(fabsf(u4.x), fabsf(u4.y))), fmaxf(fabsf(u4.z), fabsf(u4.w)));
+      }
+    }
+  }
+  __syncthreads();
+
   if (m >= ff) {
     mode = 0;
   } else if (m <= 0) {
     mode = 1;
   } else {
-    key_thr = radix_select_kth([&](int j) { return float_key(fabsf(tt[j])); }, ff, m, tie_need, sm);
+    key_thr = radix_select_kth([&](int j) { return float_key(fabsf(tv[j])); }, ff, m, tie_need, sm);
     mode = 3;
     const float thr32 = key_to_float(key_thr);
     // error window: |g|, |u| carry at most 2^-18 of their largest magnitude of float32 accumulation error
-    const float* gg = p.g + (size_t)b * ff;
-    const float* uu = p.u + (size_t)b * ff;
-    float gmax = 0.f, umax = 0.f;
-    for (int j = tid; j < ff; j += SEL_THREADS) {
-      gmax = fmaxf(gmax, fabsf(gg[j]));
-      umax = fmaxf(umax, fabsf(uu[j]));
-    }
     gmax = warp_max(gmax);
     umax = warp_max(umax);
     if (lane == 0) {
@@ -85,7 +96,7 @@ __global__ void __launch_bounds__(SEL_THREADS) channel_select_kernel(const ChanD
     const float hi = thr32 + delta, lo = thr32 - delta;
     int n_in = 0;
     for (int j = tid; j < ff; j += SEL_THREADS) {
-      const float s = fabsf(tt[j]);
+      const float s = fabsf(tv[j]);
       if (s > hi) {
         ++n_in;
       } else if (s >= lo) {
@@ -149,7 +160,7 @@ __global__ void __launch_bounds__(SEL_THREADS) channel_select_kernel(const ChanD
   auto klass = [&](int j) -> int {
     if (mode == 0) return 2;
     if (mode == 1) return 0;
-    const float s = fabsf(tt[j]);
+    const float s = fabsf(tv[j]);
     if (mode == 2) {
       if (s > thr) return 2;
       if (s >= thr_lo) {  // within the window: look the channel up in the decided list
@@ -166,7 +177,7 @@ __global__ void __launch_bounds__(SEL_THREADS) channel_select_kernel(const ChanD
   auto emit = [&](int j, bool keep) {
     uint16_t hi = 0, lo = 0;
     if (keep) {
-      const float v = tt[j];
+      const float v = tv[j];
       hi = f2bf(v);
       lo = f2bf(v - bf2f(hi));
       p.live[j >> 5] = 1;
@@ -186,7 +197,9 @@ void launch_channel_select(const ChannelSelectArgs& a, cudaStream_t st) {
   c.t_hi = static_cast<uint16_t*>(a.t_hi); c.t_lo = static_cast<uint16_t*>(a.t_lo);
   c.live = a.live; c.status = a.status;
   cudaMemsetAsync(a.live, 0, sizeof(int32_t) * (a.ff / 32), st);
-  SOL_LAUNCH("channel_select", channel_select_kernel, dim3(a.B), dim3(SEL_THREADS), 0, st, c);
+  const int smem = a.ff * 4;
+  ensure_dynamic_smem(reinterpret_cast<const void*>(&channel_select_kernel), smem);
+  SOL_LAUNCH("channel_select", channel_select_kernel, dim3(a.B), dim3(SEL_THREADS), smem, st, c);
 }
 
 }  // namespace sol

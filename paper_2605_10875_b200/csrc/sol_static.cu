@@ -46,7 +46,7 @@ sol_status_t scratch_of_current_device(unsigned char** out) {
 }
 
 struct StaticLayout {
-  size_t status, q_rot, q_split, logits, sigma, kept_idx, kept_cnt, part, total;
+  size_t status, q_rot, q_split, logits, sigma, kept_idx, kept_cnt, part, work_items, work_ctr, total;
   int splits;
 };
 
@@ -54,7 +54,7 @@ StaticLayout layout_for(const sol_shape_t& s, int B, int max_pages) {
   StaticLayout L;
   const size_t Hq = s.n_q_heads, Hkv = s.n_kv_heads, hd = s.head_dim, G = Hq / Hkv, HG = (G + 3) / 4;
   const size_t Tmax = (size_t)max_pages * s.page_size;
-  L.splits = (int)((Tmax + sol::ATTN_SPLIT_LEN - 1) / sol::ATTN_SPLIT_LEN);
+  L.splits = sol::attn_splits(s.head_dim, max_pages, s.page_size);
   size_t at = 0;
   auto take = [&](size_t bytes) {
     const size_t o = at;
@@ -69,6 +69,8 @@ StaticLayout layout_for(const sol_shape_t& s, int B, int max_pages) {
   L.kept_idx = take(B * Hkv * Tmax * 4);
   L.kept_cnt = take(B * Hkv * 4);
   L.part = take(B * Hkv * (size_t)L.splits * G * (hd + 2) * 4);
+  L.work_items = take(B * Hkv * (size_t)L.splits * 4);
+  L.work_ctr = take((2 + B * Hkv) * 4);
   L.total = at;
   return L;
 }
@@ -91,7 +93,7 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
   if (!shape || !q_bf16 || !kv || !kv->k_pool || !kv->v_pool || !kv->page_table || !kv->seq_lens ||
       kv->max_pages_per_seq <= 0 || kv->num_pages <= 0 || !r_permille || !out_bf16 || B < 0)
     return SOL_ERR_INVALID_ARG;
-  if (!attention_shape_ok(shape) || B > 128) return SOL_ERR_UNSUPPORTED;
+  if (!attention_shape_ok(shape) || B > 128 || kv->max_pages_per_seq > sol::MAX_PAGES_PER_SEQ) return SOL_ERR_UNSUPPORTED;
   if (B == 0) return SOL_OK;
   const StaticLayout L = layout_for(*shape, B, kv->max_pages_per_seq);
   if (L.total > kScratchBytes) return SOL_ERR_WORKSPACE_TOO_SMALL;  // the fixed scratch cannot hold this problem
@@ -119,6 +121,8 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
   a.kept_cnt = kept_cnt ? kept_cnt : reinterpret_cast<int32_t*>(base + L.kept_cnt);
   a.part = reinterpret_cast<float*>(base + L.part);
   a.splits = L.splits;
+  a.work_items = reinterpret_cast<int32_t*>(base + L.work_items);
+  a.work_ctr = reinterpret_cast<int32_t*>(base + L.work_ctr);
   a.out_f32 = nullptr;
   a.out_bf16 = out_bf16;
   a.out_hi = nullptr;
