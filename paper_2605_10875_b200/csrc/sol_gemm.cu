@@ -1,40 +1,67 @@
-// Weight-streaming skinny GEMMs.  The batch (16..128 rows) is the small side;
-// each weight byte is read from HBM exactly once, so these kernels are bound
-// by HBM bandwidth and are built around keeping many bulk copies in flight:
-// a producer warp streams weight tiles into a shared-memory ring with
-// cp.async.bulk (the 1-D TMA path, completion on mbarriers), eight consumer
-// warps feed them to bf16 tensor-core MMAs with fp32 accumulation.
+// Weight-streaming skinny GEMMs on the Blackwell tensor cores.
 //
-//   gemm_nk   : Y[M][N] = A[M][K] . W[N][K]^T   (QKV, output and gate/up projections)
-//   gemm_down : Y[M][d] = T[M][ff] . W[ff][d]   (down projection; rows of W whose
-//               32-channel granule no token keeps are neither copied nor multiplied)
-#include "sol_common.cuh"
+// The batch (16..128 rows after padding) is the small side, so every weight
+// byte is read from HBM exactly once and the kernels are bound by HBM
+// bandwidth.  They are built so that one thread keeps large TMA copies in
+// flight and nobody touches the data with ordinary instructions:
+//
+//   * weights and activations arrive by TMA tiled loads through tensor maps
+//     (128-byte swizzle, several 64-wide k chunks per copy) into a ring of
+//     shared-memory stages guarded by mbarriers (bounded waits);
+//   * one thread issues tcgen05.mma (bf16 x bf16 -> float32) with the WEIGHT
+//     tile as the 128-row M side and the batch as the N side, accumulating in
+//     tensor memory; tcgen05.commit releases each stage when its MMAs finish;
+//   * four warps read the accumulators back with tcgen05.ld and apply the
+//     epilogue (quantizer scale / residual / SwiGLU), writing out[m][n] with
+//     the weight row n along the lanes (coalesced).
+//
+//   umma_nk   : Y[M][N] = A[M][K] . W[N][K]^T   (QKV, output and gate/up projections).  Each CTA owns
+//               a contiguous range of `rows` weight rows (a multiple of 8 chosen so that one wave of
+//               CTAs covers all SMs) over the whole of K.  The MMA always spans 128 rows; rows beyond
+//               the CTA's range read whatever follows in shared memory and land in accumulator lanes
+//               that are never stored (an output row depends only on its own weight row).
+//   umma_down : Y[M][d] = T[M][ff] . W[ff][d]   (down projection).  W rows are intermediate channels,
+//               so the weight tile is the MN-major operand.  CTA = (128 output columns, range of 64-
+//               channel blocks); blocks in which no token keeps a channel are neither copied nor
+//               multiplied; partial sums per range are reduced by reduce_out.
+#include <cstring>
+#include <mutex>
+#include <unordered_map>
+
+#include <cudaTypedefs.h>
+
 #include "sol_internal.h"
+#include "sol_umma.cuh"
 
 namespace sol {
 
-// ============================================================================
-// gemm_nk
-// ============================================================================
-constexpr int NK_CONSUMERS = 8;                 // consumer warps
-constexpr int NK_THREADS = (NK_CONSUMERS + 1) * 32;
-constexpr int NK_KC = 256;                      // k columns per stage
-constexpr int NK_ROWS = 32;                     // weight rows per stage (4 n-tiles)
-constexpr int NK_ROW_BYTES = NK_KC * 2;         // 512
-constexpr int NK_ROW_STRIDE = NK_ROW_BYTES + 64;  // +64: conflict-free 128-bit fragment loads
-constexpr int NK_STAGE_BYTES = NK_ROWS * NK_ROW_STRIDE;  // 18432
-constexpr int NK_STAGES = 8;
-constexpr int NK_RED_BYTES = NK_CONSUMERS * 4 * 128 * 4;  // 16 KB cross-warp reduction buffer
-constexpr int NK_SMEM = NK_STAGES * NK_STAGE_BYTES + NK_RED_BYTES + 2 * NK_STAGES * 8 + 64;
+constexpr int UM_THREADS = 192;      // warps 0-3: epilogue, warp 4: TMA producer, warp 5: MMA issuer + TMEM owner
+constexpr int UM_MAX_STAGES = 8;
+constexpr int UM_TILE_SPAN = 16384;  // bytes one 128-row operand read spans from the start of a chunk tile
+constexpr int UM_SMEM_BUDGET = 196 * 1024;
 
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(NK_CONSUMERS * 32)); }
+struct UmBarriers {
+  uint64_t full[UM_MAX_STAGES];
+  uint64_t empty[UM_MAX_STAGES];
+  uint64_t accum;
+  uint32_t tmem_base;
+  int n_issued;
+};
 
+__device__ __forceinline__ unsigned char* align_1024(unsigned char* p) {
+  const uint32_t a = smem_u32(p);
+  return p + (((a + 1023u) & ~1023u) - a);
+}
+
+// ============================================================================
+// umma_nk
+// ============================================================================
 struct NKDev {
-  const uint16_t* a_hi;
-  const uint16_t* a_lo;
-  const uint16_t* w0;
-  const uint16_t* w1;
-  int M, K, N, MT;
+  int M, Mpad, K, N;  // N: weight rows (EPI_SWIGLU: channels, with a gate and an up row each)
+  int rows;           // weight rows per CTA
+  int cps, stages;    // 64-wide k chunks per stage, ring depth
+  int n_b;            // activation operands: 1, or 2 for a high + low bf16 pair
+  uint32_t tmem_cols;
   const float* row_scale;
   const void* resid;
   int resid_f32;
@@ -42,388 +69,438 @@ struct NKDev {
   float* out1;
   float* out2;
   int* status;
-  int n_tiles;  // virtual n-tiles of 8 rows (EPI_SWIGLU: 2 per 8 channels, gate then up)
 };
 
-template <int EPI, int MT>
-__global__ void __launch_bounds__(NK_THREADS, 1) gemm_nk_kernel(const NKDev p) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  unsigned char* stages = smem;
-  float* red = reinterpret_cast<float*>(smem + NK_STAGES * NK_STAGE_BYTES);
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + NK_STAGES * NK_STAGE_BYTES + NK_RED_BYTES);
-  uint64_t* empty = full + NK_STAGES;
+template <int EPI>
+__global__ void __launch_bounds__(UM_THREADS, 1)
+umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant__ CUtensorMap tm_w1,
+               const __grid_constant__ CUtensorMap tm_x0, const __grid_constant__ CUtensorMap tm_x1, const NKDev p) {
+  extern __shared__ unsigned char smem_raw[];
+  constexpr int NW = EPI == EPI_SWIGLU ? 2 : 1;
+  unsigned char* stages = align_1024(smem_raw);
+  const int w_tile = p.rows * 128, x_tile = p.Mpad * 128;  // bytes per 64-wide k chunk
+  const int stage_bytes = p.cps * (NW * w_tile + p.n_b * x_tile);
+  UmBarriers* bars = reinterpret_cast<UmBarriers*>(stages + (size_t)p.stages * stage_bytes + UM_TILE_SPAN);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < NK_STAGES; ++s) {
-      mbar_init(&full[s], 1);
-      mbar_init(&empty[s], NK_CONSUMERS);
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&bars->full[s], 1);
+      mbar_init(&bars->empty[s], 1);
     }
+    mbar_init(&bars->accum, 1);
     fence_mbar_init();
   }
+  if (warp == 5) tmem_alloc(&bars->tmem_base, p.tmem_cols);
+  tc_fence_before();
   __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
 
-  // this CTA's range of n-tiles, in units of 2 so gate/up pairs stay together
-  const int pairs = p.n_tiles / 2;
-  const int pr0 = (int)(((long long)pairs * blockIdx.x) / gridDim.x);
-  const int pr1 = (int)(((long long)pairs * (blockIdx.x + 1)) / gridDim.x);
-  const int vt0 = 2 * pr0, vt1 = 2 * pr1;
-  const int kchunks = p.K / NK_KC;
+  const int row0 = blockIdx.x * p.rows;
+  const int n_iter = p.K / 64 / p.cps;
 
-  // row r of virtual n-tile vt -> weight row pointer
-  auto w_row = [&](int vt, int r) -> const uint16_t* {
-    if (EPI == EPI_SWIGLU) {
-      const uint16_t* base = (vt & 1) ? p.w1 : p.w0;
-      return base + (size_t)((vt >> 1) * 8 + r) * p.K;
-    }
-    return p.w0 + (size_t)(vt * 8 + r) * p.K;
-  };
-
-  if (warp == NK_CONSUMERS) {
-    // ------------------------------ producer -------------------------------
-    bool ok = true;
-    uint32_t it = 0;
-    for (int vb = vt0; vb < vt1; vb += 4) {
-      const int nt = min(4, vt1 - vb);
-      for (int kc = 0; kc < kchunks; ++kc, ++it) {
-        const int s = it % NK_STAGES;
-        const uint32_t ph = (it / NK_STAGES) & 1;
-        if (ok) ok = mbar_wait(&empty[s], ph ^ 1, p.status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) continue;
-        if (lane == 0) mbar_expect_tx(&full[s], nt * 8 * NK_ROW_BYTES);
-        __syncwarp();
-        if (lane < nt * 8) {
-          const uint16_t* src = w_row(vb + (lane >> 3), lane & 7) + (size_t)kc * NK_KC;
-          bulk_g2s(stages + (size_t)s * NK_STAGE_BYTES + lane * NK_ROW_STRIDE, src, NK_ROW_BYTES, &full[s]);
-        }
+  if (warp == 4) {
+    // ------------------------------ TMA producer -----------------------------
+    if (lane == 0) {
+      tma_prefetch_map(&tm_w0);
+      tma_prefetch_map(&tm_x0);
+      for (int it = 0; it < n_iter; ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!mbar_wait(&bars->empty[s], ph ^ 1, p.status)) break;
+        unsigned char* st = stages + (size_t)s * stage_bytes;
+        mbar_expect_tx(&bars->full[s], stage_bytes);
+        tma_load_3d(st, &tm_w0, 0, row0, it * p.cps, &bars->full[s]);
+        if (NW == 2) tma_load_3d(st + p.cps * w_tile, &tm_w1, 0, row0, it * p.cps, &bars->full[s]);
+        unsigned char* xs = st + NW * p.cps * w_tile;
+        tma_load_3d(xs, &tm_x0, 0, 0, it * p.cps, &bars->full[s]);
+        if (p.n_b == 2) tma_load_3d(xs + p.cps * x_tile, &tm_x1, 0, 0, it * p.cps, &bars->full[s]);
       }
     }
-    return;
-  }
-
-  // -------------------------------- consumers --------------------------------
-  const int g = lane >> 2, t = lane & 3;
-  bool ok = true;
-  uint32_t it = 0;
-  for (int vb = vt0; vb < vt1; vb += 4) {
-    const int nt = min(4, vt1 - vb);
-    float acc[MT][4][4];
+  } else if (warp == 5) {
+    // ------------------------------- MMA issuer ------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16_m128(p.Mpad, 0, 0);
+      bool acc = false, ok = true;
+      for (int it = 0; it < n_iter; ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        ok = mbar_wait(&bars->full[s], ph, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
+        const uint32_t xs = st + NW * p.cps * w_tile;
+        for (int c = 0; c < p.cps; ++c) {
 #pragma unroll
-    for (int m = 0; m < MT; ++m)
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-#pragma unroll
-        for (int r = 0; r < 4; ++r) acc[m][j][r] = 0.f;
-
-    for (int kc = 0; kc < kchunks; ++kc, ++it) {
-      const int s = it % NK_STAGES;
-      const uint32_t ph = (it / NK_STAGES) & 1;
-      const size_t kofs = (size_t)kc * NK_KC + warp * 32 + t * 8;
-      // activation fragments come from global memory (L1/L2 resident); with a single m-tile they are
-      // fetched before the wait so their latency overlaps it
-      auto load_a = [&](int m, uint4 (&ah)[2], uint4 (&al)[2]) {
-        ah[0] = *reinterpret_cast<const uint4*>(p.a_hi + (size_t)(m * 16 + g) * p.K + kofs);
-        ah[1] = *reinterpret_cast<const uint4*>(p.a_hi + (size_t)(m * 16 + g + 8) * p.K + kofs);
-        if (p.a_lo != nullptr) {
-          al[0] = *reinterpret_cast<const uint4*>(p.a_lo + (size_t)(m * 16 + g) * p.K + kofs);
-          al[1] = *reinterpret_cast<const uint4*>(p.a_lo + (size_t)(m * 16 + g + 8) * p.K + kofs);
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t b0 = umma_smem_desc(xs + c * x_tile + ks * 32, 16, 1024);
+            const uint64_t b1 = umma_smem_desc(xs + (p.cps + c) * x_tile + ks * 32, 16, 1024);
+            const uint64_t a0 = umma_smem_desc(st + c * w_tile + ks * 32, 16, 1024);
+            umma_bf16(tmem, a0, b0, idesc, acc);
+            if (p.n_b == 2) umma_bf16(tmem, a0, b1, idesc, true);
+            if (NW == 2) {
+              const uint64_t a1 = umma_smem_desc(st + (p.cps + c) * w_tile + ks * 32, 16, 1024);
+              umma_bf16(tmem + p.Mpad, a1, b0, idesc, acc);
+              if (p.n_b == 2) umma_bf16(tmem + p.Mpad, a1, b1, idesc, true);
+            }
+            acc = true;
+          }
         }
-      };
-      uint4 ah[2], al[2];
-      if (MT == 1) load_a(0, ah, al);
-      if (ok) ok = mbar_wait(&full[s], ph, p.status);
-      if (ok) {
-        const uint32_t base = smem_u32(stages + (size_t)s * NK_STAGE_BYTES) + g * NK_ROW_STRIDE + (warp * 32 + t * 8) * 2;
-        uint4 w[4];
+        umma_commit(&bars->empty[s]);  // the stage is free again once these MMAs have read it
+      }
+      if (ok) umma_commit(&bars->accum);
+    }
+  } else {
+    // -------------------------------- epilogue -------------------------------
+    if (warp * 32 < p.rows) {
+      const bool ok = mbar_wait(&bars->accum, 0, p.status);
+      tc_fence_after();
+      const int r = warp * 32 + lane, n = row0 + r;
+      const bool valid = r < p.rows && n < p.N;
+      const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
+      for (int c0 = 0; c0 < p.Mpad && ok; c0 += 16) {
+        float v[16], u[16];
+        tmem_ld16(tl + c0, v);
+        if (NW == 2) tmem_ld16(tl + p.Mpad + c0, u);
+        if (valid) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-          if (j < nt) w[j] = lds128(base + j * 8 * NK_ROW_STRIDE);
-#pragma unroll
-        for (int m = 0; m < MT; ++m) {
-          if (MT > 1) load_a(m, ah, al);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            if (j < nt) {
-              mma_bf16(acc[m][j], ah[0].x, ah[1].x, ah[0].y, ah[1].y, w[j].x, w[j].y);
-              mma_bf16(acc[m][j], ah[0].z, ah[1].z, ah[0].w, ah[1].w, w[j].z, w[j].w);
-              if (p.a_lo != nullptr) {
-                mma_bf16(acc[m][j], al[0].x, al[1].x, al[0].y, al[1].y, w[j].x, w[j].y);
-                mma_bf16(acc[m][j], al[0].z, al[1].z, al[0].w, al[1].w, w[j].z, w[j].w);
+          for (int i = 0; i < 16; ++i) {
+            const int m = c0 + i;
+            if (m < p.M) {
+              const float sc = p.row_scale ? p.row_scale[m] : 1.0f;
+              const size_t o = (size_t)m * p.N + n;
+              if (EPI == EPI_SWIGLU) {
+                const float gg = v[i] * sc, uu = u[i] * sc;
+                p.out0[o] = gg;
+                p.out1[o] = uu;
+                p.out2[o] = (gg / (1.0f + expf(-gg))) * uu;
+              } else if (EPI == EPI_RESIDUAL) {
+                const float res = p.resid_f32 ? static_cast<const float*>(p.resid)[o]
+                                              : bf2f(static_cast<const uint16_t*>(p.resid)[o]);
+                p.out0[o] = v[i] * sc + res;
+              } else {
+                p.out0[o] = v[i] * sc;
               }
             }
           }
         }
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty[s]);
-    }
-
-    // cross-warp reduction (each warp holds a K sub-slice) and epilogue, one m-tile at a time
-#pragma unroll
-    for (int m = 0; m < MT; ++m) {
-      consumer_bar();  // previous round's readers are done with `red`
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-        *reinterpret_cast<float4*>(red + ((warp * 4 + j) * 128 + lane * 4)) =
-            make_float4(acc[m][j][0], acc[m][j][1], acc[m][j][2], acc[m][j][3]);
-      consumer_bar();
-      // thread -> (tile pair pr, lane l, register r); tiles 2pr and 2pr+1
-      const int pr = threadIdx.x >> 7, idx = threadIdx.x & 127;
-      const int l = idx >> 2, r = idx & 3;
-      float v0 = 0.f, v1 = 0.f;
-#pragma unroll
-      for (int w = 0; w < NK_CONSUMERS; ++w) {
-        v0 += red[(w * 4 + 2 * pr) * 128 + idx];
-        v1 += red[(w * 4 + 2 * pr + 1) * 128 + idx];
-      }
-      const int row = m * 16 + (l >> 2) + ((r & 2) ? 8 : 0);
-      const int col = (l & 3) * 2 + (r & 1);
-      if (row < p.M) {
-        const float sc = p.row_scale ? p.row_scale[row] : 1.0f;
-        v0 *= sc;
-        v1 *= sc;
-        if (EPI == EPI_SWIGLU) {
-          if (2 * pr < nt) {
-            const int ch = ((vb >> 1) + pr) * 8 + col;
-            const size_t o = (size_t)row * p.N + ch;
-            const float gg = v0, uu = v1;
-            p.out0[o] = gg;
-            p.out1[o] = uu;
-            p.out2[o] = (gg / (1.0f + expf(-gg))) * uu;
-          }
-        } else {
-#pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            const int j = 2 * pr + q;
-            if (j < nt) {
-              const int n = (vb + j) * 8 + col;
-              const size_t o = (size_t)row * p.N + n;
-              float v = q ? v1 : v0;
-              if (EPI == EPI_RESIDUAL) {
-                v += p.resid_f32 ? static_cast<const float*>(p.resid)[o]
-                                 : bf2f(static_cast<const uint16_t*>(p.resid)[o]);
-              }
-              p.out0[o] = v;
-            }
-          }
-        }
-      }
     }
   }
-}
-
-template <int EPI>
-static void launch_nk_mt(const NKDev& d, int grid, cudaStream_t st) {
-  const char* name = EPI == EPI_SWIGLU ? "gemm_gate_up_swiglu" : (EPI == EPI_RESIDUAL ? "gemm_out_proj" : "gemm_qkv");
-#define SOL_NK_CASE(MTV)                                                                                      \
-  case MTV: {                                                                                                 \
-    ensure_dynamic_smem(reinterpret_cast<const void*>(&gemm_nk_kernel<EPI, MTV>), NK_SMEM);                   \
-    SOL_LAUNCH(name, (gemm_nk_kernel<EPI, MTV>), dim3(grid), dim3(NK_THREADS), NK_SMEM, st, d);               \
-  } break;
-  switch (d.MT) {
-    SOL_NK_CASE(1)
-    SOL_NK_CASE(2)
-    SOL_NK_CASE(4)
-    SOL_NK_CASE(8)
-    default: break;
-  }
-#undef SOL_NK_CASE
-}
-
-static int round_mt(int M) {
-  int mt = (M + 15) / 16;
-  return mt <= 1 ? 1 : (mt <= 2 ? 2 : (mt <= 4 ? 4 : 8));
-}
-
-void launch_gemm_nk(const GemmNK& p, GemmEpilogue epi, cudaStream_t st) {
-  NKDev d;
-  d.a_hi = static_cast<const uint16_t*>(p.a_hi);
-  d.a_lo = static_cast<const uint16_t*>(p.a_lo);
-  d.w0 = static_cast<const uint16_t*>(p.w0);
-  d.w1 = static_cast<const uint16_t*>(p.w1);
-  d.M = p.M; d.K = p.K; d.N = p.N; d.MT = round_mt(p.M);
-  d.row_scale = p.row_scale; d.resid = p.resid; d.resid_f32 = p.resid_f32;
-  d.out0 = p.out0; d.out1 = p.out1; d.out2 = p.out2; d.status = p.status;
-  d.n_tiles = (epi == EPI_SWIGLU) ? 2 * (p.N / 8) : p.N / 8;
-  const int grid = min(sm_count(), max(1, d.n_tiles / 2));
-  if (epi == EPI_SWIGLU) launch_nk_mt<EPI_SWIGLU>(d, grid, st);
-  else if (epi == EPI_RESIDUAL) launch_nk_mt<EPI_RESIDUAL>(d, grid, st);
-  else launch_nk_mt<EPI_SCALE>(d, grid, st);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem, p.tmem_cols);
 }
 
 // ============================================================================
-// gemm_down
+// umma_down
 // ============================================================================
-constexpr int DN_CONSUMERS = 8;
-constexpr int DN_THREADS = (DN_CONSUMERS + 1) * 32;
-constexpr int DN_KG = 32;                        // channels per stage (one granule)
-constexpr int DN_NS = 256;                       // output columns per CTA
-constexpr int DN_W_STRIDE = DN_NS * 2 + 16;      // 528: conflict-free ldmatrix rows
-constexpr int DN_W_BYTES = DN_KG * DN_W_STRIDE;  // 16896
-constexpr int DN_A_STRIDE = DN_KG * 2 + 16;      // 80
-constexpr int DN_SMEM_BUDGET = 200 * 1024;
-
 struct DownDev {
-  const uint16_t* t_hi;
-  const uint16_t* t_lo;
-  const uint16_t* w;
-  const int32_t* live;
   int M, Mpad, ff, d;
-  float* partial;
-  int chunks, stages, stage_bytes;
+  int chunks, stages;
+  uint32_t tmem_cols;
+  const int32_t* live;  // [ff/32]
+  float* partial;       // [chunks][Mpad][d]
   int* status;
 };
 
-template <int MT>
-__global__ void __launch_bounds__(DN_THREADS, 1) gemm_down_kernel(const DownDev p) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  const int NST = p.stages;
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)NST * p.stage_bytes);
-  uint64_t* empty = full + NST;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < NST; ++s) {
-      mbar_init(&full[s], 1);
-      mbar_init(&empty[s], DN_CONSUMERS);
-    }
-    fence_mbar_init();
-  }
-  __syncthreads();
-
-  const int slab = blockIdx.x;   // 256 output columns
-  const int chunk = blockIdx.y;  // range of granules
-  const int granules = p.ff / DN_KG;
-  const int g0 = (int)(((long long)granules * chunk) / p.chunks);
-  const int g1 = (int)(((long long)granules * (chunk + 1)) / p.chunks);
-  const int a_bytes = MT * 16 * DN_A_STRIDE;
-
-  if (warp == DN_CONSUMERS) {
-    bool ok = true;
-    uint32_t it = 0;
-    for (int gi = g0; gi < g1; ++gi) {
-      if (p.live[gi] == 0) continue;
-      const int s = it % NST;
-      const uint32_t ph = (it / NST) & 1;
-      ++it;
-      if (ok) ok = mbar_wait(&empty[s], ph ^ 1, p.status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) continue;
-      unsigned char* st = smem + (size_t)s * p.stage_bytes;
-      if (lane == 0) mbar_expect_tx(&full[s], DN_KG * DN_NS * 2 + 2 * MT * 16 * DN_KG * 2);
-      __syncwarp();
-      // weight rows: one 512-byte copy per channel
-      bulk_g2s(st + lane * DN_W_STRIDE, p.w + (size_t)(gi * DN_KG + lane) * p.d + slab * DN_NS, DN_NS * 2, &full[s]);
-      // activation tiles: 64 bytes per batch row, high and low parts
-      for (int r = lane; r < MT * 16; r += 32) {
-        const size_t src = (size_t)r * p.ff + (size_t)gi * DN_KG;
-        bulk_g2s(st + DN_W_BYTES + r * DN_A_STRIDE, p.t_hi + src, DN_KG * 2, &full[s]);
-        bulk_g2s(st + DN_W_BYTES + a_bytes + r * DN_A_STRIDE, p.t_lo + src, DN_KG * 2, &full[s]);
-      }
-    }
-    return;
-  }
-
-  float acc[MT][4][4];
-#pragma unroll
-  for (int m = 0; m < MT; ++m)
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-#pragma unroll
-      for (int r = 0; r < 4; ++r) acc[m][j][r] = 0.f;
-
-  bool ok = true;
-  uint32_t it = 0;
-  const int mi = lane >> 3, mr = lane & 7;  // ldmatrix: this lane addresses row mr of matrix mi
-  for (int gi = g0; gi < g1; ++gi) {
-    if (p.live[gi] == 0) continue;
-    const int s = it % NST;
-    const uint32_t ph = (it / NST) & 1;
-    ++it;
-    if (ok) ok = mbar_wait(&full[s], ph, p.status);
-    if (ok) {
-      const uint32_t st = smem_u32(smem + (size_t)s * p.stage_bytes);
-#pragma unroll
-      for (int ks = 0; ks < 2; ++ks) {
-        uint32_t bfr[2][4];  // [pair of n-tiles][b0,b1 of tile a, b0,b1 of tile a+1]
-#pragma unroll
-        for (int pr = 0; pr < 2; ++pr) {
-          const int krow = ks * 16 + (mi & 1) * 8 + mr;
-          const int ncol = warp * 32 + (2 * pr + (mi >> 1)) * 8;
-          ldsm_x4_trans(bfr[pr], st + krow * DN_W_STRIDE + ncol * 2);
-        }
-#pragma unroll
-        for (int m = 0; m < MT; ++m) {
-          uint32_t ah[4], al[4];
-          const int mrow = m * 16 + (mi & 1) * 8 + mr;
-          const int kcol = ks * 16 + (mi >> 1) * 8;
-          ldsm_x4(ah, st + DN_W_BYTES + mrow * DN_A_STRIDE + kcol * 2);
-          ldsm_x4(al, st + DN_W_BYTES + a_bytes + mrow * DN_A_STRIDE + kcol * 2);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t b0 = bfr[j >> 1][(j & 1) * 2], b1 = bfr[j >> 1][(j & 1) * 2 + 1];
-            mma_bf16(acc[m][j], ah[0], ah[1], ah[2], ah[3], b0, b1);
-            mma_bf16(acc[m][j], al[0], al[1], al[2], al[3], b0, b1);
-          }
-        }
-      }
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&empty[s]);
-  }
-
-  // partial sums of this chunk
-  const int g = lane >> 2, t = lane & 3;
-  float* out = p.partial + (size_t)chunk * p.Mpad * p.d;
-#pragma unroll
-  for (int m = 0; m < MT; ++m)
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int col = slab * DN_NS + warp * 32 + j * 8 + t * 2;
-      const int r0 = m * 16 + g, r1 = r0 + 8;
-      if (r0 < p.M) *reinterpret_cast<float2*>(out + (size_t)r0 * p.d + col) = make_float2(acc[m][j][0], acc[m][j][1]);
-      if (r1 < p.M) *reinterpret_cast<float2*>(out + (size_t)r1 * p.d + col) = make_float2(acc[m][j][2], acc[m][j][3]);
-    }
+__device__ __forceinline__ bool block_live(const int32_t* live, int jb, int granules) {
+  return live[2 * jb] != 0 || (2 * jb + 1 < granules && live[2 * jb + 1] != 0);
 }
 
-int down_chunks(int ff, int d) {
-  const int slabs = d / DN_NS;
-  const int granules = ff / DN_KG;
-  int c = sm_count() / (slabs > 0 ? slabs : 1);
-  if (c < 1) c = 1;
-  if (c > granules) c = granules;
+__global__ void __launch_bounds__(UM_THREADS, 1)
+umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_hi,
+                 const __grid_constant__ CUtensorMap tm_lo, const DownDev p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* stages = align_1024(smem_raw);
+  const int t_tile = p.Mpad * 128;
+  const int stage_bytes = UM_TILE_SPAN + 2 * t_tile;
+  UmBarriers* bars = reinterpret_cast<UmBarriers*>(stages + (size_t)p.stages * stage_bytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&bars->full[s], 1);
+      mbar_init(&bars->empty[s], 1);
+    }
+    mbar_init(&bars->accum, 1);
+    bars->n_issued = 0;
+    fence_mbar_init();
+  }
+  if (warp == 5) tmem_alloc(&bars->tmem_base, p.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
+
+  const int slab = blockIdx.x, chunk = blockIdx.y;
+  const int granules = p.ff / 32, jblocks = (p.ff + 63) / 64;
+  const int jb0 = (int)(((long long)jblocks * chunk) / p.chunks);
+  const int jb1 = (int)(((long long)jblocks * (chunk + 1)) / p.chunks);
+
+  if (warp == 4) {
+    if (lane == 0) {
+      tma_prefetch_map(&tm_w);
+      int it = 0;
+      for (int jb = jb0; jb < jb1; ++jb) {
+        if (!block_live(p.live, jb, granules)) continue;
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        ++it;
+        if (!mbar_wait(&bars->empty[s], ph ^ 1, p.status)) break;
+        unsigned char* st = stages + (size_t)s * stage_bytes;
+        mbar_expect_tx(&bars->full[s], stage_bytes);
+        tma_load_3d(st, &tm_w, 0, jb * 64, slab * 2, &bars->full[s]);
+        tma_load_2d(st + UM_TILE_SPAN, &tm_hi, jb * 64, 0, &bars->full[s]);
+        tma_load_2d(st + UM_TILE_SPAN + t_tile, &tm_lo, jb * 64, 0, &bars->full[s]);
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16_m128(p.Mpad, 1, 0);
+      bool acc = false, ok = true;
+      int it = 0;
+      for (int jb = jb0; jb < jb1; ++jb) {
+        if (!block_live(p.live, jb, granules)) continue;
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        ++it;
+        ok = mbar_wait(&bars->full[s], ph, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+          // weight tile: two 64-column blocks of [64 channels][128 bytes]; 16 channels = two 8-row groups
+          const uint64_t a = umma_smem_desc(st + ks * 2048, 8192, 1024);
+          const uint64_t bh = umma_smem_desc(st + UM_TILE_SPAN + ks * 32, 16, 1024);
+          const uint64_t bl = umma_smem_desc(st + UM_TILE_SPAN + t_tile + ks * 32, 16, 1024);
+          umma_bf16(tmem, a, bh, idesc, acc);
+          umma_bf16(tmem, a, bl, idesc, true);
+          acc = true;
+        }
+        umma_commit(&bars->empty[s]);
+      }
+      *reinterpret_cast<volatile int*>(&bars->n_issued) = acc ? 1 : 0;
+      __threadfence_block();
+      if (ok) umma_commit(&bars->accum);
+    }
+  } else {
+    const bool ok = mbar_wait(&bars->accum, 0, p.status);
+    tc_fence_after();
+    const bool any = *reinterpret_cast<volatile int*>(&bars->n_issued) > 0;
+    const int n = slab * 128 + warp * 32 + lane;
+    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
+    float* out = p.partial + (size_t)chunk * p.Mpad * p.d;
+    for (int c0 = 0; c0 < p.Mpad && ok; c0 += 16) {
+      float v[16];
+      if (any) {
+        tmem_ld16(tl + c0, v);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int m = c0 + i;
+        if (m < p.M) out[(size_t)m * p.d + n] = v[i];
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem, p.tmem_cols);
+}
+
+// ============================================================================
+// tensor maps (host)
+// ============================================================================
+namespace {
+
+struct MapKey {
+  uintptr_t ptr;
+  uint64_t dim[3];
+  uint64_t stride[2];
+  uint32_t box[3];
+  uint32_t rank;
+  bool operator==(const MapKey& o) const {
+    return ptr == o.ptr && rank == o.rank && dim[0] == o.dim[0] && dim[1] == o.dim[1] && dim[2] == o.dim[2] &&
+           stride[0] == o.stride[0] && stride[1] == o.stride[1] && box[0] == o.box[0] && box[1] == o.box[1] &&
+           box[2] == o.box[2];
+  }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    uint64_t h = k.ptr * 0x9e3779b97f4a7c15ull;
+    auto mix = [&](uint64_t v) { h = (h ^ v) * 0x100000001b3ull + (h >> 29); };
+    mix(k.dim[0]); mix(k.dim[1]); mix(k.dim[2]); mix(k.stride[0]); mix(k.stride[1]);
+    mix(k.box[0]); mix(k.box[1]); mix(k.box[2]); mix(k.rank);
+    return (size_t)h;
+  }
+};
+
+PFN_cuTensorMapEncodeTiled encode_fn() {
+  static PFN_cuTensorMapEncodeTiled fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<PFN_cuTensorMapEncodeTiled>(p);
+  }();
+  return fn;
+}
+
+// bf16 tensor map with 128-byte swizzle; encoded maps are remembered (the encoding is a pure function
+// of the key, and the same weight matrices come back every step).
+bool tensor_map(CUtensorMap* out, const void* ptr, uint32_t rank, const uint64_t* dim, const uint64_t* stride,
+                const uint32_t* box) {
+  static std::mutex mu;
+  static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+  MapKey k;
+  memset(&k, 0, sizeof(k));
+  k.ptr = reinterpret_cast<uintptr_t>(ptr);
+  k.rank = rank;
+  for (uint32_t i = 0; i < rank; ++i) {
+    k.dim[i] = dim[i];
+    k.box[i] = box[i];
+    if (i + 1 < rank) k.stride[i] = stride[i];
+  }
+  std::lock_guard<std::mutex> lock(mu);
+  auto it = cache.find(k);
+  if (it != cache.end()) {
+    *out = it->second;
+    return true;
+  }
+  PFN_cuTensorMapEncodeTiled fn = encode_fn();
+  if (!fn) {
+    record_cuda_error(cudaErrorNotSupported, "cuTensorMapEncodeTiled entry point");
+    return false;
+  }
+  const cuuint32_t ones[3] = {1, 1, 1};
+  CUtensorMap m;
+  const CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(ptr), dim, stride, box, ones,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return false;
+  }
+  if (cache.size() > (1u << 16)) cache.clear();
+  cache.emplace(k, m);
+  *out = m;
+  return true;
+}
+
+// [rows][K] row-major bf16 viewed as (64 k, rows, K/64 chunks): a box of (64, box_rows, cps) lands in
+// shared memory as cps consecutive [box_rows][64] tiles, each in the 128-byte-swizzled K-major layout.
+bool kmajor_map(CUtensorMap* out, const void* ptr, int rows, int K, int box_rows, int cps) {
+  const uint64_t dim[3] = {64, (uint64_t)rows, (uint64_t)(K / 64)};
+  const uint64_t stride[2] = {(uint64_t)K * 2, 128};
+  const uint32_t box[3] = {64, (uint32_t)box_rows, (uint32_t)cps};
+  return tensor_map(out, ptr, 3, dim, stride, box);
+}
+
+uint32_t pow2_cols(int n) {
+  uint32_t c = 32;
+  while ((int)c < n) c <<= 1;
   return c;
 }
 
-void launch_gemm_down(const GemmDown& p, cudaStream_t st) {
-  DownDev d;
-  d.t_hi = static_cast<const uint16_t*>(p.t_hi);
-  d.t_lo = static_cast<const uint16_t*>(p.t_lo);
-  d.w = static_cast<const uint16_t*>(p.w);
-  d.live = p.live;
-  d.M = p.M; d.ff = p.ff; d.d = p.d;
-  const int mt = round_mt(p.M);
-  d.Mpad = mt * 16;
-  d.partial = p.partial; d.chunks = p.chunks; d.status = p.status;
-  d.stage_bytes = DN_W_BYTES + 2 * mt * 16 * DN_A_STRIDE;
-  d.stage_bytes = (d.stage_bytes + 127) / 128 * 128;
-  d.stages = DN_SMEM_BUDGET / d.stage_bytes;
-  if (d.stages > 8) d.stages = 8;
-  const int smem = d.stages * d.stage_bytes + 2 * d.stages * 8 + 64;
-  dim3 grid(p.d / DN_NS, p.chunks);
-#define SOL_DN_CASE(MTV)                                                                                  \
-  case MTV: {                                                                                             \
-    ensure_dynamic_smem(reinterpret_cast<const void*>(&gemm_down_kernel<MTV>), smem);                     \
-    SOL_LAUNCH("gemm_down_gathered", gemm_down_kernel<MTV>, grid, dim3(DN_THREADS), smem, st, d);         \
-  } break;
-  switch (mt) {
-    SOL_DN_CASE(1)
-    SOL_DN_CASE(2)
-    SOL_DN_CASE(4)
-    SOL_DN_CASE(8)
-    default: break;
+int round_mpad(int M) {
+  const int mt = (M + 15) / 16;
+  return 16 * (mt <= 1 ? 1 : (mt <= 2 ? 2 : (mt <= 4 ? 4 : 8)));
+}
+
+}  // namespace
+
+// ============================================================================
+// launchers
+// ============================================================================
+void launch_gemm_nk(const GemmNK& g, GemmEpilogue epi, cudaStream_t st) {
+  const int nw = epi == EPI_SWIGLU ? 2 : 1;
+  NKDev d;
+  memset(&d, 0, sizeof(d));
+  d.M = g.M; d.Mpad = round_mpad(g.M); d.K = g.K; d.N = g.N;
+  d.n_b = g.a_lo ? 2 : 1;
+  const int sms = sm_count();
+  int rows = ((g.N + sms - 1) / sms + 7) / 8 * 8;
+  if (rows > 128) rows = 128;
+  d.rows = rows;
+  const int chunk_bytes = 128 * (nw * rows + d.n_b * d.Mpad);
+  const int chunks = g.K / 64;
+  int cps = 4;
+  while (cps > 1 && (cps * chunk_bytes > 36 * 1024 || chunks % cps)) cps >>= 1;
+  d.cps = cps;
+  const int stage_bytes = cps * chunk_bytes;
+  int stages = UM_SMEM_BUDGET / stage_bytes;
+  if (stages > UM_MAX_STAGES) stages = UM_MAX_STAGES;
+  if (stages > chunks / cps) stages = chunks / cps;
+  if (stages < 1) stages = 1;
+  d.stages = stages;
+  d.tmem_cols = pow2_cols(nw * d.Mpad);
+  d.row_scale = g.row_scale; d.resid = g.resid; d.resid_f32 = g.resid_f32;
+  d.out0 = g.out0; d.out1 = g.out1; d.out2 = g.out2; d.status = g.status;
+
+  CUtensorMap w0, w1, x0, x1;
+  bool ok = kmajor_map(&w0, g.w0, g.N, g.K, rows, cps);
+  ok = ok && kmajor_map(&w1, nw == 2 ? g.w1 : g.w0, g.N, g.K, rows, cps);
+  ok = ok && kmajor_map(&x0, g.a_hi, d.Mpad, g.K, d.Mpad, cps);
+  ok = ok && kmajor_map(&x1, g.a_lo ? g.a_lo : g.a_hi, d.Mpad, g.K, d.Mpad, cps);
+  if (!ok) return;
+  const int smem = 1024 + stages * stage_bytes + UM_TILE_SPAN + (int)sizeof(UmBarriers);
+  const dim3 grid((g.N + rows - 1) / rows);
+  if (epi == EPI_SWIGLU) {
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_nk_kernel<EPI_SWIGLU>), smem);
+    SOL_LAUNCH("gemm_gate_up_swiglu", umma_nk_kernel<EPI_SWIGLU>, grid, dim3(UM_THREADS), smem, st, w0, w1, x0, x1, d);
+  } else if (epi == EPI_RESIDUAL) {
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_nk_kernel<EPI_RESIDUAL>), smem);
+    SOL_LAUNCH("gemm_out_proj", umma_nk_kernel<EPI_RESIDUAL>, grid, dim3(UM_THREADS), smem, st, w0, w1, x0, x1, d);
+  } else {
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_nk_kernel<EPI_SCALE>), smem);
+    SOL_LAUNCH("gemm_qkv", umma_nk_kernel<EPI_SCALE>, grid, dim3(UM_THREADS), smem, st, w0, w1, x0, x1, d);
   }
-#undef SOL_DN_CASE
+}
+
+int down_chunks(int ff, int d) {
+  const int slabs = d / 128;
+  const int jblocks = (ff + 63) / 64;
+  int c = sm_count() / (slabs > 0 ? slabs : 1);
+  if (c < 1) c = 1;
+  if (c > jblocks) c = jblocks;
+  return c;
+}
+
+void launch_gemm_down(const GemmDown& g, cudaStream_t st) {
+  DownDev d;
+  memset(&d, 0, sizeof(d));
+  d.M = g.M; d.Mpad = round_mpad(g.M); d.ff = g.ff; d.d = g.d;
+  d.chunks = g.chunks;
+  const int stage_bytes = UM_TILE_SPAN + 2 * d.Mpad * 128;
+  int stages = UM_SMEM_BUDGET / stage_bytes;
+  if (stages > UM_MAX_STAGES) stages = UM_MAX_STAGES;
+  d.stages = stages;
+  d.tmem_cols = pow2_cols(d.Mpad);
+  d.live = g.live; d.partial = g.partial; d.status = g.status;
+
+  CUtensorMap w, hi, lo;
+  // W[ff][d] viewed as (64 columns, ff channels, d/64 column blocks): a box of (64, 64, 2) lands as two
+  // [64 channels][64 columns] blocks, the MN-major operand layout for 128 output columns
+  const uint64_t wdim[3] = {64, (uint64_t)g.ff, (uint64_t)(g.d / 64)};
+  const uint64_t wstride[2] = {(uint64_t)g.d * 2, 128};
+  const uint32_t wbox[3] = {64, 64, 2};
+  bool ok = tensor_map(&w, g.w, 3, wdim, wstride, wbox);
+  // activations [Mpad][ff]: (ff, Mpad) with a box of (64 channels, Mpad rows); channels past ff read as zero
+  const uint64_t tdim[2] = {(uint64_t)g.ff, (uint64_t)d.Mpad};
+  const uint64_t tstride[1] = {(uint64_t)g.ff * 2};
+  const uint32_t tbox[2] = {64, (uint32_t)d.Mpad};
+  ok = ok && tensor_map(&hi, g.t_hi, 2, tdim, tstride, tbox);
+  ok = ok && tensor_map(&lo, g.t_lo, 2, tdim, tstride, tbox);
+  if (!ok) return;
+  const int smem = 1024 + stages * stage_bytes + (int)sizeof(UmBarriers);
+  ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_down_kernel), smem);
+  SOL_LAUNCH("gemm_down_gathered", umma_down_kernel, dim3(g.d / 128, g.chunks), dim3(UM_THREADS), smem, st, w, hi, lo, d);
 }
 
 // ============================================================================

@@ -76,7 +76,6 @@ __global__ void __launch_bounds__(SEL_THREADS) channel_select_kernel(const ChanD
     key_thr = radix_select_kth([&](int j) { return float_key(fabsf(tv[j])); }, ff, m, tie_need, sm);
     mode = 3;
     const float thr32 = key_to_float(key_thr);
-    // error window: |g|, |u| carry at most 2^-18 of their largest magnitude of float32 accumulation error
     gmax = warp_max(gmax);
     umax = warp_max(umax);
     if (lane == 0) {
@@ -91,7 +90,10 @@ __global__ void __launch_bounds__(SEL_THREADS) channel_select_kernel(const ChanD
       gmax = fmaxf(gmax, sm.f[i]);
       umax = fmaxf(umax, __int_as_float(sm.i[i]));
     }
-    const float eps = 3.814697265625e-06f * fmaxf(gmax, umax);   // 2^-18 * scale: bound on the error of g_j, u_j
+    // error taken for g_j, u_j: the tensor cores add each 16-long slice of the dot product to the running
+    // float32 sum with truncation, so the error grows with the d/16 steps: (d/16) * 2^-24 of the largest
+    // magnitude, and never less than 2^-18 of it
+    const float eps = fmaxf(3.814697265625e-06f, (float)(d / 16) * 5.9604644775390625e-08f) * fmaxf(gmax, umax);
     const float delta = 2.0f * eps * (1.1f * umax + gmax) + 1e-6f * thr32;  // |silu'| <= 1.1, |silu(g)| <= |g|
     const float hi = thr32 + delta, lo = thr32 - delta;
     int n_in = 0;
