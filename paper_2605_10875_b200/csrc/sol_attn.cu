@@ -258,21 +258,22 @@ struct SelectDev {
   int* status;
 };
 
-// One CTA per (sequence, kv-head).  The scores are copied to shared memory once; every later pass
-// (radix digits, window scan, compaction) reads them from there.  Decided candidates are marked by
-// overwriting the shared copy with +-inf.
-__global__ void __launch_bounds__(SEL_THREADS) token_select_kernel(const SelectDev p) {
-  extern __shared__ __align__(16) float sv[];  // [T] scores of this (sequence, kv-head)
+// One CTA per (sequence, kv-head).  Every thread keeps KPT consecutive scores in registers (as order-
+// preserving keys) for all passes; candidates near the threshold are settled in float64.
+template <int THREADS, int KPT>
+__global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p) {
   __shared__ SelectSmem sm;
   __shared__ double qsum[128];
 
   const int kvh = blockIdx.x, b = blockIdx.y;
   const int Hkv = p.sh.n_kv_heads, hd = p.sh.head_dim, G = p.sh.n_q_heads / Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr int WARPS = THREADS / 32;
   const int bk = b * Hkv + kvh;
   const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
   const size_t row = (size_t)bk * p.Tmax;
   const float* sig = p.sigma + row;
+  const int j0 = tid * KPT;
 
   int total = 0;
   if (T > 0) {
@@ -283,13 +284,14 @@ __global__ void __launch_bounds__(SEL_THREADS) token_select_kernel(const SelectD
     if (bud > T) bud = T;
     const int k = min(T, max((int)bud, nf));
     auto forced = [&](int j) { return j < n_sink || j >= T - n_win; };
+    if (tid < 4) sm.counts[tid] = 0;
 
-    // mode 0: keep all; 1: forced only; 2: kept iff score > thr (candidates already decided and
-    // overwritten with +-inf); 3: key threshold with index-ordered ties (float32 ordering)
-    float thr = 0.f;
+    // mode 0: keep all; 1: forced only; 2: kept iff score above the window or a candidate decided in
+    // float64; 3: key threshold with index-ordered ties (float32 ordering, candidate list overflowed)
+    int mode, tie_need = 0, n_cand = 0;
     uint32_t key_thr = 0;
-    int tie_need = 0;
-    int mode;
+    float hi = 0.f, lo = 0.f;
+    uint32_t key[KPT];  // 0: absent, 0xffffffff: forced
 
     if (k >= T) {
       mode = 0;
@@ -297,54 +299,67 @@ __global__ void __launch_bounds__(SEL_THREADS) token_select_kernel(const SelectD
       mode = 1;
     } else {
       float mx = 0.f;
-      for (int j = tid; j < T; j += SEL_THREADS) {
-        const float s = sig[j] + 0.0f;
-        sv[j] = s;
-        if (!forced(j)) mx = fmaxf(mx, fabsf(s));
+#pragma unroll
+      for (int i = 0; i < KPT; i += 4) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (j0 + i < T) v = *reinterpret_cast<const float4*>(sig + j0 + i);
+        const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int j = j0 + i + e;
+          uint32_t kk = 0;
+          if (j < T) {
+            if (forced(j)) {
+              kk = 0xffffffffu;
+            } else {
+              const float sv = vv[e] + 0.0f;
+              kk = float_key(sv);
+              mx = fmaxf(mx, fabsf(sv));
+            }
+          }
+          key[i + e] = kk;
+        }
       }
-      mx = warp_max(mx);
-      if (lane == 0) sm.f[warp] = mx;
-      if (tid < 4) sm.counts[tid] = 0;
-      __syncthreads();
-      mx = sm.f[0];
-      for (int i = 1; i < SEL_WARPS; ++i) mx = fmaxf(mx, sm.f[i]);
-
-      key_thr = radix_select_kth([&](int j) { return forced(j) ? 0xffffffffu : float_key(sv[j]); }, T, k, tie_need, sm);
+      mx = block_max<THREADS>(mx, 0, sm);
+      key_thr = select_kth<THREADS, KPT>(key, k, tie_need, sm);
       mode = 3;
 
       // ---- window around the threshold, re-scored in float64 ----
       const float thr32 = key_to_float(key_thr);
       // 2^-16 of the largest score: far above the float32 accumulation error of a head_dim-long dot product
       const float delta = mx * 1.52587890625e-05f;
-      const float hi = thr32 + delta, lo = thr32 - delta;
+      hi = thr32 + delta;
+      lo = thr32 - delta;
       int n_in = 0;
-      for (int j = tid; j < T; j += SEL_THREADS) {
-        if (forced(j)) continue;
-        const float s = sv[j];
-        if (s > hi) {
+#pragma unroll
+      for (int i = 0; i < KPT; ++i) {
+        const uint32_t kk = key[i];
+        if (kk == 0u || kk == 0xffffffffu) continue;
+        const float sv = key_to_float(kk);
+        if (sv > hi) {
           ++n_in;
-        } else if (s >= lo) {
+        } else if (sv >= lo) {
           const int slot = atomicAdd(&sm.counts[0], 1);
-          if (slot < SEL_CAND_CAP) sm.cand_idx[slot] = j;
+          if (slot < SEL_CAND_CAP) sm.cand_idx[slot] = j0 + i;
         }
       }
-      if (n_in) atomicAdd(&sm.counts[1], n_in);
-      __syncthreads();
-      const int n_cand = sm.counts[0];
-      const int need = k - nf - sm.counts[1];
+      n_in = block_count<THREADS>(n_in, 0, sm);
+      n_cand = sm.counts[0];
+      const int need = k - nf - n_in;
       if (n_cand > SEL_CAND_CAP) {
         if (tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
+        n_cand = 0;
       } else {
         if (n_cand != need) {
           if (tid == 0) atomicAdd(p.status + ST_TOK_REFINED, n_cand);
-          for (int e = tid; e < hd; e += SEL_THREADS) {
+          for (int e = tid; e < hd; e += THREADS) {
             double a = 0.0;
             for (int h = 0; h < G; ++h) a += (double)p.q_rot[((size_t)b * p.sh.n_q_heads + kvh * G + h) * hd + e];
             qsum[e] = a;
           }
           __syncthreads();
           const uint16_t* kp = static_cast<const uint16_t*>(p.kv.k_pool);
-          for (int c = warp; c < n_cand; c += SEL_WARPS) {
+          for (int c = warp; c < n_cand; c += WARPS) {
             const int j = sm.cand_idx[c];
             const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + j / PAGE];
             double a = 0.0;
@@ -356,39 +371,43 @@ __global__ void __launch_bounds__(SEL_THREADS) token_select_kernel(const SelectD
             if (lane == 0) sm.cand_val[c] = a;
           }
           __syncthreads();
-          rank_candidates(n_cand, need, sm, [&](int c, bool keep) { sv[sm.cand_idx[c]] = keep ? INFINITY : -INFINITY; });
+          rank_candidates<THREADS>(n_cand, need, sm);
         } else {
-          for (int c = tid; c < n_cand; c += SEL_THREADS) sv[sm.cand_idx[c]] = INFINITY;
+          for (int c = tid; c < n_cand; c += THREADS) sm.cand_keep[c] = 1;
         }
-        thr = hi;
         mode = 2;
         __syncthreads();
       }
     }
 
-    auto klass = [&](int j) -> int {
-      if (mode == 0) return 2;
-      if (forced(j)) return 2;
-      if (mode == 1) return 0;
-      const float s = sv[j];
-      if (mode == 2) return s > thr ? 2 : 0;
-      const uint32_t key = float_key(s);
-      return key > key_thr ? 2 : (key == key_thr ? 1 : 0);
+    auto klass = [&](int i) -> int {
+      const int j = j0 + i;
+      if (j >= T) return 0;
+      if (mode == 0 || forced(j)) return 2;
+      if (mode == 2) {
+        const float sv = key_to_float(key[i]);
+        if (sv > hi) return 2;
+        if (sv >= lo) {  // within the window: look the token up in the decided list
+          for (int q = 0; q < n_cand; ++q)
+            if (sm.cand_idx[q] == j) return sm.cand_keep[q] ? 2 : 0;
+        }
+        return 0;
+      }
+      if (mode == 3) return key[i] > key_thr ? 2 : (key[i] == key_thr ? 1 : 0);
+      return 0;
     };
-    ordered_compact(klass, [](int, bool) {}, T, mode == 3 ? tie_need : 0, p.kept_idx + row, p.kept_cnt + bk, sm);
-    total = k;  // the compaction keeps exactly k indices
-  } else if (tid == 0) {
-    p.kept_cnt[bk] = 0;
+    total = compact_indices<THREADS, KPT>(klass, [](int, bool) {}, mode == 3 ? tie_need : 0, p.kept_idx + row, sm);
   }
+  if (tid == 0) p.kept_cnt[bk] = total;
 
   // pass-2 work items of this (sequence, kv-head): one per split_len kept tokens, at least one so
   // that the output is always written
   const int ns = max(1, (total + p.split_len - 1) / p.split_len);
   __syncthreads();
-  if (tid == 0) sm.pick[0] = atomicAdd(p.work_ctr, ns);
+  if (tid == 0) sm.counts[3] = atomicAdd(p.work_ctr, ns);
   __syncthreads();
-  const int base = sm.pick[0];
-  for (int i = tid; i < ns; i += SEL_THREADS) p.work_items[base + i] = bk * p.S + i;
+  const int base = sm.counts[3];
+  for (int i = tid; i < ns; i += THREADS) p.work_items[base + i] = bk * p.S + i;
 }
 
 // ============================================================================
@@ -709,9 +728,12 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   se.sigma = a.sigma; se.kept_idx = a.kept_idx; se.kept_cnt = a.kept_cnt;
   se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
   {
-    const int smem = Tmax * 4;
-    ensure_dynamic_smem(reinterpret_cast<const void*>(&token_select_kernel), smem);
-    SOL_LAUNCH("token_select", token_select_kernel, dim3(Hkv, a.B), dim3(SEL_THREADS), smem, st, se);
+    const dim3 grid(Hkv, a.B);
+    if (Tmax <= 1024) SOL_LAUNCH("token_select", (token_select_kernel<256, 4>), grid, dim3(256), 0, st, se);
+    else if (Tmax <= 4096) SOL_LAUNCH("token_select", (token_select_kernel<256, 16>), grid, dim3(256), 0, st, se);
+    else if (Tmax <= 16384) SOL_LAUNCH("token_select", (token_select_kernel<1024, 16>), grid, dim3(1024), 0, st, se);
+    else if (Tmax <= 32768) SOL_LAUNCH("token_select", (token_select_kernel<1024, 32>), grid, dim3(1024), 0, st, se);
+    else SOL_LAUNCH("token_select", (token_select_kernel<1024, 48>), grid, dim3(1024), 0, st, se);
   }
 
   GatherDev gd;

@@ -38,7 +38,7 @@ namespace sol {
 constexpr int UM_THREADS = 192;      // warps 0-3: epilogue, warp 4: TMA producer, warp 5: MMA issuer + TMEM owner
 constexpr int UM_MAX_STAGES = 8;
 constexpr int UM_TILE_SPAN = 16384;  // bytes one 128-row operand read spans from the start of a chunk tile
-constexpr int UM_SMEM_BUDGET = 196 * 1024;
+constexpr int UM_SMEM_BUDGET = 204 * 1024;
 
 struct UmBarriers {
   uint64_t full[UM_MAX_STAGES];
@@ -120,37 +120,40 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
     }
   } else if (warp == 5) {
     // ------------------------------- MMA issuer ------------------------------
-    if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16_m128(p.Mpad, 0, 0);
-      bool acc = false, ok = true;
-      for (int it = 0; it < n_iter; ++it) {
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
-        ok = mbar_wait(&bars->full[s], ph, p.status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
-        const uint32_t xs = st + NW * p.cps * w_tile;
-        for (int c = 0; c < p.cps; ++c) {
+    // The mbarrier wait orders the TMA writes before the MMA reads; no tcgen05 fence is needed per stage.
+    const uint32_t idesc = umma_idesc_bf16_m128(p.Mpad, 0, 0);
+    bool acc = false, ok = true;
+    for (int it = 0; it < n_iter; ++it) {
+      const int s = it % p.stages;
+      const uint32_t ph = (it / p.stages) & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[s], ph, p.status));
+      if (!ok) break;
+      const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
+      const uint32_t xs = st + NW * p.cps * w_tile;
+      const uint64_t a_base = umma_smem_desc(st, 16, 1024), b_base = umma_smem_desc(xs, 16, 1024);
+      for (int c = 0; c < p.cps; ++c) {
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
-            const uint64_t b0 = umma_smem_desc(xs + c * x_tile + ks * 32, 16, 1024);
-            const uint64_t b1 = umma_smem_desc(xs + (p.cps + c) * x_tile + ks * 32, 16, 1024);
-            const uint64_t a0 = umma_smem_desc(st + c * w_tile + ks * 32, 16, 1024);
+        for (int ks = 0; ks < 4; ++ks) {
+          // descriptors advance in units of 16 bytes: a chunk tile per c, 32 bytes per 16-wide k step
+          const uint64_t a0 = a_base + (uint64_t)((c * w_tile + ks * 32) >> 4);
+          const uint64_t a1 = a_base + (uint64_t)(((p.cps + c) * w_tile + ks * 32) >> 4);
+          const uint64_t b0 = b_base + (uint64_t)((c * x_tile + ks * 32) >> 4);
+          const uint64_t b1 = b_base + (uint64_t)(((p.cps + c) * x_tile + ks * 32) >> 4);
+          if (elect_one()) {
             umma_bf16(tmem, a0, b0, idesc, acc);
             if (p.n_b == 2) umma_bf16(tmem, a0, b1, idesc, true);
             if (NW == 2) {
-              const uint64_t a1 = umma_smem_desc(st + (p.cps + c) * w_tile + ks * 32, 16, 1024);
               umma_bf16(tmem + p.Mpad, a1, b0, idesc, acc);
               if (p.n_b == 2) umma_bf16(tmem + p.Mpad, a1, b1, idesc, true);
             }
-            acc = true;
           }
+          acc = true;
         }
-        umma_commit(&bars->empty[s]);  // the stage is free again once these MMAs have read it
       }
-      if (ok) umma_commit(&bars->accum);
+      if (elect_one()) umma_commit(&bars->empty[s]);  // the stage is free again once these MMAs have read it
+      __syncwarp();
     }
+    if (ok && elect_one()) umma_commit(&bars->accum);
   } else {
     // -------------------------------- epilogue -------------------------------
     if (warp * 32 < p.rows) {
@@ -257,35 +260,38 @@ umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
       }
     }
   } else if (warp == 5) {
-    if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16_m128(p.Mpad, 1, 0);
-      bool acc = false, ok = true;
-      int it = 0;
-      for (int jb = jb0; jb < jb1; ++jb) {
-        if (!block_live(p.live, jb, granules)) continue;
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
-        ++it;
-        ok = mbar_wait(&bars->full[s], ph, p.status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
+    const uint32_t idesc = umma_idesc_bf16_m128(p.Mpad, 1, 0);
+    bool acc = false, ok = true;
+    int it = 0;
+    for (int jb = jb0; jb < jb1; ++jb) {
+      if (!block_live(p.live, jb, granules)) continue;
+      const int s = it % p.stages;
+      const uint32_t ph = (it / p.stages) & 1;
+      ++it;
+      ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[s], ph, p.status));
+      if (!ok) break;
+      const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
+      // weight tile: two 64-column blocks of [64 channels][128 bytes]; 16 channels = two 8-row groups
+      const uint64_t a_base = umma_smem_desc(st, 8192, 1024);
+      const uint64_t h_base = umma_smem_desc(st + UM_TILE_SPAN, 16, 1024);
+      const uint64_t l_base = umma_smem_desc(st + UM_TILE_SPAN + t_tile, 16, 1024);
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-          // weight tile: two 64-column blocks of [64 channels][128 bytes]; 16 channels = two 8-row groups
-          const uint64_t a = umma_smem_desc(st + ks * 2048, 8192, 1024);
-          const uint64_t bh = umma_smem_desc(st + UM_TILE_SPAN + ks * 32, 16, 1024);
-          const uint64_t bl = umma_smem_desc(st + UM_TILE_SPAN + t_tile + ks * 32, 16, 1024);
-          umma_bf16(tmem, a, bh, idesc, acc);
-          umma_bf16(tmem, a, bl, idesc, true);
-          acc = true;
+      for (int ks = 0; ks < 4; ++ks) {
+        if (elect_one()) {
+          umma_bf16(tmem, a_base + (uint64_t)((ks * 2048) >> 4), h_base + (uint64_t)((ks * 32) >> 4), idesc, acc);
+          umma_bf16(tmem, a_base + (uint64_t)((ks * 2048) >> 4), l_base + (uint64_t)((ks * 32) >> 4), idesc, true);
         }
-        umma_commit(&bars->empty[s]);
+        acc = true;
       }
+      if (elect_one()) umma_commit(&bars->empty[s]);
+      __syncwarp();
+    }
+    if (lane == 0) {
       *reinterpret_cast<volatile int*>(&bars->n_issued) = acc ? 1 : 0;
       __threadfence_block();
-      if (ok) umma_commit(&bars->accum);
     }
+    __syncwarp();
+    if (ok && elect_one()) umma_commit(&bars->accum);
   } else {
     const bool ok = mbar_wait(&bars->accum, 0, p.status);
     tc_fence_after();

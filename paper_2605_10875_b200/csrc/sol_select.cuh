@@ -1,105 +1,158 @@
 // Block-wide exact top-k building blocks shared by the token and the channel
-// selection kernels (one 1024-thread CTA per selection problem):
+// selection kernels (one CTA per selection problem).
 //
-//   radix_select_kth   the k-th largest 32-bit key among n, 8 bits per pass,
-//                      plus how many keys equal to it are still needed
-//   ordered_compact    writes the kept indices in ascending order; class 2 is
-//                      kept, class 1 ("tie") is kept in ascending index order
-//                      until tie_need runs out, class 0 is dropped
-//   rank_candidates    ranks a short candidate list by (value descending,
-//                      index ascending)
+// Every thread holds KPT consecutive 32-bit keys in registers (key order =
+// value order, see float_key); nothing is re-read from memory between passes.
+//
+//   select_kth        the k-th largest key of the block (histogram of the top
+//                     key bits, then exact ranking inside the threshold bin),
+//                     plus how many keys equal to it are still needed
+//   block_count/max   reductions over the block
+//   rank_candidates   ranks a short candidate list by (value descending,
+//                     index ascending)
+//   compact_indices   writes the kept indices in ascending order
 #pragma once
 #include "sol_common.cuh"
 
 namespace sol {
 
-constexpr int SEL_THREADS = 1024;
-constexpr int SEL_WARPS = SEL_THREADS / 32;
-constexpr int SEL_HGROUPS = 8;
 constexpr int SEL_CAND_CAP = 1024;
+constexpr int SEL_RANK_CAP = 32;  // a threshold bin this small is ranked exactly instead of split further
+constexpr int SEL_BINS = 4096;
+constexpr int SEL_MAX_WARPS = 32;
 
 struct SelectSmem {
-  uint32_t hist[SEL_HGROUPS * 256];
-  int pick[2];
-  float f[SEL_WARPS];
-  int i[SEL_WARPS * 2];
+  uint32_t hist[SEL_BINS];
+  uint32_t rank_key[SEL_RANK_CAP];
+  int pick[3];
+  int scan[2][SEL_MAX_WARPS];  // per-warp totals of block_count / compact_indices / select_kth
+  float f[2][SEL_MAX_WARPS];
   int cand_idx[SEL_CAND_CAP];
   double cand_val[SEL_CAND_CAP];
+  unsigned char cand_keep[SEL_CAND_CAP];
   int counts[4];
 };
-
-// Warp 0 finds the digit that holds the `remaining`-th largest key and the
-// number of keys in higher digits.
-__device__ __forceinline__ void pick_digit(const uint32_t* hist, int remaining, int* out2) {
-  if (threadIdx.x < 32) {
-    const int lane = threadIdx.x;
-    int cnt[8];
-    int tot = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      int c = 0;
-      for (int gI = 0; gI < SEL_HGROUPS; ++gI) c += hist[gI * 256 + lane * 8 + i];
-      cnt[i] = c;
-      tot += c;
-    }
-    int run = tot;  // becomes the inclusive suffix sum over lanes >= lane
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int v = __shfl_down_sync(0xffffffffu, run, o);
-      if (lane + o < 32) run += v;
-    }
-    const int above = run - tot;
-    if (above < remaining && remaining <= above + tot) {
-      int a = above;
-      for (int i = 7; i >= 0; --i) {
-        if (remaining <= a + cnt[i]) {
-          out2[0] = lane * 8 + i;
-          out2[1] = a;
-          break;
-        }
-        a += cnt[i];
-      }
-    }
-  }
-}
-
-// key(j) -> uint32 for j in [0, n).  Requires 1 <= k <= n.  All threads call.
-template <typename KeyFn>
-__device__ __forceinline__ uint32_t radix_select_kth(KeyFn key, int n, int k, int& tie_need, SelectSmem& sm) {
-  const int tid = threadIdx.x, warp = tid >> 5;
-  uint32_t prefix = 0, mask = 0;
-  int remaining = k;
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    for (int i = tid; i < SEL_HGROUPS * 256; i += SEL_THREADS) sm.hist[i] = 0;
-    __syncthreads();
-    uint32_t* myh = sm.hist + (warp & (SEL_HGROUPS - 1)) * 256;
-    for (int j = tid; j < n; j += SEL_THREADS) {
-      const uint32_t kk = key(j);
-      if ((kk & mask) == prefix) atomicAdd(&myh[(kk >> shift) & 255u], 1u);
-    }
-    __syncthreads();
-    pick_digit(sm.hist, remaining, sm.pick);
-    __syncthreads();
-    prefix |= ((uint32_t)sm.pick[0]) << shift;
-    mask |= 255u << shift;
-    remaining -= sm.pick[1];
-    __syncthreads();
-  }
-  tie_need = remaining;
-  return prefix;
-}
 
 // Inverse of float_key.
 __device__ __forceinline__ float key_to_float(uint32_t key) {
   return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
 }
 
-// Ranks the first n_cand candidates; decide(c, keep) is called once per
-// candidate with keep = (rank < need).
-template <typename DecideFn>
-__device__ __forceinline__ void rank_candidates(int n_cand, int need, SelectSmem& sm, DecideFn decide) {
-  for (int c = threadIdx.x; c < n_cand; c += SEL_THREADS) {
+// The k-th largest of the block's keys (1 <= k <= number of keys).  Absent elements carry key 0 and
+// count like any other key, so k must not exceed the number of present elements.  tie_need = how many
+// keys equal to the result belong to the top k.  All threads call.
+//
+// One histogram pass over the top 12 key bits (shared-memory atomics) finds the bin that holds the
+// k-th key; if that bin is small its keys are listed and ranked exactly, otherwise the next 12 (then
+// the last 8) bits are histogrammed within it.
+template <int THREADS, int KPT>
+__device__ __forceinline__ uint32_t select_kth(const uint32_t (&key)[KPT], int k, int& tie_need, SelectSmem& sm) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  uint32_t prefix = 0, mask = 0;
+  int remaining = k, pop = 0;
+#pragma unroll 1
+  for (int level = 0; level < 3; ++level) {
+    const int bits = level == 2 ? 8 : 12, shift = level == 0 ? 20 : (level == 1 ? 8 : 0);
+    const int nb = 1 << bits;
+    for (int i = tid; i < nb; i += THREADS) sm.hist[i] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < KPT; ++i)
+      if ((key[i] & mask) == prefix) atomicAdd(&sm.hist[(key[i] >> shift) & (uint32_t)(nb - 1)], 1u);
+    __syncthreads();
+    // bins in descending order: thread t owns bins nb-1-t*bpt .. nb-bpt-t*bpt
+    const int bpt = nb >= THREADS ? nb / THREADS : 1;
+    const bool active = tid * bpt < nb;
+    int mine = 0;
+    if (active)
+      for (int q = 0; q < bpt; ++q) mine += (int)sm.hist[nb - 1 - tid * bpt - q];
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) sm.scan[0][warp] = incl;
+    __syncthreads();
+    int before = incl - mine;
+    for (int w = 0; w < warp; ++w) before += sm.scan[0][w];
+    if (active && before < remaining && remaining <= before + mine) {
+      int a = before;
+      for (int q = 0; q < bpt; ++q) {
+        const int bin = nb - 1 - tid * bpt - q;
+        const int c = (int)sm.hist[bin];
+        if (remaining <= a + c) {
+          sm.pick[0] = bin;
+          sm.pick[1] = a;
+          sm.pick[2] = c;
+          break;
+        }
+        a += c;
+      }
+    }
+    __syncthreads();
+    prefix |= (uint32_t)sm.pick[0] << shift;
+    mask |= (uint32_t)(nb - 1) << shift;
+    remaining -= sm.pick[1];
+    pop = sm.pick[2];
+    if (pop <= SEL_RANK_CAP) break;
+  }
+  if (mask == 0xffffffffu) {  // every bit decided: the keys left are all equal to the result
+    tie_need = remaining;
+    return prefix;
+  }
+  // list the keys under the prefix and rank them exactly
+  if (tid == 0) sm.counts[2] = 0;
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < KPT; ++i)
+    if ((key[i] & mask) == prefix) sm.rank_key[atomicAdd(&sm.counts[2], 1)] = key[i];
+  __syncthreads();
+  for (int c = tid; c < pop; c += THREADS) {
+    const uint32_t kc = sm.rank_key[c];
+    int gt = 0, ge = 0;
+    for (int o = 0; o < pop; ++o) {
+      const uint32_t ko = sm.rank_key[o];
+      gt += ko > kc;
+      ge += ko >= kc;
+    }
+    if (gt < remaining && remaining <= ge) {  // equal keys all write the same pair
+      sm.pick[0] = (int)kc;
+      sm.pick[1] = remaining - gt;
+    }
+  }
+  __syncthreads();
+  tie_need = sm.pick[1];
+  return (uint32_t)sm.pick[0];
+}
+
+// Sum of v over the block, returned to every thread.  `slot` (0 or 1) picks the scratch row so that
+// two calls in a row need no barrier between them.
+template <int THREADS>
+__device__ __forceinline__ int block_count(int v, int slot, SelectSmem& sm) {
+  constexpr int WARPS = THREADS / 32;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  v = __reduce_add_sync(0xffffffffu, v);
+  if (lane == 0) sm.scan[slot][warp] = v;
+  __syncthreads();
+  return __reduce_add_sync(0xffffffffu, lane < WARPS ? sm.scan[slot][lane] : 0);
+}
+
+template <int THREADS>
+__device__ __forceinline__ float block_max(float v, int slot, SelectSmem& sm) {
+  constexpr int WARPS = THREADS / 32;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  v = warp_max(v);
+  if (lane == 0) sm.f[slot][warp] = v;
+  __syncthreads();
+  return warp_max(lane < WARPS ? sm.f[slot][lane] : 0.f);
+}
+
+// Ranks the first n_cand candidates (cand_val, cand_idx) and sets cand_keep[c] = (rank < need).
+// A barrier must separate the writes of cand_val from this call and this call from the readers.
+template <int THREADS>
+__device__ __forceinline__ void rank_candidates(int n_cand, int need, SelectSmem& sm) {
+  for (int c = threadIdx.x; c < n_cand; c += THREADS) {
     const double v = sm.cand_val[c];
     const int j = sm.cand_idx[c];
     int rank = 0;
@@ -107,58 +160,68 @@ __device__ __forceinline__ void rank_candidates(int n_cand, int need, SelectSmem
       const double vo = sm.cand_val[o];
       rank += (vo > v) || (vo == v && sm.cand_idx[o] < j);
     }
-    decide(c, rank < need);
+    sm.cand_keep[c] = rank < need ? 1 : 0;
   }
 }
 
-// klass(j) in {0,1,2}; emit(j, keep) is called for every j in [0, n) (may be a
-// no-op); kept indices go to out[] ascending; returns nothing, thread 0
-// writes the kept count to *out_cnt.  All threads call.
-template <typename ClassFn, typename EmitFn>
-__device__ __forceinline__ void ordered_compact(ClassFn klass, EmitFn emit, int n, int tie_need, int32_t* out,
-                                                int32_t* out_cnt, SelectSmem& sm) {
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int per_warp = ((n + SEL_WARPS - 1) / SEL_WARPS + 31) / 32 * 32;
-  const int w0 = warp * per_warp, w1 = min(n, w0 + per_warp);
+// klass(i) in {0 dropped, 1 tie, 2 kept} for element j = tid*KPT + i (called twice per element).  Ties
+// are kept in ascending index order until tie_need runs out.  Kept indices go to out[] ascending;
+// emit(i, keep) reports the final decision of every element.  Returns the kept total to every thread.
+// All threads call; uses sm.scan.
+template <int THREADS, int KPT, typename ClassFn, typename EmitFn>
+__device__ __forceinline__ int compact_indices(ClassFn klass, EmitFn emit, int tie_need, int32_t* out, SelectSmem& sm) {
+  constexpr int WARPS = THREADS / 32;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int c2 = 0, c1 = 0;
-  for (int j = w0 + lane; j < w0 + per_warp; j += 32) {
-    const int c = j < w1 ? klass(j) : 0;
-    c2 += __popc(__ballot_sync(0xffffffffu, c == 2));
-    c1 += __popc(__ballot_sync(0xffffffffu, c == 1));
+#pragma unroll
+  for (int i = 0; i < KPT; ++i) {
+    const int c = klass(i);
+    c2 += c == 2;
+    c1 += c == 1;
   }
-  __syncthreads();
-  if (lane == 0) {
-    sm.i[warp] = c2;
-    sm.i[SEL_WARPS + warp] = c1;
+  // exclusive prefix of ties over the block (threads in index order), then of kept elements
+  int t_incl = c1;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, t_incl, o);
+    if (lane >= o) t_incl += v;
   }
+  __syncthreads();  // earlier readers of sm.scan are done
+  if (lane == 31) sm.scan[0][warp] = t_incl;
   __syncthreads();
-  int tie_before = 0, kept_before = 0, total = 0;
-  {
-    int tb = 0;
-    for (int w = 0; w < SEL_WARPS; ++w) {
-      const int t1 = sm.i[SEL_WARPS + w];
-      const int kept_w = sm.i[w] + min(max(tie_need - tb, 0), t1);
-      if (w < warp) {
-        kept_before += kept_w;
-        tie_before = tb + t1;
-      }
-      total += kept_w;
-      tb += t1;
+  int t_before = t_incl - c1;
+  for (int w = 0; w < warp; ++w) t_before += sm.scan[0][w];
+  const int my_ties = min(max(tie_need - t_before, 0), c1);
+  const int mine = c2 + my_ties;
+  int k_incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, k_incl, o);
+    if (lane >= o) k_incl += v;
+  }
+  if (lane == 31) sm.scan[1][warp] = k_incl;
+  __syncthreads();
+  int pos = k_incl - mine, total = 0;
+  for (int w = 0; w < WARPS; ++w) {
+    const int v = sm.scan[1][w];
+    if (w < warp) pos += v;
+    total += v;
+  }
+  int ties_left = my_ties;
+  const int j0 = threadIdx.x * KPT;
+#pragma unroll
+  for (int i = 0; i < KPT; ++i) {
+    const int c = klass(i);
+    bool kp = c == 2;
+    if (c == 1 && ties_left > 0) {
+      kp = true;
+      --ties_left;
     }
+    if (kp) out[pos++] = j0 + i;
+    emit(i, kp);
   }
-  if (tid == 0) *out_cnt = total;
-  int pos = kept_before, ties = tie_before;
-  for (int j = w0 + lane; j < w0 + per_warp; j += 32) {
-    const int c = j < w1 ? klass(j) : 0;
-    const unsigned m1 = __ballot_sync(0xffffffffu, c == 1);
-    const int my_tie_rank = ties + __popc(m1 & ((1u << lane) - 1));
-    const bool keep = c == 2 || (c == 1 && my_tie_rank < tie_need);
-    const unsigned mk = __ballot_sync(0xffffffffu, keep);
-    if (keep) out[pos + __popc(mk & ((1u << lane) - 1))] = j;
-    if (j < w1) emit(j, keep);
-    pos += __popc(mk);
-    ties += __popc(m1);
-  }
+  __syncthreads();  // sm.scan may be reused by the caller
+  return total;
 }
 
 }  // namespace sol
