@@ -272,7 +272,7 @@ static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, cons
   dn.status = status;
   launch_gemm_down(dn, st);
   launch_reduce_out(dn.partial, dn.chunks, B, pad_rows(B), s.d_model, resid, resid_f32, out_bf16, out_f32, out_f32_b,
-                    st);
+                    cs.live, s.d_ff / 32, st);
 }
 
 static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol_layer_weights_t& w,

@@ -56,6 +56,8 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
   const int pos = T - 1;
   const bool layer = p.qkv != nullptr;
   const bool rope = layer && p.sh.rope_theta > 0.f;
+  pdl_trigger();
+  pdl_wait();
 
   if (tid == 0) {
     p.work_ctr[2 + b * Hkv + kvh] = 0;
@@ -158,11 +160,13 @@ __global__ void __launch_bounds__(SC_WARPS * 32) attn_score_kernel(const ScoreDe
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SC_WARPS * PAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.z, kvh = blockIdx.y;
+  pdl_trigger();
   if (threadIdx.x == 0) {
     for (int i = 0; i < SC_WARPS; ++i) mbar_init(&bars[i], 1);
     fence_mbar_init();
   }
   __syncthreads();
+  pdl_wait();
 
   const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
   const int lp = blockIdx.x * SC_WARPS + warp;  // logical page
@@ -270,6 +274,8 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int WARPS = THREADS / 32;
   const int bk = b * Hkv + kvh;
+  pdl_trigger();
+  pdl_wait();
   const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
   const size_t row = (size_t)bk * p.Tmax;
   const float* sig = p.sigma + row;
@@ -487,6 +493,8 @@ __global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev
   const int G = p.G, Hkv = p.Hkv;
   const uint16_t* vp = static_cast<const uint16_t*>(p.kv.v_pool);
   constexpr int CH = HD / 8;  // 16-byte chunks per row
+  pdl_trigger();
+  pdl_wait();
 
   for (;;) {
     if (tid == 0) {

@@ -101,6 +101,13 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   return v;
 }
 
+// ---- programmatic dependent launch ---------------------------------------------
+// pdl_trigger: the next kernel in the stream may be scheduled from now on (it still waits in
+// pdl_wait for this grid to finish).  pdl_wait: returns once every earlier kernel has completed and
+// its writes are visible; until then only constants (weights, shapes) may be read.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- small reductions ---------------------------------------------------------
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

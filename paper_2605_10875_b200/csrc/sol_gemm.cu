@@ -83,6 +83,7 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
   UmBarriers* bars = reinterpret_cast<UmBarriers*>(stages + (size_t)p.stages * stage_bytes + UM_TILE_SPAN);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_trigger();
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(&bars->full[s], 1);
@@ -102,10 +103,25 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
 
   if (warp == 4) {
     // ------------------------------ TMA producer -----------------------------
+    // Weights do not depend on earlier kernels: the first ring of weight tiles is requested before
+    // pdl_wait(), the activation tiles of those stages after it.
     if (lane == 0) {
       tma_prefetch_map(&tm_w0);
       tma_prefetch_map(&tm_x0);
-      for (int it = 0; it < n_iter; ++it) {
+      const int pre = min(n_iter, p.stages);
+      for (int it = 0; it < pre; ++it) {
+        unsigned char* st = stages + (size_t)it * stage_bytes;
+        mbar_expect_tx(&bars->full[it], stage_bytes);
+        tma_load_3d(st, &tm_w0, 0, row0, it * p.cps, &bars->full[it]);
+        if (NW == 2) tma_load_3d(st + p.cps * w_tile, &tm_w1, 0, row0, it * p.cps, &bars->full[it]);
+      }
+      pdl_wait();
+      for (int it = 0; it < pre; ++it) {
+        unsigned char* xs = stages + (size_t)it * stage_bytes + NW * p.cps * w_tile;
+        tma_load_3d(xs, &tm_x0, 0, 0, it * p.cps, &bars->full[it]);
+        if (p.n_b == 2) tma_load_3d(xs + p.cps * x_tile, &tm_x1, 0, 0, it * p.cps, &bars->full[it]);
+      }
+      for (int it = pre; it < n_iter; ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
         if (!mbar_wait(&bars->empty[s], ph ^ 1, p.status)) break;
@@ -156,6 +172,7 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
     if (ok && elect_one()) umma_commit(&bars->accum);
   } else {
     // -------------------------------- epilogue -------------------------------
+    pdl_wait();  // the epilogue reads scales / the residual and overwrites buffers earlier kernels used
     if (warp * 32 < p.rows) {
       const bool ok = mbar_wait(&bars->accum, 0, p.status);
       tc_fence_after();
@@ -222,6 +239,7 @@ umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
   UmBarriers* bars = reinterpret_cast<UmBarriers*>(stages + (size_t)p.stages * stage_bytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_trigger();
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(&bars->full[s], 1);
@@ -235,6 +253,7 @@ umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();  // which channel blocks are live is decided by the selection kernel
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
 
   const int slab = blockIdx.x, chunk = blockIdx.y;
@@ -514,8 +533,13 @@ void launch_gemm_down(const GemmDown& g, cudaStream_t st) {
 // ============================================================================
 __global__ void reduce_out_kernel(const float* __restrict__ partial, int chunks, int M, int Mpad, int d,
                                   const void* __restrict__ resid, int resid_f32, uint16_t* __restrict__ out_bf16,
-                                  float* __restrict__ out_f32, float* __restrict__ out_f32_b) {
-  const int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+                                  float* __restrict__ out_f32, float* __restrict__ out_f32_b, int32_t* __restrict__ live,
+                                  int n_live) {
+  pdl_trigger();
+  pdl_wait();
+  const int gi = blockIdx.x * blockDim.x + threadIdx.x;
+  if (gi < n_live) live[gi] = 0;  // the down projection has read the flags; the next selection starts from zero
+  const int i = gi * 4;
   if (i >= M * d) return;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int c = 0; c < chunks; ++c) {
@@ -542,10 +566,11 @@ __global__ void reduce_out_kernel(const float* __restrict__ partial, int chunks,
 }
 
 void launch_reduce_out(const float* partial, int chunks, int M, int Mpad, int d, const void* resid, int resid_f32,
-                       void* out_bf16, float* out_f32, float* out_f32_b, cudaStream_t st) {
-  const int n4 = M * d / 4;
+                       void* out_bf16, float* out_f32, float* out_f32_b, int32_t* live, int n_live, cudaStream_t st) {
+  int n4 = M * d / 4;
+  if (n4 < n_live) n4 = n_live;
   SOL_LAUNCH("down_reduce_residual", reduce_out_kernel, dim3((n4 + 255) / 256), dim3(256), 0, st, partial, chunks, M,
-             Mpad, d, resid, resid_f32, static_cast<uint16_t*>(out_bf16), out_f32, out_f32_b);
+             Mpad, d, resid, resid_f32, static_cast<uint16_t*>(out_bf16), out_f32, out_f32_b, live, n_live);
 }
 
 }  // namespace sol

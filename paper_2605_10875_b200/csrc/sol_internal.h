@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
+#include <string.h>
 
 #include "../../include/sol.h"
 
@@ -16,11 +17,25 @@ void note_launch_end(cudaStream_t st);
 bool record_cuda_error(cudaError_t e, const char* where);  // true if e != success
 bool take_cuda_failure();  // true if a CUDA call of this thread failed since the last check; clears the mark
 
-#define SOL_LAUNCH(name, kernel, grid, block, smem, st, ...)             \
-  do {                                                                   \
-    ::sol::note_launch_begin(name, st);                                  \
-    kernel<<<grid, block, smem, st>>>(__VA_ARGS__);                      \
-    ::sol::note_launch_end(st);                                          \
+// Every kernel is launched with programmatic stream serialization: it may start while the kernel
+// before it in the stream is still running, does its set-up (and, for the GEMMs, starts streaming
+// weights), and calls pdl_wait() before it touches anything an earlier kernel produced.
+#define SOL_LAUNCH(name, kernel, grid, block, smem, st, ...)                                   \
+  do {                                                                                         \
+    ::sol::note_launch_begin(name, st);                                                        \
+    cudaLaunchConfig_t sol_cfg_;                                                               \
+    memset(&sol_cfg_, 0, sizeof(sol_cfg_));                                                    \
+    sol_cfg_.gridDim = grid;                                                                   \
+    sol_cfg_.blockDim = block;                                                                 \
+    sol_cfg_.dynamicSmemBytes = smem;                                                          \
+    sol_cfg_.stream = st;                                                                      \
+    cudaLaunchAttribute sol_attr_[1];                                                          \
+    sol_attr_[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                      \
+    sol_attr_[0].val.programmaticStreamSerializationAllowed = 1;                               \
+    sol_cfg_.attrs = sol_attr_;                                                                \
+    sol_cfg_.numAttrs = 1;                                                                     \
+    ::sol::record_cuda_error(cudaLaunchKernelEx(&sol_cfg_, kernel, __VA_ARGS__), name);        \
+    ::sol::note_launch_end(st);                                                                \
   } while (0)
 
 int sm_count();
@@ -67,8 +82,9 @@ struct GemmDown {
 int down_chunks(int ff, int d);
 void launch_gemm_down(const GemmDown& p, cudaStream_t st);
 // out = resid + sum over chunks of partial; out_bf16 / out_f32 optional.
+// Also clears the n_live "granule is live" flags, which every reader has finished with by then.
 void launch_reduce_out(const float* partial, int chunks, int M, int Mpad, int d, const void* resid, int resid_f32,
-                       void* out_bf16, float* out_f32, float* out_f32_b, cudaStream_t st);
+                       void* out_bf16, float* out_f32, float* out_f32_b, int32_t* live, int n_live, cudaStream_t st);
 
 // ---- attention (sol_attn.cu) ------------------------------------------------
 struct AttnArgs {
@@ -123,7 +139,7 @@ struct ChannelSelectArgs {
   int32_t* kept_cnt;   // [B]
   void* t_hi;          // bf16 [Mpad][ff]
   void* t_lo;
-  int32_t* live;       // [ff/32], zeroed by the launcher
+  int32_t* live;       // [ff/32], all zero on entry (cleared by reduce_out after the down projection)
   int* status;
 };
 void launch_channel_select(const ChannelSelectArgs& a, cudaStream_t st);

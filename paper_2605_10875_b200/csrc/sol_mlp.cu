@@ -54,6 +54,8 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int WARPS = THREADS / 32;
   const int ff = p.ff, d = p.d;
+  pdl_trigger();
+  pdl_wait();
   const float* tt = p.t + (size_t)b * ff;
   const int m = (int)(((long long)(1000 - p.p_permille[b]) * ff + 999) / 1000);
   const int j0 = tid * KPT;
@@ -240,7 +242,6 @@ void launch_channel_select(const ChannelSelectArgs& a, cudaStream_t st) {
   c.kept_ch = a.kept_ch; c.kept_cnt = a.kept_cnt;
   c.t_hi = static_cast<uint16_t*>(a.t_hi); c.t_lo = static_cast<uint16_t*>(a.t_lo);
   c.live = a.live; c.status = a.status;
-  cudaMemsetAsync(a.live, 0, sizeof(int32_t) * (a.ff / 32), st);
   const dim3 grid(a.B);
   if (a.ff <= 2048) SOL_LAUNCH("channel_select", (channel_select_kernel<256, 8>), grid, dim3(256), 0, st, c);
   else if (a.ff <= 8192) SOL_LAUNCH("channel_select", (channel_select_kernel<512, 16>), grid, dim3(512), 0, st, c);

@@ -32,6 +32,8 @@ norm_quant_kernel(const void* __restrict__ in, const uint16_t* __restrict__ gamm
                   const int32_t* __restrict__ bits, int d, uint16_t* __restrict__ a_op, float* __restrict__ scale,
                   float* __restrict__ xn, int8_t* __restrict__ codes, int* __restrict__ status) {
   __shared__ float sh[NQ_THREADS / 32];
+  pdl_trigger();
+  pdl_wait();
   const int row = blockIdx.x;
   const int nvec = d / NQ_VEC;
   float x[NQ_MAX_PER_THREAD][NQ_VEC];
