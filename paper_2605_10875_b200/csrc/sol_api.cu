@@ -99,7 +99,7 @@ static int pad_rows(int B) {
 
 struct Layout {
   size_t status, stage_h_in, stage_act, stage_h_out, a_op, scale, qkv, q_rot, q_split, logits, sigma, kept_idx,
-      kept_cnt, part, work_items, work_ctr, attn_hi, attn_lo, attn_f32, h_mid, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, down_part,
+      kept_cnt, part, work_items, work_ctr, attn_hi, attn_lo, attn_f32, h_mid, o_part, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, down_part,
       h_a, h_b, total;
   int splits, chunks, Mpad, Tmax;
 };
@@ -139,7 +139,7 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   L.stage_h_out = take(B * d * 2);
   L.a_op = take(Mpad * d * 2);
   L.scale = take(Mpad * 4);
-  L.qkv = take(B * Nqkv * 4);
+  L.qkv = take((size_t)NK_MAX_KSPLIT * B * Nqkv * 4);  // split-K partial sums of the QKV projection
   L.q_rot = take(B * Hq * hd * 4);
   L.q_split = take(B * Hkv * HG * 16 * hd * 2);
   L.logits = take(B * Hkv * Tmax * G * 4);
@@ -153,6 +153,7 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   L.attn_lo = take(Mpad * Hq * hd * 2);
   L.attn_f32 = take(B * Hq * hd * 4);
   L.h_mid = take(B * d * 4);
+  L.o_part = take((size_t)NK_MAX_KSPLIT * B * d * 4);  // split-K partial sums of the output projection
   L.g = take(B * ff * 4);
   L.u = take(B * ff * 4);
   L.t = take(B * ff * 4);
@@ -190,7 +191,8 @@ static bool kv_ok(const sol_kv_t* kv) {
 // compositions
 // ---------------------------------------------------------------------------
 static void run_attention(const sol_shape_t& s, const Layout& L, void* ws, const sol_kv_t& kv, int B,
-                          const int32_t* r_permille, const float* qkv, int ldq, const void* q_bf16, void* out_bf16,
+                          const int32_t* r_permille, const float* qkv, int ldq, int qkv_ksplit, const float* qkv_scale,
+                          const void* q_bf16, void* out_bf16,
                           float* out_f32, bool want_split, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t st) {
   AttnArgs a;
   a.shape = s;
@@ -199,6 +201,8 @@ static void run_attention(const sol_shape_t& s, const Layout& L, void* ws, const
   a.r_permille = r_permille;
   a.qkv_f32 = qkv;
   a.ldq = ldq;
+  a.qkv_ksplit = qkv_ksplit;
+  a.qkv_scale = qkv_scale;
   a.q_bf16 = q_bf16;
   a.q_rot = at<float>(ws, L.q_rot);
   a.q_split = at<void>(ws, L.q_split);
@@ -284,45 +288,56 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   const int Nqkv = (Hq + 2 * Hkv) * hd;
   float* scale = at<float>(ws, L.scale);
 
-  launch_norm_quant(h_in, in_f32, w.gamma1, s.rms_eps, bits, B, d, at<void>(ws, L.a_op), scale,
-                    tr ? tr->xn1 : nullptr, tr ? tr->codes1 : nullptr, status, st);
+  NormQuantArgs n1;
+  memset(&n1, 0, sizeof(n1));
+  n1.in = h_in; n1.in_f32 = in_f32; n1.gamma_bf16 = w.gamma1; n1.eps = s.rms_eps; n1.bits = bits; n1.B = B; n1.d = d;
+  n1.a_op = at<void>(ws, L.a_op); n1.scale = scale; n1.xn = tr ? tr->xn1 : nullptr; n1.codes = tr ? tr->codes1 : nullptr;
+  n1.status = status;
+  launch_norm_quant(n1, st);
   if (tr && tr->scales1) cudaMemcpyAsync(tr->scales1, scale, sizeof(float) * B, cudaMemcpyDeviceToDevice, st);
 
+  // QKV projection, split over K: raw partial sums, summed and scaled by the kernel that rotates and appends
   GemmNK q;
   memset(&q, 0, sizeof(q));
+  q.name = "gemm_qkv";
   q.a_hi = at<void>(ws, L.a_op);
   q.w0 = w.w_qkv;
   q.M = B;
   q.K = d;
   q.N = Nqkv;
-  q.row_scale = scale;
   q.out0 = at<float>(ws, L.qkv);
   q.status = status;
-  launch_gemm_nk(q, EPI_SCALE, st);
+  launch_gemm_nk(q, EPI_PARTIAL, st);
 
-  run_attention(s, L, ws, kv, B, r, at<float>(ws, L.qkv), Nqkv, nullptr, nullptr, tr ? tr->attn_out : nullptr, true,
-                tr ? tr->kept_idx : nullptr, tr ? tr->kept_cnt : nullptr, st);
+  run_attention(s, L, ws, kv, B, r, at<float>(ws, L.qkv), Nqkv, nk_ksplit(Nqkv, d), scale, nullptr, nullptr,
+                tr ? tr->attn_out : nullptr, true, tr ? tr->kept_idx : nullptr, tr ? tr->kept_cnt : nullptr, st);
   if (tr && tr->q_rot)
     cudaMemcpyAsync(tr->q_rot, at<float>(ws, L.q_rot), sizeof(float) * B * Hq * hd, cudaMemcpyDeviceToDevice, st);
 
+  // output projection, split over K; the second RMSNorm kernel adds the partial sums to the residual
   GemmNK o;
   memset(&o, 0, sizeof(o));
+  o.name = "gemm_out_proj";
   o.a_hi = at<void>(ws, L.attn_hi);
   o.a_lo = at<void>(ws, L.attn_lo);
   o.w0 = w.w_o;
   o.M = B;
   o.K = Hq * hd;
   o.N = d;
-  o.resid = h_in;
-  o.resid_f32 = in_f32 ? 1 : 0;
-  o.out0 = at<float>(ws, L.h_mid);
+  o.out0 = at<float>(ws, L.o_part);
   o.status = status;
-  launch_gemm_nk(o, EPI_RESIDUAL, st);
+  launch_gemm_nk(o, EPI_PARTIAL, st);
+
+  NormQuantArgs n2;
+  memset(&n2, 0, sizeof(n2));
+  n2.in = h_in; n2.in_f32 = in_f32; n2.part = at<float>(ws, L.o_part); n2.ksplit = nk_ksplit(d, Hq * hd);
+  n2.sum_out = at<float>(ws, L.h_mid);
+  n2.gamma_bf16 = w.gamma2; n2.eps = s.rms_eps; n2.bits = bits; n2.B = B; n2.d = d;
+  n2.a_op = at<void>(ws, L.a_op); n2.scale = scale; n2.xn = tr ? tr->xn2 : nullptr; n2.codes = tr ? tr->codes2 : nullptr;
+  n2.status = status;
+  launch_norm_quant(n2, st);
   if (tr && tr->h_mid)
     cudaMemcpyAsync(tr->h_mid, at<float>(ws, L.h_mid), sizeof(float) * B * d, cudaMemcpyDeviceToDevice, st);
-
-  launch_norm_quant(at<float>(ws, L.h_mid), true, w.gamma2, s.rms_eps, bits, B, d, at<void>(ws, L.a_op), scale,
-                    tr ? tr->xn2 : nullptr, tr ? tr->codes2 : nullptr, status, st);
   if (tr && tr->scales2) cudaMemcpyAsync(tr->scales2, scale, sizeof(float) * B, cudaMemcpyDeviceToDevice, st);
 
   run_mlp(s, L, ws, B, w.w_gate, w.w_up, w.w_down_t, p, at<float>(ws, L.h_mid), 1, h_out_bf16, h_out_f32,
@@ -376,8 +391,10 @@ sol_status_t sol_quant_act(const void* x_bf16, int32_t B, int32_t d, const int32
   if (!x_bf16 || !bits || !codes || !scales || B < 0 || d <= 0) return SOL_ERR_INVALID_ARG;
   if (d % 8 || d > 8192) return SOL_ERR_UNSUPPORTED;
   if (B == 0) return SOL_OK;
-  launch_norm_quant(x_bf16, false, nullptr, 0.f, bits, B, d, xhat_bf16, scales, nullptr, codes, nullptr,
-                    (cudaStream_t)stream);
+  NormQuantArgs n;
+  memset(&n, 0, sizeof(n));
+  n.in = x_bf16; n.bits = bits; n.B = B; n.d = d; n.a_op = xhat_bf16; n.scale = scales; n.codes = codes;
+  launch_norm_quant(n, (cudaStream_t)stream);
   return finish();
 }
 
@@ -389,8 +406,8 @@ sol_status_t sol_sparse_decode_attn(const sol_shape_t* shape, const void* q_bf16
   if (B == 0) return SOL_OK;
   const Layout L = make_layout(*shape, B, kv->max_pages_per_seq);
   if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
-  run_attention(*shape, L, ws, *kv, B, r_permille, nullptr, 0, q_bf16, out_bf16, nullptr, false, kept_idx, kept_cnt,
-                (cudaStream_t)stream);
+  run_attention(*shape, L, ws, *kv, B, r_permille, nullptr, 0, 0, nullptr, q_bf16, out_bf16, nullptr, false, kept_idx,
+                kept_cnt, (cudaStream_t)stream);
   return finish();
 }
 
@@ -406,8 +423,10 @@ sol_status_t sol_pruned_swiglu_mlp(const sol_shape_t* shape, const void* x_bf16,
   if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
   // bf16 passthrough into the padded operand buffer, scale 1
-  launch_norm_quant(x_bf16, false, nullptr, 0.f, nullptr, B, shape->d_model, at<void>(ws, L.a_op),
-                    at<float>(ws, L.scale), nullptr, nullptr, nullptr, st);
+  NormQuantArgs n;
+  memset(&n, 0, sizeof(n));
+  n.in = x_bf16; n.B = B; n.d = shape->d_model; n.a_op = at<void>(ws, L.a_op); n.scale = at<float>(ws, L.scale);
+  launch_norm_quant(n, st);
   run_mlp(*shape, L, ws, B, w_gate, w_up, w_down_t, p_permille, nullptr, 0, out_bf16, nullptr, nullptr, nullptr,
           kept_ch, kept_ch_cnt, st);
   return finish();

@@ -34,8 +34,9 @@ constexpr int PAGE = 64;
 struct PrepDev {
   sol_shape_t sh;
   sol_kv_t kv;
-  const float* qkv;  // [B][ldq] or nullptr
-  int ldq;
+  const float* qkv;  // [ksplit][B][ldq] partial sums of the QKV projection, or nullptr
+  int ldq, ksplit, B;
+  const float* qkv_scale;  // [B]
   const uint16_t* q_bf16;  // [B][Hq][hd] or nullptr
   float* q_rot;
   uint16_t* q_split;
@@ -58,6 +59,14 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
   const bool rope = layer && p.sh.rope_theta > 0.f;
   pdl_trigger();
   pdl_wait();
+
+  // element `col` of this sequence's q/k/v row: the K slices summed in order, times the quantizer scale
+  const float row_scale = (layer && p.qkv_scale) ? p.qkv_scale[b] : 1.0f;
+  auto qkv_at = [&](int col) -> float {
+    float a = 0.f;
+    for (int z = 0; z < p.ksplit; ++z) a += p.qkv[((size_t)z * p.B + b) * p.ldq + col];
+    return a * row_scale;
+  };
 
   if (tid == 0) {
     p.work_ctr[2 + b * Hkv + kvh] = 0;
@@ -89,8 +98,7 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
     const int gi = i / half, f = i % half, h = kvh * G + gi;
     float q0, q1;
     if (layer) {
-      const float* src = p.qkv + (size_t)b * p.ldq + h * hd;
-      const float x0 = src[f], x1 = src[f + half];
+      const float x0 = qkv_at(h * hd + f), x1 = qkv_at(h * hd + f + half);
       q0 = x0 * cs[f] + (-x1) * sn[f];
       q1 = x1 * cs[f] + x0 * sn[f];
     } else {
@@ -127,15 +135,14 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
   }
   uint16_t* kp = static_cast<uint16_t*>(p.kv.k_pool);
   uint16_t* vp = static_cast<uint16_t*>(p.kv.v_pool);
-  const float* ks = p.qkv + (size_t)b * p.ldq + (Hq + kvh) * hd;
-  const float* vs = p.qkv + (size_t)b * p.ldq + (Hq + Hkv + kvh) * hd;
+  const int kcol = (Hq + kvh) * hd, vcol = (Hq + Hkv + kvh) * hd;
   const size_t dst = (((size_t)page * Hkv + kvh) * PAGE + slot) * hd;
   for (int f = tid; f < half; f += PREP_THREADS) {
-    const float x0 = ks[f], x1 = ks[f + half];
+    const float x0 = qkv_at(kcol + f), x1 = qkv_at(kcol + f + half);
     kp[dst + f] = f2bf(x0 * cs[f] + (-x1) * sn[f]);
     kp[dst + f + half] = f2bf(x1 * cs[f] + x0 * sn[f]);
-    vp[dst + f] = f2bf(vs[f]);
-    vp[dst + f + half] = f2bf(vs[f + half]);
+    vp[dst + f] = f2bf(qkv_at(vcol + f));
+    vp[dst + f + half] = f2bf(qkv_at(vcol + f + half));
   }
 }
 
@@ -717,7 +724,8 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   const int Tmax = a.kv.max_pages_per_seq * PAGE;
 
   PrepDev pd;
-  pd.sh = sh; pd.kv = a.kv; pd.qkv = a.qkv_f32; pd.ldq = a.ldq;
+  pd.sh = sh; pd.kv = a.kv; pd.qkv = a.qkv_f32; pd.ldq = a.ldq; pd.ksplit = a.qkv_ksplit; pd.B = a.B;
+  pd.qkv_scale = a.qkv_scale;
   pd.q_bf16 = static_cast<const uint16_t*>(a.q_bf16);
   pd.q_rot = a.q_rot; pd.q_split = static_cast<uint16_t*>(a.q_split); pd.work_ctr = a.work_ctr; pd.status = a.status;
   SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(Hkv, a.B), dim3(PREP_THREADS), 0, st, pd);

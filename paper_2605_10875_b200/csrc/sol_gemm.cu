@@ -59,12 +59,12 @@ __device__ __forceinline__ unsigned char* align_1024(unsigned char* p) {
 struct NKDev {
   int M, Mpad, K, N;  // N: weight rows (EPI_SWIGLU: channels, with a gate and an up row each)
   int rows;           // weight rows per CTA
+  int ksplit;         // K slices (blockIdx.y); EPI_PARTIAL writes one partial per slice
   int cps, stages;    // 64-wide k chunks per stage, ring depth
-  int n_b;            // activation operands: 1, or 2 for a high + low bf16 pair
+  int n_b;            // 1, or 2: the activation rows are a high-part block followed by a low-part block of
+                      // Mpad rows each; one MMA of N = 2 Mpad multiplies both, the epilogue adds the halves
   uint32_t tmem_cols;
   const float* row_scale;
-  const void* resid;
-  int resid_f32;
   float* out0;
   float* out1;
   float* out2;
@@ -74,12 +74,13 @@ struct NKDev {
 template <int EPI>
 __global__ void __launch_bounds__(UM_THREADS, 1)
 umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant__ CUtensorMap tm_w1,
-               const __grid_constant__ CUtensorMap tm_x0, const __grid_constant__ CUtensorMap tm_x1, const NKDev p) {
+               const __grid_constant__ CUtensorMap tm_x0, const NKDev p) {
   extern __shared__ unsigned char smem_raw[];
   constexpr int NW = EPI == EPI_SWIGLU ? 2 : 1;
   unsigned char* stages = align_1024(smem_raw);
-  const int w_tile = p.rows * 128, x_tile = p.Mpad * 128;  // bytes per 64-wide k chunk
-  const int stage_bytes = p.cps * (NW * w_tile + p.n_b * x_tile);
+  const int nb_rows = p.n_b * p.Mpad;                      // N of the MMA
+  const int w_tile = p.rows * 128, x_tile = nb_rows * 128;  // bytes per 64-wide k chunk
+  const int stage_bytes = p.cps * (NW * w_tile + x_tile);
   UmBarriers* bars = reinterpret_cast<UmBarriers*>(stages + (size_t)p.stages * stage_bytes + UM_TILE_SPAN);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -99,7 +100,11 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
 
   const int row0 = blockIdx.x * p.rows;
-  const int n_iter = p.K / 64 / p.cps;
+  // this CTA's K slice, in 64-wide chunks (cps == 1 whenever K is split)
+  const int chunks = p.K / 64;
+  const int ch0 = (int)(((long long)chunks * blockIdx.y) / p.ksplit);
+  const int ch1 = (int)(((long long)chunks * (blockIdx.y + 1)) / p.ksplit);
+  const int n_iter = (ch1 - ch0) / p.cps;
 
   if (warp == 4) {
     // ------------------------------ TMA producer -----------------------------
@@ -112,14 +117,13 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
       for (int it = 0; it < pre; ++it) {
         unsigned char* st = stages + (size_t)it * stage_bytes;
         mbar_expect_tx(&bars->full[it], stage_bytes);
-        tma_load_3d(st, &tm_w0, 0, row0, it * p.cps, &bars->full[it]);
-        if (NW == 2) tma_load_3d(st + p.cps * w_tile, &tm_w1, 0, row0, it * p.cps, &bars->full[it]);
+        tma_load_3d(st, &tm_w0, 0, row0, ch0 + it * p.cps, &bars->full[it]);
+        if (NW == 2) tma_load_3d(st + p.cps * w_tile, &tm_w1, 0, row0, ch0 + it * p.cps, &bars->full[it]);
       }
       pdl_wait();
       for (int it = 0; it < pre; ++it) {
         unsigned char* xs = stages + (size_t)it * stage_bytes + NW * p.cps * w_tile;
-        tma_load_3d(xs, &tm_x0, 0, 0, it * p.cps, &bars->full[it]);
-        if (p.n_b == 2) tma_load_3d(xs + p.cps * x_tile, &tm_x1, 0, 0, it * p.cps, &bars->full[it]);
+        tma_load_3d(xs, &tm_x0, 0, 0, ch0 + it * p.cps, &bars->full[it]);
       }
       for (int it = pre; it < n_iter; ++it) {
         const int s = it % p.stages;
@@ -127,17 +131,16 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
         if (!mbar_wait(&bars->empty[s], ph ^ 1, p.status)) break;
         unsigned char* st = stages + (size_t)s * stage_bytes;
         mbar_expect_tx(&bars->full[s], stage_bytes);
-        tma_load_3d(st, &tm_w0, 0, row0, it * p.cps, &bars->full[s]);
-        if (NW == 2) tma_load_3d(st + p.cps * w_tile, &tm_w1, 0, row0, it * p.cps, &bars->full[s]);
+        tma_load_3d(st, &tm_w0, 0, row0, ch0 + it * p.cps, &bars->full[s]);
+        if (NW == 2) tma_load_3d(st + p.cps * w_tile, &tm_w1, 0, row0, ch0 + it * p.cps, &bars->full[s]);
         unsigned char* xs = st + NW * p.cps * w_tile;
-        tma_load_3d(xs, &tm_x0, 0, 0, it * p.cps, &bars->full[s]);
-        if (p.n_b == 2) tma_load_3d(xs + p.cps * x_tile, &tm_x1, 0, 0, it * p.cps, &bars->full[s]);
+        tma_load_3d(xs, &tm_x0, 0, 0, ch0 + it * p.cps, &bars->full[s]);
       }
     }
   } else if (warp == 5) {
     // ------------------------------- MMA issuer ------------------------------
     // The mbarrier wait orders the TMA writes before the MMA reads; no tcgen05 fence is needed per stage.
-    const uint32_t idesc = umma_idesc_bf16_m128(p.Mpad, 0, 0);
+    const uint32_t idesc = umma_idesc_bf16_m128(nb_rows, 0, 0);
     bool acc = false, ok = true;
     for (int it = 0; it < n_iter; ++it) {
       const int s = it % p.stages;
@@ -154,14 +157,9 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
           const uint64_t a0 = a_base + (uint64_t)((c * w_tile + ks * 32) >> 4);
           const uint64_t a1 = a_base + (uint64_t)(((p.cps + c) * w_tile + ks * 32) >> 4);
           const uint64_t b0 = b_base + (uint64_t)((c * x_tile + ks * 32) >> 4);
-          const uint64_t b1 = b_base + (uint64_t)(((p.cps + c) * x_tile + ks * 32) >> 4);
           if (elect_one()) {
             umma_bf16(tmem, a0, b0, idesc, acc);
-            if (p.n_b == 2) umma_bf16(tmem, a0, b1, idesc, true);
-            if (NW == 2) {
-              umma_bf16(tmem + p.Mpad, a1, b0, idesc, acc);
-              if (p.n_b == 2) umma_bf16(tmem + p.Mpad, a1, b1, idesc, true);
-            }
+            if (NW == 2) umma_bf16(tmem + nb_rows, a1, b0, idesc, acc);
           }
           acc = true;
         }
@@ -182,25 +180,27 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
       for (int c0 = 0; c0 < p.Mpad && ok; c0 += 16) {
         float v[16], u[16];
         tmem_ld16(tl + c0, v);
-        if (NW == 2) tmem_ld16(tl + p.Mpad + c0, u);
+        if (NW == 2) tmem_ld16(tl + nb_rows + c0, u);
+        if (p.n_b == 2) {  // high-part and low-part products
+          float w2[16];
+          tmem_ld16(tl + p.Mpad + c0, w2);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] += w2[i];
+        }
         if (valid) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const int m = c0 + i;
             if (m < p.M) {
-              const float sc = p.row_scale ? p.row_scale[m] : 1.0f;
               const size_t o = (size_t)m * p.N + n;
               if (EPI == EPI_SWIGLU) {
+                const float sc = p.row_scale ? p.row_scale[m] : 1.0f;
                 const float gg = v[i] * sc, uu = u[i] * sc;
                 p.out0[o] = gg;
                 p.out1[o] = uu;
                 p.out2[o] = (gg / (1.0f + expf(-gg))) * uu;
-              } else if (EPI == EPI_RESIDUAL) {
-                const float res = p.resid_f32 ? static_cast<const float*>(p.resid)[o]
-                                              : bf2f(static_cast<const uint16_t*>(p.resid)[o]);
-                p.out0[o] = v[i] * sc + res;
               } else {
-                p.out0[o] = v[i] * sc;
+                p.out0[(size_t)blockIdx.y * p.M * p.N + o] = v[i];
               }
             }
           }
@@ -230,8 +230,7 @@ __device__ __forceinline__ bool block_live(const int32_t* live, int jb, int gran
 }
 
 __global__ void __launch_bounds__(UM_THREADS, 1)
-umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_hi,
-                 const __grid_constant__ CUtensorMap tm_lo, const DownDev p) {
+umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_t, const DownDev p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* stages = align_1024(smem_raw);
   const int t_tile = p.Mpad * 128;
@@ -274,12 +273,11 @@ umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
         unsigned char* st = stages + (size_t)s * stage_bytes;
         mbar_expect_tx(&bars->full[s], stage_bytes);
         tma_load_3d(st, &tm_w, 0, jb * 64, slab * 2, &bars->full[s]);
-        tma_load_2d(st + UM_TILE_SPAN, &tm_hi, jb * 64, 0, &bars->full[s]);
-        tma_load_2d(st + UM_TILE_SPAN + t_tile, &tm_lo, jb * 64, 0, &bars->full[s]);
+        tma_load_2d(st + UM_TILE_SPAN, &tm_t, jb * 64, 0, &bars->full[s]);  // high rows then low rows
       }
     }
   } else if (warp == 5) {
-    const uint32_t idesc = umma_idesc_bf16_m128(p.Mpad, 1, 0);
+    const uint32_t idesc = umma_idesc_bf16_m128(2 * p.Mpad, 1, 0);
     bool acc = false, ok = true;
     int it = 0;
     for (int jb = jb0; jb < jb1; ++jb) {
@@ -292,14 +290,11 @@ umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
       const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
       // weight tile: two 64-column blocks of [64 channels][128 bytes]; 16 channels = two 8-row groups
       const uint64_t a_base = umma_smem_desc(st, 8192, 1024);
-      const uint64_t h_base = umma_smem_desc(st + UM_TILE_SPAN, 16, 1024);
-      const uint64_t l_base = umma_smem_desc(st + UM_TILE_SPAN + t_tile, 16, 1024);
+      const uint64_t t_base = umma_smem_desc(st + UM_TILE_SPAN, 16, 1024);  // [2 Mpad rows][64 channels]
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks) {
-        if (elect_one()) {
-          umma_bf16(tmem, a_base + (uint64_t)((ks * 2048) >> 4), h_base + (uint64_t)((ks * 32) >> 4), idesc, acc);
-          umma_bf16(tmem, a_base + (uint64_t)((ks * 2048) >> 4), l_base + (uint64_t)((ks * 32) >> 4), idesc, true);
-        }
+        if (elect_one())
+          umma_bf16(tmem, a_base + (uint64_t)((ks * 2048) >> 4), t_base + (uint64_t)((ks * 32) >> 4), idesc, acc);
         acc = true;
       }
       if (elect_one()) umma_commit(&bars->empty[s]);
@@ -321,7 +316,11 @@ umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
     for (int c0 = 0; c0 < p.Mpad && ok; c0 += 16) {
       float v[16];
       if (any) {
+        float w2[16];
         tmem_ld16(tl + c0, v);
+        tmem_ld16(tl + p.Mpad + c0, w2);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] += w2[i];
       } else {
 #pragma unroll
         for (int i = 0; i < 16; ++i) v[i] = 0.f;
@@ -443,48 +442,79 @@ int round_mpad(int M) {
 // ============================================================================
 // launchers
 // ============================================================================
+// Split-K geometry of the EPI_PARTIAL projections: full 128-row weight tiles (so that one TMA box and
+// one MMA cover as many weight bytes as possible) and as many K slices as it takes to give every SM a CTA.
+static void nk_partial_geometry(int N, int K, int* rows, int* tiles, int* ksplit) {
+  int r = (N + 7) / 8 * 8;
+  if (r > 128) r = 128;
+  const int t = (N + r - 1) / r;
+  const int chunks = K / 64;
+  int z = sm_count() / t;
+  if (z > chunks) z = chunks;
+  if (z > NK_MAX_KSPLIT) z = NK_MAX_KSPLIT;
+  if (z < 1) z = 1;
+  *rows = r;
+  *tiles = t;
+  *ksplit = z;
+}
+
+int nk_ksplit(int N, int K) {
+  int rows, tiles, z;
+  nk_partial_geometry(N, K, &rows, &tiles, &z);
+  return z;
+}
+
 void launch_gemm_nk(const GemmNK& g, GemmEpilogue epi, cudaStream_t st) {
   const int nw = epi == EPI_SWIGLU ? 2 : 1;
   NKDev d;
   memset(&d, 0, sizeof(d));
   d.M = g.M; d.Mpad = round_mpad(g.M); d.K = g.K; d.N = g.N;
   d.n_b = g.a_lo ? 2 : 1;
-  const int sms = sm_count();
-  int rows = ((g.N + sms - 1) / sms + 7) / 8 * 8;
-  if (rows > 128) rows = 128;
-  d.rows = rows;
-  const int chunk_bytes = 128 * (nw * rows + d.n_b * d.Mpad);
+  if (g.a_lo && static_cast<const char*>(g.a_lo) != static_cast<const char*>(g.a_hi) + (size_t)d.Mpad * g.K * 2) {
+    record_cuda_error(cudaErrorInvalidValue, "split activation operand must be contiguous (high rows, then low rows)");
+    return;
+  }
   const int chunks = g.K / 64;
-  int cps = 4;
+  int rows, tiles, ksplit = 1;
+  if (epi == EPI_PARTIAL) {
+    nk_partial_geometry(g.N, g.K, &rows, &tiles, &ksplit);
+  } else {
+    // whole K per CTA, one wave of CTAs: `rows` channels (a gate and an up row each) per CTA
+    const int sms = sm_count();
+    rows = ((g.N + sms - 1) / sms + 7) / 8 * 8;
+    if (rows > 128) rows = 128;
+    tiles = (g.N + rows - 1) / rows;
+  }
+  d.rows = rows;
+  d.ksplit = ksplit;
+  const int chunk_bytes = 128 * (nw * rows + d.n_b * d.Mpad);
+  int cps = ksplit > 1 ? 1 : 4;
   while (cps > 1 && (cps * chunk_bytes > 36 * 1024 || chunks % cps)) cps >>= 1;
   d.cps = cps;
   const int stage_bytes = cps * chunk_bytes;
+  const int iters = (chunks / ksplit + (chunks % ksplit ? 1 : 0)) / cps;  // of the longest slice
   int stages = UM_SMEM_BUDGET / stage_bytes;
   if (stages > UM_MAX_STAGES) stages = UM_MAX_STAGES;
-  if (stages > chunks / cps) stages = chunks / cps;
+  if (stages > iters) stages = iters;
   if (stages < 1) stages = 1;
   d.stages = stages;
-  d.tmem_cols = pow2_cols(nw * d.Mpad);
-  d.row_scale = g.row_scale; d.resid = g.resid; d.resid_f32 = g.resid_f32;
+  d.tmem_cols = pow2_cols(nw * d.n_b * d.Mpad);
+  d.row_scale = g.row_scale;
   d.out0 = g.out0; d.out1 = g.out1; d.out2 = g.out2; d.status = g.status;
 
-  CUtensorMap w0, w1, x0, x1;
+  CUtensorMap w0, w1, x0;
   bool ok = kmajor_map(&w0, g.w0, g.N, g.K, rows, cps);
   ok = ok && kmajor_map(&w1, nw == 2 ? g.w1 : g.w0, g.N, g.K, rows, cps);
-  ok = ok && kmajor_map(&x0, g.a_hi, d.Mpad, g.K, d.Mpad, cps);
-  ok = ok && kmajor_map(&x1, g.a_lo ? g.a_lo : g.a_hi, d.Mpad, g.K, d.Mpad, cps);
+  ok = ok && kmajor_map(&x0, g.a_hi, d.n_b * d.Mpad, g.K, d.n_b * d.Mpad, cps);
   if (!ok) return;
   const int smem = 1024 + stages * stage_bytes + UM_TILE_SPAN + (int)sizeof(UmBarriers);
-  const dim3 grid((g.N + rows - 1) / rows);
+  const dim3 grid(tiles, ksplit);
   if (epi == EPI_SWIGLU) {
     ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_nk_kernel<EPI_SWIGLU>), smem);
-    SOL_LAUNCH("gemm_gate_up_swiglu", umma_nk_kernel<EPI_SWIGLU>, grid, dim3(UM_THREADS), smem, st, w0, w1, x0, x1, d);
-  } else if (epi == EPI_RESIDUAL) {
-    ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_nk_kernel<EPI_RESIDUAL>), smem);
-    SOL_LAUNCH("gemm_out_proj", umma_nk_kernel<EPI_RESIDUAL>, grid, dim3(UM_THREADS), smem, st, w0, w1, x0, x1, d);
+    SOL_LAUNCH("gemm_gate_up_swiglu", umma_nk_kernel<EPI_SWIGLU>, grid, dim3(UM_THREADS), smem, st, w0, w1, x0, d);
   } else {
-    ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_nk_kernel<EPI_SCALE>), smem);
-    SOL_LAUNCH("gemm_qkv", umma_nk_kernel<EPI_SCALE>, grid, dim3(UM_THREADS), smem, st, w0, w1, x0, x1, d);
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_nk_kernel<EPI_PARTIAL>), smem);
+    SOL_LAUNCH(g.name ? g.name : "gemm_partial", umma_nk_kernel<EPI_PARTIAL>, grid, dim3(UM_THREADS), smem, st, w0, w1, x0, d);
   }
 }
 
@@ -506,26 +536,29 @@ void launch_gemm_down(const GemmDown& g, cudaStream_t st) {
   int stages = UM_SMEM_BUDGET / stage_bytes;
   if (stages > UM_MAX_STAGES) stages = UM_MAX_STAGES;
   d.stages = stages;
-  d.tmem_cols = pow2_cols(d.Mpad);
+  d.tmem_cols = pow2_cols(2 * d.Mpad);
   d.live = g.live; d.partial = g.partial; d.status = g.status;
 
-  CUtensorMap w, hi, lo;
+  if (static_cast<const char*>(g.t_lo) != static_cast<const char*>(g.t_hi) + (size_t)d.Mpad * g.ff * 2) {
+    record_cuda_error(cudaErrorInvalidValue, "split activation operand must be contiguous (high rows, then low rows)");
+    return;
+  }
+  CUtensorMap w, tm;
   // W[ff][d] viewed as (64 columns, ff channels, d/64 column blocks): a box of (64, 64, 2) lands as two
   // [64 channels][64 columns] blocks, the MN-major operand layout for 128 output columns
   const uint64_t wdim[3] = {64, (uint64_t)g.ff, (uint64_t)(g.d / 64)};
   const uint64_t wstride[2] = {(uint64_t)g.d * 2, 128};
   const uint32_t wbox[3] = {64, 64, 2};
   bool ok = tensor_map(&w, g.w, 3, wdim, wstride, wbox);
-  // activations [Mpad][ff]: (ff, Mpad) with a box of (64 channels, Mpad rows); channels past ff read as zero
-  const uint64_t tdim[2] = {(uint64_t)g.ff, (uint64_t)d.Mpad};
+  // activations [2 Mpad][ff] (high rows, then low rows): (ff, 2 Mpad) with a box of (64 channels, all rows); channels past ff read as zero
+  const uint64_t tdim[2] = {(uint64_t)g.ff, (uint64_t)(2 * d.Mpad)};
   const uint64_t tstride[1] = {(uint64_t)g.ff * 2};
-  const uint32_t tbox[2] = {64, (uint32_t)d.Mpad};
-  ok = ok && tensor_map(&hi, g.t_hi, 2, tdim, tstride, tbox);
-  ok = ok && tensor_map(&lo, g.t_lo, 2, tdim, tstride, tbox);
+  const uint32_t tbox[2] = {64, (uint32_t)(2 * d.Mpad)};
+  ok = ok && tensor_map(&tm, g.t_hi, 2, tdim, tstride, tbox);
   if (!ok) return;
   const int smem = 1024 + stages * stage_bytes + (int)sizeof(UmBarriers);
   ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_down_kernel), smem);
-  SOL_LAUNCH("gemm_down_gathered", umma_down_kernel, dim3(g.d / 128, g.chunks), dim3(UM_THREADS), smem, st, w, hi, lo, d);
+  SOL_LAUNCH("gemm_down_gathered", umma_down_kernel, dim3(g.d / 128, g.chunks), dim3(UM_THREADS), smem, st, w, tm, d);
 }
 
 // ============================================================================

@@ -45,24 +45,45 @@ void ensure_dynamic_smem(const void* kernel, int bytes);
 constexpr int MAX_PAGES_PER_SEQ = 768;  // 49152 tokens: the selection kernel keeps one float per token in shared memory
 
 // ---- quantizer / RMSNorm (sol_quant.cu) ------------------------------------
-// One token per CTA.  in: bf16 or float32 [B][d].  gamma == nullptr: no norm.
-// Outputs (each optional): a_op bf16 [B][d] (codes as bf16, or x as bf16 for
-// 16 bits), scale [B], xn float32 [B][d], codes int8 [B][d].
-void launch_norm_quant(const void* in, bool in_f32, const void* gamma_bf16, float eps, const int32_t* bits, int B,
-                       int d, void* a_op, float* scale, float* xn, int8_t* codes, int* status, cudaStream_t st);
+// One token per CTA.  The row is in[B][d] (bf16 or float32) plus, when `part` is given, the ksplit
+// partial sums part[z][B][d] of a split-K projection (the output projection: in is the residual).
+// gamma == nullptr: no norm.  Outputs (each optional): sum_out float32 [B][d] (the row before the
+// norm), a_op bf16 [B][d] (codes as bf16, or x as bf16 for 16 bits), scale [B], xn float32 [B][d],
+// codes int8 [B][d].
+struct NormQuantArgs {
+  const void* in;
+  bool in_f32;
+  const float* part;
+  int ksplit;
+  float* sum_out;
+  const void* gamma_bf16;
+  float eps;
+  const int32_t* bits;
+  int B, d;
+  void* a_op;
+  float* scale;
+  float* xn;
+  int8_t* codes;
+  int* status;
+};
+void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st);
 
 // ---- weight-streaming GEMMs (sol_gemm.cu) ----------------------------------
-enum GemmEpilogue { EPI_SCALE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2 };
+// EPI_PARTIAL: split-K; out0 is [ksplit][M][N] raw partial sums (no scale, no residual), summed by the
+// consumer kernel.  EPI_SWIGLU: whole K per CTA; g, u and t = silu(g) u with the row scale applied.
+enum GemmEpilogue { EPI_PARTIAL = 0, EPI_SWIGLU = 2 };
+// K slices launch_gemm_nk uses for an [N][K] weight matrix in EPI_PARTIAL mode (<= NK_MAX_KSPLIT).
+constexpr int NK_MAX_KSPLIT = 16;
+int nk_ksplit(int N, int K);
 struct GemmNK {
+  const char* name;       // kernel name for the per-kernel timing table
   const void* a_hi;       // bf16 [Mpad][K]
   const void* a_lo;       // bf16 [Mpad][K] or nullptr; the product uses a_hi + a_lo
   const void* w0;         // bf16 [N][K]   (EPI_SWIGLU: gate [ff][K])
   const void* w1;         // EPI_SWIGLU: up [ff][K]
   int M, K, N;            // EPI_SWIGLU: N = ff
-  const float* row_scale; // [M] or nullptr
-  const void* resid;      // EPI_RESIDUAL: [M][N] bf16 or float32
-  int resid_f32;
-  float* out0;            // [M][N]  (EPI_SWIGLU: g)
+  const float* row_scale; // EPI_SWIGLU: [M] or nullptr
+  float* out0;            // EPI_PARTIAL: [ksplit][M][N]; EPI_SWIGLU: g [M][N]
   float* out1;            // EPI_SWIGLU: u
   float* out2;            // EPI_SWIGLU: t = silu(g) * u
   int* status;
@@ -94,8 +115,10 @@ struct AttnArgs {
   const int32_t* r_permille;
   // inputs of the query preparation: either float32 qkv rows [B][ldq] (layer path: rotate q and k,
   // append k and v) or bf16 q [B][Hq][hd] (stand-alone path: no rotation, no append)
-  const float* qkv_f32;
+  const float* qkv_f32;   // [qkv_ksplit][B][ldq] partial sums of the QKV projection
   int ldq;
+  int qkv_ksplit;
+  const float* qkv_scale; // [B] quantizer scale applied to the summed rows
   const void* q_bf16;
   // scratch
   float* q_rot;      // [B][Hq][hd]

@@ -28,7 +28,8 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float* sh) {
 
 template <bool IN_F32>
 __global__ void __launch_bounds__(NQ_THREADS)
-norm_quant_kernel(const void* __restrict__ in, const uint16_t* __restrict__ gamma, float eps,
+norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, int ksplit, size_t part_stride,
+                  float* __restrict__ sum_out, const uint16_t* __restrict__ gamma, float eps,
                   const int32_t* __restrict__ bits, int d, uint16_t* __restrict__ a_op, float* __restrict__ scale,
                   float* __restrict__ xn, int8_t* __restrict__ codes, int* __restrict__ status) {
   __shared__ float sh[NQ_THREADS / 32];
@@ -55,6 +56,19 @@ norm_quant_kernel(const void* __restrict__ in, const uint16_t* __restrict__ gamm
         uint4 w = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(in) + (size_t)row * d)[v];
         x[i][0] = bf16_lo(w.x); x[i][1] = bf16_hi(w.x); x[i][2] = bf16_lo(w.y); x[i][3] = bf16_hi(w.y);
         x[i][4] = bf16_lo(w.z); x[i][5] = bf16_hi(w.z); x[i][6] = bf16_lo(w.w); x[i][7] = bf16_hi(w.w);
+      }
+      if (part != nullptr) {  // partial sums of the projection that produced this row, in slice order
+        for (int z = 0; z < ksplit; ++z) {
+          const float4* q = reinterpret_cast<const float4*>(part + (size_t)z * part_stride + (size_t)row * d) + 2 * v;
+          const float4 a = q[0], b = q[1];
+          x[i][0] += a.x; x[i][1] += a.y; x[i][2] += a.z; x[i][3] += a.w;
+          x[i][4] += b.x; x[i][5] += b.y; x[i][6] += b.z; x[i][7] += b.w;
+        }
+      }
+      if (sum_out != nullptr) {
+        float4* o = reinterpret_cast<float4*>(sum_out + (size_t)row * d) + 2 * v;
+        o[0] = make_float4(x[i][0], x[i][1], x[i][2], x[i][3]);
+        o[1] = make_float4(x[i][4], x[i][5], x[i][6], x[i][7]);
       }
 #pragma unroll
       for (int e = 0; e < NQ_VEC; ++e) ss += x[i][e] * x[i][e];
@@ -141,16 +155,16 @@ norm_quant_kernel(const void* __restrict__ in, const uint16_t* __restrict__ gamm
   }
 }
 
-void launch_norm_quant(const void* in, bool in_f32, const void* gamma_bf16, float eps, const int32_t* bits, int B,
-                       int d, void* a_op, float* scale, float* xn, int8_t* codes, int* status, cudaStream_t st) {
-  if (in_f32)
-    SOL_LAUNCH("norm_quant", norm_quant_kernel<true>, dim3(B), dim3(NQ_THREADS), 0, st, in,
-               static_cast<const uint16_t*>(gamma_bf16), eps, bits, d, static_cast<uint16_t*>(a_op), scale, xn,
-               codes, status);
+void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st) {
+  const size_t stride = (size_t)a.B * a.d;
+  if (a.in_f32)
+    SOL_LAUNCH("norm_quant", norm_quant_kernel<true>, dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit, stride,
+               a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d, static_cast<uint16_t*>(a.a_op),
+               a.scale, a.xn, a.codes, a.status);
   else
-    SOL_LAUNCH("norm_quant", norm_quant_kernel<false>, dim3(B), dim3(NQ_THREADS), 0, st, in,
-               static_cast<const uint16_t*>(gamma_bf16), eps, bits, d, static_cast<uint16_t*>(a_op), scale, xn,
-               codes, status);
+    SOL_LAUNCH("norm_quant", norm_quant_kernel<false>, dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit, stride,
+               a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d, static_cast<uint16_t*>(a.a_op),
+               a.scale, a.xn, a.codes, a.status);
 }
 
 }  // namespace sol

@@ -112,6 +112,8 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
   a.r_permille = r_permille;
   a.qkv_f32 = nullptr;
   a.ldq = 0;
+  a.qkv_ksplit = 0;
+  a.qkv_scale = nullptr;
   a.q_bf16 = q_bf16;
   a.q_rot = reinterpret_cast<float*>(base + L.q_rot);
   a.q_split = base + L.q_split;
