@@ -99,7 +99,7 @@ static int pad_rows(int B) {
 
 struct Layout {
   size_t status, stage_h_in, stage_act, stage_h_out, a_op, scale, qkv, q_rot, q_split, logits, sigma, kept_idx,
-      kept_cnt, part, work_items, work_ctr, attn_hi, attn_lo, attn_f32, h_mid, o_part, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, down_part,
+      kept_cnt, part, work_items, work_ctr, attn_hi, attn_lo, attn_f32, h_mid, o_part, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, ch_sel, ch_cand_val, ch_cand_idx, ch_keep, down_part,
       h_a, h_b, total;
   int splits, chunks, Mpad, Tmax;
 };
@@ -162,6 +162,10 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   L.kept_ch = take(B * ff * 4);
   L.kept_ch_cnt = take((size_t)B * 4);
   L.live = take(ff / 32 * 4);
+  L.ch_sel = take((size_t)B * CH_SEL_WORDS * 4);
+  L.ch_cand_val = take((size_t)B * CH_CAND_CAP * 8);
+  L.ch_cand_idx = take((size_t)B * CH_CAND_CAP * 4);
+  L.ch_keep = take((size_t)B * ff);
   L.down_part = take((size_t)L.chunks * Mpad * d * 4);
   L.h_a = take(B * d * 4);
   L.h_b = take(B * d * 4);
@@ -240,6 +244,7 @@ static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, cons
   gu.out0 = at<float>(ws, L.g);
   gu.out1 = at<float>(ws, L.u);
   gu.out2 = t_trace ? t_trace : at<float>(ws, L.t);
+  gu.sel = at<uint32_t>(ws, L.ch_sel);
   gu.status = status;
   launch_gemm_nk(gu, EPI_SWIGLU, st);
 
@@ -255,7 +260,12 @@ static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, cons
   cs.scale = at<float>(ws, L.scale);
   cs.w_gate = w_gate;
   cs.w_up = w_up;
-  cs.kept_ch = kept_ch ? kept_ch : at<int32_t>(ws, L.kept_ch);
+  cs.sel = at<uint32_t>(ws, L.ch_sel);
+  cs.cand_val = at<double>(ws, L.ch_cand_val);
+  cs.cand_idx = at<int32_t>(ws, L.ch_cand_idx);
+  cs.keep = at<unsigned char>(ws, L.ch_keep);
+  cs.scratch_idx = at<int32_t>(ws, L.kept_ch);
+  cs.kept_ch = kept_ch;
   cs.kept_cnt = kept_ch_cnt ? kept_ch_cnt : at<int32_t>(ws, L.kept_ch_cnt);
   cs.t_hi = at<void>(ws, L.t_hi);
   cs.t_lo = at<void>(ws, L.t_lo);
@@ -335,6 +345,8 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   n2.gamma_bf16 = w.gamma2; n2.eps = s.rms_eps; n2.bits = bits; n2.B = B; n2.d = d;
   n2.a_op = at<void>(ws, L.a_op); n2.scale = scale; n2.xn = tr ? tr->xn2 : nullptr; n2.codes = tr ? tr->codes2 : nullptr;
   n2.status = status;
+  n2.clear = at<uint32_t>(ws, L.ch_sel);
+  n2.clear_words = CH_SEL_WORDS;
   launch_norm_quant(n2, st);
   if (tr && tr->h_mid)
     cudaMemcpyAsync(tr->h_mid, at<float>(ws, L.h_mid), sizeof(float) * B * d, cudaMemcpyDeviceToDevice, st);
@@ -426,6 +438,8 @@ sol_status_t sol_pruned_swiglu_mlp(const sol_shape_t* shape, const void* x_bf16,
   NormQuantArgs n;
   memset(&n, 0, sizeof(n));
   n.in = x_bf16; n.B = B; n.d = shape->d_model; n.a_op = at<void>(ws, L.a_op); n.scale = at<float>(ws, L.scale);
+  n.clear = at<uint32_t>(ws, L.ch_sel);
+  n.clear_words = CH_SEL_WORDS;
   launch_norm_quant(n, st);
   run_mlp(*shape, L, ws, B, w_gate, w_up, w_down_t, p_permille, nullptr, 0, out_bf16, nullptr, nullptr, nullptr,
           kept_ch, kept_ch_cnt, st);

@@ -101,6 +101,22 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   return v;
 }
 
+// ---- histogram of |t| shared by the gate/up epilogue (which fills it) and the channel selection ----
+// 4096 bins: 32 octaves from 2^-24 to 2^8 with 128 steps each (the top mantissa bits); smaller values
+// share bin 0, larger ones bin 4095.  Bin order is value order.
+constexpr int CH_BINS = 4096;
+__device__ __forceinline__ int chan_bin(float a) {  // a >= 0
+  const int b = (int)(__float_as_uint(a) >> 16) - (103 << 7);
+  return min(max(b, 0), CH_BINS - 1);
+}
+__device__ __forceinline__ float chan_bin_lo(int b) {  // smallest value of bin b (0 for bin 0)
+  return b <= 0 ? 0.f : __uint_as_float((uint32_t)(b + (103 << 7)) << 16);
+}
+// Per-token scratch words of the channel selection, cleared by the RMSNorm kernel before the projection:
+// the histogram, then these.
+enum : int { CH_GMAX = CH_BINS, CH_UMAX, CH_N_ABOVE, CH_N_CAND, CH_DONE, CH_FALLBACK, CH_SEL_WORDS = CH_BINS + 8 };
+constexpr int CH_CAND_CAP = 1024;  // exactly re-scored candidates per token before the single-CTA path takes over
+
 // ---- programmatic dependent launch ---------------------------------------------
 // pdl_trigger: the next kernel in the stream may be scheduled from now on (it still waits in
 // pdl_wait for this grid to finish).  pdl_wait: returns once every earlier kernel has completed and

@@ -68,6 +68,7 @@ struct NKDev {
   float* out0;
   float* out1;
   float* out2;
+  uint32_t* sel;
   int* status;
 };
 
@@ -187,21 +188,34 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
 #pragma unroll
           for (int i = 0; i < 16; ++i) v[i] += w2[i];
         }
-        if (valid) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int m = c0 + i;
-            if (m < p.M) {
-              const size_t o = (size_t)m * p.N + n;
-              if (EPI == EPI_SWIGLU) {
-                const float sc = p.row_scale ? p.row_scale[m] : 1.0f;
-                const float gg = v[i] * sc, uu = u[i] * sc;
+        for (int i = 0; i < 16; ++i) {
+          const int m = c0 + i;
+          if (m < p.M) {  // warp-uniform
+            const size_t o = (size_t)m * p.N + n;
+            if (EPI == EPI_SWIGLU) {
+              const float sc = p.row_scale ? p.row_scale[m] : 1.0f;
+              const float gg = v[i] * sc, uu = u[i] * sc;
+              const float tv = (gg / (1.0f + expf(-gg))) * uu;
+              if (valid) {
                 p.out0[o] = gg;
                 p.out1[o] = uu;
-                p.out2[o] = (gg / (1.0f + expf(-gg))) * uu;
-              } else {
-                p.out0[(size_t)blockIdx.y * p.M * p.N + o] = v[i];
+                p.out2[o] = tv;
               }
+              if (p.sel != nullptr) {
+                // what the channel selection needs from all of a token's channels: a histogram of |t|
+                // and the largest |g|, |u| (non-negative floats order like their bit patterns)
+                uint32_t* sel = p.sel + (size_t)m * CH_SEL_WORDS;
+                if (valid) atomicAdd(sel + chan_bin(fabsf(tv)), 1u);
+                const uint32_t gm = __reduce_max_sync(0xffffffffu, valid ? __float_as_uint(fabsf(gg)) : 0u);
+                const uint32_t um = __reduce_max_sync(0xffffffffu, valid ? __float_as_uint(fabsf(uu)) : 0u);
+                if (lane == 0) {
+                  atomicMax(sel + CH_GMAX, gm);
+                  atomicMax(sel + CH_UMAX, um);
+                }
+              }
+            } else if (valid) {
+              p.out0[(size_t)blockIdx.y * p.M * p.N + o] = v[i];
             }
           }
         }
@@ -500,7 +514,7 @@ void launch_gemm_nk(const GemmNK& g, GemmEpilogue epi, cudaStream_t st) {
   d.stages = stages;
   d.tmem_cols = pow2_cols(nw * d.n_b * d.Mpad);
   d.row_scale = g.row_scale;
-  d.out0 = g.out0; d.out1 = g.out1; d.out2 = g.out2; d.status = g.status;
+  d.out0 = g.out0; d.out1 = g.out1; d.out2 = g.out2; d.sel = g.sel; d.status = g.status;
 
   CUtensorMap w0, w1, x0;
   bool ok = kmajor_map(&w0, g.w0, g.N, g.K, rows, cps);

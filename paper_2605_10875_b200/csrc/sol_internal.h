@@ -65,6 +65,8 @@ struct NormQuantArgs {
   float* xn;
   int8_t* codes;
   int* status;
+  uint32_t* clear;   // optional: [B][clear_words] words zeroed, row by row, for the kernels that follow
+  int clear_words;
 };
 void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st);
 
@@ -86,6 +88,7 @@ struct GemmNK {
   float* out0;            // EPI_PARTIAL: [ksplit][M][N]; EPI_SWIGLU: g [M][N]
   float* out1;            // EPI_SWIGLU: u
   float* out2;            // EPI_SWIGLU: t = silu(g) * u
+  uint32_t* sel;          // EPI_SWIGLU: [M][CH_SEL_WORDS] histogram of |t| and max |g|, |u| per token (pre-cleared)
   int* status;
 };
 void launch_gemm_nk(const GemmNK& p, GemmEpilogue epi, cudaStream_t st);
@@ -158,7 +161,12 @@ struct ChannelSelectArgs {
   const float* scale;  // [B]
   const void* w_gate;  // bf16 [ff][d]
   const void* w_up;
-  int32_t* kept_ch;    // [B][ff]
+  uint32_t* sel;       // [B][CH_SEL_WORDS] filled by the gate/up epilogue
+  double* cand_val;    // [B][CH_CAND_CAP]
+  int32_t* cand_idx;   // [B][CH_CAND_CAP]
+  unsigned char* keep; // [B][ff] 1 = kept
+  int32_t* scratch_idx; // [B][ff] scratch of the single-CTA path
+  int32_t* kept_ch;    // optional [B][ff]: ascending list, written only when requested
   int32_t* kept_cnt;   // [B]
   void* t_hi;          // bf16 [Mpad][ff]
   void* t_lo;

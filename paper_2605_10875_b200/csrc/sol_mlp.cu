@@ -2,13 +2,21 @@
 //
 // For token i keep the m = ceil((1 - p_i) * ff) channels with the largest
 // |t_j| = |silu(g_j) * u_j| (the count mirrors the paper's m = ceil(rho * d),
-// "Per-token channel selection", with rho = 1 - p).  One CTA per token: exact
-// k-th largest of the float32 |t| held in registers, then every channel within
-// a small window of the threshold has g_j and u_j recomputed exactly from the
-// weight rows, so the kept set does not depend on float32 rounding.  Emits
-// the ascending kept-channel list, the masked activations as two bf16 parts
-// (hi + lo) for the tensor-core down projection, and the "granule is live"
-// flags that let the down projection skip weight rows nobody keeps.
+// "Per-token channel selection", with rho = 1 - p; ties: lower index).
+//
+// The gate/up projection leaves, per token, a 4096-bin histogram of |t| and
+// the largest |g|, |u|.  channel_select_multi spreads every token over
+// ff/1024 CTAs: each finds the histogram bin that holds the m-th largest |t|,
+// keeps what lies above that bin (by more than the float32 error bound of t),
+// drops what lies below, and recomputes the few channels in between exactly
+// from the weight rows; the last CTA of a token ranks those candidates and
+// patches the kept ones in.  Outputs: the masked activations as two bf16
+// parts (hi + lo) for the tensor-core down projection, a keep mask, and the
+// "granule is live" flags that let the down projection skip weight rows
+// nobody keeps.  A token with more candidates than the list holds (massive
+// ties) is redone by the single-CTA kernel channel_select, which is exact for
+// any input; channel_list turns the mask into the ascending index list when a
+// caller asks for it.
 #include <math.h>
 
 #include "sol_common.cuh"
@@ -27,7 +35,12 @@ struct ChanDev {
   const float* scale;
   const uint16_t* w_gate;
   const uint16_t* w_up;
+  uint32_t* sel;
+  double* cand_val;
+  int32_t* cand_idx;
+  unsigned char* keep;
   int32_t* kept_ch;
+  int32_t* scratch_idx;  // [B][ff] list written by the single-CTA kernel (not an output)
   int32_t* kept_cnt;
   uint16_t* t_hi;
   uint16_t* t_lo;
@@ -56,6 +69,7 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
   const int ff = p.ff, d = p.d;
   pdl_trigger();
   pdl_wait();
+  if (p.sel[(size_t)b * CH_SEL_WORDS + CH_FALLBACK] == 0u) return;  // the multi-CTA kernel settled this token
   const float* tt = p.t + (size_t)b * ff;
   const int m = (int)(((long long)(1000 - p.p_permille[b]) * ff + 999) / 1000);
   const int j0 = tid * KPT;
@@ -221,6 +235,7 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
       hw[e >> 1] |= (uint32_t)hv << 16;
       lw[e >> 1] |= (uint32_t)lv << 16;
     }
+    if (j0 + i < ff) p.keep[(size_t)b * ff + j0 + i] = keep ? 1 : 0;
     if (e == 7 && j0 + i < ff) {
       *reinterpret_cast<uint4*>(th + j0 + i - 7) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
       *reinterpret_cast<uint4*>(tl + j0 + i - 7) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
@@ -230,8 +245,233 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
       any = false;
     }
   };
-  const int total = compact_indices<THREADS, KPT>(klass, emit, mode == 3 ? tie_need : 0, p.kept_ch + (size_t)b * ff, sm);
+  // the index list itself is written by channel_list from the mask; here it goes to the candidate scratch
+  const int total = compact_indices<THREADS, KPT>(klass, emit, mode == 3 ? tie_need : 0, p.scratch_idx + (size_t)b * ff, sm);
   if (tid == 0) p.kept_cnt[b] = total;
+}
+
+// ============================================================================
+// channel_select_multi
+// ============================================================================
+constexpr int CM_THREADS = 256;
+constexpr int CM_SLICE = CM_THREADS * 4;  // channels per CTA
+
+struct ChanMultiSmem {
+  int scan[CM_THREADS / 32];
+  int pick[2];
+  int n_local;
+  int flag;
+  int local_idx[CM_SLICE];
+  double val[CH_CAND_CAP];
+  int idx[CH_CAND_CAP];
+};
+
+__global__ void __launch_bounds__(CM_THREADS) channel_select_multi_kernel(const ChanDev p) {
+  __shared__ ChanMultiSmem sm;
+  const int slice = blockIdx.x, b = blockIdx.y, S = gridDim.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr int WARPS = CM_THREADS / 32;
+  const int ff = p.ff, d = p.d;
+  pdl_trigger();
+  pdl_wait();
+  uint32_t* sel = p.sel + (size_t)b * CH_SEL_WORDS;
+  const int m = (int)(((long long)(1000 - p.p_permille[b]) * ff + 999) / 1000);
+  const int j0 = slice * CM_SLICE + tid * 4;
+  const bool in = j0 < ff;  // ff is a multiple of 4: a thread's group is present or absent as a whole
+  if (tid == 0) sm.n_local = 0;
+
+  // ---- the histogram bin of the m-th largest |t| (every CTA of the token finds the same one) ----
+  float hi_edge = 0.f, lo_edge = 0.f;  // keep at or above hi_edge, drop below lo_edge, exact in between
+  if (m >= ff) {
+    hi_edge = 0.f;  // everything is kept
+    lo_edge = 0.f;
+  } else if (m <= 0) {
+    hi_edge = INFINITY;
+    lo_edge = INFINITY;
+  } else {
+    constexpr int BPT = CH_BINS / CM_THREADS;  // bins per thread, descending
+    int mine = 0;
+#pragma unroll
+    for (int q = 0; q < BPT; ++q) mine += (int)sel[CH_BINS - 1 - tid * BPT - q];
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) sm.scan[warp] = incl;
+    __syncthreads();
+    int before = incl - mine;
+    for (int w = 0; w < warp; ++w) before += sm.scan[w];
+    if (before < m && m <= before + mine) {
+      int a = before;
+      for (int q = 0; q < BPT; ++q) {
+        const int bin = CH_BINS - 1 - tid * BPT - q;
+        const int c = (int)sel[bin];
+        if (m <= a + c) {
+          sm.pick[0] = bin;
+          break;
+        }
+        a += c;
+      }
+    }
+    __syncthreads();
+    const int tb = sm.pick[0];
+    const float gmax = __uint_as_float(sel[CH_GMAX]), umax = __uint_as_float(sel[CH_UMAX]);
+    const float bin_lo = chan_bin_lo(tb), bin_hi = tb >= CH_BINS - 1 ? INFINITY : chan_bin_lo(tb + 1);
+    // error taken for g_j, u_j: the tensor cores add each 16-long slice of the dot product to the running
+    // float32 sum with truncation, so the error grows with the d/16 steps: (d/16) * 2^-24 of the largest
+    // magnitude, and never less than 2^-18 of it; carried into t through |silu'| <= 1.1, |silu(g)| <= |g|
+    const float eps = fmaxf(3.814697265625e-06f, (float)(d / 16) * 5.9604644775390625e-08f) * fmaxf(gmax, umax);
+    const float delta = 2.0f * eps * (1.1f * umax + gmax) + 1e-6f * (tb >= CH_BINS - 1 ? bin_lo : bin_hi);
+    lo_edge = bin_lo - delta;
+    hi_edge = bin_hi + delta;
+  }
+
+  // ---- classify this CTA's channels ----
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (in) v = *reinterpret_cast<const float4*>(p.t + (size_t)b * ff + j0);
+  const float vv[4] = {v.x, v.y, v.z, v.w};
+  uint32_t hw[2] = {0, 0}, lw[2] = {0, 0}, kw = 0;
+  int n_above = 0;
+  bool any = false;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float a = fabsf(vv[e]);
+    if (!in) continue;
+    if (a >= hi_edge) {
+      const uint16_t hv = f2bf(vv[e]);
+      const uint16_t lv = f2bf(vv[e] - bf2f(hv));
+      hw[e >> 1] |= (uint32_t)hv << (16 * (e & 1));
+      lw[e >> 1] |= (uint32_t)lv << (16 * (e & 1));
+      kw |= 1u << (8 * e);
+      ++n_above;
+      any = true;
+    } else if (a >= lo_edge) {
+      sm.local_idx[atomicAdd(&sm.n_local, 1)] = j0 + e;
+    }
+  }
+  if (in) {
+    *reinterpret_cast<uint2*>(p.t_hi + (size_t)b * ff + j0) = make_uint2(hw[0], hw[1]);
+    *reinterpret_cast<uint2*>(p.t_lo + (size_t)b * ff + j0) = make_uint2(lw[0], lw[1]);
+    *reinterpret_cast<uint32_t*>(p.keep + (size_t)b * ff + j0) = kw;
+    if (any) p.live[j0 >> 5] = 1;
+  }
+  n_above = __reduce_add_sync(0xffffffffu, n_above);
+  if (lane == 0 && n_above) atomicAdd(sel + CH_N_ABOVE, (uint32_t)n_above);
+  __syncthreads();
+
+  // ---- exact |t| of the channels in between, from the weight rows ----
+  // g_j = scale * sum_e x_e w_je with x the quantizer codes (or the bf16 row): every product of two bf16
+  // numbers is an exact float32, so the sums are gathered exactly in float pairs
+  const int n_local = sm.n_local;
+  if (n_local > 0) {
+    const double sc = (double)p.scale[b];
+    const uint16_t* x = p.a_op + (size_t)b * d;
+    for (int c = warp; c < n_local; c += WARPS) {
+      const int j = sm.local_idx[c];
+      const uint16_t* wg = p.w_gate + (size_t)j * d;
+      const uint16_t* wu = p.w_up + (size_t)j * d;
+      float gh = 0.f, gl = 0.f, uh = 0.f, ul = 0.f;
+      for (int e0 = lane * 8; e0 < d; e0 += 1024) {  // four 256-wide slices per round, loads before uses
+        uint4 xv[4], gv[4], uv[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const int e = e0 + r * 256;
+          if (e < d) {
+            xv[r] = *reinterpret_cast<const uint4*>(x + e);
+            gv[r] = *reinterpret_cast<const uint4*>(wg + e);
+            uv[r] = *reinterpret_cast<const uint4*>(wu + e);
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          if (e0 + r * 256 >= d) break;
+          const uint32_t xa[4] = {xv[r].x, xv[r].y, xv[r].z, xv[r].w}, ga[4] = {gv[r].x, gv[r].y, gv[r].z, gv[r].w},
+                         ua[4] = {uv[r].x, uv[r].y, uv[r].z, uv[r].w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float x0 = bf16_lo(xa[q]), x1 = bf16_hi(xa[q]);
+            pair_add(gh, gl, __fmul_rn(x0, bf16_lo(ga[q])));
+            pair_add(gh, gl, __fmul_rn(x1, bf16_hi(ga[q])));
+            pair_add(uh, ul, __fmul_rn(x0, bf16_lo(ua[q])));
+            pair_add(uh, ul, __fmul_rn(x1, bf16_hi(ua[q])));
+          }
+        }
+      }
+      const double ag = warp_sum_d((double)gh + (double)gl) * sc;
+      const double au = warp_sum_d((double)uh + (double)ul) * sc;
+      if (lane == 0) {
+        const uint32_t slot = atomicAdd(sel + CH_N_CAND, 1u);
+        if (slot < (uint32_t)CH_CAND_CAP) {
+          p.cand_val[(size_t)b * CH_CAND_CAP + slot] = fabs(ag / (1.0 + exp(-ag)) * au);
+          p.cand_idx[(size_t)b * CH_CAND_CAP + slot] = j;
+        }
+      }
+    }
+  }
+
+  // ---- the last CTA of the token ranks the candidates and patches the kept ones in ----
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) sm.flag = atomicAdd(sel + CH_DONE, 1u) == (uint32_t)(S - 1) ? 1 : 0;
+  __syncthreads();
+  if (!sm.flag) return;
+  __threadfence();
+  const int n_cand = (int)__ldcg(sel + CH_N_CAND);
+  const int need = m - (int)__ldcg(sel + CH_N_ABOVE);
+  if (m >= ff || m <= 0) {
+    if (tid == 0) p.kept_cnt[b] = m >= ff ? ff : 0;
+    return;
+  }
+  if (n_cand > CH_CAND_CAP || need < 0 || need > n_cand) {  // more candidates than the list holds: redo the token
+    if (tid == 0) {
+      sel[CH_FALLBACK] = 1u;
+      atomicAdd(p.status + ST_CH_OVERFLOW, 1);
+    }
+    return;
+  }
+  for (int c = tid; c < n_cand; c += CM_THREADS) {
+    sm.val[c] = __ldcg(p.cand_val + (size_t)b * CH_CAND_CAP + c);
+    sm.idx[c] = __ldcg(p.cand_idx + (size_t)b * CH_CAND_CAP + c);
+  }
+  __syncthreads();
+  for (int c = tid; c < n_cand; c += CM_THREADS) {
+    const double vc = sm.val[c];
+    const int j = sm.idx[c];
+    int rank = 0;
+    for (int o = 0; o < n_cand; ++o) {
+      const double vo = sm.val[o];
+      rank += (vo > vc) || (vo == vc && sm.idx[o] < j);
+    }
+    if (rank < need) {
+      const float tv = p.t[(size_t)b * ff + j];
+      const uint16_t hv = f2bf(tv);
+      p.t_hi[(size_t)b * ff + j] = hv;
+      p.t_lo[(size_t)b * ff + j] = f2bf(tv - bf2f(hv));
+      p.keep[(size_t)b * ff + j] = 1;
+      p.live[j >> 5] = 1;
+    }
+  }
+  if (tid == 0) {
+    p.kept_cnt[b] = m;
+    atomicAdd(p.status + ST_CH_REFINED, n_cand);
+  }
+}
+
+// ============================================================================
+// channel_list: keep mask -> ascending index list (only when a caller asks for the list)
+// ============================================================================
+template <int THREADS, int KPT>
+__global__ void __launch_bounds__(THREADS) channel_list_kernel(const unsigned char* __restrict__ keep, int ff,
+                                                               int32_t* __restrict__ kept_ch) {
+  __shared__ SelectSmem sm;
+  pdl_trigger();
+  pdl_wait();
+  const int b = blockIdx.x, j0 = threadIdx.x * KPT;
+  const unsigned char* k = keep + (size_t)b * ff;
+  auto klass = [&](int i) -> int { return (j0 + i < ff && k[j0 + i]) ? 2 : 0; };
+  compact_indices<THREADS, KPT>(klass, [](int, bool) {}, 0, kept_ch + (size_t)b * ff, sm);
 }
 
 void launch_channel_select(const ChannelSelectArgs& a, cudaStream_t st) {
@@ -239,15 +479,24 @@ void launch_channel_select(const ChannelSelectArgs& a, cudaStream_t st) {
   c.d = a.d; c.ff = a.ff; c.p_permille = a.p_permille; c.g = a.g; c.u = a.u; c.t = a.t;
   c.a_op = static_cast<const uint16_t*>(a.a_op); c.scale = a.scale;
   c.w_gate = static_cast<const uint16_t*>(a.w_gate); c.w_up = static_cast<const uint16_t*>(a.w_up);
-  c.kept_ch = a.kept_ch; c.kept_cnt = a.kept_cnt;
+  c.sel = a.sel; c.cand_val = a.cand_val; c.cand_idx = a.cand_idx; c.keep = a.keep;
+  c.kept_ch = a.kept_ch; c.scratch_idx = a.scratch_idx; c.kept_cnt = a.kept_cnt;
   c.t_hi = static_cast<uint16_t*>(a.t_hi); c.t_lo = static_cast<uint16_t*>(a.t_lo);
   c.live = a.live; c.status = a.status;
+  const dim3 mgrid((a.ff + CM_SLICE - 1) / CM_SLICE, a.B);
+  SOL_LAUNCH("channel_select", channel_select_multi_kernel, mgrid, dim3(CM_THREADS), 0, st, c);
   const dim3 grid(a.B);
-  if (a.ff <= 2048) SOL_LAUNCH("channel_select", (channel_select_kernel<256, 8>), grid, dim3(256), 0, st, c);
-  else if (a.ff <= 8192) SOL_LAUNCH("channel_select", (channel_select_kernel<512, 16>), grid, dim3(512), 0, st, c);
-  else if (a.ff <= 16384) SOL_LAUNCH("channel_select", (channel_select_kernel<1024, 16>), grid, dim3(1024), 0, st, c);
-  else if (a.ff <= 32768) SOL_LAUNCH("channel_select", (channel_select_kernel<1024, 32>), grid, dim3(1024), 0, st, c);
-  else SOL_LAUNCH("channel_select", (channel_select_kernel<1024, 48>), grid, dim3(1024), 0, st, c);
+  // tokens the multi-CTA kernel handed over (it sets their flag); every other CTA leaves at once
+  if (a.ff <= 2048) SOL_LAUNCH("channel_select_exact", (channel_select_kernel<256, 8>), grid, dim3(256), 0, st, c);
+  else if (a.ff <= 8192) SOL_LAUNCH("channel_select_exact", (channel_select_kernel<512, 16>), grid, dim3(512), 0, st, c);
+  else if (a.ff <= 16384) SOL_LAUNCH("channel_select_exact", (channel_select_kernel<1024, 16>), grid, dim3(1024), 0, st, c);
+  else if (a.ff <= 32768) SOL_LAUNCH("channel_select_exact", (channel_select_kernel<1024, 32>), grid, dim3(1024), 0, st, c);
+  else SOL_LAUNCH("channel_select_exact", (channel_select_kernel<1024, 48>), grid, dim3(1024), 0, st, c);
+  if (a.kept_ch != nullptr) {
+    if (a.ff <= 4096) SOL_LAUNCH("channel_list", (channel_list_kernel<256, 16>), grid, dim3(256), 0, st, a.keep, a.ff, a.kept_ch);
+    else if (a.ff <= 16384) SOL_LAUNCH("channel_list", (channel_list_kernel<1024, 16>), grid, dim3(1024), 0, st, a.keep, a.ff, a.kept_ch);
+    else SOL_LAUNCH("channel_list", (channel_list_kernel<1024, 48>), grid, dim3(1024), 0, st, a.keep, a.ff, a.kept_ch);
+  }
 }
 
 }  // namespace sol

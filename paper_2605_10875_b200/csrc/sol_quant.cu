@@ -31,11 +31,14 @@ __global__ void __launch_bounds__(NQ_THREADS)
 norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, int ksplit, size_t part_stride,
                   float* __restrict__ sum_out, const uint16_t* __restrict__ gamma, float eps,
                   const int32_t* __restrict__ bits, int d, uint16_t* __restrict__ a_op, float* __restrict__ scale,
-                  float* __restrict__ xn, int8_t* __restrict__ codes, int* __restrict__ status) {
+                  float* __restrict__ xn, int8_t* __restrict__ codes, int* __restrict__ status,
+                  uint32_t* __restrict__ clear, int clear_words) {
   __shared__ float sh[NQ_THREADS / 32];
   pdl_trigger();
   pdl_wait();
   const int row = blockIdx.x;
+  if (clear != nullptr)  // this token's scratch of the kernels that follow
+    for (int i = threadIdx.x; i < clear_words; i += NQ_THREADS) clear[(size_t)row * clear_words + i] = 0u;
   const int nvec = d / NQ_VEC;
   float x[NQ_MAX_PER_THREAD][NQ_VEC];
 
@@ -160,11 +163,11 @@ void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st) {
   if (a.in_f32)
     SOL_LAUNCH("norm_quant", norm_quant_kernel<true>, dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit, stride,
                a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d, static_cast<uint16_t*>(a.a_op),
-               a.scale, a.xn, a.codes, a.status);
+               a.scale, a.xn, a.codes, a.status, a.clear, a.clear_words);
   else
     SOL_LAUNCH("norm_quant", norm_quant_kernel<false>, dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit, stride,
                a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d, static_cast<uint16_t*>(a.a_op),
-               a.scale, a.xn, a.codes, a.status);
+               a.scale, a.xn, a.codes, a.status, a.clear, a.clear_words);
 }
 
 }  // namespace sol
