@@ -193,13 +193,15 @@ def test_mlp_llama8b_shape():
 # ------------------------------------------------------------------ layer ---
 
 
-def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1):
+def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1, sample=None):
     """Runs one layer on the GPU with every tap, then checks each stage against
     the oracle's stage applied to the inputs the GPU stage really saw, and the
     whole layer against the oracle's own layer.  A float32-vs-float64 difference
     of one ulp upstream may legally flip a quantizer code or a selection that
     sits exactly on a boundary; when that happened the end-to-end comparison is
-    reported but not asserted (the chain of stage checks still covers it)."""
+    reported but not asserted (the chain of stage checks still covers it).
+    `sample`: the GPU runs the whole batch, the oracle only these sequences
+    (full-size workloads, where the oracle cannot afford every sequence)."""
     shape, oshape = H.make_shapes(cfg, n_sink, n_window)
     B = len(seq_lens)
     seq_lens = np.asarray(seq_lens, np.int32)
@@ -212,10 +214,18 @@ def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1):
     assert st[0] == 0 and st[1] == 0 and st[2] == 0, st
     ow = H.oracle_weights(w)
     tab = np.where(table < 0, 0, table)
+    k_gpu, v_gpu = H.host_u16(kv.k_pool), H.host_u16(kv.v_pool)
+    assert (k_gpu != k_pool).sum() <= B * Hkv * hd  # nothing but the appended rows changed
+    if sample is not None:  # from here on only the sampled sequences
+        idx = np.asarray(sample)
+        taps = {key: val[idx] for key, val in taps.items()}
+        out, h_in, seq_lens, tab = out[idx], h_in[idx], seq_lens[idx], tab[idx]
+        r, p, b = np.asarray(r)[idx], np.asarray(p)[idx], np.asarray(b)[idx]
+        B = len(idx)
     h64 = O.bf16_to_f64(h_in)
 
-    # the oracle's own layer
-    okv = O.PagedKV(k_pool.copy(), v_pool.copy(), tab, seq_lens)
+    # the oracle's own layer (on the pools as generated; the GPU's copies were fetched above)
+    okv = O.PagedKV(k_pool, v_pool, tab, seq_lens)
     out_o, tr = O.decode_layer(oshape, ow, okv, h64, r, p, b)
 
     # stage 1: RMSNorm (float32 on the GPU) and quantizer (bit-exact on the GPU's own normalised row)
@@ -229,7 +239,6 @@ def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1):
     q_ref = np.stack([O.rope_rotate(qkv[i, : Hq * hd].reshape(Hq, hd), int(seq_lens[i]) - 1, oshape.rope_theta)
                       for i in range(B)])
     assert np.allclose(taps["q_rot"], q_ref, rtol=0, atol=1e-5 * max(1.0, np.abs(q_ref).max())), "q_rot"
-    k_gpu, v_gpu = H.host_u16(kv.k_pool), H.host_u16(kv.v_pool)
     # float32 accumulation of a K-long dot product: error taken as 16 u sum|x_k w_k| with u = 2^-24
     # (the worst case is K u sum|x_k w_k|); it matters only for outputs that nearly cancel to zero
     acc_tol = 2.0 ** -20 * (np.abs(x_hat1) @ np.abs(O.bf16_to_f64(w.w_qkv)).T)
@@ -244,7 +253,6 @@ def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1):
         for got, want, tol in ((k_gpu[pg, :, slot], k_ref, k_tol), (v_gpu[pg, :, slot], v_ref, v_tol)):
             # the appended row is the bf16 nearest to the float32 value: within one bf16 step of the float64 one
             assert np.all(np.abs(O.bf16_to_f64(got) - want) <= np.abs(want) * 2.0 ** -8 * 1.01 + tol + 1e-6), "append"
-    assert (k_gpu != k_pool).sum() <= B * Hkv * hd  # nothing but the appended rows changed
     # stage 3: token selection and attention on the GPU's own queries and cache
     gkv = O.PagedKV(k_gpu, v_gpu, tab, seq_lens)
     attn_o, kept_o, sigma = O.sparse_decode_attn(oshape, taps["q_rot"].astype(np.float64), gkv, r)
