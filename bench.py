@@ -35,6 +35,8 @@ UNIT = "steps/s"
 HBM_SPEC_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 ROTATE = 4  # distinct copies of weights + cache, cycled so that no step finds its inputs in L2 (--rotate)
+SERVE_STEPS = 64   # ragged serving workload: consecutive steps that append before the contexts start over
+SERVE_REDRAW = 16  # ... and steps between two draws of the per-sequence actions
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
 # the ncu capture summarised under profiles/, keyed by (workload, kernel); absent -> null.
@@ -151,14 +153,27 @@ class Replica:
 
         self.torch, self.sol, self.cfg, self.device = torch, sol, cfg, device
         self.B, self.L = cfg["batch"], cfg["layers"]
+        # the ragged serving workload runs consecutive steps that append: contexts grow by one token per
+        # step over a cycle of SERVE_STEPS steps and the actions are redrawn every SERVE_REDRAW steps
+        self.serving = cfg.get("context") is None
+        self.cycle = SERVE_STEPS if self.serving else 1
         self.seq_lens = synth.make_contexts(cfg, seed)
+        if self.serving:
+            self.seq_lens = np.maximum(self.seq_lens - (self.cycle - 1), 1).astype(np.int32)
         self.shape = sol.make_shape(cfg["d_model"], cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"], cfg["d_ff"],
                                     64, synth.RMS_EPS, cfg.get("rope_theta", 0.0), 0, 1)
-        table, n_pages = synth.make_page_table(self.seq_lens, cfg.get("shuffle_pages", True), seed)
+        table, n_pages = synth.make_page_table(self.seq_lens, cfg.get("shuffle_pages", True), seed,
+                                               spare_tokens=self.cycle - 1)
         self.max_pages, self.n_pages = table.shape[1], n_pages
         self.table = self._i32(np.where(table < 0, 0, table))
-        self.lens_dev = self._i32(self.seq_lens)
+        self.lens_dev = [self._i32(self.seq_lens + j) for j in range(self.cycle)]
         names = ("w_qkv", "w_o", "w_gate", "w_up", "w_down_t", "gamma1", "gamma2")
+        # enough distinct copies of weights + cache that no step finds its inputs in the 126 MB L2; one
+        # copy of a multi-GB workload is already far larger than L2
+        hkv, hd, d, ff = cfg["n_kv_heads"], cfg["head_dim"], cfg["d_model"], cfg["d_ff"]
+        copy_bytes = self.L * (n_pages * hkv * 64 * hd * 4 + (3 * ff * d + 2 * d * (cfg["n_q_heads"] + hkv) * hd) * 2)
+        self.rotate = ROTATE if copy_bytes < (1 << 30) else 1
+        self.copy_mb = int(copy_bytes / 1e6)
         self.weights, self.kvs, self._keep = [], [], []
         for l in range(self.L):
             w = synth.make_layer_weights(cfg, seed, l)
@@ -166,12 +181,13 @@ class Replica:
             k, v = synth.make_kv_pool(cfg, n_pages, seed, l)
             base_kv = [self._bf16(k), self._bf16(v)]
             per_copy_w, per_copy_kv = [], []
-            for c in range(ROTATE):
+            for c in range(self.rotate):
                 ws_ = base_w if c == 0 else [t.clone() for t in base_w]
                 kv_ = base_kv if c == 0 else [t.clone() for t in base_kv]
                 self._keep += ws_ + kv_
                 per_copy_w.append(sol.make_weights(*ws_))
-                per_copy_kv.append(sol.make_kv(kv_[0], kv_[1], self.table, self.lens_dev, self.max_pages, n_pages))
+                per_copy_kv.append([sol.make_kv(kv_[0], kv_[1], self.table, self.lens_dev[j], self.max_pages, n_pages)
+                                    for j in range(self.cycle)])
             self.weights.append(per_copy_w)
             self.kvs.append(per_copy_kv)
         self.ws_bytes = sol.workspace_bytes(self.shape, self.B, self.max_pages)
@@ -183,7 +199,7 @@ class Replica:
         pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
         self.h_in_host = pin(synth.make_hidden(cfg, seed).view(np.int16))
         self.h_out_host = torch.zeros((self.B, cfg["d_model"]), dtype=torch.int16).pin_memory()
-        self.lens_host = pin(self.seq_lens.astype(np.int32))
+        self.lens_host = [pin((self.seq_lens + j).astype(np.int32)) for j in range(self.cycle)]
         torch.cuda.synchronize()
 
     def _bf16(self, u16):
@@ -193,22 +209,31 @@ class Replica:
     def _i32(self, a):
         return self.torch.from_numpy(np.ascontiguousarray(np.asarray(a, np.int32))).to(self.device)
 
-    def set_actions(self, r, p, b):
-        self.r_np, self.p_np, self.b_np = [np.asarray(x, np.int32) for x in (r, p, b)]
-        self.r, self.p, self.b = self._i32(r), self._i32(p), self._i32(b)
+    def set_actions(self, r, p, b, redraws=None):
+        """redraws: further (r, p, b) sets the serving workload switches to every SERVE_REDRAW steps."""
         pin = lambda a: self.torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
-        self.r_host, self.p_host, self.b_host = pin(self.r_np), pin(self.p_np), pin(self.b_np)
+        self.r_np, self.p_np, self.b_np = [np.asarray(x, np.int32) for x in (r, p, b)]
+        self.acts, self.acts_host = [], []
+        for (rr, pp, bb) in [(r, p, b)] + list(redraws or []):
+            self.acts.append((self._i32(rr), self._i32(pp), self._i32(bb)))
+            self.acts_host.append(tuple(pin(np.asarray(x, np.int32)) for x in (rr, pp, bb)))
+        self.r, self.p, self.b = self.acts[0]
+
+    def _phase(self, i):
+        j = i % self.cycle
+        return i % self.rotate, j, (j // SERVE_REDRAW) % len(self.acts)
 
     def step(self, i):
-        c = i % ROTATE
-        self.sol.decode_step(self.shape, [w[c] for w in self.weights], [k[c] for k in self.kvs], self.B, self.h_in,
-                             self.h_out, None, self.r, self.p, self.b, self.ws, self.ws_bytes)
+        c, j, a = self._phase(i)
+        r, p, b = self.acts[a]
+        self.sol.decode_step(self.shape, [w[c] for w in self.weights], [k[c][j] for k in self.kvs], self.B, self.h_in,
+                             self.h_out, None, r, p, b, self.ws, self.ws_bytes)
 
     def step_host(self, i):
-        c = i % ROTATE
-        self.sol.decode_step_host(self.shape, [w[c] for w in self.weights], [k[c] for k in self.kvs], self.B,
-                                  self.h_in_host, self.h_out_host, self.r_host, self.p_host, self.b_host,
-                                  self.lens_host, self.ws, self.ws_bytes)
+        c, j, a = self._phase(i)
+        r, p, b = self.acts_host[a]
+        self.sol.decode_step_host(self.shape, [w[c] for w in self.weights], [k[c][j] for k in self.kvs], self.B,
+                                  self.h_in_host, self.h_out_host, r, p, b, self.lens_host[j], self.ws, self.ws_bytes)
 
     def union_rows(self):
         """Rows of W_down that at least one token keeps, from one traced call of layer 0."""
@@ -217,7 +242,7 @@ class Replica:
         kept = t.full((self.B, ff), -1, dtype=t.int32, device=self.device)
         cnt = t.zeros((self.B,), dtype=t.int32, device=self.device)
         out = t.zeros_like(self.h_out)
-        sol.decode_layer(self.shape, self.weights[0][0], self.kvs[0][0], self.B, self.h_in, out, self.r, self.p,
+        sol.decode_layer(self.shape, self.weights[0][0], self.kvs[0][0][0], self.B, self.h_in, out, self.r, self.p,
                          self.b, sol.make_trace(kept_ch=kept, kept_ch_cnt=cnt), self.ws, self.ws_bytes)
         t.cuda.synchronize()
         k, c = kept.cpu().numpy(), cnt.cpu().numpy()
@@ -227,7 +252,7 @@ class Replica:
         return len(rows)
 
     def required_bytes_per_step(self, union_rows):
-        kb = kernel_bytes(self.cfg, self.seq_lens, self.r_np, union_rows)
+        kb = kernel_bytes(self.cfg, self.seq_lens + (self.cycle - 1) // 2, self.r_np, union_rows)
         return self.L * sum(kb.values()), kb
 
 
@@ -279,7 +304,8 @@ def run_ours(args):
     cfg = synth.WORKLOADS[args.workload]
     rep = Replica(cfg, device, seed=0)
     r, p, b = synth.draw_actions(cfg, 0)
-    rep.set_actions(r, p, b)
+    redraws = [synth.draw_actions(cfg, 0, redraw=k) for k in range(1, SERVE_STEPS // SERVE_REDRAW)] if rep.serving else None
+    rep.set_actions(r, p, b, redraws)
     union = rep.union_rows()
     req_bytes, kb = rep.required_bytes_per_step(union)
     peak_gbs, peak_kind = measured_peaks()
@@ -341,7 +367,19 @@ def run_ours(args):
             sweep.append({"r": rr / 1000, "p": pp / 1000, "b": bb, "us_per_step": round(1e3 * t_ms, 2),
                           "required_mb": round(byt / 1e6, 1), "hbm_gbs": round(byt / t_ms / 1e6, 1),
                           "frac_of_measured": round(byt / t_ms / 1e6 / peak_gbs, 4)})
-        rep.set_actions(r, p, b)
+        # the same budgets as a batch mix of the two adjacent keep-rates (how a fixed schedule hits a
+        # budget that falls between discrete levels), bit-widths drawn per sequence
+        for tgt in (1000, 500, 250, 125):
+            rm, pm, bm = synth.budget_mix_actions(cfg, tgt, 0)
+            rep.set_actions(rm, pm, bm)
+            u = rep.union_rows()
+            byt, _ = rep.required_bytes_per_step(u)
+            n = min(args.steps, 300)
+            t_ms = max_over_ranks(timed_steps(rep, n, 5, barrier, rep.step)) / n
+            sweep.append({"mix_mean_r": tgt / 1000, "p": 0.0, "b": "drawn", "us_per_step": round(1e3 * t_ms, 2),
+                          "required_mb": round(byt / 1e6, 1), "hbm_gbs": round(byt / t_ms / 1e6, 1),
+                          "frac_of_measured": round(byt / t_ms / 1e6 / peak_gbs, 4)})
+        rep.set_actions(r, p, b, redraws)
 
     line = None
     if rank == 0:
@@ -353,7 +391,8 @@ def run_ours(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "layers": cfg["layers"], "batch": cfg["batch"],
                        "context": int(np.max(rep.seq_lens)), "actions": "per-sequence uniform draw, seed 0",
-                       "l2": f"inputs larger than L2: {ROTATE} rotating copies of weights and KV cache",
+                       "l2": f"inputs larger than L2: {rep.rotate} rotating cop{'ies' if rep.rotate > 1 else 'y'} of weights "
+                             f"and KV cache, {rep.copy_mb} MB each",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "required_bytes_per_step": int(req_bytes),
             "hbm_tbs": round(hbm_gbs / 1e3, 4),
