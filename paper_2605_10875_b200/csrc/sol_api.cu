@@ -99,7 +99,7 @@ static int pad_rows(int B) {
 
 struct Layout {
   size_t status, stage_h_in, stage_act, stage_h_out, a_op, scale, qkv, q_rot, q_split, logits, sigma, kept_idx,
-      kept_cnt, part, work_items, work_ctr, attn_hi, attn_lo, attn_f32, h_mid, o_part, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, ch_sel, ch_cand_val, ch_cand_idx, ch_keep, down_part,
+      kept_cnt, part, work_items, kept_row, work_ctr, attn_hi, attn_lo, attn_f32, h_mid, o_part, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, ch_sel, ch_cand_val, ch_cand_idx, ch_keep, down_part,
       h_a, h_b, total;
   int splits, chunks, Mpad, Tmax;
 };
@@ -147,7 +147,8 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   L.kept_idx = take(B * Hkv * Tmax * 4);
   L.kept_cnt = take(B * Hkv * 4);
   L.part = take(B * Hkv * L.splits * G * (hd + 2) * 4);
-  L.work_items = take(B * Hkv * (size_t)L.splits * 4);
+  L.work_items = take(B * Hkv * (size_t)L.splits * 8);
+  L.kept_row = take(B * Hkv * Tmax * 4);
   L.work_ctr = take((2 + B * Hkv) * 4);
   L.attn_hi = take(Mpad * Hq * hd * 2);
   L.attn_lo = take(Mpad * Hq * hd * 2);
@@ -217,6 +218,7 @@ static void run_attention(const sol_shape_t& s, const Layout& L, void* ws, const
   a.part = at<float>(ws, L.part);
   a.splits = attn_splits(s.head_dim, kv.max_pages_per_seq, s.page_size);
   a.work_items = at<int32_t>(ws, L.work_items);
+  a.kept_row = at<uint32_t>(ws, L.kept_row);
   a.work_ctr = at<int32_t>(ws, L.work_ctr);
   a.out_f32 = out_f32;
   a.out_bf16 = out_bf16;

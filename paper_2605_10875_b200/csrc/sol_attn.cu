@@ -264,6 +264,7 @@ struct SelectDev {
   const float* sigma;
   int32_t* kept_idx;
   int32_t* kept_cnt;
+  uint32_t* kept_row;
   int32_t* work_items;
   int32_t* work_ctr;
   int* status;
@@ -286,7 +287,10 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
   const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
   const size_t row = (size_t)bk * p.Tmax;
   const float* sig = p.sigma + row;
-  const int j0 = tid * KPT;
+  // a thread owns `per` consecutive tokens: as few as this sequence needs (a multiple of 4 for the
+  // vector loads), so a short context in a long-context batch costs what its own length costs
+  const int per = min(KPT, ((max(T, 1) + THREADS - 1) / THREADS + 3) / 4 * 4);
+  const int j0 = tid * per;
 
   int total = 0;
   if (T > 0) {
@@ -314,6 +318,7 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
       float mx = 0.f;
 #pragma unroll
       for (int i = 0; i < KPT; i += 4) {
+        if (i >= per) break;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (j0 + i < T) v = *reinterpret_cast<const float4*>(sig + j0 + i);
         const float vv[4] = {v.x, v.y, v.z, v.w};
@@ -334,7 +339,7 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
         }
       }
       mx = block_max<THREADS>(mx, 0, sm);
-      key_thr = select_kth<THREADS, KPT>(key, k, tie_need, sm);
+      key_thr = select_kth<THREADS, KPT>(key, k, tie_need, sm, per);
       mode = 3;
 
       // ---- window around the threshold, re-scored in float64 ----
@@ -346,6 +351,7 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
       int n_in = 0;
 #pragma unroll
       for (int i = 0; i < KPT; ++i) {
+        if (i >= per) break;
         const uint32_t kk = key[i];
         if (kk == 0u || kk == 0xffffffffu) continue;
         const float sv = key_to_float(kk);
@@ -409,7 +415,19 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
       if (mode == 3) return key[i] > key_thr ? 2 : (key[i] == key_thr ? 1 : 0);
       return 0;
     };
-    total = compact_indices<THREADS, KPT>(klass, [](int, bool) {}, mode == 3 ? tie_need : 0, p.kept_idx + row, sm);
+    // beside the index list, the cache row of every kept token (page table applied), so that pass 2
+    // goes from the list straight to the V rows
+    const int32_t* table = p.kv.page_table + (size_t)b * p.kv.max_pages_per_seq;
+    auto emit = [&](int i, bool keep, int pos) {
+      if (!keep) return;
+      const int j = j0 + i;
+      const int page = table[j / PAGE];
+      uint32_t ridx = 0xffffffffu;
+      if (page >= 0 && page < p.kv.num_pages) ridx = (uint32_t)((page * Hkv + kvh) * PAGE + (j % PAGE));
+      else atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+      p.kept_row[row + pos] = ridx;
+    };
+    total = compact_indices<THREADS, KPT>(klass, emit, mode == 3 ? tie_need : 0, p.kept_idx + row, sm, per);
   }
   if (tid == 0) p.kept_cnt[bk] = total;
 
@@ -420,7 +438,10 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
   if (tid == 0) sm.counts[3] = atomicAdd(p.work_ctr, ns);
   __syncthreads();
   const int base = sm.counts[3];
-  for (int i = tid; i < ns; i += THREADS) p.work_items[base + i] = bk * p.S + i;
+  for (int i = tid; i < ns; i += THREADS) {
+    p.work_items[2 * (base + i)] = bk * p.S + i;
+    p.work_items[2 * (base + i) + 1] = total;
+  }
 }
 
 // ============================================================================
@@ -431,7 +452,7 @@ struct GatherDev {
   int Hq, Hkv, G, Tmax, S;
   const float* logits;
   const int32_t* kept_idx;
-  const int32_t* kept_cnt;
+  const uint32_t* kept_row;
   const int32_t* work_items;
   int32_t* work_ctr;
   float* part;  // [B][Hkv][S][G][HD + 2]
@@ -472,7 +493,7 @@ struct GatherLayout {
   static constexpr int V_BYTES = SPLIT * ROW_STRIDE;
   static constexpr int P_BYTES = 2 * GMAX * P_STRIDE * 2;
   static constexpr int ROWIDX_BYTES = SPLIT * 4;
-  static constexpr int BYTES = V_BYTES + P_BYTES + ROWIDX_BYTES + 64;
+  static constexpr int BYTES = V_BYTES + P_BYTES + ROWIDX_BYTES + 64;  // 64: flags
   static_assert(KSTEPS >= 1 && KSTEPS <= 4, "copy groups are waited on with at most 3 in flight");
   static_assert(GA_WARPS * GMAX * (HD + 2) * 4 <= V_BYTES, "the merge scratch reuses the V tile");
 };
@@ -504,21 +525,26 @@ __global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev
   pdl_wait();
 
   for (;;) {
+    // items are claimed from a shared counter: their cost varies (the last item of a (sequence,
+    // kv-head) also merges its partials)
     if (tid == 0) {
       const int it = atomicAdd(p.work_ctr + 1, 1);
-      flag[0] = it < p.work_ctr[0] ? p.work_items[it] : -1;
+      int2 h = make_int2(-1, 0);
+      if (it < p.work_ctr[0]) h = *reinterpret_cast<const int2*>(p.work_items + 2 * it);
+      flag[0] = h.x;
+      flag[2] = h.y;
     }
     __syncthreads();
     const int item = flag[0];
     if (item < 0) break;
+    const int cnt = flag[2];
     const int bk = item / p.S, s = item % p.S;
     const int b = bk / Hkv, kvh = bk % Hkv;
-    const int cnt = p.kept_cnt[bk];
     const int n0 = s * L::SPLIT, n1 = min(cnt, n0 + L::SPLIT);
     const size_t row = (size_t)bk * p.Tmax;
     const int tok0 = warp * L::TPW;  // first token slot of this warp within the item
 
-    // ---- row addresses of this warp's tokens ----
+    // ---- cache rows (page table already applied by the selection kernel) of this warp's tokens ----
     int jj[L::TPW / 32];
 #pragma unroll
     for (int i = 0; i < L::TPW / 32; ++i) {
@@ -527,14 +553,8 @@ __global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev
       uint32_t ridx = 0xffffffffu;
       jj[i] = -1;
       if (n < n1) {
-        const int j = p.kept_idx[row + n];
-        const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + j / PAGE];
-        if (page >= 0 && page < p.kv.num_pages) {
-          ridx = (uint32_t)((page * Hkv + kvh) * PAGE + (j % PAGE));
-          jj[i] = j;
-        } else {
-          atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
-        }
+        ridx = p.kept_row[row + n];
+        if (ridx != 0xffffffffu) jj[i] = p.kept_idx[row + n];
       }
       rowidx[slot] = ridx;
     }
@@ -554,7 +574,6 @@ __global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev
       }
       cp_async_commit();
     }
-
     // ---- softmax weights relative to the warp's maximum ----
     float x[L::TPW / 32][GMAX];
     float mh[GMAX], lh[GMAX];
@@ -741,7 +760,7 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   SelectDev se;
   se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.S = a.splits;
   se.split_len = attn_split_len(hd); se.q_rot = a.q_rot;
-  se.sigma = a.sigma; se.kept_idx = a.kept_idx; se.kept_cnt = a.kept_cnt;
+  se.sigma = a.sigma; se.kept_idx = a.kept_idx; se.kept_cnt = a.kept_cnt; se.kept_row = a.kept_row;
   se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
   {
     const dim3 grid(Hkv, a.B);
@@ -754,7 +773,7 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
 
   GatherDev gd;
   gd.kv = a.kv; gd.Hq = Hq; gd.Hkv = Hkv; gd.G = G; gd.Tmax = Tmax; gd.S = a.splits;
-  gd.logits = a.logits; gd.kept_idx = a.kept_idx; gd.kept_cnt = a.kept_cnt;
+  gd.logits = a.logits; gd.kept_idx = a.kept_idx; gd.kept_row = a.kept_row;
   gd.work_items = a.work_items; gd.work_ctr = a.work_ctr; gd.part = a.part;
   gd.scale_log2 = (float)(1.4426950408889634 / sqrt((double)hd));
   gd.out_f32 = a.out_f32;

@@ -130,10 +130,11 @@ struct AttnArgs {
   float* sigma;      // [B][Hkv][Tmax]
   int32_t* kept_idx; // [B][Hkv][Tmax]
   int32_t* kept_cnt; // [B][Hkv]
+  uint32_t* kept_row; // [B][Hkv][Tmax] cache row (page-resolved) of every kept token, 0xffffffff: bad page
   float* part;       // [B][Hkv][S][G][hd + 2]
   int splits;        // S = ceil(Tmax / attn_split_len(hd))
-  int32_t* work_items;  // [B*Hkv*S] pass-2 work list, filled by the selection kernel
-  int32_t* work_ctr;    // [2 + B*Hkv]: items emitted, next item to take, finished items per (sequence, kv-head)
+  int32_t* work_items;  // [B*Hkv*S][2] pass-2 work list (item code, kept count), filled by the selection kernel
+  int32_t* work_ctr;    // [2 + B*Hkv]: items emitted, unused, finished items per (sequence, kv-head)
   // outputs (each optional)
   float* out_f32;    // [B][Hq][hd]
   void* out_bf16;    // [B][Hq][hd]

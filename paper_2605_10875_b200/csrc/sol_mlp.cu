@@ -218,7 +218,7 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
   uint16_t* tl = p.t_lo + (size_t)b * ff;
   uint32_t hw[4], lw[4];
   bool any = false;
-  auto emit = [&](int i, bool keep) {
+  auto emit = [&](int i, bool keep, int) {
     uint16_t hv = 0, lv = 0;
     if (keep) {
       const float a = key_to_float(key[i]);
@@ -471,7 +471,7 @@ __global__ void __launch_bounds__(THREADS) channel_list_kernel(const unsigned ch
   const int b = blockIdx.x, j0 = threadIdx.x * KPT;
   const unsigned char* k = keep + (size_t)b * ff;
   auto klass = [&](int i) -> int { return (j0 + i < ff && k[j0 + i]) ? 2 : 0; };
-  compact_indices<THREADS, KPT>(klass, [](int, bool) {}, 0, kept_ch + (size_t)b * ff, sm);
+  compact_indices<THREADS, KPT>(klass, [](int, bool, int) {}, 0, kept_ch + (size_t)b * ff, sm);
 }
 
 void launch_channel_select(const ChannelSelectArgs& a, cudaStream_t st) {

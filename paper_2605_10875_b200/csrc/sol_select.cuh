@@ -38,15 +38,17 @@ __device__ __forceinline__ float key_to_float(uint32_t key) {
   return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
 }
 
-// The k-th largest of the block's keys (1 <= k <= number of keys).  Absent elements carry key 0 and
-// count like any other key, so k must not exceed the number of present elements.  tie_need = how many
+// The k-th largest of the block's keys (1 <= k <= number of keys).  Only the first per_thread keys of
+// every thread take part.  Absent elements carry key 0 and count like any other key, so k must not
+// exceed the number of present elements.  tie_need = how many
 // keys equal to the result belong to the top k.  All threads call.
 //
 // One histogram pass over the top 12 key bits (shared-memory atomics) finds the bin that holds the
 // k-th key; if that bin is small its keys are listed and ranked exactly, otherwise the next 12 (then
 // the last 8) bits are histogrammed within it.
 template <int THREADS, int KPT>
-__device__ __forceinline__ uint32_t select_kth(const uint32_t (&key)[KPT], int k, int& tie_need, SelectSmem& sm) {
+__device__ __forceinline__ uint32_t select_kth(const uint32_t (&key)[KPT], int k, int& tie_need, SelectSmem& sm,
+                                               int per_thread = KPT) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint32_t prefix = 0, mask = 0;
   int remaining = k, pop = 0;
@@ -58,7 +60,7 @@ __device__ __forceinline__ uint32_t select_kth(const uint32_t (&key)[KPT], int k
     __syncthreads();
 #pragma unroll
     for (int i = 0; i < KPT; ++i)
-      if ((key[i] & mask) == prefix) atomicAdd(&sm.hist[(key[i] >> shift) & (uint32_t)(nb - 1)], 1u);
+      if (i < per_thread && (key[i] & mask) == prefix) atomicAdd(&sm.hist[(key[i] >> shift) & (uint32_t)(nb - 1)], 1u);
     __syncthreads();
     // bins in descending order: thread t owns bins nb-1-t*bpt .. nb-bpt-t*bpt
     const int bpt = nb >= THREADS ? nb / THREADS : 1;
@@ -106,7 +108,7 @@ __device__ __forceinline__ uint32_t select_kth(const uint32_t (&key)[KPT], int k
   __syncthreads();
 #pragma unroll
   for (int i = 0; i < KPT; ++i)
-    if ((key[i] & mask) == prefix) sm.rank_key[atomicAdd(&sm.counts[2], 1)] = key[i];
+    if (i < per_thread && (key[i] & mask) == prefix) sm.rank_key[atomicAdd(&sm.counts[2], 1)] = key[i];
   __syncthreads();
   for (int c = tid; c < pop; c += THREADS) {
     const uint32_t kc = sm.rank_key[c];
@@ -164,17 +166,20 @@ __device__ __forceinline__ void rank_candidates(int n_cand, int need, SelectSmem
   }
 }
 
-// klass(i) in {0 dropped, 1 tie, 2 kept} for element j = tid*KPT + i (called twice per element).  Ties
+// klass(i) in {0 dropped, 1 tie, 2 kept} for element j = tid*per_thread + i, i < per_thread <= KPT (called
+// twice per element; a thread's elements beyond per_thread must be class 0).  Ties
 // are kept in ascending index order until tie_need runs out.  Kept indices go to out[] ascending;
-// emit(i, keep) reports the final decision of every element.  Returns the kept total to every thread.
+// emit(i, keep, pos) reports the final decision of every element and, for a kept one, its place in out[].  Returns the kept total to every thread.
 // All threads call; uses sm.scan.
 template <int THREADS, int KPT, typename ClassFn, typename EmitFn>
-__device__ __forceinline__ int compact_indices(ClassFn klass, EmitFn emit, int tie_need, int32_t* out, SelectSmem& sm) {
+__device__ __forceinline__ int compact_indices(ClassFn klass, EmitFn emit, int tie_need, int32_t* out, SelectSmem& sm,
+                                               int per_thread = KPT) {
   constexpr int WARPS = THREADS / 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int c2 = 0, c1 = 0;
 #pragma unroll
   for (int i = 0; i < KPT; ++i) {
+    if (i >= per_thread) break;
     const int c = klass(i);
     c2 += c == 2;
     c1 += c == 1;
@@ -208,17 +213,19 @@ __device__ __forceinline__ int compact_indices(ClassFn klass, EmitFn emit, int t
     total += v;
   }
   int ties_left = my_ties;
-  const int j0 = threadIdx.x * KPT;
+  const int j0 = threadIdx.x * per_thread;
 #pragma unroll
   for (int i = 0; i < KPT; ++i) {
+    if (i >= per_thread) break;
     const int c = klass(i);
     bool kp = c == 2;
     if (c == 1 && ties_left > 0) {
       kp = true;
       --ties_left;
     }
-    if (kp) out[pos++] = j0 + i;
-    emit(i, kp);
+    if (kp) out[pos] = j0 + i;
+    emit(i, kp, pos);
+    if (kp) ++pos;
   }
   __syncthreads();  // sm.scan may be reused by the caller
   return total;

@@ -46,7 +46,7 @@ sol_status_t scratch_of_current_device(unsigned char** out) {
 }
 
 struct StaticLayout {
-  size_t status, q_rot, q_split, logits, sigma, kept_idx, kept_cnt, part, work_items, work_ctr, total;
+  size_t status, q_rot, q_split, logits, sigma, kept_idx, kept_cnt, part, work_items, kept_row, work_ctr, total;
   int splits;
 };
 
@@ -69,7 +69,8 @@ StaticLayout layout_for(const sol_shape_t& s, int B, int max_pages) {
   L.kept_idx = take(B * Hkv * Tmax * 4);
   L.kept_cnt = take(B * Hkv * 4);
   L.part = take(B * Hkv * (size_t)L.splits * G * (hd + 2) * 4);
-  L.work_items = take(B * Hkv * (size_t)L.splits * 4);
+  L.work_items = take(B * Hkv * (size_t)L.splits * 8);
+  L.kept_row = take(B * Hkv * Tmax * 4);
   L.work_ctr = take((2 + B * Hkv) * 4);
   L.total = at;
   return L;
@@ -124,6 +125,7 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
   a.part = reinterpret_cast<float*>(base + L.part);
   a.splits = L.splits;
   a.work_items = reinterpret_cast<int32_t*>(base + L.work_items);
+  a.kept_row = reinterpret_cast<uint32_t*>(base + L.kept_row);
   a.work_ctr = reinterpret_cast<int32_t*>(base + L.work_ctr);
   a.out_f32 = nullptr;
   a.out_bf16 = out_bf16;
