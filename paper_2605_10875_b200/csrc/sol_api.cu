@@ -149,7 +149,7 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   L.part = take(B * Hkv * L.splits * G * (hd + 2) * 4);
   L.work_items = take(B * Hkv * (size_t)L.splits * 8);
   L.kept_row = take(B * Hkv * Tmax * 4);
-  L.work_ctr = take((2 + B * Hkv) * 4);
+  L.work_ctr = take((4 + B * Hkv) * 4);
   L.attn_hi = take(Mpad * Hq * hd * 2);
   L.attn_lo = take(Mpad * Hq * hd * 2);
   L.attn_f32 = take(B * Hq * hd * 4);

@@ -45,6 +45,8 @@ struct PrepDev {
 };
 
 constexpr int PREP_THREADS = 128;
+// words of AttnArgs::work_ctr
+enum : int { WC_ITEMS = 0, WC_NEXT = 1, WC_CPI = 2, WC_DONE = 4 };
 
 // One CTA per (kv-head, sequence): the G query heads of the group, the new k row and the new v row.
 __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p) {
@@ -69,10 +71,10 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
   };
 
   if (tid == 0) {
-    p.work_ctr[2 + b * Hkv + kvh] = 0;
+    p.work_ctr[WC_DONE + b * Hkv + kvh] = 0;
     if (b == 0 && kvh == 0) {
-      p.work_ctr[0] = 0;
-      p.work_ctr[1] = 0;
+      p.work_ctr[WC_ITEMS] = 0;
+      p.work_ctr[WC_NEXT] = 0;
     }
   }
   if (tid < half) {
@@ -259,7 +261,7 @@ struct SelectDev {
   sol_shape_t sh;
   sol_kv_t kv;
   const int32_t* r_permille;
-  int Tmax, S, split_len;
+  int Tmax, S, split_len, B, target_items;
   const float* q_rot;
   const float* sigma;
   int32_t* kept_idx;
@@ -431,15 +433,33 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
   }
   if (tid == 0) p.kept_cnt[bk] = total;
 
-  // pass-2 work items of this (sequence, kv-head): one per split_len kept tokens, at least one so
-  // that the output is always written
-  const int ns = max(1, (total + p.split_len - 1) / p.split_len);
+  // Pass-2 work items of this (sequence, kv-head): runs of `cpi` chunks of split_len kept tokens (at least
+  // one item, so that the output is always written).  cpi is the same in every CTA: it is sized from the
+  // kept count of the whole batch so that the batch yields about target_items items: few, long items
+  // amortise the per-item work, enough of them keep every SM busy.
+  int kb = 0;
+  for (int i = tid; i < p.B; i += THREADS) {
+    const int Ti = min(p.kv.seq_lens[i], p.kv.max_pages_per_seq * PAGE);
+    if (Ti > 0) {
+      const int ns_ = min(max(p.sh.n_sink, 0), Ti), nw_ = min(max(p.sh.n_window, 0), Ti - ns_);
+      long long bd = ((long long)p.r_permille[i] * Ti + 999) / 1000;
+      if (bd > Ti) bd = Ti;
+      kb += (min(Ti, max((int)bd, ns_ + nw_)) + p.split_len - 1) / p.split_len;
+    }
+  }
   __syncthreads();
-  if (tid == 0) sm.counts[3] = atomicAdd(p.work_ctr, ns);
+  const int batch_chunks = block_count<THREADS>(kb, 0, sm) * Hkv;
+  const int cpi = min(8, max(1, (batch_chunks + p.target_items - 1) / p.target_items));
+  const int chunks = max(1, (total + p.split_len - 1) / p.split_len);
+  const int ns = (chunks + cpi - 1) / cpi;
+  if (tid == 0) {
+    sm.counts[3] = atomicAdd(p.work_ctr + WC_ITEMS, ns);
+    p.work_ctr[WC_CPI] = cpi;
+  }
   __syncthreads();
   const int base = sm.counts[3];
   for (int i = tid; i < ns; i += THREADS) {
-    p.work_items[2 * (base + i)] = bk * p.S + i;
+    p.work_items[2 * (base + i)] = bk * p.S + i * cpi;  // first chunk of the item
     p.work_items[2 * (base + i) + 1] = total;
   }
 }
@@ -483,54 +503,64 @@ __device__ __forceinline__ void cp_async_wait_dyn(int n) {
 constexpr int GA_WARPS = 4;
 constexpr int GA_THREADS = GA_WARPS * 32;
 
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+
 template <int HD, int GMAX>
 struct GatherLayout {
-  static constexpr int SPLIT = HD == 64 ? 256 : 128;  // kept tokens per work item (attn_split_len)
-  static constexpr int TPW = SPLIT / GA_WARPS;        // tokens per warp
-  static constexpr int KSTEPS = TPW / 16;             // MMA k-steps per warp
+  static constexpr int SPLIT = HD == 64 ? 256 : 128;  // kept tokens per chunk (attn_split_len): 32 KB of V rows
+  static constexpr int TPW = SPLIT / GA_WARPS;        // tokens per warp and chunk
+  static constexpr int NT = TPW / 32;                 // tokens per lane and chunk
+  static constexpr int KSTEPS = TPW / 16;             // MMA k-steps per warp and chunk
   static constexpr int ROW_STRIDE = HD * 2 + 16;      // bytes; +16 keeps ldmatrix rows on distinct banks
   static constexpr int P_STRIDE = SPLIT + 8;          // bf16 elements; +8 spreads the heads over the banks
+  static constexpr int STAGES = 2;
   static constexpr int V_BYTES = SPLIT * ROW_STRIDE;
+  static constexpr int LG_BYTES = SPLIT * GMAX * 4;   // logits of the chunk's tokens, [slot][GMAX]
+  static constexpr int STAGE_BYTES = V_BYTES + LG_BYTES;
   static constexpr int P_BYTES = 2 * GMAX * P_STRIDE * 2;
   static constexpr int ROWIDX_BYTES = SPLIT * 4;
-  static constexpr int BYTES = V_BYTES + P_BYTES + ROWIDX_BYTES + 64;  // 64: flags
-  static_assert(KSTEPS >= 1 && KSTEPS <= 4, "copy groups are waited on with at most 3 in flight");
-  static_assert(GA_WARPS * GMAX * (HD + 2) * 4 <= V_BYTES, "the merge scratch reuses the V tile");
+  static constexpr int BYTES = STAGES * STAGE_BYTES + P_BYTES + ROWIDX_BYTES + 64;  // 64: flags
+  static_assert(GA_WARPS * GMAX * (HD + 2) * 4 <= V_BYTES, "the merge scratch reuses the first V tile");
 };
 
-// Persistent CTAs take (sequence, kv-head, split) items from the work list.  Per item each warp owns
-// a quarter of the kept tokens: it resolves their V row addresses, starts all row copies (cp.async,
-// one commit group per 16 tokens), turns the kept logits into softmax weights relative to the warp's
-// own maximum, and multiplies weights by rows on the tensor cores as the groups land: the weights
-// (bf16 high part in MMA rows 0..G-1, low part in rows 8..8+G-1) are the A operand, the V rows the
-// B operand.  The CTA that finishes the last item of a (sequence, kv-head) merges its partials.
+// Persistent CTAs claim items from the work list: (sequence, kv-head, run of chunks).  Within an item
+// every warp owns a quarter of each chunk's kept tokens and runs its own two-stage pipeline over the
+// chunks: while chunk c is multiplied, the V rows and the logits of chunk c+1 are in flight (cp.async
+// into the other stage) and the index words of chunk c+2 are being fetched, so only the first chunk of
+// an item pays for the chain indices -> rows.  Softmax weights are relative to a running maximum per
+// head (the accumulators are rescaled when it grows); weights x rows runs on the tensor cores: the
+// weights (bf16 high part in MMA rows 0..G-1, low part in rows 8..8+G-1) are the A operand, the V
+// rows the B operand.  Per item one partial is written; the CTA that finishes the last item of a
+// (sequence, kv-head) merges its partials.
 template <int HD, int GMAX>
 __global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev p) {
   using L = GatherLayout<HD, GMAX>;
   extern __shared__ __align__(128) unsigned char smem[];
-  unsigned char* vt = smem;
-  uint16_t* p_hi = reinterpret_cast<uint16_t*>(smem + L::V_BYTES);
+  uint16_t* p_hi = reinterpret_cast<uint16_t*>(smem + L::STAGES * L::STAGE_BYTES);
   uint16_t* p_lo = p_hi + GMAX * L::P_STRIDE;
-  uint32_t* rowidx = reinterpret_cast<uint32_t*>(smem + L::V_BYTES + L::P_BYTES);
-  int* flag = reinterpret_cast<int*>(smem + L::V_BYTES + L::P_BYTES + L::ROWIDX_BYTES);
-  float* sc_acc = reinterpret_cast<float*>(smem);                        // [GA_WARPS][GMAX][HD], after the MMAs
-  float* sc_ml = sc_acc + GA_WARPS * GMAX * HD;                          // [GA_WARPS][GMAX][2]
+  uint32_t* rowidx = reinterpret_cast<uint32_t*>(smem + L::STAGES * L::STAGE_BYTES + L::P_BYTES);
+  int* flag = reinterpret_cast<int*>(smem + L::STAGES * L::STAGE_BYTES + L::P_BYTES + L::ROWIDX_BYTES);
+  float* sc_acc = reinterpret_cast<float*>(smem);  // [GA_WARPS][GMAX][HD], after the MMAs
+  float* sc_ml = sc_acc + GA_WARPS * GMAX * HD;    // [GA_WARPS][GMAX][2]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
   const int G = p.G, Hkv = p.Hkv;
   const uint16_t* vp = static_cast<const uint16_t*>(p.kv.v_pool);
   constexpr int CH = HD / 8;  // 16-byte chunks per row
+  const int tok0 = warp * L::TPW;  // first token slot of this warp within a chunk
+  const int mi = lane >> 3, mr = lane & 7;  // ldmatrix: this lane addresses row mr of matrix mi
   pdl_trigger();
   pdl_wait();
+  const int cpi = p.work_ctr[WC_CPI];
 
   for (;;) {
-    // items are claimed from a shared counter: their cost varies (the last item of a (sequence,
-    // kv-head) also merges its partials)
     if (tid == 0) {
-      const int it = atomicAdd(p.work_ctr + 1, 1);
+      const int it = atomicAdd(p.work_ctr + WC_NEXT, 1);
       int2 h = make_int2(-1, 0);
-      if (it < p.work_ctr[0]) h = *reinterpret_cast<const int2*>(p.work_items + 2 * it);
+      if (it < p.work_ctr[WC_ITEMS]) h = *reinterpret_cast<const int2*>(p.work_items + 2 * it);
       flag[0] = h.x;
       flag[2] = h.y;
     }
@@ -538,108 +568,160 @@ __global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev
     const int item = flag[0];
     if (item < 0) break;
     const int cnt = flag[2];
-    const int bk = item / p.S, s = item % p.S;
+    const int bk = item / p.S, c0 = item % p.S;
     const int b = bk / Hkv, kvh = bk % Hkv;
-    const int n0 = s * L::SPLIT, n1 = min(cnt, n0 + L::SPLIT);
     const size_t row = (size_t)bk * p.Tmax;
-    const int tok0 = warp * L::TPW;  // first token slot of this warp within the item
+    const int chunks = max(1, (cnt + L::SPLIT - 1) / L::SPLIT);
+    const int nch = min(cpi, chunks - c0);
 
-    // ---- cache rows (page table already applied by the selection kernel) of this warp's tokens ----
-    int jj[L::TPW / 32];
+    // index words of the chunk that is issued next (kept in registers one chunk ahead)
+    int pj[L::NT];
+    uint32_t pr[L::NT];
+    auto load_idx = [&](int c) {
 #pragma unroll
-    for (int i = 0; i < L::TPW / 32; ++i) {
-      const int slot = tok0 + lane + 32 * i;
-      const int n = n0 + slot;
-      uint32_t ridx = 0xffffffffu;
-      jj[i] = -1;
-      if (n < n1) {
-        ridx = p.kept_row[row + n];
-        if (ridx != 0xffffffffu) jj[i] = p.kept_idx[row + n];
-      }
-      rowidx[slot] = ridx;
-    }
-    __syncwarp();
-
-    // ---- start every row copy; rows of absent tokens are zero-filled ----
-#pragma unroll
-    for (int ks = 0; ks < L::KSTEPS; ++ks) {
-#pragma unroll
-      for (int i = 0; i < 16 * CH / 32; ++i) {
-        const int c = lane + 32 * i;
-        const int slot = tok0 + ks * 16 + c / CH, ch = c % CH;
-        const uint32_t ridx = rowidx[slot];
-        unsigned char* dst = vt + slot * L::ROW_STRIDE + ch * 16;
-        if (ridx != 0xffffffffu) cp_async16(smem_u32(dst), vp + (size_t)ridx * HD + ch * 8);
-        else *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
-      }
-      cp_async_commit();
-    }
-    // ---- softmax weights relative to the warp's maximum ----
-    float x[L::TPW / 32][GMAX];
-    float mh[GMAX], lh[GMAX];
-#pragma unroll
-    for (int h = 0; h < GMAX; ++h) mh[h] = -INFINITY;
-#pragma unroll
-    for (int i = 0; i < L::TPW / 32; ++i) {
-#pragma unroll
-      for (int h = 0; h < GMAX; ++h) {
-        x[i][h] = -INFINITY;
-        if (h < G && jj[i] >= 0) x[i][h] = p.logits[(row + jj[i]) * G + h] * p.scale_log2;
-        mh[h] = fmaxf(mh[h], x[i][h]);
-      }
-    }
-#pragma unroll
-    for (int h = 0; h < GMAX; ++h) {
-      mh[h] = warp_max(mh[h]);
-      lh[h] = 0.f;
-    }
-#pragma unroll
-    for (int i = 0; i < L::TPW / 32; ++i) {
-      const int slot = tok0 + lane + 32 * i;
-#pragma unroll
-      for (int h = 0; h < GMAX; ++h) {
-        if (h < G) {
-          const float pw = x[i][h] == -INFINITY ? 0.f : exp2f(x[i][h] - mh[h]);
-          lh[h] += pw;
-          const uint16_t hi = f2bf(pw);
-          p_hi[h * L::P_STRIDE + slot] = hi;
-          p_lo[h * L::P_STRIDE + slot] = f2bf(pw - bf2f(hi));
+      for (int i = 0; i < L::NT; ++i) {
+        const int n = (c0 + c) * L::SPLIT + tok0 + lane + 32 * i;
+        pr[i] = 0xffffffffu;
+        pj[i] = -1;
+        if (c < nch && n < cnt) {
+          pr[i] = p.kept_row[row + n];
+          if (pr[i] != 0xffffffffu) pj[i] = p.kept_idx[row + n];
         }
       }
-    }
+    };
+    // starts the copies of one chunk (this warp's tokens): logits, then V rows; one commit group
+    auto issue = [&](int stage) {
+      unsigned char* vt = smem + stage * L::STAGE_BYTES;
+      float* lg = reinterpret_cast<float*>(vt + L::V_BYTES);
 #pragma unroll
-    for (int h = 0; h < GMAX; ++h) lh[h] = warp_sum(lh[h]);
-    __syncwarp();
+      for (int i = 0; i < L::NT; ++i) {
+        const int slot = tok0 + lane + 32 * i;
+        rowidx[slot] = pr[i];
+        float* dst = lg + slot * GMAX;
+        if (pj[i] >= 0) {
+          const float* src = p.logits + (row + pj[i]) * G;
+          if (GMAX == 4 && G == 4) {
+            cp_async16(smem_u32(dst), src);
+          } else {
+            for (int h = 0; h < G; ++h) cp_async4(smem_u32(dst + h), src + h);
+          }
+        } else {
+#pragma unroll
+          for (int h = 0; h < GMAX; ++h) dst[h] = -INFINITY;  // an absent token weighs nothing
+        }
+      }
+      __syncwarp();
+#pragma unroll
+      for (int ks = 0; ks < L::KSTEPS; ++ks) {
+#pragma unroll
+        for (int i = 0; i < 16 * CH / 32; ++i) {
+          const int c = lane + 32 * i;
+          const int slot = tok0 + ks * 16 + c / CH, ch = c % CH;
+          const uint32_t ridx = rowidx[slot];
+          unsigned char* dst = vt + slot * L::ROW_STRIDE + ch * 16;
+          if (ridx != 0xffffffffu) cp_async16(smem_u32(dst), vp + (size_t)ridx * HD + ch * 8);
+          else *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      cp_async_commit();
+      __syncwarp();  // rowidx is rewritten by the next issue
+    };
 
-    // ---- weights x rows on the tensor cores, as the copy groups land ----
+    float mh[GMAX], lh[GMAX];
+#pragma unroll
+    for (int h = 0; h < GMAX; ++h) {
+      mh[h] = -INFINITY;
+      lh[h] = 0.f;
+    }
     float acc[HD / 8][4];
 #pragma unroll
     for (int nt = 0; nt < HD / 8; ++nt)
 #pragma unroll
       for (int r = 0; r < 4; ++r) acc[nt][r] = 0.f;
-    const int mi = lane >> 3, mr = lane & 7;  // ldmatrix: this lane addresses row mr of matrix mi
-#pragma unroll
-    for (int ks = 0; ks < L::KSTEPS; ++ks) {
-      cp_async_wait_dyn(L::KSTEPS - 1 - ks);
+
+    load_idx(0);
+    issue(0);
+    load_idx(1);
+#pragma unroll 1
+    for (int c = 0; c < nch; ++c) {
+      if (c + 1 < nch) {
+        issue((c + 1) & 1);
+        load_idx(c + 2);
+        cp_async_wait<1>();
+      } else {
+        cp_async_wait<0>();
+      }
       __syncwarp();
-      const int kb = tok0 + ks * 16;
-      uint32_t a0 = 0, a1 = 0, a2 = 0, a3 = 0;
-      if (g < G) {
-        a0 = *reinterpret_cast<const uint32_t*>(p_hi + g * L::P_STRIDE + kb + 2 * t);
-        a1 = *reinterpret_cast<const uint32_t*>(p_lo + g * L::P_STRIDE + kb + 2 * t);
-        a2 = *reinterpret_cast<const uint32_t*>(p_hi + g * L::P_STRIDE + kb + 8 + 2 * t);
-        a3 = *reinterpret_cast<const uint32_t*>(p_lo + g * L::P_STRIDE + kb + 8 + 2 * t);
-      }
-      const uint32_t vrow = smem_u32(vt) + (kb + (mi & 1) * 8 + mr) * L::ROW_STRIDE;
+      const unsigned char* vt = smem + (c & 1) * L::STAGE_BYTES;
+      const float* lg = reinterpret_cast<const float*>(vt + L::V_BYTES);
+
+      // ---- softmax weights relative to the running maximum ----
+      float x[L::NT][GMAX], cm[GMAX];
 #pragma unroll
-      for (int pr = 0; pr < HD / 16; ++pr) {
-        uint32_t bfr[4];
-        ldsm_x4_trans(bfr, vrow + ((2 * pr + (mi >> 1)) * 8) * 2);
-        mma_bf16(acc[2 * pr], a0, a1, a2, a3, bfr[0], bfr[1]);
-        mma_bf16(acc[2 * pr + 1], a0, a1, a2, a3, bfr[2], bfr[3]);
+      for (int h = 0; h < GMAX; ++h) cm[h] = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < L::NT; ++i) {
+        const float* src = lg + (tok0 + lane + 32 * i) * GMAX;
+#pragma unroll
+        for (int h = 0; h < GMAX; ++h) {
+          x[i][h] = h < G ? src[h] * p.scale_log2 : -INFINITY;
+          cm[h] = fmaxf(cm[h], x[i][h]);
+        }
       }
+      float my_sc = 1.f;  // rescaling of this lane's accumulator rows (head g, both parts)
+#pragma unroll
+      for (int h = 0; h < GMAX; ++h) {
+        const float nm = fmaxf(mh[h], warp_max(cm[h]));
+        const float sc = mh[h] == -INFINITY ? 0.f : exp2f(mh[h] - nm);
+        mh[h] = nm;
+        lh[h] *= sc;
+        if (h == g) my_sc = sc;
+      }
+#pragma unroll
+      for (int nt = 0; nt < HD / 8; ++nt)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) acc[nt][r] *= my_sc;
+#pragma unroll
+      for (int i = 0; i < L::NT; ++i) {
+        const int slot = tok0 + lane + 32 * i;
+#pragma unroll
+        for (int h = 0; h < GMAX; ++h) {
+          if (h < G) {
+            const float pw = x[i][h] == -INFINITY ? 0.f : exp2f(x[i][h] - mh[h]);
+            lh[h] += pw;
+            const uint16_t hi = f2bf(pw);
+            p_hi[h * L::P_STRIDE + slot] = hi;
+            p_lo[h * L::P_STRIDE + slot] = f2bf(pw - bf2f(hi));
+          }
+        }
+      }
+      __syncwarp();
+
+      // ---- weights x rows on the tensor cores ----
+#pragma unroll
+      for (int ks = 0; ks < L::KSTEPS; ++ks) {
+        const int kb = tok0 + ks * 16;
+        uint32_t a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+        if (g < G) {
+          a0 = *reinterpret_cast<const uint32_t*>(p_hi + g * L::P_STRIDE + kb + 2 * t);
+          a1 = *reinterpret_cast<const uint32_t*>(p_lo + g * L::P_STRIDE + kb + 2 * t);
+          a2 = *reinterpret_cast<const uint32_t*>(p_hi + g * L::P_STRIDE + kb + 8 + 2 * t);
+          a3 = *reinterpret_cast<const uint32_t*>(p_lo + g * L::P_STRIDE + kb + 8 + 2 * t);
+        }
+        const uint32_t vrow = smem_u32(vt) + (kb + (mi & 1) * 8 + mr) * L::ROW_STRIDE;
+#pragma unroll
+        for (int pr2 = 0; pr2 < HD / 16; ++pr2) {
+          uint32_t bfr[4];
+          ldsm_x4_trans(bfr, vrow + ((2 * pr2 + (mi >> 1)) * 8) * 2);
+          mma_bf16(acc[2 * pr2], a0, a1, a2, a3, bfr[0], bfr[1]);
+          mma_bf16(acc[2 * pr2 + 1], a0, a1, a2, a3, bfr[2], bfr[3]);
+        }
+      }
+      __syncwarp();  // the weights and this stage are rewritten from here on
     }
-    __syncthreads();  // every warp is done with the V tile: its space becomes the merge scratch
+#pragma unroll
+    for (int h = 0; h < GMAX; ++h) lh[h] = warp_sum(lh[h]);
+    __syncthreads();  // every warp is done with the stages: the first becomes the merge scratch
 
     if (g < G) {
 #pragma unroll
@@ -657,7 +739,8 @@ __global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev
       }
     }
     __syncthreads();
-    float* dst = p.part + (((size_t)bk * p.S + s) * G) * (HD + 2);
+    const int slot_no = c0 / cpi;  // this item's partial
+    float* dst = p.part + (((size_t)bk * p.S + slot_no) * G) * (HD + 2);
     for (int i = tid; i < G * HD; i += GA_THREADS) {
       const int h = i / HD, e = i % HD;
       float M = -INFINITY;
@@ -679,10 +762,10 @@ __global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev
     }
 
     // ---- the last item of this (sequence, kv-head) merges the partials ----
-    const int ns = max(1, (cnt + L::SPLIT - 1) / L::SPLIT);
+    const int ns = (chunks + cpi - 1) / cpi;
     __threadfence();
     __syncthreads();
-    if (tid == 0) flag[1] = atomicAdd(p.work_ctr + 2 + bk, 1) == ns - 1 ? 1 : 0;
+    if (tid == 0) flag[1] = atomicAdd(p.work_ctr + WC_DONE + bk, 1) == ns - 1 ? 1 : 0;
     __syncthreads();
     if (flag[1]) {
       __threadfence();
@@ -759,7 +842,7 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
 
   SelectDev se;
   se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.S = a.splits;
-  se.split_len = attn_split_len(hd); se.q_rot = a.q_rot;
+  se.split_len = attn_split_len(hd); se.q_rot = a.q_rot; se.B = a.B; se.target_items = 3 * sm_count();
   se.sigma = a.sigma; se.kept_idx = a.kept_idx; se.kept_cnt = a.kept_cnt; se.kept_row = a.kept_row;
   se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
   {
@@ -781,7 +864,7 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   gd.out_hi = static_cast<uint16_t*>(a.out_hi); gd.out_lo = static_cast<uint16_t*>(a.out_lo);
   gd.status = a.status;
   const long long items = (long long)a.B * Hkv * a.splits;
-  const int grid = (int)(items < (long long)sm_count() * 5 ? items : (long long)sm_count() * 5);
+  const int grid = (int)(items < (long long)sm_count() * 2 ? items : (long long)sm_count() * 2);
   if (hd == 64) {
     if (G <= 4) launch_gather<64, 4>(gd, grid, st);
     else launch_gather<64, 8>(gd, grid, st);

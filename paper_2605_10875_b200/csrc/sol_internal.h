@@ -134,7 +134,8 @@ struct AttnArgs {
   float* part;       // [B][Hkv][S][G][hd + 2]
   int splits;        // S = ceil(Tmax / attn_split_len(hd))
   int32_t* work_items;  // [B*Hkv*S][2] pass-2 work list (item code, kept count), filled by the selection kernel
-  int32_t* work_ctr;    // [2 + B*Hkv]: items emitted, unused, finished items per (sequence, kv-head)
+  int32_t* work_ctr;    // [4 + B*Hkv]: items emitted, next item to claim, chunks per item, unused; then the finished
+                        // items of every (sequence, kv-head)
   // outputs (each optional)
   float* out_f32;    // [B][Hq][hd]
   void* out_bf16;    // [B][Hq][hd]

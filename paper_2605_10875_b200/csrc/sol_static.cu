@@ -71,7 +71,7 @@ StaticLayout layout_for(const sol_shape_t& s, int B, int max_pages) {
   L.part = take(B * Hkv * (size_t)L.splits * G * (hd + 2) * 4);
   L.work_items = take(B * Hkv * (size_t)L.splits * 8);
   L.kept_row = take(B * Hkv * Tmax * 4);
-  L.work_ctr = take((2 + B * Hkv) * 4);
+  L.work_ctr = take((4 + B * Hkv) * 4);
   L.total = at;
   return L;
 }
