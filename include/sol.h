@@ -42,8 +42,10 @@ typedef int32_t sol_status_t;
 typedef struct CUstream_st *sol_stream_t; /* a cudaStream_t */
 
 /* Layer geometry.  Supported: head_dim 64 or 128; page_size 64;
- * n_q_heads a multiple of n_kv_heads; d_model and n_q_heads*head_dim
- * multiples of 256; d_ff a multiple of 32; batch 1..128. */
+ * n_q_heads a multiple of n_kv_heads (at most 8 query heads per kv head);
+ * d_model (<= 8192) and n_q_heads*head_dim multiples of 256; d_ff a multiple
+ * of 32, at most 49152; batch 1..128; at most 768 pages (49152 tokens) per
+ * sequence.  Anything else: SOL_ERR_UNSUPPORTED (sol_workspace_bytes: 0). */
 typedef struct sol_shape {
   int32_t d_model, n_q_heads, n_kv_heads, head_dim, d_ff, page_size;
   float rms_eps;
@@ -100,7 +102,12 @@ const char *sol_status_string(sol_status_t s);
 const char *sol_last_cuda_error(void); /* text of the last CUDA error seen by this thread's calls */
 
 /* Bytes of scratch that any call below needs for batches up to max_batch and
- * contexts up to max_pages_per_seq pages.  0 if the shape is unsupported. */
+ * contexts up to max_pages_per_seq pages.  0 if the shape is unsupported.
+ * The offsets inside the workspace depend on the batch of each call.  Results
+ * do not depend on what earlier calls left behind (every counter a call needs
+ * is cleared by the call itself), but stale "row is live" flags of a call with
+ * another batch size can cost extra weight reads: pass the workspace through
+ * sol_workspace_init again when the batch size changes. */
 size_t sol_workspace_bytes(const sol_shape_t *shape, int32_t max_batch, int32_t max_pages_per_seq);
 
 /* Must be called once per workspace before its first use (and may be called
