@@ -62,13 +62,28 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
   pdl_trigger();
   pdl_wait();
 
-  // element `col` of this sequence's q/k/v row: the K slices summed in order, times the quantizer scale
-  const float row_scale = (layer && p.qkv_scale) ? p.qkv_scale[b] : 1.0f;
-  auto qkv_at = [&](int col) -> float {
-    float a = 0.f;
-    for (int z = 0; z < p.ksplit; ++z) a += p.qkv[((size_t)z * p.B + b) * p.ldq + col];
-    return a * row_scale;
-  };
+  // this (sequence, kv-head)'s part of the q/k/v row: G query heads, the k head, the v head.  The K
+  // slices of the projection are summed in order (four loads in flight at a time) and scaled.
+  __shared__ float rowbuf[(8 + 2) * 128];
+  if (layer) {
+    const float row_scale = p.qkv_scale ? p.qkv_scale[b] : 1.0f;
+    const float* base = p.qkv + (size_t)b * p.ldq;
+    const size_t zs = (size_t)p.B * p.ldq;
+    for (int i = tid; i < (G + 2) * hd; i += PREP_THREADS) {
+      const int col = i < G * hd ? kvh * G * hd + i
+                                 : (i < (G + 1) * hd ? Hq * hd + kvh * hd + (i - G * hd)
+                                                     : (Hq + Hkv) * hd + kvh * hd + (i - (G + 1) * hd));
+      float a = 0.f;
+      for (int z0 = 0; z0 < p.ksplit; z0 += 4) {
+        float v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) v[q] = z0 + q < p.ksplit ? base[(size_t)(z0 + q) * zs + col] : 0.f;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) a += v[q];
+      }
+      rowbuf[i] = a * row_scale;
+    }
+  }
 
   if (tid == 0) {
     p.work_ctr[WC_DONE + b * Hkv + kvh] = 0;
@@ -100,7 +115,7 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
     const int gi = i / half, f = i % half, h = kvh * G + gi;
     float q0, q1;
     if (layer) {
-      const float x0 = qkv_at(h * hd + f), x1 = qkv_at(h * hd + f + half);
+      const float x0 = rowbuf[gi * hd + f], x1 = rowbuf[gi * hd + f + half];
       q0 = x0 * cs[f] + (-x1) * sn[f];
       q1 = x1 * cs[f] + x0 * sn[f];
     } else {
@@ -137,14 +152,15 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
   }
   uint16_t* kp = static_cast<uint16_t*>(p.kv.k_pool);
   uint16_t* vp = static_cast<uint16_t*>(p.kv.v_pool);
-  const int kcol = (Hq + kvh) * hd, vcol = (Hq + Hkv + kvh) * hd;
+  const float* kr = rowbuf + G * hd;
+  const float* vr = rowbuf + (G + 1) * hd;
   const size_t dst = (((size_t)page * Hkv + kvh) * PAGE + slot) * hd;
   for (int f = tid; f < half; f += PREP_THREADS) {
-    const float x0 = qkv_at(kcol + f), x1 = qkv_at(kcol + f + half);
+    const float x0 = kr[f], x1 = kr[f + half];
     kp[dst + f] = f2bf(x0 * cs[f] + (-x1) * sn[f]);
     kp[dst + f + half] = f2bf(x1 * cs[f] + x0 * sn[f]);
-    vp[dst + f] = f2bf(qkv_at(vcol + f));
-    vp[dst + f + half] = f2bf(qkv_at(vcol + f + half));
+    vp[dst + f] = f2bf(vr[f]);
+    vp[dst + f + half] = f2bf(vr[f + half]);
   }
 }
 

@@ -589,9 +589,16 @@ __global__ void reduce_out_kernel(const float* __restrict__ partial, int chunks,
   const int i = gi * 4;
   if (i >= M * d) return;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int c = 0; c < chunks; ++c) {
-    const float4 v = *reinterpret_cast<const float4*>(partial + (size_t)c * Mpad * d + i);
-    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+  for (int c0 = 0; c0 < chunks; c0 += 4) {  // four partials' loads in flight, added in order
+    float4 v[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      v[q] = c0 + q < chunks ? *reinterpret_cast<const float4*>(partial + (size_t)(c0 + q) * Mpad * d + i)
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      acc.x += v[q].x; acc.y += v[q].y; acc.z += v[q].z; acc.w += v[q].w;
+    }
   }
   if (resid != nullptr) {
     if (resid_f32) {

@@ -61,11 +61,23 @@ norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, i
         x[i][4] = bf16_lo(w.z); x[i][5] = bf16_hi(w.z); x[i][6] = bf16_lo(w.w); x[i][7] = bf16_hi(w.w);
       }
       if (part != nullptr) {  // partial sums of the projection that produced this row, in slice order
-        for (int z = 0; z < ksplit; ++z) {
-          const float4* q = reinterpret_cast<const float4*>(part + (size_t)z * part_stride + (size_t)row * d) + 2 * v;
-          const float4 a = q[0], b = q[1];
-          x[i][0] += a.x; x[i][1] += a.y; x[i][2] += a.z; x[i][3] += a.w;
-          x[i][4] += b.x; x[i][5] += b.y; x[i][6] += b.z; x[i][7] += b.w;
+        for (int z0 = 0; z0 < ksplit; z0 += 4) {  // four slices' loads in flight, added in slice order
+          float4 a[4], b[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            a[q] = b[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (z0 + q < ksplit) {
+              const float4* src =
+                  reinterpret_cast<const float4*>(part + (size_t)(z0 + q) * part_stride + (size_t)row * d) + 2 * v;
+              a[q] = src[0];
+              b[q] = src[1];
+            }
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            x[i][0] += a[q].x; x[i][1] += a[q].y; x[i][2] += a[q].z; x[i][3] += a[q].w;
+            x[i][4] += b[q].x; x[i][5] += b[q].y; x[i][6] += b[q].z; x[i][7] += b[q].w;
+          }
         }
       }
       if (sum_out != nullptr) {
