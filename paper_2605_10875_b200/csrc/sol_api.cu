@@ -98,10 +98,10 @@ static int pad_rows(int B) {
 }
 
 struct Layout {
-  size_t status, stage_h_in, stage_act, stage_h_out, a_op, scale, qkv, q_rot, q_split, logits, sigma, kept_idx,
-      kept_cnt, part, work_items, kept_row, work_ctr, attn_hi, attn_lo, attn_f32, h_mid, o_part, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, ch_sel, ch_cand_val, ch_cand_idx, ch_keep, down_part,
+  size_t status, stage_h_in, stage_act, stage_h_out, a_op, scale, qkv, attn_hi, attn_lo, attn_f32, h_mid, o_part, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, ch_sel, ch_cand_val, ch_cand_idx, ch_keep, down_part,
       h_a, h_b, total;
-  int splits, chunks, Mpad, Tmax;
+  AttnScratch attn;
+  int chunks, Mpad, Tmax;
 };
 
 static bool shape_ok(const sol_shape_t* s) {
@@ -125,7 +125,6 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   const size_t Mpad = pad_rows(B), Tmax = (size_t)max_pages * s.page_size;
   L.Mpad = (int)Mpad;
   L.Tmax = (int)Tmax;
-  L.splits = attn_splits(s.head_dim, max_pages, s.page_size);
   L.chunks = down_chunks((int)ff, (int)d);
   size_t at = 0;
   auto take = [&](size_t bytes) {
@@ -140,16 +139,8 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   L.a_op = take(Mpad * d * 2);
   L.scale = take(Mpad * 4);
   L.qkv = take((size_t)NK_MAX_KSPLIT * B * Nqkv * 4);  // split-K partial sums of the QKV projection
-  L.q_rot = take(B * Hq * hd * 4);
-  L.q_split = take(B * Hkv * HG * 16 * hd * 2);
-  L.logits = take(B * Hkv * Tmax * G * 4);
-  L.sigma = take(B * Hkv * Tmax * 4);
-  L.kept_idx = take(B * Hkv * Tmax * 4);
-  L.kept_cnt = take(B * Hkv * 4);
-  L.part = take(B * Hkv * L.splits * G * (hd + 2) * 4);
-  L.work_items = take(B * Hkv * (size_t)L.splits * 8);
-  L.kept_row = take(B * Hkv * Tmax * 4);
-  L.work_ctr = take((4 + B * Hkv) * 4);
+  L.attn = attn_scratch_layout(s, B, max_pages, at);
+  at = L.attn.end;
   L.attn_hi = take(Mpad * Hq * hd * 2);
   L.attn_lo = take(Mpad * Hq * hd * 2);
   L.attn_f32 = take(B * Hq * hd * 4);
@@ -209,17 +200,7 @@ static void run_attention(const sol_shape_t& s, const Layout& L, void* ws, const
   a.qkv_ksplit = qkv_ksplit;
   a.qkv_scale = qkv_scale;
   a.q_bf16 = q_bf16;
-  a.q_rot = at<float>(ws, L.q_rot);
-  a.q_split = at<void>(ws, L.q_split);
-  a.logits = at<float>(ws, L.logits);
-  a.sigma = at<float>(ws, L.sigma);
-  a.kept_idx = kept_idx ? kept_idx : at<int32_t>(ws, L.kept_idx);
-  a.kept_cnt = kept_cnt ? kept_cnt : at<int32_t>(ws, L.kept_cnt);
-  a.part = at<float>(ws, L.part);
-  a.splits = attn_splits(s.head_dim, kv.max_pages_per_seq, s.page_size);
-  a.work_items = at<int32_t>(ws, L.work_items);
-  a.kept_row = at<uint32_t>(ws, L.kept_row);
-  a.work_ctr = at<int32_t>(ws, L.work_ctr);
+  attn_scratch_bind(a, ws, L.attn, kept_idx, kept_cnt);
   a.out_f32 = out_f32;
   a.out_bf16 = out_bf16;
   a.out_hi = want_split ? at<void>(ws, L.attn_hi) : nullptr;
@@ -324,7 +305,7 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   run_attention(s, L, ws, kv, B, r, at<float>(ws, L.qkv), Nqkv, nk_ksplit(Nqkv, d), scale, nullptr, nullptr,
                 tr ? tr->attn_out : nullptr, true, tr ? tr->kept_idx : nullptr, tr ? tr->kept_cnt : nullptr, st);
   if (tr && tr->q_rot)
-    cudaMemcpyAsync(tr->q_rot, at<float>(ws, L.q_rot), sizeof(float) * B * Hq * hd, cudaMemcpyDeviceToDevice, st);
+    cudaMemcpyAsync(tr->q_rot, at<float>(ws, L.attn.q_rot), sizeof(float) * B * Hq * hd, cudaMemcpyDeviceToDevice, st);
 
   // output projection, split over K; the second RMSNorm kernel adds the partial sums to the residual
   GemmNK o;

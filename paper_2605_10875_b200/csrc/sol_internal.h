@@ -111,29 +111,37 @@ void launch_reduce_out(const float* partial, int chunks, int M, int Mpad, int d,
                        void* out_bf16, float* out_f32, float* out_f32_b, int32_t* live, int n_live, cudaStream_t st);
 
 // ---- attention (sol_attn.cu) ------------------------------------------------
+// Kept tokens per pass-2 chunk: 32 KB of V rows.
+inline int attn_split_len(int head_dim) { return head_dim == 64 ? 256 : 128; }
+inline int attn_splits(int head_dim, int max_pages, int page_size) {
+  const int len = attn_split_len(head_dim);
+  const int s = (max_pages * page_size + len - 1) / len;
+  return s < 1 ? 1 : s;
+}
 struct AttnArgs {
   sol_shape_t shape;
   sol_kv_t kv;
   int B;
   const int32_t* r_permille;
-  // inputs of the query preparation: either float32 qkv rows [B][ldq] (layer path: rotate q and k,
-  // append k and v) or bf16 q [B][Hq][hd] (stand-alone path: no rotation, no append)
-  const float* qkv_f32;   // [qkv_ksplit][B][ldq] partial sums of the QKV projection
+  // inputs of the query preparation: either the split-K partial sums of the QKV projection (layer
+  // path: rotate q and k, append k and v) or bf16 q [B][Hq][hd] (stand-alone path: no rotation, no append)
+  const float* qkv_f32;   // [qkv_ksplit][B][ldq]
   int ldq;
   int qkv_ksplit;
   const float* qkv_scale; // [B] quantizer scale applied to the summed rows
   const void* q_bf16;
-  // scratch
-  float* q_rot;      // [B][Hq][hd]
-  void* q_split;     // bf16 [B][Hkv][HG*16][hd]
-  float* logits;     // [B][Hkv][Tmax][G]
-  float* sigma;      // [B][Hkv][Tmax]
-  int32_t* kept_idx; // [B][Hkv][Tmax]
-  int32_t* kept_cnt; // [B][Hkv]
-  uint32_t* kept_row; // [B][Hkv][Tmax] cache row (page-resolved) of every kept token, 0xffffffff: bad page
-  float* part;       // [B][Hkv][S][G][hd + 2]
-  int splits;        // S = ceil(Tmax / attn_split_len(hd))
-  int32_t* work_items;  // [B*Hkv*S][2] pass-2 work list (item code, kept count), filled by the selection kernel
+  // scratch (attn_scratch_layout)
+  float* q_rot;         // [B][Hq][hd]
+  void* q_split;        // bf16 [B][Hkv][HG*16][hd]
+  float* logits;        // [B][Hkv][Tmax][G]
+  float* sigma;         // [B][Hkv][Tmax]
+  int32_t* kept_idx;    // [B][Hkv][Tmax] kept tokens, ascending (the caller's array when it asks for the list)
+  int32_t* kept_cnt;    // [B][Hkv]
+  uint32_t* kept_row;   // same layout as kept_idx: cache row (page table applied) of every kept token,
+                        // 0xffffffff: bad page
+  float* part;          // [B][Hkv][S][G][hd + 2]
+  int splits;           // S = ceil(Tmax / attn_split_len(hd))
+  int32_t* work_items;  // [B*Hkv*S][2] pass-2 work list (item code, kept count), filled by the selection
   int32_t* work_ctr;    // [4 + B*Hkv]: items emitted, next item to claim, chunks per item, unused; then the finished
                         // items of every (sequence, kv-head)
   // outputs (each optional)
@@ -143,12 +151,49 @@ struct AttnArgs {
   void* out_lo;
   int* status;
 };
-// Kept tokens per pass-2 work item: 32 KB of V rows.
-inline int attn_split_len(int head_dim) { return head_dim == 64 ? 256 : 128; }
-inline int attn_splits(int head_dim, int max_pages, int page_size) {
-  const int len = attn_split_len(head_dim);
-  const int s = (max_pages * page_size + len - 1) / len;
-  return s < 1 ? 1 : s;
+
+// Offsets of the attention scratch inside a buffer, starting at `at` (a multiple of 256).
+struct AttnScratch {
+  size_t q_rot, q_split, logits, sigma, kept_idx, kept_cnt, kept_row, part, work_items, work_ctr, end;
+  int splits;
+};
+inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_pages, size_t at) {
+  AttnScratch L;
+  const size_t Hq = s.n_q_heads, Hkv = s.n_kv_heads, hd = s.head_dim, G = Hq / Hkv, HG = (G + 3) / 4;
+  const size_t Tmax = (size_t)max_pages * s.page_size, BK = (size_t)B * Hkv;
+  L.splits = attn_splits(s.head_dim, max_pages, s.page_size);
+  auto take = [&](size_t bytes) {
+    const size_t o = at;
+    at += (bytes + 255) / 256 * 256;
+    return o;
+  };
+  L.q_rot = take(B * Hq * hd * 4);
+  L.q_split = take(BK * HG * 16 * hd * 2);
+  L.logits = take(BK * Tmax * G * 4);
+  L.sigma = take(BK * Tmax * 4);
+  L.kept_idx = take(BK * Tmax * 4);
+  L.kept_cnt = take(BK * 4);
+  L.kept_row = take(BK * Tmax * 4);
+  L.part = take(BK * L.splits * G * (hd + 2) * 4);
+  L.work_items = take(BK * L.splits * 8);
+  L.work_ctr = take((4 + BK) * 4);
+  L.end = at;
+  return L;
+}
+// kept_idx / kept_cnt: the caller's arrays, or nullptr to use the scratch.
+inline void attn_scratch_bind(AttnArgs& a, void* base, const AttnScratch& L, int32_t* kept_idx, int32_t* kept_cnt) {
+  unsigned char* b = static_cast<unsigned char*>(base);
+  a.q_rot = reinterpret_cast<float*>(b + L.q_rot);
+  a.q_split = b + L.q_split;
+  a.logits = reinterpret_cast<float*>(b + L.logits);
+  a.sigma = reinterpret_cast<float*>(b + L.sigma);
+  a.kept_idx = kept_idx ? kept_idx : reinterpret_cast<int32_t*>(b + L.kept_idx);
+  a.kept_cnt = kept_cnt ? kept_cnt : reinterpret_cast<int32_t*>(b + L.kept_cnt);
+  a.kept_row = reinterpret_cast<uint32_t*>(b + L.kept_row);
+  a.part = reinterpret_cast<float*>(b + L.part);
+  a.work_items = reinterpret_cast<int32_t*>(b + L.work_items);
+  a.work_ctr = reinterpret_cast<int32_t*>(b + L.work_ctr);
+  a.splits = L.splits;
 }
 void launch_attention(const AttnArgs& a, cudaStream_t st);
 

@@ -45,36 +45,8 @@ sol_status_t scratch_of_current_device(unsigned char** out) {
   return SOL_OK;
 }
 
-struct StaticLayout {
-  size_t status, q_rot, q_split, logits, sigma, kept_idx, kept_cnt, part, work_items, kept_row, work_ctr, total;
-  int splits;
-};
-
-StaticLayout layout_for(const sol_shape_t& s, int B, int max_pages) {
-  StaticLayout L;
-  const size_t Hq = s.n_q_heads, Hkv = s.n_kv_heads, hd = s.head_dim, G = Hq / Hkv, HG = (G + 3) / 4;
-  const size_t Tmax = (size_t)max_pages * s.page_size;
-  L.splits = sol::attn_splits(s.head_dim, max_pages, s.page_size);
-  size_t at = 0;
-  auto take = [&](size_t bytes) {
-    const size_t o = at;
-    at += (bytes + 255) / 256 * 256;
-    return o;
-  };
-  L.status = take(256);
-  L.q_rot = take(B * Hq * hd * 4);
-  L.q_split = take(B * Hkv * HG * 16 * hd * 2);
-  L.logits = take(B * Hkv * Tmax * G * 4);
-  L.sigma = take(B * Hkv * Tmax * 4);
-  L.kept_idx = take(B * Hkv * Tmax * 4);
-  L.kept_cnt = take(B * Hkv * 4);
-  L.part = take(B * Hkv * (size_t)L.splits * G * (hd + 2) * 4);
-  L.work_items = take(B * Hkv * (size_t)L.splits * 8);
-  L.kept_row = take(B * Hkv * Tmax * 4);
-  L.work_ctr = take((4 + B * Hkv) * 4);
-  L.total = at;
-  return L;
-}
+// status words first, then the attention scratch
+constexpr size_t kStatusBytes = 256;
 
 bool attention_shape_ok(const sol_shape_t* s) {
   if (!s) return false;
@@ -96,15 +68,15 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
     return SOL_ERR_INVALID_ARG;
   if (!attention_shape_ok(shape) || B > 128 || kv->max_pages_per_seq > sol::MAX_PAGES_PER_SEQ) return SOL_ERR_UNSUPPORTED;
   if (B == 0) return SOL_OK;
-  const StaticLayout L = layout_for(*shape, B, kv->max_pages_per_seq);
-  if (L.total > kScratchBytes) return SOL_ERR_WORKSPACE_TOO_SMALL;  // the fixed scratch cannot hold this problem
+  const sol::AttnScratch L = sol::attn_scratch_layout(*shape, B, kv->max_pages_per_seq, kStatusBytes);
+  if (L.end > kScratchBytes) return SOL_ERR_WORKSPACE_TOO_SMALL;  // the fixed scratch cannot hold this problem
 
   unsigned char* base = nullptr;
   const sol_status_t s = scratch_of_current_device(&base);
   if (s != SOL_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
   // the array keeps whatever the previous call left; only the status words must start at zero
-  if (sol::record_cuda_error(cudaMemsetAsync(base + L.status, 0, 256, st), "status memset")) return SOL_ERR_CUDA;
+  if (sol::record_cuda_error(cudaMemsetAsync(base, 0, kStatusBytes, st), "status memset")) return SOL_ERR_CUDA;
 
   sol::AttnArgs a;
   a.shape = *shape;
@@ -116,25 +88,15 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
   a.qkv_ksplit = 0;
   a.qkv_scale = nullptr;
   a.q_bf16 = q_bf16;
-  a.q_rot = reinterpret_cast<float*>(base + L.q_rot);
-  a.q_split = base + L.q_split;
-  a.logits = reinterpret_cast<float*>(base + L.logits);
-  a.sigma = reinterpret_cast<float*>(base + L.sigma);
-  a.kept_idx = kept_idx ? kept_idx : reinterpret_cast<int32_t*>(base + L.kept_idx);
-  a.kept_cnt = kept_cnt ? kept_cnt : reinterpret_cast<int32_t*>(base + L.kept_cnt);
-  a.part = reinterpret_cast<float*>(base + L.part);
-  a.splits = L.splits;
-  a.work_items = reinterpret_cast<int32_t*>(base + L.work_items);
-  a.kept_row = reinterpret_cast<uint32_t*>(base + L.kept_row);
-  a.work_ctr = reinterpret_cast<int32_t*>(base + L.work_ctr);
+  sol::attn_scratch_bind(a, base, L, kept_idx, kept_cnt);
   a.out_f32 = nullptr;
   a.out_bf16 = out_bf16;
   a.out_hi = nullptr;
   a.out_lo = nullptr;
-  a.status = reinterpret_cast<int*>(base + L.status);
+  a.status = reinterpret_cast<int*>(base);
   sol::launch_attention(a, st);
   if (status_out != nullptr &&
-      sol::record_cuda_error(cudaMemcpyAsync(status_out, base + L.status, sizeof(int32_t) * sol::ST_WORDS,
+      sol::record_cuda_error(cudaMemcpyAsync(status_out, base, sizeof(int32_t) * sol::ST_WORDS,
                                              cudaMemcpyDeviceToDevice, st), "status copy"))
     return SOL_ERR_CUDA;
   return sol::take_cuda_failure() ? SOL_ERR_CUDA : SOL_OK;
