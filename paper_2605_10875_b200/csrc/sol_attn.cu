@@ -465,7 +465,7 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
   }
   __syncthreads();
   const int batch_chunks = block_count<THREADS>(kb, 0, sm) * Hkv;
-  const int cpi = min(8, max(1, (batch_chunks + p.target_items - 1) / p.target_items));
+  const int cpi = min(ATTN_ITEM_MAX / p.split_len, max(1, (batch_chunks + p.target_items - 1) / p.target_items));
   const int chunks = max(1, (total + p.split_len - 1) / p.split_len);
   const int ns = (chunks + cpi - 1) / cpi;
   if (tid == 0) {
@@ -500,275 +500,215 @@ struct GatherDev {
   int* status;
 };
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-// waits until at most n (0..3) of this thread's copy groups are still in flight
-__device__ __forceinline__ void cp_async_wait_dyn(int n) {
-  if (n <= 0) cp_async_wait<0>();
-  else if (n == 1) cp_async_wait<1>();
-  else if (n == 2) cp_async_wait<2>();
-  else cp_async_wait<3>();
-}
-
-constexpr int GA_WARPS = 4;
+constexpr int GA_WARPS = 8;
 constexpr int GA_THREADS = GA_WARPS * 32;
+constexpr int GA_BATCH = 32;  // kept tokens per warp step: one per lane in the softmax part
+constexpr int GA_ROWS_IN_FLIGHT = 8;  // row loads a lane issues before it consumes the first
 
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
-}
-
+// Pass 2 is a gather of 128- or 256-byte V rows with G multiply-adds per element: bound by memory
+// latency, not by arithmetic, so it runs on the FMA pipes with many warps per SM and no shared-memory
+// staging of the rows.
+//
+// Persistent CTAs work through the list of items: (sequence, kv-head, run of at most 1024 kept tokens);
+// a CTA's first item is dealt by its index, the later ones are claimed from a counter one item ahead.
+// The 8 warps of a CTA take the item's tokens in batches of 32, each warp on its own:
+//   lane l of the warp fetches the index words and the G logits of token l of the batch (the next
+//   batch's while the current one is processed), the warp updates its running maximum per head and
+//   every lane computes its token's softmax weights; cache rows and weights go to a small
+//   shared-memory table; then the warp walks over the batch's rows: a row is read by HD/4 lanes (8
+//   bytes each, 8 rows in flight per lane) and multiplied into the lane's float32 accumulators
+//   (G heads x 4 columns).
+// Per item one partial (accumulators, maximum, sum; merged over the warps) is written; the CTA that
+// finishes the last item of a (sequence, kv-head) merges its partials.
 template <int HD, int GMAX>
-struct GatherLayout {
-  static constexpr int SPLIT = HD == 64 ? 256 : 128;  // kept tokens per chunk (attn_split_len): 32 KB of V rows
-  static constexpr int TPW = SPLIT / GA_WARPS;        // tokens per warp and chunk
-  static constexpr int NT = TPW / 32;                 // tokens per lane and chunk
-  static constexpr int KSTEPS = TPW / 16;             // MMA k-steps per warp and chunk
-  static constexpr int ROW_STRIDE = HD * 2 + 16;      // bytes; +16 keeps ldmatrix rows on distinct banks
-  static constexpr int P_STRIDE = SPLIT + 8;          // bf16 elements; +8 spreads the heads over the banks
-  static constexpr int STAGES = 2;
-  static constexpr int V_BYTES = SPLIT * ROW_STRIDE;
-  static constexpr int LG_BYTES = SPLIT * GMAX * 4;   // logits of the chunk's tokens, [slot][GMAX]
-  static constexpr int STAGE_BYTES = V_BYTES + LG_BYTES;
-  static constexpr int P_BYTES = 2 * GMAX * P_STRIDE * 2;
-  static constexpr int ROWIDX_BYTES = SPLIT * 4;
-  static constexpr int BYTES = STAGES * STAGE_BYTES + P_BYTES + ROWIDX_BYTES + 64;  // 64: flags
-  static_assert(GA_WARPS * GMAX * (HD + 2) * 4 <= V_BYTES, "the merge scratch reuses the first V tile");
-};
-
-// Persistent CTAs claim items from the work list: (sequence, kv-head, run of chunks).  Within an item
-// every warp owns a quarter of each chunk's kept tokens and runs its own two-stage pipeline over the
-// chunks: while chunk c is multiplied, the V rows and the logits of chunk c+1 are in flight (cp.async
-// into the other stage) and the index words of chunk c+2 are being fetched, so only the first chunk of
-// an item pays for the chain indices -> rows.  Softmax weights are relative to a running maximum per
-// head (the accumulators are rescaled when it grows); weights x rows runs on the tensor cores: the
-// weights (bf16 high part in MMA rows 0..G-1, low part in rows 8..8+G-1) are the A operand, the V
-// rows the B operand.  Per item one partial is written; the CTA that finishes the last item of a
-// (sequence, kv-head) merges its partials.
-template <int HD, int GMAX>
-__global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev p) {
-  using L = GatherLayout<HD, GMAX>;
-  extern __shared__ __align__(128) unsigned char smem[];
-  uint16_t* p_hi = reinterpret_cast<uint16_t*>(smem + L::STAGES * L::STAGE_BYTES);
-  uint16_t* p_lo = p_hi + GMAX * L::P_STRIDE;
-  uint32_t* rowidx = reinterpret_cast<uint32_t*>(smem + L::STAGES * L::STAGE_BYTES + L::P_BYTES);
-  int* flag = reinterpret_cast<int*>(smem + L::STAGES * L::STAGE_BYTES + L::P_BYTES + L::ROWIDX_BYTES);
-  float* sc_acc = reinterpret_cast<float*>(smem);  // [GA_WARPS][GMAX][HD], after the MMAs
-  float* sc_ml = sc_acc + GA_WARPS * GMAX * HD;    // [GA_WARPS][GMAX][2]
+__global__ void __launch_bounds__(GA_THREADS, GMAX == 4 ? 4 : 2) attn_gather_kernel(const GatherDev p) {
+  constexpr int SPLIT = HD == 64 ? 256 : 128;  // kept tokens per chunk (attn_split_len): the unit of the item list
+  constexpr int LPT = HD / 4;                  // lanes per row
+  constexpr int TPS = 32 / LPT;                // rows per warp-wide load
+  constexpr int U = GA_ROWS_IN_FLIGHT;
+  static_assert(GA_BATCH % (U * TPS) == 0, "a batch is a whole number of load groups");
+  __shared__ uint32_t s_row[GA_WARPS][GA_BATCH];
+  __shared__ __align__(16) float s_w[GA_WARPS][GA_BATCH][GMAX];
+  __shared__ __align__(16) float sc_acc[GA_WARPS][GMAX][HD];
+  __shared__ float sc_ml[GA_WARPS][GMAX][2];
+  __shared__ __align__(16) int hdr[2][4];  // (sequence, kv-head) or -1, first token, tokens, kept count
+  __shared__ int flag;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = lane >> 2, t = lane & 3;
   const int G = p.G, Hkv = p.Hkv;
   const uint16_t* vp = static_cast<const uint16_t*>(p.kv.v_pool);
-  constexpr int CH = HD / 8;  // 16-byte chunks per row
-  const int tok0 = warp * L::TPW;  // first token slot of this warp within a chunk
-  const int mi = lane >> 3, mr = lane & 7;  // ldmatrix: this lane addresses row mr of matrix mi
+  const int sub = lane / LPT, col = (lane % LPT) * 4;  // which row of a load step, which four columns
   pdl_trigger();
   pdl_wait();
   const int cpi = p.work_ctr[WC_CPI];
+  const int n_items = p.work_ctr[WC_ITEMS];
+  auto header_of = [&](int2 w) {
+    const int bk = w.x / p.S, n0 = (w.x % p.S) * SPLIT;
+    return make_int4(bk, n0, max(0, min(w.y - n0, cpi * SPLIT)), w.y);
+  };
+  if (tid == 0) {
+    int4 h = make_int4(-1, 0, 0, 0);
+    if ((int)blockIdx.x < n_items) h = header_of(*reinterpret_cast<const int2*>(p.work_items + 2 * blockIdx.x));
+    *reinterpret_cast<int4*>(hdr[0]) = h;
+  }
+  __syncthreads();
 
-  for (;;) {
-    if (tid == 0) {
-      const int it = atomicAdd(p.work_ctr + WC_NEXT, 1);
-      int2 h = make_int2(-1, 0);
-      if (it < p.work_ctr[WC_ITEMS]) h = *reinterpret_cast<const int2*>(p.work_items + 2 * it);
-      flag[0] = h.x;
-      flag[2] = h.y;
-    }
-    __syncthreads();
-    const int item = flag[0];
-    if (item < 0) break;
-    const int cnt = flag[2];
-    const int bk = item / p.S, c0 = item % p.S;
+#pragma unroll 1
+  for (int it = 0;; ++it) {
+    const int4 cur = *reinterpret_cast<const int4*>(hdr[it & 1]);
+    if (cur.x < 0) break;
+    int claimed = 0;
+    if (tid == 0) claimed = (int)gridDim.x + atomicAdd(p.work_ctr + WC_NEXT, 1);
+    const int bk = cur.x, len = cur.z, cnt = cur.w;
     const int b = bk / Hkv, kvh = bk % Hkv;
     const size_t row = (size_t)bk * p.Tmax;
-    const int chunks = max(1, (cnt + L::SPLIT - 1) / L::SPLIT);
-    const int nch = min(cpi, chunks - c0);
+    const uint32_t* krow = p.kept_row + row + cur.y;
+    const int32_t* kidx = p.kept_idx + row + cur.y;
+    const float* lgrow = p.logits + row * G;
+    const int nb = (len + GA_BATCH - 1) / GA_BATCH;
 
-    // index words of the chunk that is issued next (kept in registers one chunk ahead)
-    int pj[L::NT];
-    uint32_t pr[L::NT];
-    auto load_idx = [&](int c) {
-#pragma unroll
-      for (int i = 0; i < L::NT; ++i) {
-        const int n = (c0 + c) * L::SPLIT + tok0 + lane + 32 * i;
-        pr[i] = 0xffffffffu;
-        pj[i] = -1;
-        if (c < nch && n < cnt) {
-          pr[i] = p.kept_row[row + n];
-          if (pr[i] != 0xffffffffu) pj[i] = p.kept_idx[row + n];
-        }
+    auto load_idx = [&](int q, uint32_t& r, int& j) {
+      const int n = q * GA_BATCH + lane;
+      r = 0xffffffffu;
+      j = 0;
+      if (q < nb && n < len) {
+        r = krow[n];
+        j = kidx[n];
       }
     };
-    // starts the copies of one chunk (this warp's tokens): logits, then V rows; one commit group
-    auto issue = [&](int stage) {
-      unsigned char* vt = smem + stage * L::STAGE_BYTES;
-      float* lg = reinterpret_cast<float*>(vt + L::V_BYTES);
+    auto load_logits = [&](uint32_t r, int j, float (&x)[GMAX]) {
 #pragma unroll
-      for (int i = 0; i < L::NT; ++i) {
-        const int slot = tok0 + lane + 32 * i;
-        rowidx[slot] = pr[i];
-        float* dst = lg + slot * GMAX;
-        if (pj[i] >= 0) {
-          const float* src = p.logits + (row + pj[i]) * G;
-          if (GMAX == 4 && G == 4) {
-            cp_async16(smem_u32(dst), src);
-          } else {
-            for (int h = 0; h < G; ++h) cp_async4(smem_u32(dst + h), src + h);
-          }
-        } else {
+      for (int h = 0; h < GMAX; ++h) x[h] = -INFINITY;  // an absent token weighs nothing
+      if (r == 0xffffffffu) return;
+      const float* src = lgrow + (size_t)j * G;
+      if (GMAX == 4 && G == 4) {
+        const float4 v = *reinterpret_cast<const float4*>(src);
+        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+      } else {
 #pragma unroll
-          for (int h = 0; h < GMAX; ++h) dst[h] = -INFINITY;  // an absent token weighs nothing
-        }
+        for (int h = 0; h < GMAX; ++h)
+          if (h < G) x[h] = src[h];
       }
-      __syncwarp();
-#pragma unroll
-      for (int ks = 0; ks < L::KSTEPS; ++ks) {
-#pragma unroll
-        for (int i = 0; i < 16 * CH / 32; ++i) {
-          const int c = lane + 32 * i;
-          const int slot = tok0 + ks * 16 + c / CH, ch = c % CH;
-          const uint32_t ridx = rowidx[slot];
-          unsigned char* dst = vt + slot * L::ROW_STRIDE + ch * 16;
-          if (ridx != 0xffffffffu) cp_async16(smem_u32(dst), vp + (size_t)ridx * HD + ch * 8);
-          else *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
-        }
-      }
-      cp_async_commit();
-      __syncwarp();  // rowidx is rewritten by the next issue
     };
 
-    float mh[GMAX], lh[GMAX];
+    float mh[GMAX], ls[GMAX], acc[GMAX][4];
 #pragma unroll
     for (int h = 0; h < GMAX; ++h) {
       mh[h] = -INFINITY;
-      lh[h] = 0.f;
+      ls[h] = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[h][c] = 0.f;
     }
-    float acc[HD / 8][4];
-#pragma unroll
-    for (int nt = 0; nt < HD / 8; ++nt)
-#pragma unroll
-      for (int r = 0; r < 4; ++r) acc[nt][r] = 0.f;
+    uint32_t r_c, r_n;
+    int j_c, j_n;
+    float x_c[GMAX];
+    load_idx(warp, r_c, j_c);
+    load_idx(warp + GA_WARPS, r_n, j_n);
+    load_logits(r_c, j_c, x_c);
 
-    load_idx(0);
-    issue(0);
-    load_idx(1);
 #pragma unroll 1
-    for (int c = 0; c < nch; ++c) {
-      if (c + 1 < nch) {
-        issue((c + 1) & 1);
-        load_idx(c + 2);
-        cp_async_wait<1>();
-      } else {
-        cp_async_wait<0>();
-      }
-      __syncwarp();
-      const unsigned char* vt = smem + (c & 1) * L::STAGE_BYTES;
-      const float* lg = reinterpret_cast<const float*>(vt + L::V_BYTES);
+    for (int q = warp; q < nb; q += GA_WARPS) {
+      // the next batch's logits and the index words of the batch after it start now
+      float x_n[GMAX];
+      load_logits(r_n, j_n, x_n);
+      uint32_t r_nn;
+      int j_nn;
+      load_idx(q + 2 * GA_WARPS, r_nn, j_nn);
 
       // ---- softmax weights relative to the running maximum ----
-      float x[L::NT][GMAX], cm[GMAX];
-#pragma unroll
-      for (int h = 0; h < GMAX; ++h) cm[h] = -INFINITY;
-#pragma unroll
-      for (int i = 0; i < L::NT; ++i) {
-        const float* src = lg + (tok0 + lane + 32 * i) * GMAX;
-#pragma unroll
-        for (int h = 0; h < GMAX; ++h) {
-          x[i][h] = h < G ? src[h] * p.scale_log2 : -INFINITY;
-          cm[h] = fmaxf(cm[h], x[i][h]);
-        }
-      }
-      float my_sc = 1.f;  // rescaling of this lane's accumulator rows (head g, both parts)
 #pragma unroll
       for (int h = 0; h < GMAX; ++h) {
-        const float nm = fmaxf(mh[h], warp_max(cm[h]));
+        const float x = x_c[h] * p.scale_log2;
+        const float nm = fmaxf(mh[h], warp_max(x));
         const float sc = mh[h] == -INFINITY ? 0.f : exp2f(mh[h] - nm);
+        const float pw = x == -INFINITY ? 0.f : exp2f(x - nm);
         mh[h] = nm;
-        lh[h] *= sc;
-        if (h == g) my_sc = sc;
+        ls[h] = ls[h] * sc + pw;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[h][c] *= sc;
+        s_w[warp][lane][h] = pw;
       }
+      s_row[warp][lane] = r_c;
+      __syncwarp();
+
+      // ---- weights x rows ----
+      const int nt = min(GA_BATCH, len - q * GA_BATCH);
+#pragma unroll 1
+      for (int k0 = 0; k0 < nt; k0 += U * TPS) {
+        uint2 v[U];
 #pragma unroll
-      for (int nt = 0; nt < HD / 8; ++nt)
+        for (int u = 0; u < U; ++u) {
+          const uint32_t r = s_row[warp][k0 + u * TPS + sub];
+          v[u] = make_uint2(0u, 0u);
+          if (r != 0xffffffffu) v[u] = __ldcs(reinterpret_cast<const uint2*>(vp + (size_t)r * HD + col));
+        }
 #pragma unroll
-        for (int r = 0; r < 4; ++r) acc[nt][r] *= my_sc;
+        for (int u = 0; u < U; ++u) {
+          const float* w = s_w[warp][k0 + u * TPS + sub];
+          const float f0 = __uint_as_float(v[u].x << 16), f1 = __uint_as_float(v[u].x & 0xffff0000u);
+          const float f2 = __uint_as_float(v[u].y << 16), f3 = __uint_as_float(v[u].y & 0xffff0000u);
 #pragma unroll
-      for (int i = 0; i < L::NT; ++i) {
-        const int slot = tok0 + lane + 32 * i;
+          for (int h4 = 0; h4 < GMAX; h4 += 4) {
+            const float4 w4 = *reinterpret_cast<const float4*>(w + h4);
+            const float ww[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
-        for (int h = 0; h < GMAX; ++h) {
-          if (h < G) {
-            const float pw = x[i][h] == -INFINITY ? 0.f : exp2f(x[i][h] - mh[h]);
-            lh[h] += pw;
-            const uint16_t hi = f2bf(pw);
-            p_hi[h * L::P_STRIDE + slot] = hi;
-            p_lo[h * L::P_STRIDE + slot] = f2bf(pw - bf2f(hi));
+            for (int e = 0; e < 4; ++e) {
+              acc[h4 + e][0] = fmaf(ww[e], f0, acc[h4 + e][0]);
+              acc[h4 + e][1] = fmaf(ww[e], f1, acc[h4 + e][1]);
+              acc[h4 + e][2] = fmaf(ww[e], f2, acc[h4 + e][2]);
+              acc[h4 + e][3] = fmaf(ww[e], f3, acc[h4 + e][3]);
+            }
           }
         }
       }
-      __syncwarp();
+      __syncwarp();  // the tables are rewritten for the next batch
+      r_c = r_n;
+      j_c = j_n;
+#pragma unroll
+      for (int h = 0; h < GMAX; ++h) x_c[h] = x_n[h];
+      r_n = r_nn;
+      j_n = j_nn;
+    }
 
-      // ---- weights x rows on the tensor cores ----
+    // ---- one partial per item: merge the warps ----
+    if (TPS == 2) {  // two rows per load step: the half-warps hold partial sums of the same columns
 #pragma unroll
-      for (int ks = 0; ks < L::KSTEPS; ++ks) {
-        const int kb = tok0 + ks * 16;
-        uint32_t a0 = 0, a1 = 0, a2 = 0, a3 = 0;
-        if (g < G) {
-          a0 = *reinterpret_cast<const uint32_t*>(p_hi + g * L::P_STRIDE + kb + 2 * t);
-          a1 = *reinterpret_cast<const uint32_t*>(p_lo + g * L::P_STRIDE + kb + 2 * t);
-          a2 = *reinterpret_cast<const uint32_t*>(p_hi + g * L::P_STRIDE + kb + 8 + 2 * t);
-          a3 = *reinterpret_cast<const uint32_t*>(p_lo + g * L::P_STRIDE + kb + 8 + 2 * t);
-        }
-        const uint32_t vrow = smem_u32(vt) + (kb + (mi & 1) * 8 + mr) * L::ROW_STRIDE;
+      for (int h = 0; h < GMAX; ++h)
 #pragma unroll
-        for (int pr2 = 0; pr2 < HD / 16; ++pr2) {
-          uint32_t bfr[4];
-          ldsm_x4_trans(bfr, vrow + ((2 * pr2 + (mi >> 1)) * 8) * 2);
-          mma_bf16(acc[2 * pr2], a0, a1, a2, a3, bfr[0], bfr[1]);
-          mma_bf16(acc[2 * pr2 + 1], a0, a1, a2, a3, bfr[2], bfr[3]);
-        }
-      }
-      __syncwarp();  // the weights and this stage are rewritten from here on
+        for (int c = 0; c < 4; ++c) acc[h][c] += __shfl_xor_sync(0xffffffffu, acc[h][c], 16);
     }
 #pragma unroll
-    for (int h = 0; h < GMAX; ++h) lh[h] = warp_sum(lh[h]);
-    __syncthreads();  // every warp is done with the stages: the first becomes the merge scratch
-
-    if (g < G) {
+    for (int h = 0; h < GMAX; ++h) ls[h] = warp_sum(ls[h]);
+    if (sub == 0) {
 #pragma unroll
-      for (int nt = 0; nt < HD / 8; ++nt) {
-        float* d = sc_acc + ((size_t)(warp * GMAX + g) * HD) + nt * 8 + 2 * t;
-        d[0] = acc[nt][0] + acc[nt][2];
-        d[1] = acc[nt][1] + acc[nt][3];
-      }
+      for (int h = 0; h < GMAX; ++h)
+        *reinterpret_cast<float4*>(&sc_acc[warp][h][col]) = make_float4(acc[h][0], acc[h][1], acc[h][2], acc[h][3]);
     }
     if (lane == 0) {
 #pragma unroll
       for (int h = 0; h < GMAX; ++h) {
-        sc_ml[(warp * GMAX + h) * 2] = mh[h];
-        sc_ml[(warp * GMAX + h) * 2 + 1] = lh[h];
+        sc_ml[warp][h][0] = mh[h];
+        sc_ml[warp][h][1] = ls[h];
       }
     }
+    // the header of the claimed item is fetched while the partial is put together
+    int2 claimed_words = make_int2(0, 0);
+    if (tid == 0 && claimed < n_items) claimed_words = *reinterpret_cast<const int2*>(p.work_items + 2 * claimed);
     __syncthreads();
-    const int slot_no = c0 / cpi;  // this item's partial
+    const int slot_no = (cur.y / SPLIT) / cpi;  // this item's partial
     float* dst = p.part + (((size_t)bk * p.S + slot_no) * G) * (HD + 2);
-    for (int i = tid; i < G * HD; i += GA_THREADS) {
-      const int h = i / HD, e = i % HD;
+    for (int e0 = tid; e0 < G * HD; e0 += GA_THREADS) {
+      const int h = e0 / HD, e = e0 % HD;
       float M = -INFINITY;
 #pragma unroll
-      for (int w = 0; w < GA_WARPS; ++w) M = fmaxf(M, sc_ml[(w * GMAX + h) * 2]);
+      for (int w = 0; w < GA_WARPS; ++w) M = fmaxf(M, sc_ml[w][h][0]);
       float a = 0.f, l = 0.f;
 #pragma unroll
       for (int w = 0; w < GA_WARPS; ++w) {
-        const float mw = sc_ml[(w * GMAX + h) * 2];
+        const float mw = sc_ml[w][h][0];
         const float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
-        a += sc_acc[(size_t)(w * GMAX + h) * HD + e] * f;
-        l += sc_ml[(w * GMAX + h) * 2 + 1] * f;
+        a += sc_acc[w][h][e] * f;
+        l += sc_ml[w][h][1] * f;
       }
       dst[h * (HD + 2) + e] = a;
       if (e == 0) {
@@ -778,16 +718,22 @@ __global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev
     }
 
     // ---- the last item of this (sequence, kv-head) merges the partials ----
+    const int chunks = max(1, (cnt + SPLIT - 1) / SPLIT);
     const int ns = (chunks + cpi - 1) / cpi;
     __threadfence();
     __syncthreads();
-    if (tid == 0) flag[1] = atomicAdd(p.work_ctr + WC_DONE + bk, 1) == ns - 1 ? 1 : 0;
+    if (tid == 0) {
+      flag = atomicAdd(p.work_ctr + WC_DONE + bk, 1) == ns - 1 ? 1 : 0;
+      int4 h = make_int4(-1, 0, 0, 0);
+      if (claimed < n_items) h = header_of(claimed_words);
+      *reinterpret_cast<int4*>(hdr[(it + 1) & 1]) = h;
+    }
     __syncthreads();
-    if (flag[1]) {
+    if (flag) {
       __threadfence();
       const float* src0 = p.part + ((size_t)bk * p.S * G) * (HD + 2);
-      for (int i = tid; i < G * HD; i += GA_THREADS) {
-        const int h = i / HD, e = i % HD;
+      for (int e0 = tid; e0 < G * HD; e0 += GA_THREADS) {
+        const int h = e0 / HD, e = e0 % HD;
         float m = -INFINITY, l = 0.f, a = 0.f;
         for (int q = 0; q < ns; ++q) {
           const float* src = src0 + ((size_t)q * G + h) * (HD + 2);
@@ -810,7 +756,7 @@ __global__ void __launch_bounds__(GA_THREADS) attn_gather_kernel(const GatherDev
         }
       }
     }
-    __syncthreads();  // the scratch and the flags are reused by the next item
+    __syncthreads();  // the merge scratch, the flag and the headers are reused by the next item
   }
 }
 
@@ -829,11 +775,19 @@ static void launch_score(const ScoreDev& d, int HG, dim3 grid, cudaStream_t st) 
   }
 }
 
+// One CTA per item, at most as many CTAs as are resident at once (they are persistent).
 template <int HD, int GMAX>
-static void launch_gather(const GatherDev& d, int grid, cudaStream_t st) {
-  using L = GatherLayout<HD, GMAX>;
-  ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_gather_kernel<HD, GMAX>), L::BYTES);
-  SOL_LAUNCH("attn_gather_v", (attn_gather_kernel<HD, GMAX>), dim3(grid), dim3(GA_THREADS), L::BYTES, st, d);
+static void launch_gather(const GatherDev& d, long long items, cudaStream_t st) {
+  static int per_sm = 0;  // the same on every device this library supports
+  if (per_sm == 0) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attn_gather_kernel<HD, GMAX>, GA_THREADS, 0) != cudaSuccess || n < 1)
+      n = 1;
+    per_sm = n;
+  }
+  const long long resident = (long long)sm_count() * per_sm;
+  const int grid = (int)(items < resident ? items : resident);
+  SOL_LAUNCH("attn_gather_v", (attn_gather_kernel<HD, GMAX>), dim3(grid), dim3(GA_THREADS), 0, st, d);
 }
 
 void launch_attention(const AttnArgs& a, cudaStream_t st) {
@@ -880,13 +834,12 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   gd.out_hi = static_cast<uint16_t*>(a.out_hi); gd.out_lo = static_cast<uint16_t*>(a.out_lo);
   gd.status = a.status;
   const long long items = (long long)a.B * Hkv * a.splits;
-  const int grid = (int)(items < (long long)sm_count() * 2 ? items : (long long)sm_count() * 2);
   if (hd == 64) {
-    if (G <= 4) launch_gather<64, 4>(gd, grid, st);
-    else launch_gather<64, 8>(gd, grid, st);
+    if (G <= 4) launch_gather<64, 4>(gd, items, st);
+    else launch_gather<64, 8>(gd, items, st);
   } else {
-    if (G <= 4) launch_gather<128, 4>(gd, grid, st);
-    else launch_gather<128, 8>(gd, grid, st);
+    if (G <= 4) launch_gather<128, 4>(gd, items, st);
+    else launch_gather<128, 8>(gd, items, st);
   }
 }
 
