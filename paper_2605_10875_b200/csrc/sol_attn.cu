@@ -288,17 +288,22 @@ struct SelectDev {
   int* status;
 };
 
-// One CTA per (sequence, kv-head).  Every thread keeps KPT consecutive scores in registers (as order-
-// preserving keys) for all passes; candidates near the threshold are settled in float64.
-template <int THREADS, int KPT>
+// One CTA per (sequence, kv-head).  Every thread owns `per` consecutive tokens; their scores sit in
+// shared memory (as order-preserving keys, slot i of thread t at [i * THREADS + t]) for all passes, and
+// every loop over them is a rolled one: the kernel is a long chain of short passes, and unrolled over
+// register arrays it spent more time waiting for instructions than for data.  Candidates near the
+// threshold are settled in float64.
+template <int THREADS>
 __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p) {
   __shared__ SelectSmem sm;
   __shared__ double qsum[128];
+  extern __shared__ __align__(16) uint32_t skey[];  // [per][THREADS]
 
   const int kvh = blockIdx.x, b = blockIdx.y;
   const int Hkv = p.sh.n_kv_heads, hd = p.sh.head_dim, G = p.sh.n_q_heads / Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int WARPS = THREADS / 32;
+  constexpr int KPT = 0;  // rolled key loops
   const int bk = b * Hkv + kvh;
   pdl_trigger();
   pdl_wait();
@@ -307,8 +312,9 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
   const float* sig = p.sigma + row;
   // a thread owns `per` consecutive tokens: as few as this sequence needs (a multiple of 4 for the
   // vector loads), so a short context in a long-context batch costs what its own length costs
-  const int per = min(KPT, ((max(T, 1) + THREADS - 1) / THREADS + 3) / 4 * 4);
+  const int per = ((max(T, 1) + THREADS - 1) / THREADS + 3) / 4 * 4;
   const int j0 = tid * per;
+  auto key = [&](int i) { return skey[i * THREADS + tid]; };  // 0: absent, 0xffffffff: forced
 
   int total = 0;
   if (T > 0) {
@@ -321,22 +327,24 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
     auto forced = [&](int j) { return j < n_sink || j >= T - n_win; };
     if (tid < 4) sm.counts[tid] = 0;
 
-    // mode 0: keep all; 1: forced only; 2: kept iff score above the window or a candidate decided in
-    // float64; 3: key threshold with index-ordered ties (float32 ordering, candidate list overflowed)
-    int mode, tie_need = 0, n_cand = 0;
+    // mode 0: keep all; 1: forced only; 2: the key slots hold classes (settled by the window pass and
+    // the float64 ranking); 3: key threshold with index-ordered ties (float32 ordering, the candidate
+    // list overflowed)
+    constexpr uint32_t CLS_DROP = 0u, CLS_KEEP = 2u, CLS_CAND = 3u;
+    int mode, tie_need = 0;
     uint32_t key_thr = 0;
-    float hi = 0.f, lo = 0.f;
-    uint32_t key[KPT];  // 0: absent, 0xffffffff: forced
+    int my_keep = 0, my_ties = 0;  // of this thread's tokens: kept for sure, tied at the threshold
 
     if (k >= T) {
       mode = 0;
+      my_keep = min(max(T - j0, 0), per);
     } else if (k <= nf) {
       mode = 1;
+      for (int i = 0; i < per; ++i) my_keep += j0 + i < T && forced(j0 + i);
     } else {
       float mx = 0.f;
-#pragma unroll
-      for (int i = 0; i < KPT; i += 4) {
-        if (i >= per) break;
+#pragma unroll 1
+      for (int i = 0; i < per; i += 4) {
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (j0 + i < T) v = *reinterpret_cast<const float4*>(sig + j0 + i);
         const float vv[4] = {v.x, v.y, v.z, v.w};
@@ -353,39 +361,49 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
               mx = fmaxf(mx, fabsf(sv));
             }
           }
-          key[i + e] = kk;
+          skey[(i + e) * THREADS + tid] = kk;
         }
       }
       mx = block_max<THREADS>(mx, 0, sm);
-      key_thr = select_kth<THREADS, KPT>(key, k, tie_need, sm, per);
-      mode = 3;
+      key_thr = select_kth<THREADS, KPT, true>(key, k, tie_need, sm, per);
 
       // ---- window around the threshold, re-scored in float64 ----
       const float thr32 = key_to_float(key_thr);
       // 2^-16 of the largest score: far above the float32 accumulation error of a head_dim-long dot product
       const float delta = mx * 1.52587890625e-05f;
-      hi = thr32 + delta;
-      lo = thr32 - delta;
-      int n_in = 0;
-#pragma unroll
-      for (int i = 0; i < KPT; ++i) {
-        if (i >= per) break;
-        const uint32_t kk = key[i];
-        if (kk == 0u || kk == 0xffffffffu) continue;
-        const float sv = key_to_float(kk);
-        if (sv > hi) {
-          ++n_in;
-        } else if (sv >= lo) {
-          const int slot = atomicAdd(&sm.counts[0], 1);
-          if (slot < SEL_CAND_CAP) sm.cand_idx[slot] = j0 + i;
+      const float hi = thr32 + delta, lo = thr32 - delta;
+      // One pass counts what is clear of the window and lists the candidates inside it.
+      int n_in = 0, my_cand = 0;
+#pragma unroll 1
+      for (int i = 0; i < per; ++i) {
+        const uint32_t kk = key(i);
+        if (kk == 0xffffffffu) {
+          ++my_keep;
+        } else if (kk != 0u) {
+          const float sv = key_to_float(kk);
+          if (sv > hi) {
+            ++n_in;
+          } else if (sv >= lo) {
+            ++my_cand;
+            const int slot = atomicAdd(&sm.counts[0], 1);
+            if (slot < SEL_CAND_CAP) sm.cand_idx[slot] = j0 + i;
+          }
         }
       }
+      my_keep += n_in;
       n_in = block_count<THREADS>(n_in, 0, sm);
-      n_cand = sm.counts[0];
+      const int n_cand = sm.counts[0];
       const int need = k - nf - n_in;
       if (n_cand > SEL_CAND_CAP) {
         if (tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
-        n_cand = 0;
+        mode = 3;
+        my_keep = 0;
+#pragma unroll 1
+        for (int i = 0; i < per; ++i) {
+          const uint32_t kk = key(i);
+          my_keep += kk > key_thr && kk != 0u;
+          my_ties += kk == key_thr;
+        }
       } else {
         if (n_cand != need) {
           if (tid == 0) atomicAdd(p.status + ST_TOK_REFINED, n_cand);
@@ -414,24 +432,35 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
         }
         mode = 2;
         __syncthreads();
+        // the key slot of every candidate takes its class: a kept one sorts above every key, a dropped
+        // one below (token j is slot j % per of thread j / per), so that one comparison with the window
+        // classifies any slot from here on
+        for (int c = tid; c < n_cand; c += THREADS) {
+          const int j = sm.cand_idx[c];
+          skey[(j % per) * THREADS + j / per] = sm.cand_keep[c] ? 0xffffffffu : 0u;
+        }
+        __syncthreads();
+        if (my_cand > 0) {  // few threads own candidates: they count their kept ones
+#pragma unroll 1
+          for (int i = 0; i < per; ++i) {
+            const uint32_t kk = key(i);
+            // a forced token or a kept candidate now; the forced ones were counted above
+            my_keep += kk == 0xffffffffu && !(j0 + i < T && forced(j0 + i));
+          }
+        }
+        key_thr = float_key(hi);  // kept: keys above the window (candidates inside it are settled)
       }
     }
 
+    // class of this thread's i-th token: 2 kept, 1 tie, 0 dropped
     auto klass = [&](int i) -> int {
       const int j = j0 + i;
       if (j >= T) return 0;
-      if (mode == 0 || forced(j)) return 2;
-      if (mode == 2) {
-        const float sv = key_to_float(key[i]);
-        if (sv > hi) return 2;
-        if (sv >= lo) {  // within the window: look the token up in the decided list
-          for (int q = 0; q < n_cand; ++q)
-            if (sm.cand_idx[q] == j) return sm.cand_keep[q] ? 2 : 0;
-        }
-        return 0;
-      }
-      if (mode == 3) return key[i] > key_thr ? 2 : (key[i] == key_thr ? 1 : 0);
-      return 0;
+      if (mode == 0) return 2;
+      if (mode == 1) return forced(j) ? 2 : 0;
+      const uint32_t kk = key(i);
+      if (mode == 2) return kk > key_thr ? 2 : 0;
+      return kk > key_thr ? 2 : (kk == key_thr ? 1 : 0);
     };
     // beside the index list, the cache row of every kept token (page table applied), so that pass 2
     // goes from the list straight to the V rows
@@ -445,7 +474,8 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
       else atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
       p.kept_row[row + pos] = ridx;
     };
-    total = compact_indices<THREADS, KPT>(klass, emit, mode == 3 ? tie_need : 0, p.kept_idx + row, sm, per);
+    total = compact_counted<THREADS, KPT>(my_keep, my_ties, klass, emit, mode == 3 ? tie_need : 0, p.kept_idx + row,
+                                          sm, per);
   }
   if (tid == 0) p.kept_cnt[bk] = total;
 
@@ -816,12 +846,17 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   se.sigma = a.sigma; se.kept_idx = a.kept_idx; se.kept_cnt = a.kept_cnt; se.kept_row = a.kept_row;
   se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
   {
+    // keys of the longest row in shared memory: 4 bytes per token, rounded up to four per thread
     const dim3 grid(Hkv, a.B);
-    if (Tmax <= 1024) SOL_LAUNCH("token_select", (token_select_kernel<256, 4>), grid, dim3(256), 0, st, se);
-    else if (Tmax <= 4096) SOL_LAUNCH("token_select", (token_select_kernel<256, 16>), grid, dim3(256), 0, st, se);
-    else if (Tmax <= 16384) SOL_LAUNCH("token_select", (token_select_kernel<1024, 16>), grid, dim3(1024), 0, st, se);
-    else if (Tmax <= 32768) SOL_LAUNCH("token_select", (token_select_kernel<1024, 32>), grid, dim3(1024), 0, st, se);
-    else SOL_LAUNCH("token_select", (token_select_kernel<1024, 48>), grid, dim3(1024), 0, st, se);
+    if (Tmax <= 1024) {
+      const int smem = ((Tmax + 256 - 1) / 256 + 3) / 4 * 4 * 256 * 4;
+      ensure_dynamic_smem(reinterpret_cast<const void*>(&token_select_kernel<256>), smem);
+      SOL_LAUNCH("token_select", token_select_kernel<256>, grid, dim3(256), smem, st, se);
+    } else {
+      const int smem = ((Tmax + 1024 - 1) / 1024 + 3) / 4 * 4 * 1024 * 4;
+      ensure_dynamic_smem(reinterpret_cast<const void*>(&token_select_kernel<1024>), smem);
+      SOL_LAUNCH("token_select", token_select_kernel<1024>, grid, dim3(1024), smem, st, se);
+    }
   }
 
   GatherDev gd;

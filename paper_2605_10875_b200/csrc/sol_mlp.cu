@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
   } else {
     gmax = block_max<THREADS>(gmax, 0, sm);
     umax = block_max<THREADS>(umax, 1, sm);
-    key_thr = select_kth<THREADS, KPT>(key, m, tie_need, sm);
+    key_thr = select_kth<THREADS, KPT>([&](int i) { return key[i]; }, m, tie_need, sm, KPT);
     mode = 3;
     const float thr32 = key_to_float(key_thr);
     // error taken for g_j, u_j: the tensor cores add each 16-long slice of the dot product to the running
@@ -246,7 +246,8 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
     }
   };
   // the index list itself is written by channel_list from the mask; here it goes to the candidate scratch
-  const int total = compact_indices<THREADS, KPT>(klass, emit, mode == 3 ? tie_need : 0, p.scratch_idx + (size_t)b * ff, sm);
+  const int total =
+      compact_indices<THREADS, KPT>(klass, emit, mode == 3 ? tie_need : 0, p.scratch_idx + (size_t)b * ff, sm, KPT);
   if (tid == 0) p.kept_cnt[b] = total;
 }
 
@@ -471,7 +472,7 @@ __global__ void __launch_bounds__(THREADS) channel_list_kernel(const unsigned ch
   const int b = blockIdx.x, j0 = threadIdx.x * KPT;
   const unsigned char* k = keep + (size_t)b * ff;
   auto klass = [&](int i) -> int { return (j0 + i < ff && k[j0 + i]) ? 2 : 0; };
-  compact_indices<THREADS, KPT>(klass, [](int, bool, int) {}, 0, kept_ch + (size_t)b * ff, sm);
+  compact_indices<THREADS, KPT>(klass, [](int, bool, int) {}, 0, kept_ch + (size_t)b * ff, sm, KPT);
 }
 
 void launch_channel_select(const ChannelSelectArgs& a, cudaStream_t st) {

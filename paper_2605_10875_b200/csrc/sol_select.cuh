@@ -1,8 +1,11 @@
 // Block-wide exact top-k building blocks shared by the token and the channel
 // selection kernels (one CTA per selection problem).
 //
-// Every thread holds KPT consecutive 32-bit keys in registers (key order =
-// value order, see float_key); nothing is re-read from memory between passes.
+// Every thread owns a run of consecutive elements whose 32-bit keys (key order
+// = value order, see float_key) are read through an accessor key(i): a
+// register array walked by fully unrolled loops (KPT > 0), or shared memory
+// walked by rolled loops (KPT == 0: small code, any run length); nothing is
+// re-read from global memory between passes.
 //
 //   select_kth        the k-th largest key of the block (histogram of the top
 //                     key bits, then exact ranking inside the threshold bin),
@@ -17,7 +20,7 @@
 namespace sol {
 
 constexpr int SEL_CAND_CAP = 1024;
-constexpr int SEL_RANK_CAP = 32;  // a threshold bin this small is ranked exactly instead of split further
+constexpr int SEL_RANK_CAP = 128;  // a threshold bin this small is ranked exactly instead of split further
 constexpr int SEL_BINS = 4096;
 constexpr int SEL_MAX_WARPS = 32;
 
@@ -33,36 +36,65 @@ struct SelectSmem {
   int counts[4];
 };
 
+// f(i) for the first `per` elements of a thread: unrolled over KPT register slots, or (KPT == 0) a
+// rolled loop.
+template <int KPT, typename F>
+__device__ __forceinline__ void for_keys(int per, F f) {
+  if constexpr (KPT > 0) {
+#pragma unroll
+    for (int i = 0; i < KPT; ++i) {
+      if (i >= per) break;
+      f(i);
+    }
+  } else {
+#pragma unroll 1
+    for (int i = 0; i < per; ++i) f(i);
+  }
+}
+
 // Inverse of float_key.
 __device__ __forceinline__ float key_to_float(uint32_t key) {
   return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
 }
 
-// The k-th largest of the block's keys (1 <= k <= number of keys).  Only the first per_thread keys of
-// every thread take part.  Absent elements carry key 0 and count like any other key, so k must not
+// Order-preserving bin (0..4095) of a key by the value it stands for: the sign, then 32 binades of
+// magnitude (2^-18 .. 2^14, clamped at both ends) with 64 steps each.  Keys of one sign, binade and
+// step share their upper 15 bits, so a bin that is not a clamped one is a key prefix.  Scores spread
+// over hundreds of these bins where the upper 12 key bits (3 mantissa bits) put most of them into a
+// dozen, which serialises the shared-memory atomics of the histogram.
+constexpr int VB_EXP0 = 109;  // biased exponent of the smallest resolved binade
+__device__ __forceinline__ int key_value_bin(uint32_t key) {
+  const uint32_t u = (key & 0x80000000u) ? (key & 0x7fffffffu) : ~key;  // the float's bits
+  int m = (int)((u & 0x7fffffffu) >> 17) - (VB_EXP0 << 6);
+  m = min(max(m, 0), SEL_BINS / 2 - 1);
+  return (u >> 31) ? SEL_BINS / 2 - 1 - m : SEL_BINS / 2 + m;
+}
+
+// The k-th largest of the block's keys (1 <= k <= number of keys); key(i), i < per_thread, are a
+// thread's keys.  Absent elements carry key 0 and count like any other key, so k must not
 // exceed the number of present elements.  tie_need = how many
 // keys equal to the result belong to the top k.  All threads call.
 //
-// One histogram pass over the top 12 key bits (shared-memory atomics) finds the bin that holds the
-// k-th key; if that bin is small its keys are listed and ranked exactly, otherwise the next 12 (then
-// the last 8) bits are histogrammed within it.
-template <int THREADS, int KPT>
-__device__ __forceinline__ uint32_t select_kth(const uint32_t (&key)[KPT], int k, int& tie_need, SelectSmem& sm,
-                                               int per_thread = KPT) {
+// A histogram pass (shared-memory atomics) finds the bin that holds the k-th key; if that bin is small
+// its keys are listed and ranked exactly, otherwise the next key bits are histogrammed within it.
+// Plain schedule: 12 + 12 + 8 key bits.  VALUE_BINS: the first pass uses key_value_bin (15 key bits
+// unless the bin is a clamped one, then the plain schedule starts over), then 12 + 5 bits.
+template <int THREADS, int KPT, bool VALUE_BINS = false, typename KeyFn, typename Smem>
+__device__ __forceinline__ uint32_t select_kth(KeyFn key, int k, int& tie_need, Smem& sm, int per_thread) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint32_t prefix = 0, mask = 0;
   int remaining = k, pop = 0;
-#pragma unroll 1
-  for (int level = 0; level < 3; ++level) {
-    const int bits = level == 2 ? 8 : 12, shift = level == 0 ? 20 : (level == 1 ? 8 : 0);
-    const int nb = 1 << bits;
+  // One pass: histogram of digit(key) (negative: the key does not take part) over nb bins, then the bin
+  // that holds rank `remaining` (bins in descending order).  Leaves bin, keys above it, its size in sm.pick.
+  auto run_level = [&](int nb, auto digit) {
     for (int i = tid; i < nb; i += THREADS) sm.hist[i] = 0;
     __syncthreads();
-#pragma unroll
-    for (int i = 0; i < KPT; ++i)
-      if (i < per_thread && (key[i] & mask) == prefix) atomicAdd(&sm.hist[(key[i] >> shift) & (uint32_t)(nb - 1)], 1u);
+    for_keys<KPT>(per_thread, [&](int i) {
+      const int d = digit(key(i));
+      if (d >= 0) atomicAdd(&sm.hist[d], 1u);
+    });
     __syncthreads();
-    // bins in descending order: thread t owns bins nb-1-t*bpt .. nb-bpt-t*bpt
+    // thread t owns bins nb-1-t*bpt .. nb-bpt-t*bpt
     const int bpt = nb >= THREADS ? nb / THREADS : 1;
     const bool active = tid * bpt < nb;
     int mine = 0;
@@ -93,11 +125,37 @@ __device__ __forceinline__ uint32_t select_kth(const uint32_t (&key)[KPT], int k
       }
     }
     __syncthreads();
+  };
+  auto radix_level = [&](int bits, int shift) {
+    const uint32_t dm = (1u << bits) - 1u;
+    run_level(1 << bits, [&](uint32_t kk) { return (kk & mask) == prefix ? (int)((kk >> shift) & dm) : -1; });
     prefix |= (uint32_t)sm.pick[0] << shift;
-    mask |= (uint32_t)(nb - 1) << shift;
+    mask |= dm << shift;
     remaining -= sm.pick[1];
     pop = sm.pick[2];
-    if (pop <= SEL_RANK_CAP) break;
+  };
+
+  bool done = false;
+  if (VALUE_BINS) {
+    run_level(SEL_BINS, [&](uint32_t kk) { return key_value_bin(kk); });
+    const int bin = sm.pick[0];
+    const int m = bin >= SEL_BINS / 2 ? bin - SEL_BINS / 2 : SEL_BINS / 2 - 1 - bin;
+    if (m >= 1 && m < SEL_BINS / 2 - 1) {  // not a clamped bin: its keys share their upper 15 bits
+      const uint32_t u = (uint32_t)(m + (VB_EXP0 << 6)) << 17;
+      prefix = bin >= SEL_BINS / 2 ? (u | 0x80000000u) : (~(u | 0x80000000u) & 0xfffe0000u);
+      mask = 0xfffe0000u;
+      remaining -= sm.pick[1];
+      pop = sm.pick[2];
+      if (pop > SEL_RANK_CAP) radix_level(12, 5);
+      if (pop > SEL_RANK_CAP) radix_level(5, 0);
+      done = true;
+    }
+    __syncthreads();  // sm.pick is rewritten by the passes below
+  }
+  if (!done) {
+    radix_level(12, 20);
+    if (pop > SEL_RANK_CAP) radix_level(12, 8);
+    if (pop > SEL_RANK_CAP) radix_level(8, 0);
   }
   if (mask == 0xffffffffu) {  // every bit decided: the keys left are all equal to the result
     tie_need = remaining;
@@ -106,9 +164,10 @@ __device__ __forceinline__ uint32_t select_kth(const uint32_t (&key)[KPT], int k
   // list the keys under the prefix and rank them exactly
   if (tid == 0) sm.counts[2] = 0;
   __syncthreads();
-#pragma unroll
-  for (int i = 0; i < KPT; ++i)
-    if (i < per_thread && (key[i] & mask) == prefix) sm.rank_key[atomicAdd(&sm.counts[2], 1)] = key[i];
+  for_keys<KPT>(per_thread, [&](int i) {
+    const uint32_t kk = key(i);
+    if ((kk & mask) == prefix) sm.rank_key[atomicAdd(&sm.counts[2], 1)] = kk;
+  });
   __syncthreads();
   for (int c = tid; c < pop; c += THREADS) {
     const uint32_t kc = sm.rank_key[c];
@@ -166,24 +225,33 @@ __device__ __forceinline__ void rank_candidates(int n_cand, int need, SelectSmem
   }
 }
 
-// klass(i) in {0 dropped, 1 tie, 2 kept} for element j = tid*per_thread + i, i < per_thread <= KPT (called
-// twice per element; a thread's elements beyond per_thread must be class 0).  Ties
+// klass(i) in {0 dropped, 1 tie, 2 kept} for element j = first + tid*per_thread + i, i < per_thread (called
+// twice per element).  Ties
 // are kept in ascending index order until tie_need runs out.  Kept indices go to out[] ascending;
 // emit(i, keep, pos) reports the final decision of every element and, for a kept one, its place in out[].  Returns the kept total to every thread.
 // All threads call; uses sm.scan.
-template <int THREADS, int KPT, typename ClassFn, typename EmitFn>
-__device__ __forceinline__ int compact_indices(ClassFn klass, EmitFn emit, int tie_need, int32_t* out, SelectSmem& sm,
-                                               int per_thread = KPT) {
-  constexpr int WARPS = THREADS / 32;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+template <int THREADS, int KPT, typename ClassFn, typename EmitFn, typename Smem>
+__device__ __forceinline__ int compact_counted(int c2, int c1, ClassFn klass, EmitFn emit, int tie_need, int32_t* out,
+                                               Smem& sm, int per_thread, int first = 0);
+
+template <int THREADS, int KPT, typename ClassFn, typename EmitFn, typename Smem>
+__device__ __forceinline__ int compact_indices(ClassFn klass, EmitFn emit, int tie_need, int32_t* out, Smem& sm,
+                                               int per_thread, int first = 0) {
   int c2 = 0, c1 = 0;
-#pragma unroll
-  for (int i = 0; i < KPT; ++i) {
-    if (i >= per_thread) break;
+  for_keys<KPT>(per_thread, [&](int i) {
     const int c = klass(i);
     c2 += c == 2;
     c1 += c == 1;
-  }
+  });
+  return compact_counted<THREADS, KPT>(c2, c1, klass, emit, tie_need, out, sm, per_thread, first);
+}
+
+// The same when the caller already knows how many of its elements are of class 2 (c2) and 1 (c1).
+template <int THREADS, int KPT, typename ClassFn, typename EmitFn, typename Smem>
+__device__ __forceinline__ int compact_counted(int c2, int c1, ClassFn klass, EmitFn emit, int tie_need, int32_t* out,
+                                               Smem& sm, int per_thread, int first) {
+  constexpr int WARPS = THREADS / 32;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // exclusive prefix of ties over the block (threads in index order), then of kept elements
   int t_incl = c1;
 #pragma unroll
@@ -213,10 +281,8 @@ __device__ __forceinline__ int compact_indices(ClassFn klass, EmitFn emit, int t
     total += v;
   }
   int ties_left = my_ties;
-  const int j0 = threadIdx.x * per_thread;
-#pragma unroll
-  for (int i = 0; i < KPT; ++i) {
-    if (i >= per_thread) break;
+  const int j0 = first + threadIdx.x * per_thread;
+  for_keys<KPT>(per_thread, [&](int i) {
     const int c = klass(i);
     bool kp = c == 2;
     if (c == 1 && ties_left > 0) {
@@ -226,7 +292,7 @@ __device__ __forceinline__ int compact_indices(ClassFn klass, EmitFn emit, int t
     if (kp) out[pos] = j0 + i;
     emit(i, kp, pos);
     if (kp) ++pos;
-  }
+  });
   __syncthreads();  // sm.scan may be reused by the caller
   return total;
 }
