@@ -173,6 +173,10 @@ struct ScoreDev {
   const uint16_t* q_split;
   float* logits;
   float* sigma;
+  // for the choice of the pass-2 item length
+  int B, n_sink, n_window, split_len, target_items;
+  const int32_t* r_permille;
+  int32_t* work_ctr;
   int* status;
 };
 
@@ -192,6 +196,43 @@ __global__ void __launch_bounds__(SC_WARPS * 32) attn_score_kernel(const ScoreDe
   }
   __syncthreads();
   pdl_wait();
+
+  // Length of the pass-2 work items, in chunks of split_len kept tokens (the first CTA finds it for the batch,
+  // from the kept counts the budgets imply): the smallest run length (up to ATTN_ITEM_CHUNKS) that gives
+  // every resident CTA of pass 2 at most one item, so that there is no second, partly filled round of
+  // items; when even the longest runs leave more items than CTAs there is work for many rounds, and runs
+  // of 8 chunks, claimed one by one, balance it.
+  if (blockIdx.x == 0 && kvh == 0 && b == 0) {
+    __shared__ int n_items[ATTN_ITEM_CHUNKS];
+        if (threadIdx.x < ATTN_ITEM_CHUNKS) n_items[threadIdx.x] = 0;
+    __syncthreads();
+    for (int i0 = warp * 32; i0 < p.B; i0 += SC_WARPS * 32) {  // one sequence per lane
+      const int i = i0 + lane;
+      int ch = 0;
+      if (i < p.B) {
+        const int Ti = min(p.kv.seq_lens[i], p.kv.max_pages_per_seq * PAGE);
+        ch = 1;
+        if (Ti > 0) {
+          const int ns_ = min(max(p.n_sink, 0), Ti), nw_ = min(max(p.n_window, 0), Ti - ns_);
+          long long bd = ((long long)p.r_permille[i] * Ti + 999) / 1000;
+          if (bd > Ti) bd = Ti;
+          ch = max(1, (min(Ti, max((int)bd, ns_ + nw_)) + p.split_len - 1) / p.split_len);
+        }
+      }
+#pragma unroll
+      for (int c = 1; c <= ATTN_ITEM_CHUNKS; ++c) {
+        const int n = __reduce_add_sync(0xffffffffu, (ch + c - 1) / c);
+        if (lane == 0) atomicAdd(&n_items[c - 1], n);
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int cpi = 8;
+      for (int c = ATTN_ITEM_CHUNKS; c >= 1; --c)
+        if ((long long)n_items[c - 1] * p.Hkv <= p.target_items) cpi = c;
+      p.work_ctr[WC_CPI] = cpi;
+    }
+  }
 
   const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
   const int lp = blockIdx.x * SC_WARPS + warp;  // logical page
@@ -277,7 +318,7 @@ struct SelectDev {
   sol_shape_t sh;
   sol_kv_t kv;
   const int32_t* r_permille;
-  int Tmax, S, split_len, B, target_items;
+  int Tmax, S, split_len, B;
   const float* q_rot;
   const float* sigma;
   int32_t* kept_idx;
@@ -480,28 +521,11 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
   if (tid == 0) p.kept_cnt[bk] = total;
 
   // Pass-2 work items of this (sequence, kv-head): runs of `cpi` chunks of split_len kept tokens (at least
-  // one item, so that the output is always written).  cpi is the same in every CTA: it is sized from the
-  // kept count of the whole batch so that the batch yields about target_items items: few, long items
-  // amortise the per-item work, enough of them keep every SM busy.
-  int kb = 0;
-  for (int i = tid; i < p.B; i += THREADS) {
-    const int Ti = min(p.kv.seq_lens[i], p.kv.max_pages_per_seq * PAGE);
-    if (Ti > 0) {
-      const int ns_ = min(max(p.sh.n_sink, 0), Ti), nw_ = min(max(p.sh.n_window, 0), Ti - ns_);
-      long long bd = ((long long)p.r_permille[i] * Ti + 999) / 1000;
-      if (bd > Ti) bd = Ti;
-      kb += (min(Ti, max((int)bd, ns_ + nw_)) + p.split_len - 1) / p.split_len;
-    }
-  }
-  __syncthreads();
-  const int batch_chunks = block_count<THREADS>(kb, 0, sm) * Hkv;
-  const int cpi = min(ATTN_ITEM_MAX / p.split_len, max(1, (batch_chunks + p.target_items - 1) / p.target_items));
+  // one item, so that the output is always written); cpi was chosen by the query preparation kernel.
+  const int cpi = p.work_ctr[WC_CPI];
   const int chunks = max(1, (total + p.split_len - 1) / p.split_len);
   const int ns = (chunks + cpi - 1) / cpi;
-  if (tid == 0) {
-    sm.counts[3] = atomicAdd(p.work_ctr + WC_ITEMS, ns);
-    p.work_ctr[WC_CPI] = cpi;
-  }
+  if (tid == 0) sm.counts[3] = atomicAdd(p.work_ctr + WC_ITEMS, ns);
   __syncthreads();
   const int base = sm.counts[3];
   for (int i = tid; i < ns; i += THREADS) {
@@ -836,17 +860,21 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   sd.kv = a.kv; sd.Hkv = Hkv; sd.G = G; sd.HG = HG; sd.Tmax = Tmax;
   sd.q_split = static_cast<const uint16_t*>(a.q_split);
   sd.logits = a.logits; sd.sigma = a.sigma; sd.status = a.status;
+  sd.B = a.B; sd.n_sink = sh.n_sink; sd.n_window = sh.n_window; sd.split_len = attn_split_len(hd);
+  sd.target_items = sm_count() * (G <= 4 ? 4 : 2);  // the pass-2 CTAs resident at once
+  sd.r_permille = a.r_permille; sd.work_ctr = a.work_ctr;
   dim3 sgrid((a.kv.max_pages_per_seq + SC_WARPS - 1) / SC_WARPS, Hkv, a.B);
   if (hd == 64) launch_score<64>(sd, HG, sgrid, st);
   else launch_score<128>(sd, HG, sgrid, st);
 
   SelectDev se;
   se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.S = a.splits;
-  se.split_len = attn_split_len(hd); se.q_rot = a.q_rot; se.B = a.B; se.target_items = 3 * sm_count();
+  se.split_len = attn_split_len(hd); se.q_rot = a.q_rot; se.B = a.B;
   se.sigma = a.sigma; se.kept_idx = a.kept_idx; se.kept_cnt = a.kept_cnt; se.kept_row = a.kept_row;
   se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
   {
-    // keys of the longest row in shared memory: 4 bytes per token, rounded up to four per thread
+    // keys of the longest row in shared memory: 4 bytes per token, rounded up to four per thread; rows up
+    // to 1024 tokens take 256 threads, longer ones 1024
     const dim3 grid(Hkv, a.B);
     if (Tmax <= 1024) {
       const int smem = ((Tmax + 256 - 1) / 256 + 3) / 4 * 4 * 256 * 4;

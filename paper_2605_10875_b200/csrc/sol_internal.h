@@ -118,7 +118,7 @@ inline int attn_splits(int head_dim, int max_pages, int page_size) {
   const int s = (max_pages * page_size + len - 1) / len;
   return s < 1 ? 1 : s;
 }
-constexpr int ATTN_ITEM_MAX = 1024;  // kept tokens per pass-2 work item at most
+constexpr int ATTN_ITEM_CHUNKS = 16;  // chunks of attn_split_len kept tokens per pass-2 work item at most
 struct AttnArgs {
   sol_shape_t shape;
   sol_kv_t kv;
