@@ -190,6 +190,10 @@ __global__ void __launch_bounds__(SC_WARPS * 32) attn_score_kernel(const ScoreDe
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.z, kvh = blockIdx.y;
   pdl_trigger();
+  // The grid covers the longest row the page table allows; the CTAs beyond this sequence's length leave
+  // before anything else (the lengths are an input of the step, not the work of an earlier kernel).  The
+  // first CTA stays: it also sizes the pass-2 items.
+  if (blockIdx.x * SC_WARPS * PAGE >= p.kv.seq_lens[b] && (blockIdx.x | blockIdx.y | blockIdx.z) != 0) return;
   if (threadIdx.x == 0) {
     for (int i = 0; i < SC_WARPS; ++i) mbar_init(&bars[i], 1);
     fence_mbar_init();
