@@ -282,7 +282,9 @@ __global__ void __launch_bounds__(CM_THREADS) channel_select_multi_kernel(const 
   if (tid == 0) sm.n_local = 0;
 
   // ---- the histogram bin of the m-th largest |t| (every CTA of the token finds the same one) ----
-  float hi_edge = 0.f, lo_edge = 0.f;  // keep at or above hi_edge, drop below lo_edge, exact in between
+  // keep at or above hi_edge + e_j, drop below lo_edge - e_j, exact in between; e_j = eps * (1.1 |u_j| + |g_j|)
+  // bounds the error of this channel's own float32 |t|
+  float hi_edge = 0.f, lo_edge = 0.f, eps = 0.f;
   if (m >= ff) {
     hi_edge = 0.f;  // everything is kept
     lo_edge = 0.f;
@@ -323,16 +325,24 @@ __global__ void __launch_bounds__(CM_THREADS) channel_select_multi_kernel(const 
     // error taken for g_j, u_j: the tensor cores add each 16-long slice of the dot product to the running
     // float32 sum with truncation, so the error grows with the d/16 steps: (d/16) * 2^-24 of the largest
     // magnitude, and never less than 2^-18 of it; carried into t through |silu'| <= 1.1, |silu(g)| <= |g|
-    const float eps = fmaxf(3.814697265625e-06f, (float)(d / 16) * 5.9604644775390625e-08f) * fmaxf(gmax, umax);
-    const float delta = 2.0f * eps * (1.1f * umax + gmax) + 1e-6f * (tb >= CH_BINS - 1 ? bin_lo : bin_hi);
+    eps = fmaxf(3.814697265625e-06f, (float)(d / 16) * 5.9604644775390625e-08f) * fmaxf(gmax, umax);
+    // the m-th largest exact |t| lies within the largest error any channel can carry of the bin; a channel is
+    // settled when its own error cannot carry it across that
+    const float delta = eps * (1.1f * umax + gmax) + 1e-6f * (tb >= CH_BINS - 1 ? bin_lo : bin_hi);
     lo_edge = bin_lo - delta;
     hi_edge = bin_hi + delta;
   }
 
   // ---- classify this CTA's channels ----
-  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (in) v = *reinterpret_cast<const float4*>(p.t + (size_t)b * ff + j0);
-  const float vv[4] = {v.x, v.y, v.z, v.w};
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f), gq = v, uq = v;
+  if (in) {
+    v = *reinterpret_cast<const float4*>(p.t + (size_t)b * ff + j0);
+    if (eps > 0.f) {
+      gq = *reinterpret_cast<const float4*>(p.g + (size_t)b * ff + j0);
+      uq = *reinterpret_cast<const float4*>(p.u + (size_t)b * ff + j0);
+    }
+  }
+  const float vv[4] = {v.x, v.y, v.z, v.w}, gg[4] = {gq.x, gq.y, gq.z, gq.w}, uu[4] = {uq.x, uq.y, uq.z, uq.w};
   uint32_t hw[2] = {0, 0}, lw[2] = {0, 0}, kw = 0;
   int n_above = 0;
   bool any = false;
@@ -340,7 +350,8 @@ __global__ void __launch_bounds__(CM_THREADS) channel_select_multi_kernel(const 
   for (int e = 0; e < 4; ++e) {
     const float a = fabsf(vv[e]);
     if (!in) continue;
-    if (a >= hi_edge) {
+    const float ej = eps * (1.1f * fabsf(uu[e]) + fabsf(gg[e]));
+    if (a >= hi_edge + ej) {
       const uint16_t hv = f2bf(vv[e]);
       const uint16_t lv = f2bf(vv[e] - bf2f(hv));
       hw[e >> 1] |= (uint32_t)hv << (16 * (e & 1));
@@ -348,7 +359,7 @@ __global__ void __launch_bounds__(CM_THREADS) channel_select_multi_kernel(const 
       kw |= 1u << (8 * e);
       ++n_above;
       any = true;
-    } else if (a >= lo_edge) {
+    } else if (a >= lo_edge - ej) {
       sm.local_idx[atomicAdd(&sm.n_local, 1)] = j0 + e;
     }
   }
