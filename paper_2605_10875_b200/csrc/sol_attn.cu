@@ -419,7 +419,7 @@ __global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p
       const float hi = thr32 + delta, lo = thr32 - delta;
       // One pass counts what is clear of the window and lists the candidates inside it.
       int n_in = 0, my_cand = 0;
-#pragma unroll 1
+#pragma unroll 4
       for (int i = 0; i < per; ++i) {
         const uint32_t kk = key(i);
         if (kk == 0xffffffffu) {

@@ -46,9 +46,17 @@ __device__ __forceinline__ void for_keys(int per, F f) {
       if (i >= per) break;
       f(i);
     }
-  } else {
+  } else {  // four at a time: the loads of a group are independent, the loop overhead is shared
+    int i = 0;
 #pragma unroll 1
-    for (int i = 0; i < per; ++i) f(i);
+    for (; i + 4 <= per; i += 4) {
+      f(i);
+      f(i + 1);
+      f(i + 2);
+      f(i + 3);
+    }
+#pragma unroll 1
+    for (; i < per; ++i) f(i);
   }
 }
 

@@ -150,6 +150,11 @@ def test_attention_head_dim_128_ragged():
     _attention_case(cfg, lens, [125, 1000, 500, 250, 500], seed=5)
 
 
+def test_attention_head_dim_128_group_of_8():
+    cfg = dict(L8B, n_q_heads=16, n_kv_heads=2)
+    _attention_case(cfg, [700, 64, 1500, 129], [250, 500, 125, 1000], seed=8, n_sink=1, n_window=2)
+
+
 @pytest.mark.parametrize("hq,hkv", [(8, 1), (4, 4), (12, 2)])
 def test_attention_other_group_sizes(hq, hkv):
     cfg = dict(TINY, n_q_heads=hq, n_kv_heads=hkv, d_model=256 if (hq * 64) % 256 == 0 else 768)
