@@ -150,6 +150,13 @@ def test_attention_head_dim_128_ragged():
     _attention_case(cfg, lens, [125, 1000, 500, 250, 500], seed=5)
 
 
+def test_attention_longest_supported_row():
+    """768 pages = 49152 tokens, the longest row the library takes (its selection keeps every key of the
+    row in shared memory), next to a short one."""
+    par, st, _ = _attention_case(TINY, [49152, 300], [125, 500], seed=9, n_sink=4, n_window=2)
+    assert par.sets == 2 * TINY["n_kv_heads"]
+
+
 def test_attention_head_dim_128_group_of_8():
     cfg = dict(L8B, n_q_heads=16, n_kv_heads=2)
     _attention_case(cfg, [700, 64, 1500, 129], [250, 500, 125, 1000], seed=8, n_sink=1, n_window=2)
