@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
   pdl_wait();
 
   // this (sequence, kv-head)'s part of the q/k/v row: G query heads, the k head, the v head.  The K
-  // slices of the projection are summed in order (eight loads in flight at a time) and scaled.
+  // slices of the projection are summed in order (four loads in flight at a time) and scaled.
   __shared__ float rowbuf[(8 + 2) * 128];
   if (layer) {
     const float row_scale = p.qkv_scale ? p.qkv_scale[b] : 1.0f;
@@ -74,12 +74,12 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
                                  : (i < (G + 1) * hd ? Hq * hd + kvh * hd + (i - G * hd)
                                                      : (Hq + Hkv) * hd + kvh * hd + (i - (G + 1) * hd));
       float a = 0.f;
-      for (int z0 = 0; z0 < p.ksplit; z0 += 8) {
-        float v[8];
+      for (int z0 = 0; z0 < p.ksplit; z0 += 4) {
+        float v[4];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) v[q] = z0 + q < p.ksplit ? base[(size_t)(z0 + q) * zs + col] : 0.f;
+        for (int q = 0; q < 4; ++q) v[q] = z0 + q < p.ksplit ? base[(size_t)(z0 + q) * zs + col] : 0.f;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) a += v[q];
+        for (int q = 0; q < 4; ++q) a += v[q];
       }
       rowbuf[i] = a * row_scale;
     }

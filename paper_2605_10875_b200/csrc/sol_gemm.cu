@@ -589,14 +589,14 @@ __global__ void reduce_out_kernel(const float* __restrict__ partial, int chunks,
   const int i = gi * 4;
   if (i >= M * d) return;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int c0 = 0; c0 < chunks; c0 += 8) {  // eight partials' loads in flight, added in order
-    float4 v[8];
+  for (int c0 = 0; c0 < chunks; c0 += 4) {  // four partials' loads in flight, added in order
+    float4 v[4];
 #pragma unroll
-    for (int q = 0; q < 8; ++q)
+    for (int q = 0; q < 4; ++q)
       v[q] = c0 + q < chunks ? *reinterpret_cast<const float4*>(partial + (size_t)(c0 + q) * Mpad * d + i)
                              : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
+    for (int q = 0; q < 4; ++q) {
       acc.x += v[q].x; acc.y += v[q].y; acc.z += v[q].z; acc.w += v[q].w;
     }
   }
