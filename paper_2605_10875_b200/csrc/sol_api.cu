@@ -501,6 +501,16 @@ sol_status_t sol_decode_step(const sol_shape_t* shape, int32_t n_layers, const s
                           p_permille, bits, ws, L, (cudaStream_t)stream);
 }
 
+// The per-sequence actions and lengths of a step (at most 128 sequences) travel as kernel parameters:
+// one launch instead of four small host-to-device copies, and the values are taken at the call.
+struct StepActions {
+  int32_t v[4][128];  // keep-rate, prune rate, bit-width, sequence length
+};
+__global__ void upload_actions_kernel(const StepActions a, int B, int32_t* __restrict__ dst) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < 4 * B) dst[i] = a.v[i / B][i % B];
+}
+
 sol_status_t sol_decode_step_host(const sol_shape_t* shape, int32_t n_layers, const sol_layer_weights_t* layers,
                                   const sol_kv_t* kvs, int32_t B, const void* h_in_bf16_host, void* h_out_bf16_host,
                                   const int32_t* r_permille_host, const int32_t* p_permille_host,
@@ -527,10 +537,15 @@ sol_status_t sol_decode_step_host(const sol_shape_t* shape, int32_t n_layers, co
   int32_t* act = at<int32_t>(ws, L.stage_act);
   bool bad = false;
   bad |= record_cuda_error(cudaMemcpyAsync(at<void>(ws, L.stage_h_in), h_in_bf16_host, hb, cudaMemcpyHostToDevice, st), "h2d h_in");
-  bad |= record_cuda_error(cudaMemcpyAsync(act, r_permille_host, ab, cudaMemcpyHostToDevice, st), "h2d r");
-  bad |= record_cuda_error(cudaMemcpyAsync(act + B, p_permille_host, ab, cudaMemcpyHostToDevice, st), "h2d p");
-  bad |= record_cuda_error(cudaMemcpyAsync(act + 2 * B, bits_host, ab, cudaMemcpyHostToDevice, st), "h2d bits");
-  bad |= record_cuda_error(cudaMemcpyAsync(act + 3 * B, seq_lens_host, ab, cudaMemcpyHostToDevice, st), "h2d seq_lens");
+  {
+    StepActions sa;
+    memcpy(sa.v[0], r_permille_host, ab);
+    memcpy(sa.v[1], p_permille_host, ab);
+    memcpy(sa.v[2], bits_host, ab);
+    memcpy(sa.v[3], seq_lens_host, ab);
+    upload_actions_kernel<<<(4 * B + 127) / 128, 128, 0, st>>>(sa, B, act);
+    bad |= record_cuda_error(cudaGetLastError(), "upload of the actions");
+  }
   if (bad) return finish();
   s = decode_step_impl(shape, n_layers, layers, kvs, act + 3 * B, B, at<void>(ws, L.stage_h_in),
                        at<void>(ws, L.stage_h_out), nullptr, act, act + B, act + 2 * B, ws, L, st);
