@@ -203,11 +203,12 @@ sol_status_t sol_decode_step(const sol_shape_t *shape, int32_t n_layers, const s
 
 /* The same step for a caller whose per-step data lives on the HOST: h_in,
  * the three action arrays, seq_lens and h_out are host pointers (pinned
- * memory makes the copies asynchronous).  They are copied to staging areas
- * inside the workspace, the step runs with kvs[l].seq_lens replaced by the
- * staged copy, and the result is copied back; the call returns after the
- * stream has been synchronised.  Weights, pools and page tables stay on the
- * device. */
+ * memory makes the copies of h_in and h_out asynchronous; the four int32
+ * arrays are read during the call and travel as kernel parameters).  They
+ * land in staging areas inside the workspace, the step runs with
+ * kvs[l].seq_lens replaced by the staged copy, and the result is copied back;
+ * the call returns after the stream has been synchronised.  Weights, pools and
+ * page tables stay on the device. */
 sol_status_t sol_decode_step_host(const sol_shape_t *shape, int32_t n_layers, const sol_layer_weights_t *layers,
                                   const sol_kv_t *kvs, int32_t B, const void *h_in_bf16_host,
                                   void *h_out_bf16_host, const int32_t *r_permille_host,
