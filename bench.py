@@ -281,32 +281,62 @@ def timed_steps(rep, steps, warmup, barrier, fn):
     return e0.elapsed_time(e1)  # ms
 
 
+class Ranks:
+    """The process-group side of the benchmark: one process per GPU, every rank an independent replica.
+    The ranks meet only at barriers and to take the slowest rank's time; `backend` "gloo" with device
+    "cpu" runs the same plumbing without a GPU (the multi-process tests)."""
+
+    def __init__(self, backend="nccl", device=None):
+        import torch
+        import torch.distributed as dist
+
+        self.torch, self.dist = torch, dist
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        self.device = device if device is not None else f"cuda:{self.local}"
+        if self.world > 1:
+            if backend == "nccl":
+                dist.init_process_group("nccl", device_id=torch.device(self.device))
+            else:
+                dist.init_process_group(backend)
+
+    @property
+    def is_root(self):
+        return self.rank == 0
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+
+    def max_over_ranks(self, ms):
+        if self.world == 1:
+            return ms
+        t = self.torch.tensor([ms], dtype=self.torch.float64, device=self.device)
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def whole_job_rate(self, steps_per_rank, ms):
+        """Steps per second of all ranks together: every rank ran steps_per_rank steps in (at most) ms."""
+        return self.world * steps_per_rank / (ms / 1e3)
+
+    def close(self):
+        if self.world > 1:
+            self.dist.barrier()
+            self.dist.destroy_process_group()
+
+
 def run_ours(args):
     import torch
-    import torch.distributed as dist
 
     from paper_2605_10875_b200 import binding as sol
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
-    torch.cuda.set_device(local)
-    device = f"cuda:{local}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(device))
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-
-    def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    ranks = Ranks("nccl")
+    world, rank, local, device = ranks.world, ranks.rank, ranks.local, ranks.device
+    barrier, max_over_ranks = ranks.barrier, ranks.max_over_ranks
 
     sol.lib()
     cfg = synth.WORKLOADS[args.workload]
@@ -325,7 +355,7 @@ def run_ours(args):
     launches = sol.launch_count(reset=True) * args.steps // (args.steps + args.warmup)
     status = sol.read_device_status(rep.ws)
     ms_per_step = ms / args.steps
-    value = world * args.steps / (ms / 1e3)
+    value = ranks.whole_job_rate(args.steps, ms)
 
     # --- the same steps with per-kernel CUDA events, for the dominant kernel's roofline ---
     prof_steps = min(args.steps, 200)
@@ -359,7 +389,7 @@ def run_ours(args):
     e2e_steps = min(args.steps, 500)
     ms_e2e = max_over_ranks(timed_steps(rep, e2e_steps, 3, barrier, rep.step_host))
     hb = rep.B * cfg["d_model"] * 2
-    e2e = {"value": round(world * e2e_steps / (ms_e2e / 1e3), 2), "unit": UNIT, "steps": e2e_steps,
+    e2e = {"value": round(ranks.whole_job_rate(e2e_steps, ms_e2e), 2), "unit": UNIT, "steps": e2e_steps,
            "h2d_bytes_per_step": hb + 4 * rep.B * 4, "d2h_bytes_per_step": hb}
 
     # --- budget sweep: every sequence with the same action ---
@@ -411,9 +441,7 @@ def run_ours(args):
             "budget_sweep": sweep,
         }
         print(json.dumps(line, default=_plain), flush=True)
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    ranks.close()
     return line
 
 

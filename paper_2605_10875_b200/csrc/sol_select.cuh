@@ -102,12 +102,12 @@ __device__ __forceinline__ uint32_t select_kth(KeyFn key, int k, int& tie_need, 
       if (d >= 0) atomicAdd(&sm.hist[d], 1u);
     });
     __syncthreads();
-    // thread t owns bins nb-1-t*bpt .. nb-bpt-t*bpt
-    const int bpt = nb >= THREADS ? nb / THREADS : 1;
+    // thread t owns bins nb-1-t*bpt .. nb-bpt-t*bpt (those that exist)
+    const int bpt = (nb + THREADS - 1) / THREADS;
     const bool active = tid * bpt < nb;
     int mine = 0;
     if (active)
-      for (int q = 0; q < bpt; ++q) mine += (int)sm.hist[nb - 1 - tid * bpt - q];
+      for (int q = 0; q < bpt && nb - 1 - tid * bpt - q >= 0; ++q) mine += (int)sm.hist[nb - 1 - tid * bpt - q];
     int incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -122,6 +122,7 @@ __device__ __forceinline__ uint32_t select_kth(KeyFn key, int k, int& tie_need, 
       int a = before;
       for (int q = 0; q < bpt; ++q) {
         const int bin = nb - 1 - tid * bpt - q;
+        if (bin < 0) break;
         const int c = (int)sm.hist[bin];
         if (remaining <= a + c) {
           sm.pick[0] = bin;
