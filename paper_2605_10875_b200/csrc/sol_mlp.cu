@@ -263,6 +263,7 @@ struct ChanMultiSmem {
   int n_local;
   int flag;
   int local_idx[CM_SLICE];
+  __align__(16) uint16_t x[8192];  // the token's operand row (d_model <= 8192)
   double val[CH_CAND_CAP];
   int idx[CH_CAND_CAP];
 };
@@ -379,27 +380,31 @@ __global__ void __launch_bounds__(CM_THREADS) channel_select_multi_kernel(const 
   const int n_local = sm.n_local;
   if (n_local > 0) {
     const double sc = (double)p.scale[b];
-    const uint16_t* x = p.a_op + (size_t)b * d;
+    // the token's operand row, shared by all candidates of the CTA
+    for (int e = tid * 8; e < d; e += CM_THREADS * 8)
+      *reinterpret_cast<uint4*>(sm.x + e) = *reinterpret_cast<const uint4*>(p.a_op + (size_t)b * d + e);
+    __syncthreads();
     for (int c = warp; c < n_local; c += WARPS) {
       const int j = sm.local_idx[c];
       const uint16_t* wg = p.w_gate + (size_t)j * d;
       const uint16_t* wu = p.w_up + (size_t)j * d;
       float gh = 0.f, gl = 0.f, uh = 0.f, ul = 0.f;
-      for (int e0 = lane * 8; e0 < d; e0 += 1024) {  // four 256-wide slices per round, loads before uses
-        uint4 xv[4], gv[4], uv[4];
+      for (int e0 = lane * 8; e0 < d; e0 += 2048) {  // eight 256-wide slices of both rows per round, loads before uses
+        uint4 gv[8], uv[8];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
+        for (int r = 0; r < 8; ++r) {
           const int e = e0 + r * 256;
           if (e < d) {
-            xv[r] = *reinterpret_cast<const uint4*>(x + e);
             gv[r] = *reinterpret_cast<const uint4*>(wg + e);
             uv[r] = *reinterpret_cast<const uint4*>(wu + e);
           }
         }
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          if (e0 + r * 256 >= d) break;
-          const uint32_t xa[4] = {xv[r].x, xv[r].y, xv[r].z, xv[r].w}, ga[4] = {gv[r].x, gv[r].y, gv[r].z, gv[r].w},
+        for (int r = 0; r < 8; ++r) {
+          const int e = e0 + r * 256;
+          if (e >= d) break;
+          const uint4 xv = *reinterpret_cast<const uint4*>(sm.x + e);
+          const uint32_t xa[4] = {xv.x, xv.y, xv.z, xv.w}, ga[4] = {gv[r].x, gv[r].y, gv[r].z, gv[r].w},
                          ua[4] = {uv[r].x, uv[r].y, uv[r].z, uv[r].w};
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
