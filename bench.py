@@ -42,12 +42,12 @@ SERVE_REDRAW = 16  # ... and steps between two draws of the per-sequence actions
 # the ncu capture summarised under profiles/, keyed by (workload, kernel); absent -> null.
 NCU_TRAFFIC_BYTES = {
     # profiles/ncu_full_llama1b_layer_all_kernels.txt (one launch each, same workload and actions)
-    ("llama1b_layer", "attn_score"): 67395328 + 1481216,
-    ("llama1b_layer", "attn_gather_v"): 34698752 + 4352,
-    ("llama1b_layer", "gemm_gate_up_swiglu"): 67371264 + 875008,
-    ("llama1b_layer", "gemm_down_gathered"): 34107136 + 0,
+    ("llama1b_layer", "attn_score"): 67394816 + 1545216,
+    ("llama1b_layer", "attn_gather_v"): 34699008 + 6656,
+    ("llama1b_layer", "gemm_gate_up_swiglu"): 67371264 + 910848,
+    ("llama1b_layer", "gemm_down_gathered"): 34107392 + 0,
     ("llama1b_layer", "gemm_qkv"): 12682240 + 0,
-    ("llama1b_layer", "gemm_out_proj"): 8553728 + 0,
+    ("llama1b_layer", "gemm_out_proj"): 8553216 + 0,
 }
 
 
