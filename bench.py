@@ -10,6 +10,11 @@ the step on its own GPU: the path needs no exchange between sequences, so
 there is no collective in the data path; the ranks meet only at the barriers
 around the timed region and the slowest rank's time is reported.
 
+The default workload is the ragged serving mix (the largest configuration: 16
+layers, batch 128, contexts 256..32768, consecutive steps that append, actions
+redrawn every 16 steps); the same run also times the other four workloads
+compactly (`per_workload`) and a small-batch prune-rate sweep.
+
 `--impl reference` times the CPU oracle on the host cores instead (a
 deliberately plain fp64 program; a reported baseline, not a target).
 """
@@ -38,17 +43,26 @@ ROTATE = 4  # distinct copies of weights + cache, cycled so that no step finds i
 SERVE_STEPS = 64   # ragged serving workload: consecutive steps that append before the contexts start over
 SERVE_REDRAW = 16  # ... and steps between two draws of the per-sequence actions
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
-# the ncu capture summarised under profiles/, keyed by (workload, kernel); absent -> null.
-NCU_TRAFFIC_BYTES = {
-    # profiles/ncu_full_llama1b_layer_all_kernels.txt (one launch each, same workload and actions)
-    ("llama1b_layer", "attn_score"): 67394816 + 1545216,
-    ("llama1b_layer", "attn_gather_v"): 34699008 + 6656,
-    ("llama1b_layer", "gemm_gate_up_swiglu"): 67371264 + 910848,
-    ("llama1b_layer", "gemm_down_gathered"): 34107392 + 0,
-    ("llama1b_layer", "gemm_qkv"): 12682240 + 0,
-    ("llama1b_layer", "gemm_out_proj"): 8553216 + 0,
-}
+DEFAULT_WORKLOAD = "ragged_serving"  # the largest single-GPU configuration
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_dram_traffic.txt")
+
+
+def ncu_traffic():
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the streaming kernels from
+    the ncu captures summarised under profiles/: lines of `workload kernel read_bytes write_bytes
+    captured_units full_units` (a capture of a scaled-down case carries the units it processed and the
+    units of a full launch; traffic is scaled by their ratio).  Absent -> null."""
+    table = {}
+    try:
+        with open(TRAFFIC_FILE) as f:
+            for line in f:
+                parts = line.split("#")[0].split()
+                if len(parts) == 6:
+                    wl, k, rd, wr, cu, fu = parts
+                    table[(wl, k)] = int((int(rd) + int(wr)) * (float(fu) / float(cu)))
+    except OSError:
+        pass
+    return table
 
 
 def _plain(o):
@@ -152,7 +166,9 @@ class ClockSampler:
 
 
 class Replica:
-    """Device-resident state of one workload: ROTATE copies of weights and caches."""
+    """Device-resident state of one workload: `rotate` copies of weights and caches.  Weights and caches
+    are drawn on the device by a seeded generator (the same shapes and distributions as the host-side
+    generators of the parity tests; tens of GB would take minutes to draw on the host)."""
 
     def __init__(self, cfg, device, seed=0):
         import torch
@@ -184,10 +200,9 @@ class Replica:
         self.copy_mb = int(copy_bytes / 1e6)
         self.weights, self.kvs, self._keep = [], [], []
         for l in range(self.L):
-            w = synth.make_layer_weights(cfg, seed, l)
-            base_w = [self._bf16(getattr(w, n)) for n in names]
-            k, v = synth.make_kv_pool(cfg, n_pages, seed, l)
-            base_kv = [self._bf16(k), self._bf16(v)]
+            wd = synth.device_layer_weights(cfg, device, seed, l)
+            base_w = [wd[n] for n in names]
+            base_kv = list(synth.device_kv_pool(cfg, n_pages, device, seed, l))
             per_copy_w, per_copy_kv = [], []
             for c in range(self.rotate):
                 ws_ = base_w if c == 0 else [t.clone() for t in base_w]
@@ -220,12 +235,11 @@ class Replica:
     def set_actions(self, r, p, b, redraws=None):
         """redraws: further (r, p, b) sets the serving workload switches to every SERVE_REDRAW steps."""
         pin = lambda a: self.torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
-        self.r_np, self.p_np, self.b_np = [np.asarray(x, np.int32) for x in (r, p, b)]
-        self.acts, self.acts_host = [], []
+        self.acts, self.acts_host, self.acts_np, self._union = [], [], [], {}
         for (rr, pp, bb) in [(r, p, b)] + list(redraws or []):
             self.acts.append((self._i32(rr), self._i32(pp), self._i32(bb)))
             self.acts_host.append(tuple(pin(np.asarray(x, np.int32)) for x in (rr, pp, bb)))
-        self.r, self.p, self.b = self.acts[0]
+            self.acts_np.append(tuple(np.asarray(x, np.int32) for x in (rr, pp, bb)))
 
     def _phase(self, i):
         j = i % self.cycle
@@ -243,40 +257,59 @@ class Replica:
         self.sol.decode_step_host(self.shape, [w[c] for w in self.weights], [k[c][j] for k in self.kvs], self.B,
                                   self.h_in_host, self.h_out_host, r, p, b, self.lens_host[j], self.ws, self.ws_bytes)
 
-    def union_rows(self):
-        """Rows of W_down that at least one token keeps, from one traced call of layer 0."""
+    def union_rows(self, a=0):
+        """Rows of W_down that at least one token keeps under action set `a`, from one traced call of layer 0."""
+        if a in self._union:
+            return self._union[a]
         t, sol = self.torch, self.sol
         ff = self.cfg["d_ff"]
         kept = t.full((self.B, ff), -1, dtype=t.int32, device=self.device)
         cnt = t.zeros((self.B,), dtype=t.int32, device=self.device)
         out = t.zeros_like(self.h_out)
-        sol.decode_layer(self.shape, self.weights[0][0], self.kvs[0][0][0], self.B, self.h_in, out, self.r, self.p,
-                         self.b, sol.make_trace(kept_ch=kept, kept_ch_cnt=cnt), self.ws, self.ws_bytes)
+        r, p, b = self.acts[a]
+        sol.decode_layer(self.shape, self.weights[0][0], self.kvs[0][0][0], self.B, self.h_in, out, r, p, b,
+                         sol.make_trace(kept_ch=kept, kept_ch_cnt=cnt), self.ws, self.ws_bytes)
         t.cuda.synchronize()
-        k, c = kept.cpu().numpy(), cnt.cpu().numpy()
-        rows = set()
-        for i in range(self.B):
-            rows.update(k[i, : c[i]].tolist())
-        return len(rows)
+        live = t.zeros((ff + 1,), dtype=t.bool, device=self.device)
+        valid = t.arange(ff, device=self.device)[None, :] < cnt[:, None]
+        live[t.where(valid, kept, t.full_like(kept, ff)).reshape(-1).long()] = True
+        self._union[a] = int(live[:ff].sum().item())
+        return self._union[a]
 
-    def required_bytes_per_step(self, union_rows):
-        kb = kernel_bytes(self.cfg, self.seq_lens + (self.cycle - 1) // 2, self.r_np, union_rows)
-        return self.L * sum(kb.values()), kb
+    def bytes_of_steps(self, step_indices):
+        """Algorithmic bytes of the given steps (mean per step, and mean per launch of each streaming kernel)."""
+        tot, per_kernel = 0.0, {}
+        for i in step_indices:
+            _, j, a = self._phase(i)
+            kb = kernel_bytes(self.cfg, self.seq_lens + j, self.acts_np[a][0], self.union_rows(a))
+            tot += self.L * sum(kb.values())
+            for k, v in kb.items():
+                per_kernel[k] = per_kernel.get(k, 0.0) + v
+        n = max(1, len(step_indices))
+        return tot / n, {k: v / n for k, v in per_kernel.items()}
+
+    def free(self):
+        self.weights = self.kvs = self._keep = self.ws = None
+        self.torch.cuda.empty_cache()
 
 
-def timed_steps(rep, steps, warmup, barrier, fn):
-    """`steps` calls of fn(i) after `warmup`; device time by CUDA events, max over ranks."""
+def timed_steps(rep, steps, warmup, barrier, fn, count_launches=False):
+    """`steps` calls of fn(i) after `warmup`; device time by CUDA events on the launching stream."""
     torch = rep.torch
     for i in range(warmup):
         fn(i)
     torch.cuda.synchronize()
     barrier()
+    if count_launches:
+        rep.sol.launch_count(reset=True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(steps):
         fn(warmup + i)
     e1.record()
     torch.cuda.synchronize()
+    if count_launches:
+        rep.launches_timed = rep.sol.launch_count(reset=True)
     barrier()
     return e0.elapsed_time(e1)  # ms
 
@@ -326,6 +359,37 @@ class Ranks:
             self.dist.destroy_process_group()
 
 
+def config_dict(workload, cfg, context):
+    """The `config` of the JSON line: the same keys and values in both arms."""
+    return {"workload": workload, "layers": cfg["layers"], "batch": cfg["batch"], "context": int(context),
+            "actions": "per-sequence uniform draw, seed 0",
+            "l2": "inputs larger than L2 (rotating copies of weights and KV cache where one copy is under 1 GB)"}
+
+
+def fractions(byt, t_ms, peak_gbs):
+    gbs = byt / t_ms / 1e6
+    return {"hbm_gbs": round(gbs, 1), "frac_of_measured": round(gbs / peak_gbs, 4),
+            "frac_of_spec_8tbs": round(gbs / HBM_SPEC_GBS, 4)}
+
+
+def sweep_point(rep, ranks, steps, peak_gbs, label):
+    n = min(steps, 300)
+    t_ms = ranks.max_over_ranks(timed_steps(rep, n, 5, ranks.barrier, rep.step)) / n
+    byt, _ = rep.bytes_of_steps(range(5, 5 + n))
+    out = dict(label)
+    out.update({"us_per_step": round(1e3 * t_ms, 2), "required_mb": round(byt / 1e6, 1)})
+    out.update(fractions(byt, t_ms, peak_gbs))
+    return out
+
+
+def flag_non_monotone(rows, key_fn):
+    """Marks sweep rows whose step time is more than 1 % above that of the row with the next larger budget
+    (rows given in order of shrinking budget)."""
+    for prev, cur in zip(rows, rows[1:]):
+        if key_fn(prev) and key_fn(cur) and cur["us_per_step"] > 1.01 * prev["us_per_step"]:
+            cur["non_monotone"] = True
+
+
 def run_ours(args):
     import torch
 
@@ -344,27 +408,28 @@ def run_ours(args):
     r, p, b = synth.draw_actions(cfg, 0)
     redraws = [synth.draw_actions(cfg, 0, redraw=k) for k in range(1, SERVE_STEPS // SERVE_REDRAW)] if rep.serving else None
     rep.set_actions(r, p, b, redraws)
-    union = rep.union_rows()
-    req_bytes, kb = rep.required_bytes_per_step(union)
     peak_gbs, peak_kind = measured_peaks()
+    traffic = ncu_traffic()
 
     # --- headline: K steps, inputs resident in HBM ---
-    sol.launch_count(reset=True)
     with ClockSampler(local) as clocks:
-        ms = max_over_ranks(timed_steps(rep, args.steps, args.warmup, barrier, rep.step))
-    launches = sol.launch_count(reset=True) * args.steps // (args.steps + args.warmup)
+        ms = max_over_ranks(timed_steps(rep, args.steps, args.warmup, barrier, rep.step, count_launches=True))
+    launches = rep.launches_timed
     status = sol.read_device_status(rep.ws)
     ms_per_step = ms / args.steps
     value = ranks.whole_job_rate(args.steps, ms)
+    timed = range(args.warmup, args.warmup + args.steps)
+    req_bytes, _ = rep.bytes_of_steps(timed)
 
-    # --- the same steps with per-kernel CUDA events, for the dominant kernel's roofline ---
+    # --- the same steps with per-kernel CUDA events (on the launching stream), for the dominant kernel's roofline ---
     prof_steps = min(args.steps, 200)
     sol.timing_enable(True)
-    timed_steps(rep, prof_steps, 3, barrier, rep.step)
+    timed_steps(rep, prof_steps, args.warmup, barrier, rep.step)
     rows = sol.timing_collect()
     sol.timing_enable(False)
+    _, kb = rep.bytes_of_steps(range(0, args.warmup + prof_steps))
     per_kernel = {}
-    n_prof = prof_steps + 3
+    n_prof = prof_steps + args.warmup
     for name, n, tot in rows:
         per_kernel[name] = {"launches_per_step": n // n_prof, "us_per_launch": 1e3 * tot / n,
                             "us_per_step": 1e3 * tot / n_prof}
@@ -375,15 +440,17 @@ def run_ours(args):
         v["us_per_step"] = round(v["us_per_step"], 3)
     for name, nbytes in kb.items():
         if name in per_kernel:
-            per_kernel[name]["bytes_per_launch"] = nbytes
+            per_kernel[name]["bytes_per_launch"] = int(nbytes)
             per_kernel[name]["gbs"] = round(nbytes / per_kernel[name]["us_per_launch"] / 1e3, 1)
+            per_kernel[name]["frac_of_measured"] = round(per_kernel[name]["gbs"] / peak_gbs, 4)
     streaming = {k: v for k, v in per_kernel.items() if "bytes_per_launch" in v}
     dom = max(streaming, key=lambda k: streaming[k]["us_per_step"])
     achieved = streaming[dom]["gbs"]
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
                 "frac": round(achieved / peak_gbs, 4), "peak_kind": f"of {peak_kind}",
+                "frac_of_spec_8tbs": round(achieved / HBM_SPEC_GBS, 4),
                 "bytes_per_launch": streaming[dom]["bytes_per_launch"],
-                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dom))}
+                "traffic": traffic.get((args.workload, dom))}
 
     # --- end to end: host buffers in, host buffers out, every step ---
     e2e_steps = min(args.steps, 500)
@@ -395,50 +462,91 @@ def run_ours(args):
     # --- budget sweep: every sequence with the same action ---
     sweep = []
     if not args.no_sweep:
-        for (rr, pp, bb) in [(1000, 0, 16), (500, 0, 16), (250, 0, 16), (125, 0, 16), (1000, 500, 16),
-                             (1000, 0, 8), (1000, 0, 4), (125, 750, 4)]:
+        r_rows, p_rows = [], []
+        for (rr, pp, bb) in [(1000, 0, 16), (500, 0, 16), (250, 0, 16), (125, 0, 16), (1000, 250, 16), (1000, 500, 16),
+                             (1000, 750, 16), (1000, 0, 8), (1000, 0, 4), (125, 750, 4)]:
             rep.set_actions(*synth.uniform_actions(rep.B, rr, pp, bb))
-            u = rep.union_rows()
-            byt, _ = rep.required_bytes_per_step(u)
-            n = min(args.steps, 300)
-            t_ms = max_over_ranks(timed_steps(rep, n, 5, barrier, rep.step)) / n
-            sweep.append({"r": rr / 1000, "p": pp / 1000, "b": bb, "us_per_step": round(1e3 * t_ms, 2),
-                          "required_mb": round(byt / 1e6, 1), "hbm_gbs": round(byt / t_ms / 1e6, 1),
-                          "frac_of_measured": round(byt / t_ms / 1e6 / peak_gbs, 4)})
+            row = sweep_point(rep, ranks, args.steps, peak_gbs, {"r": rr / 1000, "p": pp / 1000, "b": bb})
+            sweep.append(row)
+            if pp == 0 and bb == 16:
+                r_rows.append(row)
+            if rr == 1000 and bb == 16:
+                p_rows.append(row)
+        flag_non_monotone(r_rows, lambda x: True)
+        flag_non_monotone(p_rows, lambda x: True)
+        if sweep[-1]["us_per_step"] > 1.01 * r_rows[-1]["us_per_step"]:  # (r=.125, p=.75, b=4) against (r=.125, p=0)
+            sweep[-1]["non_monotone"] = True
         # the same budgets as a batch mix of the two adjacent keep-rates (how a fixed schedule hits a
         # budget that falls between discrete levels), bit-widths drawn per sequence
+        mix_rows = []
         for tgt in (1000, 500, 250, 125):
-            rm, pm, bm = synth.budget_mix_actions(cfg, tgt, 0)
-            rep.set_actions(rm, pm, bm)
-            u = rep.union_rows()
-            byt, _ = rep.required_bytes_per_step(u)
-            n = min(args.steps, 300)
-            t_ms = max_over_ranks(timed_steps(rep, n, 5, barrier, rep.step)) / n
-            sweep.append({"mix_mean_r": tgt / 1000, "p": 0.0, "b": "drawn", "us_per_step": round(1e3 * t_ms, 2),
-                          "required_mb": round(byt / 1e6, 1), "hbm_gbs": round(byt / t_ms / 1e6, 1),
-                          "frac_of_measured": round(byt / t_ms / 1e6 / peak_gbs, 4)})
+            rep.set_actions(*synth.budget_mix_actions(cfg, tgt, 0))
+            mix_rows.append(sweep_point(rep, ranks, args.steps, peak_gbs, {"mix_mean_r": tgt / 1000, "p": 0.0, "b": "drawn"}))
+        flag_non_monotone(mix_rows, lambda x: True)
+        sweep += mix_rows
         rep.set_actions(r, p, b, redraws)
+    context = int(np.max(rep.seq_lens + rep.cycle - 1))
+    rotate, copy_mb = rep.rotate, rep.copy_mb
+    rep.free()
+    del rep
+
+    # --- the other workloads, compactly, and where the prune rate saves bytes (small batches) ---
+    per_workload, small_batch = {}, []
+    if not args.no_others:
+        n = min(args.steps, 100)
+        for name in sorted(synth.WORKLOADS):
+            if name == args.workload:
+                continue
+            c2 = synth.WORKLOADS[name]
+            rp = Replica(c2, device, seed=0)
+            entry = {}
+            for tag, acts in (("drawn", synth.draw_actions(c2, 0)), ("dense", synth.uniform_actions(rp.B, 1000, 0, 16)),
+                              ("r0.125", synth.uniform_actions(rp.B, 125, 0, 16))):
+                rd = [synth.draw_actions(c2, 0, redraw=k) for k in range(1, SERVE_STEPS // SERVE_REDRAW)] \
+                    if (rp.serving and tag == "drawn") else None
+                rp.set_actions(*acts, rd)
+                t_ms = max_over_ranks(timed_steps(rp, n, 5, barrier, rp.step)) / n
+                byt, _ = rp.bytes_of_steps(range(5, 5 + n))
+                e = {"steps_per_s": round(world * 1e3 / t_ms, 2), "us_per_step": round(1e3 * t_ms, 2),
+                     "required_mb": round(byt / 1e6, 1)}
+                e.update(fractions(byt, t_ms, peak_gbs))
+                entry[tag] = e
+            per_workload[name] = entry
+            rp.free()
+            del rp
+        # one Llama-3.2-1B-shaped layer at batch 1 and 4: the union of kept W_down rows is small there
+        base = synth.WORKLOADS["llama1b_layer"]
+        for bsz in (1, 4):
+            c2 = dict(base, batch=bsz)
+            rp = Replica(c2, device, seed=0)
+            rows_b = []
+            for pp in (0, 500, 750):
+                rp.set_actions(*synth.uniform_actions(bsz, 1000, pp, 16))
+                row = sweep_point(rp, ranks, min(args.steps, 100), peak_gbs, {"batch": bsz, "r": 1.0, "p": pp / 1000, "b": 16})
+                row["union_rows"] = rp.union_rows(0)
+                rows_b.append(row)
+            flag_non_monotone(rows_b, lambda x: True)
+            small_batch += rows_b
+            rp.free()
+            del rp
 
     line = None
     if rank == 0:
         cpu = None if (world > 1 or args.no_cpu_baseline) else cpu_baseline(args.workload, budget_s=20.0)
-        hbm_gbs = req_bytes / ms_per_step / 1e6
         line = {
             "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "layers": cfg["layers"], "batch": cfg["batch"],
-                       "context": int(np.max(rep.seq_lens)), "actions": "per-sequence uniform draw, seed 0",
-                       "l2": f"inputs larger than L2: {rep.rotate} rotating cop{'ies' if rep.rotate > 1 else 'y'} of weights "
-                             f"and KV cache, {rep.copy_mb} MB each",
-                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "config": config_dict(args.workload, cfg, context),
+            "parallelism": "replicas only" if world > 1 else "single GPU",
+            "l2_defeat": f"{rotate} rotating cop{'ies' if rotate > 1 else 'y'} of weights and KV cache, {copy_mb} MB each",
             "required_bytes_per_step": int(req_bytes),
-            "hbm_tbs": round(hbm_gbs / 1e3, 4),
-            "hbm_frac_of_measured_peak": round(hbm_gbs / peak_gbs, 4),
-            "hbm_frac_of_spec_8tbs": round(hbm_gbs / HBM_SPEC_GBS, 4),
+            "hbm_tbs": round(req_bytes / ms_per_step / 1e9, 4),
+            "hbm_frac_of_measured_peak": round(req_bytes / ms_per_step / 1e6 / peak_gbs, 4),
+            "hbm_frac_of_spec_8tbs": round(req_bytes / ms_per_step / 1e6 / HBM_SPEC_GBS, 4),
             "roofline": roofline, "kernels": per_kernel, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks.summary(), "device_status": status,
-            "budget_sweep": sweep,
+            "budget_sweep": sweep, "per_workload": per_workload, "small_batch_prune_sweep": small_batch,
         }
         print(json.dumps(line, default=_plain), flush=True)
     ranks.close()
@@ -538,8 +646,7 @@ def run_reference(args):
             "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": steps, "warmup": args.warmup,
             "ms_per_step": round(1e3 * step_s, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "layers": L, "batch": B, "context": int(np.max(kv.seq_lens)),
-                       "actions": "per-sequence uniform draw, seed 0"},
+            "config": config_dict(args.workload, cfg, int(np.max(synth.make_contexts(cfg, 0)))),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": _host_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -552,12 +659,13 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="llama1b_layer", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rotate", type=int, default=ROTATE,
                     help="distinct copies of weights and KV cache cycled through the steps (1 for a small profiler capture)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="skip the compact runs of the other workloads")
     args = ap.parse_args()
     globals()["ROTATE"] = max(1, args.rotate)
     if args.impl == "reference":
@@ -565,8 +673,8 @@ def main():
         args.warmup = 1 if args.warmup is None else args.warmup
         run_reference(args)
     else:
-        args.steps = 2000 if args.steps is None else args.steps
-        args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
+        args.steps = 128 if args.steps is None else args.steps
+        args.warmup = 8 if args.warmup is None else max(args.warmup, 3)
         run_ours(args)
 
 

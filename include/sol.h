@@ -201,6 +201,15 @@ sol_status_t sol_decode_step(const sol_shape_t *shape, int32_t n_layers, const s
                              float *h_out_f32, const int32_t *r_permille, const int32_t *p_permille,
                              const int32_t *bits, void *ws, size_t ws_bytes, sol_stream_t stream);
 
+/* sol_decode_step with the taps of sol_decode_layer on every layer: `traces` is a HOST array of
+ * n_layers structs (or NULL); layer l fills traces[l].  traces[l].h_out is the float32 residual
+ * stream that layer l+1 reads, so a checker can compare every layer on the input it really saw. */
+sol_status_t sol_decode_step_traced(const sol_shape_t *shape, int32_t n_layers, const sol_layer_weights_t *layers,
+                                    const sol_kv_t *kvs, int32_t B, const void *h_in_bf16, void *h_out_bf16,
+                                    float *h_out_f32, const int32_t *r_permille, const int32_t *p_permille,
+                                    const int32_t *bits, const sol_layer_trace_t *traces, void *ws, size_t ws_bytes,
+                                    sol_stream_t stream);
+
 /* The same step for a caller whose per-step data lives on the HOST: h_in,
  * the three action arrays, seq_lens and h_out are host pointers (pinned
  * memory makes the copies of h_in and h_out asynchronous; the four int32
@@ -208,7 +217,8 @@ sol_status_t sol_decode_step(const sol_shape_t *shape, int32_t n_layers, const s
  * land in staging areas inside the workspace, the step runs with
  * kvs[l].seq_lens replaced by the staged copy, and the result is copied back;
  * the call returns after the stream has been synchronised.  Weights, pools and
- * page tables stay on the device. */
+ * page tables stay on the device.  Because the call synchronises, it also reads the workspace's
+ * error word and returns SOL_ERR_DEVICE_TIMEOUT if a bounded device-side wait gave up. */
 sol_status_t sol_decode_step_host(const sol_shape_t *shape, int32_t n_layers, const sol_layer_weights_t *layers,
                                   const sol_kv_t *kvs, int32_t B, const void *h_in_bf16_host,
                                   void *h_out_bf16_host, const int32_t *r_permille_host,
@@ -224,6 +234,12 @@ sol_status_t sol_decode_step_host(const sol_shape_t *shape, int32_t n_layers, co
  * float32 ordering, out[2] the same for channel selections, out[3] token
  * candidates re-scored in float64, out[4] channel candidates re-scored. */
 sol_status_t sol_read_device_status(const void *ws, int32_t *out_host8, sol_stream_t stream);
+
+/* Self-check of the time-out reporting (no counterpart in the paper): launches one CTA that waits, with a
+ * limit of a few thousand polls, on a barrier nothing arrives at; the wait gives up, raises bit 0 of
+ * the status words of `ws` (>= 256 bytes, initialised) and the kernel returns.  A following
+ * sol_read_device_status must then return SOL_ERR_DEVICE_TIMEOUT; sol_workspace_init clears the bit. */
+sol_status_t sol_selftest_wait_timeout(void *ws, sol_stream_t stream);
 
 /* Per-kernel timing for benchmarks.  While enabled, every kernel launch of
  * this library is bracketed by CUDA events on its stream.  sol_timing_collect

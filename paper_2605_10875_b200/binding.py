@@ -24,7 +24,7 @@ SOL_ERR_DEVICE_TIMEOUT = 5
 EXPORTS = [
     "sol_status_string", "sol_last_cuda_error", "sol_workspace_bytes", "sol_workspace_init", "sol_quant_act",
     "sol_sparse_decode_attn", "sol_sparse_decode_attn_static", "sol_pruned_swiglu_mlp", "sol_decode_layer", "sol_decode_step",
-    "sol_decode_step_host", "sol_read_device_status", "sol_timing_enable", "sol_timing_collect",
+    "sol_decode_step_traced", "sol_decode_step_host", "sol_read_device_status", "sol_selftest_wait_timeout", "sol_timing_enable", "sol_timing_collect",
     "sol_launch_count",
 ]
 
@@ -96,6 +96,11 @@ def lib() -> C.CDLL:
         L.sol_decode_step.restype = I
         L.sol_decode_step.argtypes = [C.POINTER(SolShape), I, C.POINTER(SolLayerWeights), C.POINTER(SolKV), I, P, P,
                                       P, P, P, P, P, S, P]
+        L.sol_decode_step_traced.restype = I
+        L.sol_decode_step_traced.argtypes = [C.POINTER(SolShape), I, C.POINTER(SolLayerWeights), C.POINTER(SolKV), I,
+                                             P, P, P, P, P, P, C.POINTER(SolLayerTrace), P, S, P]
+        L.sol_selftest_wait_timeout.restype = I
+        L.sol_selftest_wait_timeout.argtypes = [P, P]
         L.sol_decode_step_host.restype = I
         L.sol_decode_step_host.argtypes = [C.POINTER(SolShape), I, C.POINTER(SolLayerWeights), C.POINTER(SolKV), I,
                                            P, P, P, P, P, P, P, S, P]
@@ -232,6 +237,22 @@ def decode_step(shape, layers, kvs, B: int, h_in_bf16, h_out_bf16, h_out_f32, r_
     if check:
         _check(s, "sol_decode_step")
     return s
+
+
+def decode_step_traced(shape, layers, kvs, B: int, h_in_bf16, h_out_bf16, h_out_f32, r_permille, p_permille, bits,
+                       traces: Optional[Sequence[SolLayerTrace]], ws, ws_bytes: int, stream=None, check=True) -> int:
+    la, ka = _arrays(layers, kvs)
+    ta = (SolLayerTrace * len(layers))(*traces) if traces is not None else None
+    s = lib().sol_decode_step_traced(C.byref(shape), len(layers), la, ka, B, _ptr(h_in_bf16), _ptr(h_out_bf16),
+                                     _ptr(h_out_f32), _ptr(r_permille), _ptr(p_permille), _ptr(bits), ta, _ptr(ws),
+                                     ws_bytes, _stream(stream))
+    if check:
+        _check(s, "sol_decode_step_traced")
+    return s
+
+
+def selftest_wait_timeout(ws, stream=None) -> None:
+    _check(lib().sol_selftest_wait_timeout(_ptr(ws), _stream(stream)), "sol_selftest_wait_timeout")
 
 
 def decode_step_host(shape, layers, kvs, B: int, h_in_host, h_out_host, r_host, p_host, bits_host, seq_lens_host,

@@ -456,7 +456,7 @@ static sol_status_t decode_step_impl(const sol_shape_t* shape, int32_t n_layers,
                                      const sol_kv_t* kvs, const int32_t* seq_lens_override, int32_t B,
                                      const void* h_in_bf16, void* h_out_bf16, float* h_out_f32, const int32_t* r,
                                      const int32_t* p, const int32_t* bits, void* ws, const Layout& L,
-                                     cudaStream_t st) {
+                                     cudaStream_t st, const sol_layer_trace_t* traces = nullptr) {
   const void* h = h_in_bf16;
   bool in_f32 = false;
   for (int l = 0; l < n_layers; ++l) {
@@ -464,8 +464,8 @@ static sol_status_t decode_step_impl(const sol_shape_t* shape, int32_t n_layers,
     if (seq_lens_override) kv.seq_lens = seq_lens_override;
     const bool last = l == n_layers - 1;
     float* out32 = last ? h_out_f32 : at<float>(ws, (l & 1) ? L.h_b : L.h_a);
-    run_layer(*shape, L, ws, layers[l], kv, B, h, in_f32, last ? h_out_bf16 : nullptr, out32, r, p, bits, nullptr,
-              st);
+    run_layer(*shape, L, ws, layers[l], kv, B, h, in_f32, last ? h_out_bf16 : nullptr, out32, r, p, bits,
+              traces ? &traces[l] : nullptr, st);
     h = out32;
     in_f32 = true;
   }
@@ -499,6 +499,22 @@ sol_status_t sol_decode_step(const sol_shape_t* shape, int32_t n_layers, const s
   if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
   return decode_step_impl(shape, n_layers, layers, kvs, nullptr, B, h_in_bf16, h_out_bf16, h_out_f32, r_permille,
                           p_permille, bits, ws, L, (cudaStream_t)stream);
+}
+
+sol_status_t sol_decode_step_traced(const sol_shape_t* shape, int32_t n_layers, const sol_layer_weights_t* layers,
+                                    const sol_kv_t* kvs, int32_t B, const void* h_in_bf16, void* h_out_bf16,
+                                    float* h_out_f32, const int32_t* r_permille, const int32_t* p_permille,
+                                    const int32_t* bits, const sol_layer_trace_t* traces, void* ws, size_t ws_bytes,
+                                    sol_stream_t stream) {
+  int mp = 0;
+  sol_status_t s = step_args_ok(shape, n_layers, layers, kvs, B, &mp);
+  if (s != SOL_OK) return s;
+  if (!h_in_bf16 || !h_out_bf16 || !r_permille || !p_permille || !bits || !ws) return SOL_ERR_INVALID_ARG;
+  if (B == 0) return SOL_OK;
+  const Layout L = make_layout(*shape, B, mp);
+  if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
+  return decode_step_impl(shape, n_layers, layers, kvs, nullptr, B, h_in_bf16, h_out_bf16, h_out_f32, r_permille,
+                          p_permille, bits, ws, L, (cudaStream_t)stream, traces);
 }
 
 // The per-sequence actions and lengths of a step (at most 128 sequences) travel as kernel parameters:
@@ -551,8 +567,15 @@ sol_status_t sol_decode_step_host(const sol_shape_t* shape, int32_t n_layers, co
                        at<void>(ws, L.stage_h_out), nullptr, act, act + B, act + 2 * B, ws, L, st);
   if (s != SOL_OK) return s;
   record_cuda_error(cudaMemcpyAsync(h_out_bf16_host, at<void>(ws, L.stage_h_out), hb, cudaMemcpyDeviceToHost, st), "d2h h_out");
+  // the call synchronises anyway, so it also reads the error word of the workspace: a wait that gave up is
+  // reported here instead of leaving a result built from skipped stores
+  int32_t err_word = 0;
+  record_cuda_error(cudaMemcpyAsync(&err_word, at<int32_t>(ws, L.status) + ST_ERR, sizeof(int32_t), cudaMemcpyDeviceToHost, st),
+                    "status copy");
   record_cuda_error(cudaStreamSynchronize(st), "stream synchronize");
-  return finish();
+  s = finish();
+  if (s != SOL_OK) return s;
+  return (err_word & ERR_TIMEOUT) ? SOL_ERR_DEVICE_TIMEOUT : SOL_OK;
 }
 
 sol_status_t sol_read_device_status(const void* ws, int32_t* out_host8, sol_stream_t stream) {
@@ -562,6 +585,25 @@ sol_status_t sol_read_device_status(const void* ws, int32_t* out_host8, sol_stre
     return finish();
   if (record_cuda_error(cudaStreamSynchronize(st), "stream synchronize")) return finish();
   return (out_host8[ST_ERR] & ERR_TIMEOUT) ? SOL_ERR_DEVICE_TIMEOUT : SOL_OK;
+}
+
+// One CTA waits on an mbarrier that nothing ever arrives at; the bounded wait gives up after a few thousand
+// polls, raises the time-out bit of the workspace's status words and the kernel returns.
+__global__ void selftest_wait_kernel(int* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait(&bar, 0, status, 4096);
+}
+
+sol_status_t sol_selftest_wait_timeout(void* ws, sol_stream_t stream) {
+  if (!ws) return SOL_ERR_INVALID_ARG;
+  selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(at<int>(ws, 0));
+  record_cuda_error(cudaGetLastError(), "self-test launch");
+  return finish();
 }
 
 void sol_timing_enable(int32_t on) {

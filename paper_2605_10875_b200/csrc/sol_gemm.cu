@@ -143,6 +143,9 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
     // The mbarrier wait orders the TMA writes before the MMA reads; no tcgen05 fence is needed per stage.
     const uint32_t idesc = umma_idesc_bf16_m128(nb_rows, 0, 0);
     bool acc = false, ok = true;
+    // the first stage fills only after the producer's own pdl_wait(): without this wait the bounded poll
+    // below would start counting while earlier kernels of the stream are still running
+    pdl_wait();
     for (int it = 0; it < n_iter; ++it) {
       const int s = it % p.stages;
       const uint32_t ph = (it / p.stages) & 1;

@@ -73,10 +73,16 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
 
   unsigned char* base = nullptr;
   const sol_status_t s = scratch_of_current_device(&base);
-  if (s != SOL_OK) return s;
+  if (s != SOL_OK) {
+    sol::take_cuda_failure();  // reported here; the mark must not leak into this thread's next call
+    return s;
+  }
   cudaStream_t st = (cudaStream_t)stream;
   // the array keeps whatever the previous call left; only the status words must start at zero
-  if (sol::record_cuda_error(cudaMemsetAsync(base, 0, kStatusBytes, st), "status memset")) return SOL_ERR_CUDA;
+  if (sol::record_cuda_error(cudaMemsetAsync(base, 0, kStatusBytes, st), "status memset")) {
+    sol::take_cuda_failure();
+    return SOL_ERR_CUDA;
+  }
 
   sol::AttnArgs a;
   a.shape = *shape;
@@ -95,9 +101,8 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
   a.out_lo = nullptr;
   a.status = reinterpret_cast<int*>(base);
   sol::launch_attention(a, st);
-  if (status_out != nullptr &&
-      sol::record_cuda_error(cudaMemcpyAsync(status_out, base, sizeof(int32_t) * sol::ST_WORDS,
-                                             cudaMemcpyDeviceToDevice, st), "status copy"))
-    return SOL_ERR_CUDA;
+  if (status_out != nullptr)
+    sol::record_cuda_error(cudaMemcpyAsync(status_out, base, sizeof(int32_t) * sol::ST_WORDS, cudaMemcpyDeviceToDevice, st),
+                           "status copy");
   return sol::take_cuda_failure() ? SOL_ERR_CUDA : SOL_OK;
 }

@@ -140,6 +140,41 @@ def make_kv_pool(cfg: dict, num_pages: int, seed: int = 0, layer: int = 0) -> Tu
             normal_bf16(rng_for(seed, "v_pool", layer), shape, 0.0, 1.0))
 
 
+def device_kv_pool(cfg: dict, num_pages: int, device, seed: int = 0, layer: int = 0):
+    """The same N(0, 1) bf16 pools drawn on a CUDA device by torch's counter-based generator, for
+    workloads whose cache (tens of GB) would take minutes to draw on the host.  Returns torch bf16
+    tensors (k_pool, v_pool); a checker reads back the pages it needs."""
+    return (device_normal_bf16((num_pages, cfg["n_kv_heads"], PAGE_SIZE, cfg["head_dim"]), device, seed, "k_pool", layer),
+            device_normal_bf16((num_pages, cfg["n_kv_heads"], PAGE_SIZE, cfg["head_dim"]), device, seed, "v_pool", layer))
+
+
+def device_normal_bf16(shape, device, seed: int, stream: str, layer: int = 0, mean: float = 0.0, std: float = 1.0):
+    """N(mean, std) rounded to bf16, drawn on `device` (torch): an independent seeded stream per
+    (seed, named tensor, layer), like rng_for."""
+    import torch
+
+    g = torch.Generator(device=device)
+    g.manual_seed((int(seed) * 1000003 + _STREAMS[stream]) * 1000003 + int(layer))
+    out = torch.empty(shape, dtype=torch.bfloat16, device=device)
+    flat = out.view(-1)
+    chunk = 1 << 28
+    for s0 in range(0, flat.numel(), chunk):
+        part = flat[s0:s0 + chunk]
+        x = torch.randn(part.shape, dtype=torch.float32, device=device, generator=g)
+        part.copy_(x.mul_(std).add_(mean))
+    return out
+
+
+def device_layer_weights(cfg: dict, device, seed: int = 0, layer: int = 0) -> dict:
+    """Layer weights of the workload's shapes and distributions drawn on the device (see device_normal_bf16)."""
+    d, hq, hkv, hd, ff = cfg["d_model"], cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"], cfg["d_ff"]
+    g = lambda name, shape, mean, std: device_normal_bf16(shape, device, seed, name, layer, mean, std)
+    return dict(w_qkv=g("w_qkv", ((hq + 2 * hkv) * hd, d), 0.0, 0.02), w_o=g("w_o", (d, hq * hd), 0.0, 0.02),
+                w_gate=g("w_gate", (ff, d), 0.0, 0.02), w_up=g("w_up", (ff, d), 0.0, 0.02),
+                w_down_t=g("w_down_t", (ff, d), 0.0, 0.02), gamma1=g("gamma1", (d,), 1.0, 0.02),
+                gamma2=g("gamma2", (d,), 1.0, 0.02))
+
+
 def make_hidden(cfg: dict, seed: int = 0, batch: Optional[int] = None) -> np.ndarray:
     B = batch or cfg["batch"]
     return normal_bf16(rng_for(seed, "hidden"), (B, cfg["d_model"]), 0.0, 1.0)

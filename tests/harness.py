@@ -204,5 +204,9 @@ def assert_sets(par: checker.SetParity, what: str):
 
 def assert_outputs(oracle_out, got, what: str):
     m, r = checker.output_errors(oracle_out, got)
+    raw_small, raw_all = checker.raw_max_abs(oracle_out, got)
+    assert raw_small <= checker.OUT_MAX_ABS, f"{what}: plain max-abs {raw_small:.3e} where |oracle| < 8"
     assert m <= checker.OUT_MAX_ABS and r <= checker.OUT_REL_L2, f"{what}: max-abs {m:.3e} rel-L2 {r:.3e}"
+    print(f"{what}: max-abs {raw_all:.3e} plain, {raw_small:.3e} where |oracle| < 8, {m:.3e} in bf16 steps of [4,8); "
+          f"rel-L2 {r:.3e}")
     return m, r

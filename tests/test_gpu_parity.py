@@ -229,39 +229,22 @@ def test_mlp_llama8b_shape():
 # ------------------------------------------------------------------ layer ---
 
 
-def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1, sample=None):
-    """Runs one layer on the GPU with every tap, then checks each stage against
-    the oracle's stage applied to the inputs the GPU stage really saw, and the
-    whole layer against the oracle's own layer.  A float32-vs-float64 difference
-    of one ulp upstream may legally flip a quantizer code or a selection that
-    sits exactly on a boundary; when that happened the end-to-end comparison is
-    reported but not asserted (the chain of stage checks still covers it).
-    `sample`: the GPU runs the whole batch, the oracle only these sequences
-    (full-size workloads, where the oracle cannot afford every sequence)."""
-    shape, oshape = H.make_shapes(cfg, n_sink, n_window)
-    B = len(seq_lens)
-    seq_lens = np.asarray(seq_lens, np.int32)
-    d, Hq, Hkv, hd = cfg["d_model"], oshape.n_q_heads, oshape.n_kv_heads, oshape.head_dim
-    w = synth.make_layer_weights(cfg, seed)
-    k_pool, v_pool, table = H.make_case_kv(cfg, seq_lens, seed)
-    h_in = synth.make_hidden(cfg, seed, B)
-    kv = H.device_kv(k_pool, v_pool, table, seq_lens)
-    out, taps, st = H.gpu_layer(shape, H.device_weights(w), kv, h_in, r, p, b)
-    assert st[0] == 0 and st[1] == 0 and st[2] == 0, st
-    ow = H.oracle_weights(w)
-    tab = np.where(table < 0, 0, table)
-    k_gpu, v_gpu = H.host_u16(kv.k_pool), H.host_u16(kv.v_pool)
-    assert (k_gpu != k_pool).sum() <= B * Hkv * hd  # nothing but the appended rows changed
-    if sample is not None:  # from here on only the sampled sequences
-        idx = np.asarray(sample)
-        taps = {key: val[idx] for key, val in taps.items()}
-        out, h_in, seq_lens, tab = out[idx], h_in[idx], seq_lens[idx], tab[idx]
-        r, p, b = np.asarray(r)[idx], np.asarray(p)[idx], np.asarray(b)[idx]
-        B = len(idx)
-    h64 = O.bf16_to_f64(h_in)
+def check_stages(oshape, w, h64, tab, seq_lens, r, p, b, taps, k_before, v_before, k_after, v_after, out=None,
+                 status=None):
+    """Every stage of one layer against the oracle's stage applied to the inputs that stage really saw on
+    the GPU (teacher forcing), then the whole layer against the oracle's own layer.
 
-    # the oracle's own layer (on the pools as generated; the GPU's copies were fetched above)
-    okv = O.PagedKV(k_pool, v_pool, tab, seq_lens)
+    h64 [n][d] is the layer's input as the GPU saw it; taps are the GPU's taps for the same n sequences;
+    k_before / v_before are the cache pools before the layer ran and k_after / v_after after it (all
+    indexed by the page table rows `tab`); out (optional) is the layer's bf16 output as float64.
+    A float32-vs-float64 difference of one ulp upstream may legally flip a quantizer code or a selection
+    that sits exactly on a boundary; when that happened the end-to-end comparison is reported, not
+    asserted (the chain of stage checks still covers the layer); `end_to_end_asserted` says which."""
+    B, d = h64.shape
+    Hq, Hkv, hd = oshape.n_q_heads, oshape.n_kv_heads, oshape.head_dim
+    ow = H.oracle_weights(w)
+    # the oracle's own layer on the cache as it was before the layer (it appends into its copy)
+    okv = O.PagedKV(k_before, v_before, tab, seq_lens)
     out_o, tr = O.decode_layer(oshape, ow, okv, h64, r, p, b)
 
     # stage 1: RMSNorm (float32 on the GPU) and quantizer (bit-exact on the GPU's own normalised row)
@@ -286,11 +269,11 @@ def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1, sample=Non
         k_tol = acc_tol[i, Hq * hd:(Hq + Hkv) * hd].reshape(Hkv, hd)
         k_tol = k_tol + np.roll(k_tol, hd // 2, axis=1)  # a rotated element mixes e and e +- hd/2
         v_tol = acc_tol[i, (Hq + Hkv) * hd:].reshape(Hkv, hd)
-        for got, want, tol in ((k_gpu[pg, :, slot], k_ref, k_tol), (v_gpu[pg, :, slot], v_ref, v_tol)):
+        for got, want, tol in ((k_after[pg, :, slot], k_ref, k_tol), (v_after[pg, :, slot], v_ref, v_tol)):
             # the appended row is the bf16 nearest to the float32 value: within one bf16 step of the float64 one
             assert np.all(np.abs(O.bf16_to_f64(got) - want) <= np.abs(want) * 2.0 ** -8 * 1.01 + tol + 1e-6), "append"
     # stage 3: token selection and attention on the GPU's own queries and cache
-    gkv = O.PagedKV(k_gpu, v_gpu, tab, seq_lens)
+    gkv = O.PagedKV(k_after, v_after, tab, seq_lens)
     attn_o, kept_o, sigma = O.sparse_decode_attn(oshape, taps["q_rot"].astype(np.float64), gkv, r)
     kept = [[taps["kept_idx"][i, h, : taps["kept_cnt"][i, h]] for h in range(Hkv)] for i in range(B)]
     tok = H.check_token_sets(oshape, sigma, kept_o, kept, seq_lens)
@@ -299,7 +282,7 @@ def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1, sample=Non
         assert np.allclose(taps["attn_out"], attn_o, rtol=0, atol=1e-4 * max(1.0, np.abs(attn_o).max())), "attn_out"
     # stage 4: output projection + residual on the GPU's own attention output
     h_mid_ref = h64 + taps["attn_out"].astype(np.float64).reshape(B, Hq * hd) @ O.bf16_to_f64(w.w_o).T
-    assert np.allclose(taps["h_mid"], h_mid_ref, rtol=0, atol=1e-4), "h_mid"
+    assert np.allclose(taps["h_mid"], h_mid_ref, rtol=0, atol=1e-4 * max(1.0, np.abs(h_mid_ref).max() / 8)), "h_mid"
     # stage 5: second RMSNorm + quantizer
     xn2_ref = np.stack([O.rmsnorm(taps["h_mid"][i].astype(np.float64), O.bf16_to_f64(w.gamma2), oshape.rms_eps)
                         for i in range(B)])
@@ -321,27 +304,64 @@ def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1, sample=Non
     g_o, u_o = x_hat2 @ O.bf16_to_f64(w.w_gate).T, x_hat2 @ O.bf16_to_f64(w.w_up).T
     t_tol = 1e-4 * np.abs(t_o) + 1.1 * np.abs(u_o) * g_tol + np.abs(g_o) * u_tol + 1e-6
     assert np.all(np.abs(taps["t"] - t_o) <= t_tol), "t"
+    h_out_ref = taps["h_mid"].astype(np.float64) + mlp_o
     if ch.exact == ch.sets:
-        assert np.allclose(taps["h_out"], taps["h_mid"].astype(np.float64) + mlp_o, rtol=0, atol=2e-4), "h_out"
+        assert np.allclose(taps["h_out"], h_out_ref, rtol=0, atol=2e-4 * max(1.0, np.abs(h_out_ref).max() / 8)), "h_out"
+    # the layer's output against the oracle's stage on the GPU's own h_mid and quantized MLP input, at the
+    # task's output tolerances (max-abs 2e-2, relative L2 1e-2): this is the per-layer output rule
+    # of a many-layer step, where the end-to-end comparison below drifts
+    H.assert_outputs(h_out_ref, taps["h_out"], "layer output on its own inputs")
     # stage 7: the bf16 output is the float32 result rounded to nearest-even
-    assert np.array_equal(synth.to_bf16(taps["h_out"]), synth.to_bf16(out.astype(np.float32))), "bf16 rounding"
+    if out is not None:
+        assert np.array_equal(synth.to_bf16(taps["h_out"]), synth.to_bf16(out.astype(np.float32))), "bf16 rounding"
 
     # end to end against the oracle's own layer
     flips = int((taps["codes1"] != tr.codes1).sum() + (taps["codes2"] != tr.codes2).sum())
     own_tok = H.check_token_sets(oshape, tr.extra["sigma"], tr.kept_tokens, kept, seq_lens)
     own_ch = H.check_channel_sets(tr.t, tr.kept_channels, kept_ch)
     diverged = flips > 0 or own_tok.exact != own_tok.sets or own_ch.exact != own_ch.sets
-    err = checker.output_errors(out_o, out)
+    got = out if out is not None else taps["h_out"].astype(np.float64)
+    err = checker.output_errors(out_o, got)
     if not diverged:
-        H.assert_outputs(out_o, out, "layer output")
+        H.assert_outputs(out_o, got, "layer output")
     return dict(err=err, code_flips=flips, tokens=tok, channels=ch, own_tokens=own_tok, own_channels=own_ch,
-                status=st, end_to_end_asserted=not diverged)
+                status=status, end_to_end_asserted=not diverged)
+
+
+def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1, sample=None):
+    """Runs one layer on the GPU with every tap and checks it with check_stages.
+    `sample`: the GPU runs the whole batch, the oracle only these sequences
+    (full-size workloads, where the oracle cannot afford every sequence)."""
+    shape, oshape = H.make_shapes(cfg, n_sink, n_window)
+    B = len(seq_lens)
+    seq_lens = np.asarray(seq_lens, np.int32)
+    Hkv, hd = oshape.n_kv_heads, oshape.head_dim
+    w = synth.make_layer_weights(cfg, seed)
+    k_pool, v_pool, table = H.make_case_kv(cfg, seq_lens, seed)
+    h_in = synth.make_hidden(cfg, seed, B)
+    kv = H.device_kv(k_pool, v_pool, table, seq_lens)
+    out, taps, st = H.gpu_layer(shape, H.device_weights(w), kv, h_in, r, p, b)
+    assert st[0] == 0 and st[1] == 0 and st[2] == 0, st
+    tab = np.where(table < 0, 0, table)
+    k_gpu, v_gpu = H.host_u16(kv.k_pool), H.host_u16(kv.v_pool)
+    assert (k_gpu != k_pool).sum() <= B * Hkv * hd  # nothing but the appended rows changed
+    if sample is not None:  # from here on only the sampled sequences
+        idx = np.asarray(sample)
+        taps = {key: val[idx] for key, val in taps.items()}
+        out, h_in, seq_lens, tab = out[idx], h_in[idx], seq_lens[idx], tab[idx]
+        r, p, b = np.asarray(r)[idx], np.asarray(p)[idx], np.asarray(b)[idx]
+    return check_stages(oshape, w, O.bf16_to_f64(h_in), tab, seq_lens, r, p, b, taps, k_pool, v_pool, k_gpu, v_gpu,
+                        out=out, status=st)
 
 
 def test_layer_tiny_workload():
     r, p, b = synth.draw_actions(TINY, 0)
-    res = check_layer(TINY, synth.make_contexts(TINY, 0), r, p, b)
-    print("tiny layer:", res)
+    asserted = []
+    for seed in (0, 1, 2, 3):  # every seed passes the stage chain; the end-to-end rule must be the gate on one at least
+        res = check_layer(TINY, synth.make_contexts(TINY, 0), r, p, b, seed=seed)
+        asserted.append(res["end_to_end_asserted"])
+        print("tiny layer, seed", seed, res)
+    assert any(asserted), asserted
 
 
 def test_layer_dense_action():
@@ -359,6 +379,22 @@ def test_layer_llama1b_full():
     r, p, b = synth.draw_actions(L1B, 0)
     res = check_layer(L1B, synth.make_contexts(L1B, 0), r, p, b)
     print("llama1b layer:", res)
+
+
+def test_layer_llama1b_end_to_end_rule_asserted():
+    """The whole layer against the oracle's own run at the task's output tolerances, asserted: with the
+    bf16 passthrough (no quantizer grid for a one-ulp difference to cross) and a seed on which no
+    selection sits on a boundary, nothing diverges and the end-to-end comparison is the gate."""
+    B = L1B["batch"]
+    r, p, _ = synth.draw_actions(L1B, 0)
+    asserted = []
+    for seed in (0, 1, 2):
+        res = check_layer(L1B, synth.make_contexts(L1B, 0), r, p, [16] * B, seed=seed)
+        asserted.append(res["end_to_end_asserted"])
+        print("llama1b layer, 16 bits, seed", seed, res)
+        if asserted[-1]:
+            break
+    assert any(asserted), asserted
 
 
 def test_layer_llama8b_shape_reduced_context():
@@ -474,3 +510,26 @@ def test_repeat_calls_are_bit_identical():
         outs.append((out, taps["kept_idx"].copy(), taps["kept_ch"].copy(), taps["h_out"].copy()))
     for a, c in zip(outs[0], outs[1]):
         assert np.array_equal(a, c)
+
+
+# ------------------------------------------------------- device-side time-out ---
+
+
+def test_bounded_wait_gives_up_and_is_reported():
+    """A wait on a barrier that nothing arrives at runs out after a few thousand polls: the kernel
+    returns, the status word carries the time-out bit, the host call reports it, and the context is
+    still usable afterwards."""
+    shape, _ = H.make_shapes(TINY)
+    ws = H.Workspace(shape, 4, 8)
+    assert ws.status()[0] == 0
+    sol.selftest_wait_timeout(ws.buf)
+    out = sol.read_device_status(ws.buf, check=False)
+    assert out[0] & 1
+    with pytest.raises(sol.SolError) as e:
+        sol.read_device_status(ws.buf)
+    assert e.value.status == sol.SOL_ERR_DEVICE_TIMEOUT
+    sol.workspace_init(ws.buf, ws.bytes)
+    torch.cuda.synchronize()
+    assert ws.status()[0] == 0
+    # the device still computes: a small attention case runs and matches the oracle
+    _attention_case(TINY, [130, 64], [500, 250], seed=12)
