@@ -41,12 +41,17 @@ struct PrepDev {
   float* q_rot;
   uint16_t* q_split;
   int32_t* work_ctr;  // zeroed here: [0] items emitted, [1] next item, [2 + b*Hkv + kvh] finished items
+  uint32_t* row_hist; // zeroed here: [B*Hkv][SEL_BINS] score histogram of rows that span several selection CTAs
+  uint32_t* row_ctl;  // zeroed here: [B*Hkv][RC_WORDS]
   int* status;
 };
 
 constexpr int PREP_THREADS = 128;
 // words of AttnArgs::work_ctr
 enum : int { WC_ITEMS = 0, WC_NEXT = 1, WC_CPI = 2, WC_DONE = 4 };
+// words of AttnArgs::row_ctl, per (sequence, kv-head): token selection CTAs finished, largest |score| (float
+// bits), the keep edge (float bits), the selection mode
+enum : int { RC_DONE = 0, RC_MAX = 1, RC_EDGE = 2, RC_MODE = 3, RC_WORDS = 4 };
 
 // One CTA per (kv-head, sequence): the G query heads of the group, the new k row and the new v row.
 __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p) {
@@ -91,6 +96,12 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
       p.work_ctr[WC_ITEMS] = 0;
       p.work_ctr[WC_NEXT] = 0;
     }
+  }
+  // scratch of the token selection of this (sequence, kv-head)
+  if (tid < RC_WORDS) p.row_ctl[(size_t)(b * Hkv + kvh) * RC_WORDS + tid] = 0u;
+  if (T > 2048) {  // rows of one selection CTA keep their histogram in shared memory
+    uint4* hz = reinterpret_cast<uint4*>(p.row_hist + (size_t)(b * Hkv + kvh) * SEL_BINS);
+    for (int i = tid; i < SEL_BINS / 4; i += PREP_THREADS) hz[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   if (tid < half) {
     float c = 1.f, s = 0.f;
@@ -309,232 +320,462 @@ __global__ void __launch_bounds__(SC_WARPS * 32) attn_score_kernel(const ScoreDe
       sig1 += q1;
     }
     if (t == 0) {
-      if (tok0 < T) p.sigma[row0 + tok0] = sig0;
-      if (tok1 < T) p.sigma[row0 + tok1] = sig1;
+      if (tok0 < T) p.sigma[row0 + tok0] = sig0 + 0.0f;  // -0 becomes +0: the selection compares floats and keys
+      if (tok1 < T) p.sigma[row0 + tok1] = sig1 + 0.0f;
     }
   }
 }
 
 // ============================================================================
-// token_select
+// token_select + token_compact
 // ============================================================================
+// Exact top-k of a (sequence, kv-head) row of scores, spread over one CTA per 2048 tokens.
+//
+//   phase 1 (every CTA of the row): histogram of the CTA's scores over 4096 value bins in shared memory,
+//            flushed (non-empty bins only) to the row's histogram in global memory, and the largest |score|;
+//   phase 2 (the CTA that finishes last; rows of one CTA go straight on): the bin that holds the k-th
+//            largest score; one pass over the row's scores counts, per 2048-token segment, what lies above
+//            that bin (by more than a small window) and lists what lies in it or within the window; the
+//            list is ranked in float32, everything within the window of the k-th value is re-scored in
+//            float64 from the cache rows, and the listed tokens that are kept get their score replaced by
+//            +inf, as do the forced tokens.  From then on "kept" is the single comparison score > edge.
+//
+// token_compact (one CTA per 2048 tokens again) turns that comparison into the ascending index list and
+// the page-resolved cache row of every kept token, at the offsets phase 2 derived from the segment counts.
+constexpr int TS_THREADS = 256;
+constexpr int TS_SEG = 2048;                                      // tokens per CTA
+constexpr int TS_MAX_SEGS = MAX_PAGES_PER_SEQ * PAGE / TS_SEG;     // 24
+constexpr float TS_FLT_MAX = 3.402823466e+38f;
+
 struct SelectDev {
   sol_shape_t sh;
   sol_kv_t kv;
   const int32_t* r_permille;
-  int Tmax, S, split_len, B;
+  int Tmax, S, split_len, B, nseg_max;
   const float* q_rot;
-  const float* sigma;
-  int32_t* kept_idx;
+  float* sigma;          // kept listed tokens and forced tokens are overwritten with +inf
+  uint32_t* row_hist;    // [B*Hkv][SEL_BINS], zero on entry
+  uint32_t* row_ctl;     // [B*Hkv][RC_WORDS], zero on entry
+  int32_t* seg_off;      // [B*Hkv][nseg_max] first place of each segment's kept tokens in the row's list
   int32_t* kept_cnt;
-  uint32_t* kept_row;
   int32_t* work_items;
   int32_t* work_ctr;
   int* status;
 };
 
-// One CTA per (sequence, kv-head).  Every thread owns `per` consecutive tokens; their scores sit in
-// shared memory (as order-preserving keys, slot i of thread t at [i * THREADS + t]) for all passes, and
-// every loop over them is a rolled one: the kernel is a long chain of short passes, and unrolled over
-// register arrays it spent more time waiting for instructions than for data.  Candidates near the
-// threshold are settled in float64.
-template <int THREADS>
-__global__ void __launch_bounds__(THREADS) token_select_kernel(const SelectDev p) {
-  __shared__ SelectSmem sm;
-  __shared__ double qsum[128];
-  extern __shared__ __align__(16) uint32_t skey[];  // [per][THREADS]
+// Exclusive prefix sum of v over the 256 threads (in thread order) and the block total.
+__device__ __forceinline__ int ts_block_scan(int v, int& total, int* warp_tot) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += x;
+  }
+  __syncthreads();  // earlier readers of warp_tot are done
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  int before = incl - v;
+  total = 0;
+#pragma unroll
+  for (int w = 0; w < TS_THREADS / 32; ++w) {
+    const int x = warp_tot[w];
+    if (w < warp) before += x;
+    total += x;
+  }
+  return before;
+}
 
-  const int kvh = blockIdx.x, b = blockIdx.y;
+__global__ void __launch_bounds__(TS_THREADS) token_select_kernel(const SelectDev p) {
+  __shared__ SelectSmem sm;
+  __shared__ float sup_val[SEL_CAND_CAP];
+  __shared__ double qsum[128];
+  __shared__ int seg_cnt[TS_MAX_SEGS];
+  __shared__ int s_flag;
+
+  const int seg = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int Hkv = p.sh.n_kv_heads, hd = p.sh.head_dim, G = p.sh.n_q_heads / Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  constexpr int WARPS = THREADS / 32;
-  constexpr int KPT = 0;  // rolled key loops
+  constexpr int WARPS = TS_THREADS / 32;
   const int bk = b * Hkv + kvh;
   pdl_trigger();
-  pdl_wait();
+  // the lengths are an input of the step, not the work of an earlier kernel
   const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
+  if (seg * TS_SEG >= max(T, 1)) return;
+  pdl_wait();
   const size_t row = (size_t)bk * p.Tmax;
-  const float* sig = p.sigma + row;
-  // a thread owns `per` consecutive tokens: as few as this sequence needs (a multiple of 4 for the
-  // vector loads), so a short context in a long-context batch costs what its own length costs
-  const int per = ((max(T, 1) + THREADS - 1) / THREADS + 3) / 4 * 4;
-  const int j0 = tid * per;
-  auto key = [&](int i) { return skey[i * THREADS + tid]; };  // 0: absent, 0xffffffff: forced
+  float* sig = p.sigma + row;
+  uint32_t* ctl = p.row_ctl + (size_t)bk * RC_WORDS;
+  uint32_t* gh = p.row_hist + (size_t)bk * SEL_BINS;
+  int32_t* soff = p.seg_off + (size_t)bk * p.nseg_max;
+  const int nseg = max(1, (T + TS_SEG - 1) / TS_SEG);
 
-  int total = 0;
-  if (T > 0) {
-    const int n_sink = min(max(p.sh.n_sink, 0), T);
-    const int n_win = min(max(p.sh.n_window, 0), T - n_sink);
-    const int nf = n_sink + n_win;
-    long long bud = ((long long)p.r_permille[b] * T + 999) / 1000;
-    if (bud > T) bud = T;
-    const int k = min(T, max((int)bud, nf));
-    auto forced = [&](int j) { return j < n_sink || j >= T - n_win; };
-    if (tid < 4) sm.counts[tid] = 0;
+  const int n_sink = min(max(p.sh.n_sink, 0), max(T, 0));
+  const int n_win = min(max(p.sh.n_window, 0), max(T, 0) - n_sink);
+  const int nf = n_sink + n_win;
+  long long bud = ((long long)p.r_permille[b] * T + 999) / 1000;
+  if (bud > T) bud = T;
+  const int k = T > 0 ? min(T, max((int)bud, nf)) : 0;
+  auto forced = [&](int j) { return j < n_sink || j >= T - n_win; };
+  // mode 0: keep all; 1: forced only; 2: selection; 3 (phase 2 only): float32 order with index-ordered ties
+  int mode = k >= T ? 0 : (k <= nf ? 1 : 2);
 
-    // mode 0: keep all; 1: forced only; 2: the key slots hold classes (settled by the window pass and
-    // the float64 ranking); 3: key threshold with index-ordered ties (float32 ordering, the candidate
-    // list overflowed)
-    constexpr uint32_t CLS_DROP = 0u, CLS_KEEP = 2u, CLS_CAND = 3u;
-    int mode, tie_need = 0;
-    uint32_t key_thr = 0;
-    int my_keep = 0, my_ties = 0;  // of this thread's tokens: kept for sure, tied at the threshold
-
-    if (k >= T) {
-      mode = 0;
-      my_keep = min(max(T - j0, 0), per);
-    } else if (k <= nf) {
-      mode = 1;
-      for (int i = 0; i < per; ++i) my_keep += j0 + i < T && forced(j0 + i);
-    } else {
-      float mx = 0.f;
-#pragma unroll 1
-      for (int i = 0; i < per; i += 4) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (j0 + i < T) v = *reinterpret_cast<const float4*>(sig + j0 + i);
-        const float vv[4] = {v.x, v.y, v.z, v.w};
+  // ------------------------------------------------------------- phase 1 ----
+  float mx = 0.f;
+  if (mode == 2) {
+    for (int i = tid; i < SEL_BINS; i += TS_THREADS) sm.hist[i] = 0;
+    __syncthreads();
+    const int j0 = seg * TS_SEG + tid * 8;
+    if (j0 < T) {
+      const float4 v0 = *reinterpret_cast<const float4*>(sig + j0), v1 = *reinterpret_cast<const float4*>(sig + j0 + 4);
+      const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int j = j0 + i + e;
-          uint32_t kk = 0;
-          if (j < T) {
-            if (forced(j)) {
-              kk = 0xffffffffu;
-            } else {
-              const float sv = vv[e] + 0.0f;
-              kk = float_key(sv);
-              mx = fmaxf(mx, fabsf(sv));
-            }
-          }
-          skey[(i + e) * THREADS + tid] = kk;
+      for (int e = 0; e < 8; ++e) {
+        const int j = j0 + e;
+        if (j < T && !forced(j)) {
+          const float sv = vv[e] + 0.0f;
+          atomicAdd(&sm.hist[key_value_bin(float_key(sv))], 1u);
+          mx = fmaxf(mx, fabsf(sv));
         }
-      }
-      mx = block_max<THREADS>(mx, 0, sm);
-      key_thr = select_kth<THREADS, KPT, true>(key, k, tie_need, sm, per);
-
-      // ---- window around the threshold, re-scored in float64 ----
-      const float thr32 = key_to_float(key_thr);
-      // 2^-16 of the largest score: far above the float32 accumulation error of a head_dim-long dot product
-      const float delta = mx * 1.52587890625e-05f;
-      const float hi = thr32 + delta, lo = thr32 - delta;
-      // One pass counts what is clear of the window and lists the candidates inside it.
-      int n_in = 0, my_cand = 0;
-#pragma unroll 4
-      for (int i = 0; i < per; ++i) {
-        const uint32_t kk = key(i);
-        if (kk == 0xffffffffu) {
-          ++my_keep;
-        } else if (kk != 0u) {
-          const float sv = key_to_float(kk);
-          if (sv > hi) {
-            ++n_in;
-          } else if (sv >= lo) {
-            ++my_cand;
-            const int slot = atomicAdd(&sm.counts[0], 1);
-            if (slot < SEL_CAND_CAP) sm.cand_idx[slot] = j0 + i;
-          }
-        }
-      }
-      my_keep += n_in;
-      n_in = block_count<THREADS>(n_in, 0, sm);
-      const int n_cand = sm.counts[0];
-      const int need = k - nf - n_in;
-      if (n_cand > SEL_CAND_CAP) {
-        if (tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
-        mode = 3;
-        my_keep = 0;
-#pragma unroll 1
-        for (int i = 0; i < per; ++i) {
-          const uint32_t kk = key(i);
-          my_keep += kk > key_thr && kk != 0u;
-          my_ties += kk == key_thr;
-        }
-      } else {
-        if (n_cand != need) {
-          if (tid == 0) atomicAdd(p.status + ST_TOK_REFINED, n_cand);
-          for (int e = tid; e < hd; e += THREADS) {
-            double a = 0.0;
-            for (int h = 0; h < G; ++h) a += (double)p.q_rot[((size_t)b * p.sh.n_q_heads + kvh * G + h) * hd + e];
-            qsum[e] = a;
-          }
-          __syncthreads();
-          const uint16_t* kp = static_cast<const uint16_t*>(p.kv.k_pool);
-          for (int c = warp; c < n_cand; c += WARPS) {
-            const int j = sm.cand_idx[c];
-            const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + j / PAGE];
-            double a = 0.0;
-            if (page >= 0 && page < p.kv.num_pages) {
-              const uint16_t* kr = kp + (((size_t)page * Hkv + kvh) * PAGE + (j % PAGE)) * hd;
-              for (int e = lane; e < hd; e += 32) a += qsum[e] * (double)bf2f(kr[e]);
-            }
-            a = warp_sum_d(a);
-            if (lane == 0) sm.cand_val[c] = a;
-          }
-          __syncthreads();
-          rank_candidates<THREADS>(n_cand, need, sm);
-        } else {
-          for (int c = tid; c < n_cand; c += THREADS) sm.cand_keep[c] = 1;
-        }
-        mode = 2;
-        __syncthreads();
-        // the key slot of every candidate takes its class: a kept one sorts above every key, a dropped
-        // one below (token j is slot j % per of thread j / per), so that one comparison with the window
-        // classifies any slot from here on
-        for (int c = tid; c < n_cand; c += THREADS) {
-          const int j = sm.cand_idx[c];
-          skey[(j % per) * THREADS + j / per] = sm.cand_keep[c] ? 0xffffffffu : 0u;
-        }
-        __syncthreads();
-        if (my_cand > 0) {  // few threads own candidates: they count their kept ones
-#pragma unroll 1
-          for (int i = 0; i < per; ++i) {
-            const uint32_t kk = key(i);
-            // a forced token or a kept candidate now; the forced ones were counted above
-            my_keep += kk == 0xffffffffu && !(j0 + i < T && forced(j0 + i));
-          }
-        }
-        key_thr = float_key(hi);  // kept: keys above the window (candidates inside it are settled)
       }
     }
-
-    // class of this thread's i-th token: 2 kept, 1 tie, 0 dropped
-    auto klass = [&](int i) -> int {
-      const int j = j0 + i;
-      if (j >= T) return 0;
-      if (mode == 0) return 2;
-      if (mode == 1) return forced(j) ? 2 : 0;
-      const uint32_t kk = key(i);
-      if (mode == 2) return kk > key_thr ? 2 : 0;
-      return kk > key_thr ? 2 : (kk == key_thr ? 1 : 0);
-    };
-    // beside the index list, the cache row of every kept token (page table applied), so that pass 2
-    // goes from the list straight to the V rows
-    const int32_t* table = p.kv.page_table + (size_t)b * p.kv.max_pages_per_seq;
-    auto emit = [&](int i, bool keep, int pos) {
-      if (!keep) return;
-      const int j = j0 + i;
-      const int page = table[j / PAGE];
-      uint32_t ridx = 0xffffffffu;
-      if (page >= 0 && page < p.kv.num_pages) ridx = (uint32_t)((page * Hkv + kvh) * PAGE + (j % PAGE));
-      else atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
-      p.kept_row[row + pos] = ridx;
-    };
-    total = compact_counted<THREADS, KPT>(my_keep, my_ties, klass, emit, mode == 3 ? tie_need : 0, p.kept_idx + row,
-                                          sm, per);
+    mx = block_max<TS_THREADS>(mx, 0, sm);
+    __syncthreads();
+    if (nseg > 1) {
+      for (int i = tid; i < SEL_BINS; i += TS_THREADS) {
+        const uint32_t c = sm.hist[i];
+        if (c) atomicAdd(gh + i, c);
+      }
+      if (tid == 0) atomicMax(ctl + RC_MAX, __float_as_uint(mx));
+    }
   }
-  if (tid == 0) p.kept_cnt[bk] = total;
+  if (nseg > 1) {  // only the CTA that arrives last goes on
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_flag = atomicAdd(ctl + RC_DONE, 1u) == (uint32_t)(nseg - 1) ? 1 : 0;
+    __syncthreads();
+    if (!s_flag) return;
+    __threadfence();
+  }
+
+  // ------------------------------------------------------------- phase 2 ----
+  if (tid < TS_MAX_SEGS) seg_cnt[tid] = 0;
+  if (tid < 4) sm.counts[tid] = 0;
+  float edge = TS_FLT_MAX;  // kept <=> score > edge (after the patches below)
+  if (mode == 2) {
+    if (nseg > 1) {
+      for (int i = tid; i < SEL_BINS; i += TS_THREADS) sm.hist[i] = __ldcg(gh + i);
+      mx = __uint_as_float(__ldcg(ctl + RC_MAX));
+    }
+    __syncthreads();
+    const int need_total = k - nf;
+    // the bin that holds the `want`-th largest of the histogrammed scores, and how many lie above it:
+    // thread t owns bins 4095 - 16 t .. 4080 - 16 t
+    auto rank_bin = [&](int want) {
+      constexpr int BPT = SEL_BINS / TS_THREADS;
+      int mine = 0;
+#pragma unroll
+      for (int q = 0; q < BPT; ++q) mine += (int)sm.hist[SEL_BINS - 1 - tid * BPT - q];
+      int total;
+      const int before = ts_block_scan(mine, total, sm.scan[0]);
+      if (before < want && want <= before + mine) {
+        int a = before;
+        for (int q = 0; q < BPT; ++q) {
+          const int bin = SEL_BINS - 1 - tid * BPT - q;
+          const int c = (int)sm.hist[bin];
+          if (want <= a + c) {
+            sm.pick[0] = bin;
+            sm.pick[2] = a;
+            break;
+          }
+          a += c;
+        }
+      }
+      __syncthreads();
+    };
+    rank_bin(need_total);
+    const int vbin = sm.pick[0], above_bin = sm.pick[2];
+    uint32_t klo, khi;
+    value_bin_key_range(vbin, klo, khi);
+    // 2^-16 of the largest score: far above the float32 accumulation error of a head_dim-long dot product
+    const float delta = mx * 1.52587890625e-05f;
+    float lo = key_to_float(klo) - delta;
+    edge = fminf(key_to_float(khi) + delta, TS_FLT_MAX);
+
+    // one pass over the row: count what is above the edge per segment, list what lies between lo and the edge
+    auto run_pass = [&]() -> int {
+      int n_above_edge = 0;
+#pragma unroll 1
+      for (int wbase = warp * 256; wbase < T; wbase += TS_THREADS * 8) {  // a warp's 256 tokens lie in one segment
+        const int base = wbase + lane * 8;
+        int c8 = 0;
+        if (base < T) {
+          const float4 v0 = *reinterpret_cast<const float4*>(sig + base), v1 = *reinterpret_cast<const float4*>(sig + base + 4);
+          const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const int j = base + e;
+            if (j < T && !forced(j)) {
+              if (vv[e] > edge) {
+                ++c8;
+              } else if (vv[e] >= lo) {
+                const int slot = atomicAdd(&sm.counts[0], 1);
+                if (slot < SEL_CAND_CAP) {
+                  sm.cand_idx[slot] = j;
+                  sup_val[slot] = vv[e];
+                }
+              }
+            }
+          }
+        }
+        n_above_edge += c8;
+        c8 = __reduce_add_sync(0xffffffffu, c8);
+        if (c8 && lane == 0) atomicAdd(&seg_cnt[wbase / TS_SEG], c8);
+      }
+      n_above_edge = block_count<TS_THREADS>(n_above_edge, 0, sm);
+      __syncthreads();
+      return n_above_edge;
+    };
+    int n_hi = run_pass();
+    const bool prefix_bin = vbin != 0 && vbin != SEL_BINS / 2 - 1 && vbin != SEL_BINS / 2 && vbin != SEL_BINS - 1;
+    if (sm.counts[0] > SEL_CAND_CAP && prefix_bin) {
+      // The bin and its window hold more scores than the list: histogram the next 12 key bits of the bin's
+      // keys (they share their upper 15 bits), take the sub-bin of the k-th score and list again.
+      for (int i = tid; i < SEL_BINS; i += TS_THREADS) sm.hist[i] = 0;
+      if (tid < TS_MAX_SEGS) seg_cnt[tid] = 0;
+      if (tid == 0) sm.counts[0] = 0;
+      __syncthreads();
+#pragma unroll 1
+      for (int j = tid; j < T; j += TS_THREADS) {
+        if (forced(j)) continue;
+        const uint32_t kk = float_key(sig[j] + 0.0f);
+        if (kk >= klo && kk <= khi) atomicAdd(&sm.hist[(kk >> 5) & 0xfffu], 1u);
+      }
+      __syncthreads();
+      rank_bin(need_total - above_bin);
+      const uint32_t klo2 = (klo & 0xfffe0000u) | ((uint32_t)sm.pick[0] << 5), khi2 = klo2 | 31u;
+      lo = key_to_float(klo2) - delta;
+      edge = fminf(key_to_float(khi2) + delta, TS_FLT_MAX);
+      n_hi = run_pass();
+    }
+    const int ns = sm.counts[0];
+    const int need_s = need_total - n_hi;
+    if (ns > SEL_CAND_CAP || need_s < 1 || need_s > ns) {
+      mode = 3;
+    } else {
+      // float32 rank inside the list: the element of rank need_s - 1 carries the k-th value
+      for (int c = tid; c < ns; c += TS_THREADS) {
+        const float v = sup_val[c];
+        const int j = sm.cand_idx[c];
+        int rank = 0;
+        for (int o = 0; o < ns; ++o) {
+          const float vo = sup_val[o];
+          rank += (vo > v) || (vo == v && sm.cand_idx[o] < j);
+        }
+        if (rank == need_s - 1) sm.pick[1] = __float_as_int(v);
+      }
+      __syncthreads();
+      const float thr32 = __int_as_float(sm.pick[1]);
+      const float whi = thr32 + delta, wlo = thr32 - delta;
+      // classes: above the window (kept, ranks first), inside it (re-scored), below it (dropped)
+      int n_above = 0, n_in = 0;
+      for (int c = tid; c < ns; c += TS_THREADS) {
+        const float v = sup_val[c];
+        unsigned char cls = 0;
+        if (v > whi) {
+          cls = 1;
+          ++n_above;
+          sm.cand_val[c] = 1.0e300;
+        } else if (v >= wlo) {
+          cls = 2;
+          ++n_in;
+          sm.cand_val[c] = (double)v;
+        } else {
+          sm.cand_val[c] = -1.0e300;
+        }
+        sm.cand_keep[c] = cls;
+      }
+      n_above = block_count<TS_THREADS>(n_above, 0, sm);
+      n_in = block_count<TS_THREADS>(n_in, 1, sm);
+      __syncthreads();
+      if (n_above + n_in != need_s) {  // the window holds more than are needed: settle it in float64
+        if (tid == 0) atomicAdd(p.status + ST_TOK_REFINED, n_in);
+        for (int e = tid; e < hd; e += TS_THREADS) {
+          double a = 0.0;
+          for (int h = 0; h < G; ++h) a += (double)p.q_rot[((size_t)b * p.sh.n_q_heads + kvh * G + h) * hd + e];
+          qsum[e] = a;
+        }
+        __syncthreads();
+        const uint16_t* kp = static_cast<const uint16_t*>(p.kv.k_pool);
+        for (int c = warp; c < ns; c += WARPS) {
+          if (sm.cand_keep[c] != 2) continue;  // warp-uniform
+          const int j = sm.cand_idx[c];
+          const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + j / PAGE];
+          double a = 0.0;
+          if (page >= 0 && page < p.kv.num_pages) {
+            const uint16_t* kr = kp + (((size_t)page * Hkv + kvh) * PAGE + (j % PAGE)) * hd;
+            for (int e = lane; e < hd; e += 32) a += qsum[e] * (double)bf2f(kr[e]);
+          }
+          a = warp_sum_d(a);
+          if (lane == 0) sm.cand_val[c] = a;
+        }
+        __syncthreads();
+      }
+      rank_candidates<TS_THREADS>(ns, need_s, sm);  // cand_keep[c] = 1 for the need_s best of the list
+      __syncthreads();
+      for (int c = tid; c < ns; c += TS_THREADS) {
+        if (sm.cand_keep[c]) {
+          const int j = sm.cand_idx[c];
+          sig[j] = INFINITY;
+          atomicAdd(&seg_cnt[j / TS_SEG], 1);
+        }
+      }
+    }
+  }
+
+  if (mode == 3) {
+    // More scores inside the list's range than it holds (long runs of equal or nearly equal scores): exact
+    // float32 order with ties to the lower index, by a radix select over the row's keys in global memory.
+    if (tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
+    __syncthreads();
+    if (tid < TS_MAX_SEGS) seg_cnt[tid] = 0;
+    const int per = (T + TS_THREADS - 1) / TS_THREADS;
+    auto key = [&](int i) -> uint32_t {
+      const int j = i * TS_THREADS + tid;
+      return (j < T && !forced(j)) ? float_key(sig[j] + 0.0f) : 0u;
+    };
+    int tie_need = 0;
+    const uint32_t key_thr = select_kth<TS_THREADS, 0, true>(key, k - nf, tie_need, sm, per);
+    edge = fminf(key_to_float(key_thr), TS_FLT_MAX);
+    int ties_taken = 0;
+#pragma unroll 1
+    for (int base0 = 0; base0 < T; base0 += TS_SEG) {  // in index order: ties are kept until tie_need runs out
+      const int j0 = base0 + tid * 8;
+      int above = 0, ties = 0;
+      uint32_t tie_mask = 0;
+      if (j0 < T) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int j = j0 + e;
+          if (j < T && !forced(j)) {
+            const uint32_t kk = float_key(sig[j] + 0.0f);
+            above += kk > key_thr;
+            if (kk == key_thr) {
+              ++ties;
+              tie_mask |= 1u << e;
+            }
+          }
+        }
+      }
+      int tot_ties;
+      const int t_before = ties_taken + ts_block_scan(ties, tot_ties, sm.scan[0]);
+      int taken = 0;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        if (((tie_mask >> e) & 1u) && t_before + taken < tie_need) {
+          sig[j0 + e] = INFINITY;
+          ++taken;
+        }
+      }
+      const int kept_here = block_count<TS_THREADS>(above + taken, 1, sm);
+      if (tid == 0) seg_cnt[base0 / TS_SEG] = kept_here;
+      ties_taken += tot_ties;
+    }
+    __syncthreads();
+  }
+
+  // forced tokens are kept whatever their score
+  if (mode != 0) {
+    for (int f = tid; f < nf; f += TS_THREADS) {
+      const int j = f < n_sink ? f : T - n_win + (f - n_sink);
+      sig[j] = INFINITY;
+      atomicAdd(&seg_cnt[j / TS_SEG], 1);
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int total = 0;
+    for (int s = 0; s < nseg; ++s) {
+      soff[s] = total;
+      total += mode == 0 ? min(TS_SEG, T - s * TS_SEG) : seg_cnt[s];
+    }
+    if (T <= 0) total = 0;
+    ctl[RC_MODE] = (uint32_t)mode;
+    ctl[RC_EDGE] = __float_as_uint(edge);
+    p.kept_cnt[bk] = total;
+    sm.counts[2] = total;
+  }
+  __syncthreads();
+  const int total = sm.counts[2];
 
   // Pass-2 work items of this (sequence, kv-head): runs of `cpi` chunks of split_len kept tokens (at least
-  // one item, so that the output is always written); cpi was chosen by the query preparation kernel.
+  // one item, so that the output is always written); cpi was chosen by the first CTA of the score pass.
   const int cpi = p.work_ctr[WC_CPI];
   const int chunks = max(1, (total + p.split_len - 1) / p.split_len);
-  const int ns = (chunks + cpi - 1) / cpi;
-  if (tid == 0) sm.counts[3] = atomicAdd(p.work_ctr + WC_ITEMS, ns);
+  const int ns_items = (chunks + cpi - 1) / cpi;
+  if (tid == 0) sm.counts[3] = atomicAdd(p.work_ctr + WC_ITEMS, ns_items);
   __syncthreads();
-  const int base = sm.counts[3];
-  for (int i = tid; i < ns; i += THREADS) {
-    p.work_items[2 * (base + i)] = bk * p.S + i * cpi;  // first chunk of the item
-    p.work_items[2 * (base + i) + 1] = total;
+  const int item0 = sm.counts[3];
+  for (int i = tid; i < ns_items; i += TS_THREADS) {
+    p.work_items[2 * (item0 + i)] = bk * p.S + i * cpi;  // first chunk of the item
+    p.work_items[2 * (item0 + i) + 1] = total;
+  }
+}
+
+struct CompactDev {
+  sol_kv_t kv;
+  int Hkv, Tmax, nseg_max;
+  const float* sigma;
+  const uint32_t* row_ctl;
+  const int32_t* seg_off;
+  int32_t* kept_idx;   // [B*Hkv][Tmax] ascending
+  uint32_t* kept_row;  // same layout: cache row (page table applied), 0xffffffff: bad page
+  int* status;
+};
+
+__global__ void __launch_bounds__(TS_THREADS) token_compact_kernel(const CompactDev p) {
+  __shared__ int warp_tot[TS_THREADS / 32];
+  const int seg = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x;
+  pdl_trigger();
+  const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);
+  if (seg * TS_SEG >= T) return;
+  pdl_wait();
+  const int bk = b * p.Hkv + kvh;
+  const size_t row = (size_t)bk * p.Tmax;
+  const uint32_t mode = p.row_ctl[(size_t)bk * RC_WORDS + RC_MODE];
+  const float edge = __uint_as_float(p.row_ctl[(size_t)bk * RC_WORDS + RC_EDGE]);
+  const int off = p.seg_off[(size_t)bk * p.nseg_max + seg];
+  const int j0 = seg * TS_SEG + tid * 8;
+  uint32_t keep = 0;
+  if (j0 < T) {
+    if (mode == 0) {
+      keep = T - j0 >= 8 ? 0xffu : ((1u << (T - j0)) - 1u);
+    } else {
+      const float4 v0 = *reinterpret_cast<const float4*>(p.sigma + row + j0);
+      const float4 v1 = *reinterpret_cast<const float4*>(p.sigma + row + j0 + 4);
+      const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if (j0 + e < T && vv[e] > edge) keep |= 1u << e;
+    }
+  }
+  int total;
+  int pos = off + ts_block_scan(__popc(keep), total, warp_tot);
+  if (keep) {
+    // eight consecutive tokens share a page
+    const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + j0 / PAGE];
+    const bool ok = page >= 0 && page < p.kv.num_pages;
+    if (!ok) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+    const uint32_t r0 = (uint32_t)((page * p.Hkv + kvh) * PAGE + (j0 % PAGE));
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      if ((keep >> e) & 1u) {
+        p.kept_idx[row + pos] = j0 + e;
+        p.kept_row[row + pos] = ok ? r0 + e : 0xffffffffu;
+        ++pos;
+      }
+    }
   }
 }
 
@@ -858,6 +1099,7 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   pd.qkv_scale = a.qkv_scale;
   pd.q_bf16 = static_cast<const uint16_t*>(a.q_bf16);
   pd.q_rot = a.q_rot; pd.q_split = static_cast<uint16_t*>(a.q_split); pd.work_ctr = a.work_ctr; pd.status = a.status;
+  pd.row_hist = a.row_hist; pd.row_ctl = a.row_ctl;
   SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(Hkv, a.B), dim3(PREP_THREADS), 0, st, pd);
 
   ScoreDev sd;
@@ -874,22 +1116,16 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   SelectDev se;
   se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.S = a.splits;
   se.split_len = attn_split_len(hd); se.q_rot = a.q_rot; se.B = a.B;
-  se.sigma = a.sigma; se.kept_idx = a.kept_idx; se.kept_cnt = a.kept_cnt; se.kept_row = a.kept_row;
-  se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
-  {
-    // keys of the longest row in shared memory: 4 bytes per token, rounded up to four per thread; rows up
-    // to 1024 tokens take 256 threads, longer ones 1024
-    const dim3 grid(Hkv, a.B);
-    if (Tmax <= 1024) {
-      const int smem = ((Tmax + 256 - 1) / 256 + 3) / 4 * 4 * 256 * 4;
-      ensure_dynamic_smem(reinterpret_cast<const void*>(&token_select_kernel<256>), smem);
-      SOL_LAUNCH("token_select", token_select_kernel<256>, grid, dim3(256), smem, st, se);
-    } else {
-      const int smem = ((Tmax + 1024 - 1) / 1024 + 3) / 4 * 4 * 1024 * 4;
-      ensure_dynamic_smem(reinterpret_cast<const void*>(&token_select_kernel<1024>), smem);
-      SOL_LAUNCH("token_select", token_select_kernel<1024>, grid, dim3(1024), smem, st, se);
-    }
-  }
+  se.nseg_max = attn_select_segs(a.kv.max_pages_per_seq, PAGE);
+  se.sigma = a.sigma; se.row_hist = a.row_hist; se.row_ctl = a.row_ctl; se.seg_off = a.seg_off;
+  se.kept_cnt = a.kept_cnt; se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
+  const dim3 seg_grid(se.nseg_max, Hkv, a.B);
+  SOL_LAUNCH("token_select", token_select_kernel, seg_grid, dim3(TS_THREADS), 0, st, se);
+
+  CompactDev cd;
+  cd.kv = a.kv; cd.Hkv = Hkv; cd.Tmax = Tmax; cd.nseg_max = se.nseg_max; cd.sigma = a.sigma; cd.row_ctl = a.row_ctl;
+  cd.seg_off = a.seg_off; cd.kept_idx = a.kept_idx; cd.kept_row = a.kept_row; cd.status = a.status;
+  SOL_LAUNCH("token_compact", token_compact_kernel, seg_grid, dim3(TS_THREADS), 0, st, cd);
 
   GatherDev gd;
   gd.kv = a.kv; gd.Hq = Hq; gd.Hkv = Hkv; gd.G = G; gd.Tmax = Tmax; gd.S = a.splits;

@@ -118,6 +118,11 @@ inline int attn_splits(int head_dim, int max_pages, int page_size) {
   const int s = (max_pages * page_size + len - 1) / len;
   return s < 1 ? 1 : s;
 }
+// CTAs per row of the token selection: one per 2048 tokens.
+inline int attn_select_segs(int max_pages, int page_size) {
+  const int s = (max_pages * page_size + 2047) / 2048;
+  return s < 1 ? 1 : s;
+}
 constexpr int ATTN_ITEM_CHUNKS = 16;  // chunks of attn_split_len kept tokens per pass-2 work item at most
 struct AttnArgs {
   sol_shape_t shape;
@@ -136,6 +141,9 @@ struct AttnArgs {
   void* q_split;        // bf16 [B][Hkv][HG*16][hd]
   float* logits;        // [B][Hkv][Tmax][G]
   float* sigma;         // [B][Hkv][Tmax]
+  uint32_t* row_hist;   // [B][Hkv][4096] histogram of a row's scores (rows that span several selection CTAs)
+  uint32_t* row_ctl;    // [B][Hkv][4] selection state of a row
+  int32_t* seg_off;     // [B][Hkv][segments] offsets of the 2048-token segments in the row's kept list
   int32_t* kept_idx;    // [B][Hkv][Tmax] kept tokens, ascending (the caller's array when it asks for the list)
   int32_t* kept_cnt;    // [B][Hkv]
   uint32_t* kept_row;   // same layout as kept_idx: cache row (page table applied) of every kept token,
@@ -155,7 +163,7 @@ struct AttnArgs {
 
 // Offsets of the attention scratch inside a buffer, starting at `at` (a multiple of 256).
 struct AttnScratch {
-  size_t q_rot, q_split, logits, sigma, kept_idx, kept_cnt, kept_row, part, work_items, work_ctr, end;
+  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_off, kept_idx, kept_cnt, kept_row, part, work_items, work_ctr, end;
   int splits;
 };
 inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_pages, size_t at) {
@@ -172,6 +180,9 @@ inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_page
   L.q_split = take(BK * HG * 16 * hd * 2);
   L.logits = take(BK * Tmax * G * 4);
   L.sigma = take(BK * Tmax * 4);
+  L.row_hist = take(BK * 4096 * 4);
+  L.row_ctl = take(BK * 4 * 4);
+  L.seg_off = take(BK * (size_t)attn_select_segs(max_pages, s.page_size) * 4);
   L.kept_idx = take(BK * Tmax * 4);
   L.kept_cnt = take(BK * 4);
   L.kept_row = take(BK * Tmax * 4);
@@ -188,6 +199,9 @@ inline void attn_scratch_bind(AttnArgs& a, void* base, const AttnScratch& L, int
   a.q_split = b + L.q_split;
   a.logits = reinterpret_cast<float*>(b + L.logits);
   a.sigma = reinterpret_cast<float*>(b + L.sigma);
+  a.row_hist = reinterpret_cast<uint32_t*>(b + L.row_hist);
+  a.row_ctl = reinterpret_cast<uint32_t*>(b + L.row_ctl);
+  a.seg_off = reinterpret_cast<int32_t*>(b + L.seg_off);
   a.kept_idx = kept_idx ? kept_idx : reinterpret_cast<int32_t*>(b + L.kept_idx);
   a.kept_cnt = kept_cnt ? kept_cnt : reinterpret_cast<int32_t*>(b + L.kept_cnt);
   a.kept_row = reinterpret_cast<uint32_t*>(b + L.kept_row);

@@ -78,6 +78,23 @@ __device__ __forceinline__ int key_value_bin(uint32_t key) {
   return (u >> 31) ? SEL_BINS / 2 - 1 - m : SEL_BINS / 2 + m;
 }
 
+// Smallest and largest key of a value bin: key_value_bin(key) == bin exactly for klo <= key <= khi (keys of
+// NaNs aside: the clamped end bins stop at the keys of -inf and +inf).
+__device__ __forceinline__ void value_bin_key_range(int bin, uint32_t& klo, uint32_t& khi) {
+  const bool pos = bin >= SEL_BINS / 2;
+  const int m = pos ? bin - SEL_BINS / 2 : SEL_BINS / 2 - 1 - bin;
+  // magnitudes of the bin as float bit patterns without the sign
+  const uint32_t mlo = m == 0 ? 0u : (uint32_t)(m + (VB_EXP0 << 6)) << 17;
+  const uint32_t mhi = m == SEL_BINS / 2 - 1 ? 0x7f800000u : (((uint32_t)(m + (VB_EXP0 << 6)) + 1u) << 17) - 1u;
+  if (pos) {
+    klo = mlo | 0x80000000u;
+    khi = mhi | 0x80000000u;
+  } else {
+    klo = 0x7fffffffu - mhi;
+    khi = 0x7fffffffu - mlo;
+  }
+}
+
 // The k-th largest of the block's keys (1 <= k <= number of keys); key(i), i < per_thread, are a
 // thread's keys.  Absent elements carry key 0 and count like any other key, so k must not
 // exceed the number of present elements.  tie_need = how many
