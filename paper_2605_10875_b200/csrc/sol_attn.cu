@@ -43,15 +43,17 @@ struct PrepDev {
   int32_t* work_ctr;  // zeroed here: [0] items emitted, [1] next item, [2 + b*Hkv + kvh] finished items
   uint32_t* row_hist; // zeroed here: [B*Hkv][SEL_BINS] score histogram of rows that span several selection CTAs
   uint32_t* row_ctl;  // zeroed here: [B*Hkv][RC_WORDS]
+  uint32_t* seg_pub;  // zeroed here: [B*Hkv][nseg_max]
+  int nseg_max;
   int* status;
 };
 
 constexpr int PREP_THREADS = 128;
 // words of AttnArgs::work_ctr
 enum : int { WC_ITEMS = 0, WC_NEXT = 1, WC_CPI = 2, WC_DONE = 4 };
-// words of AttnArgs::row_ctl, per (sequence, kv-head): token selection CTAs finished, largest |score| (float
-// bits), the keep edge (float bits), the selection mode
-enum : int { RC_DONE = 0, RC_MAX = 1, RC_EDGE = 2, RC_MODE = 3, RC_WORDS = 4 };
+// words of AttnArgs::row_ctl, per (sequence, kv-head): histogram CTAs finished, largest |score|, keep edge,
+// drop edge, window (float bits), tickets drawn by the scan CTAs, candidates listed, scan CTAs finished
+enum : int { RC_DONE1 = 0, RC_MAX, RC_EDGE, RC_LO, RC_DELTA, RC_TICKET, RC_NCAND, RC_DONE2, RC_WORDS };
 
 // One CTA per (kv-head, sequence): the G query heads of the group, the new k row and the new v row.
 __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p) {
@@ -99,7 +101,8 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
   }
   // scratch of the token selection of this (sequence, kv-head)
   if (tid < RC_WORDS) p.row_ctl[(size_t)(b * Hkv + kvh) * RC_WORDS + tid] = 0u;
-  if (T > 2048) {  // rows of one selection CTA keep their histogram in shared memory
+  if (tid < p.nseg_max) p.seg_pub[(size_t)(b * Hkv + kvh) * p.nseg_max + tid] = 0u;
+  if (T > 8192) {  // rows of one histogram CTA keep their histogram in shared memory
     uint4* hz = reinterpret_cast<uint4*>(p.row_hist + (size_t)(b * Hkv + kvh) * SEL_BINS);
     for (int i = tid; i < SEL_BINS / 4; i += PREP_THREADS) hz[i] = make_uint4(0u, 0u, 0u, 0u);
   }
@@ -327,25 +330,32 @@ __global__ void __launch_bounds__(SC_WARPS * 32) attn_score_kernel(const ScoreDe
 }
 
 // ============================================================================
-// token_select + token_compact
+// token selection: token_hist, token_scan (+ token_list)
 // ============================================================================
-// Exact top-k of a (sequence, kv-head) row of scores, spread over one CTA per 2048 tokens.
+// Exact top-k of a (sequence, kv-head) row of scores in two kernels, both spread over the row.
 //
-//   phase 1 (every CTA of the row): histogram of the CTA's scores over 4096 value bins in shared memory,
-//            flushed (non-empty bins only) to the row's histogram in global memory, and the largest |score|;
-//   phase 2 (the CTA that finishes last; rows of one CTA go straight on): the bin that holds the k-th
-//            largest score; one pass over the row's scores counts, per 2048-token segment, what lies above
-//            that bin (by more than a small window) and lists what lies in it or within the window; the
-//            list is ranked in float32, everything within the window of the k-th value is re-scored in
-//            float64 from the cache rows, and the listed tokens that are kept get their score replaced by
-//            +inf, as do the forced tokens.  From then on "kept" is the single comparison score > edge.
+//   token_hist   one CTA per 8192 tokens: histogram of its scores over 4096 value bins in shared memory,
+//                flushed (non-empty bins) to the row's histogram in global memory, and the largest |score|.
+//                The CTA that finishes last (rows of one CTA go straight on) finds the bin of the k-th
+//                largest score and publishes two values: everything above `edge` (the bin's upper end plus
+//                a small window) is kept, everything below `lo` is dropped.
+//   token_scan   one CTA per 2048 tokens: kept tokens (above the edge, or forced) go to the row's list at
+//                the place given by the counts of the CTAs before it (each CTA publishes its count and
+//                adds up those of its predecessors; tickets make sure the predecessors are running);
+//                the few tokens between lo and edge are appended to a candidate list.  The CTA that
+//                finishes last ranks the candidates in float32, re-scores those within the window of the
+//                k-th value in float64 from the cache rows, and appends the kept ones (ascending) to the list.
+//   token_list   only when a caller asks for the kept indices: the ascending list, from the patched scores
+//                (kept candidates and forced tokens get +inf, so "kept" is the comparison score > edge).
 //
-// token_compact (one CTA per 2048 tokens again) turns that comparison into the ascending index list and
-// the page-resolved cache row of every kept token, at the offsets phase 2 derived from the segment counts.
+// The row's list (token index and page-resolved cache row of every kept token) is what pass 2 reads: segment
+// by segment ascending, the settled candidates last; the order is the same on every run.
 constexpr int TS_THREADS = 256;
-constexpr int TS_SEG = 2048;                                      // tokens per CTA
+constexpr int TH_SEG = 8192;                                      // tokens per token_hist CTA
+constexpr int TS_SEG = 2048;                                      // tokens per token_scan CTA
 constexpr int TS_MAX_SEGS = MAX_PAGES_PER_SEQ * PAGE / TS_SEG;     // 24
 constexpr float TS_FLT_MAX = 3.402823466e+38f;
+constexpr uint32_t TS_READY = 0x80000000u;
 
 struct SelectDev {
   sol_shape_t sh;
@@ -353,10 +363,14 @@ struct SelectDev {
   const int32_t* r_permille;
   int Tmax, S, split_len, B, nseg_max;
   const float* q_rot;
-  float* sigma;          // kept listed tokens and forced tokens are overwritten with +inf
+  float* sigma;          // kept candidates and forced tokens are overwritten with +inf (for token_list)
   uint32_t* row_hist;    // [B*Hkv][SEL_BINS], zero on entry
   uint32_t* row_ctl;     // [B*Hkv][RC_WORDS], zero on entry
-  int32_t* seg_off;      // [B*Hkv][nseg_max] first place of each segment's kept tokens in the row's list
+  uint32_t* seg_pub;     // [B*Hkv][nseg_max] kept count of each 2048-token segment | TS_READY, zero on entry
+  int32_t* cand_idx;     // [B*Hkv][SEL_CAND_CAP]
+  float* cand_val;       // [B*Hkv][SEL_CAND_CAP]
+  int32_t* list_idx;     // [B*Hkv][Tmax] token index of every kept token
+  uint32_t* list_row;    // same layout: its cache row (page table applied), 0xffffffff: bad page
   int32_t* kept_cnt;
   int32_t* work_items;
   int32_t* work_ctr;
@@ -386,183 +400,354 @@ __device__ __forceinline__ int ts_block_scan(int v, int& total, int* warp_tot) {
   return before;
 }
 
-__global__ void __launch_bounds__(TS_THREADS) token_select_kernel(const SelectDev p) {
-  __shared__ SelectSmem sm;
-  __shared__ float sup_val[SEL_CAND_CAP];
-  __shared__ double qsum[128];
-  __shared__ int seg_cnt[TS_MAX_SEGS];
-  __shared__ int s_flag;
+// What every selection kernel derives from a row's length and keep-rate.
+struct RowPlan {
+  int T, n_sink, n_win, nf, k, mode;  // mode 0: keep all; 1: forced only; 2: selection
+  __device__ __forceinline__ bool forced(int j) const { return j < n_sink || j >= T - n_win; }
+};
+__device__ __forceinline__ RowPlan row_plan(const sol_shape_t& sh, const sol_kv_t& kv, const int32_t* r_permille, int b) {
+  RowPlan r;
+  r.T = min(kv.seq_lens[b], kv.max_pages_per_seq * PAGE);  // never index past the page table
+  const int Tp = max(r.T, 0);
+  r.n_sink = min(max(sh.n_sink, 0), Tp);
+  r.n_win = min(max(sh.n_window, 0), Tp - r.n_sink);
+  r.nf = r.n_sink + r.n_win;
+  long long bud = ((long long)r_permille[b] * Tp + 999) / 1000;
+  if (bud > Tp) bud = Tp;
+  r.k = min(Tp, max((int)bud, r.nf));
+  r.mode = r.k >= Tp ? 0 : (r.k <= r.nf ? 1 : 2);
+  return r;
+}
 
+__global__ void __launch_bounds__(TS_THREADS) token_hist_kernel(const SelectDev p) {
+  __shared__ uint32_t hist[SEL_BINS];
+  __shared__ int scan_tot[TS_THREADS / 32];
+  __shared__ float fmax_w[TS_THREADS / 32];
+  __shared__ int pick[2];
+  __shared__ int s_flag;
   const int seg = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  pdl_trigger();
+  // lengths and keep-rates are inputs of the step, not the work of an earlier kernel
+  const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, b);
+  const int T = rp.T;
+  if (rp.mode != 2 || seg * TH_SEG >= T) return;
+  for (int i = tid; i < SEL_BINS; i += TS_THREADS) hist[i] = 0;
+  pdl_wait();
+  __syncthreads();
+  const int bk = b * p.sh.n_kv_heads + kvh;
+  const float* sig = p.sigma + (size_t)bk * p.Tmax;
+  uint32_t* ctl = p.row_ctl + (size_t)bk * RC_WORDS;
+  uint32_t* gh = p.row_hist + (size_t)bk * SEL_BINS;
+  const int nseg = (T + TH_SEG - 1) / TH_SEG;
+
+  // ---- this CTA's scores: 32 per thread, all loads issued before the first use ----
+  float mx = 0.f;
+  {
+    constexpr int VPT = TH_SEG / TS_THREADS / 4;  // float4 loads per thread
+    float4 v[VPT];
+#pragma unroll
+    for (int q = 0; q < VPT; ++q) {
+      const int j = seg * TH_SEG + (q * TS_THREADS + tid) * 4;
+      v[q] = j < T ? *reinterpret_cast<const float4*>(sig + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int q = 0; q < VPT; ++q) {
+      const int j0 = seg * TH_SEG + (q * TS_THREADS + tid) * 4;
+      const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int j = j0 + e;
+        if (j < T && !rp.forced(j)) {
+          atomicAdd(&hist[key_value_bin(float_key(vv[e]))], 1u);
+          mx = fmaxf(mx, fabsf(vv[e]));
+        }
+      }
+    }
+  }
+  mx = warp_max(mx);
+  if (lane == 0) fmax_w[warp] = mx;
+  __syncthreads();
+  mx = 0.f;
+#pragma unroll
+  for (int w = 0; w < TS_THREADS / 32; ++w) mx = fmaxf(mx, fmax_w[w]);
+  if (nseg > 1) {  // only the CTA that arrives last goes on
+    for (int i = tid; i < SEL_BINS; i += TS_THREADS) {
+      const uint32_t c = hist[i];
+      if (c) atomicAdd(gh + i, c);
+    }
+    if (tid == 0) atomicMax(ctl + RC_MAX, __float_as_uint(mx));
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_flag = atomicAdd(ctl + RC_DONE1, 1u) == (uint32_t)(nseg - 1) ? 1 : 0;
+    __syncthreads();
+    if (!s_flag) return;
+    __threadfence();
+    for (int i = tid; i < SEL_BINS; i += TS_THREADS) hist[i] = __ldcg(gh + i);
+    mx = __uint_as_float(__ldcg(ctl + RC_MAX));
+    __syncthreads();
+  }
+
+  // ---- the bin that holds the `want`-th largest of the histogrammed scores, and how many lie above it:
+  //      thread t owns bins 4095 - 16 t .. 4080 - 16 t
+  auto rank_bin = [&](int want) {
+    constexpr int BPT = SEL_BINS / TS_THREADS;
+    int mine = 0;
+#pragma unroll
+    for (int q = 0; q < BPT; ++q) mine += (int)hist[SEL_BINS - 1 - tid * BPT - q];
+    int total;
+    const int before = ts_block_scan(mine, total, scan_tot);
+    if (before < want && want <= before + mine) {
+      int a = before;
+      for (int q = 0; q < BPT; ++q) {
+        const int bin = SEL_BINS - 1 - tid * BPT - q;
+        const int c = (int)hist[bin];
+        if (want <= a + c) {
+          pick[0] = bin;
+          pick[1] = a;
+          break;
+        }
+        a += c;
+      }
+    }
+    __syncthreads();
+  };
+  const int need_total = rp.k - rp.nf;
+  rank_bin(need_total);
+  const int vbin = pick[0], above_bin = pick[1];
+  const int pop = (int)hist[vbin];
+  uint32_t klo, khi;
+  value_bin_key_range(vbin, klo, khi);
+  __syncthreads();
+  const bool prefix_bin = vbin != 0 && vbin != SEL_BINS / 2 - 1 && vbin != SEL_BINS / 2 && vbin != SEL_BINS - 1;
+  if (pop > SEL_CAND_CAP / 2 && prefix_bin) {
+    // A crowded bin (many nearly equal scores): histogram the next 12 key bits of the bin's keys (they share
+    // their upper 15 bits) and take the sub-bin of the k-th score, so that the candidate list stays short.
+    for (int i = tid; i < SEL_BINS; i += TS_THREADS) hist[i] = 0;
+    __syncthreads();
+#pragma unroll 4
+    for (int j = tid; j < T; j += TS_THREADS) {
+      if (rp.forced(j)) continue;
+      const uint32_t kk = float_key(sig[j]);
+      if (kk >= klo && kk <= khi) atomicAdd(&hist[(kk >> 5) & 0xfffu], 1u);
+    }
+    __syncthreads();
+    rank_bin(need_total - above_bin);
+    klo = (klo & 0xfffe0000u) | ((uint32_t)pick[0] << 5);
+    khi = klo | 31u;
+  }
+  if (tid == 0) {
+    // window: 2^-16 of the largest score, far above the float32 accumulation error of a head_dim-long dot product
+    const float delta = mx * 1.52587890625e-05f;
+    ctl[RC_DELTA] = __float_as_uint(delta);
+    ctl[RC_LO] = __float_as_uint(key_to_float(klo) - delta);
+    ctl[RC_EDGE] = __float_as_uint(fminf(key_to_float(khi) + delta, TS_FLT_MAX));
+  }
+}
+
+__global__ void __launch_bounds__(TS_THREADS) token_scan_kernel(const SelectDev p) {
+  __shared__ SelectSmem sm;
+  __shared__ double qsum[128];
+  __shared__ int s_seg, s_off, s_flag;
+
+  const int kvh = blockIdx.y, b = blockIdx.z;
   const int Hkv = p.sh.n_kv_heads, hd = p.sh.head_dim, G = p.sh.n_q_heads / Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int WARPS = TS_THREADS / 32;
   const int bk = b * Hkv + kvh;
   pdl_trigger();
-  // the lengths are an input of the step, not the work of an earlier kernel
-  const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
-  if (seg * TS_SEG >= max(T, 1)) return;
+  const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, b);
+  const int T = rp.T;
+  if ((int)blockIdx.x * TS_SEG >= max(T, 1)) return;
   pdl_wait();
   const size_t row = (size_t)bk * p.Tmax;
   float* sig = p.sigma + row;
   uint32_t* ctl = p.row_ctl + (size_t)bk * RC_WORDS;
-  uint32_t* gh = p.row_hist + (size_t)bk * SEL_BINS;
-  int32_t* soff = p.seg_off + (size_t)bk * p.nseg_max;
+  uint32_t* pub = p.seg_pub + (size_t)bk * p.nseg_max;
+  int32_t* lidx = p.list_idx + row;
+  uint32_t* lrow = p.list_row + row;
+  const int32_t* table = p.kv.page_table + (size_t)b * p.kv.max_pages_per_seq;
   const int nseg = max(1, (T + TS_SEG - 1) / TS_SEG);
+  // The segment this CTA works on is the ticket it draws: a CTA only ever waits for CTAs with a smaller
+  // ticket, which are therefore already running.
+  if (tid == 0) s_seg = nseg > 1 ? (int)atomicAdd(ctl + RC_TICKET, 1u) : 0;
+  __syncthreads();
+  const int seg = s_seg;
+  const int mode = rp.mode;
+  const float edge = mode == 2 ? __uint_as_float(ctl[RC_EDGE]) : TS_FLT_MAX;
+  const float lo = mode == 2 ? __uint_as_float(ctl[RC_LO]) : TS_FLT_MAX;
 
-  const int n_sink = min(max(p.sh.n_sink, 0), max(T, 0));
-  const int n_win = min(max(p.sh.n_window, 0), max(T, 0) - n_sink);
-  const int nf = n_sink + n_win;
-  long long bud = ((long long)p.r_permille[b] * T + 999) / 1000;
-  if (bud > T) bud = T;
-  const int k = T > 0 ? min(T, max((int)bud, nf)) : 0;
-  auto forced = [&](int j) { return j < n_sink || j >= T - n_win; };
-  // mode 0: keep all; 1: forced only; 2: selection; 3 (phase 2 only): float32 order with index-ordered ties
-  int mode = k >= T ? 0 : (k <= nf ? 1 : 2);
-
-  // ------------------------------------------------------------- phase 1 ----
-  float mx = 0.f;
-  if (mode == 2) {
-    for (int i = tid; i < SEL_BINS; i += TS_THREADS) sm.hist[i] = 0;
-    __syncthreads();
-    const int j0 = seg * TS_SEG + tid * 8;
-    if (j0 < T) {
-      const float4 v0 = *reinterpret_cast<const float4*>(sig + j0), v1 = *reinterpret_cast<const float4*>(sig + j0 + 4);
-      const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+  // ---- classify this CTA's 2048 tokens: 8 consecutive ones per thread ----
+  const int j0 = seg * TS_SEG + tid * 8;
+  uint32_t keep = 0;
+  if (j0 < T) {
+    if (mode == 0) {
+      keep = T - j0 >= 8 ? 0xffu : ((1u << (T - j0)) - 1u);
+    } else {
+      float vv[8];
+      if (mode == 2) {
+        const float4 v0 = *reinterpret_cast<const float4*>(sig + j0), v1 = *reinterpret_cast<const float4*>(sig + j0 + 4);
+        vv[0] = v0.x; vv[1] = v0.y; vv[2] = v0.z; vv[3] = v0.w; vv[4] = v1.x; vv[5] = v1.y; vv[6] = v1.z; vv[7] = v1.w;
+      }
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int j = j0 + e;
-        if (j < T && !forced(j)) {
-          const float sv = vv[e] + 0.0f;
-          atomicAdd(&sm.hist[key_value_bin(float_key(sv))], 1u);
-          mx = fmaxf(mx, fabsf(sv));
+        if (j >= T) continue;
+        if (rp.forced(j)) {
+          keep |= 1u << e;
+        } else if (mode == 2) {
+          if (vv[e] > edge) {
+            keep |= 1u << e;
+          } else if (vv[e] >= lo) {
+            const uint32_t slot = atomicAdd(ctl + RC_NCAND, 1u);
+            if (slot < (uint32_t)SEL_CAND_CAP) {
+              p.cand_idx[(size_t)bk * SEL_CAND_CAP + slot] = j;
+              p.cand_val[(size_t)bk * SEL_CAND_CAP + slot] = vv[e];
+            }
+          }
         }
       }
     }
-    mx = block_max<TS_THREADS>(mx, 0, sm);
-    __syncthreads();
+  }
+  int total;
+  const int before = ts_block_scan(__popc(keep), total, sm.scan[0]);
+
+  // ---- this segment's place in the row's list: the kept counts of the segments before it ----
+  if (tid == 0) {
+    int off = 0;
     if (nseg > 1) {
-      for (int i = tid; i < SEL_BINS; i += TS_THREADS) {
-        const uint32_t c = sm.hist[i];
-        if (c) atomicAdd(gh + i, c);
+      __threadfence();
+      atomicExch(pub + seg, (uint32_t)total | TS_READY);
+      for (int q = 0; q < seg; ++q) {
+        uint32_t v = 0;
+        uint32_t tries = 0;
+        while (((v = atomicAdd(pub + q, 0u)) & TS_READY) == 0u) {
+          if (++tries > WAIT_LIMIT) {  // never seen; reported, the row's list is then incomplete
+            atomicOr(p.status + ST_ERR, ERR_TIMEOUT);
+            break;
+          }
+        }
+        off += (int)(v & ~TS_READY);
       }
-      if (tid == 0) atomicMax(ctl + RC_MAX, __float_as_uint(mx));
+    }
+    s_off = off;
+  }
+  // staged in shared memory so that the list is written with full-width stores
+  int32_t* st_idx = reinterpret_cast<int32_t*>(sm.hist);
+  uint32_t* st_row = sm.hist + TS_SEG;
+  if (keep) {
+    // eight consecutive tokens share a page
+    const int page = table[j0 / PAGE];
+    const bool ok = page >= 0 && page < p.kv.num_pages;
+    if (!ok) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+    const uint32_t r0 = (uint32_t)((page * Hkv + kvh) * PAGE + (j0 % PAGE));
+    int pos = before;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      if ((keep >> e) & 1u) {
+        st_idx[pos] = j0 + e;
+        st_row[pos] = ok ? r0 + e : 0xffffffffu;
+        ++pos;
+      }
     }
   }
-  if (nseg > 1) {  // only the CTA that arrives last goes on
+  __syncthreads();
+  const int off = s_off;
+  for (int i = tid; i < total; i += TS_THREADS) {
+    lidx[off + i] = st_idx[i];
+    lrow[off + i] = st_row[i];
+  }
+
+  // ---- the CTA that finishes last settles the candidates ----
+  if (nseg > 1) {
     __threadfence();
     __syncthreads();
-    if (tid == 0) s_flag = atomicAdd(ctl + RC_DONE, 1u) == (uint32_t)(nseg - 1) ? 1 : 0;
+    if (tid == 0) s_flag = atomicAdd(ctl + RC_DONE2, 1u) == (uint32_t)(nseg - 1) ? 1 : 0;
     __syncthreads();
     if (!s_flag) return;
     __threadfence();
   }
-
-  // ------------------------------------------------------------- phase 2 ----
-  if (tid < TS_MAX_SEGS) seg_cnt[tid] = 0;
+  int n_list = 0;  // kept so far: what the segments wrote
+  if (nseg > 1) {
+    for (int q = 0; q < nseg; ++q) n_list += (int)(__ldcg(pub + q) & ~TS_READY);
+  } else {
+    n_list = total;
+  }
   if (tid < 4) sm.counts[tid] = 0;
-  float edge = TS_FLT_MAX;  // kept <=> score > edge (after the patches below)
+  __syncthreads();
   if (mode == 2) {
-    if (nseg > 1) {
-      for (int i = tid; i < SEL_BINS; i += TS_THREADS) sm.hist[i] = __ldcg(gh + i);
-      mx = __uint_as_float(__ldcg(ctl + RC_MAX));
-    }
-    __syncthreads();
-    const int need_total = k - nf;
-    // the bin that holds the `want`-th largest of the histogrammed scores, and how many lie above it:
-    // thread t owns bins 4095 - 16 t .. 4080 - 16 t
-    auto rank_bin = [&](int want) {
-      constexpr int BPT = SEL_BINS / TS_THREADS;
-      int mine = 0;
-#pragma unroll
-      for (int q = 0; q < BPT; ++q) mine += (int)sm.hist[SEL_BINS - 1 - tid * BPT - q];
-      int total;
-      const int before = ts_block_scan(mine, total, sm.scan[0]);
-      if (before < want && want <= before + mine) {
-        int a = before;
-        for (int q = 0; q < BPT; ++q) {
-          const int bin = SEL_BINS - 1 - tid * BPT - q;
-          const int c = (int)sm.hist[bin];
-          if (want <= a + c) {
-            sm.pick[0] = bin;
-            sm.pick[2] = a;
-            break;
-          }
-          a += c;
-        }
-      }
-      __syncthreads();
-    };
-    rank_bin(need_total);
-    const int vbin = sm.pick[0], above_bin = sm.pick[2];
-    uint32_t klo, khi;
-    value_bin_key_range(vbin, klo, khi);
-    // 2^-16 of the largest score: far above the float32 accumulation error of a head_dim-long dot product
-    const float delta = mx * 1.52587890625e-05f;
-    float lo = key_to_float(klo) - delta;
-    edge = fminf(key_to_float(khi) + delta, TS_FLT_MAX);
-
-    // one pass over the row: count what is above the edge per segment, list what lies between lo and the edge
-    auto run_pass = [&]() -> int {
-      int n_above_edge = 0;
+    const int ns_all = (int)__ldcg(ctl + RC_NCAND);
+    const int need_s = rp.k - n_list;
+    const float delta = __uint_as_float(ctl[RC_DELTA]);
+    if (ns_all > SEL_CAND_CAP || need_s < 0 || need_s > ns_all) {
+      // More scores between the edges than the list holds (long runs of equal scores): float32 order with
+      // ties to the lower index, by a radix select over the row's keys that lie between the edges.
+      if (tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
+      auto between = [&](int j, float& v) {
+        if (j >= T || rp.forced(j)) return false;
+        v = sig[j];
+        return v <= edge && v >= lo;
+      };
+      const int per = (T + TS_THREADS - 1) / TS_THREADS;
+      auto key = [&](int i) -> uint32_t {
+        float v;
+        return between(i * TS_THREADS + tid, v) ? float_key(v) : 0u;
+      };
+      int tie_need = 0;
+      const int want = min(max(need_s, 1), max(ns_all, 1));
+      const uint32_t key_thr = select_kth<TS_THREADS, 0, true>(key, want, tie_need, sm, per);
+      int ties_taken = 0, at = n_list;
 #pragma unroll 1
-      for (int wbase = warp * 256; wbase < T; wbase += TS_THREADS * 8) {  // a warp's 256 tokens lie in one segment
-        const int base = wbase + lane * 8;
-        int c8 = 0;
-        if (base < T) {
-          const float4 v0 = *reinterpret_cast<const float4*>(sig + base), v1 = *reinterpret_cast<const float4*>(sig + base + 4);
-          const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+      for (int base0 = 0; base0 < T && need_s > 0; base0 += TS_SEG) {  // in index order: ties are kept until tie_need runs out
+        const int q0 = base0 + tid * 8;
+        uint32_t above_mask = 0, tie_mask = 0;
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const int j = base + e;
-            if (j < T && !forced(j)) {
-              if (vv[e] > edge) {
-                ++c8;
-              } else if (vv[e] >= lo) {
-                const int slot = atomicAdd(&sm.counts[0], 1);
-                if (slot < SEL_CAND_CAP) {
-                  sm.cand_idx[slot] = j;
-                  sup_val[slot] = vv[e];
-                }
-              }
-            }
+        for (int e = 0; e < 8; ++e) {
+          float v;
+          if (between(q0 + e, v)) {
+            const uint32_t kk = float_key(v);
+            if (kk > key_thr) above_mask |= 1u << e;
+            if (kk == key_thr) tie_mask |= 1u << e;
           }
         }
-        n_above_edge += c8;
-        c8 = __reduce_add_sync(0xffffffffu, c8);
-        if (c8 && lane == 0) atomicAdd(&seg_cnt[wbase / TS_SEG], c8);
+        int tot_ties;
+        const int t_before = ties_taken + ts_block_scan(__popc(tie_mask), tot_ties, sm.scan[0]);
+        uint32_t take = above_mask;
+        int taken = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (((tie_mask >> e) & 1u) && t_before + taken < tie_need) {
+            take |= 1u << e;
+            ++taken;
+          }
+        }
+        int tot_take;
+        int pos = at + ts_block_scan(__popc(take), tot_take, sm.scan[1]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if ((take >> e) & 1u) {
+            const int j = q0 + e;
+            const int page = table[j / PAGE];
+            const bool ok = page >= 0 && page < p.kv.num_pages;
+            if (!ok) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+            lidx[pos] = j;
+            lrow[pos] = ok ? (uint32_t)((page * Hkv + kvh) * PAGE + (j % PAGE)) : 0xffffffffu;
+            sig[j] = INFINITY;
+            ++pos;
+          }
+        }
+        at += tot_take;
+        ties_taken += tot_ties;
       }
-      n_above_edge = block_count<TS_THREADS>(n_above_edge, 0, sm);
-      __syncthreads();
-      return n_above_edge;
-    };
-    int n_hi = run_pass();
-    const bool prefix_bin = vbin != 0 && vbin != SEL_BINS / 2 - 1 && vbin != SEL_BINS / 2 && vbin != SEL_BINS - 1;
-    if (sm.counts[0] > SEL_CAND_CAP && prefix_bin) {
-      // The bin and its window hold more scores than the list: histogram the next 12 key bits of the bin's
-      // keys (they share their upper 15 bits), take the sub-bin of the k-th score and list again.
-      for (int i = tid; i < SEL_BINS; i += TS_THREADS) sm.hist[i] = 0;
-      if (tid < TS_MAX_SEGS) seg_cnt[tid] = 0;
-      if (tid == 0) sm.counts[0] = 0;
-      __syncthreads();
-#pragma unroll 1
-      for (int j = tid; j < T; j += TS_THREADS) {
-        if (forced(j)) continue;
-        const uint32_t kk = float_key(sig[j] + 0.0f);
-        if (kk >= klo && kk <= khi) atomicAdd(&sm.hist[(kk >> 5) & 0xfffu], 1u);
+      n_list = at;
+    } else if (need_s > 0) {
+      const int ns = ns_all;
+      float* sup_val = sm.f32;
+      for (int c = tid; c < ns; c += TS_THREADS) {
+        sm.cand_idx[c] = __ldcg(p.cand_idx + (size_t)bk * SEL_CAND_CAP + c);
+        sup_val[c] = __ldcg(p.cand_val + (size_t)bk * SEL_CAND_CAP + c);
       }
       __syncthreads();
-      rank_bin(need_total - above_bin);
-      const uint32_t klo2 = (klo & 0xfffe0000u) | ((uint32_t)sm.pick[0] << 5), khi2 = klo2 | 31u;
-      lo = key_to_float(klo2) - delta;
-      edge = fminf(key_to_float(khi2) + delta, TS_FLT_MAX);
-      n_hi = run_pass();
-    }
-    const int ns = sm.counts[0];
-    const int need_s = need_total - n_hi;
-    if (ns > SEL_CAND_CAP || need_s < 1 || need_s > ns) {
-      mode = 3;
-    } else {
       // float32 rank inside the list: the element of rank need_s - 1 carries the k-th value
       for (int c = tid; c < ns; c += TS_THREADS) {
         const float v = sup_val[c];
@@ -610,7 +795,7 @@ __global__ void __launch_bounds__(TS_THREADS) token_select_kernel(const SelectDe
         for (int c = warp; c < ns; c += WARPS) {
           if (sm.cand_keep[c] != 2) continue;  // warp-uniform
           const int j = sm.cand_idx[c];
-          const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + j / PAGE];
+          const int page = table[j / PAGE];
           double a = 0.0;
           if (page >= 0 && page < p.kv.num_pages) {
             const uint16_t* kr = kp + (((size_t)page * Hkv + kvh) * PAGE + (j % PAGE)) * hd;
@@ -623,159 +808,83 @@ __global__ void __launch_bounds__(TS_THREADS) token_select_kernel(const SelectDe
       }
       rank_candidates<TS_THREADS>(ns, need_s, sm);  // cand_keep[c] = 1 for the need_s best of the list
       __syncthreads();
+      // the kept candidates join the row's list in ascending index order
       for (int c = tid; c < ns; c += TS_THREADS) {
-        if (sm.cand_keep[c]) {
-          const int j = sm.cand_idx[c];
-          sig[j] = INFINITY;
-          atomicAdd(&seg_cnt[j / TS_SEG], 1);
-        }
+        if (!sm.cand_keep[c]) continue;
+        const int j = sm.cand_idx[c];
+        int pos = 0;
+        for (int o = 0; o < ns; ++o) pos += sm.cand_keep[o] && sm.cand_idx[o] < j;
+        const int page = table[j / PAGE];
+        const bool ok = page >= 0 && page < p.kv.num_pages;
+        if (!ok) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+        lidx[n_list + pos] = j;
+        lrow[n_list + pos] = ok ? (uint32_t)((page * Hkv + kvh) * PAGE + (j % PAGE)) : 0xffffffffu;
+        sig[j] = INFINITY;
       }
+      n_list += need_s;
     }
   }
-
-  if (mode == 3) {
-    // More scores inside the list's range than it holds (long runs of equal or nearly equal scores): exact
-    // float32 order with ties to the lower index, by a radix select over the row's keys in global memory.
-    if (tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
-    __syncthreads();
-    if (tid < TS_MAX_SEGS) seg_cnt[tid] = 0;
-    const int per = (T + TS_THREADS - 1) / TS_THREADS;
-    auto key = [&](int i) -> uint32_t {
-      const int j = i * TS_THREADS + tid;
-      return (j < T && !forced(j)) ? float_key(sig[j] + 0.0f) : 0u;
-    };
-    int tie_need = 0;
-    const uint32_t key_thr = select_kth<TS_THREADS, 0, true>(key, k - nf, tie_need, sm, per);
-    edge = fminf(key_to_float(key_thr), TS_FLT_MAX);
-    int ties_taken = 0;
-#pragma unroll 1
-    for (int base0 = 0; base0 < T; base0 += TS_SEG) {  // in index order: ties are kept until tie_need runs out
-      const int j0 = base0 + tid * 8;
-      int above = 0, ties = 0;
-      uint32_t tie_mask = 0;
-      if (j0 < T) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int j = j0 + e;
-          if (j < T && !forced(j)) {
-            const uint32_t kk = float_key(sig[j] + 0.0f);
-            above += kk > key_thr;
-            if (kk == key_thr) {
-              ++ties;
-              tie_mask |= 1u << e;
-            }
-          }
-        }
-      }
-      int tot_ties;
-      const int t_before = ties_taken + ts_block_scan(ties, tot_ties, sm.scan[0]);
-      int taken = 0;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        if (((tie_mask >> e) & 1u) && t_before + taken < tie_need) {
-          sig[j0 + e] = INFINITY;
-          ++taken;
-        }
-      }
-      const int kept_here = block_count<TS_THREADS>(above + taken, 1, sm);
-      if (tid == 0) seg_cnt[base0 / TS_SEG] = kept_here;
-      ties_taken += tot_ties;
-    }
-    __syncthreads();
-  }
-
-  // forced tokens are kept whatever their score
+  // forced tokens read as kept for token_list whatever their score
   if (mode != 0) {
-    for (int f = tid; f < nf; f += TS_THREADS) {
-      const int j = f < n_sink ? f : T - n_win + (f - n_sink);
-      sig[j] = INFINITY;
-      atomicAdd(&seg_cnt[j / TS_SEG], 1);
-    }
+    for (int f = tid; f < rp.nf; f += TS_THREADS) sig[f < rp.n_sink ? f : T - rp.n_win + (f - rp.n_sink)] = INFINITY;
   }
-  __syncthreads();
-  if (tid == 0) {
-    int total = 0;
-    for (int s = 0; s < nseg; ++s) {
-      soff[s] = total;
-      total += mode == 0 ? min(TS_SEG, T - s * TS_SEG) : seg_cnt[s];
-    }
-    if (T <= 0) total = 0;
-    ctl[RC_MODE] = (uint32_t)mode;
-    ctl[RC_EDGE] = __float_as_uint(edge);
-    p.kept_cnt[bk] = total;
-    sm.counts[2] = total;
-  }
-  __syncthreads();
-  const int total = sm.counts[2];
+  const int total_kept = T > 0 ? n_list : 0;
+  if (tid == 0) p.kept_cnt[bk] = total_kept;
 
   // Pass-2 work items of this (sequence, kv-head): runs of `cpi` chunks of split_len kept tokens (at least
   // one item, so that the output is always written); cpi was chosen by the first CTA of the score pass.
   const int cpi = p.work_ctr[WC_CPI];
-  const int chunks = max(1, (total + p.split_len - 1) / p.split_len);
+  const int chunks = max(1, (total_kept + p.split_len - 1) / p.split_len);
   const int ns_items = (chunks + cpi - 1) / cpi;
+  __syncthreads();
   if (tid == 0) sm.counts[3] = atomicAdd(p.work_ctr + WC_ITEMS, ns_items);
   __syncthreads();
   const int item0 = sm.counts[3];
   for (int i = tid; i < ns_items; i += TS_THREADS) {
     p.work_items[2 * (item0 + i)] = bk * p.S + i * cpi;  // first chunk of the item
-    p.work_items[2 * (item0 + i) + 1] = total;
+    p.work_items[2 * (item0 + i) + 1] = total_kept;
   }
 }
 
-struct CompactDev {
+struct ListDev {
+  sol_shape_t sh;
   sol_kv_t kv;
-  int Hkv, Tmax, nseg_max;
+  const int32_t* r_permille;
+  int Tmax;
   const float* sigma;
   const uint32_t* row_ctl;
-  const int32_t* seg_off;
-  int32_t* kept_idx;   // [B*Hkv][Tmax] ascending
-  uint32_t* kept_row;  // same layout: cache row (page table applied), 0xffffffff: bad page
-  int* status;
+  int32_t* kept_idx;  // [B*Hkv][Tmax] ascending
 };
 
-__global__ void __launch_bounds__(TS_THREADS) token_compact_kernel(const CompactDev p) {
+// One CTA per (sequence, kv-head): the kept token indices in ascending order, for a caller that asks for them.
+__global__ void __launch_bounds__(TS_THREADS) token_list_kernel(const ListDev p) {
   __shared__ int warp_tot[TS_THREADS / 32];
-  const int seg = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
-  const int tid = threadIdx.x;
+  const int kvh = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
   pdl_trigger();
-  const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);
-  if (seg * TS_SEG >= T) return;
+  const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, b);
   pdl_wait();
-  const int bk = b * p.Hkv + kvh;
+  const int bk = b * p.sh.n_kv_heads + kvh;
   const size_t row = (size_t)bk * p.Tmax;
-  const uint32_t mode = p.row_ctl[(size_t)bk * RC_WORDS + RC_MODE];
-  const float edge = __uint_as_float(p.row_ctl[(size_t)bk * RC_WORDS + RC_EDGE]);
-  const int off = p.seg_off[(size_t)bk * p.nseg_max + seg];
-  const int j0 = seg * TS_SEG + tid * 8;
-  uint32_t keep = 0;
-  if (j0 < T) {
-    if (mode == 0) {
-      keep = T - j0 >= 8 ? 0xffu : ((1u << (T - j0)) - 1u);
-    } else {
+  const float edge = rp.mode == 2 ? __uint_as_float(p.row_ctl[(size_t)bk * RC_WORDS + RC_EDGE]) : TS_FLT_MAX;
+  int at = 0;
+#pragma unroll 1
+  for (int base0 = 0; base0 < rp.T; base0 += TS_SEG) {
+    const int j0 = base0 + tid * 8;
+    uint32_t keep = 0;
+    if (j0 < rp.T) {
       const float4 v0 = *reinterpret_cast<const float4*>(p.sigma + row + j0);
       const float4 v1 = *reinterpret_cast<const float4*>(p.sigma + row + j0 + 4);
       const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
 #pragma unroll
       for (int e = 0; e < 8; ++e)
-        if (j0 + e < T && vv[e] > edge) keep |= 1u << e;
+        if (j0 + e < rp.T && (rp.mode == 0 || vv[e] > edge)) keep |= 1u << e;
     }
-  }
-  int total;
-  int pos = off + ts_block_scan(__popc(keep), total, warp_tot);
-  if (keep) {
-    // eight consecutive tokens share a page
-    const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + j0 / PAGE];
-    const bool ok = page >= 0 && page < p.kv.num_pages;
-    if (!ok) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
-    const uint32_t r0 = (uint32_t)((page * p.Hkv + kvh) * PAGE + (j0 % PAGE));
+    int total;
+    int pos = at + ts_block_scan(__popc(keep), total, warp_tot);
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      if ((keep >> e) & 1u) {
-        p.kept_idx[row + pos] = j0 + e;
-        p.kept_row[row + pos] = ok ? r0 + e : 0xffffffffu;
-        ++pos;
-      }
-    }
+    for (int e = 0; e < 8; ++e)
+      if ((keep >> e) & 1u) p.kept_idx[row + pos++] = j0 + e;
+    at += total;
   }
 }
 
@@ -1099,7 +1208,8 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   pd.qkv_scale = a.qkv_scale;
   pd.q_bf16 = static_cast<const uint16_t*>(a.q_bf16);
   pd.q_rot = a.q_rot; pd.q_split = static_cast<uint16_t*>(a.q_split); pd.work_ctr = a.work_ctr; pd.status = a.status;
-  pd.row_hist = a.row_hist; pd.row_ctl = a.row_ctl;
+  pd.row_hist = a.row_hist; pd.row_ctl = a.row_ctl; pd.seg_pub = a.seg_pub;
+  pd.nseg_max = attn_select_segs(a.kv.max_pages_per_seq, PAGE);
   SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(Hkv, a.B), dim3(PREP_THREADS), 0, st, pd);
 
   ScoreDev sd;
@@ -1117,19 +1227,21 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.S = a.splits;
   se.split_len = attn_split_len(hd); se.q_rot = a.q_rot; se.B = a.B;
   se.nseg_max = attn_select_segs(a.kv.max_pages_per_seq, PAGE);
-  se.sigma = a.sigma; se.row_hist = a.row_hist; se.row_ctl = a.row_ctl; se.seg_off = a.seg_off;
+  se.sigma = a.sigma; se.row_hist = a.row_hist; se.row_ctl = a.row_ctl; se.seg_pub = a.seg_pub;
+  se.cand_idx = a.cand_idx; se.cand_val = a.cand_val; se.list_idx = a.list_idx; se.list_row = a.kept_row;
   se.kept_cnt = a.kept_cnt; se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
-  const dim3 seg_grid(se.nseg_max, Hkv, a.B);
-  SOL_LAUNCH("token_select", token_select_kernel, seg_grid, dim3(TS_THREADS), 0, st, se);
-
-  CompactDev cd;
-  cd.kv = a.kv; cd.Hkv = Hkv; cd.Tmax = Tmax; cd.nseg_max = se.nseg_max; cd.sigma = a.sigma; cd.row_ctl = a.row_ctl;
-  cd.seg_off = a.seg_off; cd.kept_idx = a.kept_idx; cd.kept_row = a.kept_row; cd.status = a.status;
-  SOL_LAUNCH("token_compact", token_compact_kernel, seg_grid, dim3(TS_THREADS), 0, st, cd);
+  SOL_LAUNCH("token_hist", token_hist_kernel, dim3((Tmax + TH_SEG - 1) / TH_SEG, Hkv, a.B), dim3(TS_THREADS), 0, st, se);
+  SOL_LAUNCH("token_scan", token_scan_kernel, dim3(se.nseg_max, Hkv, a.B), dim3(TS_THREADS), 0, st, se);
+  if (a.kept_idx_out != nullptr) {
+    ListDev ld;
+    ld.sh = sh; ld.kv = a.kv; ld.r_permille = a.r_permille; ld.Tmax = Tmax; ld.sigma = a.sigma; ld.row_ctl = a.row_ctl;
+    ld.kept_idx = a.kept_idx_out;
+    SOL_LAUNCH("token_list", token_list_kernel, dim3(Hkv, a.B), dim3(TS_THREADS), 0, st, ld);
+  }
 
   GatherDev gd;
   gd.kv = a.kv; gd.Hq = Hq; gd.Hkv = Hkv; gd.G = G; gd.Tmax = Tmax; gd.S = a.splits;
-  gd.logits = a.logits; gd.kept_idx = a.kept_idx; gd.kept_row = a.kept_row;
+  gd.logits = a.logits; gd.kept_idx = a.list_idx; gd.kept_row = a.kept_row;
   gd.work_items = a.work_items; gd.work_ctr = a.work_ctr; gd.part = a.part;
   gd.scale_log2 = (float)(1.4426950408889634 / sqrt((double)hd));
   gd.out_f32 = a.out_f32;

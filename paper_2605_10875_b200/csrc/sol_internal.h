@@ -142,9 +142,12 @@ struct AttnArgs {
   float* logits;        // [B][Hkv][Tmax][G]
   float* sigma;         // [B][Hkv][Tmax]
   uint32_t* row_hist;   // [B][Hkv][4096] histogram of a row's scores (rows that span several selection CTAs)
-  uint32_t* row_ctl;    // [B][Hkv][4] selection state of a row
-  int32_t* seg_off;     // [B][Hkv][segments] offsets of the 2048-token segments in the row's kept list
-  int32_t* kept_idx;    // [B][Hkv][Tmax] kept tokens, ascending (the caller's array when it asks for the list)
+  uint32_t* row_ctl;    // [B][Hkv][8] selection state of a row
+  uint32_t* seg_pub;    // [B][Hkv][segments] kept count of each 2048-token segment of the row (| ready bit)
+  int32_t* cand_idx;    // [B][Hkv][1024] tokens between the selection's edges
+  float* cand_val;      // [B][Hkv][1024] their scores
+  int32_t* list_idx;    // [B][Hkv][Tmax] token index of every kept token, in the order pass 2 reads them
+  int32_t* kept_idx_out; // optional: the caller's [B][Hkv][Tmax] array for the ascending index list
   int32_t* kept_cnt;    // [B][Hkv]
   uint32_t* kept_row;   // same layout as kept_idx: cache row (page table applied) of every kept token,
                         // 0xffffffff: bad page
@@ -163,7 +166,7 @@ struct AttnArgs {
 
 // Offsets of the attention scratch inside a buffer, starting at `at` (a multiple of 256).
 struct AttnScratch {
-  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_off, kept_idx, kept_cnt, kept_row, part, work_items, work_ctr, end;
+  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_pub, cand_idx, cand_val, kept_idx, kept_cnt, kept_row, part, work_items, work_ctr, end;
   int splits;
 };
 inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_pages, size_t at) {
@@ -181,8 +184,10 @@ inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_page
   L.logits = take(BK * Tmax * G * 4);
   L.sigma = take(BK * Tmax * 4);
   L.row_hist = take(BK * 4096 * 4);
-  L.row_ctl = take(BK * 4 * 4);
-  L.seg_off = take(BK * (size_t)attn_select_segs(max_pages, s.page_size) * 4);
+  L.row_ctl = take(BK * 8 * 4);
+  L.seg_pub = take(BK * (size_t)attn_select_segs(max_pages, s.page_size) * 4);
+  L.cand_idx = take(BK * 1024 * 4);
+  L.cand_val = take(BK * 1024 * 4);
   L.kept_idx = take(BK * Tmax * 4);
   L.kept_cnt = take(BK * 4);
   L.kept_row = take(BK * Tmax * 4);
@@ -201,8 +206,11 @@ inline void attn_scratch_bind(AttnArgs& a, void* base, const AttnScratch& L, int
   a.sigma = reinterpret_cast<float*>(b + L.sigma);
   a.row_hist = reinterpret_cast<uint32_t*>(b + L.row_hist);
   a.row_ctl = reinterpret_cast<uint32_t*>(b + L.row_ctl);
-  a.seg_off = reinterpret_cast<int32_t*>(b + L.seg_off);
-  a.kept_idx = kept_idx ? kept_idx : reinterpret_cast<int32_t*>(b + L.kept_idx);
+  a.seg_pub = reinterpret_cast<uint32_t*>(b + L.seg_pub);
+  a.cand_idx = reinterpret_cast<int32_t*>(b + L.cand_idx);
+  a.cand_val = reinterpret_cast<float*>(b + L.cand_val);
+  a.list_idx = reinterpret_cast<int32_t*>(b + L.kept_idx);
+  a.kept_idx_out = kept_idx;
   a.kept_cnt = kept_cnt ? kept_cnt : reinterpret_cast<int32_t*>(b + L.kept_cnt);
   a.kept_row = reinterpret_cast<uint32_t*>(b + L.kept_row);
   a.part = reinterpret_cast<float*>(b + L.part);

@@ -33,6 +33,7 @@ struct SelectSmem {
   int cand_idx[SEL_CAND_CAP];
   double cand_val[SEL_CAND_CAP];
   unsigned char cand_keep[SEL_CAND_CAP];
+  float f32[SEL_CAND_CAP];
   int counts[4];
 };
 
