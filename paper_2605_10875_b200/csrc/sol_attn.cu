@@ -28,6 +28,44 @@ namespace sol {
 
 constexpr int PAGE = 64;
 
+// Flat work lists of the attention kernels (AttnArgs::plan): cumulative counts over the sequences of the
+// batch, PLAN_STRIDE words each: 64-token pages (score pass), 8192-token segments of rows that need a
+// selection (histogram), 2048-token segments (scan).  Entry b is the count before sequence b, entry B the total.
+enum : int { PLAN_PAGES = 0, PLAN_HSEG = 1, PLAN_SSEG = 2, PLAN_LISTS = 3 };
+constexpr int PLAN_STRIDE = 132;
+constexpr int TH_SEG = 8192;  // tokens per token_hist CTA
+constexpr int TS_SEG = 2048;  // tokens per token_scan CTA
+
+// What every selection kernel derives from a row's length and keep-rate.
+struct RowPlan {
+  int T, n_sink, n_win, nf, k, mode;  // mode 0: keep all; 1: forced only; 2: selection
+  __device__ __forceinline__ bool forced(int j) const { return j < n_sink || j >= T - n_win; }
+};
+__device__ __forceinline__ RowPlan row_plan(const sol_shape_t& sh, const sol_kv_t& kv, const int32_t* r_permille, int b) {
+  RowPlan r;
+  r.T = min(kv.seq_lens[b], kv.max_pages_per_seq * PAGE);  // never index past the page table
+  const int Tp = max(r.T, 0);
+  r.n_sink = min(max(sh.n_sink, 0), Tp);
+  r.n_win = min(max(sh.n_window, 0), Tp - r.n_sink);
+  r.nf = r.n_sink + r.n_win;
+  long long bud = ((long long)r_permille[b] * Tp + 999) / 1000;
+  if (bud > Tp) bud = Tp;
+  r.k = min(Tp, max((int)bud, r.nf));
+  r.mode = r.k >= Tp ? 0 : (r.k <= r.nf ? 1 : 2);
+  return r;
+}
+
+// The sequence that holds flat unit `u` of a cumulative list (cum[b] <= u < cum[b + 1]); n entries + total.
+__device__ __forceinline__ int plan_find(const int* cum, int n, int u) {
+  int lo = 0, hi = n - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (cum[mid] <= u) lo = mid;
+    else hi = mid - 1;
+  }
+  return lo;
+}
+
 // ============================================================================
 // attn_prep
 // ============================================================================
@@ -45,6 +83,9 @@ struct PrepDev {
   uint32_t* row_ctl;  // zeroed here: [B*Hkv][RC_WORDS]
   uint32_t* seg_pub;  // zeroed here: [B*Hkv][nseg_max]
   int nseg_max;
+  int32_t* plan;      // written here by the first CTA: [PLAN_LISTS][PLAN_STRIDE]
+  const int32_t* r_permille;
+  int split_len, target_items;  // for the choice of the pass-2 item length
   int* status;
 };
 
@@ -68,6 +109,59 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
   const bool rope = layer && p.sh.rope_theta > 0.f;
   pdl_trigger();
   pdl_wait();
+
+  // The first CTA lays out the work of the kernels that follow: cumulative page and segment counts over the
+  // batch, and the length of the pass-2 work items in chunks of split_len kept tokens: the smallest run
+  // length (up to ATTN_ITEM_CHUNKS) that gives every resident CTA of pass 2 at most one item, so that there
+  // is no second, partly filled round of items; when even the longest runs leave more items than CTAs there
+  // is work for many rounds, and runs of 8 chunks, claimed one by one, balance it.
+  if (kvh == 0 && b == 0) {
+    __shared__ int wsum[PLAN_LISTS][PREP_THREADS / 32];
+    __shared__ int n_items[ATTN_ITEM_CHUNKS];
+    if (tid < ATTN_ITEM_CHUNKS) n_items[tid] = 0;
+    int cnt[PLAN_LISTS] = {0, 0, 0};
+    int ch = 0;
+    if (tid < p.B) {
+      const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, tid);
+      const int Tp = max(rp.T, 0);
+      cnt[PLAN_PAGES] = (Tp + PAGE - 1) / PAGE;
+      cnt[PLAN_HSEG] = rp.mode == 2 ? (Tp + TH_SEG - 1) / TH_SEG : 0;
+      cnt[PLAN_SSEG] = max(1, (Tp + TS_SEG - 1) / TS_SEG);
+      ch = max(1, (rp.k + p.split_len - 1) / p.split_len);
+    }
+    const int w = tid >> 5, l = tid & 31;
+    int incl[PLAN_LISTS];
+#pragma unroll
+    for (int q = 0; q < PLAN_LISTS; ++q) {
+      incl[q] = cnt[q];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int x = __shfl_up_sync(0xffffffffu, incl[q], o);
+        if (l >= o) incl[q] += x;
+      }
+      if (l == 31) wsum[q][w] = incl[q];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < PLAN_LISTS; ++q) {
+      int before = 0;
+      for (int x = 0; x < w; ++x) before += wsum[q][x];
+      if (tid < p.B) p.plan[q * PLAN_STRIDE + tid + 1] = before + incl[q];
+      if (tid == 0) p.plan[q * PLAN_STRIDE] = 0;
+    }
+#pragma unroll
+    for (int c = 1; c <= ATTN_ITEM_CHUNKS; ++c) {
+      const int n = __reduce_add_sync(0xffffffffu, tid < p.B ? (ch + c - 1) / c : 0);
+      if (l == 0) atomicAdd(&n_items[c - 1], n);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int cpi = 8;
+      for (int c = ATTN_ITEM_CHUNKS; c >= 1; --c)
+        if ((long long)n_items[c - 1] * Hkv <= p.target_items) cpi = c;
+      p.work_ctr[WC_CPI] = cpi;
+    }
+  }
 
   // this (sequence, kv-head)'s part of the q/k/v row: G query heads, the k head, the v head.  The K
   // slices of the projection are summed in order (four loads in flight at a time) and scaled.
@@ -183,149 +277,183 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
 // ============================================================================
 struct ScoreDev {
   sol_kv_t kv;
-  int Hkv, G, HG, Tmax;
+  int Hkv, G, HG, Tmax, B;
   const uint16_t* q_split;
+  const int32_t* plan;
   float* logits;
   float* sigma;
-  // for the choice of the pass-2 item length
-  int B, n_sink, n_window, split_len, target_items;
-  const int32_t* r_permille;
-  int32_t* work_ctr;
   int* status;
 };
 
-constexpr int SC_WARPS = 4;  // pages per CTA
+// Persistent warps over the flat list of (sequence, kv-head, page) units, in that order: every warp takes an
+// equal contiguous run of units, so it streams the pages of one row after the other and reloads the query
+// fragments only at row boundaries.  A warp owns two page buffers: while it multiplies one page, the bulk
+// copy of the next one is in flight (its page-table entry was fetched an iteration earlier).
+struct PageCursor {
+  int b, kvh, lp, np;  // sequence, kv-head, logical page, pages of the sequence
+};
+__device__ __forceinline__ void cursor_seek(PageCursor& c, const int* cum, int B, int Hkv, int unit) {
+  const int pg = unit;  // units of sequence b: cum[b] * Hkv .. cum[b + 1] * Hkv - 1
+  int lo = 0, hi = B - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (cum[mid] * Hkv <= pg) lo = mid;
+    else hi = mid - 1;
+  }
+  c.b = lo;
+  c.np = cum[lo + 1] - cum[lo];
+  const int rem = pg - cum[lo] * Hkv;
+  c.kvh = c.np > 0 ? rem / c.np : 0;
+  c.lp = c.np > 0 ? rem % c.np : 0;
+}
+__device__ __forceinline__ void cursor_next(PageCursor& c, const int* cum, int B, int Hkv) {
+  if (++c.lp < c.np) return;
+  c.lp = 0;
+  if (++c.kvh < Hkv) return;
+  c.kvh = 0;
+  do {
+    ++c.b;
+    c.np = c.b < B ? cum[c.b + 1] - cum[c.b] : 1;
+  } while (c.np == 0);
+}
 
-template <int HD, int HG>
-__global__ void __launch_bounds__(SC_WARPS * 32) attn_score_kernel(const ScoreDev p) {
+template <int HD, int HG, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32) attn_score_kernel(const ScoreDev p) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int PAGE_BYTES = PAGE * HD * 2;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SC_WARPS * PAGE_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + WARPS * 2 * PAGE_BYTES);
+  int* cum = reinterpret_cast<int*>(bars + WARPS * 2);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = blockIdx.z, kvh = blockIdx.y;
   pdl_trigger();
-  // The grid covers the longest row the page table allows; the CTAs beyond this sequence's length leave
-  // before anything else (the lengths are an input of the step, not the work of an earlier kernel).  The
-  // first CTA stays: it also sizes the pass-2 items.
-  if (blockIdx.x * SC_WARPS * PAGE >= p.kv.seq_lens[b] && (blockIdx.x | blockIdx.y | blockIdx.z) != 0) return;
   if (threadIdx.x == 0) {
-    for (int i = 0; i < SC_WARPS; ++i) mbar_init(&bars[i], 1);
+    for (int i = 0; i < WARPS * 2; ++i) mbar_init(&bars[i], 1);
     fence_mbar_init();
   }
-  __syncthreads();
   pdl_wait();
+  for (int i = threadIdx.x; i <= p.B; i += WARPS * 32) cum[i] = p.plan[PLAN_PAGES * PLAN_STRIDE + i];
+  __syncthreads();
+  const int Hkv = p.Hkv;
+  const int n_units = cum[p.B] * Hkv;
+  const int total_warps = gridDim.x * WARPS;
+  const int run = (n_units + total_warps - 1) / total_warps;
+  const int u0 = (blockIdx.x * WARPS + warp) * run, u1 = min(n_units, u0 + run);
+  if (u0 >= u1) return;
 
-  // Length of the pass-2 work items, in chunks of split_len kept tokens (the first CTA finds it for the batch,
-  // from the kept counts the budgets imply): the smallest run length (up to ATTN_ITEM_CHUNKS) that gives
-  // every resident CTA of pass 2 at most one item, so that there is no second, partly filled round of
-  // items; when even the longest runs leave more items than CTAs there is work for many rounds, and runs
-  // of 8 chunks, claimed one by one, balance it.
-  if (blockIdx.x == 0 && kvh == 0 && b == 0) {
-    __shared__ int n_items[ATTN_ITEM_CHUNKS];
-        if (threadIdx.x < ATTN_ITEM_CHUNKS) n_items[threadIdx.x] = 0;
-    __syncthreads();
-    for (int i0 = warp * 32; i0 < p.B; i0 += SC_WARPS * 32) {  // one sequence per lane
-      const int i = i0 + lane;
-      int ch = 0;
-      if (i < p.B) {
-        const int Ti = min(p.kv.seq_lens[i], p.kv.max_pages_per_seq * PAGE);
-        ch = 1;
-        if (Ti > 0) {
-          const int ns_ = min(max(p.n_sink, 0), Ti), nw_ = min(max(p.n_window, 0), Ti - ns_);
-          long long bd = ((long long)p.r_permille[i] * Ti + 999) / 1000;
-          if (bd > Ti) bd = Ti;
-          ch = max(1, (min(Ti, max((int)bd, ns_ + nw_)) + p.split_len - 1) / p.split_len);
-        }
-      }
-#pragma unroll
-      for (int c = 1; c <= ATTN_ITEM_CHUNKS; ++c) {
-        const int n = __reduce_add_sync(0xffffffffu, (ch + c - 1) / c);
-        if (lane == 0) atomicAdd(&n_items[c - 1], n);
+  unsigned char* tile0 = smem + warp * 2 * PAGE_BYTES;
+  uint64_t* bar0 = bars + warp * 2;
+  const uint16_t* kp = static_cast<const uint16_t*>(p.kv.k_pool);
+  // page id of a unit (warp-uniform load); -1: out of range
+  auto page_of = [&](const PageCursor& c) {
+    const int page = p.kv.page_table[(size_t)c.b * p.kv.max_pages_per_seq + c.lp];
+    return (page < 0 || page >= p.kv.num_pages) ? -1 : page;
+  };
+  // starts the copy of a unit's page into buffer `s`; a bad page id leaves the buffer alone (its scores are
+  // then computed from whatever it holds and the error is flagged)
+  auto issue = [&](const PageCursor& c, int page, int s) {
+    if (lane == 0) {
+      if (page >= 0) {
+        mbar_expect_tx(&bar0[s], PAGE_BYTES);
+        bulk_g2s(tile0 + s * PAGE_BYTES, kp + ((size_t)page * Hkv + c.kvh) * PAGE * HD, PAGE_BYTES, &bar0[s]);
+      } else {
+        atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+        mbar_arrive(&bar0[s]);
       }
     }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      int cpi = 8;
-      for (int c = ATTN_ITEM_CHUNKS; c >= 1; --c)
-        if ((long long)n_items[c - 1] * p.Hkv <= p.target_items) cpi = c;
-      p.work_ctr[WC_CPI] = cpi;
-    }
+  };
+
+  PageCursor cur, nxt;
+  cursor_seek(cur, cum, p.B, Hkv, u0);
+  nxt = cur;
+  issue(cur, page_of(cur), 0);
+  int page_nxt = -1;
+  if (u0 + 1 < u1) {
+    cursor_next(nxt, cum, p.B, Hkv);
+    page_nxt = page_of(nxt);
   }
 
-  const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
-  const int lp = blockIdx.x * SC_WARPS + warp;  // logical page
-  if (lp * PAGE >= T || lp >= p.kv.max_pages_per_seq) return;
-  const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + lp];
-  if (page < 0 || page >= p.kv.num_pages) {
-    if (lane == 0) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
-    return;
-  }
-  unsigned char* tile = smem + warp * PAGE_BYTES;
-  if (lane == 0) {
-    mbar_expect_tx(&bars[warp], PAGE_BYTES);
-    bulk_g2s(tile, static_cast<const uint16_t*>(p.kv.k_pool) + ((size_t)page * p.Hkv + kvh) * PAGE * HD, PAGE_BYTES,
-             &bars[warp]);
-  }
-
-  // query operand fragments: B[k][n] = q_split[n][k]; this lane holds rows g and 8+g, 8 k-values per pair step
   const int g = lane >> 2, t = lane & 3;
   constexpr int KS = HD / 32;  // pair steps (two MMAs of k=16 each)
   uint4 qf[HG][KS][2];
-#pragma unroll
-  for (int hg = 0; hg < HG; ++hg) {
-    const uint16_t* qb = p.q_split + ((size_t)((b * p.Hkv + kvh) * HG + hg) * 16) * HD;
-#pragma unroll
-    for (int s = 0; s < KS; ++s) {
-      qf[hg][s][0] = *reinterpret_cast<const uint4*>(qb + (size_t)g * HD + s * 32 + t * 8);
-      qf[hg][s][1] = *reinterpret_cast<const uint4*>(qb + (size_t)(8 + g) * HD + s * 32 + t * 8);
-    }
-  }
+  int q_b = -1, q_kvh = -1;
 
-  const bool ok = mbar_wait(&bars[warp], 0, p.status);
-  if (!ok) return;
-
-  const uint32_t tb = smem_u32(tile);
-  const size_t row0 = ((size_t)b * p.Hkv + kvh) * p.Tmax;
 #pragma unroll 1
-  for (int mt = 0; mt < PAGE / 16; ++mt) {
-    uint4 ka[KS][2];
-#pragma unroll
-    for (int s = 0; s < KS; ++s) {
-      ka[s][0] = lds128(tb + (mt * 16 + g) * (HD * 2) + (s * 32 + t * 8) * 2);
-      ka[s][1] = lds128(tb + (mt * 16 + g + 8) * (HD * 2) + (s * 32 + t * 8) * 2);
-    }
-    float sig0 = 0.f, sig1 = 0.f;  // tokens g and g+8 of this m-tile
-    const int tok0 = lp * PAGE + mt * 16 + g, tok1 = tok0 + 8;
-#pragma unroll
-    for (int hg = 0; hg < HG; ++hg) {
-      float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int s = 0; s < KS; ++s) {
-        mma_bf16(d0, ka[s][0].x, ka[s][1].x, ka[s][0].y, ka[s][1].y, qf[hg][s][0].x, qf[hg][s][0].y);
-        mma_bf16(d0, ka[s][0].z, ka[s][1].z, ka[s][0].w, ka[s][1].w, qf[hg][s][0].z, qf[hg][s][0].w);
-        mma_bf16(d1, ka[s][0].x, ka[s][1].x, ka[s][0].y, ka[s][1].y, qf[hg][s][1].x, qf[hg][s][1].y);
-        mma_bf16(d1, ka[s][0].z, ka[s][1].z, ka[s][0].w, ka[s][1].w, qf[hg][s][1].z, qf[hg][s][1].w);
+  for (int u = u0, n = 0; u < u1; ++u, ++n) {
+    const int s = n & 1;
+    // the next unit's copy goes into the other buffer, which every lane finished reading an iteration ago
+    PageCursor nn = nxt;
+    int page_nn = -1;
+    if (u + 1 < u1) {
+      issue(nxt, page_nxt, s ^ 1);
+      if (u + 2 < u1) {
+        cursor_next(nn, cum, p.B, Hkv);
+        page_nn = page_of(nn);
       }
-      // columns 2t, 2t+1 of the first n-tile are head t's hi and mid parts; column 2t of the second its lo part
-      const float s0 = d0[0] + (d0[1] + d1[0]);
-      const float s1 = d0[2] + (d0[3] + d1[2]);
-      const int head = hg * 4 + t;
-      if (head < p.G) {
-        if (tok0 < T) p.logits[(row0 + tok0) * p.G + head] = s0;
-        if (tok1 < T) p.logits[(row0 + tok1) * p.G + head] = s1;
+    }
+    // query operand fragments: B[k][n] = q_split[n][k]; this lane holds rows g and 8+g, 8 k-values per pair step
+    if (cur.b != q_b || cur.kvh != q_kvh) {
+      q_b = cur.b;
+      q_kvh = cur.kvh;
+#pragma unroll
+      for (int hg = 0; hg < HG; ++hg) {
+        const uint16_t* qb = p.q_split + ((size_t)((cur.b * Hkv + cur.kvh) * HG + hg) * 16) * HD;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+          qf[hg][ks][0] = *reinterpret_cast<const uint4*>(qb + (size_t)g * HD + ks * 32 + t * 8);
+          qf[hg][ks][1] = *reinterpret_cast<const uint4*>(qb + (size_t)(8 + g) * HD + ks * 32 + t * 8);
+        }
       }
-      float q0 = s0, q1 = s1;  // rows of absent heads are zero, so they add nothing
-      q0 += __shfl_xor_sync(0xffffffffu, q0, 1);
-      q1 += __shfl_xor_sync(0xffffffffu, q1, 1);
-      q0 += __shfl_xor_sync(0xffffffffu, q0, 2);
-      q1 += __shfl_xor_sync(0xffffffffu, q1, 2);
-      sig0 += q0;
-      sig1 += q1;
     }
-    if (t == 0) {
-      if (tok0 < T) p.sigma[row0 + tok0] = sig0 + 0.0f;  // -0 becomes +0: the selection compares floats and keys
-      if (tok1 < T) p.sigma[row0 + tok1] = sig1 + 0.0f;
+    const int T = min(p.kv.seq_lens[cur.b], p.kv.max_pages_per_seq * PAGE);
+    if (!mbar_wait(&bar0[s], (n >> 1) & 1, p.status)) return;
+
+    const uint32_t tb = smem_u32(tile0 + s * PAGE_BYTES);
+    const size_t row0 = ((size_t)cur.b * Hkv + cur.kvh) * p.Tmax;
+#pragma unroll 1
+    for (int mt = 0; mt < PAGE / 16; ++mt) {
+      if (cur.lp * PAGE + mt * 16 >= T) break;
+      uint4 ka[KS][2];
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        ka[ks][0] = lds128(tb + (mt * 16 + g) * (HD * 2) + (ks * 32 + t * 8) * 2);
+        ka[ks][1] = lds128(tb + (mt * 16 + g + 8) * (HD * 2) + (ks * 32 + t * 8) * 2);
+      }
+      float sig0 = 0.f, sig1 = 0.f;  // tokens g and g+8 of this m-tile
+      const int tok0 = cur.lp * PAGE + mt * 16 + g, tok1 = tok0 + 8;
+#pragma unroll
+      for (int hg = 0; hg < HG; ++hg) {
+        float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+          mma_bf16(d0, ka[ks][0].x, ka[ks][1].x, ka[ks][0].y, ka[ks][1].y, qf[hg][ks][0].x, qf[hg][ks][0].y);
+          mma_bf16(d0, ka[ks][0].z, ka[ks][1].z, ka[ks][0].w, ka[ks][1].w, qf[hg][ks][0].z, qf[hg][ks][0].w);
+          mma_bf16(d1, ka[ks][0].x, ka[ks][1].x, ka[ks][0].y, ka[ks][1].y, qf[hg][ks][1].x, qf[hg][ks][1].y);
+          mma_bf16(d1, ka[ks][0].z, ka[ks][1].z, ka[ks][0].w, ka[ks][1].w, qf[hg][ks][1].z, qf[hg][ks][1].w);
+        }
+        // columns 2t, 2t+1 of the first n-tile are head t's hi and mid parts; column 2t of the second its lo part
+        const float s0 = d0[0] + (d0[1] + d1[0]);
+        const float s1 = d0[2] + (d0[3] + d1[2]);
+        const int head = hg * 4 + t;
+        if (head < p.G) {
+          if (tok0 < T) p.logits[(row0 + tok0) * p.G + head] = s0;
+          if (tok1 < T) p.logits[(row0 + tok1) * p.G + head] = s1;
+        }
+        float q0 = s0, q1 = s1;  // rows of absent heads are zero, so they add nothing
+        q0 += __shfl_xor_sync(0xffffffffu, q0, 1);
+        q1 += __shfl_xor_sync(0xffffffffu, q1, 1);
+        q0 += __shfl_xor_sync(0xffffffffu, q0, 2);
+        q1 += __shfl_xor_sync(0xffffffffu, q1, 2);
+        sig0 += q0;
+        sig1 += q1;
+      }
+      if (t == 0) {
+        if (tok0 < T) p.sigma[row0 + tok0] = sig0 + 0.0f;  // -0 becomes +0: the selection compares floats and keys
+        if (tok1 < T) p.sigma[row0 + tok1] = sig1 + 0.0f;
+      }
     }
+    __syncwarp();
+    cur = nxt;
+    nxt = nn;
+    page_nxt = page_nn;
   }
 }
 
@@ -351,8 +479,6 @@ __global__ void __launch_bounds__(SC_WARPS * 32) attn_score_kernel(const ScoreDe
 // The row's list (token index and page-resolved cache row of every kept token) is what pass 2 reads: segment
 // by segment ascending, the settled candidates last; the order is the same on every run.
 constexpr int TS_THREADS = 256;
-constexpr int TH_SEG = 8192;                                      // tokens per token_hist CTA
-constexpr int TS_SEG = 2048;                                      // tokens per token_scan CTA
 constexpr int TS_MAX_SEGS = MAX_PAGES_PER_SEQ * PAGE / TS_SEG;     // 24
 constexpr float TS_FLT_MAX = 3.402823466e+38f;
 constexpr uint32_t TS_READY = 0x80000000u;
@@ -362,6 +488,7 @@ struct SelectDev {
   sol_kv_t kv;
   const int32_t* r_permille;
   int Tmax, S, split_len, B, nseg_max;
+  const int32_t* plan;
   const float* q_rot;
   float* sigma;          // kept candidates and forced tokens are overwritten with +inf (for token_list)
   uint32_t* row_hist;    // [B*Hkv][SEL_BINS], zero on entry
@@ -400,40 +527,27 @@ __device__ __forceinline__ int ts_block_scan(int v, int& total, int* warp_tot) {
   return before;
 }
 
-// What every selection kernel derives from a row's length and keep-rate.
-struct RowPlan {
-  int T, n_sink, n_win, nf, k, mode;  // mode 0: keep all; 1: forced only; 2: selection
-  __device__ __forceinline__ bool forced(int j) const { return j < n_sink || j >= T - n_win; }
+struct HistSmem {
+  uint32_t hist[SEL_BINS];
+  int scan_tot[TS_THREADS / 32];
+  float fmax_w[TS_THREADS / 32];
+  int pick[2];
+  int s_flag;
+  int cum[PLAN_STRIDE];
 };
-__device__ __forceinline__ RowPlan row_plan(const sol_shape_t& sh, const sol_kv_t& kv, const int32_t* r_permille, int b) {
-  RowPlan r;
-  r.T = min(kv.seq_lens[b], kv.max_pages_per_seq * PAGE);  // never index past the page table
-  const int Tp = max(r.T, 0);
-  r.n_sink = min(max(sh.n_sink, 0), Tp);
-  r.n_win = min(max(sh.n_window, 0), Tp - r.n_sink);
-  r.nf = r.n_sink + r.n_win;
-  long long bud = ((long long)r_permille[b] * Tp + 999) / 1000;
-  if (bud > Tp) bud = Tp;
-  r.k = min(Tp, max((int)bud, r.nf));
-  r.mode = r.k >= Tp ? 0 : (r.k <= r.nf ? 1 : 2);
-  return r;
-}
 
-__global__ void __launch_bounds__(TS_THREADS) token_hist_kernel(const SelectDev p) {
-  __shared__ uint32_t hist[SEL_BINS];
-  __shared__ int scan_tot[TS_THREADS / 32];
-  __shared__ float fmax_w[TS_THREADS / 32];
-  __shared__ int pick[2];
-  __shared__ int s_flag;
-  const int seg = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+// One (sequence, kv-head, 8192-token segment) of token_hist.
+__device__ __forceinline__ void token_hist_item(const SelectDev& p, HistSmem& hs, int b, int kvh, int seg) {
+  uint32_t* hist = hs.hist;
+  int* scan_tot = hs.scan_tot;
+  float* fmax_w = hs.fmax_w;
+  int* pick = hs.pick;
+  int& s_flag = hs.s_flag;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  pdl_trigger();
-  // lengths and keep-rates are inputs of the step, not the work of an earlier kernel
   const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, b);
   const int T = rp.T;
   if (rp.mode != 2 || seg * TH_SEG >= T) return;
   for (int i = tid; i < SEL_BINS; i += TS_THREADS) hist[i] = 0;
-  pdl_wait();
   __syncthreads();
   const int bk = b * p.sh.n_kv_heads + kvh;
   const float* sig = p.sigma + (size_t)bk * p.Tmax;
@@ -545,21 +659,42 @@ __global__ void __launch_bounds__(TS_THREADS) token_hist_kernel(const SelectDev 
   }
 }
 
-__global__ void __launch_bounds__(TS_THREADS) token_scan_kernel(const SelectDev p) {
-  __shared__ SelectSmem sm;
-  __shared__ double qsum[128];
-  __shared__ int s_seg, s_off, s_flag;
+// Persistent CTAs over the flat list of (sequence, kv-head, segment) units of the rows that need a selection.
+__global__ void __launch_bounds__(TS_THREADS) token_hist_kernel(const SelectDev p) {
+  __shared__ HistSmem hs;
+  pdl_trigger();
+  pdl_wait();
+  for (int i = threadIdx.x; i <= p.B; i += TS_THREADS) hs.cum[i] = p.plan[PLAN_HSEG * PLAN_STRIDE + i];
+  __syncthreads();
+  const int Hkv = p.sh.n_kv_heads;
+  const int n_units = hs.cum[p.B] * Hkv;
+  for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const int b = plan_find(hs.cum, p.B, u / Hkv);
+    const int n = hs.cum[b + 1] - hs.cum[b], rem = u - hs.cum[b] * Hkv;
+    token_hist_item(p, hs, b, rem / n, rem % n);
+    __syncthreads();
+  }
+}
 
-  const int kvh = blockIdx.y, b = blockIdx.z;
+struct ScanSmem {
+  SelectSmem sm;
+  double qsum[128];
+  int s_off, s_flag;
+  int cum[PLAN_STRIDE];
+};
+
+// One (sequence, kv-head, 2048-token segment) of token_scan.
+__device__ __forceinline__ void token_scan_item(const SelectDev& p, ScanSmem& ss, int b, int kvh, int seg) {
+  SelectSmem& sm = ss.sm;
+  double* qsum = ss.qsum;
+  int& s_off = ss.s_off;
+  int& s_flag = ss.s_flag;
   const int Hkv = p.sh.n_kv_heads, hd = p.sh.head_dim, G = p.sh.n_q_heads / Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int WARPS = TS_THREADS / 32;
   const int bk = b * Hkv + kvh;
-  pdl_trigger();
   const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, b);
   const int T = rp.T;
-  if ((int)blockIdx.x * TS_SEG >= max(T, 1)) return;
-  pdl_wait();
   const size_t row = (size_t)bk * p.Tmax;
   float* sig = p.sigma + row;
   uint32_t* ctl = p.row_ctl + (size_t)bk * RC_WORDS;
@@ -568,11 +703,6 @@ __global__ void __launch_bounds__(TS_THREADS) token_scan_kernel(const SelectDev 
   uint32_t* lrow = p.list_row + row;
   const int32_t* table = p.kv.page_table + (size_t)b * p.kv.max_pages_per_seq;
   const int nseg = max(1, (T + TS_SEG - 1) / TS_SEG);
-  // The segment this CTA works on is the ticket it draws: a CTA only ever waits for CTAs with a smaller
-  // ticket, which are therefore already running.
-  if (tid == 0) s_seg = nseg > 1 ? (int)atomicAdd(ctl + RC_TICKET, 1u) : 0;
-  __syncthreads();
-  const int seg = s_seg;
   const int mode = rp.mode;
   const float edge = mode == 2 ? __uint_as_float(ctl[RC_EDGE]) : TS_FLT_MAX;
   const float lo = mode == 2 ? __uint_as_float(ctl[RC_LO]) : TS_FLT_MAX;
@@ -613,24 +743,29 @@ __global__ void __launch_bounds__(TS_THREADS) token_scan_kernel(const SelectDev 
   const int before = ts_block_scan(__popc(keep), total, sm.scan[0]);
 
   // ---- this segment's place in the row's list: the kept counts of the segments before it ----
-  if (tid == 0) {
+  // The first warp publishes this segment's count and adds up those of the earlier segments, one per lane.
+  // The units of a row are taken in ascending order by CTAs that are all resident, so an earlier segment
+  // is always being worked on or done.
+  if (warp == 0) {
     int off = 0;
-    if (nseg > 1) {
+    if (lane == 0) {
       __threadfence();
       atomicExch(pub + seg, (uint32_t)total | TS_READY);
-      for (int q = 0; q < seg; ++q) {
-        uint32_t v = 0;
-        uint32_t tries = 0;
-        while (((v = atomicAdd(pub + q, 0u)) & TS_READY) == 0u) {
+    }
+    if (nseg > 1) {
+      if (lane < seg) {
+        uint32_t v = 0, tries = 0;
+        while (((v = atomicAdd(pub + lane, 0u)) & TS_READY) == 0u) {
           if (++tries > WAIT_LIMIT) {  // never seen; reported, the row's list is then incomplete
             atomicOr(p.status + ST_ERR, ERR_TIMEOUT);
             break;
           }
         }
-        off += (int)(v & ~TS_READY);
+        off = (int)(v & ~TS_READY);
       }
+      off = __reduce_add_sync(0xffffffffu, off);
     }
-    s_off = off;
+    if (lane == 0) s_off = off;
   }
   // staged in shared memory so that the list is written with full-width stores
   int32_t* st_idx = reinterpret_cast<int32_t*>(sm.hist);
@@ -658,21 +793,35 @@ __global__ void __launch_bounds__(TS_THREADS) token_scan_kernel(const SelectDev 
     lrow[off + i] = st_row[i];
   }
 
-  // ---- the CTA that finishes last settles the candidates ----
-  if (nseg > 1) {
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_flag = atomicAdd(ctl + RC_DONE2, 1u) == (uint32_t)(nseg - 1) ? 1 : 0;
-    __syncthreads();
-    if (!s_flag) return;
-    __threadfence();
-  }
+}
+
+// One CTA per (sequence, kv-head), after token_scan: ranks the candidates between the edges in float32,
+// re-scores those within the window of the k-th value in float64 from the cache rows, appends the kept ones
+// (ascending) to the row's list, and emits the row's pass-2 work items.
+__global__ void __launch_bounds__(TS_THREADS) token_settle_kernel(const SelectDev p) {
+  __shared__ SelectSmem sm;
+  __shared__ double qsum[128];
+  const int kvh = blockIdx.x, b = blockIdx.y;
+  const int Hkv = p.sh.n_kv_heads, hd = p.sh.head_dim, G = p.sh.n_q_heads / Hkv;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr int WARPS = TS_THREADS / 32;
+  const int bk = b * Hkv + kvh;
+  pdl_trigger();
+  const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, b);
+  pdl_wait();
+  const int T = rp.T, mode = rp.mode;
+  const size_t row = (size_t)bk * p.Tmax;
+  float* sig = p.sigma + row;
+  uint32_t* ctl = p.row_ctl + (size_t)bk * RC_WORDS;
+  const uint32_t* pub = p.seg_pub + (size_t)bk * p.nseg_max;
+  int32_t* lidx = p.list_idx + row;
+  uint32_t* lrow = p.list_row + row;
+  const int32_t* table = p.kv.page_table + (size_t)b * p.kv.max_pages_per_seq;
+  const int nseg = max(1, (T + TS_SEG - 1) / TS_SEG);
+  const float edge = mode == 2 ? __uint_as_float(ctl[RC_EDGE]) : TS_FLT_MAX;
+  const float lo = mode == 2 ? __uint_as_float(ctl[RC_LO]) : TS_FLT_MAX;
   int n_list = 0;  // kept so far: what the segments wrote
-  if (nseg > 1) {
-    for (int q = 0; q < nseg; ++q) n_list += (int)(__ldcg(pub + q) & ~TS_READY);
-  } else {
-    n_list = total;
-  }
+  for (int q = 0; q < nseg; ++q) n_list += (int)(pub[q] & ~TS_READY);
   if (tid < 4) sm.counts[tid] = 0;
   __syncthreads();
   if (mode == 2) {
@@ -843,6 +992,24 @@ __global__ void __launch_bounds__(TS_THREADS) token_scan_kernel(const SelectDev 
   for (int i = tid; i < ns_items; i += TS_THREADS) {
     p.work_items[2 * (item0 + i)] = bk * p.S + i * cpi;  // first chunk of the item
     p.work_items[2 * (item0 + i) + 1] = total_kept;
+  }
+}
+
+// Persistent CTAs over the flat list of (sequence, kv-head, segment) units; a CTA takes its units in
+// ascending order, and all CTAs of the grid are resident at once (the launch sizes the grid so).
+__global__ void __launch_bounds__(TS_THREADS) token_scan_kernel(const SelectDev p) {
+  __shared__ ScanSmem ss;
+  pdl_trigger();
+  pdl_wait();
+  for (int i = threadIdx.x; i <= p.B; i += TS_THREADS) ss.cum[i] = p.plan[PLAN_SSEG * PLAN_STRIDE + i];
+  __syncthreads();
+  const int Hkv = p.sh.n_kv_heads;
+  const int n_units = ss.cum[p.B] * Hkv;
+  for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const int b = plan_find(ss.cum, p.B, u / Hkv);
+    const int n = ss.cum[b + 1] - ss.cum[b], rem = u - ss.cum[b] * Hkv;
+    token_scan_item(p, ss, b, rem / n, rem % n);
+    __syncthreads();
   }
 }
 
@@ -1171,16 +1338,25 @@ __global__ void __launch_bounds__(GA_THREADS, GMAX == 4 ? 4 : 2) attn_gather_ker
 // ============================================================================
 // host side
 // ============================================================================
-template <int HD>
-static void launch_score(const ScoreDev& d, int HG, dim3 grid, cudaStream_t st) {
-  const int smem = SC_WARPS * PAGE * HD * 2 + SC_WARPS * 8 + 32;
-  if (HG == 1) {
-    ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_score_kernel<HD, 1>), smem);
-    SOL_LAUNCH("attn_score", (attn_score_kernel<HD, 1>), grid, dim3(SC_WARPS * 32), smem, st, d);
-  } else {
-    ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_score_kernel<HD, 2>), smem);
-    SOL_LAUNCH("attn_score", (attn_score_kernel<HD, 2>), grid, dim3(SC_WARPS * 32), smem, st, d);
+// Persistent grid: as many CTAs as are resident at once (two page buffers per warp, about 200 KB per SM in flight).
+template <int HD, int HG, int WARPS>
+static void launch_score_t(const ScoreDev& d, cudaStream_t st) {
+  const int smem = WARPS * 2 * PAGE * HD * 2 + WARPS * 2 * 8 + (PLAN_STRIDE + 4) * 4;
+  static int per_sm = 0;
+  ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_score_kernel<HD, HG, WARPS>), smem);
+  if (per_sm == 0) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attn_score_kernel<HD, HG, WARPS>, WARPS * 32, smem) != cudaSuccess || n < 1)
+      n = 1;
+    per_sm = n;
   }
+  SOL_LAUNCH("attn_score", (attn_score_kernel<HD, HG, WARPS>), dim3(sm_count() * per_sm), dim3(WARPS * 32), smem, st, d);
+}
+template <int HD>
+static void launch_score(const ScoreDev& d, int HG, cudaStream_t st) {
+  constexpr int WARPS = HD == 64 ? 4 : 3;  // 64 / 96 KB of page buffers per CTA: three / two CTAs per SM
+  if (HG == 1) launch_score_t<HD, 1, WARPS>(d, st);
+  else launch_score_t<HD, 2, WARPS>(d, st);
 }
 
 // One CTA per item, at most as many CTAs as are resident at once (they are persistent).
@@ -1210,18 +1386,16 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   pd.q_rot = a.q_rot; pd.q_split = static_cast<uint16_t*>(a.q_split); pd.work_ctr = a.work_ctr; pd.status = a.status;
   pd.row_hist = a.row_hist; pd.row_ctl = a.row_ctl; pd.seg_pub = a.seg_pub;
   pd.nseg_max = attn_select_segs(a.kv.max_pages_per_seq, PAGE);
+  pd.plan = a.plan; pd.r_permille = a.r_permille; pd.split_len = attn_split_len(hd);
+  pd.target_items = sm_count() * (G <= 4 ? 4 : 2);  // the pass-2 CTAs resident at once
   SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(Hkv, a.B), dim3(PREP_THREADS), 0, st, pd);
 
   ScoreDev sd;
-  sd.kv = a.kv; sd.Hkv = Hkv; sd.G = G; sd.HG = HG; sd.Tmax = Tmax;
-  sd.q_split = static_cast<const uint16_t*>(a.q_split);
+  sd.kv = a.kv; sd.Hkv = Hkv; sd.G = G; sd.HG = HG; sd.Tmax = Tmax; sd.B = a.B;
+  sd.q_split = static_cast<const uint16_t*>(a.q_split); sd.plan = a.plan;
   sd.logits = a.logits; sd.sigma = a.sigma; sd.status = a.status;
-  sd.B = a.B; sd.n_sink = sh.n_sink; sd.n_window = sh.n_window; sd.split_len = attn_split_len(hd);
-  sd.target_items = sm_count() * (G <= 4 ? 4 : 2);  // the pass-2 CTAs resident at once
-  sd.r_permille = a.r_permille; sd.work_ctr = a.work_ctr;
-  dim3 sgrid((a.kv.max_pages_per_seq + SC_WARPS - 1) / SC_WARPS, Hkv, a.B);
-  if (hd == 64) launch_score<64>(sd, HG, sgrid, st);
-  else launch_score<128>(sd, HG, sgrid, st);
+  if (hd == 64) launch_score<64>(sd, HG, st);
+  else launch_score<128>(sd, HG, st);
 
   SelectDev se;
   se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.S = a.splits;
@@ -1230,8 +1404,27 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   se.sigma = a.sigma; se.row_hist = a.row_hist; se.row_ctl = a.row_ctl; se.seg_pub = a.seg_pub;
   se.cand_idx = a.cand_idx; se.cand_val = a.cand_val; se.list_idx = a.list_idx; se.list_row = a.kept_row;
   se.kept_cnt = a.kept_cnt; se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
-  SOL_LAUNCH("token_hist", token_hist_kernel, dim3((Tmax + TH_SEG - 1) / TH_SEG, Hkv, a.B), dim3(TS_THREADS), 0, st, se);
-  SOL_LAUNCH("token_scan", token_scan_kernel, dim3(se.nseg_max, Hkv, a.B), dim3(TS_THREADS), 0, st, se);
+  se.plan = a.plan;
+  {
+    // persistent grids: never more CTAs than are resident at once, never more than there can be units
+    static int hist_per_sm = 0, scan_per_sm = 0;
+    if (hist_per_sm == 0) {
+      int n = 0;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_hist_kernel, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
+      hist_per_sm = n;
+      n = 0;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_scan_kernel, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
+      scan_per_sm = n;
+    }
+    const long long hist_units = (long long)a.B * Hkv * ((Tmax + TH_SEG - 1) / TH_SEG);
+    const long long scan_units = (long long)a.B * Hkv * se.nseg_max;
+    const long long hist_res = (long long)sm_count() * hist_per_sm, scan_res = (long long)sm_count() * scan_per_sm;
+    SOL_LAUNCH("token_hist", token_hist_kernel, dim3((unsigned)(hist_units < hist_res ? hist_units : hist_res)),
+               dim3(TS_THREADS), 0, st, se);
+    SOL_LAUNCH("token_scan", token_scan_kernel, dim3((unsigned)(scan_units < scan_res ? scan_units : scan_res)),
+               dim3(TS_THREADS), 0, st, se);
+    SOL_LAUNCH("token_settle", token_settle_kernel, dim3(Hkv, a.B), dim3(TS_THREADS), 0, st, se);
+  }
   if (a.kept_idx_out != nullptr) {
     ListDev ld;
     ld.sh = sh; ld.kv = a.kv; ld.r_permille = a.r_permille; ld.Tmax = Tmax; ld.sigma = a.sigma; ld.row_ctl = a.row_ctl;

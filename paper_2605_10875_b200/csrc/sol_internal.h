@@ -153,6 +153,8 @@ struct AttnArgs {
                         // 0xffffffff: bad page
   float* part;          // [B][Hkv][S][G][hd + 2]
   int splits;           // S = ceil(Tmax / attn_split_len(hd))
+  int32_t* plan;        // [3][132] cumulative page / segment counts over the batch: the flat work lists of pass 1 and
+                        // of the selection, written by the query preparation
   int32_t* work_items;  // [B*Hkv*S][2] pass-2 work list (item code, kept count), filled by the selection
   int32_t* work_ctr;    // [4 + B*Hkv]: items emitted, next item to claim, chunks per item, unused; then the finished
                         // items of every (sequence, kv-head)
@@ -166,7 +168,7 @@ struct AttnArgs {
 
 // Offsets of the attention scratch inside a buffer, starting at `at` (a multiple of 256).
 struct AttnScratch {
-  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_pub, cand_idx, cand_val, kept_idx, kept_cnt, kept_row, part, work_items, work_ctr, end;
+  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_pub, cand_idx, cand_val, kept_idx, kept_cnt, kept_row, part, plan, work_items, work_ctr, end;
   int splits;
 };
 inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_pages, size_t at) {
@@ -192,6 +194,7 @@ inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_page
   L.kept_cnt = take(BK * 4);
   L.kept_row = take(BK * Tmax * 4);
   L.part = take(BK * L.splits * G * (hd + 2) * 4);
+  L.plan = take(3 * 132 * 4);
   L.work_items = take(BK * L.splits * 8);
   L.work_ctr = take((4 + BK) * 4);
   L.end = at;
@@ -214,6 +217,7 @@ inline void attn_scratch_bind(AttnArgs& a, void* base, const AttnScratch& L, int
   a.kept_cnt = kept_cnt ? kept_cnt : reinterpret_cast<int32_t*>(b + L.kept_cnt);
   a.kept_row = reinterpret_cast<uint32_t*>(b + L.kept_row);
   a.part = reinterpret_cast<float*>(b + L.part);
+  a.plan = reinterpret_cast<int32_t*>(b + L.plan);
   a.work_items = reinterpret_cast<int32_t*>(b + L.work_items);
   a.work_ctr = reinterpret_cast<int32_t*>(b + L.work_ctr);
   a.splits = L.splits;
