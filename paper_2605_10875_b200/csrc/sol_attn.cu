@@ -29,7 +29,7 @@ namespace sol {
 constexpr int PAGE = 64;
 
 // Flat work lists of the attention kernels (AttnArgs::plan): cumulative counts over the sequences of the
-// batch, PLAN_STRIDE words each: 64-token pages (score pass), 8192-token segments of rows that need a
+// batch, PLAN_STRIDE words each: 64-token pages, 8192-token segments of rows that need a
 // selection (histogram), 2048-token segments (scan).  Entry b is the count before sequence b, entry B the total.
 enum : int { PLAN_PAGES = 0, PLAN_HSEG = 1, PLAN_SSEG = 2, PLAN_LISTS = 3 };
 constexpr int PLAN_STRIDE = 132;
@@ -277,183 +277,107 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
 // ============================================================================
 struct ScoreDev {
   sol_kv_t kv;
-  int Hkv, G, HG, Tmax, B;
+  int Hkv, G, HG, Tmax;
   const uint16_t* q_split;
-  const int32_t* plan;
   float* logits;
   float* sigma;
   int* status;
 };
 
-// Persistent warps over the flat list of (sequence, kv-head, page) units, in that order: every warp takes an
-// equal contiguous run of units, so it streams the pages of one row after the other and reloads the query
-// fragments only at row boundaries.  A warp owns two page buffers: while it multiplies one page, the bulk
-// copy of the next one is in flight (its page-table entry was fetched an iteration earlier).
-struct PageCursor {
-  int b, kvh, lp, np;  // sequence, kv-head, logical page, pages of the sequence
-};
-__device__ __forceinline__ void cursor_seek(PageCursor& c, const int* cum, int B, int Hkv, int unit) {
-  const int pg = unit;  // units of sequence b: cum[b] * Hkv .. cum[b + 1] * Hkv - 1
-  int lo = 0, hi = B - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (cum[mid] * Hkv <= pg) lo = mid;
-    else hi = mid - 1;
-  }
-  c.b = lo;
-  c.np = cum[lo + 1] - cum[lo];
-  const int rem = pg - cum[lo] * Hkv;
-  c.kvh = c.np > 0 ? rem / c.np : 0;
-  c.lp = c.np > 0 ? rem % c.np : 0;
-}
-__device__ __forceinline__ void cursor_next(PageCursor& c, const int* cum, int B, int Hkv) {
-  if (++c.lp < c.np) return;
-  c.lp = 0;
-  if (++c.kvh < Hkv) return;
-  c.kvh = 0;
-  do {
-    ++c.b;
-    c.np = c.b < B ? cum[c.b + 1] - cum[c.b] : 1;
-  } while (c.np == 0);
-}
+constexpr int SC_WARPS = 4;  // pages per CTA
 
-template <int HD, int HG, int WARPS>
-__global__ void __launch_bounds__(WARPS * 32) attn_score_kernel(const ScoreDev p) {
+template <int HD, int HG>
+__global__ void __launch_bounds__(SC_WARPS * 32) attn_score_kernel(const ScoreDev p) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int PAGE_BYTES = PAGE * HD * 2;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + WARPS * 2 * PAGE_BYTES);
-  int* cum = reinterpret_cast<int*>(bars + WARPS * 2);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SC_WARPS * PAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.z, kvh = blockIdx.y;
   pdl_trigger();
+  // The grid covers the longest row the page table allows; the CTAs beyond this sequence's length leave
+  // before anything else (the lengths are an input of the step, not the work of an earlier kernel).
+  if (blockIdx.x * SC_WARPS * PAGE >= p.kv.seq_lens[b]) return;
   if (threadIdx.x == 0) {
-    for (int i = 0; i < WARPS * 2; ++i) mbar_init(&bars[i], 1);
+    for (int i = 0; i < SC_WARPS; ++i) mbar_init(&bars[i], 1);
     fence_mbar_init();
   }
-  pdl_wait();
-  for (int i = threadIdx.x; i <= p.B; i += WARPS * 32) cum[i] = p.plan[PLAN_PAGES * PLAN_STRIDE + i];
   __syncthreads();
-  const int Hkv = p.Hkv;
-  const int n_units = cum[p.B] * Hkv;
-  const int total_warps = gridDim.x * WARPS;
-  const int run = (n_units + total_warps - 1) / total_warps;
-  const int u0 = (blockIdx.x * WARPS + warp) * run, u1 = min(n_units, u0 + run);
-  if (u0 >= u1) return;
+  pdl_wait();
 
-  unsigned char* tile0 = smem + warp * 2 * PAGE_BYTES;
-  uint64_t* bar0 = bars + warp * 2;
-  const uint16_t* kp = static_cast<const uint16_t*>(p.kv.k_pool);
-  // page id of a unit (warp-uniform load); -1: out of range
-  auto page_of = [&](const PageCursor& c) {
-    const int page = p.kv.page_table[(size_t)c.b * p.kv.max_pages_per_seq + c.lp];
-    return (page < 0 || page >= p.kv.num_pages) ? -1 : page;
-  };
-  // starts the copy of a unit's page into buffer `s`; a bad page id leaves the buffer alone (its scores are
-  // then computed from whatever it holds and the error is flagged)
-  auto issue = [&](const PageCursor& c, int page, int s) {
-    if (lane == 0) {
-      if (page >= 0) {
-        mbar_expect_tx(&bar0[s], PAGE_BYTES);
-        bulk_g2s(tile0 + s * PAGE_BYTES, kp + ((size_t)page * Hkv + c.kvh) * PAGE * HD, PAGE_BYTES, &bar0[s]);
-      } else {
-        atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
-        mbar_arrive(&bar0[s]);
-      }
-    }
-  };
-
-  PageCursor cur, nxt;
-  cursor_seek(cur, cum, p.B, Hkv, u0);
-  nxt = cur;
-  issue(cur, page_of(cur), 0);
-  int page_nxt = -1;
-  if (u0 + 1 < u1) {
-    cursor_next(nxt, cum, p.B, Hkv);
-    page_nxt = page_of(nxt);
+  const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
+  const int lp = blockIdx.x * SC_WARPS + warp;  // logical page
+  if (lp * PAGE >= T || lp >= p.kv.max_pages_per_seq) return;
+  const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + lp];
+  if (page < 0 || page >= p.kv.num_pages) {
+    if (lane == 0) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+    return;
+  }
+  unsigned char* tile = smem + warp * PAGE_BYTES;
+  if (lane == 0) {
+    mbar_expect_tx(&bars[warp], PAGE_BYTES);
+    bulk_g2s(tile, static_cast<const uint16_t*>(p.kv.k_pool) + ((size_t)page * p.Hkv + kvh) * PAGE * HD, PAGE_BYTES,
+             &bars[warp]);
   }
 
+  // query operand fragments: B[k][n] = q_split[n][k]; this lane holds rows g and 8+g, 8 k-values per pair step
   const int g = lane >> 2, t = lane & 3;
   constexpr int KS = HD / 32;  // pair steps (two MMAs of k=16 each)
   uint4 qf[HG][KS][2];
-  int q_b = -1, q_kvh = -1;
+#pragma unroll
+  for (int hg = 0; hg < HG; ++hg) {
+    const uint16_t* qb = p.q_split + ((size_t)((b * p.Hkv + kvh) * HG + hg) * 16) * HD;
+#pragma unroll
+    for (int s = 0; s < KS; ++s) {
+      qf[hg][s][0] = *reinterpret_cast<const uint4*>(qb + (size_t)g * HD + s * 32 + t * 8);
+      qf[hg][s][1] = *reinterpret_cast<const uint4*>(qb + (size_t)(8 + g) * HD + s * 32 + t * 8);
+    }
+  }
 
-#pragma unroll 1
-  for (int u = u0, n = 0; u < u1; ++u, ++n) {
-    const int s = n & 1;
-    // the next unit's copy goes into the other buffer, which every lane finished reading an iteration ago
-    PageCursor nn = nxt;
-    int page_nn = -1;
-    if (u + 1 < u1) {
-      issue(nxt, page_nxt, s ^ 1);
-      if (u + 2 < u1) {
-        cursor_next(nn, cum, p.B, Hkv);
-        page_nn = page_of(nn);
-      }
-    }
-    // query operand fragments: B[k][n] = q_split[n][k]; this lane holds rows g and 8+g, 8 k-values per pair step
-    if (cur.b != q_b || cur.kvh != q_kvh) {
-      q_b = cur.b;
-      q_kvh = cur.kvh;
-#pragma unroll
-      for (int hg = 0; hg < HG; ++hg) {
-        const uint16_t* qb = p.q_split + ((size_t)((cur.b * Hkv + cur.kvh) * HG + hg) * 16) * HD;
-#pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-          qf[hg][ks][0] = *reinterpret_cast<const uint4*>(qb + (size_t)g * HD + ks * 32 + t * 8);
-          qf[hg][ks][1] = *reinterpret_cast<const uint4*>(qb + (size_t)(8 + g) * HD + ks * 32 + t * 8);
-        }
-      }
-    }
-    const int T = min(p.kv.seq_lens[cur.b], p.kv.max_pages_per_seq * PAGE);
-    if (!mbar_wait(&bar0[s], (n >> 1) & 1, p.status)) return;
+  const bool ok = mbar_wait(&bars[warp], 0, p.status);
+  if (!ok) return;
 
-    const uint32_t tb = smem_u32(tile0 + s * PAGE_BYTES);
-    const size_t row0 = ((size_t)cur.b * Hkv + cur.kvh) * p.Tmax;
+  const uint32_t tb = smem_u32(tile);
+  const size_t row0 = ((size_t)b * p.Hkv + kvh) * p.Tmax;
 #pragma unroll 1
-    for (int mt = 0; mt < PAGE / 16; ++mt) {
-      if (cur.lp * PAGE + mt * 16 >= T) break;
-      uint4 ka[KS][2];
+  for (int mt = 0; mt < PAGE / 16; ++mt) {
+    uint4 ka[KS][2];
 #pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-        ka[ks][0] = lds128(tb + (mt * 16 + g) * (HD * 2) + (ks * 32 + t * 8) * 2);
-        ka[ks][1] = lds128(tb + (mt * 16 + g + 8) * (HD * 2) + (ks * 32 + t * 8) * 2);
-      }
-      float sig0 = 0.f, sig1 = 0.f;  // tokens g and g+8 of this m-tile
-      const int tok0 = cur.lp * PAGE + mt * 16 + g, tok1 = tok0 + 8;
-#pragma unroll
-      for (int hg = 0; hg < HG; ++hg) {
-        float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-          mma_bf16(d0, ka[ks][0].x, ka[ks][1].x, ka[ks][0].y, ka[ks][1].y, qf[hg][ks][0].x, qf[hg][ks][0].y);
-          mma_bf16(d0, ka[ks][0].z, ka[ks][1].z, ka[ks][0].w, ka[ks][1].w, qf[hg][ks][0].z, qf[hg][ks][0].w);
-          mma_bf16(d1, ka[ks][0].x, ka[ks][1].x, ka[ks][0].y, ka[ks][1].y, qf[hg][ks][1].x, qf[hg][ks][1].y);
-          mma_bf16(d1, ka[ks][0].z, ka[ks][1].z, ka[ks][0].w, ka[ks][1].w, qf[hg][ks][1].z, qf[hg][ks][1].w);
-        }
-        // columns 2t, 2t+1 of the first n-tile are head t's hi and mid parts; column 2t of the second its lo part
-        const float s0 = d0[0] + (d0[1] + d1[0]);
-        const float s1 = d0[2] + (d0[3] + d1[2]);
-        const int head = hg * 4 + t;
-        if (head < p.G) {
-          if (tok0 < T) p.logits[(row0 + tok0) * p.G + head] = s0;
-          if (tok1 < T) p.logits[(row0 + tok1) * p.G + head] = s1;
-        }
-        float q0 = s0, q1 = s1;  // rows of absent heads are zero, so they add nothing
-        q0 += __shfl_xor_sync(0xffffffffu, q0, 1);
-        q1 += __shfl_xor_sync(0xffffffffu, q1, 1);
-        q0 += __shfl_xor_sync(0xffffffffu, q0, 2);
-        q1 += __shfl_xor_sync(0xffffffffu, q1, 2);
-        sig0 += q0;
-        sig1 += q1;
-      }
-      if (t == 0) {
-        if (tok0 < T) p.sigma[row0 + tok0] = sig0 + 0.0f;  // -0 becomes +0: the selection compares floats and keys
-        if (tok1 < T) p.sigma[row0 + tok1] = sig1 + 0.0f;
-      }
+    for (int s = 0; s < KS; ++s) {
+      ka[s][0] = lds128(tb + (mt * 16 + g) * (HD * 2) + (s * 32 + t * 8) * 2);
+      ka[s][1] = lds128(tb + (mt * 16 + g + 8) * (HD * 2) + (s * 32 + t * 8) * 2);
     }
-    __syncwarp();
-    cur = nxt;
-    nxt = nn;
-    page_nxt = page_nn;
+    float sig0 = 0.f, sig1 = 0.f;  // tokens g and g+8 of this m-tile
+    const int tok0 = lp * PAGE + mt * 16 + g, tok1 = tok0 + 8;
+#pragma unroll
+    for (int hg = 0; hg < HG; ++hg) {
+      float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int s = 0; s < KS; ++s) {
+        mma_bf16(d0, ka[s][0].x, ka[s][1].x, ka[s][0].y, ka[s][1].y, qf[hg][s][0].x, qf[hg][s][0].y);
+        mma_bf16(d0, ka[s][0].z, ka[s][1].z, ka[s][0].w, ka[s][1].w, qf[hg][s][0].z, qf[hg][s][0].w);
+        mma_bf16(d1, ka[s][0].x, ka[s][1].x, ka[s][0].y, ka[s][1].y, qf[hg][s][1].x, qf[hg][s][1].y);
+        mma_bf16(d1, ka[s][0].z, ka[s][1].z, ka[s][0].w, ka[s][1].w, qf[hg][s][1].z, qf[hg][s][1].w);
+      }
+      // columns 2t, 2t+1 of the first n-tile are head t's hi and mid parts; column 2t of the second its lo part
+      const float s0 = d0[0] + (d0[1] + d1[0]);
+      const float s1 = d0[2] + (d0[3] + d1[2]);
+      const int head = hg * 4 + t;
+      if (head < p.G) {
+        if (tok0 < T) p.logits[(row0 + tok0) * p.G + head] = s0;
+        if (tok1 < T) p.logits[(row0 + tok1) * p.G + head] = s1;
+      }
+      float q0 = s0, q1 = s1;  // rows of absent heads are zero, so they add nothing
+      q0 += __shfl_xor_sync(0xffffffffu, q0, 1);
+      q1 += __shfl_xor_sync(0xffffffffu, q1, 1);
+      q0 += __shfl_xor_sync(0xffffffffu, q0, 2);
+      q1 += __shfl_xor_sync(0xffffffffu, q1, 2);
+      sig0 += q0;
+      sig1 += q1;
+    }
+    if (t == 0) {
+      if (tok0 < T) p.sigma[row0 + tok0] = sig0 + 0.0f;  // -0 becomes +0: the selection compares floats and keys
+      if (tok1 < T) p.sigma[row0 + tok1] = sig1 + 0.0f;
+    }
   }
 }
 
@@ -1338,25 +1262,16 @@ __global__ void __launch_bounds__(GA_THREADS, GMAX == 4 ? 4 : 2) attn_gather_ker
 // ============================================================================
 // host side
 // ============================================================================
-// Persistent grid: as many CTAs as are resident at once (two page buffers per warp, about 200 KB per SM in flight).
-template <int HD, int HG, int WARPS>
-static void launch_score_t(const ScoreDev& d, cudaStream_t st) {
-  const int smem = WARPS * 2 * PAGE * HD * 2 + WARPS * 2 * 8 + (PLAN_STRIDE + 4) * 4;
-  static int per_sm = 0;
-  ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_score_kernel<HD, HG, WARPS>), smem);
-  if (per_sm == 0) {
-    int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attn_score_kernel<HD, HG, WARPS>, WARPS * 32, smem) != cudaSuccess || n < 1)
-      n = 1;
-    per_sm = n;
-  }
-  SOL_LAUNCH("attn_score", (attn_score_kernel<HD, HG, WARPS>), dim3(sm_count() * per_sm), dim3(WARPS * 32), smem, st, d);
-}
 template <int HD>
-static void launch_score(const ScoreDev& d, int HG, cudaStream_t st) {
-  constexpr int WARPS = HD == 64 ? 4 : 3;  // 64 / 96 KB of page buffers per CTA: three / two CTAs per SM
-  if (HG == 1) launch_score_t<HD, 1, WARPS>(d, st);
-  else launch_score_t<HD, 2, WARPS>(d, st);
+static void launch_score(const ScoreDev& d, int HG, dim3 grid, cudaStream_t st) {
+  const int smem = SC_WARPS * PAGE * HD * 2 + SC_WARPS * 8 + 32;
+  if (HG == 1) {
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_score_kernel<HD, 1>), smem);
+    SOL_LAUNCH("attn_score", (attn_score_kernel<HD, 1>), grid, dim3(SC_WARPS * 32), smem, st, d);
+  } else {
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_score_kernel<HD, 2>), smem);
+    SOL_LAUNCH("attn_score", (attn_score_kernel<HD, 2>), grid, dim3(SC_WARPS * 32), smem, st, d);
+  }
 }
 
 // One CTA per item, at most as many CTAs as are resident at once (they are persistent).
@@ -1391,11 +1306,12 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(Hkv, a.B), dim3(PREP_THREADS), 0, st, pd);
 
   ScoreDev sd;
-  sd.kv = a.kv; sd.Hkv = Hkv; sd.G = G; sd.HG = HG; sd.Tmax = Tmax; sd.B = a.B;
-  sd.q_split = static_cast<const uint16_t*>(a.q_split); sd.plan = a.plan;
+  sd.kv = a.kv; sd.Hkv = Hkv; sd.G = G; sd.HG = HG; sd.Tmax = Tmax;
+  sd.q_split = static_cast<const uint16_t*>(a.q_split);
   sd.logits = a.logits; sd.sigma = a.sigma; sd.status = a.status;
-  if (hd == 64) launch_score<64>(sd, HG, st);
-  else launch_score<128>(sd, HG, st);
+  dim3 sgrid((a.kv.max_pages_per_seq + SC_WARPS - 1) / SC_WARPS, Hkv, a.B);
+  if (hd == 64) launch_score<64>(sd, HG, sgrid, st);
+  else launch_score<128>(sd, HG, sgrid, st);
 
   SelectDev se;
   se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.S = a.splits;
