@@ -20,6 +20,8 @@
 // additive -inf mask on dropped keys.
 #include <math.h>
 
+#include <type_traits>
+
 #include "sol_common.cuh"
 #include "sol_internal.h"
 #include "sol_select.cuh"
@@ -125,8 +127,12 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
       const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, tid);
       const int Tp = max(rp.T, 0);
       cnt[PLAN_PAGES] = (Tp + PAGE - 1) / PAGE;
-      cnt[PLAN_HSEG] = rp.mode == 2 ? (Tp + TH_SEG - 1) / TH_SEG : 0;
-      cnt[PLAN_SSEG] = max(1, (Tp + TS_SEG - 1) / TS_SEG);
+      // when no row can be longer than TH_SEG tokens a row is one histogram unit whatever its mode (that CTA
+      // does the whole selection of the row); otherwise: histogram units for the rows that need a selection,
+      // scan units for all
+      const bool local = p.kv.max_pages_per_seq * PAGE <= TH_SEG;
+      cnt[PLAN_HSEG] = local ? 1 : (rp.mode == 2 ? (Tp + TH_SEG - 1) / TH_SEG : 0);
+      cnt[PLAN_SSEG] = local ? 0 : max(1, (Tp + TS_SEG - 1) / TS_SEG);
       ch = max(1, (rp.k + p.split_len - 1) / p.split_len);
     }
     const int w = tid >> 5, l = tid & 31;
@@ -451,8 +457,15 @@ __device__ __forceinline__ int ts_block_scan(int v, int& total, int* warp_tot) {
   return before;
 }
 
-struct HistSmem {
+// Shared memory of token_hist: the histogram alone when rows go on to token_scan (more CTAs per SM), the
+// whole selection scratch when the CTA takes its row through the selection itself.
+struct HistOnly {
   uint32_t hist[SEL_BINS];
+};
+template <bool LOCAL>
+struct HistSmem {
+  typename std::conditional<LOCAL, SelectSmem, HistOnly>::type sm;  // its histogram is the one filled here
+  double qsum[LOCAL ? 128 : 1];
   int scan_tot[TS_THREADS / 32];
   float fmax_w[TS_THREADS / 32];
   int pick[2];
@@ -460,9 +473,16 @@ struct HistSmem {
   int cum[PLAN_STRIDE];
 };
 
-// One (sequence, kv-head, 8192-token segment) of token_hist.
-__device__ __forceinline__ void token_hist_item(const SelectDev& p, HistSmem& hs, int b, int kvh, int seg) {
-  uint32_t* hist = hs.hist;
+__device__ __forceinline__ void settle_row(const SelectDev& p, SelectSmem& sm, double* qsum, const RowPlan& rp, int b,
+                                           int kvh, int n_list, float edge, float lo, float delta, int ns_all,
+                                           bool cands_in_smem);
+
+// One (sequence, kv-head, 8192-token segment) of token_hist.  When the page table allows no row longer than
+// 8192 tokens every row is one unit, and its CTA takes the row through the whole selection (edges, list,
+// candidates, work items): token_scan and token_settle are then not launched.
+template <bool LOCAL>
+__device__ __forceinline__ void token_hist_item(const SelectDev& p, HistSmem<LOCAL>& hs, int b, int kvh, int seg) {
+  uint32_t* hist = hs.sm.hist;
   int* scan_tot = hs.scan_tot;
   float* fmax_w = hs.fmax_w;
   int* pick = hs.pick;
@@ -470,14 +490,18 @@ __device__ __forceinline__ void token_hist_item(const SelectDev& p, HistSmem& hs
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, b);
   const int T = rp.T;
-  if (rp.mode != 2 || seg * TH_SEG >= T) return;
-  for (int i = tid; i < SEL_BINS; i += TS_THREADS) hist[i] = 0;
-  __syncthreads();
-  const int bk = b * p.sh.n_kv_heads + kvh;
+  constexpr bool local = LOCAL;  // no row of this call is longer than one unit
+  if (!local && (rp.mode != 2 || seg * TH_SEG >= T)) return;
+  const int Hkv = p.sh.n_kv_heads;
+  const int bk = b * Hkv + kvh;
   const float* sig = p.sigma + (size_t)bk * p.Tmax;
   uint32_t* ctl = p.row_ctl + (size_t)bk * RC_WORDS;
   uint32_t* gh = p.row_hist + (size_t)bk * SEL_BINS;
-  const int nseg = (T + TH_SEG - 1) / TH_SEG;
+  const int nseg = max(1, (T + TH_SEG - 1) / TH_SEG);
+  float lo = TS_FLT_MAX, edge = TS_FLT_MAX, delta = 0.f;
+  if (rp.mode == 2) {
+  for (int i = tid; i < SEL_BINS; i += TS_THREADS) hist[i] = 0;
+  __syncthreads();
 
   // ---- this CTA's scores: 32 per thread, all loads issued before the first use ----
   float mx = 0.f;
@@ -574,18 +598,99 @@ __device__ __forceinline__ void token_hist_item(const SelectDev& p, HistSmem& hs
     klo = (klo & 0xfffe0000u) | ((uint32_t)pick[0] << 5);
     khi = klo | 31u;
   }
-  if (tid == 0) {
-    // window: 2^-16 of the largest score, far above the float32 accumulation error of a head_dim-long dot product
-    const float delta = mx * 1.52587890625e-05f;
+  // window: 2^-16 of the largest score, far above the float32 accumulation error of a head_dim-long dot product
+  delta = mx * 1.52587890625e-05f;
+  lo = key_to_float(klo) - delta;
+  edge = fminf(key_to_float(khi) + delta, TS_FLT_MAX);
+  if (tid == 0) {  // for token_scan / token_settle of a long row, and for token_list
     ctl[RC_DELTA] = __float_as_uint(delta);
-    ctl[RC_LO] = __float_as_uint(key_to_float(klo) - delta);
-    ctl[RC_EDGE] = __float_as_uint(fminf(key_to_float(khi) + delta, TS_FLT_MAX));
+    ctl[RC_LO] = __float_as_uint(lo);
+    ctl[RC_EDGE] = __float_as_uint(edge);
   }
+  if (!local) return;
+  }  // mode 2
+
+  // ---- a row of one unit: its list and its candidates, 2048 tokens at a time, then the settling ----
+  if constexpr (LOCAL) {
+  SelectSmem& sm = hs.sm;
+  __syncthreads();  // the histogram is not read any more: its space stages the list
+  if (tid < 4) sm.counts[tid] = 0;
+  __syncthreads();
+  const size_t row = (size_t)bk * p.Tmax;
+  int32_t* lidx = p.list_idx + row;
+  uint32_t* lrow = p.list_row + row;
+  const int32_t* table = p.kv.page_table + (size_t)b * p.kv.max_pages_per_seq;
+  int32_t* st_idx = reinterpret_cast<int32_t*>(sm.hist);
+  uint32_t* st_row = sm.hist + TS_SEG;
+  int n_list = 0;
+#pragma unroll 1
+  for (int base0 = 0; base0 < T; base0 += TS_SEG) {
+    const int j0 = base0 + tid * 8;
+    uint32_t keep = 0;
+    if (j0 < T) {
+      if (rp.mode == 0) {
+        keep = T - j0 >= 8 ? 0xffu : ((1u << (T - j0)) - 1u);
+      } else {
+        float vv[8];
+        if (rp.mode == 2) {
+          const float4 v0 = *reinterpret_cast<const float4*>(sig + j0), v1 = *reinterpret_cast<const float4*>(sig + j0 + 4);
+          vv[0] = v0.x; vv[1] = v0.y; vv[2] = v0.z; vv[3] = v0.w; vv[4] = v1.x; vv[5] = v1.y; vv[6] = v1.z; vv[7] = v1.w;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int j = j0 + e;
+          if (j >= T) continue;
+          if (rp.forced(j)) {
+            keep |= 1u << e;
+          } else if (rp.mode == 2) {
+            if (vv[e] > edge) {
+              keep |= 1u << e;
+            } else if (vv[e] >= lo) {
+              const int slot = atomicAdd(&sm.counts[0], 1);
+              if (slot < SEL_CAND_CAP) {
+                sm.cand_idx[slot] = j;
+                sm.f32[slot] = vv[e];
+              }
+            }
+          }
+        }
+      }
+    }
+    int total;
+    const int before = ts_block_scan(__popc(keep), total, scan_tot);
+    if (keep) {
+      // eight consecutive tokens share a page
+      const int page = table[j0 / PAGE];
+      const bool ok = page >= 0 && page < p.kv.num_pages;
+      if (!ok) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+      const uint32_t r0 = (uint32_t)((page * Hkv + kvh) * PAGE + (j0 % PAGE));
+      int pos = before;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        if ((keep >> e) & 1u) {
+          st_idx[pos] = j0 + e;
+          st_row[pos] = ok ? r0 + e : 0xffffffffu;
+          ++pos;
+        }
+      }
+    }
+    __syncthreads();
+    for (int i = tid; i < total; i += TS_THREADS) {
+      lidx[n_list + i] = st_idx[i];
+      lrow[n_list + i] = st_row[i];
+    }
+    n_list += total;
+    __syncthreads();  // the staging space is rewritten by the next 2048 tokens
+  }
+  const int ns_all = sm.counts[0];
+  settle_row(p, sm, hs.qsum, rp, b, kvh, n_list, edge, lo, delta, ns_all, true);
+  }  // LOCAL
 }
 
 // Persistent CTAs over the flat list of (sequence, kv-head, segment) units of the rows that need a selection.
+template <bool LOCAL>
 __global__ void __launch_bounds__(TS_THREADS) token_hist_kernel(const SelectDev p) {
-  __shared__ HistSmem hs;
+  __shared__ HistSmem<LOCAL> hs;
   pdl_trigger();
   pdl_wait();
   for (int i = threadIdx.x; i <= p.B; i += TS_THREADS) hs.cum[i] = p.plan[PLAN_HSEG * PLAN_STRIDE + i];
@@ -595,7 +700,7 @@ __global__ void __launch_bounds__(TS_THREADS) token_hist_kernel(const SelectDev 
   for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
     const int b = plan_find(hs.cum, p.B, u / Hkv);
     const int n = hs.cum[b + 1] - hs.cum[b], rem = u - hs.cum[b] * Hkv;
-    token_hist_item(p, hs, b, rem / n, rem % n);
+    token_hist_item<LOCAL>(p, hs, b, rem / n, rem % n);
     __syncthreads();
   }
 }
@@ -719,39 +824,29 @@ __device__ __forceinline__ void token_scan_item(const SelectDev& p, ScanSmem& ss
 
 }
 
-// One CTA per (sequence, kv-head), after token_scan: ranks the candidates between the edges in float32,
-// re-scores those within the window of the k-th value in float64 from the cache rows, appends the kept ones
-// (ascending) to the row's list, and emits the row's pass-2 work items.
-__global__ void __launch_bounds__(TS_THREADS) token_settle_kernel(const SelectDev p) {
-  __shared__ SelectSmem sm;
-  __shared__ double qsum[128];
-  const int kvh = blockIdx.x, b = blockIdx.y;
+// The end of a row's selection, by one CTA: n_list tokens are already in the row's list (everything above the
+// edge, and the forced tokens); ns_all candidates lie between the edges (in shared memory: sm.cand_idx and
+// sm.f32, or in the row's global candidate list).  Ranks the candidates in float32, re-scores those within
+// the window of the k-th value in float64 from the cache rows, appends the kept ones (ascending) to the
+// list, and emits the row's pass-2 work items.
+__device__ __forceinline__ void settle_row(const SelectDev& p, SelectSmem& sm, double* qsum, const RowPlan& rp, int b,
+                                           int kvh, int n_list, float edge, float lo, float delta, int ns_all,
+                                           bool cands_in_smem) {
   const int Hkv = p.sh.n_kv_heads, hd = p.sh.head_dim, G = p.sh.n_q_heads / Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int WARPS = TS_THREADS / 32;
   const int bk = b * Hkv + kvh;
-  pdl_trigger();
-  const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, b);
-  pdl_wait();
   const int T = rp.T, mode = rp.mode;
   const size_t row = (size_t)bk * p.Tmax;
   float* sig = p.sigma + row;
-  uint32_t* ctl = p.row_ctl + (size_t)bk * RC_WORDS;
-  const uint32_t* pub = p.seg_pub + (size_t)bk * p.nseg_max;
   int32_t* lidx = p.list_idx + row;
   uint32_t* lrow = p.list_row + row;
   const int32_t* table = p.kv.page_table + (size_t)b * p.kv.max_pages_per_seq;
-  const int nseg = max(1, (T + TS_SEG - 1) / TS_SEG);
-  const float edge = mode == 2 ? __uint_as_float(ctl[RC_EDGE]) : TS_FLT_MAX;
-  const float lo = mode == 2 ? __uint_as_float(ctl[RC_LO]) : TS_FLT_MAX;
-  int n_list = 0;  // kept so far: what the segments wrote
-  for (int q = 0; q < nseg; ++q) n_list += (int)(pub[q] & ~TS_READY);
+  __syncthreads();
   if (tid < 4) sm.counts[tid] = 0;
   __syncthreads();
   if (mode == 2) {
-    const int ns_all = (int)__ldcg(ctl + RC_NCAND);
     const int need_s = rp.k - n_list;
-    const float delta = __uint_as_float(ctl[RC_DELTA]);
     if (ns_all > SEL_CAND_CAP || need_s < 0 || need_s > ns_all) {
       // More scores between the edges than the list holds (long runs of equal scores): float32 order with
       // ties to the lower index, by a radix select over the row's keys that lie between the edges.
@@ -816,9 +911,11 @@ __global__ void __launch_bounds__(TS_THREADS) token_settle_kernel(const SelectDe
     } else if (need_s > 0) {
       const int ns = ns_all;
       float* sup_val = sm.f32;
-      for (int c = tid; c < ns; c += TS_THREADS) {
-        sm.cand_idx[c] = __ldcg(p.cand_idx + (size_t)bk * SEL_CAND_CAP + c);
-        sup_val[c] = __ldcg(p.cand_val + (size_t)bk * SEL_CAND_CAP + c);
+      if (!cands_in_smem) {
+        for (int c = tid; c < ns; c += TS_THREADS) {
+          sm.cand_idx[c] = __ldcg(p.cand_idx + (size_t)bk * SEL_CAND_CAP + c);
+          sup_val[c] = __ldcg(p.cand_val + (size_t)bk * SEL_CAND_CAP + c);
+        }
       }
       __syncthreads();
       // float32 rank inside the list: the element of rank need_s - 1 carries the k-th value
@@ -937,6 +1034,26 @@ __global__ void __launch_bounds__(TS_THREADS) token_scan_kernel(const SelectDev 
   }
 }
 
+// One CTA per (sequence, kv-head) of the rows that token_scan worked on.
+__global__ void __launch_bounds__(TS_THREADS) token_settle_kernel(const SelectDev p) {
+  __shared__ SelectSmem sm;
+  __shared__ double qsum[128];
+  const int kvh = blockIdx.x, b = blockIdx.y;
+  pdl_trigger();
+  const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, b);
+  pdl_wait();
+  const int bk = b * p.sh.n_kv_heads + kvh;
+  const uint32_t* ctl = p.row_ctl + (size_t)bk * RC_WORDS;
+  const uint32_t* pub = p.seg_pub + (size_t)bk * p.nseg_max;
+  const int nseg = max(1, (rp.T + TS_SEG - 1) / TS_SEG);
+  int n_list = 0;  // kept so far: what the segments wrote
+  for (int q = 0; q < nseg; ++q) n_list += (int)(pub[q] & ~TS_READY);
+  const bool sel = rp.mode == 2;
+  settle_row(p, sm, qsum, rp, b, kvh, n_list, sel ? __uint_as_float(ctl[RC_EDGE]) : TS_FLT_MAX,
+             sel ? __uint_as_float(ctl[RC_LO]) : TS_FLT_MAX, sel ? __uint_as_float(ctl[RC_DELTA]) : 0.f,
+             sel ? (int)ctl[RC_NCAND] : 0, false);
+}
+
 struct ListDev {
   sol_shape_t sh;
   sol_kv_t kv;
@@ -999,44 +1116,70 @@ struct GatherDev {
   int* status;
 };
 
-constexpr int GA_WARPS = 8;
-constexpr int GA_THREADS = GA_WARPS * 32;
 constexpr int GA_BATCH = 32;  // kept tokens per warp step: one per lane in the softmax part
-constexpr int GA_ROWS_IN_FLIGHT = 8;  // row loads a lane issues before it consumes the first
 
-// Pass 2 is a gather of 128- or 256-byte V rows with G multiply-adds per element: bound by memory
-// latency, not by arithmetic, so it runs on the FMA pipes with many warps per SM and no shared-memory
-// staging of the rows.
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src, bool valid) {
+  const uint32_t n = valid ? 16u : 0u;  // 0: the 16 bytes are filled with zeros and the source is not read
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// Pass 2 is a gather of 128- or 256-byte V rows with G multiply-adds per element: bound by how many row
+// fetches are in flight, so the rows travel by asynchronous 16-byte copies into per-warp rings of shared
+// memory (about 190 KB per SM, three quarters of it in flight) and the registers only hold accumulators.
 //
-// Persistent CTAs work through the list of items: (sequence, kv-head, run of at most 1024 kept tokens);
-// a CTA's first item is dealt by its index, the later ones are claimed from a counter one item ahead.
-// The 8 warps of a CTA take the item's tokens in batches of 32, each warp on its own:
-//   lane l of the warp fetches the index words and the G logits of token l of the batch (the next
-//   batch's while the current one is processed), the warp updates its running maximum per head and
-//   every lane computes its token's softmax weights; cache rows and weights go to a small
-//   shared-memory table; then the warp walks over the batch's rows: a row is read by HD/4 lanes (8
-//   bytes each, 8 rows in flight per lane) and multiplied into the lane's float32 accumulators
-//   (G heads x 4 columns).
+// One persistent CTA per SM works through the list of items: (sequence, kv-head, run of at most
+// ATTN_ITEM_CHUNKS chunks of kept tokens); a CTA's first item is dealt by its index, the later ones are
+// claimed from a counter one item ahead.  The warps of a CTA take the item's tokens in batches of 32, each
+// warp on its own, NST batches deep:
+//   lane l fetches the list words of token l of a batch (cache row, token index) two steps before the
+//   batch's rows are requested and its G logits one step before they are used; when a batch's rows have
+//   landed the warp updates its running maximum per head, every lane computes its token's softmax weights,
+//   and the warp walks over the rows: a row is read by HD/4 lanes (8 bytes each) and multiplied into the
+//   lane's float32 accumulators (G heads x 4 columns).
 // Per item one partial (accumulators, maximum, sum; merged over the warps) is written; the CTA that
 // finishes the last item of a (sequence, kv-head) merges its partials.
 template <int HD, int GMAX>
-__global__ void __launch_bounds__(GA_THREADS, GMAX == 4 ? 4 : 2) attn_gather_kernel(const GatherDev p) {
+struct GatherCfg {
+  static constexpr int WARPS = HD == 64 ? 12 : 8;
+  static constexpr int NST = HD == 64 ? 4 : 3;              // batches of rows per warp ring
+  static constexpr int STAGE_BYTES = GA_BATCH * HD * 2;      // 4 KB / 8 KB
+  static constexpr int THREADS = WARPS * 32;
+  static constexpr int RING_BYTES = WARPS * NST * STAGE_BYTES;  // 192 KB
+  static constexpr int TAB_BYTES = WARPS * (NST + 1) * GA_BATCH * 8;
+  static constexpr int W_BYTES = WARPS * GA_BATCH * GMAX * 4;
+  static constexpr int ML_BYTES = WARPS * GMAX * 2 * 4;
+  static constexpr int SMEM = RING_BYTES + TAB_BYTES + W_BYTES + ML_BYTES + 64;
+  static_assert(WARPS * GMAX * HD * 4 <= RING_BYTES, "the merge scratch fits the ring");
+};
+
+template <int HD, int GMAX>
+__global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_kernel(const GatherDev p) {
+  using C = GatherCfg<HD, GMAX>;
+  constexpr int WARPS = C::WARPS, NST = C::NST, THREADS = C::THREADS;
   constexpr int SPLIT = HD == 64 ? 256 : 128;  // kept tokens per chunk (attn_split_len): the unit of the item list
   constexpr int LPT = HD / 4;                  // lanes per row
-  constexpr int TPS = 32 / LPT;                // rows per warp-wide load
-  constexpr int U = GA_ROWS_IN_FLIGHT;
-  static_assert(GA_BATCH % (U * TPS) == 0, "a batch is a whole number of load groups");
-  __shared__ uint32_t s_row[GA_WARPS][GA_BATCH];
-  __shared__ __align__(16) float s_w[GA_WARPS][GA_BATCH][GMAX];
-  __shared__ __align__(16) float sc_acc[GA_WARPS][GMAX][HD];
-  __shared__ float sc_ml[GA_WARPS][GMAX][2];
-  __shared__ __align__(16) int hdr[2][4];  // (sequence, kv-head) or -1, first token, tokens, kept count
-  __shared__ int flag;
+  constexpr int TPS = 32 / LPT;                // rows per warp-wide read
+  constexpr int CPR = HD / 8;                  // 16-byte pieces per row
+  extern __shared__ __align__(128) unsigned char gsm[];
+  unsigned char* ring = gsm;
+  int2* s_tab = reinterpret_cast<int2*>(gsm + C::RING_BYTES);                       // [WARPS][NST + 1][32] (cache row, token)
+  float* s_w = reinterpret_cast<float*>(gsm + C::RING_BYTES + C::TAB_BYTES);        // [WARPS][32][GMAX]
+  float* sc_ml = reinterpret_cast<float*>(gsm + C::RING_BYTES + C::TAB_BYTES + C::W_BYTES);  // [WARPS][GMAX][2]
+  int* hdr = reinterpret_cast<int*>(gsm + C::RING_BYTES + C::TAB_BYTES + C::W_BYTES + C::ML_BYTES);  // [2][4], then the flag
+  float* sc_acc = reinterpret_cast<float*>(ring);  // [WARPS][GMAX][HD], after an item's batches are done
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.G, Hkv = p.Hkv;
   const uint16_t* vp = static_cast<const uint16_t*>(p.kv.v_pool);
-  const int sub = lane / LPT, col = (lane % LPT) * 4;  // which row of a load step, which four columns
+  const int sub = lane / LPT, col = (lane % LPT) * 4;  // which row of a read step, which four columns
+  unsigned char* my_ring = ring + (size_t)warp * NST * C::STAGE_BYTES;
+  int2* my_tab = s_tab + warp * (NST + 1) * GA_BATCH;
+  float* my_w = s_w + warp * GA_BATCH * GMAX;
   pdl_trigger();
   pdl_wait();
   const int cpi = p.work_ctr[WC_CPI];
@@ -1048,13 +1191,13 @@ __global__ void __launch_bounds__(GA_THREADS, GMAX == 4 ? 4 : 2) attn_gather_ker
   if (tid == 0) {
     int4 h = make_int4(-1, 0, 0, 0);
     if ((int)blockIdx.x < n_items) h = header_of(*reinterpret_cast<const int2*>(p.work_items + 2 * blockIdx.x));
-    *reinterpret_cast<int4*>(hdr[0]) = h;
+    *reinterpret_cast<int4*>(hdr) = h;
   }
   __syncthreads();
 
 #pragma unroll 1
   for (int it = 0;; ++it) {
-    const int4 cur = *reinterpret_cast<const int4*>(hdr[it & 1]);
+    const int4 cur = *reinterpret_cast<const int4*>(hdr + 4 * (it & 1));
     if (cur.x < 0) break;
     int claimed = 0;
     if (tid == 0) claimed = (int)gridDim.x + atomicAdd(p.work_ctr + WC_NEXT, 1);
@@ -1064,22 +1207,35 @@ __global__ void __launch_bounds__(GA_THREADS, GMAX == 4 ? 4 : 2) attn_gather_ker
     const uint32_t* krow = p.kept_row + row + cur.y;
     const int32_t* kidx = p.kept_idx + row + cur.y;
     const float* lgrow = p.logits + row * G;
-    const int nb = (len + GA_BATCH - 1) / GA_BATCH;
+    const int nb = (len + GA_BATCH - 1) / GA_BATCH;       // batches of the item
+    const int my_nb = nb > warp ? (nb - warp + WARPS - 1) / WARPS : 0;  // this warp's: warp, warp + WARPS, ...
 
-    auto load_idx = [&](int q, uint32_t& r, int& j) {
-      const int n = q * GA_BATCH + lane;
-      r = 0xffffffffu;
-      j = 0;
-      if (q < nb && n < len) {
-        r = krow[n];
-        j = kidx[n];
-      }
+    // list words of this warp's m-th batch: lane l holds token l
+    auto load_tab = [&](int m) {
+      int2 e = make_int2(-1, 0);
+      const int n = (warp + m * WARPS) * GA_BATCH + lane;
+      if (m < my_nb && n < len) e = make_int2((int)krow[n], kidx[n]);
+      return e;
     };
-    auto load_logits = [&](uint32_t r, int j, float (&x)[GMAX]) {
+    // requests the rows of the m-th batch (its list words are in the table) into ring slot m % NST
+    auto request_rows = [&](int m) {
+      if (m < my_nb) {
+        const int2* tab = my_tab + (m % (NST + 1)) * GA_BATCH;
+        const uint32_t dst0 = smem_u32(my_ring + (m % NST) * C::STAGE_BYTES);
+#pragma unroll
+        for (int i = 0; i < CPR; ++i) {
+          const int c = i * 32 + lane, r = c / CPR, part = c % CPR;
+          const int ridx = tab[r].x;
+          cp_async16(dst0 + c * 16, vp + (size_t)(ridx < 0 ? 0 : ridx) * HD + part * 8, ridx >= 0);
+        }
+      }
+      cp_async_commit();  // an empty group keeps the count of groups per step fixed
+    };
+    auto load_logits = [&](int2 e, float (&x)[GMAX]) {
 #pragma unroll
       for (int h = 0; h < GMAX; ++h) x[h] = -INFINITY;  // an absent token weighs nothing
-      if (r == 0xffffffffu) return;
-      const float* src = lgrow + (size_t)j * G;
+      if (e.x < 0) return;
+      const float* src = lgrow + (size_t)e.y * G;
       if (GMAX == 4 && G == 4) {
         const float4 v = *reinterpret_cast<const float4*>(src);
         x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
@@ -1098,21 +1254,24 @@ __global__ void __launch_bounds__(GA_THREADS, GMAX == 4 ? 4 : 2) attn_gather_ker
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[h][c] = 0.f;
     }
-    uint32_t r_c, r_n;
-    int j_c, j_n;
+    // prologue: list words of the first NST batches, rows of the first NST - 1, logits of the first
+#pragma unroll
+    for (int m = 0; m < NST; ++m) my_tab[(m % (NST + 1)) * GA_BATCH + lane] = load_tab(m);
+    __syncwarp();
+#pragma unroll
+    for (int m = 0; m < NST - 1; ++m) request_rows(m);
+    int2 e_far = load_tab(NST);  // held in a register until its table slot is free
     float x_c[GMAX];
-    load_idx(warp, r_c, j_c);
-    load_idx(warp + GA_WARPS, r_n, j_n);
-    load_logits(r_c, j_c, x_c);
+    load_logits(my_tab[lane], x_c);
 
 #pragma unroll 1
-    for (int q = warp; q < nb; q += GA_WARPS) {
-      // the next batch's logits and the index words of the batch after it start now
+    for (int m = 0; m < my_nb; ++m) {
+      // the table slot of batch m - 1 is free now: batch m + NST moves in; rows of batch m + NST - 1 are requested
+      my_tab[((m + NST) % (NST + 1)) * GA_BATCH + lane] = e_far;
+      request_rows(m + NST - 1);
+      e_far = load_tab(m + NST + 1);
       float x_n[GMAX];
-      load_logits(r_n, j_n, x_n);
-      uint32_t r_nn;
-      int j_nn;
-      load_idx(q + 2 * GA_WARPS, r_nn, j_nn);
+      load_logits(m + 1 < my_nb ? my_tab[((m + 1) % (NST + 1)) * GA_BATCH + lane] : make_int2(-1, 0), x_n);
 
       // ---- softmax weights relative to the running maximum ----
 #pragma unroll
@@ -1125,52 +1284,43 @@ __global__ void __launch_bounds__(GA_THREADS, GMAX == 4 ? 4 : 2) attn_gather_ker
         ls[h] = ls[h] * sc + pw;
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[h][c] *= sc;
-        s_w[warp][lane][h] = pw;
+        my_w[lane * GMAX + h] = pw;
       }
-      s_row[warp][lane] = r_c;
-      __syncwarp();
+      cp_async_wait<NST - 1>();  // this lane's pieces of batch m have landed ...
+      __syncwarp();              // ... and so have the other lanes'; the weights are in the table
 
       // ---- weights x rows ----
-      const int nt = min(GA_BATCH, len - q * GA_BATCH);
-#pragma unroll 1
-      for (int k0 = 0; k0 < nt; k0 += U * TPS) {
-        uint2 v[U];
+      const int nt = min(GA_BATCH, len - (warp + m * WARPS) * GA_BATCH);
+      const unsigned char* st = my_ring + (m % NST) * C::STAGE_BYTES;
+#pragma unroll 4
+      for (int k0 = 0; k0 < GA_BATCH; k0 += TPS) {
+        if (k0 >= nt) break;
+        const int r = k0 + sub;  // rows past the batch's end were filled with zeros and weigh nothing
+        const uint2 v = *reinterpret_cast<const uint2*>(st + (size_t)r * HD * 2 + col * 2);
+        const float* w = my_w + r * GMAX;
+        const float f0 = __uint_as_float(v.x << 16), f1 = __uint_as_float(v.x & 0xffff0000u);
+        const float f2 = __uint_as_float(v.y << 16), f3 = __uint_as_float(v.y & 0xffff0000u);
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-          const uint32_t r = s_row[warp][k0 + u * TPS + sub];
-          v[u] = make_uint2(0u, 0u);
-          if (r != 0xffffffffu) v[u] = __ldcs(reinterpret_cast<const uint2*>(vp + (size_t)r * HD + col));
-        }
+        for (int h4 = 0; h4 < GMAX; h4 += 4) {
+          const float4 w4 = *reinterpret_cast<const float4*>(w + h4);
+          const float ww[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-          const float* w = s_w[warp][k0 + u * TPS + sub];
-          const float f0 = __uint_as_float(v[u].x << 16), f1 = __uint_as_float(v[u].x & 0xffff0000u);
-          const float f2 = __uint_as_float(v[u].y << 16), f3 = __uint_as_float(v[u].y & 0xffff0000u);
-#pragma unroll
-          for (int h4 = 0; h4 < GMAX; h4 += 4) {
-            const float4 w4 = *reinterpret_cast<const float4*>(w + h4);
-            const float ww[4] = {w4.x, w4.y, w4.z, w4.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              acc[h4 + e][0] = fmaf(ww[e], f0, acc[h4 + e][0]);
-              acc[h4 + e][1] = fmaf(ww[e], f1, acc[h4 + e][1]);
-              acc[h4 + e][2] = fmaf(ww[e], f2, acc[h4 + e][2]);
-              acc[h4 + e][3] = fmaf(ww[e], f3, acc[h4 + e][3]);
-            }
+          for (int e = 0; e < 4; ++e) {
+            acc[h4 + e][0] = fmaf(ww[e], f0, acc[h4 + e][0]);
+            acc[h4 + e][1] = fmaf(ww[e], f1, acc[h4 + e][1]);
+            acc[h4 + e][2] = fmaf(ww[e], f2, acc[h4 + e][2]);
+            acc[h4 + e][3] = fmaf(ww[e], f3, acc[h4 + e][3]);
           }
         }
       }
-      __syncwarp();  // the tables are rewritten for the next batch
-      r_c = r_n;
-      j_c = j_n;
+      __syncwarp();  // the weights and the ring slot are rewritten by the next steps
 #pragma unroll
       for (int h = 0; h < GMAX; ++h) x_c[h] = x_n[h];
-      r_n = r_nn;
-      j_n = j_nn;
     }
+    cp_async_wait<0>();
 
     // ---- one partial per item: merge the warps ----
-    if (TPS == 2) {  // two rows per load step: the half-warps hold partial sums of the same columns
+    if (TPS == 2) {  // two rows per read step: the half-warps hold partial sums of the same columns
 #pragma unroll
       for (int h = 0; h < GMAX; ++h)
 #pragma unroll
@@ -1178,16 +1328,17 @@ __global__ void __launch_bounds__(GA_THREADS, GMAX == 4 ? 4 : 2) attn_gather_ker
     }
 #pragma unroll
     for (int h = 0; h < GMAX; ++h) ls[h] = warp_sum(ls[h]);
+    __syncthreads();  // every warp is done with its ring: the merge scratch lies over it
     if (sub == 0) {
 #pragma unroll
       for (int h = 0; h < GMAX; ++h)
-        *reinterpret_cast<float4*>(&sc_acc[warp][h][col]) = make_float4(acc[h][0], acc[h][1], acc[h][2], acc[h][3]);
+        *reinterpret_cast<float4*>(&sc_acc[(warp * GMAX + h) * HD + col]) = make_float4(acc[h][0], acc[h][1], acc[h][2], acc[h][3]);
     }
     if (lane == 0) {
 #pragma unroll
       for (int h = 0; h < GMAX; ++h) {
-        sc_ml[warp][h][0] = mh[h];
-        sc_ml[warp][h][1] = ls[h];
+        sc_ml[(warp * GMAX + h) * 2] = mh[h];
+        sc_ml[(warp * GMAX + h) * 2 + 1] = ls[h];
       }
     }
     // the header of the claimed item is fetched while the partial is put together
@@ -1196,18 +1347,18 @@ __global__ void __launch_bounds__(GA_THREADS, GMAX == 4 ? 4 : 2) attn_gather_ker
     __syncthreads();
     const int slot_no = (cur.y / SPLIT) / cpi;  // this item's partial
     float* dst = p.part + (((size_t)bk * p.S + slot_no) * G) * (HD + 2);
-    for (int e0 = tid; e0 < G * HD; e0 += GA_THREADS) {
+    for (int e0 = tid; e0 < G * HD; e0 += THREADS) {
       const int h = e0 / HD, e = e0 % HD;
       float M = -INFINITY;
 #pragma unroll
-      for (int w = 0; w < GA_WARPS; ++w) M = fmaxf(M, sc_ml[w][h][0]);
+      for (int w = 0; w < WARPS; ++w) M = fmaxf(M, sc_ml[(w * GMAX + h) * 2]);
       float a = 0.f, l = 0.f;
 #pragma unroll
-      for (int w = 0; w < GA_WARPS; ++w) {
-        const float mw = sc_ml[w][h][0];
+      for (int w = 0; w < WARPS; ++w) {
+        const float mw = sc_ml[(w * GMAX + h) * 2];
         const float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
-        a += sc_acc[w][h][e] * f;
-        l += sc_ml[w][h][1] * f;
+        a += sc_acc[(w * GMAX + h) * HD + e] * f;
+        l += sc_ml[(w * GMAX + h) * 2 + 1] * f;
       }
       dst[h * (HD + 2) + e] = a;
       if (e == 0) {
@@ -1222,16 +1373,16 @@ __global__ void __launch_bounds__(GA_THREADS, GMAX == 4 ? 4 : 2) attn_gather_ker
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-      flag = atomicAdd(p.work_ctr + WC_DONE + bk, 1) == ns - 1 ? 1 : 0;
+      hdr[8] = atomicAdd(p.work_ctr + WC_DONE + bk, 1) == ns - 1 ? 1 : 0;
       int4 h = make_int4(-1, 0, 0, 0);
       if (claimed < n_items) h = header_of(claimed_words);
-      *reinterpret_cast<int4*>(hdr[(it + 1) & 1]) = h;
+      *reinterpret_cast<int4*>(hdr + 4 * ((it + 1) & 1)) = h;
     }
     __syncthreads();
-    if (flag) {
+    if (hdr[8]) {
       __threadfence();
       const float* src0 = p.part + ((size_t)bk * p.S * G) * (HD + 2);
-      for (int e0 = tid; e0 < G * HD; e0 += GA_THREADS) {
+      for (int e0 = tid; e0 < G * HD; e0 += THREADS) {
         const int h = e0 / HD, e = e0 % HD;
         float m = -INFINITY, l = 0.f, a = 0.f;
         for (int q = 0; q < ns; ++q) {
@@ -1274,19 +1425,14 @@ static void launch_score(const ScoreDev& d, int HG, dim3 grid, cudaStream_t st) 
   }
 }
 
-// One CTA per item, at most as many CTAs as are resident at once (they are persistent).
+// One CTA per item, at most one per SM (they are persistent).
 template <int HD, int GMAX>
 static void launch_gather(const GatherDev& d, long long items, cudaStream_t st) {
-  static int per_sm = 0;  // the same on every device this library supports
-  if (per_sm == 0) {
-    int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attn_gather_kernel<HD, GMAX>, GA_THREADS, 0) != cudaSuccess || n < 1)
-      n = 1;
-    per_sm = n;
-  }
-  const long long resident = (long long)sm_count() * per_sm;
+  using C = GatherCfg<HD, GMAX>;
+  ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_gather_kernel<HD, GMAX>), C::SMEM);
+  const long long resident = sm_count();
   const int grid = (int)(items < resident ? items : resident);
-  SOL_LAUNCH("attn_gather_v", (attn_gather_kernel<HD, GMAX>), dim3(grid), dim3(GA_THREADS), 0, st, d);
+  SOL_LAUNCH("attn_gather_v", (attn_gather_kernel<HD, GMAX>), dim3(grid), dim3(C::THREADS), C::SMEM, st, d);
 }
 
 void launch_attention(const AttnArgs& a, cudaStream_t st) {
@@ -1302,7 +1448,7 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   pd.row_hist = a.row_hist; pd.row_ctl = a.row_ctl; pd.seg_pub = a.seg_pub;
   pd.nseg_max = attn_select_segs(a.kv.max_pages_per_seq, PAGE);
   pd.plan = a.plan; pd.r_permille = a.r_permille; pd.split_len = attn_split_len(hd);
-  pd.target_items = sm_count() * (G <= 4 ? 4 : 2);  // the pass-2 CTAs resident at once
+  pd.target_items = sm_count();  // the pass-2 CTAs resident at once
   SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(Hkv, a.B), dim3(PREP_THREADS), 0, st, pd);
 
   ScoreDev sd;
@@ -1323,23 +1469,30 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   se.plan = a.plan;
   {
     // persistent grids: never more CTAs than are resident at once, never more than there can be units
-    static int hist_per_sm = 0, scan_per_sm = 0;
-    if (hist_per_sm == 0) {
+    static int hist_per_sm[2] = {0, 0}, scan_per_sm = 0;
+    if (scan_per_sm == 0) {
       int n = 0;
-      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_hist_kernel, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
-      hist_per_sm = n;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_hist_kernel<false>, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
+      hist_per_sm[0] = n;
+      n = 0;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_hist_kernel<true>, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
+      hist_per_sm[1] = n;
       n = 0;
       if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_scan_kernel, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
       scan_per_sm = n;
     }
+    const bool local = Tmax <= TH_SEG;
     const long long hist_units = (long long)a.B * Hkv * ((Tmax + TH_SEG - 1) / TH_SEG);
     const long long scan_units = (long long)a.B * Hkv * se.nseg_max;
-    const long long hist_res = (long long)sm_count() * hist_per_sm, scan_res = (long long)sm_count() * scan_per_sm;
-    SOL_LAUNCH("token_hist", token_hist_kernel, dim3((unsigned)(hist_units < hist_res ? hist_units : hist_res)),
-               dim3(TS_THREADS), 0, st, se);
-    SOL_LAUNCH("token_scan", token_scan_kernel, dim3((unsigned)(scan_units < scan_res ? scan_units : scan_res)),
-               dim3(TS_THREADS), 0, st, se);
-    SOL_LAUNCH("token_settle", token_settle_kernel, dim3(Hkv, a.B), dim3(TS_THREADS), 0, st, se);
+    const long long hist_res = (long long)sm_count() * hist_per_sm[local ? 1 : 0], scan_res = (long long)sm_count() * scan_per_sm;
+    const dim3 hist_grid((unsigned)(hist_units < hist_res ? hist_units : hist_res));
+    if (local) SOL_LAUNCH("token_hist", token_hist_kernel<true>, hist_grid, dim3(TS_THREADS), 0, st, se);
+    else SOL_LAUNCH("token_hist", token_hist_kernel<false>, hist_grid, dim3(TS_THREADS), 0, st, se);
+    if (Tmax > TH_SEG) {  // shorter rows are taken through the whole selection by token_hist
+      SOL_LAUNCH("token_scan", token_scan_kernel, dim3((unsigned)(scan_units < scan_res ? scan_units : scan_res)),
+                 dim3(TS_THREADS), 0, st, se);
+      SOL_LAUNCH("token_settle", token_settle_kernel, dim3(Hkv, a.B), dim3(TS_THREADS), 0, st, se);
+    }
   }
   if (a.kept_idx_out != nullptr) {
     ListDev ld;
