@@ -116,7 +116,8 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
   // batch, and the length of the pass-2 work items in chunks of split_len kept tokens: the smallest run
   // length (up to ATTN_ITEM_CHUNKS) that gives every resident CTA of pass 2 at most one item, so that there
   // is no second, partly filled round of items; when even the longest runs leave more items than CTAs there
-  // is work for many rounds, and runs of 8 chunks, claimed one by one, balance it.
+  // is work for many rounds, and runs of ATTN_ITEM_CHUNKS / 2 chunks (a few dozen batches per warp, enough to
+  // amortise filling a warp's ring of row copies), claimed one by one, balance it.
   if (kvh == 0 && b == 0) {
     __shared__ int wsum[PLAN_LISTS][PREP_THREADS / 32];
     __shared__ int n_items[ATTN_ITEM_CHUNKS];
@@ -162,7 +163,7 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
     }
     __syncthreads();
     if (tid == 0) {
-      int cpi = 8;
+      int cpi = ATTN_ITEM_CHUNKS / 2;
       for (int c = ATTN_ITEM_CHUNKS; c >= 1; --c)
         if ((long long)n_items[c - 1] * Hkv <= p.target_items) cpi = c;
       p.work_ctr[WC_CPI] = cpi;
@@ -1162,9 +1163,8 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
   using C = GatherCfg<HD, GMAX>;
   constexpr int WARPS = C::WARPS, NST = C::NST, THREADS = C::THREADS;
   constexpr int SPLIT = HD == 64 ? 256 : 128;  // kept tokens per chunk (attn_split_len): the unit of the item list
-  constexpr int LPT = HD / 4;                  // lanes per row
-  constexpr int TPS = 32 / LPT;                // rows per warp-wide read
   constexpr int CPR = HD / 8;                  // 16-byte pieces per row
+  constexpr int NT = HD / 8;                   // n-tiles (8 dims each) of the output
   extern __shared__ __align__(128) unsigned char gsm[];
   unsigned char* ring = gsm;
   int2* s_tab = reinterpret_cast<int2*>(gsm + C::RING_BYTES);                       // [WARPS][NST + 1][32] (cache row, token)
@@ -1176,7 +1176,7 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.G, Hkv = p.Hkv;
   const uint16_t* vp = static_cast<const uint16_t*>(p.kv.v_pool);
-  const int sub = lane / LPT, col = (lane % LPT) * 4;  // which row of a read step, which four columns
+  const int g = lane >> 2, t = lane & 3;  // row group and column pair of the MMA fragments
   unsigned char* my_ring = ring + (size_t)warp * NST * C::STAGE_BYTES;
   int2* my_tab = s_tab + warp * (NST + 1) * GA_BATCH;
   float* my_w = s_w + warp * GA_BATCH * GMAX;
@@ -1226,7 +1226,10 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
         for (int i = 0; i < CPR; ++i) {
           const int c = i * 32 + lane, r = c / CPR, part = c % CPR;
           const int ridx = tab[r].x;
-          cp_async16(dst0 + c * 16, vp + (size_t)(ridx < 0 ? 0 : ridx) * HD + part * 8, ridx >= 0);
+          // piece `part` of row r sits at piece position part ^ (r & 7): the transposing matrix loads below then
+          // touch every bank once
+          cp_async16(dst0 + r * (HD * 2) + ((part & ~7) | ((part ^ r) & 7)) * 16, vp + (size_t)(ridx < 0 ? 0 : ridx) * HD + part * 8,
+                     ridx >= 0);
         }
       }
       cp_async_commit();  // an empty group keeps the count of groups per step fixed
@@ -1246,14 +1249,19 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
       }
     };
 
-    float mh[GMAX], ls[GMAX], acc[GMAX][4];
+    // Output accumulators of the tensor-core product O[head][dim] += P[head][token] V[token][dim]: the 16 rows of
+    // the m16n8k16 tile are the G heads' weights as bf16 high parts (rows 0..7) and low parts (rows 8..15), so
+    // that the product is exact to 2^-17 of a weight; d[j] is the tile of dims 8 j .. 8 j + 7.
+    float mh[GMAX], ls[GMAX], d[NT][4];
 #pragma unroll
     for (int h = 0; h < GMAX; ++h) {
       mh[h] = -INFINITY;
       ls[h] = 0.f;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) acc[h][c] = 0.f;
     }
+#pragma unroll
+    for (int j = 0; j < NT; ++j)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) d[j][c] = 0.f;
     // prologue: list words of the first NST batches, rows of the first NST - 1, logits of the first
 #pragma unroll
     for (int m = 0; m < NST; ++m) my_tab[(m % (NST + 1)) * GA_BATCH + lane] = load_tab(m);
@@ -1274,6 +1282,7 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
       load_logits(m + 1 < my_nb ? my_tab[((m + 1) % (NST + 1)) * GA_BATCH + lane] : make_int2(-1, 0), x_n);
 
       // ---- softmax weights relative to the running maximum ----
+      float scg = 0.f;  // rescaling of this lane's accumulator rows (head g)
 #pragma unroll
       for (int h = 0; h < GMAX; ++h) {
         const float x = x_c[h] * p.scale_log2;
@@ -1282,35 +1291,42 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
         const float pw = x == -INFINITY ? 0.f : exp2f(x - nm);
         mh[h] = nm;
         ls[h] = ls[h] * sc + pw;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) acc[h][c] *= sc;
+        if (h == g) scg = sc;
         my_w[lane * GMAX + h] = pw;
       }
+#pragma unroll
+      for (int j = 0; j < NT; ++j)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) d[j][c] *= scg;
       cp_async_wait<NST - 1>();  // this lane's pieces of batch m have landed ...
       __syncwarp();              // ... and so have the other lanes'; the weights are in the table
 
-      // ---- weights x rows ----
-      const int nt = min(GA_BATCH, len - (warp + m * WARPS) * GA_BATCH);
-      const unsigned char* st = my_ring + (m % NST) * C::STAGE_BYTES;
-#pragma unroll 4
-      for (int k0 = 0; k0 < GA_BATCH; k0 += TPS) {
-        if (k0 >= nt) break;
-        const int r = k0 + sub;  // rows past the batch's end were filled with zeros and weigh nothing
-        const uint2 v = *reinterpret_cast<const uint2*>(st + (size_t)r * HD * 2 + col * 2);
-        const float* w = my_w + r * GMAX;
-        const float f0 = __uint_as_float(v.x << 16), f1 = __uint_as_float(v.x & 0xffff0000u);
-        const float f2 = __uint_as_float(v.y << 16), f3 = __uint_as_float(v.y & 0xffff0000u);
+      // ---- weights x rows on the tensor cores ----
+      const uint32_t st = smem_u32(my_ring + (m % NST) * C::STAGE_BYTES);
 #pragma unroll
-        for (int h4 = 0; h4 < GMAX; h4 += 4) {
-          const float4 w4 = *reinterpret_cast<const float4*>(w + h4);
-          const float ww[4] = {w4.x, w4.y, w4.z, w4.w};
+      for (int ks = 0; ks < GA_BATCH / 16; ++ks) {
+        // A fragment: head g's weights of tokens 2t, 2t+1, 2t+8, 2t+9 of this 16-token step, high and low parts
+        float w0 = 0.f, w1 = 0.f, w2 = 0.f, w3 = 0.f;
+        if (g < GMAX) {
+          const float* wt = my_w + (ks * 16 + 2 * t) * GMAX + g;
+          w0 = wt[0];
+          w1 = wt[GMAX];
+          w2 = wt[8 * GMAX];
+          w3 = wt[9 * GMAX];
+        }
+        const uint16_t h0 = f2bf(w0), h1 = f2bf(w1), h2 = f2bf(w2), h3 = f2bf(w3);
+        const uint32_t a0 = (uint32_t)h0 | ((uint32_t)h1 << 16), a2 = (uint32_t)h2 | ((uint32_t)h3 << 16);
+        const uint32_t a1 = pack_bf16(w0 - bf2f(h0), w1 - bf2f(h1)), a3 = pack_bf16(w2 - bf2f(h2), w3 - bf2f(h3));
+        // B fragments: lanes 0-7 / 8-15 address tokens 0-7 / 8-15 of the step for dims 8 j, lanes 16-31 the same for 8 (j + 1)
+        const int tok = ks * 16 + (lane & 15);
+        const uint32_t row_addr = st + tok * (HD * 2);
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            acc[h4 + e][0] = fmaf(ww[e], f0, acc[h4 + e][0]);
-            acc[h4 + e][1] = fmaf(ww[e], f1, acc[h4 + e][1]);
-            acc[h4 + e][2] = fmaf(ww[e], f2, acc[h4 + e][2]);
-            acc[h4 + e][3] = fmaf(ww[e], f3, acc[h4 + e][3]);
-          }
+        for (int j = 0; j < NT; j += 2) {
+          const int piece = j + (lane >> 4);
+          uint32_t bfr[4];
+          ldsm_x4_trans(bfr, row_addr + ((piece & ~7) | ((piece ^ tok) & 7)) * 16);
+          mma_bf16(d[j], a0, a1, a2, a3, bfr[0], bfr[1]);
+          mma_bf16(d[j + 1], a0, a1, a2, a3, bfr[2], bfr[3]);
         }
       }
       __syncwarp();  // the weights and the ring slot are rewritten by the next steps
@@ -1320,19 +1336,14 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
     cp_async_wait<0>();
 
     // ---- one partial per item: merge the warps ----
-    if (TPS == 2) {  // two rows per read step: the half-warps hold partial sums of the same columns
-#pragma unroll
-      for (int h = 0; h < GMAX; ++h)
-#pragma unroll
-        for (int c = 0; c < 4; ++c) acc[h][c] += __shfl_xor_sync(0xffffffffu, acc[h][c], 16);
-    }
 #pragma unroll
     for (int h = 0; h < GMAX; ++h) ls[h] = warp_sum(ls[h]);
     __syncthreads();  // every warp is done with its ring: the merge scratch lies over it
-    if (sub == 0) {
+    if (g < GMAX) {   // rows g (high parts) and g + 8 (low parts) of the tile belong to head g
 #pragma unroll
-      for (int h = 0; h < GMAX; ++h)
-        *reinterpret_cast<float4*>(&sc_acc[(warp * GMAX + h) * HD + col]) = make_float4(acc[h][0], acc[h][1], acc[h][2], acc[h][3]);
+      for (int j = 0; j < NT; ++j)
+        *reinterpret_cast<float2*>(&sc_acc[(warp * GMAX + g) * HD + j * 8 + 2 * t]) =
+            make_float2(d[j][0] + d[j][2], d[j][1] + d[j][3]);
     }
     if (lane == 0) {
 #pragma unroll

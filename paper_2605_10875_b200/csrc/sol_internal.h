@@ -123,7 +123,7 @@ inline int attn_select_segs(int max_pages, int page_size) {
   const int s = (max_pages * page_size + 2047) / 2048;
   return s < 1 ? 1 : s;
 }
-constexpr int ATTN_ITEM_CHUNKS = 16;  // chunks of attn_split_len kept tokens per pass-2 work item at most
+constexpr int ATTN_ITEM_CHUNKS = 64;  // chunks of attn_split_len kept tokens per pass-2 work item at most
 struct AttnArgs {
   sol_shape_t shape;
   sol_kv_t kv;
