@@ -87,7 +87,7 @@ struct PrepDev {
   int nseg_max;
   int32_t* plan;      // written here by the first CTA: [PLAN_LISTS][PLAN_STRIDE]
   const int32_t* r_permille;
-  int split_len, target_items;  // for the choice of the pass-2 item length
+  int split_len, target_items, max_item_chunks;  // for the choice of the pass-2 item length
   int* status;
 };
 
@@ -113,11 +113,11 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
   pdl_wait();
 
   // The first CTA lays out the work of the kernels that follow: cumulative page and segment counts over the
-  // batch, and the length of the pass-2 work items in chunks of split_len kept tokens: the smallest run
-  // length (up to ATTN_ITEM_CHUNKS) that gives every resident CTA of pass 2 at most one item, so that there
-  // is no second, partly filled round of items; when even the longest runs leave more items than CTAs there
-  // is work for many rounds, and runs of ATTN_ITEM_CHUNKS / 2 chunks (a few dozen batches per warp, enough to
-  // amortise filling a warp's ring of row copies), claimed one by one, balance it.
+  // batch, and the length of the pass-2 work items in chunks of split_len kept tokens: the smallest power of
+  // two (up to 1024 tokens) that gives every resident warp of pass 2 at most one item, so that there is no
+  // second, partly filled round of items; when even the longest runs leave more items than warps there is
+  // work for many rounds, and runs of 1024 tokens (32 batches, enough to amortise filling a warp's ring of
+  // row copies), claimed one by one, balance it.
   if (kvh == 0 && b == 0) {
     __shared__ int wsum[PLAN_LISTS][PREP_THREADS / 32];
     __shared__ int n_items[ATTN_ITEM_CHUNKS];
@@ -156,16 +156,15 @@ __global__ void __launch_bounds__(PREP_THREADS) attn_prep_kernel(const PrepDev p
       if (tid < p.B) p.plan[q * PLAN_STRIDE + tid + 1] = before + incl[q];
       if (tid == 0) p.plan[q * PLAN_STRIDE] = 0;
     }
-#pragma unroll
-    for (int c = 1; c <= ATTN_ITEM_CHUNKS; ++c) {
+    for (int c = 1, q = 0; c <= p.max_item_chunks; c <<= 1, ++q) {
       const int n = __reduce_add_sync(0xffffffffu, tid < p.B ? (ch + c - 1) / c : 0);
-      if (l == 0) atomicAdd(&n_items[c - 1], n);
+      if (l == 0) atomicAdd(&n_items[q], n);
     }
     __syncthreads();
     if (tid == 0) {
-      int cpi = ATTN_ITEM_CHUNKS / 2;
-      for (int c = ATTN_ITEM_CHUNKS; c >= 1; --c)
-        if ((long long)n_items[c - 1] * Hkv <= p.target_items) cpi = c;
+      int cpi = p.max_item_chunks;
+      for (int c = p.max_item_chunks, q = 31 - __clz(p.max_item_chunks); c >= 1; c >>= 1, --q)
+        if ((long long)n_items[q] * Hkv <= p.target_items) cpi = c;
       p.work_ctr[WC_CPI] = cpi;
     }
   }
@@ -1133,17 +1132,16 @@ __device__ __forceinline__ void cp_async_wait() {
 // fetches are in flight, so the rows travel by asynchronous 16-byte copies into per-warp rings of shared
 // memory (about 190 KB per SM, three quarters of it in flight) and the registers only hold accumulators.
 //
-// One persistent CTA per SM works through the list of items: (sequence, kv-head, run of at most
-// ATTN_ITEM_CHUNKS chunks of kept tokens); a CTA's first item is dealt by its index, the later ones are
-// claimed from a counter one item ahead.  The warps of a CTA take the item's tokens in batches of 32, each
-// warp on its own, NST batches deep:
+// The warps of one persistent CTA per SM work through the list of items, each warp on its own: an item is
+// (sequence, kv-head, run of kept tokens, at most 1024); a warp's first item is dealt by its index, the
+// later ones are claimed from a counter one item ahead.  A warp takes its item in batches of 32 tokens, NST
+// batches deep:
 //   lane l fetches the list words of token l of a batch (cache row, token index) two steps before the
 //   batch's rows are requested and its G logits one step before they are used; when a batch's rows have
 //   landed the warp updates its running maximum per head, every lane computes its token's softmax weights,
-//   and the warp walks over the rows: a row is read by HD/4 lanes (8 bytes each) and multiplied into the
-//   lane's float32 accumulators (G heads x 4 columns).
-// Per item one partial (accumulators, maximum, sum; merged over the warps) is written; the CTA that
-// finishes the last item of a (sequence, kv-head) merges its partials.
+//   and the weights (as bf16 high and low parts) multiply the rows on the tensor cores.
+// A row of one item goes straight to the output; otherwise one partial per item (accumulators, maximum,
+// sum) is written and the warp that finishes the last item of a (sequence, kv-head) merges the partials.
 template <int HD, int GMAX>
 struct GatherCfg {
   static constexpr int WARPS = HD == 64 ? 12 : 8;
@@ -1153,27 +1151,22 @@ struct GatherCfg {
   static constexpr int RING_BYTES = WARPS * NST * STAGE_BYTES;  // 192 KB
   static constexpr int TAB_BYTES = WARPS * (NST + 1) * GA_BATCH * 8;
   static constexpr int W_BYTES = WARPS * GA_BATCH * GMAX * 4;
-  static constexpr int ML_BYTES = WARPS * GMAX * 2 * 4;
-  static constexpr int SMEM = RING_BYTES + TAB_BYTES + W_BYTES + ML_BYTES + 64;
-  static_assert(WARPS * GMAX * HD * 4 <= RING_BYTES, "the merge scratch fits the ring");
+  static constexpr int SMEM = RING_BYTES + TAB_BYTES + W_BYTES;
 };
 
 template <int HD, int GMAX>
 __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_kernel(const GatherDev p) {
   using C = GatherCfg<HD, GMAX>;
-  constexpr int WARPS = C::WARPS, NST = C::NST, THREADS = C::THREADS;
+  constexpr int WARPS = C::WARPS, NST = C::NST;
   constexpr int SPLIT = HD == 64 ? 256 : 128;  // kept tokens per chunk (attn_split_len): the unit of the item list
   constexpr int CPR = HD / 8;                  // 16-byte pieces per row
   constexpr int NT = HD / 8;                   // n-tiles (8 dims each) of the output
   extern __shared__ __align__(128) unsigned char gsm[];
   unsigned char* ring = gsm;
-  int2* s_tab = reinterpret_cast<int2*>(gsm + C::RING_BYTES);                       // [WARPS][NST + 1][32] (cache row, token)
-  float* s_w = reinterpret_cast<float*>(gsm + C::RING_BYTES + C::TAB_BYTES);        // [WARPS][32][GMAX]
-  float* sc_ml = reinterpret_cast<float*>(gsm + C::RING_BYTES + C::TAB_BYTES + C::W_BYTES);  // [WARPS][GMAX][2]
-  int* hdr = reinterpret_cast<int*>(gsm + C::RING_BYTES + C::TAB_BYTES + C::W_BYTES + C::ML_BYTES);  // [2][4], then the flag
-  float* sc_acc = reinterpret_cast<float*>(ring);  // [WARPS][GMAX][HD], after an item's batches are done
+  int2* s_tab = reinterpret_cast<int2*>(gsm + C::RING_BYTES);                 // [WARPS][NST + 1][32] (cache row, token)
+  float* s_w = reinterpret_cast<float*>(gsm + C::RING_BYTES + C::TAB_BYTES);  // [WARPS][32][GMAX]
 
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.G, Hkv = p.Hkv;
   const uint16_t* vp = static_cast<const uint16_t*>(p.kv.v_pool);
   const int g = lane >> 2, t = lane & 3;  // row group and column pair of the MMA fragments
@@ -1184,42 +1177,44 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
   pdl_wait();
   const int cpi = p.work_ctr[WC_CPI];
   const int n_items = p.work_ctr[WC_ITEMS];
-  auto header_of = [&](int2 w) {
-    const int bk = w.x / p.S, n0 = (w.x % p.S) * SPLIT;
-    return make_int4(bk, n0, max(0, min(w.y - n0, cpi * SPLIT)), w.y);
-  };
-  if (tid == 0) {
+  const int total_warps = gridDim.x * WARPS;
+  // an item's header: (sequence, kv-head) or -1, first token of the run, tokens of the run, kept count of the row
+  auto header_of = [&](int item) {
     int4 h = make_int4(-1, 0, 0, 0);
-    if ((int)blockIdx.x < n_items) h = header_of(*reinterpret_cast<const int2*>(p.work_items + 2 * blockIdx.x));
-    *reinterpret_cast<int4*>(hdr) = h;
-  }
-  __syncthreads();
+    if (item < n_items) {
+      const int2 w = *reinterpret_cast<const int2*>(p.work_items + 2 * item);
+      const int n0 = (w.x % p.S) * SPLIT;
+      h = make_int4(w.x / p.S, n0, max(0, min(w.y - n0, cpi * SPLIT)), w.y);
+    }
+    return h;
+  };
+  int4 cur = header_of(blockIdx.x * WARPS + warp);  // warp-uniform
 
 #pragma unroll 1
-  for (int it = 0;; ++it) {
-    const int4 cur = *reinterpret_cast<const int4*>(hdr + 4 * (it & 1));
-    if (cur.x < 0) break;
+  while (cur.x >= 0) {
+    // the next item is claimed now and its header fetched while this one is worked on
     int claimed = 0;
-    if (tid == 0) claimed = (int)gridDim.x + atomicAdd(p.work_ctr + WC_NEXT, 1);
+    if (lane == 0) claimed = total_warps + atomicAdd(p.work_ctr + WC_NEXT, 1);
+    claimed = __shfl_sync(0xffffffffu, claimed, 0);
+    const int4 nxt = header_of(claimed);
     const int bk = cur.x, len = cur.z, cnt = cur.w;
     const int b = bk / Hkv, kvh = bk % Hkv;
     const size_t row = (size_t)bk * p.Tmax;
     const uint32_t* krow = p.kept_row + row + cur.y;
     const int32_t* kidx = p.kept_idx + row + cur.y;
     const float* lgrow = p.logits + row * G;
-    const int nb = (len + GA_BATCH - 1) / GA_BATCH;       // batches of the item
-    const int my_nb = nb > warp ? (nb - warp + WARPS - 1) / WARPS : 0;  // this warp's: warp, warp + WARPS, ...
+    const int nb = (len + GA_BATCH - 1) / GA_BATCH;  // batches of the item
 
-    // list words of this warp's m-th batch: lane l holds token l
+    // list words of the item's m-th batch: lane l holds token l
     auto load_tab = [&](int m) {
       int2 e = make_int2(-1, 0);
-      const int n = (warp + m * WARPS) * GA_BATCH + lane;
-      if (m < my_nb && n < len) e = make_int2((int)krow[n], kidx[n]);
+      const int n = m * GA_BATCH + lane;
+      if (n < len) e = make_int2((int)krow[n], kidx[n]);
       return e;
     };
     // requests the rows of the m-th batch (its list words are in the table) into ring slot m % NST
     auto request_rows = [&](int m) {
-      if (m < my_nb) {
+      if (m < nb) {
         const int2* tab = my_tab + (m % (NST + 1)) * GA_BATCH;
         const uint32_t dst0 = smem_u32(my_ring + (m % NST) * C::STAGE_BYTES);
 #pragma unroll
@@ -1273,13 +1268,13 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
     load_logits(my_tab[lane], x_c);
 
 #pragma unroll 1
-    for (int m = 0; m < my_nb; ++m) {
+    for (int m = 0; m < nb; ++m) {
       // the table slot of batch m - 1 is free now: batch m + NST moves in; rows of batch m + NST - 1 are requested
       my_tab[((m + NST) % (NST + 1)) * GA_BATCH + lane] = e_far;
       request_rows(m + NST - 1);
       e_far = load_tab(m + NST + 1);
       float x_n[GMAX];
-      load_logits(m + 1 < my_nb ? my_tab[((m + 1) % (NST + 1)) * GA_BATCH + lane] : make_int2(-1, 0), x_n);
+      load_logits(m + 1 < nb ? my_tab[((m + 1) % (NST + 1)) * GA_BATCH + lane] : make_int2(-1, 0), x_n);
 
       // ---- softmax weights relative to the running maximum ----
       float scg = 0.f;  // rescaling of this lane's accumulator rows (head g)
@@ -1335,89 +1330,103 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
     }
     cp_async_wait<0>();
 
-    // ---- one partial per item: merge the warps ----
+    // ---- the item's result: this lane holds head g's dims 8 j + 2 t, + 1 (rows g and g + 8 of the tile) ----
 #pragma unroll
     for (int h = 0; h < GMAX; ++h) ls[h] = warp_sum(ls[h]);
-    __syncthreads();  // every warp is done with its ring: the merge scratch lies over it
-    if (g < GMAX) {   // rows g (high parts) and g + 8 (low parts) of the tile belong to head g
+    float m_g = -INFINITY, l_g = 0.f;
 #pragma unroll
-      for (int j = 0; j < NT; ++j)
-        *reinterpret_cast<float2*>(&sc_acc[(warp * GMAX + g) * HD + j * 8 + 2 * t]) =
-            make_float2(d[j][0] + d[j][2], d[j][1] + d[j][3]);
-    }
-    if (lane == 0) {
-#pragma unroll
-      for (int h = 0; h < GMAX; ++h) {
-        sc_ml[(warp * GMAX + h) * 2] = mh[h];
-        sc_ml[(warp * GMAX + h) * 2 + 1] = ls[h];
+    for (int h = 0; h < GMAX; ++h) {
+      if (h == g) {
+        m_g = mh[h];
+        l_g = ls[h];
       }
     }
-    // the header of the claimed item is fetched while the partial is put together
-    int2 claimed_words = make_int2(0, 0);
-    if (tid == 0 && claimed < n_items) claimed_words = *reinterpret_cast<const int2*>(p.work_items + 2 * claimed);
-    __syncthreads();
-    const int slot_no = (cur.y / SPLIT) / cpi;  // this item's partial
-    float* dst = p.part + (((size_t)bk * p.S + slot_no) * G) * (HD + 2);
-    for (int e0 = tid; e0 < G * HD; e0 += THREADS) {
-      const int h = e0 / HD, e = e0 % HD;
-      float M = -INFINITY;
-#pragma unroll
-      for (int w = 0; w < WARPS; ++w) M = fmaxf(M, sc_ml[(w * GMAX + h) * 2]);
-      float a = 0.f, l = 0.f;
-#pragma unroll
-      for (int w = 0; w < WARPS; ++w) {
-        const float mw = sc_ml[(w * GMAX + h) * 2];
-        const float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
-        a += sc_acc[(w * GMAX + h) * HD + e] * f;
-        l += sc_ml[(w * GMAX + h) * 2 + 1] * f;
-      }
-      dst[h * (HD + 2) + e] = a;
-      if (e == 0) {
-        dst[h * (HD + 2) + HD] = M;
-        dst[h * (HD + 2) + HD + 1] = l;
-      }
-    }
-
-    // ---- the last item of this (sequence, kv-head) merges the partials ----
     const int chunks = max(1, (cnt + SPLIT - 1) / SPLIT);
-    const int ns = (chunks + cpi - 1) / cpi;
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-      hdr[8] = atomicAdd(p.work_ctr + WC_DONE + bk, 1) == ns - 1 ? 1 : 0;
-      int4 h = make_int4(-1, 0, 0, 0);
-      if (claimed < n_items) h = header_of(claimed_words);
-      *reinterpret_cast<int4*>(hdr + 4 * ((it + 1) & 1)) = h;
-    }
-    __syncthreads();
-    if (hdr[8]) {
-      __threadfence();
-      const float* src0 = p.part + ((size_t)bk * p.S * G) * (HD + 2);
-      for (int e0 = tid; e0 < G * HD; e0 += THREADS) {
-        const int h = e0 / HD, e = e0 % HD;
-        float m = -INFINITY, l = 0.f, a = 0.f;
-        for (int q = 0; q < ns; ++q) {
-          const float* src = src0 + ((size_t)q * G + h) * (HD + 2);
-          const float m2 = __ldcg(src + HD), l2 = __ldcg(src + HD + 1), a2 = __ldcg(src + e);
-          const float mn = fmaxf(m, m2);
-          const float e1 = (m == -INFINITY) ? 0.f : exp2f(m - mn);
-          const float e2 = (m2 == -INFINITY) ? 0.f : exp2f(m2 - mn);
-          l = l * e1 + l2 * e2;
-          a = a * e1 + a2 * e2;
-          m = mn;
+    const int ns = (chunks + cpi - 1) / cpi;  // items of this (sequence, kv-head)
+    auto write_out = [&](int h, int e, float o0, float o1) {
+      const size_t idx = ((size_t)b * p.Hq + kvh * G + h) * HD + e;
+      if (p.out_f32) *reinterpret_cast<float2*>(p.out_f32 + idx) = make_float2(o0, o1);
+      if (p.out_bf16) *reinterpret_cast<uint32_t*>(p.out_bf16 + idx) = pack_bf16(o0, o1);
+      if (p.out_hi) {
+        const uint16_t h0 = f2bf(o0), h1 = f2bf(o1);
+        *reinterpret_cast<uint32_t*>(p.out_hi + idx) = (uint32_t)h0 | ((uint32_t)h1 << 16);
+        *reinterpret_cast<uint32_t*>(p.out_lo + idx) = pack_bf16(o0 - bf2f(h0), o1 - bf2f(h1));
+      }
+    };
+    if (ns == 1) {  // the row is this one item: its output goes out directly
+      if (g < G) {
+        const float inv = l_g > 0.f ? 1.0f / l_g : 0.f;
+#pragma unroll
+        for (int j = 0; j < NT; ++j) write_out(g, j * 8 + 2 * t, (d[j][0] + d[j][2]) * inv, (d[j][1] + d[j][3]) * inv);
+      }
+    } else {
+      const int slot_no = (cur.y / SPLIT) / cpi;  // this item's partial
+      float* dst = p.part + (((size_t)bk * p.S + slot_no) * G) * (HD + 2);
+      if (g < G) {
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+          *reinterpret_cast<float2*>(dst + g * (HD + 2) + j * 8 + 2 * t) = make_float2(d[j][0] + d[j][2], d[j][1] + d[j][3]);
+        if (t == 0) {
+          dst[g * (HD + 2) + HD] = m_g;
+          dst[g * (HD + 2) + HD + 1] = l_g;
         }
-        const float o = l > 0.f ? a / l : 0.f;
-        const size_t idx = ((size_t)b * p.Hq + kvh * G + h) * HD + e;
-        if (p.out_f32) p.out_f32[idx] = o;
-        if (p.out_bf16) p.out_bf16[idx] = f2bf(o);
-        if (p.out_hi) {
-          const uint16_t hi = f2bf(o);
-          p.out_hi[idx] = hi;
-          p.out_lo[idx] = f2bf(o - bf2f(hi));
+      }
+      // ---- the last item of this (sequence, kv-head) merges the partials ----
+      __threadfence();
+      __syncwarp();
+      int last = 0;
+      if (lane == 0) last = atomicAdd(p.work_ctr + WC_DONE + bk, 1) == ns - 1 ? 1 : 0;
+      last = __shfl_sync(0xffffffffu, last, 0);
+      if (last) {
+        __threadfence();
+        const float* src0 = p.part + ((size_t)bk * p.S * G) * (HD + 2);
+        // factors of the partials: f[q][h] = 2^(m_q - M_h) / sum_q l_q 2^(m_q - M_h), in the warp's (idle) ring
+        float* fac = reinterpret_cast<float*>(my_ring);
+        for (int h = 0; h < G; ++h) {
+          float mm = -INFINITY;
+          for (int q = lane; q < ns; q += 32) mm = fmaxf(mm, __ldcg(src0 + ((size_t)q * G + h) * (HD + 2) + HD));
+          mm = warp_max(mm);
+          float l = 0.f;
+          for (int q = lane; q < ns; q += 32) {
+            const float* src = src0 + ((size_t)q * G + h) * (HD + 2);
+            const float m2 = __ldcg(src + HD);
+            const float f = m2 == -INFINITY ? 0.f : exp2f(m2 - mm);
+            fac[q * GMAX + h] = f;
+            l += __ldcg(src + HD + 1) * f;
+          }
+          l = warp_sum(l);
+          const float inv = l > 0.f ? 1.0f / l : 0.f;
+          for (int q = lane; q < ns; q += 32) fac[q * GMAX + h] *= inv;
+        }
+        __syncwarp();
+        for (int e0 = lane * 2; e0 < G * HD; e0 += 64) {
+          const int h = e0 / HD, e = e0 % HD;
+          const float* src = src0 + (size_t)h * (HD + 2) + e;
+          float a0 = 0.f, a1 = 0.f;
+          int q = 0;
+          for (; q + 8 <= ns; q += 8) {  // eight partials' loads in flight
+            float2 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = __ldcg(reinterpret_cast<const float2*>(src + (size_t)(q + u) * G * (HD + 2)));
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const float f = fac[(q + u) * GMAX + h];
+              a0 = fmaf(v[u].x, f, a0);
+              a1 = fmaf(v[u].y, f, a1);
+            }
+          }
+          for (; q < ns; ++q) {
+            const float2 v = __ldcg(reinterpret_cast<const float2*>(src + (size_t)q * G * (HD + 2)));
+            const float f = fac[q * GMAX + h];
+            a0 = fmaf(v.x, f, a0);
+            a1 = fmaf(v.y, f, a1);
+          }
+          write_out(h, e, a0, a1);
         }
       }
     }
-    __syncthreads();  // the merge scratch, the flag and the headers are reused by the next item
+    __syncwarp();
+    cur = nxt;
   }
 }
 
@@ -1459,7 +1468,8 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   pd.row_hist = a.row_hist; pd.row_ctl = a.row_ctl; pd.seg_pub = a.seg_pub;
   pd.nseg_max = attn_select_segs(a.kv.max_pages_per_seq, PAGE);
   pd.plan = a.plan; pd.r_permille = a.r_permille; pd.split_len = attn_split_len(hd);
-  pd.target_items = sm_count();  // the pass-2 CTAs resident at once
+  pd.target_items = sm_count() * (hd == 64 ? 12 : 8) / 4;  // a quarter of the pass-2 warps resident at once: few partials per row
+  pd.max_item_chunks = 1024 / attn_split_len(hd);
   SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(Hkv, a.B), dim3(PREP_THREADS), 0, st, pd);
 
   ScoreDev sd;

@@ -70,6 +70,59 @@ struct NormQuantArgs {
 };
 void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st);
 
+// ---- packed operand layouts ---------------------------------------------------
+// Every tensor-core operand is stored the way the MMA reads it from shared memory, so that a stage of the
+// GEMM pipelines is one or two large contiguous bulk copies: 64-wide k chunks of rows, each row 128 bytes
+// whose 16-byte pieces are permuted by (piece ^ (row & 7)) (the 128-byte swizzle of the K-major operand
+// layout).
+//   weights [N][K]      -> [tile][chunk][R rows][128 B]; the gate and up matrices share one packed matrix whose
+//                          rows alternate gate_c, up_c (so a channel's two sums sit in neighbouring
+//                          accumulator lanes)
+//   W_down_t [ff][d]    -> [128-column slab][64-channel block][2 column halves][64 channels][128 B] (the
+//                          MN-major operand)
+//   activations [M][K]  -> [chunk][n_rows][128 B]
+struct NKGeom {
+  int N, K;     // packed rows in all (gate/up: 2 ff), contraction length
+  int R;        // rows per tile (a multiple of 8, at most 128)
+  int tiles, chunks;
+};
+inline NKGeom nk_geom_plain(int N, int K) {
+  NKGeom g;
+  g.N = N;
+  g.K = K;
+  g.R = N >= 128 ? 128 : (N + 7) / 8 * 8;
+  g.tiles = (N + g.R - 1) / g.R;
+  g.chunks = K / 64;
+  return g;
+}
+// channels per tile: the fewest waves of CTAs that keep a tile within 64 channels (128 accumulator lanes)
+inline NKGeom nk_geom_gate_up(int ff, int K, int sms) {
+  int c = 64;
+  for (int w = 1; w <= 64; ++w) {
+    c = ((ff + sms * w - 1) / (sms * w) + 3) / 4 * 4;
+    if (c <= 64) break;
+  }
+  NKGeom g;
+  g.N = 2 * ff;
+  g.K = K;
+  g.R = 2 * c;
+  g.tiles = (ff + c - 1) / c;
+  g.chunks = K / 64;
+  return g;
+}
+inline size_t nk_packed_bytes(const NKGeom& g) { return (size_t)g.tiles * g.chunks * g.R * 128; }
+inline size_t down_packed_bytes(int ff, int d) { return (size_t)(d / 128) * ((ff + 63) / 64) * 16384; }
+// byte offset of 16-byte piece q (elements 8 q .. 8 q + 7 of a chunk) of packed row n in chunk `chunk`
+__host__ __device__ inline size_t nk_piece_offset(int R, int chunks, int n, int chunk, int q) {
+  const int r = n % R;
+  return (((size_t)(n / R) * chunks + chunk) * R + r) * 128 + (size_t)((q ^ (r & 7)) * 16);
+}
+// byte offset of the piece that holds elements 8 kp .. 8 kp + 7 of row m of a packed activation operand
+__host__ __device__ inline size_t act_piece_offset(int n_rows, int m, int kp) {
+  return ((size_t)(kp >> 3) * n_rows + m) * 128 + (size_t)(((kp & 7) ^ (m & 7)) * 16);
+}
+int pad_rows(int B);  // rows of an activation operand block: the batch padded to 16, 32, 64 or 128
+
 // ---- weight-streaming GEMMs (sol_gemm.cu) ----------------------------------
 // EPI_PARTIAL: split-K; out0 is [ksplit][M][N] raw partial sums (no scale, no residual), summed by the
 // consumer kernel.  EPI_SWIGLU: whole K per CTA; g, u and t = silu(g) u with the row scale applied.
@@ -79,10 +132,9 @@ constexpr int NK_MAX_KSPLIT = 16;
 int nk_ksplit(int N, int K);
 struct GemmNK {
   const char* name;       // kernel name for the per-kernel timing table
-  const void* a_hi;       // bf16 [Mpad][K]
-  const void* a_lo;       // bf16 [Mpad][K] or nullptr; the product uses a_hi + a_lo
-  const void* w0;         // bf16 [N][K]   (EPI_SWIGLU: gate [ff][K])
-  const void* w1;         // EPI_SWIGLU: up [ff][K]
+  const void* a;          // packed activation operand, n_b * Mpad rows (high rows, then low rows when n_b == 2)
+  int n_b;                // 1, or 2: the product uses the sum of the two row blocks
+  const void* w;          // packed weights (EPI_SWIGLU: the gate/up matrix)
   int M, K, N;            // EPI_SWIGLU: N = ff
   const float* row_scale; // EPI_SWIGLU: [M] or nullptr
   float* out0;            // EPI_PARTIAL: [ksplit][M][N]; EPI_SWIGLU: g [M][N]
@@ -94,9 +146,8 @@ struct GemmNK {
 void launch_gemm_nk(const GemmNK& p, GemmEpilogue epi, cudaStream_t st);
 
 struct GemmDown {
-  const void* t_hi;  // bf16 [Mpad][ff]  masked activations, high part
-  const void* t_lo;  // bf16 [Mpad][ff]  low part
-  const void* w;     // bf16 [ff][d]
+  const void* t;     // packed masked activations: 2 Mpad rows (high parts, then low parts), K = ff
+  const void* w;     // packed W_down_t
   const int32_t* live;  // [ff/32] non-zero if any token keeps a channel of the granule
   int M, ff, d;
   float* partial;    // [chunks][Mpad][d]
@@ -109,6 +160,8 @@ void launch_gemm_down(const GemmDown& p, cudaStream_t st);
 // Also clears the n_live "granule is live" flags, which every reader has finished with by then.
 void launch_reduce_out(const float* partial, int chunks, int M, int Mpad, int d, const void* resid, int resid_f32,
                        void* out_bf16, float* out_f32, float* out_f32_b, int32_t* live, int n_live, cudaStream_t st);
+// One-time packing of a weight matrix (kinds as in sol.h); src1 is the up matrix of the gate/up pair.
+void launch_pack_weights(const sol_shape_t& s, int kind, const void* src0, const void* src1, void* dst, cudaStream_t st);
 
 // ---- attention (sol_attn.cu) ------------------------------------------------
 // Kept tokens per pass-2 chunk: 32 KB of V rows.
