@@ -191,7 +191,7 @@ class Replica:
         self.max_pages, self.n_pages = table.shape[1], n_pages
         self.table = self._i32(np.where(table < 0, 0, table))
         self.lens_dev = [self._i32(self.seq_lens + j) for j in range(self.cycle)]
-        names = ("w_qkv", "w_o", "w_gate", "w_up", "w_down_t", "gamma1", "gamma2")
+        names = ("w_qkv", "w_o", "w_gate_up", "w_down", "gamma1", "gamma2")
         # enough distinct copies of weights + cache that no step finds its inputs in the 126 MB L2; one
         # copy of a multi-GB workload is already far larger than L2
         hkv, hd, d, ff = cfg["n_kv_heads"], cfg["head_dim"], cfg["d_model"], cfg["d_ff"]
@@ -200,7 +200,7 @@ class Replica:
         self.copy_mb = int(copy_bytes / 1e6)
         self.weights, self.kvs, self._keep = [], [], []
         for l in range(self.L):
-            wd = synth.device_layer_weights(cfg, device, seed, l)
+            wd = self._pack(synth.device_layer_weights(cfg, device, seed, l))  # load-time step, untimed
             base_w = [wd[n] for n in names]
             base_kv = list(synth.device_kv_pool(cfg, n_pages, device, seed, l))
             per_copy_w, per_copy_kv = [], []
@@ -224,6 +224,19 @@ class Replica:
         self.h_out_host = torch.zeros((self.B, cfg["d_model"]), dtype=torch.int16).pin_memory()
         self.lens_host = [pin((self.seq_lens + j).astype(np.int32)) for j in range(self.cycle)]
         torch.cuda.synchronize()
+
+    def _pack(self, plain):
+        """The library reads its weights in packed form (sol_pack_weights): done once here, at load time."""
+        sol, t = self.sol, self.torch
+        out = {"gamma1": plain["gamma1"], "gamma2": plain["gamma2"]}
+        for name, kind, a, b in (("w_qkv", sol.W_QKV, "w_qkv", None), ("w_o", sol.W_O, "w_o", None),
+                                 ("w_gate_up", sol.W_GATE_UP, "w_gate", "w_up"), ("w_down", sol.W_DOWN, "w_down_t", None)):
+            n = sol.packed_weight_bytes(self.shape, kind)
+            buf = t.empty(n, dtype=t.uint8, device=self.device)
+            sol.pack_weights(self.shape, kind, plain[a], plain[b] if b else None, buf, n)
+            out[name] = buf
+        t.cuda.synchronize()
+        return out
 
     def _bf16(self, u16):
         t = self.torch

@@ -65,17 +65,36 @@ typedef struct sol_kv {
   int32_t max_pages_per_seq, num_pages;
 } sol_kv_t;
 
-/* bf16 weights of one layer.  w_qkv rows: q heads, then k heads, then v heads.
- * w_down_t is W_down transposed once at load time so that row j is
- * intermediate channel j; a pruned channel is then a row that is not read. */
+/* Weight matrices are PACKED once at load time (sol_pack_weights) into the order the tensor cores read
+ * them, so that the kernels stream each matrix with large contiguous copies.  Kinds and their row-major
+ * bf16 sources:
+ *   SOL_W_QKV      [(n_q+2 n_kv)*head_dim][d_model]   rows: q heads, then k heads, then v heads
+ *   SOL_W_O        [d_model][n_q*head_dim]
+ *   SOL_W_GATE_UP  two matrices [d_ff][d_model] (gate, up), packed into one
+ *   SOL_W_DOWN     W_down transposed, [d_ff][d_model]: row j is intermediate channel j, so a pruned
+ *                  channel is a row that is not read
+ * The packed size depends on the shape and, for SOL_W_GATE_UP, on the SM count of the current device:
+ * pack on the device that runs the layer. */
+#define SOL_W_QKV 0
+#define SOL_W_O 1
+#define SOL_W_GATE_UP 2
+#define SOL_W_DOWN 3
+/* Bytes of the packed form of a matrix; 0 if the shape or kind is unsupported. */
+size_t sol_packed_weight_bytes(const sol_shape_t *shape, int32_t kind);
+/* Packs src0 (and src1: the up matrix when kind is SOL_W_GATE_UP, else NULL) into dst (dst_bytes >=
+ * sol_packed_weight_bytes), all device pointers, 16-byte aligned; enqueued on `stream`.  A pure
+ * permutation of 16-byte pieces (tiles that reach past the matrix are padded with zeros). */
+sol_status_t sol_pack_weights(const sol_shape_t *shape, int32_t kind, const void *src0, const void *src1, void *dst,
+                              size_t dst_bytes, sol_stream_t stream);
+
+/* Packed bf16 weights of one layer (see sol_pack_weights) and the RMSNorm gains. */
 typedef struct sol_layer_weights {
-  const void *w_qkv;    /* [(n_q+2 n_kv)*head_dim][d_model] */
-  const void *w_o;      /* [d_model][n_q*head_dim] */
-  const void *w_gate;   /* [d_ff][d_model] */
-  const void *w_up;     /* [d_ff][d_model] */
-  const void *w_down_t; /* [d_ff][d_model] */
-  const void *gamma1;   /* [d_model] RMSNorm gain before attention */
-  const void *gamma2;   /* [d_model] RMSNorm gain before the MLP */
+  const void *w_qkv;     /* packed SOL_W_QKV */
+  const void *w_o;       /* packed SOL_W_O */
+  const void *w_gate_up; /* packed SOL_W_GATE_UP */
+  const void *w_down;    /* packed SOL_W_DOWN */
+  const void *gamma1;    /* [d_model] RMSNorm gain before attention */
+  const void *gamma2;    /* [d_model] RMSNorm gain before the MLP */
 } sol_layer_weights_t;
 
 /* Optional taps on sol_decode_layer; any pointer may be NULL.  They exist so a
@@ -172,12 +191,13 @@ sol_status_t sol_sparse_decode_attn_static(const sol_shape_t *shape, const void 
  * m = ceil(rho*d), "Per-token channel selection"; the pruned axis is the
  * intermediate one): t_j = silu(W_g x)_j (W_u x)_j, keep the
  * m = ceil((1-p) d_ff) channels with the largest |t_j| (ties: lower index),
- * out = sum over kept j of t_j * w_down_t[j, :].  Rows of w_down_t that no
+ * out = sum over kept j of t_j * W_down[j, :].  Blocks of W_down rows that no
  * token of the batch keeps are not read.
- *   x_bf16 [B][d_model]; out_bf16 [B][d_model] (no residual added);
+ *   x_bf16 [B][d_model]; w_gate_up, w_down: packed SOL_W_GATE_UP / SOL_W_DOWN;
+ *   out_bf16 [B][d_model] (no residual added);
  *   kept_ch (optional) int32 [B][d_ff] ascending; kept_ch_cnt (optional) [B]. */
-sol_status_t sol_pruned_swiglu_mlp(const sol_shape_t *shape, const void *x_bf16, const void *w_gate,
-                                   const void *w_up, const void *w_down_t, int32_t B, const int32_t *p_permille,
+sol_status_t sol_pruned_swiglu_mlp(const sol_shape_t *shape, const void *x_bf16, const void *w_gate_up,
+                                   const void *w_down, int32_t B, const int32_t *p_permille,
                                    void *out_bf16, int32_t *kept_ch, int32_t *kept_ch_cnt, void *ws,
                                    size_t ws_bytes, sol_stream_t stream);
 

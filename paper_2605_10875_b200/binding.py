@@ -23,6 +23,7 @@ SOL_ERR_DEVICE_TIMEOUT = 5
 
 EXPORTS = [
     "sol_status_string", "sol_last_cuda_error", "sol_workspace_bytes", "sol_workspace_init", "sol_quant_act",
+    "sol_packed_weight_bytes", "sol_pack_weights",
     "sol_sparse_decode_attn", "sol_sparse_decode_attn_static", "sol_pruned_swiglu_mlp", "sol_decode_layer", "sol_decode_step",
     "sol_decode_step_traced", "sol_decode_step_host", "sol_read_device_status", "sol_selftest_wait_timeout", "sol_timing_enable", "sol_timing_collect",
     "sol_launch_count",
@@ -41,7 +42,7 @@ class SolKV(C.Structure):
 
 
 class SolLayerWeights(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("w_qkv", "w_o", "w_gate", "w_up", "w_down_t", "gamma1", "gamma2")]
+    _fields_ = [(n, C.c_void_p) for n in ("w_qkv", "w_o", "w_gate_up", "w_down", "gamma1", "gamma2")]
 
 
 TRACE_FIELDS = ("xn1", "codes1", "scales1", "q_rot", "kept_idx", "kept_cnt", "attn_out", "h_mid", "xn2", "codes2",
@@ -89,7 +90,11 @@ def lib() -> C.CDLL:
         L.sol_sparse_decode_attn_static.restype = I
         L.sol_sparse_decode_attn_static.argtypes = [C.POINTER(SolShape), P, C.POINTER(SolKV), I, P, P, P, P, P, P]
         L.sol_pruned_swiglu_mlp.restype = I
-        L.sol_pruned_swiglu_mlp.argtypes = [C.POINTER(SolShape), P, P, P, P, I, P, P, P, P, P, S, P]
+        L.sol_pruned_swiglu_mlp.argtypes = [C.POINTER(SolShape), P, P, P, I, P, P, P, P, P, S, P]
+        L.sol_packed_weight_bytes.restype = S
+        L.sol_packed_weight_bytes.argtypes = [C.POINTER(SolShape), I]
+        L.sol_pack_weights.restype = I
+        L.sol_pack_weights.argtypes = [C.POINTER(SolShape), I, P, P, P, S, P]
         L.sol_decode_layer.restype = I
         L.sol_decode_layer.argtypes = [C.POINTER(SolShape), C.POINTER(SolLayerWeights), C.POINTER(SolKV), I, P, P, P,
                                        P, P, C.POINTER(SolLayerTrace), P, S, P]
@@ -154,8 +159,24 @@ def make_kv(k_pool, v_pool, page_table, seq_lens, max_pages_per_seq: int, num_pa
     return SolKV(_ptr(k_pool), _ptr(v_pool), _ptr(page_table), _ptr(seq_lens), max_pages_per_seq, num_pages)
 
 
-def make_weights(w_qkv, w_o, w_gate, w_up, w_down_t, gamma1, gamma2) -> SolLayerWeights:
-    return SolLayerWeights(*[_ptr(x) for x in (w_qkv, w_o, w_gate, w_up, w_down_t, gamma1, gamma2)])
+W_QKV, W_O, W_GATE_UP, W_DOWN = 0, 1, 2, 3
+
+
+def packed_weight_bytes(shape: SolShape, kind: int) -> int:
+    return int(lib().sol_packed_weight_bytes(C.byref(shape), kind))
+
+
+def pack_weights(shape: SolShape, kind: int, src0, src1, dst, dst_bytes: int, stream=None, check=True) -> int:
+    """One-time packing of a row-major bf16 weight matrix (src1: the up matrix of the gate/up pair)."""
+    s = lib().sol_pack_weights(C.byref(shape), kind, _ptr(src0), _ptr(src1), _ptr(dst), dst_bytes, _stream(stream))
+    if check:
+        _check(s, "sol_pack_weights")
+    return s
+
+
+def make_weights(w_qkv, w_o, w_gate_up, w_down, gamma1, gamma2) -> SolLayerWeights:
+    """The four matrices are the PACKED buffers (pack_weights)."""
+    return SolLayerWeights(*[_ptr(x) for x in (w_qkv, w_o, w_gate_up, w_down, gamma1, gamma2)])
 
 
 def make_trace(**taps) -> SolLayerTrace:
@@ -203,9 +224,9 @@ def sparse_decode_attn_static(shape, q_bf16, kv: SolKV, B: int, r_permille, out_
     return s
 
 
-def pruned_swiglu_mlp(shape, x_bf16, w_gate, w_up, w_down_t, B: int, p_permille, out_bf16, kept_ch, kept_ch_cnt,
+def pruned_swiglu_mlp(shape, x_bf16, w_gate_up, w_down, B: int, p_permille, out_bf16, kept_ch, kept_ch_cnt,
                       ws, ws_bytes: int, stream=None, check=True) -> int:
-    s = lib().sol_pruned_swiglu_mlp(C.byref(shape), _ptr(x_bf16), _ptr(w_gate), _ptr(w_up), _ptr(w_down_t), B,
+    s = lib().sol_pruned_swiglu_mlp(C.byref(shape), _ptr(x_bf16), _ptr(w_gate_up), _ptr(w_down), B,
                                     _ptr(p_permille), _ptr(out_bf16), _ptr(kept_ch), _ptr(kept_ch_cnt), _ptr(ws),
                                     ws_bytes, _stream(stream))
     if check:

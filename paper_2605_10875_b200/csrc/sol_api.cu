@@ -92,11 +92,6 @@ void ensure_dynamic_smem(const void* kernel, int bytes) {
 // ---------------------------------------------------------------------------
 // workspace layout
 // ---------------------------------------------------------------------------
-static int pad_rows(int B) {
-  const int mt = (B + 15) / 16;
-  return 16 * (mt <= 1 ? 1 : (mt <= 2 ? 2 : (mt <= 4 ? 4 : 8)));
-}
-
 struct Layout {
   size_t status, stage_h_in, stage_act, stage_h_out, a_op, scale, qkv, attn_hi, attn_lo, attn_f32, h_mid, o_part, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, ch_sel, ch_cand_val, ch_cand_idx, ch_keep, down_part,
       h_a, h_b, total;
@@ -141,16 +136,17 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   L.qkv = take((size_t)NK_MAX_KSPLIT * B * Nqkv * 4);  // split-K partial sums of the QKV projection
   L.attn = attn_scratch_layout(s, B, max_pages, at);
   at = L.attn.end;
-  L.attn_hi = take(Mpad * Hq * hd * 2);
-  L.attn_lo = take(Mpad * Hq * hd * 2);
+  L.attn_hi = take(2 * Mpad * Hq * hd * 2);  // packed operand: high rows and low rows of every chunk side by side
+  L.attn_lo = take(256);
   L.attn_f32 = take(B * Hq * hd * 4);
   L.h_mid = take(B * d * 4);
   L.o_part = take((size_t)NK_MAX_KSPLIT * B * d * 4);  // split-K partial sums of the output projection
   L.g = take(B * ff * 4);
   L.u = take(B * ff * 4);
   L.t = take(B * ff * 4);
-  L.t_hi = take(Mpad * ff * 2);
-  L.t_lo = take(Mpad * ff * 2);
+  const size_t ffc = (ff + 63) / 64 * 64;  // the packed operand is written in whole 64-channel chunks
+  L.t_hi = take(2 * Mpad * ffc * 2);       // high rows and low rows of every chunk side by side
+  L.t_lo = take(256);
   L.kept_ch = take(B * ff * 4);
   L.kept_ch_cnt = take((size_t)B * 4);
   L.live = take(ff / 32 * 4);
@@ -203,23 +199,24 @@ static void run_attention(const sol_shape_t& s, const Layout& L, void* ws, const
   attn_scratch_bind(a, ws, L.attn, kept_idx, kept_cnt);
   a.out_f32 = out_f32;
   a.out_bf16 = out_bf16;
-  a.out_hi = want_split ? at<void>(ws, L.attn_hi) : nullptr;
-  a.out_lo = want_split ? at<void>(ws, L.attn_lo) : nullptr;
+  a.out_hi = want_split ? at<void>(ws, L.attn_hi) : nullptr;  // packed, high and low parts
+  a.out_lo = nullptr;
+  a.out_rows = L.Mpad;
   a.status = at<int>(ws, L.status);
   launch_attention(a, st);
 }
 
-// a_op / scale in the workspace hold the MLP input operand.
-static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, const void* w_gate, const void* w_up,
-                    const void* w_down_t, const int32_t* p_permille, const void* resid, int resid_f32, void* out_bf16,
+// a_op (packed) / scale in the workspace hold the MLP input operand.
+static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, const void* w_gate_up, const void* w_down,
+                    const int32_t* p_permille, const void* resid, int resid_f32, void* out_bf16,
                     float* out_f32, float* out_f32_b, float* t_trace, int32_t* kept_ch, int32_t* kept_ch_cnt,
                     cudaStream_t st) {
   int* status = at<int>(ws, L.status);
   GemmNK gu;
   memset(&gu, 0, sizeof(gu));
-  gu.a_hi = at<void>(ws, L.a_op);
-  gu.w0 = w_gate;
-  gu.w1 = w_up;
+  gu.a = at<void>(ws, L.a_op);
+  gu.n_b = 1;
+  gu.w = w_gate_up;
   gu.M = B;
   gu.K = s.d_model;
   gu.N = s.d_ff;
@@ -241,8 +238,7 @@ static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, cons
   cs.t = gu.out2;
   cs.a_op = at<void>(ws, L.a_op);
   cs.scale = at<float>(ws, L.scale);
-  cs.w_gate = w_gate;
-  cs.w_up = w_up;
+  cs.w_gate_up = w_gate_up;
   cs.sel = at<uint32_t>(ws, L.ch_sel);
   cs.cand_val = at<double>(ws, L.ch_cand_val);
   cs.cand_idx = at<int32_t>(ws, L.ch_cand_idx);
@@ -250,16 +246,14 @@ static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, cons
   cs.scratch_idx = at<int32_t>(ws, L.kept_ch);
   cs.kept_ch = kept_ch;
   cs.kept_cnt = kept_ch_cnt ? kept_ch_cnt : at<int32_t>(ws, L.kept_ch_cnt);
-  cs.t_hi = at<void>(ws, L.t_hi);
-  cs.t_lo = at<void>(ws, L.t_lo);
+  cs.t_op = at<void>(ws, L.t_hi);
   cs.live = at<int32_t>(ws, L.live);
   cs.status = status;
   launch_channel_select(cs, st);
 
   GemmDown dn;
-  dn.t_hi = cs.t_hi;
-  dn.t_lo = cs.t_lo;
-  dn.w = w_down_t;
+  dn.t = cs.t_op;
+  dn.w = w_down;
   dn.live = cs.live;
   dn.M = B;
   dn.ff = s.d_ff;
@@ -284,7 +278,8 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   NormQuantArgs n1;
   memset(&n1, 0, sizeof(n1));
   n1.in = h_in; n1.in_f32 = in_f32; n1.gamma_bf16 = w.gamma1; n1.eps = s.rms_eps; n1.bits = bits; n1.B = B; n1.d = d;
-  n1.a_op = at<void>(ws, L.a_op); n1.scale = scale; n1.xn = tr ? tr->xn1 : nullptr; n1.codes = tr ? tr->codes1 : nullptr;
+  n1.a_op = at<void>(ws, L.a_op); n1.a_op_rows = L.Mpad; n1.scale = scale; n1.xn = tr ? tr->xn1 : nullptr;
+  n1.codes = tr ? tr->codes1 : nullptr;
   n1.status = status;
   launch_norm_quant(n1, st);
   if (tr && tr->scales1) cudaMemcpyAsync(tr->scales1, scale, sizeof(float) * B, cudaMemcpyDeviceToDevice, st);
@@ -293,8 +288,9 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   GemmNK q;
   memset(&q, 0, sizeof(q));
   q.name = "gemm_qkv";
-  q.a_hi = at<void>(ws, L.a_op);
-  q.w0 = w.w_qkv;
+  q.a = at<void>(ws, L.a_op);
+  q.n_b = 1;
+  q.w = w.w_qkv;
   q.M = B;
   q.K = d;
   q.N = Nqkv;
@@ -311,9 +307,9 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   GemmNK o;
   memset(&o, 0, sizeof(o));
   o.name = "gemm_out_proj";
-  o.a_hi = at<void>(ws, L.attn_hi);
-  o.a_lo = at<void>(ws, L.attn_lo);
-  o.w0 = w.w_o;
+  o.a = at<void>(ws, L.attn_hi);
+  o.n_b = 2;
+  o.w = w.w_o;
   o.M = B;
   o.K = Hq * hd;
   o.N = d;
@@ -326,7 +322,8 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   n2.in = h_in; n2.in_f32 = in_f32; n2.part = at<float>(ws, L.o_part); n2.ksplit = nk_ksplit(d, Hq * hd);
   n2.sum_out = at<float>(ws, L.h_mid);
   n2.gamma_bf16 = w.gamma2; n2.eps = s.rms_eps; n2.bits = bits; n2.B = B; n2.d = d;
-  n2.a_op = at<void>(ws, L.a_op); n2.scale = scale; n2.xn = tr ? tr->xn2 : nullptr; n2.codes = tr ? tr->codes2 : nullptr;
+  n2.a_op = at<void>(ws, L.a_op); n2.a_op_rows = L.Mpad; n2.scale = scale; n2.xn = tr ? tr->xn2 : nullptr;
+  n2.codes = tr ? tr->codes2 : nullptr;
   n2.status = status;
   n2.clear = at<uint32_t>(ws, L.ch_sel);
   n2.clear_words = CH_SEL_WORDS;
@@ -335,13 +332,13 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
     cudaMemcpyAsync(tr->h_mid, at<float>(ws, L.h_mid), sizeof(float) * B * d, cudaMemcpyDeviceToDevice, st);
   if (tr && tr->scales2) cudaMemcpyAsync(tr->scales2, scale, sizeof(float) * B, cudaMemcpyDeviceToDevice, st);
 
-  run_mlp(s, L, ws, B, w.w_gate, w.w_up, w.w_down_t, p, at<float>(ws, L.h_mid), 1, h_out_bf16, h_out_f32,
+  run_mlp(s, L, ws, B, w.w_gate_up, w.w_down, p, at<float>(ws, L.h_mid), 1, h_out_bf16, h_out_f32,
           tr ? tr->h_out : nullptr, tr ? tr->t : nullptr, tr ? tr->kept_ch : nullptr, tr ? tr->kept_ch_cnt : nullptr,
           st);
 }
 
 static bool weights_ok(const sol_layer_weights_t* w) {
-  return w && w->w_qkv && w->w_o && w->w_gate && w->w_up && w->w_down_t && w->gamma1 && w->gamma2;
+  return w && w->w_qkv && w->w_o && w->w_gate_up && w->w_down && w->gamma1 && w->gamma2;
 }
 
 }  // namespace sol
@@ -406,26 +403,51 @@ sol_status_t sol_sparse_decode_attn(const sol_shape_t* shape, const void* q_bf16
   return finish();
 }
 
-sol_status_t sol_pruned_swiglu_mlp(const sol_shape_t* shape, const void* x_bf16, const void* w_gate, const void* w_up,
-                                   const void* w_down_t, int32_t B, const int32_t* p_permille, void* out_bf16,
+sol_status_t sol_pruned_swiglu_mlp(const sol_shape_t* shape, const void* x_bf16, const void* w_gate_up,
+                                   const void* w_down, int32_t B, const int32_t* p_permille, void* out_bf16,
                                    int32_t* kept_ch, int32_t* kept_ch_cnt, void* ws, size_t ws_bytes,
                                    sol_stream_t stream) {
-  if (!shape || !x_bf16 || !w_gate || !w_up || !w_down_t || !p_permille || !out_bf16 || !ws || B < 0)
+  if (!shape || !x_bf16 || !w_gate_up || !w_down || !p_permille || !out_bf16 || !ws || B < 0)
     return SOL_ERR_INVALID_ARG;
   if (!shape_ok(shape) || B > 128) return SOL_ERR_UNSUPPORTED;
   if (B == 0) return SOL_OK;
   const Layout L = make_layout(*shape, B, 1);
   if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
-  // bf16 passthrough into the padded operand buffer, scale 1
+  // bf16 passthrough into the padded, packed operand buffer, scale 1
   NormQuantArgs n;
   memset(&n, 0, sizeof(n));
-  n.in = x_bf16; n.B = B; n.d = shape->d_model; n.a_op = at<void>(ws, L.a_op); n.scale = at<float>(ws, L.scale);
+  n.in = x_bf16; n.B = B; n.d = shape->d_model; n.a_op = at<void>(ws, L.a_op); n.a_op_rows = L.Mpad;
+  n.scale = at<float>(ws, L.scale);
   n.clear = at<uint32_t>(ws, L.ch_sel);
   n.clear_words = CH_SEL_WORDS;
   launch_norm_quant(n, st);
-  run_mlp(*shape, L, ws, B, w_gate, w_up, w_down_t, p_permille, nullptr, 0, out_bf16, nullptr, nullptr, nullptr,
+  run_mlp(*shape, L, ws, B, w_gate_up, w_down, p_permille, nullptr, 0, out_bf16, nullptr, nullptr, nullptr,
           kept_ch, kept_ch_cnt, st);
+  return finish();
+}
+
+size_t sol_packed_weight_bytes(const sol_shape_t* shape, int32_t kind) {
+  if (!shape_ok(shape)) return 0;
+  const int d = shape->d_model, qo = shape->n_q_heads * shape->head_dim;
+  const int nqkv = (shape->n_q_heads + 2 * shape->n_kv_heads) * shape->head_dim;
+  switch (kind) {
+    case SOL_W_QKV: return nk_packed_bytes(nk_geom_plain(nqkv, d));
+    case SOL_W_O: return nk_packed_bytes(nk_geom_plain(d, qo));
+    case SOL_W_GATE_UP: return nk_packed_bytes(nk_geom_gate_up(shape->d_ff, d, sm_count()));
+    case SOL_W_DOWN: return down_packed_bytes(shape->d_ff, d);
+    default: return 0;
+  }
+}
+
+sol_status_t sol_pack_weights(const sol_shape_t* shape, int32_t kind, const void* src0, const void* src1, void* dst,
+                              size_t dst_bytes, sol_stream_t stream) {
+  if (!shape || !src0 || !dst || kind < SOL_W_QKV || kind > SOL_W_DOWN || (kind == SOL_W_GATE_UP && !src1))
+    return SOL_ERR_INVALID_ARG;
+  const size_t need = sol_packed_weight_bytes(shape, kind);
+  if (need == 0) return SOL_ERR_UNSUPPORTED;
+  if (dst_bytes < need) return SOL_ERR_WORKSPACE_TOO_SMALL;
+  launch_pack_weights(*shape, kind, src0, src1, dst, (cudaStream_t)stream);
   return finish();
 }
 

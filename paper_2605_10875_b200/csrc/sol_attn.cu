@@ -1111,8 +1111,8 @@ struct GatherDev {
   float scale_log2;
   float* out_f32;
   uint16_t* out_bf16;
-  uint16_t* out_hi;
-  uint16_t* out_lo;
+  uint16_t* out_hi;  // packed operand of the output projection (2 out_rows rows: high parts, then low parts)
+  int out_rows;
   int* status;
 };
 
@@ -1349,8 +1349,10 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
       if (p.out_bf16) *reinterpret_cast<uint32_t*>(p.out_bf16 + idx) = pack_bf16(o0, o1);
       if (p.out_hi) {
         const uint16_t h0 = f2bf(o0), h1 = f2bf(o1);
-        *reinterpret_cast<uint32_t*>(p.out_hi + idx) = (uint32_t)h0 | ((uint32_t)h1 << 16);
-        *reinterpret_cast<uint32_t*>(p.out_lo + idx) = pack_bf16(o0 - bf2f(h0), o1 - bf2f(h1));
+        const int k = (kvh * G + h) * HD + e;  // column of the projection's input; e is even, so k and k + 1 share a piece
+        unsigned char* dst = reinterpret_cast<unsigned char*>(p.out_hi) + act_piece_offset(2 * p.out_rows, b, k >> 3) + (k & 7) * 2;
+        *reinterpret_cast<uint32_t*>(dst) = (uint32_t)h0 | ((uint32_t)h1 << 16);
+        *reinterpret_cast<uint32_t*>(dst + (size_t)p.out_rows * 128) = pack_bf16(o0 - bf2f(h0), o1 - bf2f(h1));
       }
     };
     if (ns == 1) {  // the row is this one item: its output goes out directly
@@ -1529,7 +1531,7 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   gd.scale_log2 = (float)(1.4426950408889634 / sqrt((double)hd));
   gd.out_f32 = a.out_f32;
   gd.out_bf16 = static_cast<uint16_t*>(a.out_bf16);
-  gd.out_hi = static_cast<uint16_t*>(a.out_hi); gd.out_lo = static_cast<uint16_t*>(a.out_lo);
+  gd.out_hi = static_cast<uint16_t*>(a.out_hi); gd.out_rows = a.out_rows;
   gd.status = a.status;
   const long long items = (long long)a.B * Hkv * a.splits;
   if (hd == 64) {

@@ -2,40 +2,37 @@
 //
 // The batch (16..128 rows after padding) is the small side, so every weight
 // byte is read from HBM exactly once and the kernels are bound by HBM
-// bandwidth.  They are built so that one thread keeps large TMA copies in
-// flight and nobody touches the data with ordinary instructions:
+// bandwidth.  Weights are packed once at load time (sol_pack_weights) into the
+// order the tensor cores read them from shared memory, and the activation
+// operands are written in that order by the kernels that produce them, so:
 //
-//   * weights and activations arrive by TMA tiled loads through tensor maps
-//     (128-byte swizzle, several 64-wide k chunks per copy) into a ring of
-//     shared-memory stages guarded by mbarriers (bounded waits);
+//   * a pipeline stage is two large contiguous bulk copies (cp.async.bulk,
+//     8..32 KB each) into a ring of shared-memory stages guarded by mbarriers
+//     (bounded waits): one for the weight tile, one for the activation tile;
 //   * one thread issues tcgen05.mma (bf16 x bf16 -> float32) with the WEIGHT
 //     tile as the 128-row M side and the batch as the N side, accumulating in
 //     tensor memory; tcgen05.commit releases each stage when its MMAs finish;
 //   * four warps read the accumulators back with tcgen05.ld and apply the
-//     epilogue (quantizer scale / residual / SwiGLU), writing out[m][n] with
-//     the weight row n along the lanes (coalesced).
+//     epilogue, writing out[m][n] with the weight row n along the lanes.
 //
-//   umma_nk   : Y[M][N] = A[M][K] . W[N][K]^T   (QKV, output and gate/up projections).  Each CTA owns
-//               a contiguous range of `rows` weight rows (a multiple of 8 chosen so that one wave of
-//               CTAs covers all SMs) over the whole of K.  The MMA always spans 128 rows; rows beyond
-//               the CTA's range read whatever follows in shared memory and land in accumulator lanes
-//               that are never stored (an output row depends only on its own weight row).
-//   umma_down : Y[M][d] = T[M][ff] . W[ff][d]   (down projection).  W rows are intermediate channels,
-//               so the weight tile is the MN-major operand.  CTA = (128 output columns, range of 64-
-//               channel blocks); blocks in which no token keeps a channel are neither copied nor
-//               multiplied; partial sums per range are reduced by reduce_out.
+//   umma_nk   : Y[M][N] = A[M][K] . W[N][K]^T   (QKV, output and gate/up projections).  A CTA owns one tile
+//               of R weight rows; QKV / output: R = 128 and a slice of K (raw partial sums per slice, summed by
+//               the consumer); gate/up: the whole of K, rows alternating gate_c, up_c, so that a channel's two
+//               sums sit in neighbouring accumulator lanes and SwiGLU is a lane exchange.  The MMA always
+//               spans 128 rows; rows beyond the tile read whatever follows in shared memory and land in
+//               accumulator lanes that are never stored.
+//   umma_down : Y[M][d] = T[M][ff] . W[ff][d]   (down projection).  W rows are intermediate channels, so the
+//               weight tile is the MN-major operand.  CTA = (128 output columns, range of 64-channel
+//               blocks); blocks in which no token keeps a channel are neither copied nor multiplied;
+//               partial sums per range are reduced by reduce_out.
 #include <cstring>
-#include <mutex>
-#include <unordered_map>
-
-#include <cudaTypedefs.h>
 
 #include "sol_internal.h"
 #include "sol_umma.cuh"
 
 namespace sol {
 
-constexpr int UM_THREADS = 192;      // warps 0-3: epilogue, warp 4: TMA producer, warp 5: MMA issuer + TMEM owner
+constexpr int UM_THREADS = 192;      // warps 0-3: epilogue, warp 4: producer, warp 5: MMA issuer + TMEM owner
 constexpr int UM_MAX_STAGES = 8;
 constexpr int UM_TILE_SPAN = 16384;  // bytes one 128-row operand read spans from the start of a chunk tile
 constexpr int UM_SMEM_BUDGET = 204 * 1024;
@@ -57,13 +54,16 @@ __device__ __forceinline__ unsigned char* align_1024(unsigned char* p) {
 // umma_nk
 // ============================================================================
 struct NKDev {
-  int M, Mpad, K, N;  // N: weight rows (EPI_SWIGLU: channels, with a gate and an up row each)
-  int rows;           // weight rows per CTA
+  int M, Mpad, K, N;  // N: outputs per token (EPI_SWIGLU: channels, with a gate and an up row each)
+  int R;              // packed weight rows per tile
+  int chunks;         // K / 64
   int ksplit;         // K slices (blockIdx.y); EPI_PARTIAL writes one partial per slice
   int cps, stages;    // 64-wide k chunks per stage, ring depth
   int n_b;            // 1, or 2: the activation rows are a high-part block followed by a low-part block of
                       // Mpad rows each; one MMA of N = 2 Mpad multiplies both, the epilogue adds the halves
   uint32_t tmem_cols;
+  const unsigned char* w;  // packed weights
+  const unsigned char* x;  // packed activations
   const float* row_scale;
   float* out0;
   float* out1;
@@ -73,15 +73,12 @@ struct NKDev {
 };
 
 template <int EPI>
-__global__ void __launch_bounds__(UM_THREADS, 1)
-umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant__ CUtensorMap tm_w1,
-               const __grid_constant__ CUtensorMap tm_x0, const NKDev p) {
+__global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
   extern __shared__ unsigned char smem_raw[];
-  constexpr int NW = EPI == EPI_SWIGLU ? 2 : 1;
   unsigned char* stages = align_1024(smem_raw);
   const int nb_rows = p.n_b * p.Mpad;                      // N of the MMA
-  const int w_tile = p.rows * 128, x_tile = nb_rows * 128;  // bytes per 64-wide k chunk
-  const int stage_bytes = p.cps * (NW * w_tile + x_tile);
+  const int w_tile = p.R * 128, x_tile = nb_rows * 128;    // bytes per 64-wide k chunk
+  const int stage_bytes = p.cps * (w_tile + x_tile);
   UmBarriers* bars = reinterpret_cast<UmBarriers*>(stages + (size_t)p.stages * stage_bytes + UM_TILE_SPAN);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -100,31 +97,29 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
 
-  const int row0 = blockIdx.x * p.rows;
+  const int tile = blockIdx.x;
   // this CTA's K slice, in 64-wide chunks (cps == 1 whenever K is split)
-  const int chunks = p.K / 64;
-  const int ch0 = (int)(((long long)chunks * blockIdx.y) / p.ksplit);
-  const int ch1 = (int)(((long long)chunks * (blockIdx.y + 1)) / p.ksplit);
+  const int ch0 = (int)(((long long)p.chunks * blockIdx.y) / p.ksplit);
+  const int ch1 = (int)(((long long)p.chunks * (blockIdx.y + 1)) / p.ksplit);
   const int n_iter = (ch1 - ch0) / p.cps;
+  const unsigned char* w_src = p.w + ((size_t)tile * p.chunks + ch0) * w_tile;  // this tile's chunks are contiguous
+  const unsigned char* x_src = p.x + (size_t)ch0 * x_tile;                     // and so are the activation chunks
 
   if (warp == 4) {
-    // ------------------------------ TMA producer -----------------------------
+    // -------------------------------- producer -------------------------------
     // Weights do not depend on earlier kernels: the first ring of weight tiles is requested before
     // pdl_wait(), the activation tiles of those stages after it.
     if (lane == 0) {
-      tma_prefetch_map(&tm_w0);
-      tma_prefetch_map(&tm_x0);
       const int pre = min(n_iter, p.stages);
       for (int it = 0; it < pre; ++it) {
         unsigned char* st = stages + (size_t)it * stage_bytes;
         mbar_expect_tx(&bars->full[it], stage_bytes);
-        tma_load_3d(st, &tm_w0, 0, row0, ch0 + it * p.cps, &bars->full[it]);
-        if (NW == 2) tma_load_3d(st + p.cps * w_tile, &tm_w1, 0, row0, ch0 + it * p.cps, &bars->full[it]);
+        bulk_g2s(st, w_src + (size_t)it * p.cps * w_tile, p.cps * w_tile, &bars->full[it]);
       }
       pdl_wait();
       for (int it = 0; it < pre; ++it) {
-        unsigned char* xs = stages + (size_t)it * stage_bytes + NW * p.cps * w_tile;
-        tma_load_3d(xs, &tm_x0, 0, 0, ch0 + it * p.cps, &bars->full[it]);
+        unsigned char* xs = stages + (size_t)it * stage_bytes + p.cps * w_tile;
+        bulk_g2s(xs, x_src + (size_t)it * p.cps * x_tile, p.cps * x_tile, &bars->full[it]);
       }
       for (int it = pre; it < n_iter; ++it) {
         const int s = it % p.stages;
@@ -132,15 +127,13 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
         if (!mbar_wait(&bars->empty[s], ph ^ 1, p.status)) break;
         unsigned char* st = stages + (size_t)s * stage_bytes;
         mbar_expect_tx(&bars->full[s], stage_bytes);
-        tma_load_3d(st, &tm_w0, 0, row0, ch0 + it * p.cps, &bars->full[s]);
-        if (NW == 2) tma_load_3d(st + p.cps * w_tile, &tm_w1, 0, row0, ch0 + it * p.cps, &bars->full[s]);
-        unsigned char* xs = st + NW * p.cps * w_tile;
-        tma_load_3d(xs, &tm_x0, 0, 0, ch0 + it * p.cps, &bars->full[s]);
+        bulk_g2s(st, w_src + (size_t)it * p.cps * w_tile, p.cps * w_tile, &bars->full[s]);
+        bulk_g2s(st + p.cps * w_tile, x_src + (size_t)it * p.cps * x_tile, p.cps * x_tile, &bars->full[s]);
       }
     }
   } else if (warp == 5) {
     // ------------------------------- MMA issuer ------------------------------
-    // The mbarrier wait orders the TMA writes before the MMA reads; no tcgen05 fence is needed per stage.
+    // The mbarrier wait orders the copies before the MMA reads; no tcgen05 fence is needed per stage.
     const uint32_t idesc = umma_idesc_bf16_m128(nb_rows, 0, 0);
     bool acc = false, ok = true;
     // the first stage fills only after the producer's own pdl_wait(): without this wait the bounded poll
@@ -152,19 +145,15 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
       ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[s], ph, p.status));
       if (!ok) break;
       const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
-      const uint32_t xs = st + NW * p.cps * w_tile;
+      const uint32_t xs = st + p.cps * w_tile;
       const uint64_t a_base = umma_smem_desc(st, 16, 1024), b_base = umma_smem_desc(xs, 16, 1024);
       for (int c = 0; c < p.cps; ++c) {
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks) {
           // descriptors advance in units of 16 bytes: a chunk tile per c, 32 bytes per 16-wide k step
           const uint64_t a0 = a_base + (uint64_t)((c * w_tile + ks * 32) >> 4);
-          const uint64_t a1 = a_base + (uint64_t)(((p.cps + c) * w_tile + ks * 32) >> 4);
           const uint64_t b0 = b_base + (uint64_t)((c * x_tile + ks * 32) >> 4);
-          if (elect_one()) {
-            umma_bf16(tmem, a0, b0, idesc, acc);
-            if (NW == 2) umma_bf16(tmem + nb_rows, a1, b0, idesc, acc);
-          }
+          if (elect_one()) umma_bf16(tmem, a0, b0, idesc, acc);
           acc = true;
         }
       }
@@ -174,42 +163,49 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
     if (ok && elect_one()) umma_commit(&bars->accum);
   } else {
     // -------------------------------- epilogue -------------------------------
-    pdl_wait();  // the epilogue reads scales / the residual and overwrites buffers earlier kernels used
-    if (warp * 32 < p.rows) {
+    pdl_wait();  // the epilogue reads scales and overwrites buffers earlier kernels used
+    if (warp * 32 < p.R) {
       const bool ok = mbar_wait(&bars->accum, 0, p.status);
       tc_fence_after();
-      const int r = warp * 32 + lane, n = row0 + r;
-      const bool valid = r < p.rows && n < p.N;
+      const int r = warp * 32 + lane;  // row of the tile = accumulator lane
       const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
       for (int c0 = 0; c0 < p.Mpad && ok; c0 += 16) {
-        float v[16], u[16];
+        float v[16];
         tmem_ld16(tl + c0, v);
-        if (NW == 2) tmem_ld16(tl + nb_rows + c0, u);
         if (p.n_b == 2) {  // high-part and low-part products
           float w2[16];
           tmem_ld16(tl + p.Mpad + c0, w2);
 #pragma unroll
           for (int i = 0; i < 16; ++i) v[i] += w2[i];
         }
+        if (EPI == EPI_SWIGLU) {
+          // even lanes hold a channel's gate sum, their odd neighbours its up sum
+          const int ch = (tile * p.R + r) >> 1;
+          const bool valid = r < p.R && ch < p.N;
+          const bool even = (lane & 1) == 0;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int m = c0 + i;
-          if (m < p.M) {  // warp-uniform
-            const size_t o = (size_t)m * p.N + n;
-            if (EPI == EPI_SWIGLU) {
+          for (int i = 0; i < 16; ++i) {
+            const int m = c0 + i;
+            if (m < p.M) {  // warp-uniform
               const float sc = p.row_scale ? p.row_scale[m] : 1.0f;
-              const float gg = v[i] * sc, uu = u[i] * sc;
+              const float mine = v[i] * sc;
+              const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
+              const float gg = even ? mine : other, uu = even ? other : mine;
               const float tv = (gg / (1.0f + expf(-gg))) * uu;
+              const size_t o = (size_t)m * p.N + ch;
               if (valid) {
-                p.out0[o] = gg;
-                p.out1[o] = uu;
-                p.out2[o] = tv;
+                if (even) {
+                  p.out0[o] = gg;
+                  p.out2[o] = tv;
+                } else {
+                  p.out1[o] = uu;
+                }
               }
               if (p.sel != nullptr) {
                 // what the channel selection needs from all of a token's channels: a histogram of |t|
                 // and the largest |g|, |u| (non-negative floats order like their bit patterns)
                 uint32_t* sel = p.sel + (size_t)m * CH_SEL_WORDS;
-                if (valid) atomicAdd(sel + chan_bin(fabsf(tv)), 1u);
+                if (valid && even) atomicAdd(sel + chan_bin(fabsf(tv)), 1u);
                 const uint32_t gm = __reduce_max_sync(0xffffffffu, valid ? __float_as_uint(fabsf(gg)) : 0u);
                 const uint32_t um = __reduce_max_sync(0xffffffffu, valid ? __float_as_uint(fabsf(uu)) : 0u);
                 if (lane == 0) {
@@ -217,9 +213,15 @@ umma_nk_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant_
                   atomicMax(sel + CH_UMAX, um);
                 }
               }
-            } else if (valid) {
-              p.out0[(size_t)blockIdx.y * p.M * p.N + o] = v[i];
             }
+          }
+        } else {
+          const int n = tile * p.R + r;
+          const bool valid = r < p.R && n < p.N;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int m = c0 + i;
+            if (m < p.M && valid) p.out0[((size_t)blockIdx.y * p.M + m) * p.N + n] = v[i];
           }
         }
       }
@@ -237,8 +239,10 @@ struct DownDev {
   int M, Mpad, ff, d;
   int chunks, stages;
   uint32_t tmem_cols;
-  const int32_t* live;  // [ff/32]
-  float* partial;       // [chunks][Mpad][d]
+  const unsigned char* w;  // packed W_down_t: [slab][64-channel block][16 KB]
+  const unsigned char* t;  // packed masked activations: [64-channel chunk][2 Mpad rows][128 B]
+  const int32_t* live;     // [ff/32]
+  float* partial;          // [chunks][Mpad][d]
   int* status;
 };
 
@@ -246,12 +250,11 @@ __device__ __forceinline__ bool block_live(const int32_t* live, int jb, int gran
   return live[2 * jb] != 0 || (2 * jb + 1 < granules && live[2 * jb + 1] != 0);
 }
 
-__global__ void __launch_bounds__(UM_THREADS, 1)
-umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_t, const DownDev p) {
+__global__ void __launch_bounds__(UM_THREADS, 1) umma_down_kernel(const DownDev p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* stages = align_1024(smem_raw);
-  const int t_tile = p.Mpad * 128;
-  const int stage_bytes = UM_TILE_SPAN + 2 * t_tile;
+  const int t_tile = 2 * p.Mpad * 128;
+  const int stage_bytes = UM_TILE_SPAN + t_tile;
   UmBarriers* bars = reinterpret_cast<UmBarriers*>(stages + (size_t)p.stages * stage_bytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -279,7 +282,6 @@ umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
 
   if (warp == 4) {
     if (lane == 0) {
-      tma_prefetch_map(&tm_w);
       int it = 0;
       for (int jb = jb0; jb < jb1; ++jb) {
         if (!block_live(p.live, jb, granules)) continue;
@@ -289,8 +291,8 @@ umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
         if (!mbar_wait(&bars->empty[s], ph ^ 1, p.status)) break;
         unsigned char* st = stages + (size_t)s * stage_bytes;
         mbar_expect_tx(&bars->full[s], stage_bytes);
-        tma_load_3d(st, &tm_w, 0, jb * 64, slab * 2, &bars->full[s]);
-        tma_load_2d(st + UM_TILE_SPAN, &tm_t, jb * 64, 0, &bars->full[s]);  // high rows then low rows
+        bulk_g2s(st, p.w + ((size_t)slab * jblocks + jb) * UM_TILE_SPAN, UM_TILE_SPAN, &bars->full[s]);
+        bulk_g2s(st + UM_TILE_SPAN, p.t + (size_t)jb * t_tile, t_tile, &bars->full[s]);  // high rows then low rows
       }
     }
   } else if (warp == 5) {
@@ -355,93 +357,71 @@ umma_down_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant
 }
 
 // ============================================================================
-// tensor maps (host)
+// one-time packing of the weights
+// ============================================================================
+// One thread per 16-byte piece of the packed matrix.
+__global__ void pack_nk_kernel(const uint4* __restrict__ src0, const uint4* __restrict__ src1, uint4* __restrict__ dst,
+                               int n_src_rows, int K, int R, int tiles, int chunks, int interleaved) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t total = (size_t)tiles * chunks * R * 8;
+  if (i >= total) return;
+  const int q_dst = (int)(i & 7);
+  const size_t row_lin = i >> 3;  // ((tile * chunks + chunk) * R + r)
+  const int r = (int)(row_lin % R);
+  const int chunk = (int)((row_lin / R) % chunks);
+  const int tile = (int)(row_lin / ((size_t)R * chunks));
+  const int q = q_dst ^ (r & 7);  // the source piece that lives at this position
+  const int n = tile * R + r;     // packed row
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  const int src_row = interleaved ? n >> 1 : n;
+  if (src_row < n_src_rows) {
+    const uint4* src = (interleaved && (n & 1)) ? src1 : src0;
+    v = src[((size_t)src_row * K + (size_t)chunk * 64 + q * 8) / 8];
+  }
+  dst[i] = v;
+}
+
+__global__ void pack_down_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int ff, int d) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int jblocks = (ff + 63) / 64;
+  const size_t total = (size_t)(d / 128) * jblocks * 1024;  // pieces
+  if (i >= total) return;
+  const int q_dst = (int)(i & 7);
+  const int c = (int)((i >> 3) & 63);         // channel within the block
+  const int cb = (int)((i >> 9) & 1);         // 64-column half of the slab
+  const int jb = (int)((i >> 10) % jblocks);
+  const int slab = (int)((i >> 10) / jblocks);
+  const int q = q_dst ^ (c & 7);
+  const int j = jb * 64 + c;
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  if (j < ff) v = src[((size_t)j * d + slab * 128 + cb * 64 + q * 8) / 8];
+  dst[i] = v;
+}
+
+void launch_pack_weights(const sol_shape_t& s, int kind, const void* src0, const void* src1, void* dst, cudaStream_t st) {
+  const int d = s.d_model, qo = s.n_q_heads * s.head_dim, nqkv = (s.n_q_heads + 2 * s.n_kv_heads) * s.head_dim;
+  if (kind == SOL_W_DOWN) {
+    const size_t pieces = down_packed_bytes(s.d_ff, d) / 16;
+    pack_down_kernel<<<(unsigned)((pieces + 255) / 256), 256, 0, st>>>(static_cast<const uint4*>(src0), static_cast<uint4*>(dst),
+                                                                      s.d_ff, d);
+  } else {
+    NKGeom g;
+    int rows;
+    if (kind == SOL_W_QKV) { g = nk_geom_plain(nqkv, d); rows = nqkv; }
+    else if (kind == SOL_W_O) { g = nk_geom_plain(d, qo); rows = d; }
+    else { g = nk_geom_gate_up(s.d_ff, d, sm_count()); rows = s.d_ff; }
+    const size_t pieces = nk_packed_bytes(g) / 16;
+    pack_nk_kernel<<<(unsigned)((pieces + 255) / 256), 256, 0, st>>>(static_cast<const uint4*>(src0), static_cast<const uint4*>(src1),
+                                                                    static_cast<uint4*>(dst), rows, g.K, g.R, g.tiles,
+                                                                    g.chunks, kind == SOL_W_GATE_UP ? 1 : 0);
+  }
+  record_cuda_error(cudaGetLastError(), "weight packing");
+}
+
+// ============================================================================
+// launchers
 // ============================================================================
 namespace {
-
-struct MapKey {
-  uintptr_t ptr;
-  uint64_t dim[3];
-  uint64_t stride[2];
-  uint32_t box[3];
-  uint32_t rank;
-  bool operator==(const MapKey& o) const {
-    return ptr == o.ptr && rank == o.rank && dim[0] == o.dim[0] && dim[1] == o.dim[1] && dim[2] == o.dim[2] &&
-           stride[0] == o.stride[0] && stride[1] == o.stride[1] && box[0] == o.box[0] && box[1] == o.box[1] &&
-           box[2] == o.box[2];
-  }
-};
-struct MapKeyHash {
-  size_t operator()(const MapKey& k) const {
-    uint64_t h = k.ptr * 0x9e3779b97f4a7c15ull;
-    auto mix = [&](uint64_t v) { h = (h ^ v) * 0x100000001b3ull + (h >> 29); };
-    mix(k.dim[0]); mix(k.dim[1]); mix(k.dim[2]); mix(k.stride[0]); mix(k.stride[1]);
-    mix(k.box[0]); mix(k.box[1]); mix(k.box[2]); mix(k.rank);
-    return (size_t)h;
-  }
-};
-
-PFN_cuTensorMapEncodeTiled encode_fn() {
-  static PFN_cuTensorMapEncodeTiled fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    return reinterpret_cast<PFN_cuTensorMapEncodeTiled>(p);
-  }();
-  return fn;
-}
-
-// bf16 tensor map with 128-byte swizzle; encoded maps are remembered (the encoding is a pure function
-// of the key, and the same weight matrices come back every step).
-bool tensor_map(CUtensorMap* out, const void* ptr, uint32_t rank, const uint64_t* dim, const uint64_t* stride,
-                const uint32_t* box) {
-  static std::mutex mu;
-  static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
-  MapKey k;
-  memset(&k, 0, sizeof(k));
-  k.ptr = reinterpret_cast<uintptr_t>(ptr);
-  k.rank = rank;
-  for (uint32_t i = 0; i < rank; ++i) {
-    k.dim[i] = dim[i];
-    k.box[i] = box[i];
-    if (i + 1 < rank) k.stride[i] = stride[i];
-  }
-  std::lock_guard<std::mutex> lock(mu);
-  auto it = cache.find(k);
-  if (it != cache.end()) {
-    *out = it->second;
-    return true;
-  }
-  PFN_cuTensorMapEncodeTiled fn = encode_fn();
-  if (!fn) {
-    record_cuda_error(cudaErrorNotSupported, "cuTensorMapEncodeTiled entry point");
-    return false;
-  }
-  const cuuint32_t ones[3] = {1, 1, 1};
-  CUtensorMap m;
-  const CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(ptr), dim, stride, box, ones,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
-    return false;
-  }
-  if (cache.size() > (1u << 16)) cache.clear();
-  cache.emplace(k, m);
-  *out = m;
-  return true;
-}
-
-// [rows][K] row-major bf16 viewed as (64 k, rows, K/64 chunks): a box of (64, box_rows, cps) lands in
-// shared memory as cps consecutive [box_rows][64] tiles, each in the 128-byte-swizzled K-major layout.
-bool kmajor_map(CUtensorMap* out, const void* ptr, int rows, int K, int box_rows, int cps) {
-  const uint64_t dim[3] = {64, (uint64_t)rows, (uint64_t)(K / 64)};
-  const uint64_t stride[2] = {(uint64_t)K * 2, 128};
-  const uint32_t box[3] = {64, (uint32_t)box_rows, (uint32_t)cps};
-  return tensor_map(out, ptr, 3, dim, stride, box);
-}
 
 uint32_t pow2_cols(int n) {
   uint32_t c = 32;
@@ -449,89 +429,56 @@ uint32_t pow2_cols(int n) {
   return c;
 }
 
-int round_mpad(int M) {
-  const int mt = (M + 15) / 16;
+}  // namespace
+
+int pad_rows(int B) {
+  const int mt = (B + 15) / 16;
   return 16 * (mt <= 1 ? 1 : (mt <= 2 ? 2 : (mt <= 4 ? 4 : 8)));
 }
 
-}  // namespace
-
-// ============================================================================
-// launchers
-// ============================================================================
-// Split-K geometry of the EPI_PARTIAL projections: full 128-row weight tiles (so that one TMA box and
-// one MMA cover as many weight bytes as possible) and as many K slices as it takes to give every SM a CTA.
-static void nk_partial_geometry(int N, int K, int* rows, int* tiles, int* ksplit) {
-  int r = (N + 7) / 8 * 8;
-  if (r > 128) r = 128;
-  const int t = (N + r - 1) / r;
-  const int chunks = K / 64;
-  int z = sm_count() / t;
-  if (z > chunks) z = chunks;
+// Split-K of the EPI_PARTIAL projections: as many K slices as it takes to give every SM a CTA.
+int nk_ksplit(int N, int K) {
+  const NKGeom g = nk_geom_plain(N, K);
+  int z = sm_count() / g.tiles;
+  if (z > g.chunks) z = g.chunks;
   if (z > NK_MAX_KSPLIT) z = NK_MAX_KSPLIT;
   if (z < 1) z = 1;
-  *rows = r;
-  *tiles = t;
-  *ksplit = z;
-}
-
-int nk_ksplit(int N, int K) {
-  int rows, tiles, z;
-  nk_partial_geometry(N, K, &rows, &tiles, &z);
   return z;
 }
 
 void launch_gemm_nk(const GemmNK& g, GemmEpilogue epi, cudaStream_t st) {
-  const int nw = epi == EPI_SWIGLU ? 2 : 1;
   NKDev d;
   memset(&d, 0, sizeof(d));
-  d.M = g.M; d.Mpad = round_mpad(g.M); d.K = g.K; d.N = g.N;
-  d.n_b = g.a_lo ? 2 : 1;
-  if (g.a_lo && static_cast<const char*>(g.a_lo) != static_cast<const char*>(g.a_hi) + (size_t)d.Mpad * g.K * 2) {
-    record_cuda_error(cudaErrorInvalidValue, "split activation operand must be contiguous (high rows, then low rows)");
-    return;
-  }
-  const int chunks = g.K / 64;
-  int rows, tiles, ksplit = 1;
-  if (epi == EPI_PARTIAL) {
-    nk_partial_geometry(g.N, g.K, &rows, &tiles, &ksplit);
-  } else {
-    // whole K per CTA, one wave of CTAs: `rows` channels (a gate and an up row each) per CTA
-    const int sms = sm_count();
-    rows = ((g.N + sms - 1) / sms + 7) / 8 * 8;
-    if (rows > 128) rows = 128;
-    tiles = (g.N + rows - 1) / rows;
-  }
-  d.rows = rows;
-  d.ksplit = ksplit;
-  const int chunk_bytes = 128 * (nw * rows + d.n_b * d.Mpad);
-  int cps = ksplit > 1 ? 1 : 4;
-  while (cps > 1 && (cps * chunk_bytes > 36 * 1024 || chunks % cps)) cps >>= 1;
+  d.M = g.M; d.Mpad = pad_rows(g.M); d.K = g.K; d.N = g.N;
+  d.n_b = g.n_b;
+  const NKGeom geo = epi == EPI_SWIGLU ? nk_geom_gate_up(g.N, g.K, sm_count()) : nk_geom_plain(g.N, g.K);
+  d.R = geo.R;
+  d.chunks = geo.chunks;
+  d.ksplit = epi == EPI_PARTIAL ? nk_ksplit(g.N, g.K) : 1;
+  const int chunk_bytes = 128 * (d.R + d.n_b * d.Mpad);
+  int cps = d.ksplit > 1 ? 1 : 4;
+  while (cps > 1 && (cps * chunk_bytes > 36 * 1024 || d.chunks % cps)) cps >>= 1;
   d.cps = cps;
   const int stage_bytes = cps * chunk_bytes;
-  const int iters = (chunks / ksplit + (chunks % ksplit ? 1 : 0)) / cps;  // of the longest slice
+  const int iters = (d.chunks / d.ksplit + (d.chunks % d.ksplit ? 1 : 0)) / cps;  // of the longest slice
   int stages = UM_SMEM_BUDGET / stage_bytes;
   if (stages > UM_MAX_STAGES) stages = UM_MAX_STAGES;
   if (stages > iters) stages = iters;
   if (stages < 1) stages = 1;
   d.stages = stages;
-  d.tmem_cols = pow2_cols(nw * d.n_b * d.Mpad);
+  d.tmem_cols = pow2_cols(d.n_b * d.Mpad);
+  d.w = static_cast<const unsigned char*>(g.w);
+  d.x = static_cast<const unsigned char*>(g.a);
   d.row_scale = g.row_scale;
   d.out0 = g.out0; d.out1 = g.out1; d.out2 = g.out2; d.sel = g.sel; d.status = g.status;
-
-  CUtensorMap w0, w1, x0;
-  bool ok = kmajor_map(&w0, g.w0, g.N, g.K, rows, cps);
-  ok = ok && kmajor_map(&w1, nw == 2 ? g.w1 : g.w0, g.N, g.K, rows, cps);
-  ok = ok && kmajor_map(&x0, g.a_hi, d.n_b * d.Mpad, g.K, d.n_b * d.Mpad, cps);
-  if (!ok) return;
   const int smem = 1024 + stages * stage_bytes + UM_TILE_SPAN + (int)sizeof(UmBarriers);
-  const dim3 grid(tiles, ksplit);
+  const dim3 grid(geo.tiles, d.ksplit);
   if (epi == EPI_SWIGLU) {
     ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_nk_kernel<EPI_SWIGLU>), smem);
-    SOL_LAUNCH("gemm_gate_up_swiglu", umma_nk_kernel<EPI_SWIGLU>, grid, dim3(UM_THREADS), smem, st, w0, w1, x0, d);
+    SOL_LAUNCH("gemm_gate_up_swiglu", umma_nk_kernel<EPI_SWIGLU>, grid, dim3(UM_THREADS), smem, st, d);
   } else {
     ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_nk_kernel<EPI_PARTIAL>), smem);
-    SOL_LAUNCH(g.name ? g.name : "gemm_partial", umma_nk_kernel<EPI_PARTIAL>, grid, dim3(UM_THREADS), smem, st, w0, w1, x0, d);
+    SOL_LAUNCH(g.name ? g.name : "gemm_partial", umma_nk_kernel<EPI_PARTIAL>, grid, dim3(UM_THREADS), smem, st, d);
   }
 }
 
@@ -547,35 +494,19 @@ int down_chunks(int ff, int d) {
 void launch_gemm_down(const GemmDown& g, cudaStream_t st) {
   DownDev d;
   memset(&d, 0, sizeof(d));
-  d.M = g.M; d.Mpad = round_mpad(g.M); d.ff = g.ff; d.d = g.d;
+  d.M = g.M; d.Mpad = pad_rows(g.M); d.ff = g.ff; d.d = g.d;
   d.chunks = g.chunks;
   const int stage_bytes = UM_TILE_SPAN + 2 * d.Mpad * 128;
   int stages = UM_SMEM_BUDGET / stage_bytes;
   if (stages > UM_MAX_STAGES) stages = UM_MAX_STAGES;
   d.stages = stages;
   d.tmem_cols = pow2_cols(2 * d.Mpad);
+  d.w = static_cast<const unsigned char*>(g.w);
+  d.t = static_cast<const unsigned char*>(g.t);
   d.live = g.live; d.partial = g.partial; d.status = g.status;
-
-  if (static_cast<const char*>(g.t_lo) != static_cast<const char*>(g.t_hi) + (size_t)d.Mpad * g.ff * 2) {
-    record_cuda_error(cudaErrorInvalidValue, "split activation operand must be contiguous (high rows, then low rows)");
-    return;
-  }
-  CUtensorMap w, tm;
-  // W[ff][d] viewed as (64 columns, ff channels, d/64 column blocks): a box of (64, 64, 2) lands as two
-  // [64 channels][64 columns] blocks, the MN-major operand layout for 128 output columns
-  const uint64_t wdim[3] = {64, (uint64_t)g.ff, (uint64_t)(g.d / 64)};
-  const uint64_t wstride[2] = {(uint64_t)g.d * 2, 128};
-  const uint32_t wbox[3] = {64, 64, 2};
-  bool ok = tensor_map(&w, g.w, 3, wdim, wstride, wbox);
-  // activations [2 Mpad][ff] (high rows, then low rows): (ff, 2 Mpad) with a box of (64 channels, all rows); channels past ff read as zero
-  const uint64_t tdim[2] = {(uint64_t)g.ff, (uint64_t)(2 * d.Mpad)};
-  const uint64_t tstride[1] = {(uint64_t)g.ff * 2};
-  const uint32_t tbox[2] = {64, (uint32_t)(2 * d.Mpad)};
-  ok = ok && tensor_map(&tm, g.t_hi, 2, tdim, tstride, tbox);
-  if (!ok) return;
   const int smem = 1024 + stages * stage_bytes + (int)sizeof(UmBarriers);
   ensure_dynamic_smem(reinterpret_cast<const void*>(&umma_down_kernel), smem);
-  SOL_LAUNCH("gemm_down_gathered", umma_down_kernel, dim3(g.d / 128, g.chunks), dim3(UM_THREADS), smem, st, w, tm, d);
+  SOL_LAUNCH("gemm_down_gathered", umma_down_kernel, dim3(g.d / 128, g.chunks), dim3(UM_THREADS), smem, st, d);
 }
 
 // ============================================================================

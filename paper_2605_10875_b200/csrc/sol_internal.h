@@ -61,6 +61,7 @@ struct NormQuantArgs {
   const int32_t* bits;
   int B, d;
   void* a_op;
+  int a_op_rows;     // 0: a_op is a plain [B][d] matrix; otherwise the packed operand layout with this many rows
   float* scale;
   float* xn;
   int8_t* codes;
@@ -214,8 +215,9 @@ struct AttnArgs {
   // outputs (each optional)
   float* out_f32;    // [B][Hq][hd]
   void* out_bf16;    // [B][Hq][hd]
-  void* out_hi;      // bf16 [Mpad][Hq*hd]
-  void* out_lo;
+  void* out_hi;      // packed operand of the output projection: 2 out_rows rows (bf16 high parts, then low parts)
+  void* out_lo;      // unused
+  int out_rows;
   int* status;
 };
 
@@ -284,10 +286,9 @@ struct ChannelSelectArgs {
   const float* g;      // [B][ff]
   const float* u;
   const float* t;
-  const void* a_op;    // bf16 [B][d] MLP input operand
+  const void* a_op;    // packed MLP input operand (pad_rows(B) rows)
   const float* scale;  // [B]
-  const void* w_gate;  // bf16 [ff][d]
-  const void* w_up;
+  const void* w_gate_up;  // packed gate/up weights
   uint32_t* sel;       // [B][CH_SEL_WORDS] filled by the gate/up epilogue
   double* cand_val;    // [B][CH_CAND_CAP]
   int32_t* cand_idx;   // [B][CH_CAND_CAP]
@@ -295,8 +296,7 @@ struct ChannelSelectArgs {
   int32_t* scratch_idx; // [B][ff] scratch of the single-CTA path
   int32_t* kept_ch;    // optional [B][ff]: ascending list, written only when requested
   int32_t* kept_cnt;   // [B]
-  void* t_hi;          // bf16 [Mpad][ff]
-  void* t_lo;
+  void* t_op;          // packed operand of the down projection: 2 pad_rows(B) rows (bf16 high parts, then low parts)
   int32_t* live;       // [ff/32], all zero on entry (cleared by reduce_out after the down projection)
   int* status;
 };

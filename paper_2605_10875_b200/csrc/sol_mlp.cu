@@ -31,10 +31,10 @@ struct ChanDev {
   const float* g;
   const float* u;
   const float* t;
-  const uint16_t* a_op;
+  const unsigned char* a_op;  // packed operand, Mpad rows
   const float* scale;
-  const uint16_t* w_gate;
-  const uint16_t* w_up;
+  const unsigned char* w_gu;  // packed gate/up weights: rows alternate gate_c, up_c
+  int R, chunks, Mpad;        // rows per tile and 64-wide chunks of the packed weights; rows of the operand blocks
   uint32_t* sel;
   double* cand_val;
   int32_t* cand_idx;
@@ -42,8 +42,7 @@ struct ChanDev {
   int32_t* kept_ch;
   int32_t* scratch_idx;  // [B][ff] list written by the single-CTA kernel (not an output)
   int32_t* kept_cnt;
-  uint16_t* t_hi;
-  uint16_t* t_lo;
+  unsigned char* t_op;  // packed operand of the down projection: 2 Mpad rows (high parts, then low parts)
   int32_t* live;
   int* status;
 };
@@ -150,11 +149,8 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
         // g_j = scale * sum_e x_e w_je with x the quantizer codes (or the bf16 row): every product of two
         // bf16 numbers is an exact float32, so the sums are gathered exactly in float pairs
         const double sc = (double)p.scale[b];
-        const uint16_t* x = p.a_op + (size_t)b * d;
         for (int c = warp; c < n_cand; c += WARPS) {
           const int j = sm.cand_idx[c];
-          const uint16_t* wg = p.w_gate + (size_t)j * d;
-          const uint16_t* wu = p.w_up + (size_t)j * d;
           float gh = 0.f, gl = 0.f, uh = 0.f, ul = 0.f;
           // RB 256-wide slices per round, all loads of a round issued before the first use
           constexpr int RB = THREADS >= 1024 ? 2 : 4;  // 64 registers per thread at 1024 threads
@@ -163,10 +159,10 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
 #pragma unroll
             for (int r = 0; r < RB; ++r) {
               const int e = e0 + r * 256;
-              if (e < d) {
-                xv[r] = *reinterpret_cast<const uint4*>(x + e);
-                gv[r] = *reinterpret_cast<const uint4*>(wg + e);
-                uv[r] = *reinterpret_cast<const uint4*>(wu + e);
+              if (e < d) {  // the piece of elements e .. e + 7 of the operand row and of the channel's two weight rows
+                xv[r] = *reinterpret_cast<const uint4*>(p.a_op + act_piece_offset(p.Mpad, b, e >> 3));
+                gv[r] = *reinterpret_cast<const uint4*>(p.w_gu + nk_piece_offset(p.R, p.chunks, 2 * j, e >> 6, (e >> 3) & 7));
+                uv[r] = *reinterpret_cast<const uint4*>(p.w_gu + nk_piece_offset(p.R, p.chunks, 2 * j + 1, e >> 6, (e >> 3) & 7));
               }
             }
 #pragma unroll
@@ -214,8 +210,6 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
     return key[i] > key_thr ? 2 : (key[i] == key_thr ? 1 : 0);
   };
   // masked activations as bf16 high + low parts, 8 channels (16 bytes) at a time, and the live flags
-  uint16_t* th = p.t_hi + (size_t)b * ff;
-  uint16_t* tl = p.t_lo + (size_t)b * ff;
   uint32_t hw[4], lw[4];
   bool any = false;
   auto emit = [&](int i, bool keep, int) {
@@ -236,9 +230,10 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
       lw[e >> 1] |= (uint32_t)lv << 16;
     }
     if (j0 + i < ff) p.keep[(size_t)b * ff + j0 + i] = keep ? 1 : 0;
-    if (e == 7 && j0 + i < ff) {
-      *reinterpret_cast<uint4*>(th + j0 + i - 7) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-      *reinterpret_cast<uint4*>(tl + j0 + i - 7) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+    if (e == 7 && j0 + i < ff) {  // channels j0 + i - 7 .. j0 + i are one piece of the packed operand
+      unsigned char* dst = p.t_op + act_piece_offset(2 * p.Mpad, b, (j0 + i) >> 3);
+      *reinterpret_cast<uint4*>(dst) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+      *reinterpret_cast<uint4*>(dst + (size_t)p.Mpad * 128) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
     }
     if (((j0 + i) & 31) == 31 || i == KPT - 1) {  // end of a 32-channel granule or of this thread's range
       if (any && j0 + i < ff) p.live[(j0 + i) >> 5] = 1;
@@ -364,9 +359,10 @@ __global__ void __launch_bounds__(CM_THREADS) channel_select_multi_kernel(const 
       sm.local_idx[atomicAdd(&sm.n_local, 1)] = j0 + e;
     }
   }
-  if (in) {
-    *reinterpret_cast<uint2*>(p.t_hi + (size_t)b * ff + j0) = make_uint2(hw[0], hw[1]);
-    *reinterpret_cast<uint2*>(p.t_lo + (size_t)b * ff + j0) = make_uint2(lw[0], lw[1]);
+  if (in) {  // four channels: half a piece of the packed operand
+    unsigned char* dst = p.t_op + act_piece_offset(2 * p.Mpad, b, j0 >> 3) + (j0 & 7) * 2;
+    *reinterpret_cast<uint2*>(dst) = make_uint2(hw[0], hw[1]);
+    *reinterpret_cast<uint2*>(dst + (size_t)p.Mpad * 128) = make_uint2(lw[0], lw[1]);
     *reinterpret_cast<uint32_t*>(p.keep + (size_t)b * ff + j0) = kw;
     if (any) p.live[j0 >> 5] = 1;
   }
@@ -382,21 +378,19 @@ __global__ void __launch_bounds__(CM_THREADS) channel_select_multi_kernel(const 
     const double sc = (double)p.scale[b];
     // the token's operand row, shared by all candidates of the CTA
     for (int e = tid * 8; e < d; e += CM_THREADS * 8)
-      *reinterpret_cast<uint4*>(sm.x + e) = *reinterpret_cast<const uint4*>(p.a_op + (size_t)b * d + e);
+      *reinterpret_cast<uint4*>(sm.x + e) = *reinterpret_cast<const uint4*>(p.a_op + act_piece_offset(p.Mpad, b, e >> 3));
     __syncthreads();
     for (int c = warp; c < n_local; c += WARPS) {
       const int j = sm.local_idx[c];
-      const uint16_t* wg = p.w_gate + (size_t)j * d;
-      const uint16_t* wu = p.w_up + (size_t)j * d;
       float gh = 0.f, gl = 0.f, uh = 0.f, ul = 0.f;
       for (int e0 = lane * 8; e0 < d; e0 += 2048) {  // eight 256-wide slices of both rows per round, loads before uses
         uint4 gv[8], uv[8];
 #pragma unroll
         for (int r = 0; r < 8; ++r) {
           const int e = e0 + r * 256;
-          if (e < d) {
-            gv[r] = *reinterpret_cast<const uint4*>(wg + e);
-            uv[r] = *reinterpret_cast<const uint4*>(wu + e);
+          if (e < d) {  // the piece of elements e .. e + 7 of the channel's gate row and of its up row
+            gv[r] = *reinterpret_cast<const uint4*>(p.w_gu + nk_piece_offset(p.R, p.chunks, 2 * j, e >> 6, (e >> 3) & 7));
+            uv[r] = *reinterpret_cast<const uint4*>(p.w_gu + nk_piece_offset(p.R, p.chunks, 2 * j + 1, e >> 6, (e >> 3) & 7));
           }
         }
 #pragma unroll
@@ -464,8 +458,9 @@ __global__ void __launch_bounds__(CM_THREADS) channel_select_multi_kernel(const 
     if (rank < need) {
       const float tv = p.t[(size_t)b * ff + j];
       const uint16_t hv = f2bf(tv);
-      p.t_hi[(size_t)b * ff + j] = hv;
-      p.t_lo[(size_t)b * ff + j] = f2bf(tv - bf2f(hv));
+      uint16_t* dst = reinterpret_cast<uint16_t*>(p.t_op + act_piece_offset(2 * p.Mpad, b, j >> 3) + (j & 7) * 2);
+      dst[0] = hv;
+      dst[(size_t)p.Mpad * 64] = f2bf(tv - bf2f(hv));
       p.keep[(size_t)b * ff + j] = 1;
       p.live[j >> 5] = 1;
     }
@@ -494,11 +489,13 @@ __global__ void __launch_bounds__(THREADS) channel_list_kernel(const unsigned ch
 void launch_channel_select(const ChannelSelectArgs& a, cudaStream_t st) {
   ChanDev c;
   c.d = a.d; c.ff = a.ff; c.p_permille = a.p_permille; c.g = a.g; c.u = a.u; c.t = a.t;
-  c.a_op = static_cast<const uint16_t*>(a.a_op); c.scale = a.scale;
-  c.w_gate = static_cast<const uint16_t*>(a.w_gate); c.w_up = static_cast<const uint16_t*>(a.w_up);
+  c.a_op = static_cast<const unsigned char*>(a.a_op); c.scale = a.scale;
+  c.w_gu = static_cast<const unsigned char*>(a.w_gate_up);
+  const NKGeom geo = nk_geom_gate_up(a.ff, a.d, sm_count());
+  c.R = geo.R; c.chunks = geo.chunks; c.Mpad = pad_rows(a.B);
   c.sel = a.sel; c.cand_val = a.cand_val; c.cand_idx = a.cand_idx; c.keep = a.keep;
   c.kept_ch = a.kept_ch; c.scratch_idx = a.scratch_idx; c.kept_cnt = a.kept_cnt;
-  c.t_hi = static_cast<uint16_t*>(a.t_hi); c.t_lo = static_cast<uint16_t*>(a.t_lo);
+  c.t_op = static_cast<unsigned char*>(a.t_op);
   c.live = a.live; c.status = a.status;
   const dim3 mgrid((a.ff + CM_SLICE - 1) / CM_SLICE, a.B);
   SOL_LAUNCH("channel_select", channel_select_multi_kernel, mgrid, dim3(CM_THREADS), 0, st, c);

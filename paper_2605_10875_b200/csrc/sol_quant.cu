@@ -30,7 +30,8 @@ template <bool IN_F32>
 __global__ void __launch_bounds__(NQ_THREADS)
 norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, int ksplit, size_t part_stride,
                   float* __restrict__ sum_out, const uint16_t* __restrict__ gamma, float eps,
-                  const int32_t* __restrict__ bits, int d, uint16_t* __restrict__ a_op, float* __restrict__ scale,
+                  const int32_t* __restrict__ bits, int d, uint16_t* __restrict__ a_op, int a_op_rows,
+                  float* __restrict__ scale,
                   float* __restrict__ xn, int8_t* __restrict__ codes, int* __restrict__ status,
                   uint32_t* __restrict__ clear, int clear_words) {
   __shared__ float sh[NQ_THREADS / 32];
@@ -156,7 +157,9 @@ norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, i
       uint4 w;
       w.x = pack_bf16(c[0], c[1]); w.y = pack_bf16(c[2], c[3]);
       w.z = pack_bf16(c[4], c[5]); w.w = pack_bf16(c[6], c[7]);
-      reinterpret_cast<uint4*>(a_op + (size_t)row * d)[v] = w;
+      // vector v is the 16-byte piece of elements 8 v .. 8 v + 7: its place in the packed operand layout, or in the plain row
+      if (a_op_rows > 0) *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(a_op) + act_piece_offset(a_op_rows, row, v)) = w;
+      else reinterpret_cast<uint4*>(a_op + (size_t)row * d)[v] = w;
     }
     if (codes != nullptr) {
       int q[NQ_VEC];
@@ -175,11 +178,11 @@ void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st) {
   if (a.in_f32)
     SOL_LAUNCH("norm_quant", norm_quant_kernel<true>, dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit, stride,
                a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d, static_cast<uint16_t*>(a.a_op),
-               a.scale, a.xn, a.codes, a.status, a.clear, a.clear_words);
+               a.a_op_rows, a.scale, a.xn, a.codes, a.status, a.clear, a.clear_words);
   else
     SOL_LAUNCH("norm_quant", norm_quant_kernel<false>, dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit, stride,
                a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d, static_cast<uint16_t*>(a.a_op),
-               a.scale, a.xn, a.codes, a.status, a.clear, a.clear_words);
+               a.a_op_rows, a.scale, a.xn, a.codes, a.status, a.clear, a.clear_words);
 }
 
 }  // namespace sol

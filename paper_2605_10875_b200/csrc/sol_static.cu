@@ -99,6 +99,7 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
   a.out_bf16 = out_bf16;
   a.out_hi = nullptr;
   a.out_lo = nullptr;
+  a.out_rows = 0;
   a.status = reinterpret_cast<int*>(base);
   sol::launch_attention(a, st);
   if (status_out != nullptr)

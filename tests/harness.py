@@ -78,18 +78,34 @@ def make_case_kv(cfg: dict, seq_lens: np.ndarray, seed=0, layer=0, shuffle=None,
     return k_pool, v_pool, table
 
 
+def pack_layer(shape, plain: dict) -> dict:
+    """Packs the four matrices of a layer (device bf16 tensors, row-major) with sol_pack_weights; returns the
+    packed device buffers and the gains.  The row-major tensors can be dropped afterwards."""
+    out = {"gamma1": plain["gamma1"], "gamma2": plain["gamma2"]}
+    for name, kind, a, b in (("w_qkv", sol.W_QKV, "w_qkv", None), ("w_o", sol.W_O, "w_o", None),
+                             ("w_gate_up", sol.W_GATE_UP, "w_gate", "w_up"), ("w_down", sol.W_DOWN, "w_down_t", None)):
+        n = sol.packed_weight_bytes(shape, kind)
+        assert n > 0, (name, "unsupported shape")
+        buf = torch.empty(n, dtype=torch.uint8, device=plain[a].device)
+        sol.pack_weights(shape, kind, plain[a], plain[b] if b else None, buf, n)
+        out[name] = buf
+    torch.cuda.synchronize()
+    return out
+
+
 @dataclass
 class DeviceWeights:
-    tensors: dict
+    tensors: dict  # packed matrices + gains
 
     def struct(self):
         t = self.tensors
-        return sol.make_weights(t["w_qkv"], t["w_o"], t["w_gate"], t["w_up"], t["w_down_t"], t["gamma1"], t["gamma2"])
+        return sol.make_weights(t["w_qkv"], t["w_o"], t["w_gate_up"], t["w_down"], t["gamma1"], t["gamma2"])
 
 
-def device_weights(w: synth.LayerTensors) -> DeviceWeights:
-    return DeviceWeights({n: dev_bf16(getattr(w, n)) for n in
-                          ("w_qkv", "w_o", "w_gate", "w_up", "w_down_t", "gamma1", "gamma2")})
+def device_weights(w: synth.LayerTensors, shape) -> DeviceWeights:
+    """Uploads a layer's row-major weights and packs them for the library (shape: a sol shape of the layer)."""
+    plain = {n: dev_bf16(getattr(w, n)) for n in ("w_qkv", "w_o", "w_gate", "w_up", "w_down_t", "gamma1", "gamma2")}
+    return DeviceWeights(pack_layer(shape, plain))
 
 
 def oracle_weights(w: synth.LayerTensors) -> O.LayerWeights:
@@ -136,7 +152,7 @@ def gpu_mlp(shape, x_bf16: np.ndarray, w: DeviceWeights, p_permille, ws: Optiona
     kept_ch = torch.full((B, ff), -1, dtype=torch.int32, device=DEV)
     kept_cnt = torch.full((B,), -1, dtype=torch.int32, device=DEV)
     t = w.tensors
-    sol.pruned_swiglu_mlp(shape, dev_bf16(x_bf16), t["w_gate"], t["w_up"], t["w_down_t"], B, dev_i32(p_permille), out,
+    sol.pruned_swiglu_mlp(shape, dev_bf16(x_bf16), t["w_gate_up"], t["w_down"], B, dev_i32(p_permille), out,
                           kept_ch, kept_cnt, ws.buf, ws.bytes)
     torch.cuda.synchronize()
     st = ws.status()

@@ -68,14 +68,14 @@ def test_bad_arguments_are_rejected_before_any_launch():
     bad = _shape("tiny", head_dim=96)
     assert sol.sparse_decode_attn(bad, FAKE, kv, 4, FAKE, FAKE, None, None, FAKE, 1 << 30, check=False) \
         == sol.SOL_ERR_UNSUPPORTED
-    assert sol.pruned_swiglu_mlp(sh, FAKE, FAKE, FAKE, FAKE, 4, FAKE, FAKE, None, None, FAKE, 16, check=False) \
+    assert sol.pruned_swiglu_mlp(sh, FAKE, FAKE, FAKE, 4, FAKE, FAKE, None, None, FAKE, 16, check=False) \
         == sol.SOL_ERR_WORKSPACE_TOO_SMALL
-    assert sol.pruned_swiglu_mlp(sh, FAKE, FAKE, None, FAKE, 4, FAKE, FAKE, None, None, FAKE, 1 << 30, check=False) \
+    assert sol.pruned_swiglu_mlp(sh, FAKE, None, FAKE, 4, FAKE, FAKE, None, None, FAKE, 1 << 30, check=False) \
         == sol.SOL_ERR_INVALID_ARG
-    w = sol.make_weights(*([FAKE] * 7))
+    w = sol.make_weights(*([FAKE] * 6))
     assert sol.decode_layer(sh, w, kv, 4, FAKE, FAKE, FAKE, FAKE, FAKE, None, FAKE, 64, check=False) \
         == sol.SOL_ERR_WORKSPACE_TOO_SMALL
-    w_bad = sol.make_weights(FAKE, FAKE, None, FAKE, FAKE, FAKE, FAKE)
+    w_bad = sol.make_weights(FAKE, FAKE, None, FAKE, FAKE, FAKE)
     assert sol.decode_layer(sh, w_bad, kv, 4, FAKE, FAKE, FAKE, FAKE, FAKE, None, FAKE, 1 << 30, check=False) \
         == sol.SOL_ERR_INVALID_ARG
     assert sol.decode_step(sh, [w], [kv], 200, FAKE, FAKE, None, FAKE, FAKE, FAKE, FAKE, 1 << 30, check=False) \
@@ -88,7 +88,7 @@ def test_bad_arguments_are_rejected_before_any_launch():
 def test_host_entry_validates_actions():
     sh = _shape("tiny")
     kv = sol.make_kv(FAKE, FAKE, FAKE, FAKE, 8, 32)
-    w = sol.make_weights(*([FAKE] * 7))
+    w = sol.make_weights(*([FAKE] * 6))
     h = np.zeros((2, 256), np.uint16)
     out = np.zeros((2, 256), np.uint16)
     i32 = lambda *v: np.array(v, np.int32)
@@ -108,3 +108,21 @@ def test_binding_fails_loudly_without_the_library(monkeypatch):
     monkeypatch.setattr(sol, "LIB_PATH", "/nonexistent/libsol.so")
     with pytest.raises(RuntimeError):
         sol.lib()
+
+
+def test_packed_weight_sizes_and_rejections():
+    """Packed sizes are whole tiles of 128-byte rows; bad arguments are refused before any launch."""
+    before = sol.launch_count()
+    sh = _shape("llama1b_layer")
+    d, ff = 2048, 8192
+    assert sol.packed_weight_bytes(sh, sol.W_QKV) == (32 + 16) * 64 * d * 2        # 3072 rows: 24 tiles of 128, no padding
+    assert sol.packed_weight_bytes(sh, sol.W_O) == d * d * 2
+    assert sol.packed_weight_bytes(sh, sol.W_DOWN) == ff * d * 2
+    gu = sol.packed_weight_bytes(sh, sol.W_GATE_UP)
+    assert gu >= 2 * ff * d * 2 and gu % (128 * 8) == 0 and gu < 2 * ff * d * 2 * 1.1  # tiles padded to whole rows
+    assert sol.packed_weight_bytes(sh, 7) == 0
+    assert sol.packed_weight_bytes(_shape("tiny", d_model=300), sol.W_QKV) == 0
+    assert sol.pack_weights(sh, sol.W_GATE_UP, FAKE, None, FAKE, gu, check=False) == sol.SOL_ERR_INVALID_ARG
+    assert sol.pack_weights(sh, sol.W_DOWN, FAKE, None, FAKE, 16, check=False) == sol.SOL_ERR_WORKSPACE_TOO_SMALL
+    assert sol.pack_weights(sh, 9, FAKE, None, FAKE, gu, check=False) == sol.SOL_ERR_INVALID_ARG
+    assert sol.launch_count() == before

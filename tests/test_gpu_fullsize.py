@@ -70,7 +70,7 @@ class SampledStack:
         self.table = np.where(table < 0, 0, table).astype(np.int32)
         self.max_pages = table.shape[1]
         self.weights = [synth.make_layer_weights(cfg, seed, l) for l in range(n_layers)]
-        self.dws = [H.device_weights(w) for w in self.weights]
+        self.dws = [H.device_weights(w, self.shape) for w in self.weights]
         self.lens_dev = H.dev_i32(start_lens)
         table_dev = H.dev_i32(self.table)
         self.dkvs = []

@@ -178,7 +178,7 @@ def _mlp_case(cfg, B, p, seed=0, mutate=None):
         mutate(w)
     x = synth.make_hidden(cfg, seed, B)
     x = synth.to_bf16(synth.bf16_to_f32(x) * np.float32(1.0))
-    dw = H.device_weights(w)
+    dw = H.device_weights(w, shape)
     out, kept, st = H.gpu_mlp(shape, x, dw, p)
     out_o, kept_o, t_o = O.pruned_swiglu_mlp(O.bf16_to_f64(x), w.w_gate, w.w_up, w.w_down_t, p)
     assert st[0] == 0 and st[2] == 0, st
@@ -340,7 +340,7 @@ def check_layer(cfg, seq_lens, r, p, b, seed=0, n_sink=0, n_window=1, sample=Non
     k_pool, v_pool, table = H.make_case_kv(cfg, seq_lens, seed)
     h_in = synth.make_hidden(cfg, seed, B)
     kv = H.device_kv(k_pool, v_pool, table, seq_lens)
-    out, taps, st = H.gpu_layer(shape, H.device_weights(w), kv, h_in, r, p, b)
+    out, taps, st = H.gpu_layer(shape, H.device_weights(w, shape), kv, h_in, r, p, b)
     assert st[0] == 0 and st[1] == 0 and st[2] == 0, st
     tab = np.where(table < 0, 0, table)
     k_gpu, v_gpu = H.host_u16(kv.k_pool), H.host_u16(kv.v_pool)
@@ -414,7 +414,7 @@ def _step_case(cfg, n_layers, seq_lens, r, p, b, seed=0):
     ws_ = [synth.make_layer_weights(cfg, seed, l) for l in range(n_layers)]
     pools = [H.make_case_kv(cfg, seq_lens, seed, l) for l in range(n_layers)]
     h_in = synth.make_hidden(cfg, seed, B)
-    dws = [H.device_weights(w) for w in ws_]
+    dws = [H.device_weights(w, shape) for w in ws_]
     dkvs = [H.device_kv(k, v, t, seq_lens) for (k, v, t) in pools]
     return shape, oshape, ws_, pools, h_in, dws, dkvs, seq_lens
 
@@ -464,7 +464,7 @@ def test_consecutive_steps_append_to_the_cache():
     ws_ = [synth.make_layer_weights(cfg, 5, l) for l in range(L)]
     table, n_pages = synth.make_page_table(start, True, 5, spare_tokens=steps)
     pools = [synth.make_kv_pool(cfg, n_pages, 5, l) for l in range(L)]
-    dws = [H.device_weights(w) for w in ws_]
+    dws = [H.device_weights(w, shape) for w in ws_]
     dkvs = [H.device_kv(k, v, table, start) for (k, v) in pools]
     ws = H.Workspace(shape, B, table.shape[1])
     rng = np.random.default_rng(5)
@@ -500,7 +500,7 @@ def test_repeat_calls_are_bit_identical():
     r, p, b = synth.draw_actions(cfg, 1)
     shape, _ = H.make_shapes(cfg)
     lens = synth.make_contexts(cfg, 0)
-    w = H.device_weights(synth.make_layer_weights(cfg, 0))
+    w = H.device_weights(synth.make_layer_weights(cfg, 0), shape)
     k_pool, v_pool, table = H.make_case_kv(cfg, lens, 0)
     h_in = synth.make_hidden(cfg, 0)
     outs = []
@@ -510,6 +510,52 @@ def test_repeat_calls_are_bit_identical():
         outs.append((out, taps["kept_idx"].copy(), taps["kept_ch"].copy(), taps["h_out"].copy()))
     for a, c in zip(outs[0], outs[1]):
         assert np.array_equal(a, c)
+
+
+# ------------------------------------------------------------ packed weights ---
+
+
+def _np_pack_rows(rows: np.ndarray, R: int) -> np.ndarray:
+    """The documented packed layout, written out with NumPy: tiles of R rows, 64-wide k chunks, every row 128
+    bytes whose 16-byte pieces sit at position (piece ^ (row & 7)); tiles padded with zero rows."""
+    n, K = rows.shape
+    tiles, chunks = -(-n // R), K // 64
+    padded = np.zeros((tiles * R, K), np.uint16)
+    padded[:n] = rows
+    src = padded.reshape(tiles, R, chunks, 8, 8)  # tile, row, chunk, piece, element
+    out = np.zeros((tiles, chunks, R, 8, 8), np.uint16)
+    r = np.arange(R)
+    for q in range(8):
+        out[:, :, r, q ^ (r & 7), :] = src[:, r, :, q, :].transpose(1, 2, 0, 3)  # (row, tile, chunk, element) in
+    return out.reshape(-1)
+
+
+def test_pack_weights_is_the_documented_permutation():
+    cfg = dict(TINY, d_model=512, d_ff=2048 + 32)  # d_ff: tiles and 64-channel blocks with a ragged end
+    shape, _ = H.make_shapes(cfg)
+    w = synth.make_layer_weights(cfg, 3)
+    packed = H.device_weights(w, shape).tensors
+    got = {k: H.host_u16(v.view(torch.bfloat16)) for k, v in packed.items() if k.startswith("w_")}
+    assert np.array_equal(got["w_qkv"], _np_pack_rows(w.w_qkv, 128))
+    assert np.array_equal(got["w_o"], _np_pack_rows(w.w_o, 128))
+    # gate and up share one matrix whose rows alternate gate_c, up_c; channels per tile: the smallest multiple of
+    # 4 that covers d_ff in a whole number of waves of one tile per SM, at most 64
+    sms, ff = torch.cuda.get_device_properties(0).multi_processor_count, cfg["d_ff"]
+    c = next(-(-(-(-ff // (sms * wv))) // 4) * 4 for wv in range(1, 65) if -(-(-(-ff // (sms * wv))) // 4) * 4 <= 64)
+    gu = np.empty((2 * ff, cfg["d_model"]), np.uint16)
+    gu[0::2], gu[1::2] = w.w_gate, w.w_up
+    assert np.array_equal(got["w_gate_up"], _np_pack_rows(gu, 2 * c))
+    # W_down^T: [128-column slab][64-channel block][column half][64 channels][128 bytes], pieces at (piece ^ (channel & 7))
+    d = cfg["d_model"]
+    jblocks = -(-ff // 64)
+    padded = np.zeros((jblocks * 64, d), np.uint16)
+    padded[:ff] = w.w_down_t
+    src = padded.reshape(jblocks, 64, d // 128, 2, 8, 8)  # block, channel, slab, half, piece, element
+    want = np.zeros((d // 128, jblocks, 2, 64, 8, 8), np.uint16)
+    ch = np.arange(64)
+    for q in range(8):
+        want[:, :, :, ch, q ^ (ch & 7), :] = src[:, ch, :, :, q, :].transpose(2, 1, 3, 0, 4)  # (channel, block, slab, half, element) in
+    assert np.array_equal(got["w_down"], want.reshape(-1))
 
 
 # ------------------------------------------------------- device-side time-out ---
