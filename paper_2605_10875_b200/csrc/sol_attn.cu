@@ -1470,7 +1470,7 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   pd.row_hist = a.row_hist; pd.row_ctl = a.row_ctl; pd.seg_pub = a.seg_pub;
   pd.nseg_max = attn_select_segs(a.kv.max_pages_per_seq, PAGE);
   pd.plan = a.plan; pd.r_permille = a.r_permille; pd.split_len = attn_split_len(hd);
-  pd.target_items = sm_count() * (hd == 64 ? 12 : 8) / 4;  // a quarter of the pass-2 warps resident at once: few partials per row
+  pd.target_items = sm_count() * (hd == 64 ? 12 : 8);  // the pass-2 warps resident at once
   pd.max_item_chunks = 1024 / attn_split_len(hd);
   SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(Hkv, a.B), dim3(PREP_THREADS), 0, st, pd);
 

@@ -32,7 +32,8 @@
 
 namespace sol {
 
-constexpr int UM_THREADS = 192;      // warps 0-3: epilogue, warp 4: producer, warp 5: MMA issuer + TMEM owner
+constexpr int UM_THREADS = 320;      // warps 0-7: epilogue (two per 32 accumulator lanes), warp 8: producer, warp 9: MMA issuer + TMEM owner
+constexpr int UM_PRODUCER = 8, UM_MMA = 9;
 constexpr int UM_MAX_STAGES = 8;
 constexpr int UM_TILE_SPAN = 16384;  // bytes one 128-row operand read spans from the start of a chunk tile
 constexpr int UM_SMEM_BUDGET = 204 * 1024;
@@ -91,7 +92,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
     mbar_init(&bars->accum, 1);
     fence_mbar_init();
   }
-  if (warp == 5) tmem_alloc(&bars->tmem_base, p.tmem_cols);
+  if (warp == UM_MMA) tmem_alloc(&bars->tmem_base, p.tmem_cols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -105,7 +106,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
   const unsigned char* w_src = p.w + ((size_t)tile * p.chunks + ch0) * w_tile;  // this tile's chunks are contiguous
   const unsigned char* x_src = p.x + (size_t)ch0 * x_tile;                     // and so are the activation chunks
 
-  if (warp == 4) {
+  if (warp == UM_PRODUCER) {
     // -------------------------------- producer -------------------------------
     // Weights do not depend on earlier kernels: the first ring of weight tiles is requested before
     // pdl_wait(), the activation tiles of those stages after it.
@@ -131,7 +132,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
         bulk_g2s(st + p.cps * w_tile, x_src + (size_t)it * p.cps * x_tile, p.cps * x_tile, &bars->full[s]);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == UM_MMA) {
     // ------------------------------- MMA issuer ------------------------------
     // The mbarrier wait orders the copies before the MMA reads; no tcgen05 fence is needed per stage.
     const uint32_t idesc = umma_idesc_bf16_m128(nb_rows, 0, 0);
@@ -164,12 +165,14 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
   } else {
     // -------------------------------- epilogue -------------------------------
     pdl_wait();  // the epilogue reads scales and overwrites buffers earlier kernels used
-    if (warp * 32 < p.R) {
+    // warps w and w + 4 share the accumulator lanes 32 (w % 4) .. and take alternate groups of 16 tokens
+    const int quarter = warp & 3, half = warp >> 2;
+    if (quarter * 32 < p.R) {
       const bool ok = mbar_wait(&bars->accum, 0, p.status);
       tc_fence_after();
-      const int r = warp * 32 + lane;  // row of the tile = accumulator lane
-      const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
-      for (int c0 = 0; c0 < p.Mpad && ok; c0 += 16) {
+      const int r = quarter * 32 + lane;  // row of the tile = accumulator lane
+      const uint32_t tl = tmem + ((uint32_t)(quarter * 32) << 16);
+      for (int c0 = half * 16; c0 < p.Mpad && ok; c0 += 32) {
         float v[16];
         tmem_ld16(tl + c0, v);
         if (p.n_b == 2) {  // high-part and low-part products
@@ -229,7 +232,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem, p.tmem_cols);
+  if (warp == UM_MMA) tmem_dealloc(tmem, p.tmem_cols);
 }
 
 // ============================================================================
@@ -268,7 +271,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_down_kernel(const DownDev 
     bars->n_issued = 0;
     fence_mbar_init();
   }
-  if (warp == 5) tmem_alloc(&bars->tmem_base, p.tmem_cols);
+  if (warp == UM_MMA) tmem_alloc(&bars->tmem_base, p.tmem_cols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -280,7 +283,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_down_kernel(const DownDev 
   const int jb0 = (int)(((long long)jblocks * chunk) / p.chunks);
   const int jb1 = (int)(((long long)jblocks * (chunk + 1)) / p.chunks);
 
-  if (warp == 4) {
+  if (warp == UM_PRODUCER) {
     if (lane == 0) {
       int it = 0;
       for (int jb = jb0; jb < jb1; ++jb) {
@@ -295,7 +298,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_down_kernel(const DownDev 
         bulk_g2s(st + UM_TILE_SPAN, p.t + (size_t)jb * t_tile, t_tile, &bars->full[s]);  // high rows then low rows
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == UM_MMA) {
     const uint32_t idesc = umma_idesc_bf16_m128(2 * p.Mpad, 1, 0);
     bool acc = false, ok = true;
     int it = 0;
@@ -329,10 +332,11 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_down_kernel(const DownDev 
     const bool ok = mbar_wait(&bars->accum, 0, p.status);
     tc_fence_after();
     const bool any = *reinterpret_cast<volatile int*>(&bars->n_issued) > 0;
-    const int n = slab * 128 + warp * 32 + lane;
-    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
+    const int quarter = warp & 3, half = warp >> 2;  // as in umma_nk: two warps per 32 accumulator lanes
+    const int n = slab * 128 + quarter * 32 + lane;
+    const uint32_t tl = tmem + ((uint32_t)(quarter * 32) << 16);
     float* out = p.partial + (size_t)chunk * p.Mpad * p.d;
-    for (int c0 = 0; c0 < p.Mpad && ok; c0 += 16) {
+    for (int c0 = half * 16; c0 < p.Mpad && ok; c0 += 32) {
       float v[16];
       if (any) {
         float w2[16];
@@ -353,7 +357,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_down_kernel(const DownDev 
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem, p.tmem_cols);
+  if (warp == UM_MMA) tmem_dealloc(tmem, p.tmem_cols);
 }
 
 // ============================================================================
@@ -457,7 +461,7 @@ void launch_gemm_nk(const GemmNK& g, GemmEpilogue epi, cudaStream_t st) {
   d.ksplit = epi == EPI_PARTIAL ? nk_ksplit(g.N, g.K) : 1;
   const int chunk_bytes = 128 * (d.R + d.n_b * d.Mpad);
   int cps = d.ksplit > 1 ? 1 : 4;
-  while (cps > 1 && (cps * chunk_bytes > 36 * 1024 || d.chunks % cps)) cps >>= 1;
+  while (cps > 1 && (cps * chunk_bytes > 64 * 1024 || d.chunks % cps)) cps >>= 1;  // few, large stages: every stage costs a commit
   d.cps = cps;
   const int stage_bytes = cps * chunk_bytes;
   const int iters = (d.chunks / d.ksplit + (d.chunks % d.ksplit ? 1 : 0)) / cps;  // of the longest slice
