@@ -24,7 +24,9 @@ Readings taken where the paper is silent or the benchmark spec overrides it:
   * b = 16 is bf16 passthrough (the paper: "q >= 16 returns the input
     unchanged");
   * the quantizer is applied to the inputs of the QKV and gate/up
-    projections (the paper applies the same operator to the MLP output);
+    projections (the task's default placement); the paper's own placement,
+    the MLP output before the residual add, is PLACE_MLP_OUTPUT, and widths
+    of 9..15 bits (int16 codes) are supported in both;
   * token selection is exact top-k per (sequence, kv-head) on the q.k score
     summed over the query group (the paper uses Quest page bounds per head);
     forced-keep tokens (sinks, recent window; default: only the newest
@@ -176,33 +178,49 @@ def quantize_per_token(x32: np.ndarray, bits: int):
     code_j = clip(round(x_j / s), -q_max, q_max), x_hat_j = code_j * s.
 
     x32 is one token's float32 vector.  Both divisions are IEEE float32 and
-    the rounding is to nearest-even.  Returns (codes int8, scale float32,
-    x_hat float64).  bits == 16: passthrough to bf16; codes are all zero and
-    scale is 1.
+    the rounding is to nearest-even.  Returns (codes, scale float32, x_hat
+    float64); codes are int8 up to 8 bits and int16 from 9 to 15 bits (the
+    paper's action tables use widths up to 15).  bits == 16: passthrough to
+    bf16; codes are all zero and scale is 1.
     """
     x32 = np.asarray(x32, dtype=np.float32)
     if bits == 16:
         xh = bf16_to_f64(f32_to_bf16_rne(x32))
         return np.zeros(x32.shape, np.int8), np.float32(1.0), xh
-    if not 2 <= bits <= 8:
+    if not 2 <= bits <= 15:
         raise ValueError("unsupported bit-width")
+    ctype = np.int8 if bits <= 8 else np.int16
     q_max = (1 << (bits - 1)) - 1
     a = np.float32(np.max(np.abs(x32))) if x32.size else np.float32(0)
     if a == 0:
-        return np.zeros(x32.shape, np.int8), np.float32(0.0), np.zeros(x32.shape, np.float64)
+        return np.zeros(x32.shape, ctype), np.float32(0.0), np.zeros(x32.shape, np.float64)
     s = np.float32(a) / np.float32(q_max)  # IEEE fp32 division
     ratio = (x32 / s).astype(np.float32)  # IEEE fp32 division, element-wise
     c = np.clip(np.rint(ratio), -q_max, q_max)
-    codes = c.astype(np.int8)
+    codes = c.astype(ctype)
     x_hat = codes.astype(np.float64) * np.float64(s)
     return codes, np.float32(s), x_hat
+
+
+def fake_quant_mlp_output(z: np.ndarray, bits: int):
+    """The paper's own placement of the quantizer (appendix "Activation
+    quantization", "What is quantized"): the MLP block's output z, the update
+    of the residual stream, is quantized and dequantized per token before it is
+    added back; the matmuls themselves run at full precision.  Same operator as
+    quantize_per_token on fl32(z); from 16 bits on z is returned unchanged
+    ("For q >= 16 we return z unchanged": no rounding at all in this placement).
+    Returns (codes, scale float32, z_hat float64)."""
+    z = np.asarray(z, np.float64)
+    if bits >= 16:
+        return np.zeros(z.shape, np.int16), np.float32(1.0), z.copy()
+    return quantize_per_token(z.astype(np.float32), bits)
 
 
 def quant_act(x_bf16: np.ndarray, bits: Sequence[int]):
     """Batched form over bf16 rows: what the stand-alone quantize call returns."""
     x_bf16 = np.asarray(x_bf16, dtype=np.uint16)
     B, d = x_bf16.shape
-    codes = np.zeros((B, d), np.int8)
+    codes = np.zeros((B, d), np.int16 if any(8 < int(b) < 16 for b in bits) else np.int8)
     scales = np.zeros(B, np.float32)
     x_hat = np.zeros((B, d), np.float64)
     for i in range(B):
@@ -382,7 +400,7 @@ def norm_and_quantize(h: np.ndarray, gamma_bf16: np.ndarray, eps: float, bits: S
     B, d = h.shape
     gamma = bf16_to_f64(gamma_bf16)
     xn = np.zeros((B, d), np.float32)
-    codes = np.zeros((B, d), np.int8)
+    codes = np.zeros((B, d), np.int16 if any(8 < int(b) < 16 for b in bits) else np.int8)
     scales = np.zeros(B, np.float32)
     x_hat = np.zeros((B, d))
     for i in range(B):
@@ -400,9 +418,18 @@ def append_kv(shape: Shape, kv: PagedKV, i: int, k_bf16: np.ndarray, v_bf16: np.
     kv.v_pool[page, :, slot, :] = v_bf16
 
 
+PLACE_PROJ_INPUTS = 0  # the task's default: the inputs of the QKV and gate/up projections are quantized
+PLACE_MLP_OUTPUT = 1   # the paper's: the MLP output is fake-quantized before the residual add
+
+
 def decode_layer(shape: Shape, w: LayerWeights, kv: PagedKV, h_in: np.ndarray,
-                 r_permille: Sequence[int], p_permille: Sequence[int], bits: Sequence[int]):
+                 r_permille: Sequence[int], p_permille: Sequence[int], bits: Sequence[int],
+                 placement: int = PLACE_PROJ_INPUTS):
     """One decoder layer for one new token per sequence.
+
+    placement == PLACE_MLP_OUTPUT: the projections read the normalised rows
+    through the 16-bit passthrough (bf16, the operand type of the matmuls) and
+    bits[i] acts on the MLP output instead (fake_quant_mlp_output).
 
     h_in float64 [B][d].  kv is modified in place (the newest token's k and v,
     rounded to bf16, are written before attention reads the cache).  No other
@@ -412,8 +439,9 @@ def decode_layer(shape: Shape, w: LayerWeights, kv: PagedKV, h_in: np.ndarray,
     Hq, Hkv, hd = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
     tr = LayerTrace()
 
+    in_bits = bits if placement == PLACE_PROJ_INPUTS else [16] * B
     # attention input: RMSNorm, quantize, QKV projection
-    tr.xn1, tr.codes1, tr.scales1, x_hat = norm_and_quantize(h_in, w.gamma1, shape.rms_eps, bits)
+    tr.xn1, tr.codes1, tr.scales1, x_hat = norm_and_quantize(h_in, w.gamma1, shape.rms_eps, in_bits)
     qkv = x_hat @ bf16_to_f64(w.w_qkv).T  # [B][(Hq+2Hkv)*hd]
     q = qkv[:, : Hq * hd].reshape(B, Hq, hd)
     k = qkv[:, Hq * hd:(Hq + Hkv) * hd].reshape(B, Hkv, hd)
@@ -439,19 +467,26 @@ def decode_layer(shape: Shape, w: LayerWeights, kv: PagedKV, h_in: np.ndarray,
     tr.h_mid = h_mid
 
     # MLP input: RMSNorm, quantize; pruned SwiGLU; residual
-    tr.xn2, tr.codes2, tr.scales2, x_hat2 = norm_and_quantize(h_mid, w.gamma2, shape.rms_eps, bits)
+    tr.xn2, tr.codes2, tr.scales2, x_hat2 = norm_and_quantize(h_mid, w.gamma2, shape.rms_eps, in_bits)
     mlp, tr.kept_channels, tr.t = pruned_swiglu_mlp(x_hat2, w.w_gate, w.w_up, w.w_down_t, p_permille)
+    if placement == PLACE_MLP_OUTPUT:
+        tr.extra["z"] = mlp.copy()
+        z_codes, z_scales = [], np.zeros(B, np.float32)
+        for i in range(B):
+            c, z_scales[i], mlp[i] = fake_quant_mlp_output(mlp[i], int(bits[i]))
+            z_codes.append(c)
+        tr.extra["z_codes"], tr.extra["z_scales"] = z_codes, z_scales
     return h_mid + mlp, tr
 
 
 def decode_step(shape: Shape, layers: Sequence[LayerWeights], kvs: Sequence[PagedKV], h_in_bf16: np.ndarray,
-                r_permille, p_permille, bits):
+                r_permille, p_permille, bits, placement: int = PLACE_PROJ_INPUTS):
     """L layers with the same action tuple in every layer (the paper broadcasts
     one action across all layers at a decode step).  The residual stream is
     not rounded between layers.  Returns (h_out float64, [trace per layer])."""
     h = bf16_to_f64(h_in_bf16)
     traces = []
     for w, kv in zip(layers, kvs):
-        h, tr = decode_layer(shape, w, kv, h, r_permille, p_permille, bits)
+        h, tr = decode_layer(shape, w, kv, h, r_permille, p_permille, bits, placement)
         traces.append(tr)
     return h, traces

@@ -107,22 +107,22 @@ def test_quantizer_golden():
         assert float(s) == float(scale)
         assert np.array_equal(xh, c.astype(np.float64) * float(scale))
         n += 1
-    assert n >= 6
+    assert n >= 9
 
 
-@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 7, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 7, 8, 9, 11, 12, 15])
 def test_quantizer_properties(bits):
     rng = np.random.default_rng(bits)
     q_max = 2 ** (bits - 1) - 1
     for trial in range(20):
         x = (rng.standard_normal(257) * 10 ** rng.uniform(-3, 3)).astype(np.float32)
         c, s, xh = O.quantize_per_token(x, bits)
-        assert c.dtype == np.int8 and np.abs(c).max() <= q_max
+        assert c.dtype == (np.int8 if bits <= 8 else np.int16) and np.abs(c.astype(np.int64)).max() <= q_max
         # the scale is the correctly rounded quotient a / q_max
         a = float(np.abs(x).max())
         assert abs(float(s) - a / q_max) <= 2.0 ** -24 * a / q_max
-        # reconstruction error at most half a step (plus float32 rounding of x/s)
-        assert np.all(np.abs(x.astype(np.float64) - xh) <= 0.5 * float(s) * (1 + 2e-5))
+        # reconstruction error at most half a step (plus float32 rounding of x/s: up to q_max * 2^-24 of a step)
+        assert np.all(np.abs(x.astype(np.float64) - xh) <= 0.5 * float(s) * (1 + 2e-5) + float(s) * q_max * 2.0 ** -23)
         # the largest-magnitude element maps to +-q_max
         j = int(np.argmax(np.abs(x)))
         assert abs(int(c[j])) == q_max and np.sign(c[j]) == np.sign(x[j])
@@ -153,6 +153,38 @@ def test_quantizer_passthrough_16_bits():
     assert np.array_equal(xh2[0], O.bf16_to_f64(xb))
 
 
+def test_mlp_output_placement_of_the_quantizer():
+    """The paper's placement (appendix "Activation quantization", "What is quantized"): the MLP output is
+    quantized and dequantized before the residual add, the matmuls run at full precision, 16 bits and
+    more leave it unchanged.  Checked against torch float32 library ops on the un-quantized MLP update."""
+    import copy
+
+    shape, W, kv, h = _layer_case(31)
+    B = h.shape[0]
+    r, p, bits = [1000, 500, 250][:B], [0, 250, 500][:B], [16, 12, 5][:B]
+    out, tr = O.decode_layer(shape, W, copy.deepcopy(kv), h, r, p, bits, O.PLACE_MLP_OUTPUT)
+    # the same layer with every width at 16 in the default placement gives the un-quantized MLP update z
+    out16, tr16 = O.decode_layer(shape, W, copy.deepcopy(kv), h, r, p, [16] * B)
+    z = out16 - tr16.h_mid
+    assert np.allclose(tr.extra["z"], z, rtol=0, atol=1e-12)
+    assert np.array_equal(tr.h_mid, tr16.h_mid)
+    for i, b in enumerate(bits):
+        got = out[i] - tr.h_mid[i]
+        zi = tr.extra["z"][i]
+        if b >= 16:
+            assert np.array_equal(out[i], tr.h_mid[i] + zi)  # unchanged, not even rounded
+            continue
+        q_max = 2 ** (b - 1) - 1
+        z32 = torch.from_numpy(zi).to(torch.float32)
+        s = z32.abs().max() / q_max  # float32 division
+        want = (torch.clamp(torch.round(z32 / s), -q_max, q_max).to(torch.float64) * s.to(torch.float64)).numpy()
+        assert np.allclose(got, want, rtol=0, atol=1e-12), b
+        assert np.all(np.abs(want - zi) <= 0.5 * float(s) * (1 + 1e-3))
+        assert np.array_equal(tr.extra["z_codes"][i], np.round(want / float(s)).astype(np.int16))
+    # the inputs of the projections are not quantized in this placement: codes all zero, scales 1
+    assert not tr.codes1.any() and not tr.codes2.any() and np.all(tr.scales1 == 1) and np.all(tr.scales2 == 1)
+
+
 def test_quantizer_mixed_bits_per_example():
     rng = np.random.default_rng(2)
     xb = synth.to_bf16(rng.standard_normal((3, 64)).astype(np.float32))
@@ -160,8 +192,12 @@ def test_quantizer_mixed_bits_per_example():
     for i, b in enumerate([4, 16, 8]):
         c, s, h = O.quant_act(xb[i:i + 1], [b])
         assert np.array_equal(c[0], codes[i]) and s[0] == scales[i] and np.array_equal(h[0], xh[i])
-    with pytest.raises(ValueError):
-        O.quantize_per_token(np.ones(4, np.float32), 12)
+    for bad in (1, 17, 0):
+        with pytest.raises(ValueError):
+            O.quantize_per_token(np.ones(4, np.float32), bad)
+    # widths over 8 bits carry int16 codes
+    codes, scales, xh = O.quant_act(xb, [12, 16, 8])
+    assert codes.dtype == np.int16 and np.abs(codes[0].astype(np.int64)).max() == 2047
 
 
 # ------------------------------------------------------- rmsnorm / rope -----
