@@ -53,7 +53,14 @@ typedef struct sol_shape {
   int32_t n_sink, n_window; /* always-attended first / last tokens (the paper's sink and window
                                tokens, Method, "Policy inputs and architecture"); the task's
                                default is 0 and 1: only the newest token is forced */
+  int32_t quant_placement;  /* where bits[i] acts in a layer: SOL_QUANT_PROJ_INPUTS (0, the task's default) on the
+                               inputs of the QKV and gate/up projections, widths 2..8 and 16; SOL_QUANT_MLP_OUTPUT
+                               (1, the paper's: appendix "Activation quantization", "What is quantized") on the MLP
+                               output before the residual add, widths 2..15, 16 and more: unchanged; the
+                               projections then read bf16 rows */
 } sol_shape_t;
+#define SOL_QUANT_PROJ_INPUTS 0
+#define SOL_QUANT_MLP_OUTPUT 1
 
 /* Paged bf16 KV cache of one layer.  Pools: [num_pages][n_kv_heads][page_size][head_dim].
  * page_table: int32 [B][max_pages_per_seq], physical page of each logical page.
@@ -115,6 +122,9 @@ typedef struct sol_layer_trace {
   int32_t *kept_ch;     /* [B][d_ff] ascending */
   int32_t *kept_ch_cnt; /* [B] */
   float *h_out;         /* [B][d_model] float32 copy of the output */
+  float *z;             /* SOL_QUANT_MLP_OUTPUT only: [B][d_model] MLP output before the quantizer (float32) */
+  int16_t *z_codes;     /* SOL_QUANT_MLP_OUTPUT only: [B][d_model] its codes (0 for 16 bits) */
+  float *z_scales;      /* SOL_QUANT_MLP_OUTPUT only: [B] */
 } sol_layer_trace_t;
 
 const char *sol_status_string(sol_status_t s);
@@ -145,6 +155,11 @@ sol_status_t sol_workspace_init(void *ws, size_t ws_bytes, sol_stream_t stream);
  * d must be a multiple of 8.  Needs no workspace. */
 sol_status_t sol_quant_act(const void *x_bf16, int32_t B, int32_t d, const int32_t *bits, int8_t *codes,
                            float *scales, void *xhat_bf16, sol_stream_t stream);
+
+/* The same quantizer with int16 codes, for widths 2..15 (the paper's action tables use up to 15 bits);
+ * bits[i] >= 16: codes 0, scale 1.  No operand output. */
+sol_status_t sol_quant_act_wide(const void *x_bf16, int32_t B, int32_t d, const int32_t *bits, int16_t *codes,
+                                float *scales, sol_stream_t stream);
 
 /* Decode attention with a per-sequence keep-rate (appendix "Token sparsity",
  * "Budgeted token selection": budget ceil(kappa*K_t) clamped to [0, K_t];

@@ -23,7 +23,7 @@ SOL_ERR_DEVICE_TIMEOUT = 5
 
 EXPORTS = [
     "sol_status_string", "sol_last_cuda_error", "sol_workspace_bytes", "sol_workspace_init", "sol_quant_act",
-    "sol_packed_weight_bytes", "sol_pack_weights",
+    "sol_packed_weight_bytes", "sol_pack_weights", "sol_quant_act_wide",
     "sol_sparse_decode_attn", "sol_sparse_decode_attn_static", "sol_pruned_swiglu_mlp", "sol_decode_layer", "sol_decode_step",
     "sol_decode_step_traced", "sol_decode_step_host", "sol_read_device_status", "sol_selftest_wait_timeout", "sol_timing_enable", "sol_timing_collect",
     "sol_launch_count",
@@ -33,7 +33,8 @@ EXPORTS = [
 class SolShape(C.Structure):
     _fields_ = [("d_model", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("page_size", C.c_int32),
-                ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("n_sink", C.c_int32), ("n_window", C.c_int32)]
+                ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("n_sink", C.c_int32), ("n_window", C.c_int32),
+                ("quant_placement", C.c_int32)]
 
 
 class SolKV(C.Structure):
@@ -46,7 +47,7 @@ class SolLayerWeights(C.Structure):
 
 
 TRACE_FIELDS = ("xn1", "codes1", "scales1", "q_rot", "kept_idx", "kept_cnt", "attn_out", "h_mid", "xn2", "codes2",
-                "scales2", "t", "kept_ch", "kept_ch_cnt", "h_out")
+                "scales2", "t", "kept_ch", "kept_ch_cnt", "h_out", "z", "z_codes", "z_scales")
 
 
 class SolLayerTrace(C.Structure):
@@ -85,6 +86,8 @@ def lib() -> C.CDLL:
         L.sol_workspace_init.argtypes = [P, S, P]
         L.sol_quant_act.restype = I
         L.sol_quant_act.argtypes = [P, I, I, P, P, P, P, P]
+        L.sol_quant_act_wide.restype = I
+        L.sol_quant_act_wide.argtypes = [P, I, I, P, P, P, P]
         L.sol_sparse_decode_attn.restype = I
         L.sol_sparse_decode_attn.argtypes = [C.POINTER(SolShape), P, C.POINTER(SolKV), I, P, P, P, P, P, S, P]
         L.sol_sparse_decode_attn_static.restype = I
@@ -151,8 +154,9 @@ def last_cuda_error() -> str:
 
 
 def make_shape(d_model, n_q_heads, n_kv_heads, head_dim, d_ff, page_size=64, rms_eps=1e-5, rope_theta=0.0,
-               n_sink=0, n_window=1) -> SolShape:
-    return SolShape(d_model, n_q_heads, n_kv_heads, head_dim, d_ff, page_size, rms_eps, rope_theta, n_sink, n_window)
+               n_sink=0, n_window=1, quant_placement=0) -> SolShape:
+    return SolShape(d_model, n_q_heads, n_kv_heads, head_dim, d_ff, page_size, rms_eps, rope_theta, n_sink, n_window,
+                    quant_placement)
 
 
 def make_kv(k_pool, v_pool, page_table, seq_lens, max_pages_per_seq: int, num_pages: int) -> SolKV:
@@ -196,6 +200,16 @@ def quant_act(x_bf16, B: int, d: int, bits, codes, scales, xhat_bf16=None, strea
                             _stream(stream))
     if check:
         _check(s, "sol_quant_act")
+    return s
+
+
+QUANT_PROJ_INPUTS, QUANT_MLP_OUTPUT = 0, 1
+
+
+def quant_act_wide(x_bf16, B: int, d: int, bits, codes_i16, scales, stream=None, check=True) -> int:
+    s = lib().sol_quant_act_wide(_ptr(x_bf16), B, d, _ptr(bits), _ptr(codes_i16), _ptr(scales), _stream(stream))
+    if check:
+        _check(s, "sol_quant_act_wide")
     return s
 
 

@@ -109,6 +109,7 @@ static bool shape_ok(const sol_shape_t* s) {
   if ((s->n_q_heads * s->head_dim) % 256) return false;
   if (s->d_ff <= 0 || s->d_ff % 32 || s->d_ff > 49152) return false;
   if (s->n_sink < 0 || s->n_window < 0) return false;
+  if (s->quant_placement != SOL_QUANT_PROJ_INPUTS && s->quant_placement != SOL_QUANT_MLP_OUTPUT) return false;
   return true;
 }
 
@@ -210,7 +211,7 @@ static void run_attention(const sol_shape_t& s, const Layout& L, void* ws, const
 static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, const void* w_gate_up, const void* w_down,
                     const int32_t* p_permille, const void* resid, int resid_f32, void* out_bf16,
                     float* out_f32, float* out_f32_b, float* t_trace, int32_t* kept_ch, int32_t* kept_ch_cnt,
-                    cudaStream_t st) {
+                    cudaStream_t st, const int32_t* out_bits = nullptr, const sol_layer_trace_t* tr = nullptr) {
   int* status = at<int>(ws, L.status);
   GemmNK gu;
   memset(&gu, 0, sizeof(gu));
@@ -262,6 +263,17 @@ static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, cons
   dn.chunks = down_chunks(s.d_ff, s.d_model);
   dn.status = status;
   launch_gemm_down(dn, st);
+  if (out_bits != nullptr) {  // the paper's placement: the MLP output is quantized before the residual add
+    QuantOutArgs q;
+    memset(&q, 0, sizeof(q));
+    q.partial = dn.partial; q.chunks = dn.chunks; q.M = B; q.Mpad = pad_rows(B); q.d = s.d_model;
+    q.resid = resid; q.resid_f32 = resid_f32; q.bits = out_bits;
+    q.out_bf16 = out_bf16; q.out_f32 = out_f32; q.out_f32_b = out_f32_b;
+    q.z_tap = tr ? tr->z : nullptr; q.z_codes = tr ? tr->z_codes : nullptr; q.z_scale = tr ? tr->z_scales : nullptr;
+    q.live = cs.live; q.n_live = s.d_ff / 32; q.status = status;
+    launch_quant_out(q, st);
+    return;
+  }
   launch_reduce_out(dn.partial, dn.chunks, B, pad_rows(B), s.d_model, resid, resid_f32, out_bf16, out_f32, out_f32_b,
                     cs.live, s.d_ff / 32, st);
 }
@@ -274,10 +286,12 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   const int d = s.d_model, Hq = s.n_q_heads, Hkv = s.n_kv_heads, hd = s.head_dim;
   const int Nqkv = (Hq + 2 * Hkv) * hd;
   float* scale = at<float>(ws, L.scale);
+  const bool out_quant = s.quant_placement == SOL_QUANT_MLP_OUTPUT;
+  const int32_t* in_bits = out_quant ? nullptr : bits;  // no width: the rows go through as bf16
 
   NormQuantArgs n1;
   memset(&n1, 0, sizeof(n1));
-  n1.in = h_in; n1.in_f32 = in_f32; n1.gamma_bf16 = w.gamma1; n1.eps = s.rms_eps; n1.bits = bits; n1.B = B; n1.d = d;
+  n1.in = h_in; n1.in_f32 = in_f32; n1.gamma_bf16 = w.gamma1; n1.eps = s.rms_eps; n1.bits = in_bits; n1.B = B; n1.d = d;
   n1.a_op = at<void>(ws, L.a_op); n1.a_op_rows = L.Mpad; n1.scale = scale; n1.xn = tr ? tr->xn1 : nullptr;
   n1.codes = tr ? tr->codes1 : nullptr;
   n1.status = status;
@@ -321,7 +335,7 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   memset(&n2, 0, sizeof(n2));
   n2.in = h_in; n2.in_f32 = in_f32; n2.part = at<float>(ws, L.o_part); n2.ksplit = nk_ksplit(d, Hq * hd);
   n2.sum_out = at<float>(ws, L.h_mid);
-  n2.gamma_bf16 = w.gamma2; n2.eps = s.rms_eps; n2.bits = bits; n2.B = B; n2.d = d;
+  n2.gamma_bf16 = w.gamma2; n2.eps = s.rms_eps; n2.bits = in_bits; n2.B = B; n2.d = d;
   n2.a_op = at<void>(ws, L.a_op); n2.a_op_rows = L.Mpad; n2.scale = scale; n2.xn = tr ? tr->xn2 : nullptr;
   n2.codes = tr ? tr->codes2 : nullptr;
   n2.status = status;
@@ -334,7 +348,7 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
 
   run_mlp(s, L, ws, B, w.w_gate_up, w.w_down, p, at<float>(ws, L.h_mid), 1, h_out_bf16, h_out_f32,
           tr ? tr->h_out : nullptr, tr ? tr->t : nullptr, tr ? tr->kept_ch : nullptr, tr ? tr->kept_ch_cnt : nullptr,
-          st);
+          st, out_quant ? bits : nullptr, tr);
 }
 
 static bool weights_ok(const sol_layer_weights_t* w) {
@@ -386,6 +400,18 @@ sol_status_t sol_quant_act(const void* x_bf16, int32_t B, int32_t d, const int32
   NormQuantArgs n;
   memset(&n, 0, sizeof(n));
   n.in = x_bf16; n.bits = bits; n.B = B; n.d = d; n.a_op = xhat_bf16; n.scale = scales; n.codes = codes;
+  launch_norm_quant(n, (cudaStream_t)stream);
+  return finish();
+}
+
+sol_status_t sol_quant_act_wide(const void* x_bf16, int32_t B, int32_t d, const int32_t* bits, int16_t* codes,
+                                float* scales, sol_stream_t stream) {
+  if (!x_bf16 || !bits || !codes || !scales || B < 0 || d <= 0) return SOL_ERR_INVALID_ARG;
+  if (d % 8 || d > 8192) return SOL_ERR_UNSUPPORTED;
+  if (B == 0) return SOL_OK;
+  NormQuantArgs n;
+  memset(&n, 0, sizeof(n));
+  n.in = x_bf16; n.bits = bits; n.B = B; n.d = d; n.scale = scales; n.codes16 = codes;
   launch_norm_quant(n, (cudaStream_t)stream);
   return finish();
 }
@@ -564,7 +590,8 @@ sol_status_t sol_decode_step_host(const sol_shape_t* shape, int32_t n_layers, co
     if (r_permille_host[i] < 0 || r_permille_host[i] > 1000 || p_permille_host[i] < 0 || p_permille_host[i] > 1000)
       return SOL_ERR_INVALID_ARG;
     const int b = bits_host[i];
-    if (!(b == 16 || (b >= 2 && b <= 8))) return (b >= 9 && b <= 15) ? SOL_ERR_UNSUPPORTED : SOL_ERR_INVALID_ARG;
+    const int b_max = shape->quant_placement == SOL_QUANT_MLP_OUTPUT ? 15 : 8;  // operand codes are exact bf16 numbers up to 8 bits
+    if (!(b == 16 || (b >= 2 && b <= b_max))) return (b >= 9 && b <= 15) ? SOL_ERR_UNSUPPORTED : SOL_ERR_INVALID_ARG;
     if (seq_lens_host[i] < 1 || seq_lens_host[i] > mp * shape->page_size) return SOL_ERR_INVALID_ARG;
   }
   if (B == 0) return SOL_OK;

@@ -65,11 +65,32 @@ struct NormQuantArgs {
   float* scale;
   float* xn;
   int8_t* codes;
+  int16_t* codes16;  // optional: int16 codes (widths up to 15 bits where no operand is produced)
   int* status;
   uint32_t* clear;   // optional: [B][clear_words] words zeroed, row by row, for the kernels that follow
   int clear_words;
 };
 void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st);
+
+// The paper's placement of the quantizer: out = resid + fake_quant(sum of the down projection's partials),
+// per token at bits[row] (2..15; 16: unchanged).  Also clears the n_live "granule is live" flags.
+struct QuantOutArgs {
+  const float* partial;  // [chunks][Mpad][d]
+  int chunks, M, Mpad, d;
+  const void* resid;
+  int resid_f32;
+  const int32_t* bits;
+  void* out_bf16;
+  float* out_f32;
+  float* out_f32_b;
+  float* z_tap;       // optional [M][d]: the MLP output before the quantizer
+  int16_t* z_codes;   // optional [M][d]
+  float* z_scale;     // optional [M]
+  int32_t* live;
+  int n_live;
+  int* status;
+};
+void launch_quant_out(const QuantOutArgs& a, cudaStream_t st);
 
 // ---- packed operand layouts ---------------------------------------------------
 // Every tensor-core operand is stored the way the MMA reads it from shared memory, so that a stage of the

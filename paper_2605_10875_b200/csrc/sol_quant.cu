@@ -32,7 +32,7 @@ norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, i
                   float* __restrict__ sum_out, const uint16_t* __restrict__ gamma, float eps,
                   const int32_t* __restrict__ bits, int d, uint16_t* __restrict__ a_op, int a_op_rows,
                   float* __restrict__ scale,
-                  float* __restrict__ xn, int8_t* __restrict__ codes, int* __restrict__ status,
+                  float* __restrict__ xn, int8_t* __restrict__ codes, int16_t* __restrict__ codes16, int* __restrict__ status,
                   uint32_t* __restrict__ clear, int clear_words) {
   __shared__ float sh[NQ_THREADS / 32];
   pdl_trigger();
@@ -120,7 +120,10 @@ norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, i
   }
 
   int b = bits ? bits[row] : 16;
-  if (b != 16 && (b < 2 || b > 8)) {  // no kernel for this width: pass through and flag it
+  // widths of 9..15 bits need int16 codes, and their codes are no exact bf16 numbers: they are served only where
+  // no tensor-core operand is produced (the stand-alone wide quantizer call)
+  const int b_max = (codes16 != nullptr && a_op == nullptr) ? 15 : 8;
+  if (b != 16 && (b < 2 || b > b_max)) {  // no kernel for this width: pass through and flag it
     if (threadIdx.x == 0 && status != nullptr) atomicOr(status + ST_ERR, ERR_BAD_ACTION);
     b = 16;
   }
@@ -161,6 +164,17 @@ norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, i
       if (a_op_rows > 0) *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(a_op) + act_piece_offset(a_op_rows, row, v)) = w;
       else reinterpret_cast<uint4*>(a_op + (size_t)row * d)[v] = w;
     }
+    if (codes16 != nullptr) {
+      int q[NQ_VEC];
+#pragma unroll
+      for (int e = 0; e < NQ_VEC; ++e) q[e] = (b == 16) ? 0 : (int)c[e];
+      uint4 w;
+      w.x = (q[0] & 0xffff) | ((uint32_t)(q[1] & 0xffff) << 16);
+      w.y = (q[2] & 0xffff) | ((uint32_t)(q[3] & 0xffff) << 16);
+      w.z = (q[4] & 0xffff) | ((uint32_t)(q[5] & 0xffff) << 16);
+      w.w = (q[6] & 0xffff) | ((uint32_t)(q[7] & 0xffff) << 16);
+      reinterpret_cast<uint4*>(codes16 + (size_t)row * d)[v] = w;
+    }
     if (codes != nullptr) {
       int q[NQ_VEC];
 #pragma unroll
@@ -178,11 +192,112 @@ void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st) {
   if (a.in_f32)
     SOL_LAUNCH("norm_quant", norm_quant_kernel<true>, dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit, stride,
                a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d, static_cast<uint16_t*>(a.a_op),
-               a.a_op_rows, a.scale, a.xn, a.codes, a.status, a.clear, a.clear_words);
+               a.a_op_rows, a.scale, a.xn, a.codes, a.codes16, a.status, a.clear, a.clear_words);
   else
     SOL_LAUNCH("norm_quant", norm_quant_kernel<false>, dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit, stride,
                a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d, static_cast<uint16_t*>(a.a_op),
-               a.a_op_rows, a.scale, a.xn, a.codes, a.status, a.clear, a.clear_words);
+               a.a_op_rows, a.scale, a.xn, a.codes, a.codes16, a.status, a.clear, a.clear_words);
+}
+
+// ============================================================================
+// fake-quantization of the MLP output (the paper's placement of the quantizer)
+// ============================================================================
+// One token per CTA: z = sum of the down projection's partial sums; per-token symmetric quantizer at
+// bits[row] on z (appendix "Activation quantization": a = max|z|, s = a / q_max, code = clip(rne(z / s))),
+// z_hat = code * s, from 16 bits on z_hat = z; out = resid + z_hat.
+__global__ void __launch_bounds__(NQ_THREADS)
+quant_out_kernel(const float* __restrict__ partial, int chunks, size_t chunk_stride, int d, const void* __restrict__ resid,
+                 int resid_f32, const int32_t* __restrict__ bits, uint16_t* __restrict__ out_bf16, float* __restrict__ out_f32,
+                 float* __restrict__ out_f32_b, float* __restrict__ z_tap, int16_t* __restrict__ z_codes,
+                 float* __restrict__ z_scale, int32_t* __restrict__ live, int n_live, int* __restrict__ status) {
+  __shared__ float sh[NQ_THREADS / 32];
+  pdl_trigger();
+  pdl_wait();
+  const int row = blockIdx.x;
+  // the down projection has read the "granule is live" flags; the next selection starts from zero
+  for (int i = blockIdx.x * NQ_THREADS + threadIdx.x; i < n_live; i += gridDim.x * NQ_THREADS) live[i] = 0;
+  const int nvec = d / 4;
+  constexpr int VPT = 8;  // float4 vectors per thread: d <= 8192
+  float4 z[VPT];
+  float a = 0.f;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int v = threadIdx.x + i * NQ_THREADS;
+    z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (v < nvec) {
+      for (int c0 = 0; c0 < chunks; c0 += 4) {  // four partials' loads in flight, added in order
+        float4 t[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          t[q] = c0 + q < chunks ? reinterpret_cast<const float4*>(partial + (size_t)(c0 + q) * chunk_stride + (size_t)row * d)[v]
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          z[i].x += t[q].x; z[i].y += t[q].y; z[i].z += t[q].z; z[i].w += t[q].w;
+        }
+      }
+      if (z_tap) reinterpret_cast<float4*>(z_tap + (size_t)row * d)[v] = z[i];
+      a = fmaxf(a, fmaxf(fmaxf(fabsf(z[i].x), fabsf(z[i].y)), fmaxf(fabsf(z[i].z), fabsf(z[i].w))));
+    }
+  }
+  int b = bits[row];
+  if (b < 2) {
+    if (threadIdx.x == 0 && status != nullptr) atomicOr(status + ST_ERR, ERR_BAD_ACTION);
+    b = 16;
+  }
+  float s = 1.0f, q_max = 0.f;
+  if (b < 16) {
+    a = block_reduce(a, true, sh);
+    q_max = (float)((1 << (b - 1)) - 1);
+    s = __fdiv_rn(a, q_max);
+  }
+  if (threadIdx.x == 0 && z_scale) z_scale[row] = s;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int v = threadIdx.x + i * NQ_THREADS;
+    if (v >= nvec) continue;
+    float zz[4] = {z[i].x, z[i].y, z[i].z, z[i].w};
+    int cc[4] = {0, 0, 0, 0};
+    if (b < 16) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float r = (s == 0.f) ? 0.f : rintf(__fdiv_rn(zz[e], s));
+        const float c = fminf(fmaxf(r, -q_max), q_max) + 0.0f;
+        cc[e] = (int)c;
+        zz[e] = __fmul_rn(c, s);
+      }
+    }
+    if (z_codes) {
+      uint2 w;
+      w.x = (cc[0] & 0xffff) | ((uint32_t)(cc[1] & 0xffff) << 16);
+      w.y = (cc[2] & 0xffff) | ((uint32_t)(cc[3] & 0xffff) << 16);
+      reinterpret_cast<uint2*>(z_codes + (size_t)row * d)[v] = w;
+    }
+    float4 acc = make_float4(zz[0], zz[1], zz[2], zz[3]);
+    if (resid != nullptr) {
+      if (resid_f32) {
+        const float4 r = reinterpret_cast<const float4*>(static_cast<const float*>(resid) + (size_t)row * d)[v];
+        acc.x += r.x; acc.y += r.y; acc.z += r.z; acc.w += r.w;
+      } else {
+        const uint2 r = reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(resid) + (size_t)row * d)[v];
+        acc.x += bf16_lo(r.x); acc.y += bf16_hi(r.x); acc.z += bf16_lo(r.y); acc.w += bf16_hi(r.y);
+      }
+    }
+    if (out_bf16) {
+      uint2 o;
+      o.x = pack_bf16(acc.x, acc.y);
+      o.y = pack_bf16(acc.z, acc.w);
+      reinterpret_cast<uint2*>(out_bf16 + (size_t)row * d)[v] = o;
+    }
+    if (out_f32) reinterpret_cast<float4*>(out_f32 + (size_t)row * d)[v] = acc;
+    if (out_f32_b) reinterpret_cast<float4*>(out_f32_b + (size_t)row * d)[v] = acc;
+  }
+}
+
+void launch_quant_out(const QuantOutArgs& a, cudaStream_t st) {
+  SOL_LAUNCH("mlp_out_quant_residual", quant_out_kernel, dim3(a.M), dim3(NQ_THREADS), 0, st, a.partial, a.chunks,
+             (size_t)a.Mpad * a.d, a.d, a.resid, a.resid_f32, a.bits, static_cast<uint16_t*>(a.out_bf16), a.out_f32, a.out_f32_b,
+             a.z_tap, a.z_codes, a.z_scale, a.live, a.n_live, a.status);
 }
 
 }  // namespace sol

@@ -65,6 +65,22 @@ def test_quant_workload_shapes_all_bit_widths():
             assert np.array_equal(c, co) and np.array_equal(s.view(np.uint32), so.view(np.uint32)), (name, b)
 
 
+@pytest.mark.parametrize("B,d", [(6, 256), (16, 2048), (3, 8192)])
+def test_quant_wide_codes_bit_exact(B, d):
+    """Widths up to 15 bits (the paper's action tables): int16 codes, same arithmetic."""
+    rng = np.random.default_rng(B * 7 + d)
+    x = synth.to_bf16((rng.standard_normal((B, d)) * 10 ** rng.uniform(-2, 2, (B, 1))).astype(np.float32))
+    bits = rng.choice([2, 5, 8, 9, 10, 12, 15, 16], B).astype(np.int32)
+    bits[0], bits[1] = 15, 9
+    codes_o, scales_o, _ = O.quant_act(x, bits)
+    codes = torch.full((B, d), 77, dtype=torch.int16, device=H.DEV)
+    scales = torch.full((B,), -1.0, dtype=torch.float32, device=H.DEV)
+    sol.quant_act_wide(H.dev_bf16(x), B, d, H.dev_i32(bits), codes, scales)
+    torch.cuda.synchronize()
+    assert np.array_equal(codes.cpu().numpy(), codes_o.astype(np.int16))
+    assert np.array_equal(scales.cpu().numpy().view(np.uint32), scales_o.view(np.uint32))
+
+
 # -------------------------------------------------------------- attention ---
 
 
@@ -402,6 +418,63 @@ def test_layer_llama8b_shape_reduced_context():
     rng = np.random.default_rng(11)
     check_layer(L8B, [1500, 64, 333, 2048, 1, 700], rng.choice(L8B["r_set"], B), rng.choice(L8B["p_set"], B),
                 rng.choice(L8B["b_set"], B), seed=3)
+
+
+def _mlp_output_placement_case(cfg, seq_lens, r, p, b, seed):
+    """A layer with the paper's placement of the quantizer (on the MLP output, widths up to 15 bits): the
+    fake-quantization is checked bit for bit on the MLP output the GPU itself produced, the rest of the layer
+    against the oracle's layer in the same placement."""
+    shape, oshape = H.make_shapes(cfg, quant_placement=sol.QUANT_MLP_OUTPUT)
+    B = len(seq_lens)
+    seq_lens = np.asarray(seq_lens, np.int32)
+    w = synth.make_layer_weights(cfg, seed)
+    k_pool, v_pool, table = H.make_case_kv(cfg, seq_lens, seed)
+    h_in = synth.make_hidden(cfg, seed, B)
+    kv = H.device_kv(k_pool, v_pool, table, seq_lens)
+    out, taps, st = H.gpu_layer(shape, H.device_weights(w, shape), kv, h_in, r, p, b)
+    assert st[0] == 0, st
+    # no quantizer on the projections' inputs
+    assert not taps["codes1"].any() and not taps["codes2"].any()
+    assert np.all(taps["scales1"] == 1) and np.all(taps["scales2"] == 1)
+    # the quantizer on the GPU's own MLP output: codes and scales bit for bit, the update within a float32 rounding
+    for i in range(B):
+        c, s, z_hat = O.fake_quant_mlp_output(taps["z"][i].astype(np.float64), int(b[i]))
+        assert np.array_equal(taps["z_codes"][i], c.astype(np.int16)), ("z codes", i, int(b[i]))
+        assert np.float32(s) == taps["z_scales"][i], ("z scale", i)
+        want = taps["h_mid"][i].astype(np.float64) + z_hat
+        assert np.allclose(taps["h_out"][i], want, rtol=0, atol=2e-6 * max(1.0, np.abs(want).max())), ("h_out", i)
+    # the MLP output itself, and the layer, against the oracle in the same placement
+    okv = O.PagedKV(k_pool, v_pool, np.where(table < 0, 0, table), seq_lens)
+    out_o, tr = O.decode_layer(oshape, H.oracle_weights(w), okv, O.bf16_to_f64(h_in), r, p, b, O.PLACE_MLP_OUTPUT)
+    same_sets = all(np.array_equal(taps["kept_ch"][i, : taps["kept_ch_cnt"][i]], tr.kept_channels[i]) for i in range(B))
+    if same_sets:
+        assert np.allclose(taps["z"], tr.extra["z"], rtol=0, atol=2e-3 * max(1.0, np.abs(tr.extra["z"]).max())), "z"
+    # a float32-vs-float64 difference of the MLP output that crosses a rounding boundary moves that element by a
+    # whole step (a / q_max, e.g. 1/15 of the row's largest value at 5 bits): the end-to-end rule is the gate only
+    # when no code differs from the oracle's own run; the codes on the GPU's own z were checked bit for bit above
+    flips = sum(int((taps["z_codes"][i] != tr.extra["z_codes"][i]).sum()) for i in range(B))
+    err = checker.output_errors(out_o, out)
+    if flips == 0 and same_sets:
+        H.assert_outputs(out_o, out, "layer output, quantizer on the MLP output")
+    else:
+        assert err[1] <= checker.OUT_REL_L2, err  # a handful of one-step differences leave the relative L2 error small
+    return dict(err=err, z_code_flips=flips, end_to_end_asserted=flips == 0 and same_sets, status=st)
+
+
+def test_layer_quantizer_on_mlp_output_tiny():
+    cfg = dict(TINY, rope_theta=10000.0)
+    res = _mlp_output_placement_case(cfg, [512, 65, 1, 300, 129], [1000, 500, 250, 125, 1000], [0, 250, 500, 0, 750],
+                                     [16, 12, 5, 9, 15], seed=21)
+    print("tiny layer, MLP-output placement:", res)
+
+
+def test_layer_quantizer_on_mlp_output_llama1b():
+    B = L1B["batch"]
+    rng = np.random.default_rng(22)
+    r, p, _ = synth.draw_actions(L1B, 0)
+    b = rng.choice([5, 8, 11, 13, 16], B).astype(np.int32)  # the paper's widths: 5..16
+    res = _mlp_output_placement_case(L1B, synth.make_contexts(L1B, 0), r, p, b, seed=0)
+    print("llama1b layer, MLP-output placement:", res)
 
 
 # ------------------------------------------------------------------- step ---
