@@ -32,8 +32,9 @@ Readings taken where the paper is silent or the benchmark spec overrides it:
     forced-keep tokens (sinks, recent window; default: only the newest
     token) count toward the budget; softmax runs over the kept set only;
   * MLP pruning drops the p fraction of *intermediate* channels with the
-    smallest |silu(g)*u| per token (the paper gates MLP input channels);
-    the kept count mirrors the paper's ceil form;
+    smallest |silu(g)*u| per token (the task's default); the paper's own
+    form, gating the MLP block's input channels by |x|, is PRUNE_MLP_INPUT;
+    the kept count mirrors the paper's ceil form in both;
   * ties are broken toward the lower index;
   * T (seq_lens) counts the newest token, whose k/v the layer appends
     before attention reads the cache.
@@ -418,14 +419,37 @@ def append_kv(shape: Shape, kv: PagedKV, i: int, k_bf16: np.ndarray, v_bf16: np.
     kv.v_pool[page, :, slot, :] = v_bf16
 
 
+PRUNE_INTERMEDIATE = 0  # the task's default: intermediate channels by |silu(g) u| (pruned_swiglu_mlp)
+PRUNE_MLP_INPUT = 1     # the paper's: input channels of the MLP block by |x| (gate_input_channels)
+
+
+def gate_input_channels(x32: np.ndarray, p_permille: int):
+    """The paper's structured MLP pruning (appendix "Structured MLP activation pruning", "Per-token channel
+    selection"): of the MLP block's input x (one token, d_model channels) keep the m = ceil(rho * d_model)
+    channels of largest magnitude |x(j)|, rho = 1 - p, and zero the rest (a multiplicative 0/1 mask).
+    Ties go to the lower index.  The magnitudes are compared as the float32 numbers the quantizer also sees.
+    Returns (kept indices ascending, masked x float32)."""
+    x32 = np.asarray(x32, np.float32)
+    m = kept_channel_count(int(p_permille), x32.shape[0])
+    kept = select_top(np.abs(x32).astype(np.float64), m, np.zeros(0, np.int64))
+    out = np.zeros_like(x32)
+    out[kept] = x32[kept]
+    return kept, out
+
+
 PLACE_PROJ_INPUTS = 0  # the task's default: the inputs of the QKV and gate/up projections are quantized
 PLACE_MLP_OUTPUT = 1   # the paper's: the MLP output is fake-quantized before the residual add
 
 
 def decode_layer(shape: Shape, w: LayerWeights, kv: PagedKV, h_in: np.ndarray,
                  r_permille: Sequence[int], p_permille: Sequence[int], bits: Sequence[int],
-                 placement: int = PLACE_PROJ_INPUTS):
+                 placement: int = PLACE_PROJ_INPUTS, mlp_prune: int = PRUNE_INTERMEDIATE):
     """One decoder layer for one new token per sequence.
+
+    mlp_prune == PRUNE_MLP_INPUT: p_permille[i] gates the input channels of the
+    MLP block (gate_input_channels on the normalised row, before the quantizer;
+    the attention input of the layer is not pruned) and every intermediate
+    channel is kept.
 
     placement == PLACE_MLP_OUTPUT: the projections read the normalised rows
     through the 16-bit passthrough (bf16, the operand type of the matmuls) and
@@ -467,8 +491,23 @@ def decode_layer(shape: Shape, w: LayerWeights, kv: PagedKV, h_in: np.ndarray,
     tr.h_mid = h_mid
 
     # MLP input: RMSNorm, quantize; pruned SwiGLU; residual
-    tr.xn2, tr.codes2, tr.scales2, x_hat2 = norm_and_quantize(h_mid, w.gamma2, shape.rms_eps, in_bits)
-    mlp, tr.kept_channels, tr.t = pruned_swiglu_mlp(x_hat2, w.w_gate, w.w_up, w.w_down_t, p_permille)
+    if mlp_prune == PRUNE_MLP_INPUT:
+        gamma2 = bf16_to_f64(w.gamma2)
+        tr.xn2 = np.zeros((B, d), np.float32)
+        tr.codes2 = np.zeros((B, d), np.int16 if any(8 < int(b) < 16 for b in in_bits) else np.int8)
+        tr.scales2 = np.zeros(B, np.float32)
+        x_hat2 = np.zeros((B, d))
+        kept_in = []
+        for i in range(B):
+            tr.xn2[i] = rmsnorm(h_mid[i], gamma2, shape.rms_eps).astype(np.float32)
+            kept_i, masked = gate_input_channels(tr.xn2[i], int(p_permille[i]))
+            kept_in.append(kept_i)
+            tr.codes2[i], tr.scales2[i], x_hat2[i] = quantize_per_token(masked, int(in_bits[i]))
+        tr.extra["kept_inputs"] = kept_in
+        mlp, tr.kept_channels, tr.t = pruned_swiglu_mlp(x_hat2, w.w_gate, w.w_up, w.w_down_t, [0] * B)
+    else:
+        tr.xn2, tr.codes2, tr.scales2, x_hat2 = norm_and_quantize(h_mid, w.gamma2, shape.rms_eps, in_bits)
+        mlp, tr.kept_channels, tr.t = pruned_swiglu_mlp(x_hat2, w.w_gate, w.w_up, w.w_down_t, p_permille)
     if placement == PLACE_MLP_OUTPUT:
         tr.extra["z"] = mlp.copy()
         z_codes, z_scales = [], np.zeros(B, np.float32)
@@ -480,13 +519,13 @@ def decode_layer(shape: Shape, w: LayerWeights, kv: PagedKV, h_in: np.ndarray,
 
 
 def decode_step(shape: Shape, layers: Sequence[LayerWeights], kvs: Sequence[PagedKV], h_in_bf16: np.ndarray,
-                r_permille, p_permille, bits, placement: int = PLACE_PROJ_INPUTS):
+                r_permille, p_permille, bits, placement: int = PLACE_PROJ_INPUTS, mlp_prune: int = PRUNE_INTERMEDIATE):
     """L layers with the same action tuple in every layer (the paper broadcasts
     one action across all layers at a decode step).  The residual stream is
     not rounded between layers.  Returns (h_out float64, [trace per layer])."""
     h = bf16_to_f64(h_in_bf16)
     traces = []
     for w, kv in zip(layers, kvs):
-        h, tr = decode_layer(shape, w, kv, h, r_permille, p_permille, bits, placement)
+        h, tr = decode_layer(shape, w, kv, h, r_permille, p_permille, bits, placement, mlp_prune)
         traces.append(tr)
     return h, traces

@@ -185,6 +185,56 @@ def test_mlp_output_placement_of_the_quantizer():
     assert not tr.codes1.any() and not tr.codes2.any() and np.all(tr.scales1 == 1) and np.all(tr.scales2 == 1)
 
 
+def test_input_channel_gating_brute_force_ties_and_counts():
+    """The paper's MLP pruning (appendix "Structured MLP activation pruning"): m = ceil(rho d) input channels of
+    largest |x| survive.  Brute force over all subsets on a tiny row; ties to the lower index; the mask is 0/1."""
+    import itertools
+    from fractions import Fraction
+
+    rng = np.random.default_rng(41)
+    x = rng.standard_normal(9).astype(np.float32)
+    for p in (0, 100, 250, 500, 667, 900, 1000):
+        kept, masked = O.gate_input_channels(x, p)
+        m = -((-(1000 - p) * 9) // 1000)  # ceil((1 - p) d)
+        assert m == math.ceil(Fraction(1000 - p, 1000) * 9) and len(kept) == m
+        best = max(itertools.combinations(range(9), m), key=lambda c: sum(abs(float(x[j])) for j in c)) if m else ()
+        assert list(kept) == sorted(best)
+        assert np.array_equal(masked[kept], x[kept]) and np.count_nonzero(masked) == m
+    # equal magnitudes (either sign): the lower indices win
+    t = np.array([1.0, -2.0, 2.0, -1.0, 2.0, 1.0], np.float32)
+    assert list(O.gate_input_channels(t, 500)[0]) == [1, 2, 4]
+    assert list(O.gate_input_channels(t, 667)[0]) == [1, 2]   # ceil(0.333 * 6) = 2
+    assert list(O.gate_input_channels(t, 1000)[0]) == []
+
+
+def test_layer_with_input_channel_gating_is_a_dense_mlp_on_the_masked_row():
+    """PRUNE_MLP_INPUT: the MLP update equals a dense SwiGLU MLP (torch float64) on the masked, normalised row;
+    the attention half of the layer is untouched; p = 0 reproduces the unpruned layer."""
+    import copy
+
+    shape, W, kv, h = _layer_case(43)
+    B = h.shape[0]
+    r, bits = [1000, 500, 250][:B], [16] * B
+    p = [0, 500, 750][:B]
+    out, tr = O.decode_layer(shape, W, copy.deepcopy(kv), h, r, p, bits, mlp_prune=O.PRUNE_MLP_INPUT)
+    base, tr0 = O.decode_layer(shape, W, copy.deepcopy(kv), h, r, [0] * B, bits)
+    assert np.array_equal(tr.h_mid, tr0.h_mid)  # attention input not pruned
+    assert np.array_equal(out[0], base[0])      # p = 0 keeps every channel
+    Wg, Wu, Wd = (torch.from_numpy(O.bf16_to_f64(m)) for m in (W.w_gate, W.w_up, W.w_down_t))
+    d = shape.d_model
+    for i in range(B):
+        xn = torch.from_numpy(tr.xn2[i].astype(np.float64))
+        m = -((-(1000 - p[i]) * d) // 1000)
+        keep = torch.topk(xn.abs(), m).indices if m else torch.zeros(0, dtype=torch.long)
+        assert sorted(keep.tolist()) == list(tr.extra["kept_inputs"][i])
+        mask = torch.zeros(d, dtype=torch.float64)
+        mask[keep] = 1.0
+        xm = (xn * mask).to(torch.float32).to(torch.bfloat16).to(torch.float64)  # 16-bit passthrough of the masked row
+        z = (torch.nn.functional.silu(Wg @ xm) * (Wu @ xm)) @ Wd
+        assert np.allclose(out[i] - tr.h_mid[i], z.numpy(), rtol=0, atol=1e-12)
+        assert len(tr.kept_channels[i]) == shape.d_ff  # no intermediate channel is dropped
+
+
 def test_quantizer_mixed_bits_per_example():
     rng = np.random.default_rng(2)
     xb = synth.to_bf16(rng.standard_normal((3, 64)).astype(np.float32))
