@@ -416,7 +416,11 @@ def run_ours(args):
     barrier, max_over_ranks = ranks.barrier, ranks.max_over_ranks
 
     sol.lib()
-    cfg = synth.WORKLOADS[args.workload]
+    cfg = dict(synth.WORKLOADS[args.workload])
+    if args.batch:
+        cfg["batch"] = args.batch
+    if args.layers:
+        cfg["layers"] = args.layers
     rep = Replica(cfg, device, seed=0)
     r, p, b = synth.draw_actions(cfg, 0)
     redraws = [synth.draw_actions(cfg, 0, redraw=k) for k in range(1, SERVE_STEPS // SERVE_REDRAW)] if rep.serving else None
@@ -676,6 +680,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rotate", type=int, default=ROTATE,
                     help="distinct copies of weights and KV cache cycled through the steps (1 for a small profiler capture)")
+    ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (a scaled-down case for a profiler capture)")
+    ap.add_argument("--layers", type=int, default=None, help="override the workload's layer count (same purpose)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="skip the compact runs of the other workloads")

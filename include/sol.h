@@ -58,9 +58,17 @@ typedef struct sol_shape {
                                (1, the paper's: appendix "Activation quantization", "What is quantized") on the MLP
                                output before the residual add, widths 2..15, 16 and more: unchanged; the
                                projections then read bf16 rows */
+  int32_t mlp_prune;        /* what p_permille[i] prunes in a layer: SOL_PRUNE_INTERMEDIATE (0, the task's default) the
+                               intermediate channels with the smallest |silu(g) u|; SOL_PRUNE_MLP_INPUT (1, the
+                               paper's: appendix "Structured MLP activation pruning") the input channels of the MLP
+                               block with the smallest |x|: ceil((1 - p) d_model) survive (ties: lower index), the
+                               rest of the normalised row is zeroed before the quantizer; the attention input is
+                               not pruned and every intermediate channel is kept */
 } sol_shape_t;
 #define SOL_QUANT_PROJ_INPUTS 0
 #define SOL_QUANT_MLP_OUTPUT 1
+#define SOL_PRUNE_INTERMEDIATE 0
+#define SOL_PRUNE_MLP_INPUT 1
 
 /* Paged bf16 KV cache of one layer.  Pools: [num_pages][n_kv_heads][page_size][head_dim].
  * page_table: int32 [B][max_pages_per_seq], physical page of each logical page.
@@ -125,6 +133,7 @@ typedef struct sol_layer_trace {
   float *z;             /* SOL_QUANT_MLP_OUTPUT only: [B][d_model] MLP output before the quantizer (float32) */
   int16_t *z_codes;     /* SOL_QUANT_MLP_OUTPUT only: [B][d_model] its codes (0 for 16 bits) */
   float *z_scales;      /* SOL_QUANT_MLP_OUTPUT only: [B] */
+  float *xm2;           /* SOL_PRUNE_MLP_INPUT only: [B][d_model] the MLP input after the channel gating (float32) */
 } sol_layer_trace_t;
 
 const char *sol_status_string(sol_status_t s);

@@ -34,7 +34,7 @@ class SolShape(C.Structure):
     _fields_ = [("d_model", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("page_size", C.c_int32),
                 ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("n_sink", C.c_int32), ("n_window", C.c_int32),
-                ("quant_placement", C.c_int32)]
+                ("quant_placement", C.c_int32), ("mlp_prune", C.c_int32)]
 
 
 class SolKV(C.Structure):
@@ -47,7 +47,7 @@ class SolLayerWeights(C.Structure):
 
 
 TRACE_FIELDS = ("xn1", "codes1", "scales1", "q_rot", "kept_idx", "kept_cnt", "attn_out", "h_mid", "xn2", "codes2",
-                "scales2", "t", "kept_ch", "kept_ch_cnt", "h_out", "z", "z_codes", "z_scales")
+                "scales2", "t", "kept_ch", "kept_ch_cnt", "h_out", "z", "z_codes", "z_scales", "xm2")
 
 
 class SolLayerTrace(C.Structure):
@@ -154,9 +154,9 @@ def last_cuda_error() -> str:
 
 
 def make_shape(d_model, n_q_heads, n_kv_heads, head_dim, d_ff, page_size=64, rms_eps=1e-5, rope_theta=0.0,
-               n_sink=0, n_window=1, quant_placement=0) -> SolShape:
+               n_sink=0, n_window=1, quant_placement=0, mlp_prune=0) -> SolShape:
     return SolShape(d_model, n_q_heads, n_kv_heads, head_dim, d_ff, page_size, rms_eps, rope_theta, n_sink, n_window,
-                    quant_placement)
+                    quant_placement, mlp_prune)
 
 
 def make_kv(k_pool, v_pool, page_table, seq_lens, max_pages_per_seq: int, num_pages: int) -> SolKV:
@@ -204,6 +204,7 @@ def quant_act(x_bf16, B: int, d: int, bits, codes, scales, xhat_bf16=None, strea
 
 
 QUANT_PROJ_INPUTS, QUANT_MLP_OUTPUT = 0, 1
+PRUNE_INTERMEDIATE, PRUNE_MLP_INPUT = 0, 1
 
 
 def quant_act_wide(x_bf16, B: int, d: int, bits, codes_i16, scales, stream=None, check=True) -> int:

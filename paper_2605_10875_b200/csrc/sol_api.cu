@@ -93,7 +93,7 @@ void ensure_dynamic_smem(const void* kernel, int bytes) {
 // workspace layout
 // ---------------------------------------------------------------------------
 struct Layout {
-  size_t status, stage_h_in, stage_act, stage_h_out, a_op, scale, qkv, attn_hi, attn_lo, attn_f32, h_mid, o_part, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, ch_sel, ch_cand_val, ch_cand_idx, ch_keep, down_part,
+  size_t status, zero_p, stage_h_in, stage_act, stage_h_out, a_op, scale, qkv, attn_hi, attn_lo, attn_f32, h_mid, o_part, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, ch_sel, ch_cand_val, ch_cand_idx, ch_keep, down_part,
       h_a, h_b, total;
   AttnScratch attn;
   int chunks, Mpad, Tmax;
@@ -110,6 +110,7 @@ static bool shape_ok(const sol_shape_t* s) {
   if (s->d_ff <= 0 || s->d_ff % 32 || s->d_ff > 49152) return false;
   if (s->n_sink < 0 || s->n_window < 0) return false;
   if (s->quant_placement != SOL_QUANT_PROJ_INPUTS && s->quant_placement != SOL_QUANT_MLP_OUTPUT) return false;
+  if (s->mlp_prune != SOL_PRUNE_INTERMEDIATE && s->mlp_prune != SOL_PRUNE_MLP_INPUT) return false;
   return true;
 }
 
@@ -129,6 +130,7 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
     return o;
   };
   L.status = take(256);
+  L.zero_p = take(128 * 4);  // per-sequence prune rates of zero (never written after the workspace is initialised)
   L.stage_h_in = take(B * d * 2);
   L.stage_act = take(4 * (size_t)B * 4);
   L.stage_h_out = take(B * d * 2);
@@ -339,6 +341,11 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   n2.a_op = at<void>(ws, L.a_op); n2.a_op_rows = L.Mpad; n2.scale = scale; n2.xn = tr ? tr->xn2 : nullptr;
   n2.codes = tr ? tr->codes2 : nullptr;
   n2.status = status;
+  const bool gate_inputs = s.mlp_prune == SOL_PRUNE_MLP_INPUT;
+  if (gate_inputs) {  // the paper's MLP pruning: p gates the input channels, every intermediate channel is kept
+    n2.gate_p_permille = p;
+    n2.xm = tr ? tr->xm2 : nullptr;
+  }
   n2.clear = at<uint32_t>(ws, L.ch_sel);
   n2.clear_words = CH_SEL_WORDS;
   launch_norm_quant(n2, st);
@@ -346,7 +353,8 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
     cudaMemcpyAsync(tr->h_mid, at<float>(ws, L.h_mid), sizeof(float) * B * d, cudaMemcpyDeviceToDevice, st);
   if (tr && tr->scales2) cudaMemcpyAsync(tr->scales2, scale, sizeof(float) * B, cudaMemcpyDeviceToDevice, st);
 
-  run_mlp(s, L, ws, B, w.w_gate_up, w.w_down, p, at<float>(ws, L.h_mid), 1, h_out_bf16, h_out_f32,
+  run_mlp(s, L, ws, B, w.w_gate_up, w.w_down, gate_inputs ? at<int32_t>(ws, L.zero_p) : p, at<float>(ws, L.h_mid), 1,
+          h_out_bf16, h_out_f32,
           tr ? tr->h_out : nullptr, tr ? tr->t : nullptr, tr ? tr->kept_ch : nullptr, tr ? tr->kept_ch_cnt : nullptr,
           st, out_quant ? bits : nullptr, tr);
 }

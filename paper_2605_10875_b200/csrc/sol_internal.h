@@ -66,6 +66,8 @@ struct NormQuantArgs {
   float* xn;
   int8_t* codes;
   int16_t* codes16;  // optional: int16 codes (widths up to 15 bits where no operand is produced)
+  const int32_t* gate_p_permille;  // optional [B]: input-channel gating of the MLP block before the quantizer
+  float* xm;         // optional tap of the gated row
   int* status;
   uint32_t* clear;   // optional: [B][clear_words] words zeroed, row by row, for the kernels that follow
   int clear_words;

@@ -6,8 +6,11 @@
 //   q_max = 2^(b-1) - 1, a = max|x|, s = a / q_max, code = clip(rne(x / s)).
 // Both divisions are IEEE float32 (__fdiv_rn) so the codes are reproducible
 // bit for bit.
+#include <type_traits>
+
 #include "sol_common.cuh"
 #include "sol_internal.h"
+#include "sol_select.cuh"
 
 namespace sol {
 
@@ -26,15 +29,25 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float* sh) {
   return r;
 }
 
-template <bool IN_F32>
+// What the input-channel gating of the MLP block needs beside the row (GATE variant only).
+struct GateArgs {
+  const int32_t* p_permille;  // [B] prune rate: ceil((1 - p) d) channels of largest |x| survive
+  float* xm;                  // optional tap: [B][d] the masked normalised row
+};
+struct NoSmem {
+  int unused;
+};
+
+template <bool IN_F32, bool GATE>
 __global__ void __launch_bounds__(NQ_THREADS)
 norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, int ksplit, size_t part_stride,
                   float* __restrict__ sum_out, const uint16_t* __restrict__ gamma, float eps,
                   const int32_t* __restrict__ bits, int d, uint16_t* __restrict__ a_op, int a_op_rows,
                   float* __restrict__ scale,
                   float* __restrict__ xn, int8_t* __restrict__ codes, int16_t* __restrict__ codes16, int* __restrict__ status,
-                  uint32_t* __restrict__ clear, int clear_words) {
+                  uint32_t* __restrict__ clear, int clear_words, const GateArgs gate) {
   __shared__ float sh[NQ_THREADS / 32];
+  __shared__ typename std::conditional<GATE, SelectSmem, NoSmem>::type gsm;
   pdl_trigger();
   pdl_wait();
   const int row = blockIdx.x;
@@ -119,6 +132,71 @@ norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, i
     }
   }
 
+  if constexpr (GATE) {
+    // The paper's structured MLP pruning (appendix "Structured MLP activation pruning"): keep the
+    // m = ceil((1 - p) d) channels of largest |x|, ties to the lower index, zero the rest.  |x| orders like its
+    // bit pattern; element j = 8 v + e of the row is slot i * 8 + e of thread v - 256 i.
+    const int m = (int)(((long long)(1000 - gate.p_permille[row]) * d + 999) / 1000);
+    if (m < d) {
+      auto key = [&](int q) -> uint32_t {
+        const int v = threadIdx.x + (q >> 3) * NQ_THREADS;
+        return v < nvec ? __float_as_uint(fabsf(x[q >> 3][q & 7])) : 0u;
+      };
+      int tie_need = 0;
+      uint32_t thr = 0xffffffffu;
+      if (m > 0) thr = select_kth<NQ_THREADS, NQ_MAX_PER_THREAD * NQ_VEC>(key, m, tie_need, gsm, NQ_MAX_PER_THREAD * NQ_VEC);
+      // ties at the threshold are kept in index order until tie_need runs out: index order is (i, thread, e)
+      int taken = 0;  // ties granted to earlier rounds (block-uniform)
+#pragma unroll
+      for (int i = 0; i < NQ_MAX_PER_THREAD; ++i) {
+        const int v = threadIdx.x + i * NQ_THREADS;
+        uint32_t tie_mask = 0;
+#pragma unroll
+        for (int e = 0; e < NQ_VEC; ++e)
+          if (m > 0 && v < nvec && __float_as_uint(fabsf(x[i][e])) == thr) tie_mask |= 1u << e;
+        // exclusive prefix of the tie counts over the threads of this round
+        const int mine = __popc(tie_mask);
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, incl, o);
+          if ((threadIdx.x & 31) >= o) incl += y;
+        }
+        __syncthreads();
+        if ((threadIdx.x & 31) == 31) gsm.scan[0][threadIdx.x >> 5] = incl;
+        __syncthreads();
+        int before = taken + incl - mine, total = 0;
+        for (int wq = 0; wq < NQ_THREADS / 32; ++wq) {
+          const int y = gsm.scan[0][wq];
+          if (wq < (int)(threadIdx.x >> 5)) before += y;
+          total += y;
+        }
+        taken += total;
+#pragma unroll
+        for (int e = 0; e < NQ_VEC; ++e) {
+          const uint32_t kk = __float_as_uint(fabsf(x[i][e]));
+          bool keep = m > 0 && kk > thr;
+          if ((tie_mask >> e) & 1u) {
+            keep = before < tie_need;
+            ++before;
+          }
+          if (!keep) x[i][e] = 0.f;
+        }
+      }
+    }
+    if (gate.xm != nullptr) {
+#pragma unroll
+      for (int i = 0; i < NQ_MAX_PER_THREAD; ++i) {
+        const int v = threadIdx.x + i * NQ_THREADS;
+        if (v < nvec) {
+          float4* p = reinterpret_cast<float4*>(gate.xm + (size_t)row * d) + 2 * v;
+          p[0] = make_float4(x[i][0], x[i][1], x[i][2], x[i][3]);
+          p[1] = make_float4(x[i][4], x[i][5], x[i][6], x[i][7]);
+        }
+      }
+    }
+  }
+
   int b = bits ? bits[row] : 16;
   // widths of 9..15 bits need int16 codes, and their codes are no exact bf16 numbers: they are served only where
   // no tensor-core operand is produced (the stand-alone wide quantizer call)
@@ -189,14 +267,22 @@ norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, i
 
 void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st) {
   const size_t stride = (size_t)a.B * a.d;
-  if (a.in_f32)
-    SOL_LAUNCH("norm_quant", norm_quant_kernel<true>, dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit, stride,
-               a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d, static_cast<uint16_t*>(a.a_op),
-               a.a_op_rows, a.scale, a.xn, a.codes, a.codes16, a.status, a.clear, a.clear_words);
-  else
-    SOL_LAUNCH("norm_quant", norm_quant_kernel<false>, dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit, stride,
-               a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d, static_cast<uint16_t*>(a.a_op),
-               a.a_op_rows, a.scale, a.xn, a.codes, a.codes16, a.status, a.clear, a.clear_words);
+  GateArgs g;
+  g.p_permille = a.gate_p_permille;
+  g.xm = a.xm;
+#define SOL_NQ_LAUNCH(F32, GATE)                                                                                       \
+  SOL_LAUNCH("norm_quant", (norm_quant_kernel<F32, GATE>), dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit,  \
+             stride, a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d,                        \
+             static_cast<uint16_t*>(a.a_op), a.a_op_rows, a.scale, a.xn, a.codes, a.codes16, a.status, a.clear,         \
+             a.clear_words, g)
+  if (a.gate_p_permille != nullptr) {
+    if (a.in_f32) SOL_NQ_LAUNCH(true, true);
+    else SOL_NQ_LAUNCH(false, true);
+  } else {
+    if (a.in_f32) SOL_NQ_LAUNCH(true, false);
+    else SOL_NQ_LAUNCH(false, false);
+  }
+#undef SOL_NQ_LAUNCH
 }
 
 // ============================================================================

@@ -29,11 +29,11 @@ def host_u16(t: torch.Tensor) -> np.ndarray:
     return t.detach().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-def make_shapes(cfg: dict, n_sink=0, n_window=1, quant_placement=0):
+def make_shapes(cfg: dict, n_sink=0, n_window=1, quant_placement=0, mlp_prune=0):
     kw = dict(d_model=cfg["d_model"], n_q_heads=cfg["n_q_heads"], n_kv_heads=cfg["n_kv_heads"],
               head_dim=cfg["head_dim"], d_ff=cfg["d_ff"], page_size=64, rms_eps=synth.RMS_EPS,
               rope_theta=cfg.get("rope_theta", 0.0), n_sink=n_sink, n_window=n_window)
-    return sol.make_shape(quant_placement=quant_placement, **kw), O.Shape(**kw)
+    return sol.make_shape(quant_placement=quant_placement, mlp_prune=mlp_prune, **kw), O.Shape(**kw)
 
 
 class Workspace:
@@ -175,6 +175,8 @@ class LayerTaps:
                       kept_ch=i32(B, ff), kept_ch_cnt=i32(B), h_out=f32(B, d))
         if shape.quant_placement == sol.QUANT_MLP_OUTPUT:
             self.t.update(z=f32(B, d), z_codes=torch.zeros((B, d), dtype=torch.int16, device=DEV), z_scales=f32(B))
+        if shape.mlp_prune == sol.PRUNE_MLP_INPUT:
+            self.t.update(xm2=f32(B, d))
 
     def struct(self):
         return sol.make_trace(**self.t)

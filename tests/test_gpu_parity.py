@@ -477,6 +477,77 @@ def test_layer_quantizer_on_mlp_output_llama1b():
     print("llama1b layer, MLP-output placement:", res)
 
 
+def _input_gating_case(cfg, seq_lens, r, p, b, seed):
+    """A layer with the paper's MLP pruning (input-channel gating by |x|): the kept set is checked bit for bit
+    on the normalised row the GPU itself produced, the quantizer on the gated row, the rest of the layer
+    against the oracle's layer in the same mode."""
+    shape, oshape = H.make_shapes(cfg, mlp_prune=sol.PRUNE_MLP_INPUT)
+    B = len(seq_lens)
+    seq_lens = np.asarray(seq_lens, np.int32)
+    w = synth.make_layer_weights(cfg, seed)
+    k_pool, v_pool, table = H.make_case_kv(cfg, seq_lens, seed)
+    h_in = synth.make_hidden(cfg, seed, B)
+    kv = H.device_kv(k_pool, v_pool, table, seq_lens)
+    out, taps, st = H.gpu_layer(shape, H.device_weights(w, shape), kv, h_in, r, p, b)
+    assert st[0] == 0, st
+    x_hat2 = np.zeros((B, cfg["d_model"]))
+    for i in range(B):
+        kept, masked = O.gate_input_channels(taps["xn2"][i], int(p[i]))
+        assert np.array_equal(taps["xm2"][i], masked), ("gated row", i)
+        c, s, x_hat2[i] = O.quantize_per_token(taps["xm2"][i], int(b[i]))
+        assert np.array_equal(c, taps["codes2"][i]) and np.float32(s) == taps["scales2"][i], ("codes2", i)
+        assert taps["kept_ch_cnt"][i] == cfg["d_ff"]  # no intermediate channel is dropped
+    mlp_o, _, t_o = O.pruned_swiglu_mlp(x_hat2, w.w_gate, w.w_up, w.w_down_t, [0] * B)
+    want = taps["h_mid"].astype(np.float64) + mlp_o
+    H.assert_outputs(want, taps["h_out"], "MLP on the gated row")
+    assert np.allclose(taps["h_out"], want, rtol=0, atol=2e-4 * max(1.0, np.abs(want).max() / 8)), "h_out"
+    okv = O.PagedKV(k_pool, v_pool, np.where(table < 0, 0, table), seq_lens)
+    out_o, tr = O.decode_layer(oshape, H.oracle_weights(w), okv, O.bf16_to_f64(h_in), r, p, b, mlp_prune=O.PRUNE_MLP_INPUT)
+    same = all(np.array_equal(np.flatnonzero(taps["xm2"][i]), np.flatnonzero(tr.xn2[i] * np.isin(np.arange(cfg["d_model"]),
+               tr.extra["kept_inputs"][i]))) for i in range(B)) and np.array_equal(taps["codes2"], tr.codes2) \
+        and np.array_equal(taps["codes1"], tr.codes1)
+    err = checker.output_errors(out_o, out)
+    if same:
+        H.assert_outputs(out_o, out, "layer output, input-channel gating")
+    return dict(err=err, end_to_end_asserted=same, status=st)
+
+
+def test_layer_input_channel_gating_tiny():
+    cfg = dict(TINY, rope_theta=10000.0)
+    res = _input_gating_case(cfg, [512, 65, 1, 300, 129, 64], [1000, 500, 250, 125, 1000, 500], [0, 250, 500, 1000, 750, 999],
+                             [16, 8, 4, 16, 8, 16], seed=23)
+    print("tiny layer, input-channel gating:", res)
+
+
+def test_layer_input_channel_gating_llama1b():
+    r, p, b = synth.draw_actions(L1B, 0)
+    res = _input_gating_case(L1B, synth.make_contexts(L1B, 0), r, p, b, seed=0)
+    print("llama1b layer, input-channel gating:", res)
+
+
+def test_input_channel_gating_ties_go_to_the_lower_index():
+    """A hidden state of equal magnitudes and a gain of ones: every |x| ties, so the survivors are the lowest indices."""
+    cfg = dict(TINY)
+    shape, oshape = H.make_shapes(cfg, mlp_prune=sol.PRUNE_MLP_INPUT)
+    B, d = 3, cfg["d_model"]
+    w = synth.make_layer_weights(cfg, 5)
+    w.gamma2[:] = synth.to_bf16(np.ones(d, np.float32))
+    w.w_o[:] = 0  # the attention update vanishes: the MLP sees the hidden state itself
+    rng = np.random.default_rng(9)
+    h = np.where(rng.random((B, d)) < 0.5, -1.0, 1.0).astype(np.float32) * np.array([[0.5], [2.0], [1.0]], np.float32)
+    h_in = synth.to_bf16(h)
+    lens = np.array([64, 10, 200], np.int32)
+    k_pool, v_pool, table = H.make_case_kv(cfg, lens, 5)
+    kv = H.device_kv(k_pool, v_pool, table, lens)
+    p = [500, 250, 875]
+    out, taps, st = H.gpu_layer(shape, H.device_weights(w, shape), kv, h_in, [1000] * B, p, [16] * B)
+    for i in range(B):
+        m = -((-(1000 - p[i]) * d) // 1000)
+        assert np.array_equal(np.flatnonzero(taps["xm2"][i]), np.arange(m)), i
+        kept, masked = O.gate_input_channels(taps["xn2"][i], p[i])
+        assert np.array_equal(taps["xm2"][i], masked)
+
+
 # ------------------------------------------------------------------- step ---
 
 
