@@ -197,7 +197,7 @@ sol_status_t sol_sparse_decode_attn(const sol_shape_t *shape, const void *q_bf16
  *   Inputs and outputs as sol_sparse_decode_attn; kept_idx / kept_cnt optional.
  *   status_out (optional, DEVICE int32[8]) receives the status words of this
  *   call (layout as sol_read_device_status) by a copy enqueued on `stream`.
- *   Limit: B * n_kv * (max_pages_per_seq * 64 * (4 G + 12) + 16 KiB) bytes plus small
+ *   Limit: B * n_kv * (max_pages_per_seq * 64 * (4 G + 12) + 24 KiB) bytes plus small
  *   terms must fit the array (for 4 query / 2 kv heads of 64: batch 4 with contexts
  *   up to about 25 thousand tokens); a larger problem is refused with
  *   SOL_ERR_WORKSPACE_TOO_SMALL before anything is launched.

@@ -256,6 +256,8 @@ static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, cons
 
   GemmDown dn;
   dn.t = cs.t_op;
+  dn.t_f32 = cs.t;
+  dn.keep = cs.keep;
   dn.w = w_down;
   dn.live = cs.live;
   dn.M = B;

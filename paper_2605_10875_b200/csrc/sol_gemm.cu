@@ -361,6 +361,98 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_down_kernel(const DownDev 
 }
 
 // ============================================================================
+// down_rows: the down projection of a small batch, row by row
+// ============================================================================
+// At batch <= 8 the union of the channels that some token keeps is well below d_ff when tokens are pruned, and a
+// 64-channel block is almost never dead as a whole: this kernel reads W_down channel by channel and skips
+// every channel that no token keeps, so the bytes follow the union of kept rows.  CTA = (128 output columns,
+// range of channels) as in umma_down; a warp takes every eighth channel of the range: it looks the channel
+// up in the tokens' keep masks, reads the channel's 256 bytes of the slab (two 128-byte pieces of the packed
+// layout, one per column half) and multiplies them into float32 accumulators (<= 8 tokens x 4 columns per
+// lane) on the FMA pipes; the warps are merged through shared memory.
+constexpr int DR_WARPS = 8;
+constexpr int DR_MAXB = 8;
+
+struct DownRowsDev {
+  int M, Mpad, ff, d, chunks;
+  const unsigned char* w;     // packed W_down_t
+  const float* t;             // [M][ff] silu(g) u before masking
+  const unsigned char* keep;  // [M][ff] 1 = kept
+  float* partial;             // [chunks][Mpad][d]
+};
+
+__global__ void __launch_bounds__(DR_WARPS * 32) down_rows_kernel(const DownRowsDev p) {
+  __shared__ float red[DR_WARPS][DR_MAXB][128];
+  const int slab = blockIdx.x, chunk = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int jblocks = (p.ff + 63) / 64;
+  const int j0 = (int)(((long long)p.ff * chunk) / p.chunks), j1 = (int)(((long long)p.ff * (chunk + 1)) / p.chunks);
+  pdl_trigger();
+  pdl_wait();
+  float acc[DR_MAXB][4];
+#pragma unroll
+  for (int m = 0; m < DR_MAXB; ++m)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) acc[m][c] = 0.f;
+#pragma unroll 1
+  for (int jb = j0 + warp * 4; jb < j1; jb += DR_WARPS * 4) {  // four channels per step: their loads are in flight together
+    float tv[4][DR_MAXB];
+    uint32_t wv[4][2];
+    bool any[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = jb + u;
+      any[u] = false;
+#pragma unroll
+      for (int m = 0; m < DR_MAXB; ++m) {
+        tv[u][m] = 0.f;
+        if (j < j1 && m < p.M && p.keep[(size_t)m * p.ff + j]) {  // warp-uniform
+          tv[u][m] = p.t[(size_t)m * p.ff + j];
+          any[u] = true;
+        }
+      }
+      wv[u][0] = wv[u][1] = 0u;
+      if (any[u]) {
+        // channel j of the slab: block j / 64, row c = j % 64; lane l holds columns 2 l, 2 l + 1 of each 64-column half
+        const int c = j & 63;
+        const unsigned char* base = p.w + ((size_t)slab * jblocks + (j >> 6)) * UM_TILE_SPAN + c * 128 +
+                                    (((lane >> 2) ^ (c & 7)) * 16) + (lane & 3) * 4;
+        wv[u][0] = *reinterpret_cast<const uint32_t*>(base);
+        wv[u][1] = *reinterpret_cast<const uint32_t*>(base + 8192);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (!any[u]) continue;
+      const float w0 = bf16_lo(wv[u][0]), w1 = bf16_hi(wv[u][0]), w2 = bf16_lo(wv[u][1]), w3 = bf16_hi(wv[u][1]);
+#pragma unroll
+      for (int m = 0; m < DR_MAXB; ++m) {
+        acc[m][0] = fmaf(tv[u][m], w0, acc[m][0]);
+        acc[m][1] = fmaf(tv[u][m], w1, acc[m][1]);
+        acc[m][2] = fmaf(tv[u][m], w2, acc[m][2]);
+        acc[m][3] = fmaf(tv[u][m], w3, acc[m][3]);
+      }
+    }
+  }
+  // columns of the slab held by lane l: 2 l, 2 l + 1 (first half), 64 + 2 l, 64 + 2 l + 1 (second half)
+#pragma unroll
+  for (int m = 0; m < DR_MAXB; ++m) {
+    red[warp][m][2 * lane] = acc[m][0];
+    red[warp][m][2 * lane + 1] = acc[m][1];
+    red[warp][m][64 + 2 * lane] = acc[m][2];
+    red[warp][m][64 + 2 * lane + 1] = acc[m][3];
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < p.M * 128; i += DR_WARPS * 32) {
+    const int m = i >> 7, c = i & 127;
+    float a = 0.f;
+#pragma unroll
+    for (int w = 0; w < DR_WARPS; ++w) a += red[w][m][c];
+    p.partial[((size_t)chunk * p.Mpad + m) * p.d + slab * 128 + c] = a;
+  }
+}
+
+// ============================================================================
 // one-time packing of the weights
 // ============================================================================
 // One thread per 16-byte piece of the packed matrix.
@@ -496,6 +588,13 @@ int down_chunks(int ff, int d) {
 }
 
 void launch_gemm_down(const GemmDown& g, cudaStream_t st) {
+  if (g.M <= DR_MAXB && g.t_f32 != nullptr && g.keep != nullptr) {  // small batch: channel by channel, only kept rows
+    DownRowsDev r;
+    r.M = g.M; r.Mpad = pad_rows(g.M); r.ff = g.ff; r.d = g.d; r.chunks = g.chunks;
+    r.w = static_cast<const unsigned char*>(g.w); r.t = g.t_f32; r.keep = g.keep; r.partial = g.partial;
+    SOL_LAUNCH("gemm_down_gathered", down_rows_kernel, dim3(g.d / 128, g.chunks), dim3(DR_WARPS * 32), 0, st, r);
+    return;
+  }
   DownDev d;
   memset(&d, 0, sizeof(d));
   d.M = g.M; d.Mpad = pad_rows(g.M); d.ff = g.ff; d.d = g.d;

@@ -171,6 +171,8 @@ void launch_gemm_nk(const GemmNK& p, GemmEpilogue epi, cudaStream_t st);
 
 struct GemmDown {
   const void* t;     // packed masked activations: 2 Mpad rows (high parts, then low parts), K = ff
+  const float* t_f32;         // [M][ff] unmasked t and
+  const unsigned char* keep;  // [M][ff] keep mask: the small-batch kernel reads these instead of the packed operand
   const void* w;     // packed W_down_t
   const int32_t* live;  // [ff/32] non-zero if any token keeps a channel of the granule
   int M, ff, d;

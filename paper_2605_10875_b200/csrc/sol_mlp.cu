@@ -263,7 +263,7 @@ struct ChanMultiSmem {
   int idx[CH_CAND_CAP];
 };
 
-__global__ void __launch_bounds__(CM_THREADS) channel_select_multi_kernel(const ChanDev p) {
+__global__ void __launch_bounds__(CM_THREADS, 3) channel_select_multi_kernel(const ChanDev p) {
   __shared__ ChanMultiSmem sm;
   const int slice = blockIdx.x, b = blockIdx.y, S = gridDim.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
