@@ -44,6 +44,7 @@ struct UmBarriers {
   uint64_t accum;
   uint32_t tmem_base;
   int n_issued;
+  uint32_t gmax[128], umax[128];  // SwiGLU epilogue: per-token maxima of this CTA's channels (float bits)
 };
 
 __device__ __forceinline__ unsigned char* align_1024(unsigned char* p) {
@@ -92,6 +93,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
     mbar_init(&bars->accum, 1);
     fence_mbar_init();
   }
+  if (EPI == EPI_SWIGLU && threadIdx.x < 128) bars->gmax[threadIdx.x] = bars->umax[threadIdx.x] = 0u;
   if (warp == UM_MMA) tmem_alloc(&bars->tmem_base, p.tmem_cols);
   tc_fence_before();
   __syncthreads();
@@ -213,9 +215,9 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
                 if (valid && even) atomicAdd(sel + chan_bin(fabsf(tv)), 1u);
                 const uint32_t gm = __reduce_max_sync(0xffffffffu, valid ? __float_as_uint(fabsf(gg)) : 0u);
                 const uint32_t um = __reduce_max_sync(0xffffffffu, valid ? __float_as_uint(fabsf(uu)) : 0u);
-                if (lane == 0) {
-                  atomicMax(sel + CH_GMAX, gm);
-                  atomicMax(sel + CH_UMAX, um);
+                if (lane == 0) {  // merged over the CTA in shared memory first: one global update per token and CTA
+                  atomicMax(&bars->gmax[m], gm);
+                  atomicMax(&bars->umax[m], um);
                 }
               }
             }
@@ -235,6 +237,11 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
   tc_fence_before();
   __syncthreads();
   if (warp == UM_MMA) tmem_dealloc(tmem, p.tmem_cols);
+  if (EPI == EPI_SWIGLU && p.sel != nullptr && (int)threadIdx.x < p.M) {
+    uint32_t* sel = p.sel + (size_t)threadIdx.x * CH_SEL_WORDS;
+    atomicMax(sel + CH_GMAX, bars->gmax[threadIdx.x]);
+    atomicMax(sel + CH_UMAX, bars->umax[threadIdx.x]);
+  }
 }
 
 // ============================================================================
