@@ -37,6 +37,7 @@ constexpr int UM_PRODUCER = 8, UM_MMA = 9;
 constexpr int UM_MAX_STAGES = 8;
 constexpr int UM_TILE_SPAN = 16384;  // bytes one 128-row operand read spans from the start of a chunk tile
 constexpr int UM_SMEM_BUDGET = 204 * 1024;
+constexpr int UM_LIVE_CAP = 512;     // 64-channel blocks per CTA of the down projection whose live flags are staged in shared memory
 
 struct UmBarriers {
   uint64_t full[UM_MAX_STAGES];
@@ -45,6 +46,8 @@ struct UmBarriers {
   uint32_t tmem_base;
   int n_issued;
   uint32_t gmax[128], umax[128];  // SwiGLU epilogue: per-token maxima of this CTA's channels (float bits)
+  alignas(16) float scale[128];   // SwiGLU epilogue: the tokens' quantizer scales
+  unsigned char live[UM_LIVE_CAP];  // down projection: which of this CTA's 64-channel blocks hold a kept channel
 };
 
 __device__ __forceinline__ unsigned char* align_1024(unsigned char* p) {
@@ -124,14 +127,19 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
         unsigned char* xs = stages + (size_t)it * stage_bytes + p.cps * w_tile;
         bulk_g2s(xs, x_src + (size_t)it * p.cps * x_tile, p.cps * x_tile, &bars->full[it]);
       }
+      // ring position and phase are counted along: a division per stage costs the lone issuing thread ~0.1 us
+      int s = 0;
+      uint32_t ph = 1;
       for (int it = pre; it < n_iter; ++it) {
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
         if (!mbar_wait(&bars->empty[s], ph ^ 1, p.status)) break;
         unsigned char* st = stages + (size_t)s * stage_bytes;
         mbar_expect_tx(&bars->full[s], stage_bytes);
         bulk_g2s(st, w_src + (size_t)it * p.cps * w_tile, p.cps * w_tile, &bars->full[s]);
         bulk_g2s(st + p.cps * w_tile, x_src + (size_t)it * p.cps * x_tile, p.cps * x_tile, &bars->full[s]);
+        if (++s == p.stages) {
+          s = 0;
+          ph ^= 1;
+        }
       }
     }
   } else if (warp == UM_MMA) {
@@ -142,9 +150,9 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
     // the first stage fills only after the producer's own pdl_wait(): without this wait the bounded poll
     // below would start counting while earlier kernels of the stream are still running
     pdl_wait();
+    int s = 0;
+    uint32_t ph = 0;
     for (int it = 0; it < n_iter; ++it) {
-      const int s = it % p.stages;
-      const uint32_t ph = (it / p.stages) & 1;
       ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[s], ph, p.status));
       if (!ok) break;
       const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
@@ -162,11 +170,21 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
       }
       if (elect_one()) umma_commit(&bars->empty[s]);  // the stage is free again once these MMAs have read it
       __syncwarp();
+      if (++s == p.stages) {
+        s = 0;
+        ph ^= 1;
+      }
     }
     if (ok && elect_one()) umma_commit(&bars->accum);
   } else {
     // -------------------------------- epilogue -------------------------------
     pdl_wait();  // the epilogue reads scales and overwrites buffers earlier kernels used
+    if (EPI == EPI_SWIGLU) {
+      // the scales come to shared memory while the weights stream: a global load per token inside the loop
+      // below would put its latency between every two tokens
+      if ((int)threadIdx.x < p.Mpad) bars->scale[threadIdx.x] = (p.row_scale && (int)threadIdx.x < p.M) ? p.row_scale[threadIdx.x] : 1.0f;
+      asm volatile("bar.sync 1, 256;" ::: "memory");  // the eight epilogue warps
+    }
     // warps w and w + 4 share the accumulator lanes 32 (w % 4) .. and take alternate groups of 16 tokens
     const int quarter = warp & 3, half = warp >> 2;
     if (quarter * 32 < p.R) {
@@ -184,42 +202,59 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
           for (int i = 0; i < 16; ++i) v[i] += w2[i];
         }
         if (EPI == EPI_SWIGLU) {
-          // even lanes hold a channel's gate sum, their odd neighbours its up sum
+          // Even lanes hold a channel's gate sum, their odd neighbours its up sum.  The 16 tokens of the group are
+          // taken through each step together (no branch per token), so that the exchanges, exponentials and
+          // divisions of different tokens overlap: token by token the dependent chain cost ~0.6 us per token.
           const int ch = (tile * p.R + r) >> 1;
           const bool valid = r < p.R && ch < p.N;
           const bool even = (lane & 1) == 0;
+          const int nt = min(16, p.M - c0);  // tokens of this group that exist (warp-uniform)
+          float gg[16], uu[16], tv[16];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float4 sc = *reinterpret_cast<const float4*>(&bars->scale[c0 + 4 * q]);
+            v[4 * q + 0] *= sc.x;
+            v[4 * q + 1] *= sc.y;
+            v[4 * q + 2] *= sc.z;
+            v[4 * q + 3] *= sc.w;
+          }
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const int m = c0 + i;
-            if (m < p.M) {  // warp-uniform
-              const float sc = p.row_scale ? p.row_scale[m] : 1.0f;
-              const float mine = v[i] * sc;
-              const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
-              const float gg = even ? mine : other, uu = even ? other : mine;
-              // exp by the fast exponential: its relative error (about 2^-21 |g|) is far inside the error the channel
-              // selection already allows for g itself
-              const float tv = (gg / (1.0f + __expf(-gg))) * uu;
-              const size_t o = (size_t)m * p.N + ch;
-              if (valid) {
-                if (even) {
-                  p.out0[o] = gg;
-                  p.out2[o] = tv;
-                } else {
-                  p.out1[o] = uu;
-                }
+            const float other = __shfl_xor_sync(0xffffffffu, v[i], 1);
+            gg[i] = even ? v[i] : other;
+            uu[i] = even ? other : v[i];
+          }
+          // exp by the fast exponential: its relative error (about 2^-21 |g|) is far inside the error the channel
+          // selection already allows for g itself
+#pragma unroll
+          for (int i = 0; i < 16; ++i) tv[i] = (gg[i] / (1.0f + __expf(-gg[i]))) * uu[i];
+          float* const dst = even ? p.out0 : p.out1;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            if (i < nt && valid) {
+              const size_t o = (size_t)(c0 + i) * p.N + ch;
+              dst[o] = even ? gg[i] : uu[i];
+              if (even) p.out2[o] = tv[i];
+            }
+          }
+          if (p.sel != nullptr) {
+            // what the channel selection needs from all of a token's channels: a histogram of |t| and the largest
+            // |g|, |u| (non-negative floats order like their bit patterns); the maxima are merged over the CTA in
+            // shared memory first: one global update per token and CTA
+            uint32_t gsel = 0u, usel = 0u;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              if (i < nt && valid && even) atomicAdd(p.sel + (size_t)(c0 + i) * CH_SEL_WORDS + chan_bin(fabsf(tv[i])), 1u);
+              const uint32_t gm = __reduce_max_sync(0xffffffffu, valid ? __float_as_uint(fabsf(gg[i])) : 0u);
+              const uint32_t um = __reduce_max_sync(0xffffffffu, valid ? __float_as_uint(fabsf(uu[i])) : 0u);
+              if (lane == i) {
+                gsel = gm;
+                usel = um;
               }
-              if (p.sel != nullptr) {
-                // what the channel selection needs from all of a token's channels: a histogram of |t|
-                // and the largest |g|, |u| (non-negative floats order like their bit patterns)
-                uint32_t* sel = p.sel + (size_t)m * CH_SEL_WORDS;
-                if (valid && even) atomicAdd(sel + chan_bin(fabsf(tv)), 1u);
-                const uint32_t gm = __reduce_max_sync(0xffffffffu, valid ? __float_as_uint(fabsf(gg)) : 0u);
-                const uint32_t um = __reduce_max_sync(0xffffffffu, valid ? __float_as_uint(fabsf(uu)) : 0u);
-                if (lane == 0) {  // merged over the CTA in shared memory first: one global update per token and CTA
-                  atomicMax(&bars->gmax[m], gm);
-                  atomicMax(&bars->umax[m], um);
-                }
-              }
+            }
+            if (lane < nt) {
+              atomicMax(&bars->gmax[c0 + lane], gsel);
+              atomicMax(&bars->umax[c0 + lane], usel);
             }
           }
         } else {
@@ -291,31 +326,38 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_down_kernel(const DownDev 
   const int granules = p.ff / 32, jblocks = (p.ff + 63) / 64;
   const int jb0 = (int)(((long long)jblocks * chunk) / p.chunks);
   const int jb1 = (int)(((long long)jblocks * (chunk + 1)) / p.chunks);
+  // the flags of this CTA's blocks, read by all threads at once: the producer and the MMA issuer walk the
+  // same list, and a global load per block would put its latency between every two copies
+  const bool staged = jb1 - jb0 <= UM_LIVE_CAP;
+  if (staged) {
+    for (int i = threadIdx.x; i < jb1 - jb0; i += UM_THREADS) bars->live[i] = block_live(p.live, jb0 + i, granules) ? 1 : 0;
+    __syncthreads();
+  }
 
   if (warp == UM_PRODUCER) {
     if (lane == 0) {
-      int it = 0;
+      int s = 0;
+      uint32_t ph = 0;
       for (int jb = jb0; jb < jb1; ++jb) {
-        if (!block_live(p.live, jb, granules)) continue;
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
-        ++it;
+        if (!(staged ? bars->live[jb - jb0] != 0 : block_live(p.live, jb, granules))) continue;
         if (!mbar_wait(&bars->empty[s], ph ^ 1, p.status)) break;
         unsigned char* st = stages + (size_t)s * stage_bytes;
         mbar_expect_tx(&bars->full[s], stage_bytes);
         bulk_g2s(st, p.w + ((size_t)slab * jblocks + jb) * UM_TILE_SPAN, UM_TILE_SPAN, &bars->full[s]);
         bulk_g2s(st + UM_TILE_SPAN, p.t + (size_t)jb * t_tile, t_tile, &bars->full[s]);  // high rows then low rows
+        if (++s == p.stages) {
+          s = 0;
+          ph ^= 1;
+        }
       }
     }
   } else if (warp == UM_MMA) {
     const uint32_t idesc = umma_idesc_bf16_m128(2 * p.Mpad, 1, 0);
     bool acc = false, ok = true;
-    int it = 0;
+    int s = 0;
+    uint32_t ph = 0;
     for (int jb = jb0; jb < jb1; ++jb) {
-      if (!block_live(p.live, jb, granules)) continue;
-      const int s = it % p.stages;
-      const uint32_t ph = (it / p.stages) & 1;
-      ++it;
+      if (!(staged ? bars->live[jb - jb0] != 0 : block_live(p.live, jb, granules))) continue;
       ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[s], ph, p.status));
       if (!ok) break;
       const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
@@ -330,6 +372,10 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_down_kernel(const DownDev 
       }
       if (elect_one()) umma_commit(&bars->empty[s]);
       __syncwarp();
+      if (++s == p.stages) {
+        s = 0;
+        ph ^= 1;
+      }
     }
     if (lane == 0) {
       *reinterpret_cast<volatile int*>(&bars->n_issued) = acc ? 1 : 0;
