@@ -455,8 +455,9 @@ def run_ours(args):
         v["share"] = round(v["us_per_step"] / tot_us, 4)
         v["us_per_launch"] = round(v["us_per_launch"], 3)
         v["us_per_step"] = round(v["us_per_step"], 3)
-    for name, nbytes in kb.items():
+    for name, nbytes in kb.items():  # nbytes: one layer's bytes for this kernel; the attention kernels run once per group of sequences
         if name in per_kernel:
+            nbytes = nbytes * rep.L / max(1, per_kernel[name]["launches_per_step"])
             per_kernel[name]["bytes_per_launch"] = int(nbytes)
             per_kernel[name]["gbs"] = round(nbytes / per_kernel[name]["us_per_launch"] / 1e3, 1)
             per_kernel[name]["frac_of_measured"] = round(per_kernel[name]["gbs"] / peak_gbs, 4)
