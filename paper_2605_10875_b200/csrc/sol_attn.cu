@@ -35,6 +35,7 @@ constexpr int PAGE = 64;
 // selection (histogram), 2048-token segments (scan).  Entry b is the count before sequence b, entry B the total.
 enum : int { PLAN_PAGES = 0, PLAN_HSEG = 1, PLAN_SSEG = 2, PLAN_LISTS = 3 };
 constexpr int PLAN_STRIDE = 132;
+constexpr int PLAN_GROUP_TOKENS = 4 * PAGE;  // tokens of one pass-1 unit (a CTA of attn_score: one page per warp)
 constexpr int TH_SEG = 8192;  // tokens per token_hist CTA
 constexpr int TS_SEG = 2048;  // tokens per token_scan CTA
 
@@ -287,103 +288,157 @@ struct ScoreDev {
   const uint16_t* q_split;
   float* logits;
   float* sigma;
+  int B;
   int* status;
 };
 
 constexpr int SC_WARPS = 4;  // pages per CTA
+static_assert(SC_WARPS * PAGE == PLAN_GROUP_TOKENS, "a unit of attn_score is one page per warp");
+constexpr int SC_MAX_GRID = 32768;  // CTAs launched at most; beyond that a CTA takes several units
 
-template <int HD, int HG>
+template <int HD, int HG, bool FLAT>
 __global__ void __launch_bounds__(SC_WARPS * 32) attn_score_kernel(const ScoreDev p) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int PAGE_BYTES = PAGE * HD * 2;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SC_WARPS * PAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = blockIdx.z, kvh = blockIdx.y;
   pdl_trigger();
-  // The grid covers the longest row the page table allows; the CTAs beyond this sequence's length leave
-  // before anything else (the lengths are an input of the step, not the work of an earlier kernel).
-  if (blockIdx.x * SC_WARPS * PAGE >= p.kv.seq_lens[b]) return;
+  // Two ways to give the CTAs their unit (sequence, kv-head, group of four pages).  Direct (FLAT = false): a
+  // 3-D grid over the longest row the page table allows; CTAs beyond their sequence's length leave at once.
+  // That is the cheapest mapping, but an empty CTA costs ~0.5 ns of CTA issue: 70 us for the 131072 CTAs of
+  // 128 ragged sequences, four in five of them empty.  Flat (FLAT = true, chosen by the host when the direct
+  // grid would exceed SC_MAX_GRID): the units that exist are numbered along the batch; every CTA adds up the
+  // sequences' group counts itself from the lengths (an input of the step, so before the wait for the
+  // earlier kernels) and takes every gridDim.x-th unit.  The flat mapping costs each CTA two block
+  // barriers and a block-wide count, which made uniform batches 6-15 % slower, hence both.
+  __shared__ int s_cum[SC_WARPS * 32 + 1], s_len[SC_WARPS * 32], s_wsum[SC_WARPS];
+  int my_incl = 0, n_units = 1;
+  if (FLAT) {
+    const int tid = threadIdx.x;
+    int Tt = 0;
+    if (tid < p.B) Tt = min(max(p.kv.seq_lens[tid], 0), p.kv.max_pages_per_seq * PAGE);  // never index past the page table
+    my_incl = (Tt + PLAN_GROUP_TOKENS - 1) / PLAN_GROUP_TOKENS;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int x = __shfl_up_sync(0xffffffffu, my_incl, o);
+      if (lane >= o) my_incl += x;
+    }
+    if (lane == 31) s_wsum[warp] = my_incl;
+    if (tid == 0) s_cum[0] = 0;
+    __syncthreads();
+    for (int w = 0; w < warp; ++w) my_incl += s_wsum[w];
+    s_cum[tid + 1] = my_incl;
+    s_len[tid] = Tt;
+    __syncthreads();
+    n_units = s_cum[p.B] * p.Hkv;
+    if ((int)blockIdx.x >= n_units) return;
+  } else {
+    if (blockIdx.x * SC_WARPS * PAGE >= p.kv.seq_lens[blockIdx.z]) return;
+  }
   if (threadIdx.x == 0) {
     for (int i = 0; i < SC_WARPS; ++i) mbar_init(&bars[i], 1);
     fence_mbar_init();
   }
   __syncthreads();
   pdl_wait();
-
-  const int T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
-  const int lp = blockIdx.x * SC_WARPS + warp;  // logical page
-  if (lp * PAGE >= T || lp >= p.kv.max_pages_per_seq) return;
-  const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + lp];
-  if (page < 0 || page >= p.kv.num_pages) {
-    if (lane == 0) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
-    return;
-  }
-  unsigned char* tile = smem + warp * PAGE_BYTES;
-  if (lane == 0) {
-    mbar_expect_tx(&bars[warp], PAGE_BYTES);
-    bulk_g2s(tile, static_cast<const uint16_t*>(p.kv.k_pool) + ((size_t)page * p.Hkv + kvh) * PAGE * HD, PAGE_BYTES,
-             &bars[warp]);
-  }
-
-  // query operand fragments: B[k][n] = q_split[n][k]; this lane holds rows g and 8+g, 8 k-values per pair step
   const int g = lane >> 2, t = lane & 3;
   constexpr int KS = HD / 32;  // pair steps (two MMAs of k=16 each)
-  uint4 qf[HG][KS][2];
-#pragma unroll
-  for (int hg = 0; hg < HG; ++hg) {
-    const uint16_t* qb = p.q_split + ((size_t)((b * p.Hkv + kvh) * HG + hg) * 16) * HD;
-#pragma unroll
-    for (int s = 0; s < KS; ++s) {
-      qf[hg][s][0] = *reinterpret_cast<const uint4*>(qb + (size_t)g * HD + s * 32 + t * 8);
-      qf[hg][s][1] = *reinterpret_cast<const uint4*>(qb + (size_t)(8 + g) * HD + s * 32 + t * 8);
-    }
-  }
-
-  const bool ok = mbar_wait(&bars[warp], 0, p.status);
-  if (!ok) return;
-
-  const uint32_t tb = smem_u32(tile);
-  const size_t row0 = ((size_t)b * p.Hkv + kvh) * p.Tmax;
+  uint32_t phase = 0;
+  bool dead = false;  // a wait ran out: no more work, but the block-wide counts below still need this warp
 #pragma unroll 1
-  for (int mt = 0; mt < PAGE / 16; ++mt) {
-    uint4 ka[KS][2];
-#pragma unroll
-    for (int s = 0; s < KS; ++s) {
-      ka[s][0] = lds128(tb + (mt * 16 + g) * (HD * 2) + (s * 32 + t * 8) * 2);
-      ka[s][1] = lds128(tb + (mt * 16 + g + 8) * (HD * 2) + (s * 32 + t * 8) * 2);
+  for (int u = FLAT ? blockIdx.x : 0; u < n_units; u += gridDim.x) {
+    int b, kvh, grp, T;
+    if (FLAT) {
+      // sequence of unit u: how many cumulative counts lie at or below u / Hkv
+      const int key = u / p.Hkv;
+      b = __syncthreads_count((int)threadIdx.x < p.B && my_incl <= key);
+      const int first = s_cum[b], n_groups = s_cum[b + 1] - first;
+      const int rem = u - first * p.Hkv;
+      kvh = rem / n_groups;
+      grp = rem - kvh * n_groups;
+      T = s_len[b];
+    } else {
+      b = blockIdx.z;
+      kvh = blockIdx.y;
+      grp = blockIdx.x;
+      T = min(p.kv.seq_lens[b], p.kv.max_pages_per_seq * PAGE);  // never index past the page table
     }
-    float sig0 = 0.f, sig1 = 0.f;  // tokens g and g+8 of this m-tile
-    const int tok0 = lp * PAGE + mt * 16 + g, tok1 = tok0 + 8;
+    const int lp = grp * SC_WARPS + warp;  // logical page
+    if (dead || lp * PAGE >= T || lp >= p.kv.max_pages_per_seq) continue;
+    const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + lp];
+    if (page < 0 || page >= p.kv.num_pages) {
+      if (lane == 0) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+      continue;
+    }
+    unsigned char* tile = smem + warp * PAGE_BYTES;
+    if (lane == 0) {
+      mbar_expect_tx(&bars[warp], PAGE_BYTES);
+      bulk_g2s(tile, static_cast<const uint16_t*>(p.kv.k_pool) + ((size_t)page * p.Hkv + kvh) * PAGE * HD, PAGE_BYTES,
+               &bars[warp]);
+    }
+
+    // query operand fragments: B[k][n] = q_split[n][k]; this lane holds rows g and 8+g, 8 k-values per pair step
+    uint4 qf[HG][KS][2];
 #pragma unroll
     for (int hg = 0; hg < HG; ++hg) {
-      float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+      const uint16_t* qb = p.q_split + ((size_t)((b * p.Hkv + kvh) * HG + hg) * 16) * HD;
 #pragma unroll
       for (int s = 0; s < KS; ++s) {
-        mma_bf16(d0, ka[s][0].x, ka[s][1].x, ka[s][0].y, ka[s][1].y, qf[hg][s][0].x, qf[hg][s][0].y);
-        mma_bf16(d0, ka[s][0].z, ka[s][1].z, ka[s][0].w, ka[s][1].w, qf[hg][s][0].z, qf[hg][s][0].w);
-        mma_bf16(d1, ka[s][0].x, ka[s][1].x, ka[s][0].y, ka[s][1].y, qf[hg][s][1].x, qf[hg][s][1].y);
-        mma_bf16(d1, ka[s][0].z, ka[s][1].z, ka[s][0].w, ka[s][1].w, qf[hg][s][1].z, qf[hg][s][1].w);
+        qf[hg][s][0] = *reinterpret_cast<const uint4*>(qb + (size_t)g * HD + s * 32 + t * 8);
+        qf[hg][s][1] = *reinterpret_cast<const uint4*>(qb + (size_t)(8 + g) * HD + s * 32 + t * 8);
       }
-      // columns 2t, 2t+1 of the first n-tile are head t's hi and mid parts; column 2t of the second its lo part
-      const float s0 = d0[0] + (d0[1] + d1[0]);
-      const float s1 = d0[2] + (d0[3] + d1[2]);
-      const int head = hg * 4 + t;
-      if (head < p.G) {
-        if (tok0 < T) p.logits[(row0 + tok0) * p.G + head] = s0;
-        if (tok1 < T) p.logits[(row0 + tok1) * p.G + head] = s1;
+    }
+
+    if (!mbar_wait(&bars[warp], phase, p.status)) {
+      dead = true;
+      continue;
+    }
+    phase ^= 1;
+
+    const uint32_t tb = smem_u32(tile);
+    const size_t row0 = ((size_t)b * p.Hkv + kvh) * p.Tmax;
+#pragma unroll 1
+    for (int mt = 0; mt < PAGE / 16; ++mt) {
+      uint4 ka[KS][2];
+#pragma unroll
+      for (int s = 0; s < KS; ++s) {
+        ka[s][0] = lds128(tb + (mt * 16 + g) * (HD * 2) + (s * 32 + t * 8) * 2);
+        ka[s][1] = lds128(tb + (mt * 16 + g + 8) * (HD * 2) + (s * 32 + t * 8) * 2);
       }
-      float q0 = s0, q1 = s1;  // rows of absent heads are zero, so they add nothing
-      q0 += __shfl_xor_sync(0xffffffffu, q0, 1);
-      q1 += __shfl_xor_sync(0xffffffffu, q1, 1);
-      q0 += __shfl_xor_sync(0xffffffffu, q0, 2);
-      q1 += __shfl_xor_sync(0xffffffffu, q1, 2);
-      sig0 += q0;
-      sig1 += q1;
+      float sig0 = 0.f, sig1 = 0.f;  // tokens g and g+8 of this m-tile
+      const int tok0 = lp * PAGE + mt * 16 + g, tok1 = tok0 + 8;
+#pragma unroll
+      for (int hg = 0; hg < HG; ++hg) {
+        float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int s = 0; s < KS; ++s) {
+          mma_bf16(d0, ka[s][0].x, ka[s][1].x, ka[s][0].y, ka[s][1].y, qf[hg][s][0].x, qf[hg][s][0].y);
+          mma_bf16(d0, ka[s][0].z, ka[s][1].z, ka[s][0].w, ka[s][1].w, qf[hg][s][0].z, qf[hg][s][0].w);
+          mma_bf16(d1, ka[s][0].x, ka[s][1].x, ka[s][0].y, ka[s][1].y, qf[hg][s][1].x, qf[hg][s][1].y);
+          mma_bf16(d1, ka[s][0].z, ka[s][1].z, ka[s][0].w, ka[s][1].w, qf[hg][s][1].z, qf[hg][s][1].w);
+        }
+        // columns 2t, 2t+1 of the first n-tile are head t's hi and mid parts; column 2t of the second its lo part
+        const float s0 = d0[0] + (d0[1] + d1[0]);
+        const float s1 = d0[2] + (d0[3] + d1[2]);
+        const int head = hg * 4 + t;
+        if (head < p.G) {
+          if (tok0 < T) p.logits[(row0 + tok0) * p.G + head] = s0;
+          if (tok1 < T) p.logits[(row0 + tok1) * p.G + head] = s1;
+        }
+        float q0 = s0, q1 = s1;  // rows of absent heads are zero, so they add nothing
+        q0 += __shfl_xor_sync(0xffffffffu, q0, 1);
+        q1 += __shfl_xor_sync(0xffffffffu, q1, 1);
+        q0 += __shfl_xor_sync(0xffffffffu, q0, 2);
+        q1 += __shfl_xor_sync(0xffffffffu, q1, 2);
+        sig0 += q0;
+        sig1 += q1;
+      }
+      if (t == 0) {
+        if (tok0 < T) p.sigma[row0 + tok0] = sig0 + 0.0f;  // -0 becomes +0: the selection compares floats and keys
+        if (tok1 < T) p.sigma[row0 + tok1] = sig1 + 0.0f;
+      }
     }
-    if (t == 0) {
-      if (tok0 < T) p.sigma[row0 + tok0] = sig0 + 0.0f;  // -0 becomes +0: the selection compares floats and keys
-      if (tok1 < T) p.sigma[row0 + tok1] = sig1 + 0.0f;
-    }
+    __syncwarp();  // the tile is rewritten by the next unit's copy
   }
 }
 
@@ -1435,15 +1490,24 @@ __global__ void __launch_bounds__(GatherCfg<HD, GMAX>::THREADS, 1) attn_gather_k
 // ============================================================================
 // host side
 // ============================================================================
-template <int HD>
-static void launch_score(const ScoreDev& d, int HG, dim3 grid, cudaStream_t st) {
+template <int HD, int HG, bool FLAT>
+static void launch_score_as(const ScoreDev& d, dim3 grid, cudaStream_t st) {
   const int smem = SC_WARPS * PAGE * HD * 2 + SC_WARPS * 8 + 32;
-  if (HG == 1) {
-    ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_score_kernel<HD, 1>), smem);
-    SOL_LAUNCH("attn_score", (attn_score_kernel<HD, 1>), grid, dim3(SC_WARPS * 32), smem, st, d);
+  ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_score_kernel<HD, HG, FLAT>), smem);
+  SOL_LAUNCH("attn_score", (attn_score_kernel<HD, HG, FLAT>), grid, dim3(SC_WARPS * 32), smem, st, d);
+}
+// Direct 3-D grid while it stays within SC_MAX_GRID CTAs, else the flat numbering of the units that exist.
+template <int HD>
+static void launch_score(const ScoreDev& d, int HG, int groups_per_row, cudaStream_t st) {
+  const long long direct = (long long)groups_per_row * d.Hkv * d.B;
+  if (direct <= SC_MAX_GRID) {
+    const dim3 grid(groups_per_row, d.Hkv, d.B);
+    if (HG == 1) launch_score_as<HD, 1, false>(d, grid, st);
+    else launch_score_as<HD, 2, false>(d, grid, st);
   } else {
-    ensure_dynamic_smem(reinterpret_cast<const void*>(&attn_score_kernel<HD, 2>), smem);
-    SOL_LAUNCH("attn_score", (attn_score_kernel<HD, 2>), grid, dim3(SC_WARPS * 32), smem, st, d);
+    const dim3 grid(SC_MAX_GRID);
+    if (HG == 1) launch_score_as<HD, 1, true>(d, grid, st);
+    else launch_score_as<HD, 2, true>(d, grid, st);
   }
 }
 
@@ -1477,10 +1541,10 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   ScoreDev sd;
   sd.kv = a.kv; sd.Hkv = Hkv; sd.G = G; sd.HG = HG; sd.Tmax = Tmax;
   sd.q_split = static_cast<const uint16_t*>(a.q_split);
-  sd.logits = a.logits; sd.sigma = a.sigma; sd.status = a.status;
-  dim3 sgrid((a.kv.max_pages_per_seq + SC_WARPS - 1) / SC_WARPS, Hkv, a.B);
-  if (hd == 64) launch_score<64>(sd, HG, sgrid, st);
-  else launch_score<128>(sd, HG, sgrid, st);
+  sd.logits = a.logits; sd.sigma = a.sigma; sd.status = a.status; sd.B = a.B;
+  const int groups_per_row = (a.kv.max_pages_per_seq + SC_WARPS - 1) / SC_WARPS;
+  if (hd == 64) launch_score<64>(sd, HG, groups_per_row, st);
+  else launch_score<128>(sd, HG, groups_per_row, st);
 
   SelectDev se;
   se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.S = a.splits;

@@ -180,14 +180,11 @@ def test_ragged_serving_steps_across_an_action_redraw_every_layer():
         stack.step_and_check(lens, synth.make_hidden(cfg, 100 + s), r, p, b, f"ragged serving step {s}")
 
 
-def test_attention_ragged_batch_128_sets():
-    """The stand-alone attention call on the ragged batch-128 contexts (one layer's cache): index sets and
-    outputs of eight sampled sequences, among them the shortest and the longest, against the oracle."""
-    cfg = synth.WORKLOADS["ragged_serving"]
+def _attention_sets_case(cfg, lens, r, extra_sample, label):
+    """The stand-alone attention call on a batch of contexts (one layer's cache): kept counts of every sequence,
+    index sets and outputs of sampled sequences, among them the shortest and the longest, against the oracle."""
     shape, oshape = H.make_shapes(cfg)
     B, Hq, Hkv, hd = cfg["batch"], cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"]
-    lens = synth.make_contexts(cfg, 0)
-    r, _, _ = synth.draw_actions(cfg, 0)
     table, n_pages = synth.make_page_table(lens, True, 0)
     tab = np.where(table < 0, 0, table).astype(np.int32)
     k, v = synth.device_kv_pool(cfg, n_pages, H.DEV, 0, 0)
@@ -206,8 +203,7 @@ def test_attention_ragged_batch_128_sets():
     cnt = kept_cnt.cpu().numpy()
     for i in range(B):
         assert np.all(cnt[i] == O.kept_token_count(int(r[i]), int(lens[i]), 1)), i
-    sample = sorted(set([int(np.argmin(lens)), int(np.argmax(lens))] + [int(np.flatnonzero(r == x)[0]) for x in cfg["r_set"]]
-                        + [3, 50, 90, 127]))[:9]
+    sample = sorted(set([int(np.argmin(lens)), int(np.argmax(lens))] + extra_sample))[:9]
     # compact host cache of the sampled sequences
     need = [(int(lens[i]) + 63) // 64 for i in sample]
     pages = np.concatenate([tab[i, :n] for i, n in zip(sample, need)])
@@ -222,7 +218,28 @@ def test_attention_ragged_batch_128_sets():
     idx = kept_idx.cpu().numpy()
     kept = [[idx[i, h, : cnt[i, h]] for h in range(Hkv)] for i in sample]
     par = H.check_token_sets(oshape, sigma, kept_o, kept, lens[sample])
-    H.assert_sets(par, "ragged token sets")
+    H.assert_sets(par, label + " token sets")
     got = synth.bf16_to_f32(H.host_u16(out)).astype(np.float64)[sample]
-    err = H.assert_outputs(out_o, got, "ragged attention output")
-    print("ragged attention: sampled", sample, "contexts", lens[sample].tolist(), par, "status", st, "err", err)
+    err = H.assert_outputs(out_o, got, label + " attention output")
+    print(label, "attention: sampled", sample, "contexts", lens[sample].tolist(), par, "status", st, "err", err)
+
+
+def test_attention_ragged_batch_128_sets():
+    """Ragged batch-128 contexts: the scoring pass numbers the units that exist (flat grid)."""
+    cfg = synth.WORKLOADS["ragged_serving"]
+    lens = synth.make_contexts(cfg, 0)
+    r, _, _ = synth.draw_actions(cfg, 0)
+    extra = [int(np.flatnonzero(r == x)[0]) for x in cfg["r_set"]] + [3, 50, 90, 127]
+    _attention_sets_case(cfg, lens, r, extra, "ragged")
+
+
+def test_attention_batch_128_long_contexts_more_units_than_ctas():
+    """128 sequences of 15000..16384 tokens: 65536 units of the scoring pass for a grid of 32768 CTAs, so every
+    CTA takes two units (the second with the other phase of its copy barriers)."""
+    cfg = dict(synth.WORKLOADS["ragged_serving"])
+    rng = np.random.default_rng(11)
+    lens = rng.integers(15000, 16385, size=cfg["batch"]).astype(np.int32)
+    lens[5] = 16384
+    r, _, _ = synth.draw_actions(cfg, 0)
+    extra = [int(np.flatnonzero(r == x)[0]) for x in cfg["r_set"]][:3] + [127]
+    _attention_sets_case(cfg, lens, r, extra, "long contexts")
