@@ -35,6 +35,10 @@ Readings taken where the paper is silent or the benchmark spec overrides it:
     smallest |silu(g)*u| per token (the task's default); the paper's own
     form, gating the MLP block's input channels by |x|, is PRUNE_MLP_INPUT;
     the kept count mirrors the paper's ceil form in both;
+  * the paper's own selection, SELECT_QUEST_PAGES (quest_decode_attn): pages
+    of S contiguous tokens from token 0, extrema of a partial last page over
+    the keys that exist, top ceil(b_t / S) pages per QUERY head, the page of
+    the newest token always among them, every key of a kept page attended;
   * ties are broken toward the lower index;
   * T (seq_lens) counts the newest token, whose k/v the layer appends
     before attention reads the cache.
@@ -336,6 +340,97 @@ def sparse_decode_attn(shape: Shape, q: np.ndarray, kv: PagedKV, r_permille: Seq
         kept_all.append(kept_i)
         sigma_all.append(sigma_i)
     return out, kept_all, sigma_all
+
+
+# ----------------------------------------------------------------------------
+# The paper's own token sparsity: Quest page selection per query head
+# (appendix on efficiency actions, "Token sparsity via Quest": "Budgeted token
+# selection", "Quest masking in LLaMA attention", "Granularity")
+# ----------------------------------------------------------------------------
+SELECT_TOKENS = 0       # the task's default: exact top-k tokens per (sequence, kv-head) (sparse_decode_attn)
+SELECT_QUEST_PAGES = 1  # the paper's: top pages per query head by the Quest bound (quest_decode_attn)
+
+
+def quest_page_extrema(K: np.ndarray, S: int):
+    """K float64 [T][hd] -> (m_plus, m_minus), each [ceil(T/S)][hd]: per-dimension
+    m+ = max_j k_j and m- = -min_j k_j over the keys of each page of S contiguous
+    tokens.  The last page may hold fewer than S keys; the padding the paper adds
+    is masked there, so here the extrema run over the keys that exist."""
+    T = K.shape[0]
+    P = (T + S - 1) // S
+    m_plus = np.stack([K[pg * S:min((pg + 1) * S, T)].max(axis=0) for pg in range(P)])
+    m_minus = np.stack([-K[pg * S:min((pg + 1) * S, T)].min(axis=0) for pg in range(P)])
+    return m_plus, m_minus
+
+
+def quest_page_scores(q: np.ndarray, m_plus: np.ndarray, m_minus: np.ndarray) -> np.ndarray:
+    """score(page) = q_pos . m+ + q_neg . m-, with q_pos = |q| * [q >= 0] and
+    q_neg = |q| - q_pos (one query head, q float64 [hd])."""
+    a = np.abs(q)
+    q_pos = a * (q >= 0)
+    q_neg = a - q_pos
+    return m_plus @ q_pos + m_minus @ q_neg
+
+
+def quest_kept_page_count(r_permille: int, T: int, S: int, n_forced_pages: int) -> int:
+    """ceil(b_t / S) pages with b_t = ceil(kappa_t K_t) clamped to [0, K_t], never
+    more than there are pages, never fewer than the forced ones (the page of the
+    newest token, so that the step always attends to it)."""
+    if not 0 <= r_permille <= 1000:
+        raise ValueError("r_permille out of range")
+    b = min(max((int(r_permille) * int(T) + 999) // 1000, 0), T)
+    P = (T + S - 1) // S
+    return min(P, max((b + S - 1) // S, n_forced_pages))
+
+
+def quest_attention_one_group(q_group: np.ndarray, K: np.ndarray, V: np.ndarray, S: int, n_keep: int,
+                              forced_pages: np.ndarray):
+    """One (sequence, kv-head): every query head of the group picks its own
+    n_keep pages (forced ones first, then by score descending, page index
+    ascending), attends to all keys of its pages and to nothing else (additive
+    -inf on the others) with logits q . k / sqrt(hd).  Returns out [G][hd], the
+    kept page indices per head (ascending) and the scores [G][pages]."""
+    G, hd = q_group.shape
+    T = K.shape[0]
+    m_plus, m_minus = quest_page_extrema(K, S)
+    out = np.zeros((G, hd))
+    kept_pages, scores = [], []
+    for h in range(G):
+        sc = quest_page_scores(q_group[h], m_plus, m_minus)
+        pages = select_top(sc, n_keep, forced_pages)
+        tok = np.concatenate([np.arange(pg * S, min((pg + 1) * S, T)) for pg in pages])
+        logit = K[tok] @ q_group[h] / math.sqrt(hd)
+        w = np.exp(logit - logit.max())
+        w /= w.sum()
+        out[h] = w @ V[tok]
+        kept_pages.append(pages)
+        scores.append(sc)
+    return out, kept_pages, np.stack(scores)
+
+
+def quest_decode_attn(shape: Shape, q: np.ndarray, kv: PagedKV, r_permille: Sequence[int], S: int):
+    """q float64 [B][Hq][hd] (already rotated).  Returns out float64 [B][Hq][hd],
+    kept_pages[i][query head] and scores[i][query head] (per-page bounds)."""
+    B = q.shape[0]
+    G = shape.group
+    out = np.zeros((B, shape.n_q_heads, shape.head_dim))
+    kept_all, score_all = [], []
+    for i in range(B):
+        T = int(kv.seq_lens[i])
+        forced_tok = forced_keep_set(T, shape.n_sink, shape.n_window)
+        forced_pages = np.unique(forced_tok // S)
+        n_keep = quest_kept_page_count(int(r_permille[i]), T, S, len(forced_pages))
+        kept_i, score_i = [], []
+        for kvh in range(shape.n_kv_heads):
+            K = cache_rows(kv.k_pool, kv.page_table[i], T, kvh)
+            V = cache_rows(kv.v_pool, kv.page_table[i], T, kvh)
+            o, pages, sc = quest_attention_one_group(q[i, kvh * G:(kvh + 1) * G], K, V, S, n_keep, forced_pages)
+            out[i, kvh * G:(kvh + 1) * G] = o
+            kept_i.extend(pages)
+            score_i.extend(list(sc))
+        kept_all.append(kept_i)
+        score_all.append(score_i)
+    return out, kept_all, score_all
 
 
 # ----------------------------------------------------------------------------

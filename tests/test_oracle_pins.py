@@ -404,6 +404,134 @@ def test_duplicate_keys_prefer_lower_index_and_sink_window():
     assert list(kept[0][0]) == [0, 1, 9, 10, 11]
 
 
+# ---------------------------------------------------------------------------
+# the paper's own token sparsity: Quest pages per query head
+# ---------------------------------------------------------------------------
+def _quest_golden():
+    rows = []
+    for line in open(os.path.join(GOLDEN, "quest_cases.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        S, q, keys, r, scores, pages = [f.strip() for f in line.split(";")]
+        rows.append((int(S), np.array(q.split(), float), np.array([k.split() for k in keys.split("|")], float), int(r),
+                     np.array(scores.split(), float), np.array(pages.split(), int)))
+    return rows
+
+
+def test_quest_golden_scores_and_pages():
+    rows = _quest_golden()
+    assert len(rows) >= 9
+    for S, q, K, r, scores, pages in rows:
+        T = K.shape[0]
+        mp, mm = O.quest_page_extrema(K, S)
+        assert np.array_equal(O.quest_page_scores(q, mp, mm), scores)
+        forced = np.unique(O.forced_keep_set(T, 0, 1) // S)
+        n = O.quest_kept_page_count(r, T, S, len(forced))
+        assert n == len(pages)
+        _, kept, sc = O.quest_attention_one_group(q[None], K, np.zeros_like(K), S, n, forced)
+        assert np.array_equal(kept[0], pages) and np.array_equal(sc[0], scores)
+
+
+@pytest.mark.parametrize("S", [1, 4, 16])
+def test_quest_score_bounds_every_key_of_the_page(S):
+    rng = np.random.default_rng(S)
+    K = rng.normal(size=(131, 16))
+    for q in rng.normal(size=(5, 16)):
+        mp, mm = O.quest_page_extrema(K, S)
+        sc = O.quest_page_scores(q, mp, mm)
+        dots = K @ q
+        for pg in range(len(sc)):
+            top = dots[pg * S:(pg + 1) * S].max()
+            assert sc[pg] >= top - 1e-12
+            if S == 1:
+                assert abs(sc[pg] - top) < 1e-12  # a page of one key: the bound is the dot product
+        # the bound is the sum over dimensions of max(q_d min_d, q_d max_d): the largest any point of the box can give
+        lo = np.stack([K[pg * S:(pg + 1) * S].min(axis=0) for pg in range(len(sc))])
+        hi = np.stack([K[pg * S:(pg + 1) * S].max(axis=0) for pg in range(len(sc))])
+        assert np.allclose(sc, np.maximum(lo * q, hi * q).sum(axis=1), rtol=0, atol=1e-12)
+
+
+def test_quest_kept_page_count_closed_form():
+    for T in (1, 5, 16, 17, 100, 1000):
+        for S in (1, 4, 8, 16):
+            for r in (0, 1, 125, 333, 500, 999, 1000):
+                b = min(T, max(0, math.ceil(Fraction(r, 1000) * T)))
+                want = min(-(-T // S), max(-(-b // S), 1))
+                assert O.quest_kept_page_count(r, T, S, 1) == want
+    with pytest.raises(ValueError):
+        O.quest_kept_page_count(1001, 10, 4, 1)
+
+
+@pytest.mark.parametrize("S,r", [(1, 300), (4, 250), (8, 600), (16, 125)])
+def test_quest_attention_is_masked_dense_attention_per_head(S, r):
+    """Brute force: per head, rank the pages by the bound with a stable sort, expand to a token mask, and run
+    a dense softmax with an additive -inf bias in torch."""
+    rng = np.random.default_rng(100 + S)
+    T, hd, G = 77, 8, 3
+    K, V, qg = rng.normal(size=(T, hd)), rng.normal(size=(T, hd)), rng.normal(size=(G, hd))
+    P = -(-T // S)
+    last = (T - 1) // S
+    n = O.quest_kept_page_count(r, T, S, 1)
+    out, kept, sc = O.quest_attention_one_group(qg, K, V, S, n, np.array([last]))
+    for h in range(G):
+        lo = np.stack([K[pg * S:(pg + 1) * S].min(axis=0) for pg in range(P)])
+        hi = np.stack([K[pg * S:(pg + 1) * S].max(axis=0) for pg in range(P)])
+        bound = np.maximum(lo * qg[h], hi * qg[h]).sum(axis=1)
+        others = [pg for pg in sorted(range(P), key=lambda pg: (-bound[pg], pg)) if pg != last]
+        want = sorted([last] + others[: n - 1])
+        assert list(kept[h]) == want
+        bias = torch.full((T,), float("-inf"), dtype=torch.float64)
+        for pg in want:
+            bias[pg * S:(pg + 1) * S] = 0.0
+        w = torch.softmax(torch.from_numpy(K @ qg[h] / math.sqrt(hd)) + bias, dim=0)
+        assert np.allclose(out[h], (w[:, None] * torch.from_numpy(V)).sum(0).numpy(), rtol=0, atol=1e-12)
+
+
+def _small_paged_case(seed):
+    rng = np.random.default_rng(seed)
+    B, Hq, Hkv, hd, T = 3, 8, 2, 16, 53
+    shape = O.Shape(d_model=32, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=hd, d_ff=8, page_size=8)
+    n_pages = (T + 7) // 8
+    perm = rng.permutation(B * n_pages).astype(np.int32).reshape(B, n_pages)  # shuffled pages
+    k_pool = synth.to_bf16(rng.standard_normal((B * n_pages, Hkv, 8, hd)).astype(np.float32))
+    v_pool = synth.to_bf16(rng.standard_normal((B * n_pages, Hkv, 8, hd)).astype(np.float32))
+    kv = O.PagedKV(k_pool, v_pool, perm, np.array([T, T - 5, 9], np.int32))
+    return shape, kv, rng.standard_normal((B, Hq, hd)), B
+
+
+def test_quest_full_keep_rate_is_dense_and_pages_nest():
+    shape, kv, q, B = _small_paged_case(3)
+    dense, _, _ = O.sparse_decode_attn(shape, q, kv, [1000] * B)
+    for S in (4, 16):
+        out, kept, _ = O.quest_decode_attn(shape, q, kv, [1000] * B, S)
+        assert np.allclose(out, dense, rtol=0, atol=1e-12)
+        prev = None
+        for r in (0, 125, 250, 500, 1000):
+            _, kept, _ = O.quest_decode_attn(shape, q, kv, [r] * B, S)
+            for i in range(B):
+                last = (int(kv.seq_lens[i]) - 1) // S
+                assert all(last in set(pg) for pg in kept[i])
+                assert len(kept[i]) == shape.n_q_heads
+            if prev is not None:
+                assert all(set(a) <= set(b) for i in range(B) for a, b in zip(prev[i], kept[i]))
+            prev = kept
+
+
+def test_quest_heads_select_independently():
+    """Selection is per query head: changing one head's query changes only that head's pages and output."""
+    shape, kv, q, B = _small_paged_case(4)
+    out0, kept0, _ = O.quest_decode_attn(shape, q, kv, [250] * B, 8)
+    q2 = q.copy()
+    q2[:, 1] = -q2[:, 1]
+    out1, kept1, _ = O.quest_decode_attn(shape, q2, kv, [250] * B, 8)
+    for h in range(shape.n_q_heads):
+        same = all(np.array_equal(kept0[i][h], kept1[i][h]) for i in range(B))
+        if h != 1:
+            assert same and np.array_equal(out0[:, h], out1[:, h])
+    assert not np.array_equal(out0[:, 1], out1[:, 1])
+
+
 def test_attention_output_is_a_convex_combination():
     shape, q, kv = _tiny_case(11, 40, G=2, hd=8)
     out, kept, _ = O.sparse_decode_attn(shape, q, kv, [250])
