@@ -64,11 +64,23 @@ typedef struct sol_shape {
                                block with the smallest |x|: ceil((1 - p) d_model) survive (ties: lower index), the
                                rest of the normalised row is zeroed before the quantizer; the attention input is
                                not pruned and every intermediate channel is kept */
+  int32_t token_select;     /* how r_permille[i] picks the keys a step attends to: SOL_SELECT_TOKENS (0, the task's
+                               default) the ceil(r T) tokens with the largest q.k summed over the query group, per
+                               (sequence, kv head); SOL_SELECT_QUEST_PAGES (1, the paper's: appendix "Token sparsity
+                               via Quest") pages of quest_page_size contiguous tokens, scored per QUERY head by the
+                               bound q_pos.m+ + q_neg.m- from the per-dimension extrema of each page's keys; every
+                               head keeps its ceil(ceil(r T) / quest_page_size) best pages (ties: lower page; the
+                               pages that hold a forced token are always among them) and attends to all keys of
+                               its pages and to nothing else.  Needs sol_kv_t.quest_meta */
+  int32_t quest_page_size;  /* 4, 8, 16, 32 or 64, and at least n_q_heads / n_kv_heads, when token_select is
+                               SOL_SELECT_QUEST_PAGES (ignored otherwise) */
 } sol_shape_t;
 #define SOL_QUANT_PROJ_INPUTS 0
 #define SOL_QUANT_MLP_OUTPUT 1
 #define SOL_PRUNE_INTERMEDIATE 0
 #define SOL_PRUNE_MLP_INPUT 1
+#define SOL_SELECT_TOKENS 0
+#define SOL_SELECT_QUEST_PAGES 1
 
 /* Paged bf16 KV cache of one layer.  Pools: [num_pages][n_kv_heads][page_size][head_dim].
  * page_table: int32 [B][max_pages_per_seq], physical page of each logical page.
@@ -78,6 +90,11 @@ typedef struct sol_kv {
   const int32_t *page_table;
   const int32_t *seq_lens;
   int32_t max_pages_per_seq, num_pages;
+  void *quest_meta; /* SOL_SELECT_QUEST_PAGES only (else unused, may be NULL): device, bf16
+                       [num_pages][n_kv_heads][page_size / quest_page_size][2][head_dim]: for every block of
+                       quest_page_size tokens of a cache page the per-dimension maximum of its keys, then the negated
+                       minimum, over the tokens the sequence has (sol_quest_meta_bytes, sol_quest_build_meta).
+                       sol_decode_layer / sol_decode_step update the block of the token they append */
 } sol_kv_t;
 
 /* Weight matrices are PACKED once at load time (sol_pack_weights) into the order the tensor cores read
@@ -170,6 +187,15 @@ sol_status_t sol_quant_act(const void *x_bf16, int32_t B, int32_t d, const int32
 sol_status_t sol_quant_act_wide(const void *x_bf16, int32_t B, int32_t d, const int32_t *bits, int16_t *codes,
                                 float *scales, sol_stream_t stream);
 
+/* Page extrema for SOL_SELECT_QUEST_PAGES (the paper's appendix "Token sparsity via Quest": m+ = max_j k_j,
+ * m- = -min_j k_j over the keys of a page).  sol_quest_meta_bytes: size of sol_kv_t.quest_meta for a pool of
+ * num_pages pages (0: unsupported shape).  sol_quest_build_meta: fills quest_meta for every token the B
+ * sequences of `kv` hold (seq_lens counts them), e.g. after a prefill; blocks past a sequence's last token
+ * are left alone, the block that holds it takes its extrema over the tokens that exist.  Pointers: device;
+ * errors as for the other calls. */
+size_t sol_quest_meta_bytes(const sol_shape_t *shape, int32_t num_pages);
+sol_status_t sol_quest_build_meta(const sol_shape_t *shape, const sol_kv_t *kv, int32_t B, sol_stream_t stream);
+
 /* Decode attention with a per-sequence keep-rate (appendix "Token sparsity",
  * "Budgeted token selection": budget ceil(kappa*K_t) clamped to [0, K_t];
  * selection by exact token-level top-k instead of the paper's page bounds).
@@ -181,6 +207,11 @@ sol_status_t sol_quant_act_wide(const void *x_bf16, int32_t B, int32_t d, const 
  *   kept_idx (optional) int32 [B][n_kv][max_pages_per_seq*page_size], the
  *   kept token indices of each (sequence, kv-head) in ascending order;
  *   kept_cnt (optional) int32 [B][n_kv].
+ * With shape->token_select == SOL_SELECT_QUEST_PAGES the selection is the paper's (see sol_shape_t): per QUERY
+ * head; K and V rows are read only for pages that some head of the kv-head's group keeps; kv->quest_meta must
+ * be current.  kept_idx then holds int32 [B][n_q][max_pages_per_seq*page_size/quest_page_size]: the kept PAGE
+ * indices of each query head in ascending order (no larger than the token form, since quest_page_size is at
+ * least the number of query heads per kv head); kept_cnt is int32 [B][n_q].
  * The cache is only read. */
 sol_status_t sol_sparse_decode_attn(const sol_shape_t *shape, const void *q_bf16, const sol_kv_t *kv, int32_t B,
                                     const int32_t *r_permille, void *out_bf16, int32_t *kept_idx,
@@ -194,7 +225,7 @@ sol_status_t sol_sparse_decode_attn(const sol_shape_t *shape, const void *q_bf16
  * scratch is a fixed array of SOL_STATIC_SCRATCH_BYTES inside the library
  * image, present on every GPU that loads the library until the process exits.
  * The call allocates nothing.
- *   Inputs and outputs as sol_sparse_decode_attn; kept_idx / kept_cnt optional.
+ *   Inputs and outputs as sol_sparse_decode_attn (SOL_SELECT_TOKENS only); kept_idx / kept_cnt optional.
  *   status_out (optional, DEVICE int32[8]) receives the status words of this
  *   call (layout as sol_read_device_status) by a copy enqueued on `stream`.
  *   Limit: B * n_kv * (max_pages_per_seq * 64 * (4 G + 12) + 24 KiB) bytes plus small

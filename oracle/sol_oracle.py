@@ -538,7 +538,8 @@ PLACE_MLP_OUTPUT = 1   # the paper's: the MLP output is fake-quantized before th
 
 def decode_layer(shape: Shape, w: LayerWeights, kv: PagedKV, h_in: np.ndarray,
                  r_permille: Sequence[int], p_permille: Sequence[int], bits: Sequence[int],
-                 placement: int = PLACE_PROJ_INPUTS, mlp_prune: int = PRUNE_INTERMEDIATE):
+                 placement: int = PLACE_PROJ_INPUTS, mlp_prune: int = PRUNE_INTERMEDIATE,
+                 token_select: int = SELECT_TOKENS, quest_page_size: int = 16):
     """One decoder layer for one new token per sequence.
 
     mlp_prune == PRUNE_MLP_INPUT: p_permille[i] gates the input channels of the
@@ -579,7 +580,10 @@ def decode_layer(shape: Shape, w: LayerWeights, kv: PagedKV, h_in: np.ndarray,
     tr.q_rot = q_rot
 
     # attention over the kept tokens, output projection, residual
-    attn, tr.kept_tokens, sig = sparse_decode_attn(shape, q_rot, kv, r_permille)
+    if token_select == SELECT_QUEST_PAGES:  # the paper's page selection per query head; kept_tokens then holds pages
+        attn, tr.kept_tokens, sig = quest_decode_attn(shape, q_rot, kv, r_permille, quest_page_size)
+    else:
+        attn, tr.kept_tokens, sig = sparse_decode_attn(shape, q_rot, kv, r_permille)
     tr.attn_out = attn
     tr.extra["sigma"] = sig
     h_mid = h_in + attn.reshape(B, Hq * hd) @ bf16_to_f64(w.w_o).T

@@ -23,7 +23,7 @@ SOL_ERR_DEVICE_TIMEOUT = 5
 
 EXPORTS = [
     "sol_status_string", "sol_last_cuda_error", "sol_workspace_bytes", "sol_workspace_init", "sol_quant_act",
-    "sol_packed_weight_bytes", "sol_pack_weights", "sol_quant_act_wide",
+    "sol_packed_weight_bytes", "sol_pack_weights", "sol_quant_act_wide", "sol_quest_meta_bytes", "sol_quest_build_meta",
     "sol_sparse_decode_attn", "sol_sparse_decode_attn_static", "sol_pruned_swiglu_mlp", "sol_decode_layer", "sol_decode_step",
     "sol_decode_step_traced", "sol_decode_step_host", "sol_read_device_status", "sol_selftest_wait_timeout", "sol_timing_enable", "sol_timing_collect",
     "sol_launch_count",
@@ -34,12 +34,14 @@ class SolShape(C.Structure):
     _fields_ = [("d_model", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("page_size", C.c_int32),
                 ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("n_sink", C.c_int32), ("n_window", C.c_int32),
-                ("quant_placement", C.c_int32), ("mlp_prune", C.c_int32)]
+                ("quant_placement", C.c_int32), ("mlp_prune", C.c_int32), ("token_select", C.c_int32),
+                ("quest_page_size", C.c_int32)]
 
 
 class SolKV(C.Structure):
     _fields_ = [("k_pool", C.c_void_p), ("v_pool", C.c_void_p), ("page_table", C.c_void_p),
-                ("seq_lens", C.c_void_p), ("max_pages_per_seq", C.c_int32), ("num_pages", C.c_int32)]
+                ("seq_lens", C.c_void_p), ("max_pages_per_seq", C.c_int32), ("num_pages", C.c_int32),
+                ("quest_meta", C.c_void_p)]
 
 
 class SolLayerWeights(C.Structure):
@@ -96,6 +98,10 @@ def lib() -> C.CDLL:
         L.sol_pruned_swiglu_mlp.argtypes = [C.POINTER(SolShape), P, P, P, I, P, P, P, P, P, S, P]
         L.sol_packed_weight_bytes.restype = S
         L.sol_packed_weight_bytes.argtypes = [C.POINTER(SolShape), I]
+        L.sol_quest_meta_bytes.restype = S
+        L.sol_quest_meta_bytes.argtypes = [C.POINTER(SolShape), I]
+        L.sol_quest_build_meta.restype = I
+        L.sol_quest_build_meta.argtypes = [C.POINTER(SolShape), C.POINTER(SolKV), I, P]
         L.sol_pack_weights.restype = I
         L.sol_pack_weights.argtypes = [C.POINTER(SolShape), I, P, P, P, S, P]
         L.sol_decode_layer.restype = I
@@ -154,13 +160,29 @@ def last_cuda_error() -> str:
 
 
 def make_shape(d_model, n_q_heads, n_kv_heads, head_dim, d_ff, page_size=64, rms_eps=1e-5, rope_theta=0.0,
-               n_sink=0, n_window=1, quant_placement=0, mlp_prune=0) -> SolShape:
+               n_sink=0, n_window=1, quant_placement=0, mlp_prune=0, token_select=0, quest_page_size=0) -> SolShape:
     return SolShape(d_model, n_q_heads, n_kv_heads, head_dim, d_ff, page_size, rms_eps, rope_theta, n_sink, n_window,
-                    quant_placement, mlp_prune)
+                    quant_placement, mlp_prune, token_select, quest_page_size)
 
 
-def make_kv(k_pool, v_pool, page_table, seq_lens, max_pages_per_seq: int, num_pages: int) -> SolKV:
-    return SolKV(_ptr(k_pool), _ptr(v_pool), _ptr(page_table), _ptr(seq_lens), max_pages_per_seq, num_pages)
+def make_kv(k_pool, v_pool, page_table, seq_lens, max_pages_per_seq: int, num_pages: int, quest_meta=None) -> SolKV:
+    return SolKV(_ptr(k_pool), _ptr(v_pool), _ptr(page_table), _ptr(seq_lens), max_pages_per_seq, num_pages,
+                 _ptr(quest_meta))
+
+
+SELECT_TOKENS, SELECT_QUEST_PAGES = 0, 1
+
+
+def quest_meta_bytes(shape: SolShape, num_pages: int) -> int:
+    return int(lib().sol_quest_meta_bytes(C.byref(shape), num_pages))
+
+
+def quest_build_meta(shape: SolShape, kv: SolKV, B: int, stream=None, check=True) -> int:
+    """Page extrema of every token the B sequences hold, into kv.quest_meta."""
+    s = lib().sol_quest_build_meta(C.byref(shape), C.byref(kv), B, _stream(stream))
+    if check:
+        _check(s, "sol_quest_build_meta")
+    return s
 
 
 W_QKV, W_O, W_GATE_UP, W_DOWN = 0, 1, 2, 3

@@ -111,7 +111,17 @@ static bool shape_ok(const sol_shape_t* s) {
   if (s->n_sink < 0 || s->n_window < 0) return false;
   if (s->quant_placement != SOL_QUANT_PROJ_INPUTS && s->quant_placement != SOL_QUANT_MLP_OUTPUT) return false;
   if (s->mlp_prune != SOL_PRUNE_INTERMEDIATE && s->mlp_prune != SOL_PRUNE_MLP_INPUT) return false;
+  if (s->token_select != SOL_SELECT_TOKENS && s->token_select != SOL_SELECT_QUEST_PAGES) return false;
+  if (s->token_select == SOL_SELECT_QUEST_PAGES) {
+    const int S = s->quest_page_size;
+    if (S != 4 && S != 8 && S != 16 && S != 32 && S != 64) return false;
+    if (S < s->n_q_heads / s->n_kv_heads) return false;  // the callers' page lists fit the token lists' arrays
+  }
   return true;
+}
+// the page extrema are there when the shape asks for them
+static bool quest_ok(const sol_shape_t* s, const sol_kv_t* kv) {
+  return s->token_select != SOL_SELECT_QUEST_PAGES || kv->quest_meta != nullptr;
 }
 
 static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
@@ -199,7 +209,12 @@ static void run_attention(const sol_shape_t& s, const Layout& L, void* ws, const
   a.qkv_ksplit = qkv_ksplit;
   a.qkv_scale = qkv_scale;
   a.q_bf16 = q_bf16;
-  attn_scratch_bind(a, ws, L.attn, kept_idx, kept_cnt);
+  const bool quest = s.token_select == SOL_SELECT_QUEST_PAGES;
+  attn_scratch_bind(a, ws, L.attn, quest ? nullptr : kept_idx, quest ? nullptr : kept_cnt);
+  if (quest) {  // the callers' arrays take the kept pages of every query head
+    a.quest_pages_out = kept_idx;
+    a.quest_cnt_out = kept_cnt;
+  }
   a.out_f32 = out_f32;
   a.out_bf16 = out_bf16;
   a.out_hi = want_split ? at<void>(ws, L.attn_hi) : nullptr;  // packed, high and low parts
@@ -426,11 +441,31 @@ sol_status_t sol_quant_act_wide(const void* x_bf16, int32_t B, int32_t d, const 
   return finish();
 }
 
+size_t sol_quest_meta_bytes(const sol_shape_t* shape, int32_t num_pages) {
+  if (!shape_ok(shape) || shape->token_select != SOL_SELECT_QUEST_PAGES || num_pages <= 0) return 0;
+  return (size_t)num_pages * shape->n_kv_heads * (PAGE / shape->quest_page_size) * 2 * shape->head_dim * 2;
+}
+
+sol_status_t sol_quest_build_meta(const sol_shape_t* shape, const sol_kv_t* kv, int32_t B, sol_stream_t stream) {
+  if (!shape || !kv_ok(kv) || B < 0) return SOL_ERR_INVALID_ARG;
+  if (!shape_ok(shape) || shape->token_select != SOL_SELECT_QUEST_PAGES || kv->max_pages_per_seq > MAX_PAGES_PER_SEQ)
+    return SOL_ERR_UNSUPPORTED;
+  if (!kv->quest_meta) return SOL_ERR_INVALID_ARG;
+  if (B == 0) return SOL_OK;
+  // a bad page id is reported through the status words of a workspace; this call has none, so such pages are
+  // skipped here and found by the attention call
+  static int* sink = nullptr;
+  if (!sink && record_cuda_error(cudaMalloc(&sink, 64), "sol_quest_build_meta")) return finish();
+  launch_quest_meta(*shape, *kv, B, true, sink, (cudaStream_t)stream);
+  return finish();
+}
+
 sol_status_t sol_sparse_decode_attn(const sol_shape_t* shape, const void* q_bf16, const sol_kv_t* kv, int32_t B,
                                     const int32_t* r_permille, void* out_bf16, int32_t* kept_idx, int32_t* kept_cnt,
                                     void* ws, size_t ws_bytes, sol_stream_t stream) {
   if (!shape || !q_bf16 || !kv_ok(kv) || !r_permille || !out_bf16 || !ws || B < 0) return SOL_ERR_INVALID_ARG;
   if (!shape_ok(shape) || B > 128 || kv->max_pages_per_seq > MAX_PAGES_PER_SEQ) return SOL_ERR_UNSUPPORTED;
+  if (!quest_ok(shape, kv)) return SOL_ERR_INVALID_ARG;
   if (B == 0) return SOL_OK;
   const Layout L = make_layout(*shape, B, kv->max_pages_per_seq);
   if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
@@ -502,6 +537,7 @@ sol_status_t sol_decode_layer(const sol_shape_t* shape, const sol_layer_weights_
   sol_status_t s = check_actions_host_side(shape, B);
   if (s != SOL_OK) return s;
   if (kv->max_pages_per_seq > MAX_PAGES_PER_SEQ) return SOL_ERR_UNSUPPORTED;
+  if (!quest_ok(shape, kv)) return SOL_ERR_INVALID_ARG;
   if (B == 0) return SOL_OK;
   const Layout L = make_layout(*shape, B, kv->max_pages_per_seq);
   if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
@@ -536,7 +572,7 @@ static sol_status_t step_args_ok(const sol_shape_t* shape, int32_t n_layers, con
   if (!shape_ok(shape) || B > 128) return SOL_ERR_UNSUPPORTED;
   int mp = 0;
   for (int l = 0; l < n_layers; ++l) {
-    if (!weights_ok(&layers[l]) || !kv_ok(&kvs[l])) return SOL_ERR_INVALID_ARG;
+    if (!weights_ok(&layers[l]) || !kv_ok(&kvs[l]) || !quest_ok(shape, &kvs[l])) return SOL_ERR_INVALID_ARG;
     if (kvs[l].max_pages_per_seq > mp) mp = kvs[l].max_pages_per_seq;
   }
   if (mp > MAX_PAGES_PER_SEQ) return SOL_ERR_UNSUPPORTED;

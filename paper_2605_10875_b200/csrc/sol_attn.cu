@@ -28,8 +28,6 @@
 
 namespace sol {
 
-constexpr int PAGE = 64;
-
 // Flat work lists of the attention kernels (AttnArgs::plan): cumulative counts over the sequences of the
 // batch, PLAN_STRIDE words each: 64-token pages, 8192-token segments of rows that need a
 // selection (histogram), 2048-token segments (scan).  Entry b is the count before sequence b, entry B the total.
@@ -93,8 +91,6 @@ struct PrepDev {
 };
 
 constexpr int PREP_THREADS = 128;
-// words of AttnArgs::work_ctr
-enum : int { WC_ITEMS = 0, WC_NEXT = 1, WC_CPI = 2, WC_DONE = 4 };
 // words of AttnArgs::row_ctl, per (sequence, kv-head): histogram CTAs finished, largest |score|, keep edge,
 // drop edge, window (float bits), tickets drawn by the scan CTAs, candidates listed, scan CTAs finished
 enum : int { RC_DONE1 = 0, RC_MAX, RC_EDGE, RC_LO, RC_DELTA, RC_TICKET, RC_NCAND, RC_DONE2, RC_WORDS };
@@ -1538,54 +1534,61 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   pd.max_item_chunks = 1024 / attn_split_len(hd);
   SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(Hkv, a.B), dim3(PREP_THREADS), 0, st, pd);
 
-  ScoreDev sd;
-  sd.kv = a.kv; sd.Hkv = Hkv; sd.G = G; sd.HG = HG; sd.Tmax = Tmax;
-  sd.q_split = static_cast<const uint16_t*>(a.q_split);
-  sd.logits = a.logits; sd.sigma = a.sigma; sd.status = a.status; sd.B = a.B;
-  const int groups_per_row = (a.kv.max_pages_per_seq + SC_WARPS - 1) / SC_WARPS;
-  if (hd == 64) launch_score<64>(sd, HG, groups_per_row, st);
-  else launch_score<128>(sd, HG, groups_per_row, st);
+  if (sh.token_select == SOL_SELECT_QUEST_PAGES) {
+    // the paper's page selection per query head (sol_quest.cu) instead of pass 1 and the token selection; a
+    // layer step has just appended a key, so the extrema of its block are taken again first
+    if (a.qkv_f32 != nullptr) launch_quest_meta(sh, a.kv, a.B, false, a.status, st);
+    launch_quest_selection(a, st);
+  } else {
+    ScoreDev sd;
+    sd.kv = a.kv; sd.Hkv = Hkv; sd.G = G; sd.HG = HG; sd.Tmax = Tmax;
+    sd.q_split = static_cast<const uint16_t*>(a.q_split);
+    sd.logits = a.logits; sd.sigma = a.sigma; sd.status = a.status; sd.B = a.B;
+    const int groups_per_row = (a.kv.max_pages_per_seq + SC_WARPS - 1) / SC_WARPS;
+    if (hd == 64) launch_score<64>(sd, HG, groups_per_row, st);
+    else launch_score<128>(sd, HG, groups_per_row, st);
 
-  SelectDev se;
-  se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.S = a.splits;
-  se.split_len = attn_split_len(hd); se.q_rot = a.q_rot; se.B = a.B;
-  se.nseg_max = attn_select_segs(a.kv.max_pages_per_seq, PAGE);
-  se.sigma = a.sigma; se.row_hist = a.row_hist; se.row_ctl = a.row_ctl; se.seg_pub = a.seg_pub;
-  se.cand_idx = a.cand_idx; se.cand_val = a.cand_val; se.list_idx = a.list_idx; se.list_row = a.kept_row;
-  se.kept_cnt = a.kept_cnt; se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
-  se.plan = a.plan;
-  {
-    // persistent grids: never more CTAs than are resident at once, never more than there can be units
-    static int hist_per_sm[2] = {0, 0}, scan_per_sm = 0;
-    if (scan_per_sm == 0) {
-      int n = 0;
-      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_hist_kernel<false>, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
-      hist_per_sm[0] = n;
-      n = 0;
-      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_hist_kernel<true>, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
-      hist_per_sm[1] = n;
-      n = 0;
-      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_scan_kernel, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
-      scan_per_sm = n;
+    SelectDev se;
+    se.sh = sh; se.kv = a.kv; se.r_permille = a.r_permille; se.Tmax = Tmax; se.S = a.splits;
+    se.split_len = attn_split_len(hd); se.q_rot = a.q_rot; se.B = a.B;
+    se.nseg_max = attn_select_segs(a.kv.max_pages_per_seq, PAGE);
+    se.sigma = a.sigma; se.row_hist = a.row_hist; se.row_ctl = a.row_ctl; se.seg_pub = a.seg_pub;
+    se.cand_idx = a.cand_idx; se.cand_val = a.cand_val; se.list_idx = a.list_idx; se.list_row = a.kept_row;
+    se.kept_cnt = a.kept_cnt; se.work_items = a.work_items; se.work_ctr = a.work_ctr; se.status = a.status;
+    se.plan = a.plan;
+    {
+      // persistent grids: never more CTAs than are resident at once, never more than there can be units
+      static int hist_per_sm[2] = {0, 0}, scan_per_sm = 0;
+      if (scan_per_sm == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_hist_kernel<false>, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
+        hist_per_sm[0] = n;
+        n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_hist_kernel<true>, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
+        hist_per_sm[1] = n;
+        n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, token_scan_kernel, TS_THREADS, 0) != cudaSuccess || n < 1) n = 1;
+        scan_per_sm = n;
+      }
+      const bool local = Tmax <= TH_SEG;
+      const long long hist_units = (long long)a.B * Hkv * ((Tmax + TH_SEG - 1) / TH_SEG);
+      const long long scan_units = (long long)a.B * Hkv * se.nseg_max;
+      const long long hist_res = (long long)sm_count() * hist_per_sm[local ? 1 : 0], scan_res = (long long)sm_count() * scan_per_sm;
+      const dim3 hist_grid((unsigned)(hist_units < hist_res ? hist_units : hist_res));
+      if (local) SOL_LAUNCH("token_hist", token_hist_kernel<true>, hist_grid, dim3(TS_THREADS), 0, st, se);
+      else SOL_LAUNCH("token_hist", token_hist_kernel<false>, hist_grid, dim3(TS_THREADS), 0, st, se);
+      if (Tmax > TH_SEG) {  // shorter rows are taken through the whole selection by token_hist
+        SOL_LAUNCH("token_scan", token_scan_kernel, dim3((unsigned)(scan_units < scan_res ? scan_units : scan_res)),
+                   dim3(TS_THREADS), 0, st, se);
+        SOL_LAUNCH("token_settle", token_settle_kernel, dim3(Hkv, a.B), dim3(TS_THREADS), 0, st, se);
+      }
     }
-    const bool local = Tmax <= TH_SEG;
-    const long long hist_units = (long long)a.B * Hkv * ((Tmax + TH_SEG - 1) / TH_SEG);
-    const long long scan_units = (long long)a.B * Hkv * se.nseg_max;
-    const long long hist_res = (long long)sm_count() * hist_per_sm[local ? 1 : 0], scan_res = (long long)sm_count() * scan_per_sm;
-    const dim3 hist_grid((unsigned)(hist_units < hist_res ? hist_units : hist_res));
-    if (local) SOL_LAUNCH("token_hist", token_hist_kernel<true>, hist_grid, dim3(TS_THREADS), 0, st, se);
-    else SOL_LAUNCH("token_hist", token_hist_kernel<false>, hist_grid, dim3(TS_THREADS), 0, st, se);
-    if (Tmax > TH_SEG) {  // shorter rows are taken through the whole selection by token_hist
-      SOL_LAUNCH("token_scan", token_scan_kernel, dim3((unsigned)(scan_units < scan_res ? scan_units : scan_res)),
-                 dim3(TS_THREADS), 0, st, se);
-      SOL_LAUNCH("token_settle", token_settle_kernel, dim3(Hkv, a.B), dim3(TS_THREADS), 0, st, se);
+    if (a.kept_idx_out != nullptr) {
+      ListDev ld;
+      ld.sh = sh; ld.kv = a.kv; ld.r_permille = a.r_permille; ld.Tmax = Tmax; ld.sigma = a.sigma; ld.row_ctl = a.row_ctl;
+      ld.kept_idx = a.kept_idx_out;
+      SOL_LAUNCH("token_list", token_list_kernel, dim3(Hkv, a.B), dim3(TS_THREADS), 0, st, ld);
     }
-  }
-  if (a.kept_idx_out != nullptr) {
-    ListDev ld;
-    ld.sh = sh; ld.kv = a.kv; ld.r_permille = a.r_permille; ld.Tmax = Tmax; ld.sigma = a.sigma; ld.row_ctl = a.row_ctl;
-    ld.kept_idx = a.kept_idx_out;
-    SOL_LAUNCH("token_list", token_list_kernel, dim3(Hkv, a.B), dim3(TS_THREADS), 0, st, ld);
   }
 
   GatherDev gd;

@@ -203,6 +203,10 @@ inline int attn_select_segs(int max_pages, int page_size) {
   return s < 1 ? 1 : s;
 }
 constexpr int ATTN_ITEM_CHUNKS = 64;  // chunks of attn_split_len kept tokens per pass-2 work item at most
+constexpr int PAGE = 64;  // tokens of a cache page
+// words of AttnArgs::work_ctr
+enum : int { WC_ITEMS = 0, WC_NEXT = 1, WC_CPI = 2, WC_DONE = 4 };
+
 struct AttnArgs {
   sol_shape_t shape;
   sol_kv_t kv;
@@ -243,12 +247,21 @@ struct AttnArgs {
   void* out_hi;      // packed operand of the output projection: 2 out_rows rows (bf16 high parts, then low parts)
   void* out_lo;      // unused
   int out_rows;
+  // SOL_SELECT_QUEST_PAGES (launch_quest_selection)
+  unsigned char* page_mask;   // scratch [B][Hkv][Tmax / 4]: per Quest page, bit h = query head h of the group keeps it
+  int32_t* quest_pages_out;   // optional: the caller's [B][Hq][Tmax / S] kept pages of every query head, ascending
+  int32_t* quest_cnt_out;     // optional: [B][Hq]
   int* status;
 };
+// Quest page extrema of the cache (all pages of the B sequences, or only the block of each sequence's newest token).
+void launch_quest_meta(const sol_shape_t& sh, const sol_kv_t& kv, int B, bool all, int* status, cudaStream_t st);
+// Page scores and selection per query head, union token list + pass-2 work items per (sequence, kv-head), then the
+// logits of the listed tokens (minus infinity for the heads that did not pick the token's page).
+void launch_quest_selection(const AttnArgs& a, cudaStream_t st);
 
 // Offsets of the attention scratch inside a buffer, starting at `at` (a multiple of 256).
 struct AttnScratch {
-  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_pub, cand_idx, cand_val, kept_idx, kept_cnt, kept_row, part, plan, work_items, work_ctr, end;
+  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_pub, cand_idx, cand_val, kept_idx, kept_cnt, kept_row, part, plan, work_items, work_ctr, page_mask, end;
   int splits;
 };
 inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_pages, size_t at) {
@@ -277,6 +290,7 @@ inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_page
   L.plan = take(3 * 132 * 4);
   L.work_items = take(BK * L.splits * 8);
   L.work_ctr = take((4 + BK) * 4);
+  L.page_mask = take(s.token_select == SOL_SELECT_QUEST_PAGES ? BK * (Tmax / 4) : 0);
   L.end = at;
   return L;
 }
@@ -300,6 +314,9 @@ inline void attn_scratch_bind(AttnArgs& a, void* base, const AttnScratch& L, int
   a.plan = reinterpret_cast<int32_t*>(b + L.plan);
   a.work_items = reinterpret_cast<int32_t*>(b + L.work_items);
   a.work_ctr = reinterpret_cast<int32_t*>(b + L.work_ctr);
+  a.page_mask = b + L.page_mask;
+  a.quest_pages_out = nullptr;
+  a.quest_cnt_out = nullptr;
   a.splits = L.splits;
 }
 void launch_attention(const AttnArgs& a, cudaStream_t st);

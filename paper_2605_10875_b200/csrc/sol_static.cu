@@ -54,7 +54,7 @@ bool attention_shape_ok(const sol_shape_t* s) {
   if (s->page_size != 64) return false;
   if (s->n_kv_heads <= 0 || s->n_q_heads <= 0 || s->n_q_heads % s->n_kv_heads) return false;
   if (s->n_q_heads / s->n_kv_heads > 8) return false;
-  return s->n_sink >= 0 && s->n_window >= 0;
+  return s->n_sink >= 0 && s->n_window >= 0 && s->token_select == SOL_SELECT_TOKENS;
 }
 
 }  // namespace
@@ -100,6 +100,9 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
   a.out_hi = nullptr;
   a.out_lo = nullptr;
   a.out_rows = 0;
+  a.page_mask = nullptr;
+  a.quest_pages_out = nullptr;
+  a.quest_cnt_out = nullptr;
   a.status = reinterpret_cast<int*>(base);
   sol::launch_attention(a, st);
   if (status_out != nullptr)

@@ -29,11 +29,12 @@ def host_u16(t: torch.Tensor) -> np.ndarray:
     return t.detach().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-def make_shapes(cfg: dict, n_sink=0, n_window=1, quant_placement=0, mlp_prune=0):
+def make_shapes(cfg: dict, n_sink=0, n_window=1, quant_placement=0, mlp_prune=0, token_select=0, quest_page_size=0):
     kw = dict(d_model=cfg["d_model"], n_q_heads=cfg["n_q_heads"], n_kv_heads=cfg["n_kv_heads"],
               head_dim=cfg["head_dim"], d_ff=cfg["d_ff"], page_size=64, rms_eps=synth.RMS_EPS,
               rope_theta=cfg.get("rope_theta", 0.0), n_sink=n_sink, n_window=n_window)
-    return sol.make_shape(quant_placement=quant_placement, mlp_prune=mlp_prune, **kw), O.Shape(**kw)
+    return sol.make_shape(quant_placement=quant_placement, mlp_prune=mlp_prune, token_select=token_select,
+                          quest_page_size=quest_page_size, **kw), O.Shape(**kw)
 
 
 class Workspace:
@@ -56,9 +57,19 @@ class DeviceKV:
     seq_lens: torch.Tensor
     max_pages: int
     num_pages: int
+    quest_meta: Optional[torch.Tensor] = None
 
     def struct(self):
-        return sol.make_kv(self.k_pool, self.v_pool, self.page_table, self.seq_lens, self.max_pages, self.num_pages)
+        return sol.make_kv(self.k_pool, self.v_pool, self.page_table, self.seq_lens, self.max_pages, self.num_pages,
+                           self.quest_meta)
+
+    def build_quest_meta(self, shape, B: int):
+        """Allocates the page extrema for a shape in Quest mode and fills them from the cache."""
+        n = sol.quest_meta_bytes(shape, self.num_pages)
+        assert n > 0
+        self.quest_meta = torch.zeros(n // 2, dtype=torch.bfloat16, device=DEV)
+        sol.quest_build_meta(shape, self.struct(), B)
+        torch.cuda.synchronize()
 
     def to_oracle(self) -> O.PagedKV:
         return O.PagedKV(host_u16(self.k_pool), host_u16(self.v_pool), self.page_table.cpu().numpy(),
