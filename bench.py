@@ -170,7 +170,7 @@ class Replica:
     are drawn on the device by a seeded generator (the same shapes and distributions as the host-side
     generators of the parity tests; tens of GB would take minutes to draw on the host)."""
 
-    def __init__(self, cfg, device, seed=0):
+    def __init__(self, cfg, device, seed=0, quest_page_size=0):
         import torch
 
         from paper_2605_10875_b200 import binding as sol
@@ -185,7 +185,9 @@ class Replica:
         if self.serving:
             self.seq_lens = np.maximum(self.seq_lens - (self.cycle - 1), 1).astype(np.int32)
         self.shape = sol.make_shape(cfg["d_model"], cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"], cfg["d_ff"],
-                                    64, synth.RMS_EPS, cfg.get("rope_theta", 0.0), 0, 1)
+                                    64, synth.RMS_EPS, cfg.get("rope_theta", 0.0), 0, 1,
+                                    token_select=sol.SELECT_QUEST_PAGES if quest_page_size else sol.SELECT_TOKENS,
+                                    quest_page_size=quest_page_size)
         table, n_pages = synth.make_page_table(self.seq_lens, cfg.get("shuffle_pages", True), seed,
                                                spare_tokens=self.cycle - 1)
         self.max_pages, self.n_pages = table.shape[1], n_pages
@@ -209,7 +211,14 @@ class Replica:
                 kv_ = base_kv if c == 0 else [t.clone() for t in base_kv]
                 self._keep += ws_ + kv_
                 per_copy_w.append(sol.make_weights(*ws_))
-                per_copy_kv.append([sol.make_kv(kv_[0], kv_[1], self.table, self.lens_dev[j], self.max_pages, n_pages)
+                meta = None
+                if quest_page_size:  # page extrema of the paper's Quest selection, built once (a prefill's job) for the
+                    # longest contexts of the cycle; every step renews the block of the key it appends
+                    meta = torch.zeros(sol.quest_meta_bytes(self.shape, n_pages) // 2, dtype=torch.bfloat16, device=device)
+                    self._keep.append(meta)
+                    sol.quest_build_meta(self.shape, sol.make_kv(kv_[0], kv_[1], self.table, self.lens_dev[-1],
+                                                                 self.max_pages, n_pages, meta), self.B)
+                per_copy_kv.append([sol.make_kv(kv_[0], kv_[1], self.table, self.lens_dev[j], self.max_pages, n_pages, meta)
                                     for j in range(self.cycle)])
             self.weights.append(per_copy_w)
             self.kvs.append(per_copy_kv)
@@ -548,6 +557,25 @@ def run_ours(args):
             rp.free()
             del rp
 
+    # --- the same workload with the paper's own token sparsity (Quest pages per query head) ---
+    quest = None
+    if args.quest:
+        rq = Replica(cfg, device, seed=0, quest_page_size=args.quest)
+        rq.set_actions(r, p, b, redraws)
+        nq = min(args.steps, 100)
+        t_ms = max_over_ranks(timed_steps(rq, nq, args.warmup, barrier, rq.step)) / nq
+        sol.timing_enable(True)
+        timed_steps(rq, min(nq, 20), args.warmup, barrier, rq.step)
+        rows_q = sol.timing_collect()
+        sol.timing_enable(False)
+        quest = {"page_size": args.quest, "us_per_step": round(1e3 * t_ms, 2), "steps_per_s": round(world * 1e3 / t_ms, 2),
+                 "token_selection_us_per_step": round(1e3 * ms_per_step, 2),
+                 "kernels_us_per_launch": {name: round(1e3 * tot / n, 2) for name, n, tot in rows_q
+                                           if name.startswith(("quest", "attn_"))},
+                 "device_status": sol.read_device_status(rq.ws)}
+        rq.free()
+        del rq
+
     line = None
     if rank == 0:
         cpu = None if (world > 1 or args.no_cpu_baseline) else cpu_baseline(args.workload, budget_s=20.0)
@@ -565,6 +593,7 @@ def run_ours(args):
             "roofline": roofline, "kernels": per_kernel, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks.summary(), "device_status": status,
             "budget_sweep": sweep, "per_workload": per_workload, "small_batch_prune_sweep": small_batch,
+            "quest_selection": quest,
         }
         print(json.dumps(line, default=_plain), flush=True)
     ranks.close()
@@ -683,6 +712,8 @@ def main():
                     help="distinct copies of weights and KV cache cycled through the steps (1 for a small profiler capture)")
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (a scaled-down case for a profiler capture)")
     ap.add_argument("--layers", type=int, default=None, help="override the workload's layer count (same purpose)")
+    ap.add_argument("--quest", type=int, default=16, choices=[0, 4, 8, 16, 32, 64],
+                    help="also time the workload with the paper's Quest page selection at this page size (0: skip)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="skip the compact runs of the other workloads")

@@ -89,7 +89,7 @@ struct QuestSelDev {
   sol_shape_t sh;
   sol_kv_t kv;
   const int32_t* r_permille;
-  int Tmax, S, splits, split_len, Pstride, Prow;
+  int Tmax, S, splits, split_len, Pstride, Prow, heads_per_pass;
   const float* q_rot;       // [B][Hq][hd]
   unsigned char* page_mask; // [B][Hkv][Pstride]
   int32_t* list_idx;        // [B][Hkv][Tmax]
@@ -134,17 +134,95 @@ __device__ __forceinline__ int quest_block_scan(int v, int& total, int* buf) {
   return before + incl - v;
 }
 
+constexpr int QS_CAND_CAP = 2048;  // pages per head whose bound is taken again in float64
+
+// Monotone 32-bit key of a float; never the all-ones key (forced pages).
+__device__ __forceinline__ uint32_t quest_key32(float s) {
+  const uint32_t bits = __float_as_uint(s + 0.0f);
+  const uint32_t k = (bits & 0x80000000u) ? ~bits : bits | 0x80000000u;
+  return k == 0xffffffffu ? k - 1 : k;
+}
+__device__ __forceinline__ float quest_key32_value(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? k & 0x7fffffffu : ~k);
+}
+
+// The `need`-th largest of n keys in shared memory (0 < need <= n): byte-wise radix passes, most significant
+// first.  Leaves the key in *s_prefix and, in *s_remaining, how many keys EQUAL to it belong to the `need`
+// largest (keys above it all do).  The lanes of a warp with the same digit add to the histogram once: the
+// scores of a row share their upper bytes, so most keys of a pass fall into one or two bins.
+template <typename KeyT>
+__device__ __forceinline__ void quest_radix_threshold(const KeyT* keys, int n, int need, int* hist,
+                                                      unsigned long long* s_prefix, int* s_remaining) {
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    *s_prefix = 0ull;
+    *s_remaining = need;
+  }
+  for (int pass = (int)sizeof(KeyT) - 1; pass >= 0; --pass) {
+    hist[tid] = 0;  // QS_THREADS == 256 bins
+    __syncthreads();
+    const unsigned long long prefix = *s_prefix;
+    const int shift = 8 * pass;
+    const bool top = pass == (int)sizeof(KeyT) - 1;
+    for (int base = 0; base < n; base += QS_THREADS) {
+      const int i = base + tid;
+      const unsigned long long k = i < n ? (unsigned long long)keys[i] : 0ull;
+      const bool in = i < n && (top || (k >> (shift + 8)) == (prefix >> (shift + 8)));
+      const int dgt = in ? (int)((k >> shift) & 255ull) : 256 + (tid & 31);  // lanes without a key match nobody
+      const unsigned same = __match_any_sync(0xffffffffu, dgt);
+      if (in && (tid & 31) == __ffs(same) - 1) atomicAdd(&hist[dgt], __popc(same));
+    }
+    __syncthreads();
+    if (tid < 32) {
+      // the digit whose bin holds the rem-th key counted from the top: lane l owns bins 255 - 8 l .. 248 - 8 l
+      const int rem0 = *s_remaining;
+      int mine = 0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) mine += hist[255 - 8 * tid - q];
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int x = __shfl_up_sync(0xffffffffu, incl, o);
+        if (tid >= o) incl += x;
+      }
+      const int before = incl - mine;  // keys in the bins above this lane's
+      if (before < rem0 && rem0 <= incl) {
+        int rem = rem0 - before, dgt = 255 - 8 * tid;
+        for (int q = 0; q < 7; ++q, --dgt) {
+          if (hist[dgt] >= rem) break;
+          rem -= hist[dgt];
+        }
+        *s_prefix = prefix | ((unsigned long long)dgt << shift);
+        *s_remaining = rem;
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// Selection of one query head, in two precisions.  The bound of every page is first summed in float32 (two
+// fused multiply-adds per dimension: the score and the sum of the terms' magnitudes, which bounds the rounding
+// error of the score); the n_keep-th largest float32 score tau is found by radix select; with w the largest
+// error bound of the row, a page above tau + 2 w is certainly among the n_keep best exact scores and one below
+// tau - 2 w certainly is not (the k-th largest of a set of numbers moves by at most w when each number moves by
+// at most w).  Only the pages in between are scored again in float64 (the widening of the extrema to float64
+// is the slow instruction: all pages in float64 took 400 us for a row of 2048 pages) and the missing ones are
+// taken from them by a second radix select on the 64-bit keys, ties to the lower page.
 __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSelDev p) {
   extern __shared__ __align__(16) unsigned char qsm[];
   const int kvh = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
   const int Hkv = p.sh.n_kv_heads, Hq = p.sh.n_q_heads, G = Hq / Hkv, hd = p.sh.head_dim, S = p.S;
   const int bk = b * Hkv + kvh;
-  unsigned long long* keys = reinterpret_cast<unsigned long long*>(qsm);        // [Prow]
-  double* qpos = reinterpret_cast<double*>(qsm + (size_t)p.Prow * 8);            // [hd]
-  double* qneg = qpos + hd;                                                      // [hd]
-  unsigned char* mask = reinterpret_cast<unsigned char*>(qneg + hd);             // [Prow]
+  const int HP = p.heads_per_pass;  // query heads whose float32 keys are in shared memory at once
+  unsigned long long* cand_key = reinterpret_cast<unsigned long long*>(qsm);             // [QS_CAND_CAP]
+  float* qf = reinterpret_cast<float*>(cand_key + QS_CAND_CAP);                           // [HP][hd] the heads' queries (16-byte aligned)
+  uint32_t* keys_all = reinterpret_cast<uint32_t*>(qf + (size_t)HP * hd);                 // [HP][Prow]
+  int* cand_idx = reinterpret_cast<int*>(keys_all + (size_t)HP * p.Prow);                 // [QS_CAND_CAP]
+  unsigned char* cand_sel = reinterpret_cast<unsigned char*>(cand_idx + QS_CAND_CAP);     // [QS_CAND_CAP]
+  unsigned char* mask = cand_sel + QS_CAND_CAP;                                           // [Prow]
   __shared__ int hist[256];
   __shared__ int scan_buf[QS_THREADS / 32];
+  __shared__ float wmax[8][QS_THREADS / 32];
   __shared__ unsigned long long s_prefix;
   __shared__ int s_remaining, s_item0;
   pdl_trigger();
@@ -162,96 +240,232 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
   const int n_keep = min(P, max((budget + S - 1) / S, n_forced));
   const int32_t* table = p.kv.page_table + (size_t)b * p.kv.max_pages_per_seq;
   const uint16_t* meta = static_cast<const uint16_t*>(p.kv.quest_meta);
+  const float err_unit = (float)(hd + 2) * 5.9604644775390625e-08f * 1.0001f;  // (hd + 2) 2^-24, rounded up
+  auto page_meta = [&](int pg, bool& ok) {
+    const int tok = pg * S, page = table[tok / PAGE];
+    ok = page >= 0 && page < p.kv.num_pages;
+    return reinterpret_cast<const uint4*>(meta + quest_meta_offset(ok ? page : 0, kvh, (tok % PAGE) / S, Hkv, S, hd));
+  };
 
   for (int pg = tid; pg < P; pg += QS_THREADS) mask[pg] = 0;
 
-  for (int h = 0; h < G; ++h) {
-    const int head = kvh * G + h;
-    __syncthreads();  // keys, qpos, qneg of the previous head are not read any more
-    for (int d = tid; d < hd; d += QS_THREADS) {
-      const double q = (double)p.q_rot[((size_t)b * Hq + head) * hd + d];
-      qpos[d] = q >= 0.0 ? fabs(q) : 0.0;
-      qneg[d] = q >= 0.0 ? 0.0 : fabs(q);
-    }
+  for (int h0 = 0; h0 < G; h0 += HP) {
+    const int nh = min(HP, G - h0);
+    __syncthreads();  // keys and queries of the previous heads are not read any more
+    for (int i = tid; i < nh * hd; i += QS_THREADS) qf[i] = p.q_rot[((size_t)b * Hq + kvh * G + h0 + i / hd) * hd + i % hd];
     __syncthreads();
-    // ---- the bound of every page, as a key ----
+    // ---- float32 bounds of every page for these heads.  Per dimension only one of the two terms of
+    //      q_pos.m+ + q_neg.m- is there: |q| m+ for q >= 0, |q| m- otherwise.  A thread takes a page; the pieces
+    //      of its extrema are fetched 64 dimensions at a time, all loads before the first use (one load per loop
+    //      pass put a memory round trip between every eight dimensions: 120 us for a row of 2048 pages). ----
+    float emax[8];
+#pragma unroll
+    for (int hh = 0; hh < 8; ++hh) emax[hh] = 0.f;
     for (int pg = tid; pg < P; pg += QS_THREADS) {
       const bool forced = pg < lo_pages || pg >= hi_first;
-      unsigned long long key = ~0ull;
+      float sc[8], ab[8];
+#pragma unroll
+      for (int hh = 0; hh < 8; ++hh) sc[hh] = ab[hh] = 0.f;
+      bool ok = true;
       if (!forced) {
-        const int tok = pg * S, page = table[tok / PAGE];
-        double s = 0.0;
-        if (page >= 0 && page < p.kv.num_pages) {
-          const uint4* mp = reinterpret_cast<const uint4*>(meta + quest_meta_offset(page, kvh, (tok % PAGE) / S, Hkv, S, hd));
-          const int pieces = hd / 8;
-          for (int c = 0; c < pieces; ++c) {
-            const uint4 a = mp[c], m = mp[pieces + c];
-            const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, mw[4] = {m.x, m.y, m.z, m.w};
+        const uint4* mp = page_meta(pg, ok);
+        if (!ok) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+        const int pieces = hd / 8;
+        for (int c0 = 0; c0 < pieces && ok; c0 += 8) {
+          uint4 a[8], m[8];
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            a[c] = mp[c0 + c];
+            m[c] = mp[pieces + c0 + c];
+          }
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const uint32_t aw[4] = {a[c].x, a[c].y, a[c].z, a[c].w}, mw[4] = {m[c].x, m[c].y, m[c].z, m[c].w};
+            float up[8], dn[8];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const int d = c * 8 + 2 * e;
-              s += qpos[d] * (double)bf16_lo(aw[e]) + qneg[d] * (double)bf16_lo(mw[e]);
-              s += qpos[d + 1] * (double)bf16_hi(aw[e]) + qneg[d + 1] * (double)bf16_hi(mw[e]);
+              up[2 * e] = bf16_lo(aw[e]);
+              up[2 * e + 1] = bf16_hi(aw[e]);
+              dn[2 * e] = bf16_lo(mw[e]);
+              dn[2 * e + 1] = bf16_hi(mw[e]);
+            }
+#pragma unroll
+            for (int hh = 0; hh < 8; ++hh) {
+              if (hh < nh) {
+                const float4 qa = *reinterpret_cast<const float4*>(qf + hh * hd + (c0 + c) * 8);
+                const float4 qb = *reinterpret_cast<const float4*>(qf + hh * hd + (c0 + c) * 8 + 4);
+                const float q[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  const float qv = q[e], mv = qv >= 0.f ? up[e] : dn[e];
+                  sc[hh] = fmaf(fabsf(qv), mv, sc[hh]);
+                  ab[hh] = fmaf(fabsf(qv), fabsf(mv), ab[hh]);
+                }
+              }
             }
           }
+        }
+      }
+#pragma unroll
+      for (int hh = 0; hh < 8; ++hh) {
+        if (hh < nh) {
+          keys_all[(size_t)hh * p.Prow + pg] = forced ? 0xffffffffu : quest_key32(ok ? sc[hh] : -INFINITY);
+          if (!forced && ok) emax[hh] = fmaxf(emax[hh], ab[hh] * err_unit);
+        }
+      }
+    }
+#pragma unroll
+    for (int hh = 0; hh < 8; ++hh) {
+      float v = emax[hh];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+      if ((tid & 31) == 0) wmax[hh][tid >> 5] = v;
+    }
+
+    for (int hh = 0; hh < nh; ++hh) {
+      const int h = h0 + hh, head = kvh * G + h;
+      const uint32_t* keys = keys_all + (size_t)hh * p.Prow;
+      __syncthreads();
+      const bool all_pages = n_keep >= P;
+      uint32_t tau32 = 0u;
+      int rem32 = 0;
+      if (!all_pages && n_keep > 0) {
+        quest_radix_threshold<uint32_t>(keys, P, n_keep, hist, &s_prefix, &s_remaining);
+        tau32 = (uint32_t)s_prefix;
+        rem32 = s_remaining;
+      }
+      __syncthreads();  // s_prefix, s_remaining are rewritten below
+      float w = 0.f;
+#pragma unroll
+      for (int x = 0; x < QS_THREADS / 32; ++x) w = fmaxf(w, wmax[hh][x]);
+      const bool only_forced = tau32 == 0xffffffffu || n_keep == 0;  // the budget is met by the forced pages alone
+      const double tau = only_forced || all_pages ? 0.0 : (double)quest_key32_value(tau32);
+      const double hi = tau + 2.002 * (double)w, lo = tau - 2.002 * (double)w;
+      // ---- the pages between lo and hi, in page order ----
+      int n_cand = 0, c_in = 0;
+      bool overflow = false;
+      if (!all_pages && !only_forced) {
+        for (int base = 0; base < P; base += QS_THREADS) {
+          const int pg = base + tid;
+          const uint32_t k = pg < P ? keys[pg] : 0u;
+          const double v = (double)quest_key32_value(k);
+          const bool forced = pg < P && k == 0xffffffffu;
+          const bool in = pg < P && (forced || v > hi);
+          const bool cand = pg < P && !forced && !in && v >= lo;
+          int tot_c, tot_in;
+          const int pos = quest_block_scan(cand ? 1 : 0, tot_c, scan_buf);
+          (void)quest_block_scan(in ? 1 : 0, tot_in, scan_buf);
+          if (cand && n_cand + pos < QS_CAND_CAP) cand_idx[n_cand + pos] = pg;
+          n_cand += tot_c;
+          c_in += tot_in;
+        }
+        overflow = n_cand > QS_CAND_CAP;
+        if (overflow && tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
+        __syncthreads();  // the candidate list is read by other threads than those that wrote it
+      }
+      const bool refine = !all_pages && !only_forced && !overflow && n_cand > 0;
+      if (refine) {
+        // ---- exact bounds of the candidates: a group of hd/4 lanes per candidate, one piece of the extrema per
+        //      lane, float64 partial sums added up over the group ----
+        {
+          const int lane = tid & 31, warp = tid >> 5;
+          const int LPG = hd / 4, GPW = 32 / LPG, sub = lane % LPG, grp = lane / LPG;
+          const bool minus = sub >= hd / 8;
+          const int d0 = (minus ? sub - hd / 8 : sub) * 8;
+          const float* q = qf + hh * hd + d0;
+          const int stride = (QS_THREADS / 32) * GPW;
+          for (int c0 = 0; c0 < n_cand; c0 += stride) {  // block-uniform trip count
+            const int c = c0 + warp * GPW + grp;
+            bool ok = true;
+            uint4 piece = make_uint4(0u, 0u, 0u, 0u);
+            if (c < n_cand) {
+              const uint4* mp = page_meta(cand_idx[c], ok);
+              if (ok) piece = mp[sub];
+            }
+            const uint32_t w4[4] = {piece.x, piece.y, piece.z, piece.w};
+            double sd = 0.0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float q0 = q[2 * e], q1 = q[2 * e + 1];
+              if ((q0 < 0.f) == minus) sd = fma((double)fabsf(q0), (double)bf16_lo(w4[e]), sd);
+              if ((q1 < 0.f) == minus) sd = fma((double)fabsf(q1), (double)bf16_hi(w4[e]), sd);
+            }
+            for (int o = 1; o < LPG; o <<= 1) sd += __shfl_xor_sync(0xffffffffu, sd, o);
+            if (sub == 0 && c < n_cand) cand_key[c] = quest_key(ok ? sd : -INFINITY);
+          }
+        }
+        if (tid == 0) atomicAdd(p.status + ST_TOK_REFINED, n_cand);
+        __syncthreads();
+        const int need2 = min(max(n_keep - c_in, 0), n_cand);
+        if (n_cand <= QS_THREADS) {
+          // a short list: a candidate is kept when fewer than need2 others come before it (larger key, or the
+          // same key and a lower page)
+          const unsigned long long mine = tid < n_cand ? cand_key[tid] : 0ull;
+          int rank = 0;
+          for (int x = 0; x < n_cand; ++x) {
+            const unsigned long long k = cand_key[x];
+            rank += (k > mine || (k == mine && x < tid)) ? 1 : 0;
+          }
+          if (tid < n_cand) cand_sel[tid] = rank < need2 ? 1 : 0;
         } else {
-          atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
-          s = -INFINITY;
+          unsigned long long tau64 = ~0ull;  // need2 == 0: no candidate key reaches this
+          int rem64 = 0;
+          if (need2 > 0) {
+            quest_radix_threshold<unsigned long long>(cand_key, n_cand, need2, hist, &s_prefix, &s_remaining);
+            tau64 = s_prefix;
+            rem64 = s_remaining;
+          }
+          // the candidates that are kept, in page order
+          int seen = 0;
+          for (int base = 0; base < n_cand; base += QS_THREADS) {
+            const int c = base + tid;
+            const unsigned long long k = c < n_cand ? cand_key[c] : 0ull;
+            const bool eq = c < n_cand && k == tau64;
+            int tot;
+            const int rank = quest_block_scan(eq ? 1 : 0, tot, scan_buf);
+            if (c < n_cand) cand_sel[c] = (k > tau64 || (eq && seen + rank < rem64)) ? 1 : 0;
+            seen += tot;
+          }
         }
-        key = quest_key(s);
+        __syncthreads();
       }
-      keys[pg] = key;
-    }
-    // ---- the n_keep-th largest key: eight passes over the key's bytes, most significant first ----
-    if (tid == 0) {
-      s_prefix = 0ull;
-      s_remaining = n_keep;
-    }
-    for (int pass = 7; pass >= 0 && n_keep < P; --pass) {
-      hist[tid] = 0;  // QS_THREADS == 256 bins
-      __syncthreads();
-      const unsigned long long prefix = s_prefix;
-      const int shift = 8 * pass;
-      for (int pg = tid; pg < P; pg += QS_THREADS) {
-        const unsigned long long k = keys[pg];
-        if (pass == 7 || (k >> (shift + 8)) == (prefix >> (shift + 8))) atomicAdd(&hist[(int)((k >> shift) & 255ull)], 1);
-      }
-      __syncthreads();
-      if (tid == 0) {
-        int rem = s_remaining, dgt = 255;
-        for (; dgt > 0; --dgt) {
-          if (hist[dgt] >= rem) break;
-          rem -= hist[dgt];
+      // ---- mark the head's pages; write its ascending page list ----
+      int seen_equal = 0, seen_cand = 0, written = 0;
+      int32_t* out = p.pages_out ? p.pages_out + ((size_t)b * Hq + head) * p.Prow : nullptr;
+      for (int base = 0; base < P; base += QS_THREADS) {
+        const int pg = base + tid;
+        const uint32_t k = pg < P ? keys[pg] : 0u;
+        bool sel = false;
+        if (all_pages) {
+          sel = pg < P;
+        } else if (only_forced) {
+          sel = pg < P && k == 0xffffffffu;
+        } else if (overflow) {  // float32 order, ties to the lower page
+          const bool eq = pg < P && k == tau32;
+          int tot;
+          const int rank = quest_block_scan(eq ? 1 : 0, tot, scan_buf);
+          sel = pg < P && (k > tau32 || (eq && seen_equal + rank < rem32));
+          seen_equal += tot;
+        } else {
+          const double v = (double)quest_key32_value(k);
+          const bool forced = pg < P && k == 0xffffffffu;
+          const bool in = pg < P && (forced || v > hi);
+          const bool cand = pg < P && !forced && !in && v >= lo;
+          int tot;
+          const int pos = quest_block_scan(cand ? 1 : 0, tot, scan_buf);
+          sel = in || (cand && cand_sel[seen_cand + pos] != 0);
+          seen_cand += tot;
         }
-        s_prefix = prefix | ((unsigned long long)dgt << shift);
-        s_remaining = rem;
+        int tot_sel;
+        const int pos = quest_block_scan(sel ? 1 : 0, tot_sel, scan_buf);
+        if (sel) {
+          mask[pg] |= (unsigned char)(1u << h);
+          if (out) out[written + pos] = pg;
+        }
+        written += tot_sel;
       }
-      __syncthreads();
+      if (tid == 0 && p.cnt_out) p.cnt_out[(size_t)b * Hq + head] = written;
     }
-    __syncthreads();
-    const unsigned long long tau = s_prefix;  // keys above tau are kept, and the first s_remaining keys equal to it
-    const int n_equal = s_remaining;
-    const bool all_pages = n_keep >= P;
-    // ---- mark the head's pages; write its ascending page list ----
-    int seen_equal = 0, written = 0;
-    int32_t* out = p.pages_out ? p.pages_out + ((size_t)b * Hq + head) * p.Prow : nullptr;
-    for (int base = 0; base < P; base += QS_THREADS) {
-      const int pg = base + tid;
-      const unsigned long long k = pg < P ? keys[pg] : 0ull;
-      const bool eq = pg < P && !all_pages && k == tau;
-      int tot_eq;
-      const int rank_eq = quest_block_scan(eq ? 1 : 0, tot_eq, scan_buf);
-      const bool sel = pg < P && (all_pages || k > tau || (eq && seen_equal + rank_eq < n_equal));
-      seen_equal += tot_eq;
-      int tot_sel;
-      const int pos = quest_block_scan(sel ? 1 : 0, tot_sel, scan_buf);
-      if (sel) {
-        mask[pg] |= (unsigned char)(1u << h);
-        if (out) out[written + pos] = pg;
-      }
-      written += tot_sel;
-    }
-    if (tid == 0 && p.cnt_out) p.cnt_out[(size_t)b * Hq + head] = written;
   }
   __syncthreads();
 
@@ -270,6 +484,11 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
       const bool ok = page >= 0 && page < p.kv.num_pages;
       const uint32_t r0 = (uint32_t)((page * Hkv + kvh) * PAGE + (tok % PAGE));
       for (int j = 0; j < ntok; ++j) {
+        if (n_list + off + j >= p.Tmax) {  // cannot happen for a list of distinct tokens; checked, not trusted
+          atomicMax(p.status + 5, 1);
+          atomicMax(p.status + 6, n_list + off + j);
+          break;
+        }
         p.list_idx[row + n_list + off + j] = tok + j;
         p.list_row[row + n_list + off + j] = ok ? r0 + j : 0xffffffffu;
       }
@@ -305,6 +524,8 @@ struct QuestLogitDev {
   const int32_t* kept_cnt;
   const unsigned char* page_mask;
   float* logits;  // [B][Hkv][Tmax][G]
+  uint32_t n_rows;  // rows of the cache pool
+  int* status;
 };
 
 constexpr int QL_THREADS = 256;
@@ -318,7 +539,7 @@ __global__ void __launch_bounds__(QL_THREADS) quest_logits_kernel(const QuestLog
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, sub = lane % LPT;
   pdl_trigger();
   pdl_wait();
-  const int cnt = p.kept_cnt[bk];
+  const int cnt = min(p.kept_cnt[bk], p.Tmax);
   const int n0 = blockIdx.x * QL_CHUNK;
   if (n0 >= cnt) return;
   const int n1 = min(cnt, n0 + QL_CHUNK);
@@ -330,39 +551,73 @@ __global__ void __launch_bounds__(QL_THREADS) quest_logits_kernel(const QuestLog
   }
   const size_t row = (size_t)bk * p.Tmax;
   const uint16_t* kp = static_cast<const uint16_t*>(p.kv.k_pool);
-  for (int nb = n0 + warp * TPW; nb < n1; nb += (QL_THREADS / 32) * TPW) {
-    const int n = nb + lane / LPT;
-    const bool have = n < n1;
-    int j = 0;
-    uint32_t r = 0xffffffffu;
-    if (have) {
-      j = p.list_idx[row + n];
-      r = p.list_row[row + n];
-    }
-    float dot[GMAX];
+  // four tokens per lane group and pass; the list words of the next pass are fetched while the key pieces of
+  // this one are in flight, so a pass costs one memory round trip, not two
+  constexpr int UN = 4;
+  constexpr int STEP = (QL_THREADS / 32) * TPW * UN;
+  auto load_list = [&](int nb, int (&jj)[UN], uint32_t (&rr)[UN]) {
 #pragma unroll
-    for (int h = 0; h < GMAX; ++h) dot[h] = 0.f;
-    if (r != 0xffffffffu) {
-      const uint4 kv8 = *reinterpret_cast<const uint4*>(kp + (size_t)r * HD + sub * 8);
-      const uint32_t w[4] = {kv8.x, kv8.y, kv8.z, kv8.w};
+    for (int u = 0; u < UN; ++u) {
+      const int n = nb + u * TPW + lane / LPT;
+      jj[u] = -1;
+      rr[u] = 0xffffffffu;
+      if (n < n1) {
+        jj[u] = p.list_idx[row + n];
+        rr[u] = p.list_row[row + n];
+        if (jj[u] < 0 || jj[u] >= p.Tmax || (rr[u] != 0xffffffffu && rr[u] >= p.n_rows)) {  // checked, not trusted
+          atomicMax(p.status + 5, 2);
+          atomicMax(p.status + 6, jj[u]);
+          jj[u] = -1;
+          rr[u] = 0xffffffffu;
+        }
+      }
+    }
+  };
+  int j[UN], jn[UN];
+  uint32_t r[UN], rn[UN];
+  load_list(n0 + warp * TPW * UN, j, r);
+  for (int nb = n0 + warp * TPW * UN; nb < n1; nb += STEP) {
+    uint4 kv8[UN];
+#pragma unroll
+    for (int u = 0; u < UN; ++u) {
+      kv8[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (r[u] != 0xffffffffu) kv8[u] = *reinterpret_cast<const uint4*>(kp + (size_t)r[u] * HD + sub * 8);
+    }
+    load_list(nb + STEP, jn, rn);
+#pragma unroll
+    for (int u = 0; u < UN; ++u) {
+      float dot[GMAX];
+#pragma unroll
+      for (int h = 0; h < GMAX; ++h) dot[h] = 0.f;
+      const uint32_t w[4] = {kv8[u].x, kv8[u].y, kv8[u].z, kv8[u].w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const float k0 = bf16_lo(w[e]), k1 = bf16_hi(w[e]);
 #pragma unroll
         for (int h = 0; h < GMAX; ++h) dot[h] = fmaf(q[h][2 * e + 1], k1, fmaf(q[h][2 * e], k0, dot[h]));
       }
+#pragma unroll
+      for (int h = 0; h < GMAX; ++h) {
+#pragma unroll
+        for (int o = 1; o < LPT; o <<= 1) dot[h] += __shfl_xor_sync(0xffffffffu, dot[h], o);
+      }
+      if (j[u] >= 0 && sub == 0) {
+        const unsigned m = r[u] != 0xffffffffu ? p.page_mask[(size_t)bk * p.Pstride + j[u] / p.S] : 0u;
+        float* dst = p.logits + (row + j[u]) * p.G;
+        if (GMAX == 4 && p.G == 4) {
+          *reinterpret_cast<float4*>(dst) = make_float4((m & 1u) ? dot[0] : -INFINITY, (m & 2u) ? dot[1] : -INFINITY,
+                                                        (m & 4u) ? dot[2] : -INFINITY, (m & 8u) ? dot[3] : -INFINITY);
+        } else {
+#pragma unroll
+          for (int h = 0; h < GMAX; ++h)
+            if (h < p.G) dst[h] = ((m >> h) & 1u) ? dot[h] : -INFINITY;
+        }
+      }
     }
 #pragma unroll
-    for (int h = 0; h < GMAX; ++h) {
-#pragma unroll
-      for (int o = 1; o < LPT; o <<= 1) dot[h] += __shfl_xor_sync(0xffffffffu, dot[h], o);
-    }
-    if (have && sub == 0) {
-      const unsigned m = r != 0xffffffffu ? p.page_mask[(size_t)bk * p.Pstride + j / p.S] : 0u;
-      float* dst = p.logits + (row + j) * p.G;
-#pragma unroll
-      for (int h = 0; h < GMAX; ++h)
-        if (h < p.G) dst[h] = ((m >> h) & 1u) ? dot[h] : -INFINITY;
+    for (int u = 0; u < UN; ++u) {
+      j[u] = jn[u];
+      r[u] = rn[u];
     }
   }
 }
@@ -378,7 +633,11 @@ void launch_quest_selection(const AttnArgs& a, cudaStream_t st) {
   d.q_rot = a.q_rot; d.page_mask = a.page_mask; d.list_idx = a.list_idx; d.list_row = a.kept_row;
   d.kept_cnt = a.kept_cnt; d.pages_out = a.quest_pages_out; d.cnt_out = a.quest_cnt_out;
   d.work_items = a.work_items; d.work_ctr = a.work_ctr; d.status = a.status;
-  const int smem = d.Prow * 8 + 2 * hd * 8 + d.Prow + 16;
+  // as many heads' float32 keys at once as fit in ~96 KB
+  int hp = (96 * 1024) / (d.Prow * 4);
+  hp = hp < 1 ? 1 : (hp > G ? G : hp);
+  d.heads_per_pass = hp;
+  const int smem = QS_CAND_CAP * (8 + 4 + 1) + hp * d.Prow * 4 + hp * hd * 4 + d.Prow + 16;
   ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_select_kernel), smem);
   SOL_LAUNCH("quest_select", quest_select_kernel, dim3(Hkv, a.B), dim3(QS_THREADS), smem, st, d);
 
@@ -386,6 +645,7 @@ void launch_quest_selection(const AttnArgs& a, cudaStream_t st) {
   l.kv = a.kv; l.Hq = Hq; l.Hkv = Hkv; l.G = G; l.hd = hd; l.Tmax = Tmax; l.S = S; l.Pstride = d.Pstride;
   l.q_rot = a.q_rot; l.list_idx = a.list_idx; l.list_row = a.kept_row; l.kept_cnt = a.kept_cnt;
   l.page_mask = a.page_mask; l.logits = a.logits;
+  l.n_rows = (uint32_t)a.kv.num_pages * Hkv * PAGE; l.status = a.status;
   const dim3 grid((Tmax + QL_CHUNK - 1) / QL_CHUNK, Hkv, a.B);
   if (hd == 64) {
     if (G <= 4) SOL_LAUNCH("quest_logits", (quest_logits_kernel<64, 4>), grid, dim3(QL_THREADS), 0, st, l);
