@@ -243,3 +243,55 @@ def test_attention_batch_128_long_contexts_more_units_than_ctas():
     r, _, _ = synth.draw_actions(cfg, 0)
     extra = [int(np.flatnonzero(r == x)[0]) for x in cfg["r_set"]][:3] + [127]
     _attention_sets_case(cfg, lens, r, extra, "long contexts")
+
+
+def test_quest_attention_ragged_batch_128_pages():
+    """The paper's Quest selection (page size 16) on the ragged batch of 128 contexts: page counts of every query
+    head of every sequence by the budget formula, page sets and outputs of sampled sequences (the shortest and
+    the longest among them) against the oracle; rows of up to 2048 pages go through the two-precision select."""
+    cfg = synth.WORKLOADS["ragged_serving"]
+    S = 16
+    shape, oshape = H.make_shapes(cfg, token_select=sol.SELECT_QUEST_PAGES, quest_page_size=S)
+    B, Hq, Hkv, hd = cfg["batch"], cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"]
+    lens = synth.make_contexts(cfg, 0)
+    r, _, _ = synth.draw_actions(cfg, 0)
+    table, n_pages = synth.make_page_table(lens, True, 0)
+    tab = np.where(table < 0, 0, table).astype(np.int32)
+    k, v = synth.device_kv_pool(cfg, n_pages, H.DEV, 0, 0)
+    kv = H.DeviceKV(k, v, H.dev_i32(tab), H.dev_i32(lens), table.shape[1], n_pages)
+    kv.build_quest_meta(shape, B)
+    q = synth.make_queries(cfg, 0, B)
+    ws = H.Workspace(shape, B, kv.max_pages)
+    Prow = kv.max_pages * 64 // S
+    out = torch.zeros((B, Hq, hd), dtype=torch.bfloat16, device=H.DEV)
+    pages = torch.full((B, Hq, Prow), -1, dtype=torch.int32, device=H.DEV)
+    cnt = torch.full((B, Hq), -1, dtype=torch.int32, device=H.DEV)
+    sol.sparse_decode_attn(shape, H.dev_bf16(q), kv.struct(), B, H.dev_i32(r), out, pages, cnt, ws.buf, ws.bytes)
+    torch.cuda.synchronize()
+    st = ws.status()
+    assert st[0] == 0 and st[1] == 0 and st[5] == 0, st
+    cn = cnt.cpu().numpy()
+    for i in range(B):
+        assert np.all(cn[i] == O.quest_kept_page_count(int(r[i]), int(lens[i]), S, 1)), i
+    sample = sorted(set([int(np.argmin(lens)), int(np.argmax(lens))] + [int(np.flatnonzero(r == x)[0]) for x in cfg["r_set"]]
+                        + [50, 127]))[:8]
+    need = [(int(lens[i]) + 63) // 64 for i in sample]
+    pidx = torch.from_numpy(np.concatenate([tab[i, :n] for i, n in zip(sample, need)]).astype(np.int64)).to(H.DEV)
+    ctab = np.zeros((len(sample), kv.max_pages), np.int32)
+    at = 0
+    for row, n in enumerate(need):
+        ctab[row, :n] = np.arange(at, at + n)
+        at += n
+    okv = O.PagedKV(H.host_u16(k.index_select(0, pidx)), H.host_u16(v.index_select(0, pidx)), ctab, lens[sample])
+    out_o, kept_o, scores = O.quest_decode_attn(oshape, O.bf16_to_f64(q[sample]), okv, r[sample], S)
+    pg = pages.cpu().numpy()
+    from oracle import checker
+    tot = checker.SetParity()
+    for row, i in enumerate(sample):
+        forced = np.array([(int(lens[i]) - 1) // S])
+        for h in range(Hq):
+            tot.merge(checker.compare_index_set(scores[row][h], kept_o[row][h], pg[i, h, : cn[i, h]], forced))
+    H.assert_sets(tot, "quest page sets (ragged)")
+    got = synth.bf16_to_f32(H.host_u16(out)).astype(np.float64)[sample]
+    err = H.assert_outputs(out_o, got, "quest ragged attention output")
+    print("quest ragged attention: sampled", sample, "contexts", lens[sample].tolist(), tot, "status", st, "err", err)
