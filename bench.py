@@ -551,6 +551,13 @@ def run_ours(args):
                 rp.set_actions(*synth.uniform_actions(bsz, 1000, pp, 16))
                 row = sweep_point(rp, ranks, min(args.steps, 100), peak_gbs, {"batch": bsz, "r": 1.0, "p": pp / 1000, "b": 16})
                 row["union_rows"] = rp.union_rows(0)
+                # the down projection on its own (event-timed launches): its bytes are the union of kept rows
+                sol.timing_enable(True)
+                timed_steps(rp, 20, 5, barrier, rp.step)
+                trows = {name: 1e3 * tot / n for name, n, tot in sol.timing_collect()}
+                sol.timing_enable(False)
+                row["down_us_per_launch"] = round(trows.get("gemm_down_gathered", 0.0), 2)
+                row["down_mb"] = round(row["union_rows"] * c2["d_model"] * 2 / 1e6, 2)
                 rows_b.append(row)
             flag_non_monotone(rows_b, lambda x: True)
             small_batch += rows_b

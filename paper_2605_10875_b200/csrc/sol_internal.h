@@ -249,6 +249,8 @@ struct AttnArgs {
   int out_rows;
   // SOL_SELECT_QUEST_PAGES (launch_quest_selection)
   unsigned char* page_mask;   // scratch [B][Hkv][Tmax / 4]: per Quest page, bit h = query head h of the group keeps it
+  uint32_t* quest_keys;       // scratch [B][Hq][Tmax / S]: float32 bound of every page as a sortable key
+  uint32_t* quest_err;        // scratch [B][Hq]: largest rounding-error bound of the row's scores (float bits)
   int32_t* quest_pages_out;   // optional: the caller's [B][Hq][Tmax / S] kept pages of every query head, ascending
   int32_t* quest_cnt_out;     // optional: [B][Hq]
   int* status;
@@ -261,7 +263,7 @@ void launch_quest_selection(const AttnArgs& a, cudaStream_t st);
 
 // Offsets of the attention scratch inside a buffer, starting at `at` (a multiple of 256).
 struct AttnScratch {
-  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_pub, cand_idx, cand_val, kept_idx, kept_cnt, kept_row, part, plan, work_items, work_ctr, page_mask, end;
+  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_pub, cand_idx, cand_val, kept_idx, kept_cnt, kept_row, part, plan, work_items, work_ctr, page_mask, quest_keys, quest_err, end;
   int splits;
 };
 inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_pages, size_t at) {
@@ -290,7 +292,10 @@ inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_page
   L.plan = take(3 * 132 * 4);
   L.work_items = take(BK * L.splits * 8);
   L.work_ctr = take((4 + BK) * 4);
-  L.page_mask = take(s.token_select == SOL_SELECT_QUEST_PAGES ? BK * (Tmax / 4) : 0);
+  const bool quest = s.token_select == SOL_SELECT_QUEST_PAGES;
+  L.page_mask = take(quest ? BK * (Tmax / 4) : 0);
+  L.quest_keys = take(quest ? (size_t)B * Hq * (Tmax / s.quest_page_size) * 4 : 0);
+  L.quest_err = take(quest ? (size_t)B * Hq * 4 : 0);
   L.end = at;
   return L;
 }
@@ -315,6 +320,8 @@ inline void attn_scratch_bind(AttnArgs& a, void* base, const AttnScratch& L, int
   a.work_items = reinterpret_cast<int32_t*>(b + L.work_items);
   a.work_ctr = reinterpret_cast<int32_t*>(b + L.work_ctr);
   a.page_mask = b + L.page_mask;
+  a.quest_keys = reinterpret_cast<uint32_t*>(b + L.quest_keys);
+  a.quest_err = reinterpret_cast<uint32_t*>(b + L.quest_err);
   a.quest_pages_out = nullptr;
   a.quest_cnt_out = nullptr;
   a.splits = L.splits;

@@ -5,11 +5,13 @@
 //                 negated minimum (m-), as bf16 (extrema of bf16 numbers are bf16 numbers).  Either for every
 //                 page of the sequences (after a prefill) or only for the block of each sequence's newest token
 //                 (after a decode step's append).
-//   quest_select  one CTA per (sequence, kv-head): for each query head of the group the bound
-//                 q_pos.m+ + q_neg.m- of every page in float64 (a page costs 2/S of its keys' bytes), an exact
-//                 radix select of the head's ceil(b_t / S) best pages on the 64-bit keys (forced pages first,
-//                 ties to the lower page), then the union of the heads' pages as the row's token list, its
-//                 pass-2 work items, and a byte per page that says which heads keep it.
+//   quest_score   the bound q_pos.m+ + q_neg.m- of every page for every query head, in float32, as sortable keys,
+//                 with a bound of its rounding error (a page costs 2/S of its keys' bytes).
+//   quest_select  one CTA per (sequence, kv-head): for each query head of the group an exact selection of its
+//                 ceil(b_t / S) best pages: radix select on the float32 keys, float64 bounds for the few pages
+//                 within the error window of the threshold (forced pages first, ties to the lower page); then
+//                 the union of the heads' pages as the row's token list, its pass-2 work items, and a byte
+//                 per page that says which heads keep it.
 //   quest_logits  q.k of every listed token for the G heads (K rows are read only for pages in the union),
 //                 minus infinity for the heads that did not keep the token's page: pass 2 (attn_gather) then
 //                 weighs a token with zero for those heads, which is the paper's additive mask.
@@ -91,6 +93,8 @@ struct QuestSelDev {
   const int32_t* r_permille;
   int Tmax, S, splits, split_len, Pstride, Prow, heads_per_pass;
   const float* q_rot;       // [B][Hq][hd]
+  const uint32_t* keys;     // [B][Hq][Prow] float32 bounds as keys (quest_score)
+  const uint32_t* err;      // [B][Hq] largest error bound of the row, float bits
   unsigned char* page_mask; // [B][Hkv][Pstride]
   int32_t* list_idx;        // [B][Hkv][Tmax]
   uint32_t* list_row;
@@ -200,6 +204,106 @@ __device__ __forceinline__ void quest_radix_threshold(const KeyT* keys, int n, i
   }
 }
 
+// Float32 bounds of every block of every (sequence, kv-head) for the G heads of the group, as keys, and per head
+// the row's largest rounding-error bound.  Per dimension only one of the two terms of q_pos.m+ + q_neg.m- is
+// there: |q| m+ for q >= 0, |q| m- otherwise.  A thread takes a block; the pieces of its extrema are fetched 64
+// dimensions at a time, all loads before the first use (one load per loop pass put a memory round trip between
+// every eight dimensions); two fused multiply-adds per dimension: the score and the sum of the terms'
+// magnitudes, which bounds the rounding error of the score.  A grid over all blocks: inside the per-row
+// selection kernel this was the tail of the longest row (94 us for 2048 blocks).
+struct QuestScoreDev {
+  sol_shape_t sh;
+  sol_kv_t kv;
+  int S, Prow;
+  const float* q_rot;  // [B][Hq][hd]
+  uint32_t* keys;      // [B][Hq][Prow]
+  uint32_t* err;       // [B][Hq] float bits, zeroed before the launch
+  int* status;
+};
+
+__global__ void __launch_bounds__(QS_THREADS) quest_score_kernel(const QuestScoreDev p) {
+  __shared__ __align__(16) float qf[8 * 128];
+  __shared__ float wmax[8][QS_THREADS / 32];
+  const int kvh = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
+  const int Hkv = p.sh.n_kv_heads, Hq = p.sh.n_q_heads, G = Hq / Hkv, hd = p.sh.head_dim, S = p.S;
+  pdl_trigger();
+  const int T = min(max(p.kv.seq_lens[b], 0), p.kv.max_pages_per_seq * PAGE);
+  const int P = (T + S - 1) / S;
+  if ((int)blockIdx.x * QS_THREADS >= P) return;
+  pdl_wait();
+  const int n_sink = min(max(p.sh.n_sink, 0), T), n_win = min(max(p.sh.n_window, 0), T);
+  const int lo_pages = n_sink > 0 ? (n_sink - 1) / S + 1 : 0;
+  const int hi_first = n_win > 0 ? (T - n_win) / S : P;
+  for (int i = tid; i < G * hd; i += QS_THREADS) qf[i] = p.q_rot[((size_t)b * Hq + kvh * G + i / hd) * hd + i % hd];
+  __syncthreads();
+  const float err_unit = (float)(hd + 2) * 5.9604644775390625e-08f * 1.0001f;  // (hd + 2) 2^-24, rounded up
+  const int pg = blockIdx.x * QS_THREADS + tid;
+  float sc[8], ab[8];
+#pragma unroll
+  for (int hh = 0; hh < 8; ++hh) sc[hh] = ab[hh] = 0.f;
+  const bool forced = pg < lo_pages || pg >= hi_first;
+  bool ok = true;
+  if (pg < P && !forced) {
+    const int tok = pg * S, page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + tok / PAGE];
+    ok = page >= 0 && page < p.kv.num_pages;
+    if (!ok) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+    const uint4* mp = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.kv.quest_meta) +
+                                                     quest_meta_offset(ok ? page : 0, kvh, (tok % PAGE) / S, Hkv, S, hd));
+    const int pieces = hd / 8;
+    for (int c0 = 0; c0 < pieces && ok; c0 += 8) {
+      uint4 a[8], m[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        a[c] = mp[c0 + c];
+        m[c] = mp[pieces + c0 + c];
+      }
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint32_t aw[4] = {a[c].x, a[c].y, a[c].z, a[c].w}, mw[4] = {m[c].x, m[c].y, m[c].z, m[c].w};
+        float up[8], dn[8];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          up[2 * e] = bf16_lo(aw[e]);
+          up[2 * e + 1] = bf16_hi(aw[e]);
+          dn[2 * e] = bf16_lo(mw[e]);
+          dn[2 * e + 1] = bf16_hi(mw[e]);
+        }
+#pragma unroll
+        for (int hh = 0; hh < 8; ++hh) {
+          if (hh < G) {
+            const float4 qa = *reinterpret_cast<const float4*>(qf + hh * hd + (c0 + c) * 8);
+            const float4 qb = *reinterpret_cast<const float4*>(qf + hh * hd + (c0 + c) * 8 + 4);
+            const float q[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float qv = q[e], mv = qv >= 0.f ? up[e] : dn[e];
+              sc[hh] = fmaf(fabsf(qv), mv, sc[hh]);
+              ab[hh] = fmaf(fabsf(qv), fabsf(mv), ab[hh]);
+            }
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int hh = 0; hh < 8; ++hh) {
+    if (hh < G) {
+      if (pg < P) p.keys[((size_t)b * Hq + kvh * G + hh) * p.Prow + pg] = forced ? 0xffffffffu : quest_key32(ok ? sc[hh] : -INFINITY);
+      float v = (pg < P && !forced && ok) ? ab[hh] * err_unit : 0.f;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+      if ((tid & 31) == 0) wmax[hh][tid >> 5] = v;
+    }
+  }
+  __syncthreads();
+  if (tid < G) {
+    float v = 0.f;
+#pragma unroll
+    for (int x = 0; x < QS_THREADS / 32; ++x) v = fmaxf(v, wmax[tid][x]);
+    atomicMax(p.err + (size_t)b * Hq + kvh * G + tid, __float_as_uint(v));  // non-negative floats order like their bits
+  }
+}
+
 // Selection of one query head, in two precisions.  The bound of every page is first summed in float32 (two
 // fused multiply-adds per dimension: the score and the sum of the terms' magnitudes, which bounds the rounding
 // error of the score); the n_keep-th largest float32 score tau is found by radix select; with w the largest
@@ -222,7 +326,6 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
   unsigned char* mask = cand_sel + QS_CAND_CAP;                                           // [Prow]
   __shared__ int hist[256];
   __shared__ int scan_buf[QS_THREADS / 32];
-  __shared__ float wmax[8][QS_THREADS / 32];
   __shared__ unsigned long long s_prefix;
   __shared__ int s_remaining, s_item0;
   pdl_trigger();
@@ -240,7 +343,6 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
   const int n_keep = min(P, max((budget + S - 1) / S, n_forced));
   const int32_t* table = p.kv.page_table + (size_t)b * p.kv.max_pages_per_seq;
   const uint16_t* meta = static_cast<const uint16_t*>(p.kv.quest_meta);
-  const float err_unit = (float)(hd + 2) * 5.9604644775390625e-08f * 1.0001f;  // (hd + 2) 2^-24, rounded up
   auto page_meta = [&](int pg, bool& ok) {
     const int tok = pg * S, page = table[tok / PAGE];
     ok = page >= 0 && page < p.kv.num_pages;
@@ -254,72 +356,10 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
     __syncthreads();  // keys and queries of the previous heads are not read any more
     for (int i = tid; i < nh * hd; i += QS_THREADS) qf[i] = p.q_rot[((size_t)b * Hq + kvh * G + h0 + i / hd) * hd + i % hd];
     __syncthreads();
-    // ---- float32 bounds of every page for these heads.  Per dimension only one of the two terms of
-    //      q_pos.m+ + q_neg.m- is there: |q| m+ for q >= 0, |q| m- otherwise.  A thread takes a page; the pieces
-    //      of its extrema are fetched 64 dimensions at a time, all loads before the first use (one load per loop
-    //      pass put a memory round trip between every eight dimensions: 120 us for a row of 2048 pages). ----
-    float emax[8];
-#pragma unroll
-    for (int hh = 0; hh < 8; ++hh) emax[hh] = 0.f;
-    for (int pg = tid; pg < P; pg += QS_THREADS) {
-      const bool forced = pg < lo_pages || pg >= hi_first;
-      float sc[8], ab[8];
-#pragma unroll
-      for (int hh = 0; hh < 8; ++hh) sc[hh] = ab[hh] = 0.f;
-      bool ok = true;
-      if (!forced) {
-        const uint4* mp = page_meta(pg, ok);
-        if (!ok) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
-        const int pieces = hd / 8;
-        for (int c0 = 0; c0 < pieces && ok; c0 += 8) {
-          uint4 a[8], m[8];
-#pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            a[c] = mp[c0 + c];
-            m[c] = mp[pieces + c0 + c];
-          }
-#pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            const uint32_t aw[4] = {a[c].x, a[c].y, a[c].z, a[c].w}, mw[4] = {m[c].x, m[c].y, m[c].z, m[c].w};
-            float up[8], dn[8];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              up[2 * e] = bf16_lo(aw[e]);
-              up[2 * e + 1] = bf16_hi(aw[e]);
-              dn[2 * e] = bf16_lo(mw[e]);
-              dn[2 * e + 1] = bf16_hi(mw[e]);
-            }
-#pragma unroll
-            for (int hh = 0; hh < 8; ++hh) {
-              if (hh < nh) {
-                const float4 qa = *reinterpret_cast<const float4*>(qf + hh * hd + (c0 + c) * 8);
-                const float4 qb = *reinterpret_cast<const float4*>(qf + hh * hd + (c0 + c) * 8 + 4);
-                const float q[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  const float qv = q[e], mv = qv >= 0.f ? up[e] : dn[e];
-                  sc[hh] = fmaf(fabsf(qv), mv, sc[hh]);
-                  ab[hh] = fmaf(fabsf(qv), fabsf(mv), ab[hh]);
-                }
-              }
-            }
-          }
-        }
-      }
-#pragma unroll
-      for (int hh = 0; hh < 8; ++hh) {
-        if (hh < nh) {
-          keys_all[(size_t)hh * p.Prow + pg] = forced ? 0xffffffffu : quest_key32(ok ? sc[hh] : -INFINITY);
-          if (!forced && ok) emax[hh] = fmaxf(emax[hh], ab[hh] * err_unit);
-        }
-      }
-    }
-#pragma unroll
-    for (int hh = 0; hh < 8; ++hh) {
-      float v = emax[hh];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-      if ((tid & 31) == 0) wmax[hh][tid >> 5] = v;
+    // ---- the float32 keys of these heads' bounds (quest_score) ----
+    for (int hh = 0; hh < nh; ++hh) {
+      const uint32_t* src = p.keys + ((size_t)b * Hq + kvh * G + h0 + hh) * p.Prow;
+      for (int pg = tid; pg < P; pg += QS_THREADS) keys_all[(size_t)hh * p.Prow + pg] = src[pg];
     }
 
     for (int hh = 0; hh < nh; ++hh) {
@@ -335,9 +375,7 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
         rem32 = s_remaining;
       }
       __syncthreads();  // s_prefix, s_remaining are rewritten below
-      float w = 0.f;
-#pragma unroll
-      for (int x = 0; x < QS_THREADS / 32; ++x) w = fmaxf(w, wmax[hh][x]);
+      const float w = __uint_as_float(p.err[(size_t)b * Hq + head]);  // the row's largest error bound for this head
       const bool only_forced = tau32 == 0xffffffffu || n_keep == 0;  // the budget is met by the forced pages alone
       const double tau = only_forced || all_pages ? 0.0 : (double)quest_key32_value(tau32);
       const double hi = tau + 2.002 * (double)w, lo = tau - 2.002 * (double)w;
@@ -533,7 +571,10 @@ constexpr int QL_CHUNK = 1024;  // listed tokens per CTA
 
 template <int HD, int GMAX>
 __global__ void __launch_bounds__(QL_THREADS) quest_logits_kernel(const QuestLogitDev p) {
-  constexpr int LPT = HD / 8;     // lanes per token: 16 bytes of the key row each
+  // lanes per token: each takes PCS 16-byte pieces of the key row (two when the group has up to four heads: half
+  // as many exchanges per token as with one piece; one for larger groups, whose queries fill the registers)
+  constexpr int PCS = GMAX <= 4 ? 2 : 1;
+  constexpr int LPT = HD / (8 * PCS);
   constexpr int TPW = 32 / LPT;   // tokens per warp and pass
   const int kvh = blockIdx.y, b = blockIdx.z, bk = b * p.Hkv + kvh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, sub = lane % LPT;
@@ -543,11 +584,15 @@ __global__ void __launch_bounds__(QL_THREADS) quest_logits_kernel(const QuestLog
   const int n0 = blockIdx.x * QL_CHUNK;
   if (n0 >= cnt) return;
   const int n1 = min(cnt, n0 + QL_CHUNK);
-  float q[GMAX][8];
+  float q[GMAX][8 * PCS];  // this lane's dimensions: pieces sub, sub + LPT, ...
 #pragma unroll
   for (int h = 0; h < GMAX; ++h) {
 #pragma unroll
-    for (int e = 0; e < 8; ++e) q[h][e] = h < p.G ? p.q_rot[((size_t)b * p.Hq + kvh * p.G + h) * HD + sub * 8 + e] : 0.f;
+    for (int c = 0; c < PCS; ++c) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        q[h][c * 8 + e] = h < p.G ? p.q_rot[((size_t)b * p.Hq + kvh * p.G + h) * HD + (sub + c * LPT) * 8 + e] : 0.f;
+    }
   }
   const size_t row = (size_t)bk * p.Tmax;
   const uint16_t* kp = static_cast<const uint16_t*>(p.kv.k_pool);
@@ -577,11 +622,14 @@ __global__ void __launch_bounds__(QL_THREADS) quest_logits_kernel(const QuestLog
   uint32_t r[UN], rn[UN];
   load_list(n0 + warp * TPW * UN, j, r);
   for (int nb = n0 + warp * TPW * UN; nb < n1; nb += STEP) {
-    uint4 kv8[UN];
+    uint4 kv8[UN][PCS];
 #pragma unroll
     for (int u = 0; u < UN; ++u) {
-      kv8[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (r[u] != 0xffffffffu) kv8[u] = *reinterpret_cast<const uint4*>(kp + (size_t)r[u] * HD + sub * 8);
+#pragma unroll
+      for (int c = 0; c < PCS; ++c) {
+        kv8[u][c] = make_uint4(0u, 0u, 0u, 0u);
+        if (r[u] != 0xffffffffu) kv8[u][c] = *reinterpret_cast<const uint4*>(kp + (size_t)r[u] * HD + (sub + c * LPT) * 8);
+      }
     }
     load_list(nb + STEP, jn, rn);
 #pragma unroll
@@ -589,12 +637,15 @@ __global__ void __launch_bounds__(QL_THREADS) quest_logits_kernel(const QuestLog
       float dot[GMAX];
 #pragma unroll
       for (int h = 0; h < GMAX; ++h) dot[h] = 0.f;
-      const uint32_t w[4] = {kv8[u].x, kv8[u].y, kv8[u].z, kv8[u].w};
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float k0 = bf16_lo(w[e]), k1 = bf16_hi(w[e]);
+      for (int c = 0; c < PCS; ++c) {
+        const uint32_t w[4] = {kv8[u][c].x, kv8[u][c].y, kv8[u][c].z, kv8[u][c].w};
 #pragma unroll
-        for (int h = 0; h < GMAX; ++h) dot[h] = fmaf(q[h][2 * e + 1], k1, fmaf(q[h][2 * e], k0, dot[h]));
+        for (int e = 0; e < 4; ++e) {
+          const float k0 = bf16_lo(w[e]), k1 = bf16_hi(w[e]);
+#pragma unroll
+          for (int h = 0; h < GMAX; ++h) dot[h] = fmaf(q[h][c * 8 + 2 * e + 1], k1, fmaf(q[h][c * 8 + 2 * e], k0, dot[h]));
+        }
       }
 #pragma unroll
       for (int h = 0; h < GMAX; ++h) {
@@ -627,7 +678,14 @@ void launch_quest_selection(const AttnArgs& a, cudaStream_t st) {
   const int Hq = sh.n_q_heads, Hkv = sh.n_kv_heads, hd = sh.head_dim, G = Hq / Hkv, S = sh.quest_page_size;
   const int Tmax = a.kv.max_pages_per_seq * PAGE;
 
+  QuestScoreDev sc;
+  sc.sh = sh; sc.kv = a.kv; sc.S = S; sc.Prow = Tmax / S; sc.q_rot = a.q_rot; sc.keys = a.quest_keys; sc.err = a.quest_err;
+  sc.status = a.status;
+  record_cuda_error(cudaMemsetAsync(a.quest_err, 0, sizeof(uint32_t) * (size_t)a.B * Hq, st), "quest: clear the error bounds");
+  SOL_LAUNCH("quest_score", quest_score_kernel, dim3((sc.Prow + QS_THREADS - 1) / QS_THREADS, Hkv, a.B), dim3(QS_THREADS), 0, st, sc);
+
   QuestSelDev d;
+  d.keys = a.quest_keys; d.err = a.quest_err;
   d.sh = sh; d.kv = a.kv; d.r_permille = a.r_permille; d.Tmax = Tmax; d.S = S; d.splits = a.splits;
   d.split_len = attn_split_len(hd); d.Pstride = Tmax / 4; d.Prow = Tmax / S;
   d.q_rot = a.q_rot; d.page_mask = a.page_mask; d.list_idx = a.list_idx; d.list_row = a.kept_row;

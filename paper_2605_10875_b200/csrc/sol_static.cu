@@ -101,6 +101,8 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
   a.out_lo = nullptr;
   a.out_rows = 0;
   a.page_mask = nullptr;
+  a.quest_keys = nullptr;
+  a.quest_err = nullptr;
   a.quest_pages_out = nullptr;
   a.quest_cnt_out = nullptr;
   a.status = reinterpret_cast<int*>(base);

@@ -231,7 +231,7 @@ def test_mlp_llama1b_layer_full():
     print("llama1b mlp: sets", par, "status", st, "err", err)
 
 
-@pytest.mark.parametrize("B", [1, 17, 33, 64])
+@pytest.mark.parametrize("B", [1, 4, 8, 9, 17, 33, 64])
 def test_mlp_batch_sizes(B):
     cfg = dict(TINY, d_model=512, d_ff=2048 + 32)
     rng = np.random.default_rng(B)
