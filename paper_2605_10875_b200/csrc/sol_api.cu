@@ -224,11 +224,23 @@ static void run_attention(const sol_shape_t& s, const Layout& L, void* ws, const
   launch_attention(a, st);
 }
 
+// What a layer leaves to the first RMSNorm kernel of the next one when it skips its own reduction: the partial
+// sums of its down projection, the residual they are added to, and the live flags to clear.
+struct LayerCarry {
+  const float* resid;
+  const float* part;
+  int chunks;
+  size_t stride;
+  int32_t* live;
+  int n_live;
+};
+
 // a_op (packed) / scale in the workspace hold the MLP input operand.
 static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, const void* w_gate_up, const void* w_down,
                     const int32_t* p_permille, const void* resid, int resid_f32, void* out_bf16,
                     float* out_f32, float* out_f32_b, float* t_trace, int32_t* kept_ch, int32_t* kept_ch_cnt,
-                    cudaStream_t st, const int32_t* out_bits = nullptr, const sol_layer_trace_t* tr = nullptr) {
+                    cudaStream_t st, const int32_t* out_bits = nullptr, const sol_layer_trace_t* tr = nullptr,
+                    LayerCarry* carry_out = nullptr) {
   int* status = at<int>(ws, L.status);
   GemmNK gu;
   memset(&gu, 0, sizeof(gu));
@@ -293,6 +305,15 @@ static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, cons
     launch_quant_out(q, st);
     return;
   }
+  if (carry_out != nullptr) {  // the next layer's first RMSNorm kernel adds the partial sums to the residual
+    carry_out->resid = static_cast<const float*>(resid);
+    carry_out->part = dn.partial;
+    carry_out->chunks = dn.chunks;
+    carry_out->stride = (size_t)pad_rows(B) * s.d_model;
+    carry_out->live = cs.live;
+    carry_out->n_live = s.d_ff / 32;
+    return;
+  }
   launch_reduce_out(dn.partial, dn.chunks, B, pad_rows(B), s.d_model, resid, resid_f32, out_bf16, out_f32, out_f32_b,
                     cs.live, s.d_ff / 32, st);
 }
@@ -300,7 +321,7 @@ static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, cons
 static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol_layer_weights_t& w,
                       const sol_kv_t& kv, int B, const void* h_in, bool in_f32, void* h_out_bf16, float* h_out_f32,
                       const int32_t* r, const int32_t* p, const int32_t* bits, const sol_layer_trace_t* tr,
-                      cudaStream_t st) {
+                      cudaStream_t st, const LayerCarry* carry_in = nullptr, LayerCarry* carry_out = nullptr) {
   int* status = at<int>(ws, L.status);
   const int d = s.d_model, Hq = s.n_q_heads, Hkv = s.n_kv_heads, hd = s.head_dim;
   const int Nqkv = (Hq + 2 * Hkv) * hd;
@@ -310,7 +331,16 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
 
   NormQuantArgs n1;
   memset(&n1, 0, sizeof(n1));
-  n1.in = h_in; n1.in_f32 = in_f32; n1.gamma_bf16 = w.gamma1; n1.eps = s.rms_eps; n1.bits = in_bits; n1.B = B; n1.d = d;
+  if (carry_in != nullptr) {  // the previous layer left its down projection unreduced: h_in = its residual + the partials
+    n1.in = carry_in->resid; n1.in_f32 = true; n1.part = carry_in->part; n1.ksplit = carry_in->chunks;
+    n1.part_stride = carry_in->stride; n1.zero_flags = carry_in->live; n1.n_zero_flags = carry_in->n_live;
+    n1.sum_out = at<float>(ws, L.h_a);
+    h_in = n1.sum_out;
+    in_f32 = true;
+  } else {
+    n1.in = h_in; n1.in_f32 = in_f32;
+  }
+  n1.gamma_bf16 = w.gamma1; n1.eps = s.rms_eps; n1.bits = in_bits; n1.B = B; n1.d = d;
   n1.a_op = at<void>(ws, L.a_op); n1.a_op_rows = L.Mpad; n1.scale = scale; n1.xn = tr ? tr->xn1 : nullptr;
   n1.codes = tr ? tr->codes1 : nullptr;
   n1.status = status;
@@ -373,7 +403,7 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   run_mlp(s, L, ws, B, w.w_gate_up, w.w_down, gate_inputs ? at<int32_t>(ws, L.zero_p) : p, at<float>(ws, L.h_mid), 1,
           h_out_bf16, h_out_f32,
           tr ? tr->h_out : nullptr, tr ? tr->t : nullptr, tr ? tr->kept_ch : nullptr, tr ? tr->kept_ch_cnt : nullptr,
-          st, out_quant ? bits : nullptr, tr);
+          st, out_quant ? bits : nullptr, tr, carry_out);
 }
 
 static bool weights_ok(const sol_layer_weights_t* w) {
@@ -553,13 +583,21 @@ static sol_status_t decode_step_impl(const sol_shape_t* shape, int32_t n_layers,
                                      cudaStream_t st, const sol_layer_trace_t* traces = nullptr) {
   const void* h = h_in_bf16;
   bool in_f32 = false;
+  // Between two layers the reduction of the down projection (partials + residual) is left to the next layer's
+  // first RMSNorm kernel, which reads the row anyway: one launch less per layer.  Not with per-layer taps and not
+  // when the MLP output goes through the quantizer first.
+  const bool may_defer = traces == nullptr && shape->quant_placement != SOL_QUANT_MLP_OUTPUT;
+  LayerCarry carry[2];
+  bool have = false;
   for (int l = 0; l < n_layers; ++l) {
     sol_kv_t kv = kvs[l];
     if (seq_lens_override) kv.seq_lens = seq_lens_override;
     const bool last = l == n_layers - 1;
+    const bool defer = may_defer && !last;
     float* out32 = last ? h_out_f32 : at<float>(ws, (l & 1) ? L.h_b : L.h_a);
     run_layer(*shape, L, ws, layers[l], kv, B, h, in_f32, last ? h_out_bf16 : nullptr, out32, r, p, bits,
-              traces ? &traces[l] : nullptr, st);
+              traces ? &traces[l] : nullptr, st, have ? &carry[(l + 1) & 1] : nullptr, defer ? &carry[l & 1] : nullptr);
+    have = defer;
     h = out32;
     in_f32 = true;
   }

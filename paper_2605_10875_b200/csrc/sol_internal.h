@@ -55,6 +55,7 @@ struct NormQuantArgs {
   bool in_f32;
   const float* part;
   int ksplit;
+  size_t part_stride;  // floats between two partials; 0: B * d
   float* sum_out;
   const void* gamma_bf16;
   float eps;
@@ -71,6 +72,8 @@ struct NormQuantArgs {
   int* status;
   uint32_t* clear;   // optional: [B][clear_words] words zeroed, row by row, for the kernels that follow
   int clear_words;
+  int32_t* zero_flags;  // optional: n_zero_flags words zeroed by the grid as a whole (the down projection's live flags,
+  int n_zero_flags;     // when this kernel also stands in for the reduction of the previous layer's down projection)
 };
 void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st);
 

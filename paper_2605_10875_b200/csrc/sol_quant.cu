@@ -45,12 +45,15 @@ norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, i
                   const int32_t* __restrict__ bits, int d, uint16_t* __restrict__ a_op, int a_op_rows,
                   float* __restrict__ scale,
                   float* __restrict__ xn, int8_t* __restrict__ codes, int16_t* __restrict__ codes16, int* __restrict__ status,
-                  uint32_t* __restrict__ clear, int clear_words, const GateArgs gate) {
+                  uint32_t* __restrict__ clear, int clear_words, int32_t* __restrict__ zero_flags, int n_zero_flags,
+                  const GateArgs gate) {
   __shared__ float sh[NQ_THREADS / 32];
   __shared__ typename std::conditional<GATE, SelectSmem, NoSmem>::type gsm;
   pdl_trigger();
   pdl_wait();
   const int row = blockIdx.x;
+  if (zero_flags != nullptr)
+    for (int i = blockIdx.x * NQ_THREADS + threadIdx.x; i < n_zero_flags; i += gridDim.x * NQ_THREADS) zero_flags[i] = 0;
   if (clear != nullptr)  // this token's scratch of the kernels that follow
     for (int i = threadIdx.x; i < clear_words; i += NQ_THREADS) clear[(size_t)row * clear_words + i] = 0u;
   const int nvec = d / NQ_VEC;
@@ -266,7 +269,7 @@ norm_quant_kernel(const void* __restrict__ in, const float* __restrict__ part, i
 }
 
 void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st) {
-  const size_t stride = (size_t)a.B * a.d;
+  const size_t stride = a.part_stride ? a.part_stride : (size_t)a.B * a.d;
   GateArgs g;
   g.p_permille = a.gate_p_permille;
   g.xm = a.xm;
@@ -274,7 +277,7 @@ void launch_norm_quant(const NormQuantArgs& a, cudaStream_t st) {
   SOL_LAUNCH("norm_quant", (norm_quant_kernel<F32, GATE>), dim3(a.B), dim3(NQ_THREADS), 0, st, a.in, a.part, a.ksplit,  \
              stride, a.sum_out, static_cast<const uint16_t*>(a.gamma_bf16), a.eps, a.bits, a.d,                        \
              static_cast<uint16_t*>(a.a_op), a.a_op_rows, a.scale, a.xn, a.codes, a.codes16, a.status, a.clear,         \
-             a.clear_words, g)
+             a.clear_words, a.zero_flags, a.n_zero_flags, g)
   if (a.gate_p_permille != nullptr) {
     if (a.in_f32) SOL_NQ_LAUNCH(true, true);
     else SOL_NQ_LAUNCH(false, true);
