@@ -103,6 +103,24 @@ def test_quest_attention_head_dim_128():
     _quest_case(cfg, [700, 64, 1, 333], [250, 125, 500, 60], 16, seed=9)
 
 
+@pytest.mark.parametrize("hq,hkv,S", [(8, 1, 8), (4, 4, 4), (12, 2, 8), (8, 1, 64)])
+def test_quest_attention_other_group_sizes(hq, hkv, S):
+    cfg = dict(TINY, n_q_heads=hq, n_kv_heads=hkv, d_model=256 if (hq * 64) % 256 == 0 else 768)
+    _quest_case(cfg, [333, 64, 190, 700], [250, 500, 125, 60], S, seed=hq)
+
+
+def test_quest_long_row_many_pages_per_head_pass():
+    """A 20000-token row at page size 4: 5000 pages per head, more than one pass of heads through shared memory."""
+    _quest_case(TINY, [20000, 4097], [125, 500], 4, seed=21)
+
+
+def test_quest_page_size_below_group_is_refused():
+    cfg = dict(TINY, n_q_heads=8, n_kv_heads=1, d_model=256)
+    shape, _ = H.make_shapes(cfg, token_select=sol.SELECT_QUEST_PAGES, quest_page_size=4)
+    assert sol.workspace_bytes(shape, 4, 8) == 0
+    assert sol.quest_meta_bytes(shape, 16) == 0
+
+
 def test_quest_layer_updates_extrema_and_matches_oracle():
     """A whole layer step in Quest mode: the appended key enters its block's extrema before the pages are scored,
     and the layer output follows the oracle's layer with the same selection."""
