@@ -428,10 +428,10 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_down_kernel(const DownDev 
 // At batch <= 8 the union of the channels that some token keeps is well below d_ff when tokens are pruned, and a
 // 64-channel block is almost never dead as a whole: this kernel reads W_down channel by channel and skips
 // every channel that no token keeps, so the bytes follow the union of kept rows.  CTA = (128 output columns,
-// range of channels) as in umma_down; a warp takes every eighth channel of the range: it looks the channel
-// up in the tokens' keep masks, reads the channel's 256 bytes of the slab (two 128-byte pieces of the packed
-// layout, one per column half) and multiplies them into float32 accumulators (<= 8 tokens x 4 columns per
-// lane) on the FMA pipes; the warps are merged through shared memory.
+// range of channels) as in umma_down; a warp takes groups of 32 channels of the range, finds the kept ones with
+// one ballot, reads each kept channel's 256 bytes of the slab (two 128-byte pieces of the packed layout, one per
+// column half) and multiplies them into float32 accumulators (<= 8 tokens x 4 columns per lane) on the FMA
+// pipes; the warps are merged through shared memory.
 constexpr int DR_WARPS = 8;
 constexpr int DR_MAXB = 8;
 
@@ -456,43 +456,58 @@ __global__ void __launch_bounds__(DR_WARPS * 32) down_rows_kernel(const DownRows
   for (int m = 0; m < DR_MAXB; ++m)
 #pragma unroll
     for (int c = 0; c < 4; ++c) acc[m][c] = 0.f;
+  // A warp takes groups of 32 consecutive channels of the CTA's range.  Lane l first looks channel l of the group
+  // up in the tokens' keep masks and fetches the tokens' t for it (one round trip, all loads independent); the
+  // channels that some token keeps are then taken eight at a time: their weight pieces are requested together
+  // (256 bytes per channel, coalesced), the tokens' t come from the owning lane by a shuffle.  Looking one
+  // channel up after the other put three dependent round trips in front of every four channels (66 us for
+  // the whole matrix at batch 1).
 #pragma unroll 1
-  for (int jb = j0 + warp * 4; jb < j1; jb += DR_WARPS * 4) {  // four channels per step: their loads are in flight together
-    float tv[4][DR_MAXB];
-    uint32_t wv[4][2];
-    bool any[4];
+  for (int g0 = j0 + warp * 32; g0 < j1; g0 += DR_WARPS * 32) {
+    const int jl = g0 + lane;
+    float tl[DR_MAXB];
+    bool mine = false;
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int j = jb + u;
-      any[u] = false;
-#pragma unroll
-      for (int m = 0; m < DR_MAXB; ++m) {
-        tv[u][m] = 0.f;
-        if (j < j1 && m < p.M && p.keep[(size_t)m * p.ff + j]) {  // warp-uniform
-          tv[u][m] = p.t[(size_t)m * p.ff + j];
-          any[u] = true;
-        }
-      }
-      wv[u][0] = wv[u][1] = 0u;
-      if (any[u]) {
-        // channel j of the slab: block j / 64, row c = j % 64; lane l holds columns 2 l, 2 l + 1 of each 64-column half
-        const int c = j & 63;
-        const unsigned char* base = p.w + ((size_t)slab * jblocks + (j >> 6)) * UM_TILE_SPAN + c * 128 +
-                                    (((lane >> 2) ^ (c & 7)) * 16) + (lane & 3) * 4;
-        wv[u][0] = *reinterpret_cast<const uint32_t*>(base);
-        wv[u][1] = *reinterpret_cast<const uint32_t*>(base + 8192);
+    for (int m = 0; m < DR_MAXB; ++m) {
+      tl[m] = 0.f;
+      if (jl < j1 && m < p.M) {
+        const bool k = p.keep[(size_t)m * p.ff + jl] != 0;
+        const float v = p.t[(size_t)m * p.ff + jl];
+        tl[m] = k ? v : 0.f;
+        mine = mine || k;
       }
     }
+    unsigned todo = __ballot_sync(0xffffffffu, mine);
+    while (todo) {  // warp-uniform
+      int ch[8];
+      uint32_t wv[8][2];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      if (!any[u]) continue;
-      const float w0 = bf16_lo(wv[u][0]), w1 = bf16_hi(wv[u][0]), w2 = bf16_lo(wv[u][1]), w3 = bf16_hi(wv[u][1]);
+      for (int u = 0; u < 8; ++u) {
+        ch[u] = -1;
+        wv[u][0] = wv[u][1] = 0u;
+        if (todo) {
+          ch[u] = __ffs(todo) - 1;
+          todo &= todo - 1;
+          // channel j of the slab: block j / 64, row c = j % 64; lane l holds columns 2 l, 2 l + 1 of each 64-column half
+          const int j = g0 + ch[u], c = j & 63;
+          const unsigned char* base = p.w + ((size_t)slab * jblocks + (j >> 6)) * UM_TILE_SPAN + c * 128 +
+                                      (((lane >> 2) ^ (c & 7)) * 16) + (lane & 3) * 4;
+          wv[u][0] = *reinterpret_cast<const uint32_t*>(base);
+          wv[u][1] = *reinterpret_cast<const uint32_t*>(base + 8192);
+        }
+      }
 #pragma unroll
-      for (int m = 0; m < DR_MAXB; ++m) {
-        acc[m][0] = fmaf(tv[u][m], w0, acc[m][0]);
-        acc[m][1] = fmaf(tv[u][m], w1, acc[m][1]);
-        acc[m][2] = fmaf(tv[u][m], w2, acc[m][2]);
-        acc[m][3] = fmaf(tv[u][m], w3, acc[m][3]);
+      for (int u = 0; u < 8; ++u) {
+        if (ch[u] < 0) continue;  // warp-uniform
+        const float w0 = bf16_lo(wv[u][0]), w1 = bf16_hi(wv[u][0]), w2 = bf16_lo(wv[u][1]), w3 = bf16_hi(wv[u][1]);
+#pragma unroll
+        for (int m = 0; m < DR_MAXB; ++m) {
+          const float tv = __shfl_sync(0xffffffffu, tl[m], ch[u]);
+          acc[m][0] = fmaf(tv, w0, acc[m][0]);
+          acc[m][1] = fmaf(tv, w1, acc[m][1]);
+          acc[m][2] = fmaf(tv, w2, acc[m][2]);
+          acc[m][3] = fmaf(tv, w3, acc[m][3]);
+        }
       }
     }
   }
