@@ -250,20 +250,25 @@ __global__ void __launch_bounds__(THREADS) channel_select_kernel(const ChanDev p
 // channel_select_multi
 // ============================================================================
 constexpr int CM_THREADS = 256;
-constexpr int CM_SLICE = CM_THREADS * 4;  // channels per CTA
+constexpr int CM_MAX_GROUPS = 2;  // groups of four channels per thread at most (template parameter of the kernel)
 
 struct ChanMultiSmem {
   int scan[CM_THREADS / 32];
   int pick[2];
   int n_local;
   int flag;
-  int local_idx[CM_SLICE];
+  int local_idx[CM_THREADS * 4 * CM_MAX_GROUPS];
   __align__(16) uint16_t x[8192];  // the token's operand row (d_model <= 8192)
   double val[CH_CAND_CAP];
   int idx[CH_CAND_CAP];
 };
 
+// CM_GROUPS: groups of four channels per thread, so CM_THREADS * 4 * CM_GROUPS channels per CTA: the launch takes
+// two groups when one group per thread would need more CTAs than are resident at once (a second, partly filled
+// wave of these latency-bound CTAs cost 15 % at batch 128; four groups were slower again: 37 against 34 us).
+template <int CM_GROUPS>
 __global__ void __launch_bounds__(CM_THREADS, 3) channel_select_multi_kernel(const ChanDev p) {
+  constexpr int CM_SLICE = CM_THREADS * 4 * CM_GROUPS;
   __shared__ ChanMultiSmem sm;
   const int slice = blockIdx.x, b = blockIdx.y, S = gridDim.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -273,9 +278,27 @@ __global__ void __launch_bounds__(CM_THREADS, 3) channel_select_multi_kernel(con
   pdl_wait();
   uint32_t* sel = p.sel + (size_t)b * CH_SEL_WORDS;
   const int m = (int)(((long long)(1000 - p.p_permille[b]) * ff + 999) / 1000);
-  const int j0 = slice * CM_SLICE + tid * 4;
-  const bool in = j0 < ff;  // ff is a multiple of 4: a thread's group is present or absent as a whole
   if (tid == 0) sm.n_local = 0;
+  // What the later steps read is requested now, so that it arrives while the histogram is scanned: this CTA's
+  // channels of t (and of g, u when there is a selection to make) and the token's operand row for the exact
+  // re-scoring (into shared memory; a selection almost always leaves a few channels to re-score).
+  const bool selecting = m > 0 && m < ff;
+  float4 v[CM_GROUPS], gq[CM_GROUPS], uq[CM_GROUPS];
+#pragma unroll
+  for (int gi = 0; gi < CM_GROUPS; ++gi) {
+    const int j0 = slice * CM_SLICE + (gi * CM_THREADS + tid) * 4;
+    v[gi] = gq[gi] = uq[gi] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (j0 < ff) {  // ff is a multiple of 4: a thread's group is present or absent as a whole
+      v[gi] = *reinterpret_cast<const float4*>(p.t + (size_t)b * ff + j0);
+      if (selecting) {
+        gq[gi] = *reinterpret_cast<const float4*>(p.g + (size_t)b * ff + j0);
+        uq[gi] = *reinterpret_cast<const float4*>(p.u + (size_t)b * ff + j0);
+      }
+    }
+  }
+  if (selecting)
+    for (int e = tid * 8; e < d; e += CM_THREADS * 8)
+      *reinterpret_cast<uint4*>(sm.x + e) = *reinterpret_cast<const uint4*>(p.a_op + act_piece_offset(p.Mpad, b, e >> 3));
 
   // ---- the histogram bin of the m-th largest |t| (every CTA of the token finds the same one) ----
   // keep at or above hi_edge + e_j, drop below lo_edge - e_j, exact in between; e_j = eps * (1.1 |u_j| + |g_j|)
@@ -329,42 +352,40 @@ __global__ void __launch_bounds__(CM_THREADS, 3) channel_select_multi_kernel(con
     hi_edge = bin_hi + delta;
   }
 
-  // ---- classify this CTA's channels ----
-  float4 v = make_float4(0.f, 0.f, 0.f, 0.f), gq = v, uq = v;
-  if (in) {
-    v = *reinterpret_cast<const float4*>(p.t + (size_t)b * ff + j0);
-    if (eps > 0.f) {
-      gq = *reinterpret_cast<const float4*>(p.g + (size_t)b * ff + j0);
-      uq = *reinterpret_cast<const float4*>(p.u + (size_t)b * ff + j0);
-    }
-  }
-  const float vv[4] = {v.x, v.y, v.z, v.w}, gg[4] = {gq.x, gq.y, gq.z, gq.w}, uu[4] = {uq.x, uq.y, uq.z, uq.w};
-  uint32_t hw[2] = {0, 0}, lw[2] = {0, 0}, kw = 0;
+  // ---- classify this CTA's channels: CM_GROUPS groups of four per thread ----
   int n_above = 0;
-  bool any = false;
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const float a = fabsf(vv[e]);
-    if (!in) continue;
-    const float ej = eps * (1.1f * fabsf(uu[e]) + fabsf(gg[e]));
-    if (a >= hi_edge + ej) {
-      const uint16_t hv = f2bf(vv[e]);
-      const uint16_t lv = f2bf(vv[e] - bf2f(hv));
-      hw[e >> 1] |= (uint32_t)hv << (16 * (e & 1));
-      lw[e >> 1] |= (uint32_t)lv << (16 * (e & 1));
-      kw |= 1u << (8 * e);
-      ++n_above;
-      any = true;
-    } else if (a >= lo_edge - ej) {
-      sm.local_idx[atomicAdd(&sm.n_local, 1)] = j0 + e;
+  for (int gi = 0; gi < CM_GROUPS; ++gi) {
+    const int j0 = slice * CM_SLICE + (gi * CM_THREADS + tid) * 4;
+    const bool in = j0 < ff;
+    const float vv[4] = {v[gi].x, v[gi].y, v[gi].z, v[gi].w}, gg[4] = {gq[gi].x, gq[gi].y, gq[gi].z, gq[gi].w},
+                uu[4] = {uq[gi].x, uq[gi].y, uq[gi].z, uq[gi].w};
+    uint32_t hw[2] = {0, 0}, lw[2] = {0, 0}, kw = 0;
+    bool any = false;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float a = fabsf(vv[e]);
+      if (!in) continue;
+      const float ej = eps * (1.1f * fabsf(uu[e]) + fabsf(gg[e]));
+      if (a >= hi_edge + ej) {
+        const uint16_t hv = f2bf(vv[e]);
+        const uint16_t lv = f2bf(vv[e] - bf2f(hv));
+        hw[e >> 1] |= (uint32_t)hv << (16 * (e & 1));
+        lw[e >> 1] |= (uint32_t)lv << (16 * (e & 1));
+        kw |= 1u << (8 * e);
+        ++n_above;
+        any = true;
+      } else if (a >= lo_edge - ej) {
+        sm.local_idx[atomicAdd(&sm.n_local, 1)] = j0 + e;
+      }
     }
-  }
-  if (in) {  // four channels: half a piece of the packed operand
-    unsigned char* dst = p.t_op + act_piece_offset(2 * p.Mpad, b, j0 >> 3) + (j0 & 7) * 2;
-    *reinterpret_cast<uint2*>(dst) = make_uint2(hw[0], hw[1]);
-    *reinterpret_cast<uint2*>(dst + (size_t)p.Mpad * 128) = make_uint2(lw[0], lw[1]);
-    *reinterpret_cast<uint32_t*>(p.keep + (size_t)b * ff + j0) = kw;
-    if (any) p.live[j0 >> 5] = 1;
+    if (in) {  // four channels: half a piece of the packed operand
+      unsigned char* dst = p.t_op + act_piece_offset(2 * p.Mpad, b, j0 >> 3) + (j0 & 7) * 2;
+      *reinterpret_cast<uint2*>(dst) = make_uint2(hw[0], hw[1]);
+      *reinterpret_cast<uint2*>(dst + (size_t)p.Mpad * 128) = make_uint2(lw[0], lw[1]);
+      *reinterpret_cast<uint32_t*>(p.keep + (size_t)b * ff + j0) = kw;
+      if (any) p.live[j0 >> 5] = 1;
+    }
   }
   n_above = __reduce_add_sync(0xffffffffu, n_above);
   if (lane == 0 && n_above) atomicAdd(sel + CH_N_ABOVE, (uint32_t)n_above);
@@ -376,10 +397,7 @@ __global__ void __launch_bounds__(CM_THREADS, 3) channel_select_multi_kernel(con
   const int n_local = sm.n_local;
   if (n_local > 0) {
     const double sc = (double)p.scale[b];
-    // the token's operand row, shared by all candidates of the CTA
-    for (int e = tid * 8; e < d; e += CM_THREADS * 8)
-      *reinterpret_cast<uint4*>(sm.x + e) = *reinterpret_cast<const uint4*>(p.a_op + act_piece_offset(p.Mpad, b, e >> 3));
-    __syncthreads();
+    // the token's operand row (requested at the start) is in shared memory: the barrier above has passed
     for (int c = warp; c < n_local; c += WARPS) {
       const int j = sm.local_idx[c];
       float gh = 0.f, gl = 0.f, uh = 0.f, ul = 0.f;
@@ -497,8 +515,11 @@ void launch_channel_select(const ChannelSelectArgs& a, cudaStream_t st) {
   c.kept_ch = a.kept_ch; c.scratch_idx = a.scratch_idx; c.kept_cnt = a.kept_cnt;
   c.t_op = static_cast<unsigned char*>(a.t_op);
   c.live = a.live; c.status = a.status;
-  const dim3 mgrid((a.ff + CM_SLICE - 1) / CM_SLICE, a.B);
-  SOL_LAUNCH("channel_select", channel_select_multi_kernel, mgrid, dim3(CM_THREADS), 0, st, c);
+  const long long resident = 3LL * sm_count();
+  const int groups = (long long)((a.ff + CM_THREADS * 4 - 1) / (CM_THREADS * 4)) * a.B > resident ? 2 : 1;
+  const dim3 mgrid((a.ff + CM_THREADS * 4 * groups - 1) / (CM_THREADS * 4 * groups), a.B);
+  if (groups == 1) SOL_LAUNCH("channel_select", channel_select_multi_kernel<1>, mgrid, dim3(CM_THREADS), 0, st, c);
+  else SOL_LAUNCH("channel_select", channel_select_multi_kernel<2>, mgrid, dim3(CM_THREADS), 0, st, c);
   const dim3 grid(a.B);
   // tokens the multi-CTA kernel handed over (it sets their flag); every other CTA leaves at once
   if (a.ff <= 2048) SOL_LAUNCH("channel_select_exact", (channel_select_kernel<256, 8>), grid, dim3(256), 0, st, c);
