@@ -12,7 +12,7 @@
 //   * one thread issues tcgen05.mma (bf16 x bf16 -> float32) with the WEIGHT
 //     tile as the 128-row M side and the batch as the N side, accumulating in
 //     tensor memory; tcgen05.commit releases each stage when its MMAs finish;
-//   * four warps read the accumulators back with tcgen05.ld and apply the
+//   * sixteen warps read the accumulators back with tcgen05.ld and apply the
 //     epilogue, writing out[m][n] with the weight row n along the lanes.
 //
 //   umma_nk   : Y[M][N] = A[M][K] . W[N][K]^T   (QKV, output and gate/up projections).  A CTA owns one tile
@@ -32,8 +32,10 @@
 
 namespace sol {
 
-constexpr int UM_THREADS = 320;      // warps 0-7: epilogue (two per 32 accumulator lanes), warp 8: producer, warp 9: MMA issuer + TMEM owner
-constexpr int UM_PRODUCER = 8, UM_MMA = 9;
+constexpr int UM_EPI_WARPS = 16;     // epilogue warps: four per 32 accumulator lanes (a warp reaches the lanes 32 (w % 4) ..)
+constexpr int UM_THREADS = (UM_EPI_WARPS + 2) * 32;  // then warp 16: producer, warp 17: MMA issuer + TMEM owner
+constexpr int UM_PRODUCER = UM_EPI_WARPS, UM_MMA = UM_EPI_WARPS + 1;
+constexpr int UM_EPI_SETS = UM_EPI_WARPS / 4;  // warps that share a quarter of the lanes take alternate groups of tokens
 constexpr int UM_MAX_STAGES = 8;
 constexpr int UM_TILE_SPAN = 16384;  // bytes one 128-row operand read spans from the start of a chunk tile
 constexpr int UM_SMEM_BUDGET = 204 * 1024;
@@ -184,9 +186,9 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
       // the scales come to shared memory while the weights stream: a global load per token inside the loop
       // below would put its latency between every two tokens
       if ((int)threadIdx.x < p.Mpad) bars->scale[threadIdx.x] = (p.row_scale && (int)threadIdx.x < p.M) ? p.row_scale[threadIdx.x] : 1.0f;
-      asm volatile("bar.sync 1, 256;" ::: "memory");  // the eight epilogue warps
+      asm volatile("bar.sync 1, %0;" ::"n"(UM_EPI_WARPS * 32) : "memory");  // the epilogue warps
     }
-    // warps w and w + 4 share the accumulator lanes 32 (w % 4) .. and take alternate groups of 16 tokens
+    // warps w, w + 4, w + 8, w + 12 share the accumulator lanes 32 (w % 4) .. and take alternate groups of tokens
     const int quarter = warp & 3, half = warp >> 2;
     if (quarter * 32 < p.R) {
       const bool ok = mbar_wait(&bars->accum, 0, p.status);
@@ -207,7 +209,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
         const bool even = (lane & 1) == 0;
         float* const dst = even ? p.out0 : p.out1;
 #pragma unroll 1
-        for (int c0 = half * 8; c0 < p.M && ok; c0 += 16) {
+        for (int c0 = half * 8; c0 < p.M && ok; c0 += 8 * UM_EPI_SETS) {
           uint32_t ra[8], rb[8];
           tmem_ld8_issue(tl + c0, ra);
           tmem_ld8_issue(tl + (p.n_b == 2 ? p.Mpad : 0) + c0, rb);  // high-part and low-part products
@@ -257,7 +259,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
       } else {
         const int n = tile * p.R + r;
         const bool valid = r < p.R && n < p.N;
-        for (int c0 = half * 16; c0 < p.Mpad && ok; c0 += 32) {
+        for (int c0 = half * 16; c0 < p.Mpad && ok; c0 += 16 * UM_EPI_SETS) {
           float v[16];
           tmem_ld16(tl + c0, v);
           if (p.n_b == 2) {  // high-part and low-part products
@@ -394,11 +396,11 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_down_kernel(const DownDev 
     const bool ok = mbar_wait(&bars->accum, 0, p.status);
     tc_fence_after();
     const bool any = *reinterpret_cast<volatile int*>(&bars->n_issued) > 0;
-    const int quarter = warp & 3, half = warp >> 2;  // as in umma_nk: two warps per 32 accumulator lanes
+    const int quarter = warp & 3, half = warp >> 2;  // as in umma_nk: four warps per 32 accumulator lanes
     const int n = slab * 128 + quarter * 32 + lane;
     const uint32_t tl = tmem + ((uint32_t)(quarter * 32) << 16);
     float* out = p.partial + (size_t)chunk * p.Mpad * p.d;
-    for (int c0 = half * 16; c0 < p.Mpad && ok; c0 += 32) {
+    for (int c0 = half * 16; c0 < p.Mpad && ok; c0 += 16 * UM_EPI_SETS) {
       float v[16];
       if (any) {
         float w2[16];
