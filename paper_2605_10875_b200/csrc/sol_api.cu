@@ -255,6 +255,7 @@ static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, cons
   gu.out1 = at<float>(ws, L.u);
   gu.out2 = t_trace ? t_trace : at<float>(ws, L.t);
   gu.sel = at<uint32_t>(ws, L.ch_sel);
+  gu.sel_p_permille = p_permille;
   gu.status = status;
   launch_gemm_nk(gu, EPI_SWIGLU, st);
 

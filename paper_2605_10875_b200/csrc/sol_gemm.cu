@@ -49,6 +49,7 @@ struct UmBarriers {
   int n_issued;
   uint32_t gmax[4][128], umax[4][128];  // SwiGLU epilogue: per token and accumulator quarter, the largest |g| and |u| (float bits)
   alignas(16) float scale[128];   // SwiGLU epilogue: the tokens' quantizer scales
+  unsigned char need_hist[128];   // SwiGLU epilogue: the token's channel selection is a real one (0 < kept < ff)
   unsigned char live[UM_LIVE_CAP];  // down projection: which of this CTA's 64-channel blocks hold a kept channel
 };
 
@@ -76,6 +77,7 @@ struct NKDev {
   float* out1;
   float* out2;
   uint32_t* sel;
+  const int32_t* sel_p;  // [M] prune rates or nullptr
   int* status;
 };
 
@@ -186,6 +188,14 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
       // the scales come to shared memory while the weights stream: a global load per token inside the loop
       // below would put its latency between every two tokens
       if ((int)threadIdx.x < p.Mpad) bars->scale[threadIdx.x] = (p.row_scale && (int)threadIdx.x < p.M) ? p.row_scale[threadIdx.x] : 1.0f;
+      if ((int)threadIdx.x < p.Mpad) {
+        bool need = (int)threadIdx.x < p.M;
+        if (need && p.sel_p != nullptr) {  // the kept count as the selection kernel computes it
+          const int m = (int)(((long long)(1000 - p.sel_p[threadIdx.x]) * p.N + 999) / 1000);
+          need = m > 0 && m < p.N;
+        }
+        bars->need_hist[threadIdx.x] = need ? 1 : 0;
+      }
       asm volatile("bar.sync 1, %0;" ::"n"(UM_EPI_WARPS * 32) : "memory");  // the epilogue warps
     }
     // warps w, w + 4, w + 8, w + 12 share the accumulator lanes 32 (w % 4) .. and take alternate groups of tokens
@@ -239,7 +249,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) umma_nk_kernel(const NKDev p) {
             // go to the warp's own words in shared memory (no atomics); the CTA merges them at the end.
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-              if (mine + 2 * j < p.M && valid)
+              if (mine + 2 * j < p.M && valid && bars->need_hist[mine + 2 * j])
                 atomicAdd(p.sel + (size_t)(mine + 2 * j) * CH_SEL_WORDS + chan_bin(fabsf(tv[j])), 1u);
             uint32_t gs = 0u, us = 0u;
 #pragma unroll
@@ -645,7 +655,7 @@ void launch_gemm_nk(const GemmNK& g, GemmEpilogue epi, cudaStream_t st) {
   d.w = static_cast<const unsigned char*>(g.w);
   d.x = static_cast<const unsigned char*>(g.a);
   d.row_scale = g.row_scale;
-  d.out0 = g.out0; d.out1 = g.out1; d.out2 = g.out2; d.sel = g.sel; d.status = g.status;
+  d.out0 = g.out0; d.out1 = g.out1; d.out2 = g.out2; d.sel = g.sel; d.sel_p = g.sel_p_permille; d.status = g.status;
   const int smem = 1024 + stages * stage_bytes + UM_TILE_SPAN + (int)sizeof(UmBarriers);
   const dim3 grid(geo.tiles, d.ksplit);
   if (epi == EPI_SWIGLU) {

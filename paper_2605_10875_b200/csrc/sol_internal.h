@@ -168,6 +168,7 @@ struct GemmNK {
   float* out1;            // EPI_SWIGLU: u
   float* out2;            // EPI_SWIGLU: t = silu(g) * u
   uint32_t* sel;          // EPI_SWIGLU: [M][CH_SEL_WORDS] histogram of |t| and max |g|, |u| per token (pre-cleared)
+  const int32_t* sel_p_permille;  // EPI_SWIGLU, optional: [M] prune rates; tokens that keep all or no channels need no histogram
   int* status;
 };
 void launch_gemm_nk(const GemmNK& p, GemmEpilogue epi, cudaStream_t st);
