@@ -673,6 +673,143 @@ __global__ void __launch_bounds__(QL_THREADS) quest_logits_kernel(const QuestLog
   }
 }
 
+// ---- the same logits on the tensor cores, for page sizes that are multiples of 16 ----
+// The row's list holds the tokens of its kept pages in ascending order, so with pages of 16, 32 or 64 tokens every
+// run of 16 list entries is 16 consecutive cache rows of one page (only the sequence's last page can be short, and
+// it comes last).  A warp takes such a run: one bulk copy of its key rows, the rows as the M side of m16n8k16 and
+// the query (split into three bf16 parts per head, exact to 2^-24, as in the scoring pass) as the N side.  Units
+// of four runs are numbered along the batch as in the scoring pass: a thread per sequence takes the largest
+// unit count of its kv-heads, the CTA adds them up, and CTAs walk the numbered units.
+struct QuestLogitMmaDev {
+  sol_kv_t kv;
+  int B, Hq, Hkv, G, Tmax, S, Pstride;
+  const uint16_t* q_split;  // bf16 [B][Hkv][HG * 16][hd]
+  const int32_t* list_idx;
+  const uint32_t* list_row;
+  const int32_t* kept_cnt;
+  const unsigned char* page_mask;
+  float* logits;
+  uint32_t n_rows;
+  int* status;
+};
+
+constexpr int QLM_WARPS = 4;
+
+template <int HD, int HG>
+__global__ void __launch_bounds__(QLM_WARPS * 32) quest_logits_mma_kernel(const QuestLogitMmaDev p) {
+  extern __shared__ __align__(128) unsigned char qlsm[];
+  constexpr int TILE_BYTES = 16 * HD * 2;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(qlsm + QLM_WARPS * TILE_BYTES);
+  __shared__ int s_cum[QLM_WARPS * 32 + 1], s_wsum[QLM_WARPS];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  pdl_trigger();
+  if (tid == 0) {
+    for (int i = 0; i < QLM_WARPS; ++i) mbar_init(&bars[i], 1);
+    fence_mbar_init();
+    s_cum[0] = 0;
+  }
+  pdl_wait();  // the lists and their lengths come from the selection kernel
+  int my_incl = 0;
+  if (tid < p.B) {
+    int mx = 0;
+    for (int h = 0; h < p.Hkv; ++h) mx = max(mx, min(p.kept_cnt[tid * p.Hkv + h], p.Tmax));
+    my_incl = (mx + 16 * QLM_WARPS - 1) / (16 * QLM_WARPS);  // units of the sequence's longest list
+  }
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, my_incl, o);
+    if (lane >= o) my_incl += x;
+  }
+  if (lane == 31) s_wsum[warp] = my_incl;
+  __syncthreads();
+  for (int w = 0; w < warp; ++w) my_incl += s_wsum[w];
+  s_cum[tid + 1] = my_incl;
+  __syncthreads();
+  const int n_units = s_cum[p.B] * p.Hkv;
+  const int g = lane >> 2, t = lane & 3;
+  constexpr int KS = HD / 32;
+  uint32_t phase = 0;
+  bool dead = false;
+#pragma unroll 1
+  for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const int key = u / p.Hkv;
+    const int b = __syncthreads_count(tid < p.B && my_incl <= key);
+    const int first = s_cum[b], n_groups = s_cum[b + 1] - first;
+    const int rem = u - first * p.Hkv;
+    const int kvh = rem / n_groups, grp = rem - kvh * n_groups;
+    const int bk = b * p.Hkv + kvh;
+    const int cnt = min(p.kept_cnt[bk], p.Tmax);
+    const int n0 = (grp * QLM_WARPS + warp) * 16;  // this warp's run of list entries
+    if (dead || n0 >= cnt) continue;
+    const int ntok = min(16, cnt - n0);
+    const size_t row = (size_t)bk * p.Tmax;
+    const int j0 = p.list_idx[row + n0];
+    const uint32_t r0 = p.list_row[row + n0];
+    if (j0 < 0 || j0 + ntok > p.Tmax || r0 == 0xffffffffu || r0 + (uint32_t)ntok > p.n_rows) {  // checked, not trusted
+      if (lane == 0 && r0 != 0xffffffffu) atomicMax(p.status + 5, 3);
+      continue;
+    }
+    unsigned char* tile = qlsm + warp * TILE_BYTES;
+    if (lane == 0) {
+      mbar_expect_tx(&bars[warp], ntok * HD * 2);
+      bulk_g2s(tile, static_cast<const uint16_t*>(p.kv.k_pool) + (size_t)r0 * HD, ntok * HD * 2, &bars[warp]);
+    }
+    uint4 qf[HG][KS][2];
+#pragma unroll
+    for (int hg = 0; hg < HG; ++hg) {
+      const uint16_t* qb = p.q_split + ((size_t)(bk * HG + hg) * 16) * HD;
+#pragma unroll
+      for (int sx = 0; sx < KS; ++sx) {
+        qf[hg][sx][0] = *reinterpret_cast<const uint4*>(qb + (size_t)g * HD + sx * 32 + t * 8);
+        qf[hg][sx][1] = *reinterpret_cast<const uint4*>(qb + (size_t)(8 + g) * HD + sx * 32 + t * 8);
+      }
+    }
+    const unsigned m = p.page_mask[(size_t)bk * p.Pstride + j0 / p.S];
+    if (!mbar_wait(&bars[warp], phase, p.status)) {
+      dead = true;
+      continue;
+    }
+    phase ^= 1;
+    const uint32_t tb = smem_u32(tile);
+    uint4 ka[KS][2];
+#pragma unroll
+    for (int sx = 0; sx < KS; ++sx) {
+      ka[sx][0] = lds128(tb + g * (HD * 2) + (sx * 32 + t * 8) * 2);
+      ka[sx][1] = lds128(tb + (g + 8) * (HD * 2) + (sx * 32 + t * 8) * 2);
+    }
+#pragma unroll
+    for (int hg = 0; hg < HG; ++hg) {
+      float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int sx = 0; sx < KS; ++sx) {
+        mma_bf16(d0, ka[sx][0].x, ka[sx][1].x, ka[sx][0].y, ka[sx][1].y, qf[hg][sx][0].x, qf[hg][sx][0].y);
+        mma_bf16(d0, ka[sx][0].z, ka[sx][1].z, ka[sx][0].w, ka[sx][1].w, qf[hg][sx][0].z, qf[hg][sx][0].w);
+        mma_bf16(d1, ka[sx][0].x, ka[sx][1].x, ka[sx][0].y, ka[sx][1].y, qf[hg][sx][1].x, qf[hg][sx][1].y);
+        mma_bf16(d1, ka[sx][0].z, ka[sx][1].z, ka[sx][0].w, ka[sx][1].w, qf[hg][sx][1].z, qf[hg][sx][1].w);
+      }
+      // columns 2t, 2t+1 of the first n-tile are head t's high and middle parts; column 2t of the second its low part
+      const float s0 = d0[0] + (d0[1] + d1[0]);  // token g of the run
+      const float s1 = d0[2] + (d0[3] + d1[2]);  // token g + 8
+      const int head = hg * 4 + t;
+      if (head < p.G) {
+        const bool on = (m >> head) & 1u;
+        if (g < ntok) p.logits[(row + j0 + g) * p.G + head] = on ? s0 : -INFINITY;
+        if (g + 8 < ntok) p.logits[(row + j0 + g + 8) * p.G + head] = on ? s1 : -INFINITY;
+      }
+    }
+    __syncwarp();  // the tile is rewritten by the next unit's copy
+  }
+}
+
+template <int HD, int HG>
+static void launch_quest_logits_mma(const QuestLogitMmaDev& d, cudaStream_t st) {
+  const int smem = QLM_WARPS * 16 * HD * 2 + QLM_WARPS * 8 + 32;
+  const long long upper = (long long)((d.Tmax + 16 * QLM_WARPS - 1) / (16 * QLM_WARPS)) * d.Hkv * d.B;
+  const dim3 grid((unsigned)(upper < 32768 ? upper : 32768));
+  ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_logits_mma_kernel<HD, HG>), smem);
+  SOL_LAUNCH("quest_logits", (quest_logits_mma_kernel<HD, HG>), grid, dim3(QLM_WARPS * 32), smem, st, d);
+}
+
 void launch_quest_selection(const AttnArgs& a, cudaStream_t st) {
   const sol_shape_t& sh = a.shape;
   const int Hq = sh.n_q_heads, Hkv = sh.n_kv_heads, hd = sh.head_dim, G = Hq / Hkv, S = sh.quest_page_size;
@@ -704,6 +841,22 @@ void launch_quest_selection(const AttnArgs& a, cudaStream_t st) {
   l.q_rot = a.q_rot; l.list_idx = a.list_idx; l.list_row = a.kept_row; l.kept_cnt = a.kept_cnt;
   l.page_mask = a.page_mask; l.logits = a.logits;
   l.n_rows = (uint32_t)a.kv.num_pages * Hkv * PAGE; l.status = a.status;
+  if (S % 16 == 0) {  // runs of 16 list entries are runs of 16 cache rows: tensor cores
+    QuestLogitMmaDev m;
+    m.kv = a.kv; m.B = a.B; m.Hq = Hq; m.Hkv = Hkv; m.G = G; m.Tmax = Tmax; m.S = S; m.Pstride = d.Pstride;
+    m.q_split = static_cast<const uint16_t*>(a.q_split); m.list_idx = a.list_idx; m.list_row = a.kept_row;
+    m.kept_cnt = a.kept_cnt; m.page_mask = a.page_mask; m.logits = a.logits;
+    m.n_rows = (uint32_t)a.kv.num_pages * Hkv * PAGE; m.status = a.status;
+    const int HG = (G + 3) / 4;
+    if (hd == 64) {
+      if (HG == 1) launch_quest_logits_mma<64, 1>(m, st);
+      else launch_quest_logits_mma<64, 2>(m, st);
+    } else {
+      if (HG == 1) launch_quest_logits_mma<128, 1>(m, st);
+      else launch_quest_logits_mma<128, 2>(m, st);
+    }
+    return;
+  }
   const dim3 grid((Tmax + QL_CHUNK - 1) / QL_CHUNK, Hkv, a.B);
   if (hd == 64) {
     if (G <= 4) SOL_LAUNCH("quest_logits", (quest_logits_kernel<64, 4>), grid, dim3(QL_THREADS), 0, st, l);
