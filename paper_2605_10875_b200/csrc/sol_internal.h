@@ -255,6 +255,7 @@ struct AttnArgs {
   unsigned char* page_mask;   // scratch [B][Hkv][Tmax / 4]: per Quest page, bit h = query head h of the group keeps it
   uint32_t* quest_keys;       // scratch [B][Hq][Tmax / S]: float32 bound of every page as a sortable key
   uint32_t* quest_err;        // scratch [B][Hq]: largest rounding-error bound of the row's scores (float bits)
+  unsigned char* quest_hmask; // scratch [B][Hq][Tmax / S]: 1 = the query head keeps the page
   int32_t* quest_pages_out;   // optional: the caller's [B][Hq][Tmax / S] kept pages of every query head, ascending
   int32_t* quest_cnt_out;     // optional: [B][Hq]
   int* status;
@@ -267,7 +268,7 @@ void launch_quest_selection(const AttnArgs& a, cudaStream_t st);
 
 // Offsets of the attention scratch inside a buffer, starting at `at` (a multiple of 256).
 struct AttnScratch {
-  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_pub, cand_idx, cand_val, kept_idx, kept_cnt, kept_row, part, plan, work_items, work_ctr, page_mask, quest_keys, quest_err, end;
+  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_pub, cand_idx, cand_val, kept_idx, kept_cnt, kept_row, part, plan, work_items, work_ctr, page_mask, quest_keys, quest_err, quest_hmask, end;
   int splits;
 };
 inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_pages, size_t at) {
@@ -300,6 +301,7 @@ inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_page
   L.page_mask = take(quest ? BK * (Tmax / 4) : 0);
   L.quest_keys = take(quest ? (size_t)B * Hq * (Tmax / s.quest_page_size) * 4 : 0);
   L.quest_err = take(quest ? (size_t)B * Hq * 4 : 0);
+  L.quest_hmask = take(quest ? (size_t)B * Hq * (Tmax / s.quest_page_size) : 0);
   L.end = at;
   return L;
 }
@@ -326,6 +328,7 @@ inline void attn_scratch_bind(AttnArgs& a, void* base, const AttnScratch& L, int
   a.page_mask = b + L.page_mask;
   a.quest_keys = reinterpret_cast<uint32_t*>(b + L.quest_keys);
   a.quest_err = reinterpret_cast<uint32_t*>(b + L.quest_err);
+  a.quest_hmask = b + L.quest_hmask;
   a.quest_pages_out = nullptr;
   a.quest_cnt_out = nullptr;
   a.splits = L.splits;

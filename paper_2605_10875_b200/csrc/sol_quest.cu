@@ -95,6 +95,7 @@ struct QuestSelDev {
   const float* q_rot;       // [B][Hq][hd]
   const uint32_t* keys;     // [B][Hq][Prow] float32 bounds as keys (quest_score)
   const uint32_t* err;      // [B][Hq] largest error bound of the row, float bits
+  unsigned char* hmask;     // [B][Hq][Prow] 1 = the head keeps the page (quest_select -> quest_list)
   unsigned char* page_mask; // [B][Hkv][Pstride]
   int32_t* list_idx;        // [B][Hkv][Tmax]
   uint32_t* list_row;
@@ -314,20 +315,19 @@ __global__ void __launch_bounds__(QS_THREADS) quest_score_kernel(const QuestScor
 // taken from them by a second radix select on the 64-bit keys, ties to the lower page.
 __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSelDev p) {
   extern __shared__ __align__(16) unsigned char qsm[];
-  const int kvh = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int b = blockIdx.y, tid = threadIdx.x;  // blockIdx.x: the query head
   const int Hkv = p.sh.n_kv_heads, Hq = p.sh.n_q_heads, G = Hq / Hkv, hd = p.sh.head_dim, S = p.S;
-  const int bk = b * Hkv + kvh;
-  const int HP = p.heads_per_pass;  // query heads whose float32 keys are in shared memory at once
+  const int kvh = blockIdx.x / G;
+  constexpr int HP = 1;  // one query head per CTA: the heads of a group are selected side by side
   unsigned long long* cand_key = reinterpret_cast<unsigned long long*>(qsm);             // [QS_CAND_CAP]
   float* qf = reinterpret_cast<float*>(cand_key + QS_CAND_CAP);                           // [HP][hd] the heads' queries (16-byte aligned)
   uint32_t* keys_all = reinterpret_cast<uint32_t*>(qf + (size_t)HP * hd);                 // [HP][Prow]
   int* cand_idx = reinterpret_cast<int*>(keys_all + (size_t)HP * p.Prow);                 // [QS_CAND_CAP]
   unsigned char* cand_sel = reinterpret_cast<unsigned char*>(cand_idx + QS_CAND_CAP);     // [QS_CAND_CAP]
-  unsigned char* mask = cand_sel + QS_CAND_CAP;                                           // [Prow]
   __shared__ int hist[256];
   __shared__ int scan_buf[QS_THREADS / 32];
   __shared__ unsigned long long s_prefix;
-  __shared__ int s_remaining, s_item0;
+  __shared__ int s_remaining;
   pdl_trigger();
   pdl_wait();
 
@@ -349,10 +349,9 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
     return reinterpret_cast<const uint4*>(meta + quest_meta_offset(ok ? page : 0, kvh, (tok % PAGE) / S, Hkv, S, hd));
   };
 
-  for (int pg = tid; pg < P; pg += QS_THREADS) mask[pg] = 0;
-
-  for (int h0 = 0; h0 < G; h0 += HP) {
-    const int nh = min(HP, G - h0);
+  {
+    const int h0 = blockIdx.x - kvh * G;
+    const int nh = 1;
     __syncthreads();  // keys and queries of the previous heads are not read any more
     for (int i = tid; i < nh * hd; i += QS_THREADS) qf[i] = p.q_rot[((size_t)b * Hq + kvh * G + h0 + i / hd) * hd + i % hd];
     __syncthreads();
@@ -496,42 +495,63 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
         }
         int tot_sel;
         const int pos = quest_block_scan(sel ? 1 : 0, tot_sel, scan_buf);
-        if (sel) {
-          mask[pg] |= (unsigned char)(1u << h);
-          if (out) out[written + pos] = pg;
-        }
+        if (pg < P) p.hmask[((size_t)b * Hq + head) * p.Prow + pg] = sel ? 1 : 0;
+        if (sel && out) out[written + pos] = pg;
         written += tot_sel;
       }
       if (tid == 0 && p.cnt_out) p.cnt_out[(size_t)b * Hq + head] = written;
     }
   }
-  __syncthreads();
+}
 
-  // ---- the row's token list: every token of a page some head keeps, ascending ----
+// The union of the heads' pages of a (sequence, kv-head): the row's token list (every token of a page some head
+// keeps, ascending), a byte per page that says which heads keep it, and the row's pass-2 work items.
+__global__ void __launch_bounds__(QS_THREADS) quest_list_kernel(const QuestSelDev p) {
+  const int kvh = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int Hkv = p.sh.n_kv_heads, Hq = p.sh.n_q_heads, G = Hq / Hkv, S = p.S;
+  const int bk = b * Hkv + kvh;
+  __shared__ int scan_buf[QS_THREADS / 32];
+  __shared__ int s_item0;
+  pdl_trigger();
+  pdl_wait();
+  const int T = min(max(p.kv.seq_lens[b], 0), p.kv.max_pages_per_seq * PAGE);
+  const int P = (T + S - 1) / S;
+  const int32_t* table = p.kv.page_table + (size_t)b * p.kv.max_pages_per_seq;
   const size_t row = (size_t)bk * p.Tmax;
-  int n_list = 0;
+  // the kept pages in ascending order (page and first cache row), then the list entry by entry with full-width
+  // stores: every kept page but possibly the sequence's last holds S tokens, so entry n is token n % S of kept
+  // page n / S.  (A thread per page writing its S entries one by one took 71 us: each store touched a sector of
+  // its own.)
+  extern __shared__ __align__(16) unsigned char qlsm2[];
+  int* sel_page = reinterpret_cast<int*>(qlsm2);                          // [Prow]
+  uint32_t* sel_row0 = reinterpret_cast<uint32_t*>(sel_page + p.Prow);    // [Prow]
+  int n_sel = 0, n_list = 0;
   for (int base = 0; base < P; base += QS_THREADS) {
     const int pg = base + tid;
-    const unsigned char m = pg < P ? mask[pg] : 0;
+    unsigned char m = 0;
+    if (pg < P)
+      for (int h = 0; h < G; ++h) m |= (unsigned char)((p.hmask[((size_t)b * Hq + kvh * G + h) * p.Prow + pg] & 1u) << h);
     if (pg < P) p.page_mask[(size_t)bk * p.Pstride + pg] = m;
     const int ntok = m ? min(S, T - pg * S) : 0;
-    int tot;
-    const int off = quest_block_scan(ntok, tot, scan_buf);
-    if (ntok > 0) {
+    int tot_sel, tot;
+    const int pos = quest_block_scan(m ? 1 : 0, tot_sel, scan_buf);
+    (void)quest_block_scan(ntok, tot, scan_buf);
+    if (m) {
       const int tok = pg * S, page = table[tok / PAGE];
       const bool ok = page >= 0 && page < p.kv.num_pages;
-      const uint32_t r0 = (uint32_t)((page * Hkv + kvh) * PAGE + (tok % PAGE));
-      for (int j = 0; j < ntok; ++j) {
-        if (n_list + off + j >= p.Tmax) {  // cannot happen for a list of distinct tokens; checked, not trusted
-          atomicMax(p.status + 5, 1);
-          atomicMax(p.status + 6, n_list + off + j);
-          break;
-        }
-        p.list_idx[row + n_list + off + j] = tok + j;
-        p.list_row[row + n_list + off + j] = ok ? r0 + j : 0xffffffffu;
-      }
+      sel_page[n_sel + pos] = pg;
+      sel_row0[n_sel + pos] = ok ? (uint32_t)((page * Hkv + kvh) * PAGE + (tok % PAGE)) : 0xffffffffu;
     }
+    n_sel += tot_sel;
     n_list += tot;
+  }
+  __syncthreads();
+  n_list = min(n_list, p.Tmax);
+  for (int n = tid; n < n_list; n += QS_THREADS) {
+    const int i = n / S, j = n - i * S;
+    const uint32_t r0 = sel_row0[i];
+    p.list_idx[row + n] = sel_page[i] * S + j;
+    p.list_row[row + n] = r0 == 0xffffffffu ? r0 : r0 + j;
   }
   if (tid == 0) p.kept_cnt[bk] = n_list;
 
@@ -828,13 +848,13 @@ void launch_quest_selection(const AttnArgs& a, cudaStream_t st) {
   d.q_rot = a.q_rot; d.page_mask = a.page_mask; d.list_idx = a.list_idx; d.list_row = a.kept_row;
   d.kept_cnt = a.kept_cnt; d.pages_out = a.quest_pages_out; d.cnt_out = a.quest_cnt_out;
   d.work_items = a.work_items; d.work_ctr = a.work_ctr; d.status = a.status;
-  // as many heads' float32 keys at once as fit in ~96 KB
-  int hp = (96 * 1024) / (d.Prow * 4);
-  hp = hp < 1 ? 1 : (hp > G ? G : hp);
-  d.heads_per_pass = hp;
-  const int smem = QS_CAND_CAP * (8 + 4 + 1) + hp * d.Prow * 4 + hp * hd * 4 + d.Prow + 16;
+  d.heads_per_pass = 1;
+  d.hmask = a.quest_hmask;
+  const int smem = QS_CAND_CAP * (8 + 4 + 1) + d.Prow * 4 + hd * 4 + 16;
   ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_select_kernel), smem);
-  SOL_LAUNCH("quest_select", quest_select_kernel, dim3(Hkv, a.B), dim3(QS_THREADS), smem, st, d);
+  SOL_LAUNCH("quest_select", quest_select_kernel, dim3(Hq, a.B), dim3(QS_THREADS), smem, st, d);
+  ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_list_kernel), d.Prow * 8);
+  SOL_LAUNCH("quest_list", quest_list_kernel, dim3(Hkv, a.B), dim3(QS_THREADS), d.Prow * 8, st, d);
 
   QuestLogitDev l;
   l.kv = a.kv; l.Hq = Hq; l.Hkv = Hkv; l.G = G; l.hd = hd; l.Tmax = Tmax; l.S = S; l.Pstride = d.Pstride;
