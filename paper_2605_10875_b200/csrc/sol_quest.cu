@@ -7,14 +7,16 @@
 //                 (after a decode step's append).
 //   quest_score   the bound q_pos.m+ + q_neg.m- of every page for every query head, in float32, as sortable keys,
 //                 with a bound of its rounding error (a page costs 2/S of its keys' bytes).
-//   quest_select  one CTA per (sequence, kv-head): for each query head of the group an exact selection of its
-//                 ceil(b_t / S) best pages: radix select on the float32 keys, float64 bounds for the few pages
-//                 within the error window of the threshold (forced pages first, ties to the lower page); then
-//                 the union of the heads' pages as the row's token list, its pass-2 work items, and a byte
-//                 per page that says which heads keep it.
+//   quest_select  one CTA per (sequence, query head): an exact selection of the head's ceil(b_t / S) best pages: radix
+//                 select on the float32 keys, float64 bounds for the few pages within the error window of the
+//                 threshold (forced pages first, ties to the lower page); a byte per page: kept or not.
+//   quest_list    one CTA per (sequence, kv-head): the union of the group's heads' pages as the row's token list, its
+//                 pass-2 work items, and a byte per page that says which heads keep it.
 //   quest_logits  q.k of every listed token for the G heads (K rows are read only for pages in the union),
 //                 minus infinity for the heads that did not keep the token's page: pass 2 (attn_gather) then
-//                 weighs a token with zero for those heads, which is the paper's additive mask.
+//                 weighs a token with zero for those heads, which is the paper's additive mask.  On the tensor
+//                 cores when the page size is a multiple of 16 (a run of 16 list entries is then 16 consecutive
+//                 cache rows), on the FMA pipes otherwise.
 #include <math.h>
 
 #include "sol_common.cuh"
