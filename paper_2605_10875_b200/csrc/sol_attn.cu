@@ -524,7 +524,8 @@ struct HistSmem {
   int cum[PLAN_STRIDE];
 };
 
-__device__ __forceinline__ void settle_row(const SelectDev& p, SelectSmem& sm, double* qsum, const RowPlan& rp, int b,
+template <typename Smem>
+__device__ __forceinline__ void settle_row(const SelectDev& p, Smem& sm, double* qsum, const RowPlan& rp, int b,
                                            int kvh, int n_list, float edge, float lo, float delta, int ns_all,
                                            bool cands_in_smem);
 
@@ -880,7 +881,8 @@ __device__ __forceinline__ void token_scan_item(const SelectDev& p, ScanSmem& ss
 // sm.f32, or in the row's global candidate list).  Ranks the candidates in float32, re-scores those within
 // the window of the k-th value in float64 from the cache rows, appends the kept ones (ascending) to the
 // list, and emits the row's pass-2 work items.
-__device__ __forceinline__ void settle_row(const SelectDev& p, SelectSmem& sm, double* qsum, const RowPlan& rp, int b,
+template <typename Smem>
+__device__ __forceinline__ void settle_row(const SelectDev& p, Smem& sm, double* qsum, const RowPlan& rp, int b,
                                            int kvh, int n_list, float edge, float lo, float delta, int ns_all,
                                            bool cands_in_smem) {
   const int Hkv = p.sh.n_kv_heads, hd = p.sh.head_dim, G = p.sh.n_q_heads / Hkv;
@@ -1087,7 +1089,7 @@ __global__ void __launch_bounds__(TS_THREADS) token_scan_kernel(const SelectDev 
 
 // One CTA per (sequence, kv-head) of the rows that token_scan worked on.
 __global__ void __launch_bounds__(TS_THREADS) token_settle_kernel(const SelectDev p) {
-  __shared__ SelectSmem sm;
+  __shared__ SelectSmemOverlay sm;  // candidates from the global list (cands_in_smem = false): never beside the histogram
   __shared__ double qsum[128];
   const int kvh = blockIdx.x, b = blockIdx.y;
   pdl_trigger();

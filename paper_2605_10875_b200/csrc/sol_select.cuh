@@ -37,6 +37,26 @@ struct SelectSmem {
   int counts[4];
 };
 
+// The same members for a kernel that never needs the histogram and the candidate arrays at the same time (the
+// settling kernel: a row either fits the candidate list or is redone by the radix select, which alone uses the
+// histogram): they share their space, 19 KB instead of 35 KB, so that one more CTA fits on an SM.
+struct SelectSmemOverlay {
+  union {
+    uint32_t hist[SEL_BINS];
+    struct {
+      int cand_idx[SEL_CAND_CAP];
+      double cand_val[SEL_CAND_CAP];
+      float f32[SEL_CAND_CAP];
+    };
+  };
+  unsigned char cand_keep[SEL_CAND_CAP];
+  uint32_t rank_key[SEL_RANK_CAP];
+  int pick[3];
+  int scan[2][SEL_MAX_WARPS];
+  float f[2][SEL_MAX_WARPS];
+  int counts[4];
+};
+
 // f(i) for the first `per` elements of a thread: unrolled over KPT register slots, or (KPT == 0) a
 // rolled loop.
 template <int KPT, typename F>
@@ -216,8 +236,8 @@ __device__ __forceinline__ uint32_t select_kth(KeyFn key, int k, int& tie_need, 
 
 // Sum of v over the block, returned to every thread.  `slot` (0 or 1) picks the scratch row so that
 // two calls in a row need no barrier between them.
-template <int THREADS>
-__device__ __forceinline__ int block_count(int v, int slot, SelectSmem& sm) {
+template <int THREADS, typename Smem>
+__device__ __forceinline__ int block_count(int v, int slot, Smem& sm) {
   constexpr int WARPS = THREADS / 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   v = __reduce_add_sync(0xffffffffu, v);
@@ -226,8 +246,8 @@ __device__ __forceinline__ int block_count(int v, int slot, SelectSmem& sm) {
   return __reduce_add_sync(0xffffffffu, lane < WARPS ? sm.scan[slot][lane] : 0);
 }
 
-template <int THREADS>
-__device__ __forceinline__ float block_max(float v, int slot, SelectSmem& sm) {
+template <int THREADS, typename Smem>
+__device__ __forceinline__ float block_max(float v, int slot, Smem& sm) {
   constexpr int WARPS = THREADS / 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   v = warp_max(v);
@@ -238,8 +258,8 @@ __device__ __forceinline__ float block_max(float v, int slot, SelectSmem& sm) {
 
 // Ranks the first n_cand candidates (cand_val, cand_idx) and sets cand_keep[c] = (rank < need).
 // A barrier must separate the writes of cand_val from this call and this call from the readers.
-template <int THREADS>
-__device__ __forceinline__ void rank_candidates(int n_cand, int need, SelectSmem& sm) {
+template <int THREADS, typename Smem>
+__device__ __forceinline__ void rank_candidates(int n_cand, int need, Smem& sm) {
   for (int c = threadIdx.x; c < n_cand; c += THREADS) {
     const double v = sm.cand_val[c];
     const int j = sm.cand_idx[c];
