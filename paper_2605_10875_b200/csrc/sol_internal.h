@@ -256,6 +256,9 @@ struct AttnArgs {
   uint32_t* quest_keys;       // scratch [B][Hq][Tmax / S]: float32 bound of every page as a sortable key
   uint32_t* quest_err;        // scratch [B][Hq]: largest rounding-error bound of the row's scores (float bits)
   unsigned char* quest_hmask; // scratch [B][Hq][Tmax / S]: 1 = the query head keeps the page
+  uint16_t* quest_qsplit;     // scratch [B][Hkv][ceil(G / 4) * 16][2 hd] bf16: sign-split queries as a tensor-core operand
+  float* quest_l1;            // scratch [B][Hq]: |q|_1
+  int* quest_order;           // scratch [B]: the sequences, longest first
   int32_t* quest_pages_out;   // optional: the caller's [B][Hq][Tmax / S] kept pages of every query head, ascending
   int32_t* quest_cnt_out;     // optional: [B][Hq]
   int* status;
@@ -268,7 +271,7 @@ void launch_quest_selection(const AttnArgs& a, cudaStream_t st);
 
 // Offsets of the attention scratch inside a buffer, starting at `at` (a multiple of 256).
 struct AttnScratch {
-  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_pub, cand_idx, cand_val, kept_idx, kept_cnt, kept_row, part, plan, work_items, work_ctr, page_mask, quest_keys, quest_err, quest_hmask, end;
+  size_t q_rot, q_split, logits, sigma, row_hist, row_ctl, seg_pub, cand_idx, cand_val, kept_idx, kept_cnt, kept_row, part, plan, work_items, work_ctr, page_mask, quest_keys, quest_err, quest_hmask, quest_qsplit, quest_l1, quest_order, end;
   int splits;
 };
 inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_pages, size_t at) {
@@ -302,6 +305,9 @@ inline AttnScratch attn_scratch_layout(const sol_shape_t& s, int B, int max_page
   L.quest_keys = take(quest ? (size_t)B * Hq * (Tmax / s.quest_page_size) * 4 : 0);
   L.quest_err = take(quest ? (size_t)B * Hq * 4 : 0);
   L.quest_hmask = take(quest ? (size_t)B * Hq * (Tmax / s.quest_page_size) : 0);
+  L.quest_qsplit = take(quest ? (size_t)B * Hkv * ((Hq / Hkv + 3) / 4) * 16 * 2 * hd * 2 : 0);
+  L.quest_l1 = take(quest ? (size_t)B * Hq * 4 : 0);
+  L.quest_order = take(quest ? (size_t)B * 4 : 0);
   L.end = at;
   return L;
 }
@@ -329,6 +335,9 @@ inline void attn_scratch_bind(AttnArgs& a, void* base, const AttnScratch& L, int
   a.quest_keys = reinterpret_cast<uint32_t*>(b + L.quest_keys);
   a.quest_err = reinterpret_cast<uint32_t*>(b + L.quest_err);
   a.quest_hmask = b + L.quest_hmask;
+  a.quest_qsplit = reinterpret_cast<uint16_t*>(b + L.quest_qsplit);
+  a.quest_l1 = reinterpret_cast<float*>(b + L.quest_l1);
+  a.quest_order = reinterpret_cast<int*>(b + L.quest_order);
   a.quest_pages_out = nullptr;
   a.quest_cnt_out = nullptr;
   a.splits = L.splits;

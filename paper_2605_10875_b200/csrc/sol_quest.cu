@@ -93,10 +93,11 @@ struct QuestSelDev {
   sol_shape_t sh;
   sol_kv_t kv;
   const int32_t* r_permille;
-  int Tmax, S, splits, split_len, Pstride, Prow, heads_per_pass;
+  int Tmax, S, splits, split_len, Pstride, Prow;
   const float* q_rot;       // [B][Hq][hd]
   const uint32_t* keys;     // [B][Hq][Prow] float32 bounds as keys (quest_score)
   const uint32_t* err;      // [B][Hq] largest error bound of the row, float bits
+  const int* order;         // [B] the sequences, longest first (quest_query)
   unsigned char* hmask;     // [B][Hq][Prow] 1 = the head keeps the page (quest_select -> quest_list)
   unsigned char* page_mask; // [B][Hkv][Pstride]
   int32_t* list_idx;        // [B][Hkv][Tmax]
@@ -207,104 +208,230 @@ __device__ __forceinline__ void quest_radix_threshold(const KeyT* keys, int n, i
   }
 }
 
-// Float32 bounds of every block of every (sequence, kv-head) for the G heads of the group, as keys, and per head
-// the row's largest rounding-error bound.  Per dimension only one of the two terms of q_pos.m+ + q_neg.m- is
-// there: |q| m+ for q >= 0, |q| m- otherwise.  A thread takes a block; the pieces of its extrema are fetched 64
-// dimensions at a time, all loads before the first use (one load per loop pass put a memory round trip between
-// every eight dimensions); two fused multiply-adds per dimension: the score and the sum of the terms'
-// magnitudes, which bounds the rounding error of the score.  A grid over all blocks: inside the per-row
-// selection kernel this was the tail of the longest row (94 us for 2048 blocks).
 struct QuestScoreDev {
   sol_shape_t sh;
   sol_kv_t kv;
-  int S, Prow;
+  int S, Prow, B;
   const float* q_rot;  // [B][Hq][hd]
   uint32_t* keys;      // [B][Hq][Prow]
-  uint32_t* err;       // [B][Hq] float bits, zeroed before the launch
+  uint32_t* err;       // [B][Hq] float bits, zeroed by quest_query_kernel
+  uint16_t* qsplit;    // [B][Hkv][ceil(G / 4) * 16][2 hd] bf16: the sign-split queries as an operand
+  float* l1;           // [B][Hq]: |q|_1
+  int* order;          // [B]: the sequences, longest first
   int* status;
 };
 
-__global__ void __launch_bounds__(QS_THREADS) quest_score_kernel(const QuestScoreDev p) {
-  __shared__ __align__(16) float qf[8 * 128];
-  __shared__ float wmax[8][QS_THREADS / 32];
-  const int kvh = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
-  const int Hkv = p.sh.n_kv_heads, Hq = p.sh.n_q_heads, G = Hq / Hkv, hd = p.sh.head_dim, S = p.S;
+// ---- the pages' bounds on the tensor cores ----
+// A page's extrema are one row of 2 hd bf16 numbers (m+, then -m-), and the bound is its dot product with the
+// query split by sign, [max(q, 0) ; max(-q, 0)]: the scoring pass over again with the extrema as keys.
+//
+// quest_query_kernel, a CTA per (sequence, kv-head): the G heads' sign-split queries, each as three bf16 parts
+// (exact to 2^-24), laid out as the N side of m16n8k16 (head t of a group of four: hi in row 2t, mid in row
+// 2t + 1, lo in row 8 + 2t of 16 rows of 2 hd), the heads' |q|_1, and the row's error bounds reset to zero.
+//
+// quest_score_mma_kernel: a warp takes 16 consecutive pages of a (sequence, kv-head) as the M side (their rows
+// come by bulk copies, one per cache page they lie in; a lane each, so that the table look-ups go side by side)
+// and reads the N side's fragments from the operand above while the rows travel.  Units of 64 pages are numbered
+// along the batch.  Error bound of a row's scores: (terms + 2) 2^-24 |q|_1 max|m| for the float32 sums plus
+// 2^-23 |q|_1 max|m| for the split, with max|m| over the row's extrema (taken from the fragments on the way).
+// (Building the operand in shared memory inside the scoring kernel, once per (sequence, kv-head) a CTA met, took
+// 39 us on the ragged batch where this takes less: the build and its barriers stood between the units.)
+constexpr int QSM_WARPS = 4;
+constexpr int QQ_THREADS = 128;
+
+__global__ void __launch_bounds__(QQ_THREADS) quest_query_kernel(const QuestScoreDev p) {
+  extern __shared__ __align__(16) unsigned char qqsm[];
+  uint16_t* qs = reinterpret_cast<uint16_t*>(qqsm);  // [HG * 16][2 hd]
+  __shared__ float s_l1[8];
+  const int kvh = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
+  const int Hkv = p.sh.n_kv_heads, Hq = p.sh.n_q_heads, G = Hq / Hkv, hd = p.sh.head_dim, HD2 = 2 * hd;
+  const int rows = ((G + 3) / 4) * 16;
   pdl_trigger();
-  const int T = min(max(p.kv.seq_lens[b], 0), p.kv.max_pages_per_seq * PAGE);
-  const int P = (T + S - 1) / S;
-  if ((int)blockIdx.x * QS_THREADS >= P) return;
-  pdl_wait();
-  const int n_sink = min(max(p.sh.n_sink, 0), T), n_win = min(max(p.sh.n_window, 0), T);
-  const int lo_pages = n_sink > 0 ? (n_sink - 1) / S + 1 : 0;
-  const int hi_first = n_win > 0 ? (T - n_win) / S : P;
-  for (int i = tid; i < G * hd; i += QS_THREADS) qf[i] = p.q_rot[((size_t)b * Hq + kvh * G + i / hd) * hd + i % hd];
+  for (int i = tid * 8; i < rows * HD2; i += QQ_THREADS * 8) *reinterpret_cast<uint4*>(qs + i) = make_uint4(0u, 0u, 0u, 0u);
+  if (tid < 8) s_l1[tid] = 0.f;
   __syncthreads();
-  const float err_unit = (float)(hd + 2) * 5.9604644775390625e-08f * 1.0001f;  // (hd + 2) 2^-24, rounded up
-  const int pg = blockIdx.x * QS_THREADS + tid;
-  float sc[8], ab[8];
+  pdl_wait();  // the rotated queries come from the kernel before; the scratch below may still be read until then
+  for (int i = tid; i < G * hd; i += QQ_THREADS) {
+    const int gi = i / hd, d = i - gi * hd;
+    const float q = p.q_rot[((size_t)b * Hq + kvh * G + gi) * hd + d];
+    const float v = fabsf(q);
+    const int e = q >= 0.f ? d : hd + d;  // the half of the operand row that meets m+ or -m-
+    const uint16_t hi = f2bf(v);
+    const float r1 = v - bf2f(hi);
+    const uint16_t mid = f2bf(r1);
+    uint16_t* base = qs + (size_t)((gi >> 2) * 16) * HD2;
+    const int tt = gi & 3;
+    base[(2 * tt) * HD2 + e] = hi;
+    base[(2 * tt + 1) * HD2 + e] = mid;
+    base[(8 + 2 * tt) * HD2 + e] = f2bf(r1 - bf2f(mid));
+    float sum = v;  // a warp's 32 dimensions belong to one head (head_dim is a multiple of 32)
 #pragma unroll
-  for (int hh = 0; hh < 8; ++hh) sc[hh] = ab[hh] = 0.f;
-  const bool forced = pg < lo_pages || pg >= hi_first;
-  bool ok = true;
-  if (pg < P && !forced) {
-    const int tok = pg * S, page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + tok / PAGE];
-    ok = page >= 0 && page < p.kv.num_pages;
-    if (!ok) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
-    const uint4* mp = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.kv.quest_meta) +
-                                                     quest_meta_offset(ok ? page : 0, kvh, (tok % PAGE) / S, Hkv, S, hd));
-    const int pieces = hd / 8;
-    for (int c0 = 0; c0 < pieces && ok; c0 += 8) {
-      uint4 a[8], m[8];
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        a[c] = mp[c0 + c];
-        m[c] = mp[pieces + c0 + c];
-      }
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const uint32_t aw[4] = {a[c].x, a[c].y, a[c].z, a[c].w}, mw[4] = {m[c].x, m[c].y, m[c].z, m[c].w};
-        float up[8], dn[8];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          up[2 * e] = bf16_lo(aw[e]);
-          up[2 * e + 1] = bf16_hi(aw[e]);
-          dn[2 * e] = bf16_lo(mw[e]);
-          dn[2 * e + 1] = bf16_hi(mw[e]);
-        }
-#pragma unroll
-        for (int hh = 0; hh < 8; ++hh) {
-          if (hh < G) {
-            const float4 qa = *reinterpret_cast<const float4*>(qf + hh * hd + (c0 + c) * 8);
-            const float4 qb = *reinterpret_cast<const float4*>(qf + hh * hd + (c0 + c) * 8 + 4);
-            const float q[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const float qv = q[e], mv = qv >= 0.f ? up[e] : dn[e];
-              sc[hh] = fmaf(fabsf(qv), mv, sc[hh]);
-              ab[hh] = fmaf(fabsf(qv), fabsf(mv), ab[hh]);
-            }
-          }
-        }
-      }
-    }
-  }
-#pragma unroll
-  for (int hh = 0; hh < 8; ++hh) {
-    if (hh < G) {
-      if (pg < P) p.keys[((size_t)b * Hq + kvh * G + hh) * p.Prow + pg] = forced ? 0xffffffffu : quest_key32(ok ? sc[hh] : -INFINITY);
-      float v = (pg < P && !forced && ok) ? ab[hh] * err_unit : 0.f;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-      if ((tid & 31) == 0) wmax[hh][tid >> 5] = v;
-    }
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) atomicAdd(&s_l1[gi], sum);
   }
   __syncthreads();
+  uint4* dst = reinterpret_cast<uint4*>(p.qsplit + (size_t)(b * Hkv + kvh) * rows * HD2);
+  for (int i = tid; i < rows * HD2 / 8; i += QQ_THREADS) dst[i] = reinterpret_cast<const uint4*>(qs)[i];
   if (tid < G) {
-    float v = 0.f;
-#pragma unroll
-    for (int x = 0; x < QS_THREADS / 32; ++x) v = fmaxf(v, wmax[tid][x]);
-    atomicMax(p.err + (size_t)b * Hq + kvh * G + tid, __float_as_uint(v));  // non-negative floats order like their bits
+    p.l1[(size_t)b * Hq + kvh * G + tid] = s_l1[tid];
+    p.err[(size_t)b * Hq + kvh * G + tid] = 0u;
   }
+  // the first CTA also ranks the sequences by length: the selection starts its longest rows first, so that none
+  // of them begins when the others are about to end
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid < p.B) {
+    const int mine = p.kv.seq_lens[tid];
+    int rank = 0;
+    for (int j = 0; j < p.B; ++j) {
+      const int other = p.kv.seq_lens[j];
+      rank += (other > mine || (other == mine && j < tid)) ? 1 : 0;
+    }
+    p.order[rank] = tid;
+  }
+}
+
+template <int HD2, int HG>
+__global__ void __launch_bounds__(QSM_WARPS * 32) quest_score_mma_kernel(const QuestScoreDev p) {
+  extern __shared__ __align__(128) unsigned char qssm[];
+  constexpr int TILE_BYTES = 16 * HD2 * 2;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(qssm + QSM_WARPS * TILE_BYTES);
+  __shared__ int s_cum[QSM_WARPS * 32 + 1], s_wsum[QSM_WARPS];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int Hkv = p.sh.n_kv_heads, Hq = p.sh.n_q_heads, G = Hq / Hkv, hd = HD2 / 2, S = p.S;
+  const int B = p.B;
+  pdl_trigger();
+  int my_incl = 0;
+  if (tid < B) {
+    const int T = min(max(p.kv.seq_lens[tid], 0), p.kv.max_pages_per_seq * PAGE);
+    my_incl = ((T + S - 1) / S + 16 * QSM_WARPS - 1) / (16 * QSM_WARPS);
+  }
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, my_incl, o);
+    if (lane >= o) my_incl += x;
+  }
+  if (lane == 31) s_wsum[warp] = my_incl;
+  if (tid == 0) {
+    for (int i = 0; i < QSM_WARPS; ++i) mbar_init(&bars[i], 1);
+    fence_mbar_init();
+    s_cum[0] = 0;
+  }
+  __syncthreads();
+  for (int w = 0; w < warp; ++w) my_incl += s_wsum[w];
+  s_cum[tid + 1] = my_incl;
+  __syncthreads();
+  const int n_units = s_cum[B] * Hkv;
+  if ((int)blockIdx.x >= n_units) return;
+  pdl_wait();
+  const int g = lane >> 2, t = lane & 3;
+  constexpr int KS = HD2 / 32;
+  const int npk = PAGE / S;                        // pages per cache page
+  const int rpc = npk < 16 ? npk : 16;             // rows per bulk copy
+  uint32_t phase = 0;
+  bool dead = false;
+#pragma unroll 1
+  for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const int key = u / Hkv;
+    const int b = __syncthreads_count(tid < B && my_incl <= key);
+    const int first = s_cum[b], n_groups = s_cum[b + 1] - first;
+    const int rem = u - first * Hkv;
+    const int kvh = rem / n_groups, grp = rem - kvh * n_groups;
+    const int T = min(max(p.kv.seq_lens[b], 0), p.kv.max_pages_per_seq * PAGE);
+    const int P = (T + S - 1) / S;
+    const int pg0 = (grp * QSM_WARPS + warp) * 16;
+    if (dead || pg0 >= P) continue;
+    const int n_sink = min(max(p.sh.n_sink, 0), T), n_win = min(max(p.sh.n_window, 0), T);
+    const int lo_pages = n_sink > 0 ? (n_sink - 1) / S + 1 : 0;
+    const int hi_first = n_win > 0 ? (T - n_win) / S : P;
+    unsigned char* tile = qssm + warp * TILE_BYTES;
+    const int nrow = min(16, P - pg0);
+    if (lane == 0) mbar_expect_tx(&bars[warp], nrow * HD2 * 2);
+    __syncwarp();
+    {
+      const int r0 = lane * rpc;
+      if (r0 < nrow) {
+        const int tok = (pg0 + r0) * S, page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + tok / PAGE];
+        const bool ok = page >= 0 && page < p.kv.num_pages;
+        if (!ok) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
+        const int n = min(rpc, nrow - r0);
+        bulk_g2s(tile + (size_t)r0 * HD2 * 2,
+                 static_cast<const uint16_t*>(p.kv.quest_meta) + quest_meta_offset(ok ? page : 0, kvh, (tok % PAGE) / S, Hkv, S, hd),
+                 n * HD2 * 2, &bars[warp]);
+      }
+    }
+    const uint16_t* qop = p.qsplit + (size_t)(b * Hkv + kvh) * (HG * 16) * HD2;
+    uint4 qf[KS][2];
+#pragma unroll
+    for (int sx = 0; sx < KS; ++sx) {
+      qf[sx][0] = __ldg(reinterpret_cast<const uint4*>(qop + (size_t)g * HD2 + sx * 32 + t * 8));
+      qf[sx][1] = __ldg(reinterpret_cast<const uint4*>(qop + (size_t)(8 + g) * HD2 + sx * 32 + t * 8));
+    }
+    if (!mbar_wait(&bars[warp], phase, p.status)) {
+      dead = true;
+      continue;
+    }
+    phase ^= 1;
+    const uint32_t tb = smem_u32(tile);
+    const bool v0 = g < nrow, v1 = g + 8 < nrow;  // rows beyond the sequence's pages hold whatever the tile held before
+    uint4 ka[KS][2];
+    uint32_t am = 0u;  // largest magnitudes of this lane's elements, two bf16 patterns side by side
+#pragma unroll
+    for (int sx = 0; sx < KS; ++sx) {
+      ka[sx][0] = v0 ? lds128(tb + g * (HD2 * 2) + (sx * 32 + t * 8) * 2) : make_uint4(0u, 0u, 0u, 0u);
+      ka[sx][1] = v1 ? lds128(tb + (g + 8) * (HD2 * 2) + (sx * 32 + t * 8) * 2) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int x = 0; x < 2; ++x) {
+        am = __vmaxu2(am, ka[sx][x].x & 0x7fff7fffu);
+        am = __vmaxu2(am, ka[sx][x].y & 0x7fff7fffu);
+        am = __vmaxu2(am, ka[sx][x].z & 0x7fff7fffu);
+        am = __vmaxu2(am, ka[sx][x].w & 0x7fff7fffu);
+      }
+    }
+#pragma unroll
+    for (int hg = 0; hg < HG; ++hg) {
+      float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int sx = 0; sx < KS; ++sx) {
+        mma_bf16(d0, ka[sx][0].x, ka[sx][1].x, ka[sx][0].y, ka[sx][1].y, qf[sx][0].x, qf[sx][0].y);
+        mma_bf16(d0, ka[sx][0].z, ka[sx][1].z, ka[sx][0].w, ka[sx][1].w, qf[sx][0].z, qf[sx][0].w);
+        mma_bf16(d1, ka[sx][0].x, ka[sx][1].x, ka[sx][0].y, ka[sx][1].y, qf[sx][1].x, qf[sx][1].y);
+        mma_bf16(d1, ka[sx][0].z, ka[sx][1].z, ka[sx][0].w, ka[sx][1].w, qf[sx][1].z, qf[sx][1].w);
+      }
+      if (hg + 1 < HG) {  // the next four heads' fragments (more than four heads per kv-head is the rare case)
+#pragma unroll
+        for (int sx = 0; sx < KS; ++sx) {
+          qf[sx][0] = __ldg(reinterpret_cast<const uint4*>(qop + (size_t)((hg + 1) * 16 + g) * HD2 + sx * 32 + t * 8));
+          qf[sx][1] = __ldg(reinterpret_cast<const uint4*>(qop + (size_t)((hg + 1) * 16 + 8 + g) * HD2 + sx * 32 + t * 8));
+        }
+      }
+      const float s0 = d0[0] + (d0[1] + d1[0]);  // page pg0 + g
+      const float s1 = d0[2] + (d0[3] + d1[2]);  // page pg0 + g + 8
+      const int head = hg * 4 + t;
+      if (head < G) {
+        uint32_t* dst = p.keys + ((size_t)b * Hq + kvh * G + head) * p.Prow;
+        const int pa = pg0 + g, pb = pg0 + g + 8;
+        if (v0) dst[pa] = (pa < lo_pages || pa >= hi_first) ? 0xffffffffu : quest_key32(s0);
+        if (v1) dst[pb] = (pb < lo_pages || pb >= hi_first) ? 0xffffffffu : quest_key32(s1);
+      }
+    }
+    am = max(am & 0xffffu, am >> 16);
+    am = __reduce_max_sync(0xffffffffu, am);
+    if (lane < G) {
+      const float amax = __uint_as_float(am << 16);
+      const float w = ((float)(3 * HD2 + 2) * 5.9604644775390625e-08f + 1.1920928955078125e-07f) * 1.001f *
+                      p.l1[(size_t)b * Hq + kvh * G + lane] * amax;
+      atomicMax(p.err + (size_t)b * Hq + kvh * G + lane, __float_as_uint(w));  // non-negative floats order like their bits
+    }
+    __syncwarp();
+  }
+}
+
+template <int HD2, int HG>
+static void launch_quest_score_mma(const QuestScoreDev& d, int Hkv, cudaStream_t st) {
+  const int smem = QSM_WARPS * 16 * HD2 * 2 + QSM_WARPS * 8 + 32;
+  const long long upper = (long long)((d.Prow + 16 * QSM_WARPS - 1) / (16 * QSM_WARPS)) * Hkv * d.B;
+  const long long resident = (long long)sm_count() * (HD2 == 128 ? 24 : 12);  // twice what the shared memory lets stay on an SM
+  ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_score_mma_kernel<HD2, HG>), smem);
+  SOL_LAUNCH("quest_score", (quest_score_mma_kernel<HD2, HG>), dim3((unsigned)(upper < resident ? upper : resident)), dim3(QSM_WARPS * 32), smem, st, d);
 }
 
 // Selection of one query head, in two precisions.  The bound of every page is first summed in float32 (two
@@ -317,21 +444,22 @@ __global__ void __launch_bounds__(QS_THREADS) quest_score_kernel(const QuestScor
 // taken from them by a second radix select on the 64-bit keys, ties to the lower page.
 __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSelDev p) {
   extern __shared__ __align__(16) unsigned char qsm[];
-  const int b = blockIdx.y, tid = threadIdx.x;  // blockIdx.x: the query head
+  const int tid = threadIdx.x, head = blockIdx.x;  // one query head per CTA
   const int Hkv = p.sh.n_kv_heads, Hq = p.sh.n_q_heads, G = Hq / Hkv, hd = p.sh.head_dim, S = p.S;
-  const int kvh = blockIdx.x / G;
-  constexpr int HP = 1;  // one query head per CTA: the heads of a group are selected side by side
+  const int kvh = head / G;
   unsigned long long* cand_key = reinterpret_cast<unsigned long long*>(qsm);             // [QS_CAND_CAP]
-  float* qf = reinterpret_cast<float*>(cand_key + QS_CAND_CAP);                           // [HP][hd] the heads' queries (16-byte aligned)
-  uint32_t* keys_all = reinterpret_cast<uint32_t*>(qf + (size_t)HP * hd);                 // [HP][Prow]
-  int* cand_idx = reinterpret_cast<int*>(keys_all + (size_t)HP * p.Prow);                 // [QS_CAND_CAP]
+  float* qf = reinterpret_cast<float*>(cand_key + QS_CAND_CAP);                           // [hd] the head's query (16-byte aligned)
+  uint32_t* keys = reinterpret_cast<uint32_t*>(qf + hd);                                  // [Prow]
+  int* cand_idx = reinterpret_cast<int*>(keys + p.Prow);                                  // [QS_CAND_CAP]
   unsigned char* cand_sel = reinterpret_cast<unsigned char*>(cand_idx + QS_CAND_CAP);     // [QS_CAND_CAP]
+  unsigned char* pflag = cand_sel + QS_CAND_CAP;                                          // [Prow] 1 = the head keeps the page
   __shared__ int hist[256];
   __shared__ int scan_buf[QS_THREADS / 32];
   __shared__ unsigned long long s_prefix;
-  __shared__ int s_remaining;
+  __shared__ int s_remaining, s_ncand, s_cin;
   pdl_trigger();
   pdl_wait();
+  const int b = p.order[blockIdx.y];  // longest sequences first
 
   const int T = min(max(p.kv.seq_lens[b], 0), p.kv.max_pages_per_seq * PAGE);
   const int P = (T + S - 1) / S;
@@ -351,159 +479,173 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
     return reinterpret_cast<const uint4*>(meta + quest_meta_offset(ok ? page : 0, kvh, (tok % PAGE) / S, Hkv, S, hd));
   };
 
-  {
-    const int h0 = blockIdx.x - kvh * G;
-    const int nh = 1;
-    __syncthreads();  // keys and queries of the previous heads are not read any more
-    for (int i = tid; i < nh * hd; i += QS_THREADS) qf[i] = p.q_rot[((size_t)b * Hq + kvh * G + h0 + i / hd) * hd + i % hd];
-    __syncthreads();
-    // ---- the float32 keys of these heads' bounds (quest_score) ----
-    for (int hh = 0; hh < nh; ++hh) {
-      const uint32_t* src = p.keys + ((size_t)b * Hq + kvh * G + h0 + hh) * p.Prow;
-      for (int pg = tid; pg < P; pg += QS_THREADS) keys_all[(size_t)hh * p.Prow + pg] = src[pg];
+  for (int i = tid; i < hd; i += QS_THREADS) qf[i] = p.q_rot[((size_t)b * Hq + head) * hd + i];
+  {  // the float32 keys of this head's bounds (quest_score)
+    const uint32_t* src = p.keys + ((size_t)b * Hq + head) * p.Prow;
+    for (int pg = tid; pg < P; pg += QS_THREADS) keys[pg] = src[pg];
+  }
+  if (tid == 0) {
+    s_ncand = 0;
+    s_cin = 0;
+  }
+  __syncthreads();
+  const bool all_pages = n_keep >= P;
+  uint32_t tau32 = 0u;
+  int rem32 = 0;
+  if (!all_pages && n_keep > 0) {
+    quest_radix_threshold<uint32_t>(keys, P, n_keep, hist, &s_prefix, &s_remaining);
+    tau32 = (uint32_t)s_prefix;
+    rem32 = s_remaining;
+  }
+  __syncthreads();  // s_prefix, s_remaining are rewritten below
+  const float w = __uint_as_float(p.err[(size_t)b * Hq + head]);  // the row's largest error bound for this head
+  const bool only_forced = tau32 == 0xffffffffu || n_keep == 0;  // the budget is met by the forced pages alone
+  const double tau = only_forced || all_pages ? 0.0 : (double)quest_key32_value(tau32);
+  const double hi = tau + 2.002 * (double)w, lo = tau - 2.002 * (double)w;
+  auto classify = [&](int pg, bool& in, bool& cand) {
+    const uint32_t k = keys[pg];
+    const double v = (double)quest_key32_value(k);
+    in = k == 0xffffffffu || v > hi;
+    cand = !in && v >= lo;
+  };
+  // ---- the pages above hi are kept; those between lo and hi are listed (in no order: the lanes take their
+  //      slots by a counter, which spares a block-wide scan per 256 pages) ----
+  int n_cand = 0, c_in = 0;
+  bool overflow = false;
+  if (all_pages || only_forced) {
+    for (int pg = tid; pg < P; pg += QS_THREADS) pflag[pg] = (all_pages || keys[pg] == 0xffffffffu) ? 1 : 0;
+  } else {
+    int my_in = 0;
+    for (int pg = tid; pg < P; pg += QS_THREADS) {
+      bool in, cand;
+      classify(pg, in, cand);
+      my_in += in ? 1 : 0;
+      pflag[pg] = in ? 1 : 0;
+      if (cand) {
+        const int slot = atomicAdd(&s_ncand, 1);
+        if (slot < QS_CAND_CAP) cand_idx[slot] = pg;
+      }
     }
-
-    for (int hh = 0; hh < nh; ++hh) {
-      const int h = h0 + hh, head = kvh * G + h;
-      const uint32_t* keys = keys_all + (size_t)hh * p.Prow;
-      __syncthreads();
-      const bool all_pages = n_keep >= P;
-      uint32_t tau32 = 0u;
-      int rem32 = 0;
-      if (!all_pages && n_keep > 0) {
-        quest_radix_threshold<uint32_t>(keys, P, n_keep, hist, &s_prefix, &s_remaining);
-        tau32 = (uint32_t)s_prefix;
-        rem32 = s_remaining;
-      }
-      __syncthreads();  // s_prefix, s_remaining are rewritten below
-      const float w = __uint_as_float(p.err[(size_t)b * Hq + head]);  // the row's largest error bound for this head
-      const bool only_forced = tau32 == 0xffffffffu || n_keep == 0;  // the budget is met by the forced pages alone
-      const double tau = only_forced || all_pages ? 0.0 : (double)quest_key32_value(tau32);
-      const double hi = tau + 2.002 * (double)w, lo = tau - 2.002 * (double)w;
-      // ---- the pages between lo and hi, in page order ----
-      int n_cand = 0, c_in = 0;
-      bool overflow = false;
-      if (!all_pages && !only_forced) {
-        for (int base = 0; base < P; base += QS_THREADS) {
-          const int pg = base + tid;
-          const uint32_t k = pg < P ? keys[pg] : 0u;
-          const double v = (double)quest_key32_value(k);
-          const bool forced = pg < P && k == 0xffffffffu;
-          const bool in = pg < P && (forced || v > hi);
-          const bool cand = pg < P && !forced && !in && v >= lo;
-          int tot_c, tot_in;
-          const int pos = quest_block_scan(cand ? 1 : 0, tot_c, scan_buf);
-          (void)quest_block_scan(in ? 1 : 0, tot_in, scan_buf);
-          if (cand && n_cand + pos < QS_CAND_CAP) cand_idx[n_cand + pos] = pg;
-          n_cand += tot_c;
-          c_in += tot_in;
-        }
-        overflow = n_cand > QS_CAND_CAP;
-        if (overflow && tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
-        __syncthreads();  // the candidate list is read by other threads than those that wrote it
-      }
-      const bool refine = !all_pages && !only_forced && !overflow && n_cand > 0;
-      if (refine) {
-        // ---- exact bounds of the candidates: a group of hd/4 lanes per candidate, one piece of the extrema per
-        //      lane, float64 partial sums added up over the group ----
-        {
-          const int lane = tid & 31, warp = tid >> 5;
-          const int LPG = hd / 4, GPW = 32 / LPG, sub = lane % LPG, grp = lane / LPG;
-          const bool minus = sub >= hd / 8;
-          const int d0 = (minus ? sub - hd / 8 : sub) * 8;
-          const float* q = qf + hh * hd + d0;
-          const int stride = (QS_THREADS / 32) * GPW;
-          for (int c0 = 0; c0 < n_cand; c0 += stride) {  // block-uniform trip count
-            const int c = c0 + warp * GPW + grp;
-            bool ok = true;
-            uint4 piece = make_uint4(0u, 0u, 0u, 0u);
-            if (c < n_cand) {
-              const uint4* mp = page_meta(cand_idx[c], ok);
-              if (ok) piece = mp[sub];
-            }
-            const uint32_t w4[4] = {piece.x, piece.y, piece.z, piece.w};
-            double sd = 0.0;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const float q0 = q[2 * e], q1 = q[2 * e + 1];
-              if ((q0 < 0.f) == minus) sd = fma((double)fabsf(q0), (double)bf16_lo(w4[e]), sd);
-              if ((q1 < 0.f) == minus) sd = fma((double)fabsf(q1), (double)bf16_hi(w4[e]), sd);
-            }
-            for (int o = 1; o < LPG; o <<= 1) sd += __shfl_xor_sync(0xffffffffu, sd, o);
-            if (sub == 0 && c < n_cand) cand_key[c] = quest_key(ok ? sd : -INFINITY);
-          }
-        }
-        if (tid == 0) atomicAdd(p.status + ST_TOK_REFINED, n_cand);
-        __syncthreads();
-        const int need2 = min(max(n_keep - c_in, 0), n_cand);
-        if (n_cand <= QS_THREADS) {
-          // a short list: a candidate is kept when fewer than need2 others come before it (larger key, or the
-          // same key and a lower page)
-          const unsigned long long mine = tid < n_cand ? cand_key[tid] : 0ull;
-          int rank = 0;
-          for (int x = 0; x < n_cand; ++x) {
-            const unsigned long long k = cand_key[x];
-            rank += (k > mine || (k == mine && x < tid)) ? 1 : 0;
-          }
-          if (tid < n_cand) cand_sel[tid] = rank < need2 ? 1 : 0;
-        } else {
-          unsigned long long tau64 = ~0ull;  // need2 == 0: no candidate key reaches this
-          int rem64 = 0;
-          if (need2 > 0) {
-            quest_radix_threshold<unsigned long long>(cand_key, n_cand, need2, hist, &s_prefix, &s_remaining);
-            tau64 = s_prefix;
-            rem64 = s_remaining;
-          }
-          // the candidates that are kept, in page order
-          int seen = 0;
-          for (int base = 0; base < n_cand; base += QS_THREADS) {
-            const int c = base + tid;
-            const unsigned long long k = c < n_cand ? cand_key[c] : 0ull;
-            const bool eq = c < n_cand && k == tau64;
-            int tot;
-            const int rank = quest_block_scan(eq ? 1 : 0, tot, scan_buf);
-            if (c < n_cand) cand_sel[c] = (k > tau64 || (eq && seen + rank < rem64)) ? 1 : 0;
-            seen += tot;
-          }
-        }
-        __syncthreads();
-      }
-      // ---- mark the head's pages; write its ascending page list ----
-      int seen_equal = 0, seen_cand = 0, written = 0;
-      int32_t* out = p.pages_out ? p.pages_out + ((size_t)b * Hq + head) * p.Prow : nullptr;
+    for (int o = 16; o > 0; o >>= 1) my_in += __shfl_xor_sync(0xffffffffu, my_in, o);
+    if ((tid & 31) == 0 && my_in) atomicAdd(&s_cin, my_in);
+    __syncthreads();
+    n_cand = s_ncand;
+    c_in = s_cin;
+    overflow = n_cand > QS_CAND_CAP;
+    if (overflow && tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
+    if (n_cand > QS_THREADS && !overflow) {
+      // a long list goes through the radix select below, whose tie rule (the lower page first) reads the list
+      // in page order: listed again, by ordered scans
+      int at = 0;
       for (int base = 0; base < P; base += QS_THREADS) {
         const int pg = base + tid;
-        const uint32_t k = pg < P ? keys[pg] : 0u;
-        bool sel = false;
-        if (all_pages) {
-          sel = pg < P;
-        } else if (only_forced) {
-          sel = pg < P && k == 0xffffffffu;
-        } else if (overflow) {  // float32 order, ties to the lower page
-          const bool eq = pg < P && k == tau32;
-          int tot;
-          const int rank = quest_block_scan(eq ? 1 : 0, tot, scan_buf);
-          sel = pg < P && (k > tau32 || (eq && seen_equal + rank < rem32));
-          seen_equal += tot;
-        } else {
-          const double v = (double)quest_key32_value(k);
-          const bool forced = pg < P && k == 0xffffffffu;
-          const bool in = pg < P && (forced || v > hi);
-          const bool cand = pg < P && !forced && !in && v >= lo;
-          int tot;
-          const int pos = quest_block_scan(cand ? 1 : 0, tot, scan_buf);
-          sel = in || (cand && cand_sel[seen_cand + pos] != 0);
-          seen_cand += tot;
-        }
-        int tot_sel;
-        const int pos = quest_block_scan(sel ? 1 : 0, tot_sel, scan_buf);
-        if (pg < P) p.hmask[((size_t)b * Hq + head) * p.Prow + pg] = sel ? 1 : 0;
-        if (sel && out) out[written + pos] = pg;
-        written += tot_sel;
+        bool in = false, cand = false;
+        if (pg < P) classify(pg, in, cand);
+        int tot;
+        const int pos = quest_block_scan(cand ? 1 : 0, tot, scan_buf);
+        if (cand) cand_idx[at + pos] = pg;
+        at += tot;
       }
-      if (tid == 0 && p.cnt_out) p.cnt_out[(size_t)b * Hq + head] = written;
+      __syncthreads();
     }
   }
+  const bool refine = !all_pages && !only_forced && !overflow && n_cand > 0;
+  if (refine) {
+    // ---- exact bounds of the candidates: a group of hd/4 lanes per candidate, one piece of the extrema per
+    //      lane, float64 partial sums added up over the group ----
+    {
+      const int lane = tid & 31, warp = tid >> 5;
+      const int LPG = hd / 4, GPW = 32 / LPG, sub = lane % LPG, grp = lane / LPG;
+      const bool minus = sub >= hd / 8;
+      const int d0 = (minus ? sub - hd / 8 : sub) * 8;
+      const float* q = qf + d0;
+      const int stride = (QS_THREADS / 32) * GPW;
+      for (int c0 = 0; c0 < n_cand; c0 += stride) {  // block-uniform trip count
+        const int c = c0 + warp * GPW + grp;
+        bool ok = true;
+        uint4 piece = make_uint4(0u, 0u, 0u, 0u);
+        if (c < n_cand) {
+          const uint4* mp = page_meta(cand_idx[c], ok);
+          if (ok) piece = mp[sub];
+        }
+        const uint32_t w4[4] = {piece.x, piece.y, piece.z, piece.w};
+        double sd = 0.0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float q0 = q[2 * e], q1 = q[2 * e + 1];
+          if ((q0 < 0.f) == minus) sd = fma((double)fabsf(q0), (double)bf16_lo(w4[e]), sd);
+          if ((q1 < 0.f) == minus) sd = fma((double)fabsf(q1), (double)bf16_hi(w4[e]), sd);
+        }
+        for (int o = 1; o < LPG; o <<= 1) sd += __shfl_xor_sync(0xffffffffu, sd, o);
+        if (sub == 0 && c < n_cand) cand_key[c] = quest_key(ok ? sd : -INFINITY);
+      }
+    }
+    if (tid == 0) atomicAdd(p.status + ST_TOK_REFINED, n_cand);
+    __syncthreads();
+    const int need2 = min(max(n_keep - c_in, 0), n_cand);
+    if (n_cand <= QS_THREADS) {
+      // a short list: a candidate is kept when fewer than need2 others come before it (larger key, or the
+      // same key and a lower page)
+      const unsigned long long mine = tid < n_cand ? cand_key[tid] : 0ull;
+      const int my_pg = tid < n_cand ? cand_idx[tid] : 0;
+      int rank = 0;
+      for (int x = 0; x < n_cand; ++x) {
+        const unsigned long long k = cand_key[x];
+        rank += (k > mine || (k == mine && cand_idx[x] < my_pg)) ? 1 : 0;
+      }
+      if (tid < n_cand && rank < need2) pflag[my_pg] = 1;
+    } else {
+      unsigned long long tau64 = ~0ull;  // need2 == 0: no candidate key reaches this
+      int rem64 = 0;
+      if (need2 > 0) {
+        quest_radix_threshold<unsigned long long>(cand_key, n_cand, need2, hist, &s_prefix, &s_remaining);
+        tau64 = s_prefix;
+        rem64 = s_remaining;
+      }
+      // the candidates that are kept, ties in page order
+      int seen = 0;
+      for (int base = 0; base < n_cand; base += QS_THREADS) {
+        const int c = base + tid;
+        const unsigned long long k = c < n_cand ? cand_key[c] : 0ull;
+        const bool eq = c < n_cand && k == tau64;
+        int tot;
+        const int rank = quest_block_scan(eq ? 1 : 0, tot, scan_buf);
+        if (c < n_cand && (k > tau64 || (eq && seen + rank < rem64))) pflag[cand_idx[c]] = 1;
+        seen += tot;
+      }
+    }
+  } else if (overflow) {  // float32 order, ties to the lower page
+    int seen_equal = 0;
+    for (int base = 0; base < P; base += QS_THREADS) {
+      const int pg = base + tid;
+      const uint32_t k = pg < P ? keys[pg] : 0u;
+      const bool eq = pg < P && k == tau32;
+      int tot;
+      const int rank = quest_block_scan(eq ? 1 : 0, tot, scan_buf);
+      if (pg < P) pflag[pg] = (k > tau32 || (eq && seen_equal + rank < rem32)) ? 1 : 0;
+      seen_equal += tot;
+    }
+  }
+  __syncthreads();
+  // ---- the head's byte per page; its ascending page list where the caller asked for it ----
+  unsigned char* hm = p.hmask + ((size_t)b * Hq + head) * p.Prow;
+  if (p.pages_out == nullptr && p.cnt_out == nullptr) {
+    for (int pg = tid; pg < P; pg += QS_THREADS) hm[pg] = pflag[pg];
+    return;
+  }
+  int written = 0;
+  int32_t* out = p.pages_out ? p.pages_out + ((size_t)b * Hq + head) * p.Prow : nullptr;
+  for (int base = 0; base < P; base += QS_THREADS) {
+    const int pg = base + tid;
+    const bool sel = pg < P && pflag[pg] != 0;
+    int tot_sel;
+    const int pos = quest_block_scan(sel ? 1 : 0, tot_sel, scan_buf);
+    if (pg < P) hm[pg] = sel ? 1 : 0;
+    if (sel && out) out[written + pos] = pg;
+    written += tot_sel;
+  }
+  if (tid == 0 && p.cnt_out) p.cnt_out[(size_t)b * Hq + head] = written;
 }
 
 // The union of the heads' pages of a (sequence, kv-head): the row's token list (every token of a page some head
@@ -840,19 +982,28 @@ void launch_quest_selection(const AttnArgs& a, cudaStream_t st) {
   QuestScoreDev sc;
   sc.sh = sh; sc.kv = a.kv; sc.S = S; sc.Prow = Tmax / S; sc.q_rot = a.q_rot; sc.keys = a.quest_keys; sc.err = a.quest_err;
   sc.status = a.status;
-  record_cuda_error(cudaMemsetAsync(a.quest_err, 0, sizeof(uint32_t) * (size_t)a.B * Hq, st), "quest: clear the error bounds");
-  SOL_LAUNCH("quest_score", quest_score_kernel, dim3((sc.Prow + QS_THREADS - 1) / QS_THREADS, Hkv, a.B), dim3(QS_THREADS), 0, st, sc);
+  sc.B = a.B;
+  // the tensor-core kernel wants whole operand rows per cache page (S a power of two up to 64 gives that) and at
+  // most 8 heads per kv-head, which the shape check has seen to
+  sc.qsplit = a.quest_qsplit; sc.l1 = a.quest_l1; sc.order = a.quest_order;
+  SOL_LAUNCH("quest_query", quest_query_kernel, dim3(Hkv, a.B), dim3(QQ_THREADS), ((G + 3) / 4) * 16 * 2 * hd * 2, st, sc);
+  if (hd == 64) {
+    if (G <= 4) launch_quest_score_mma<128, 1>(sc, Hkv, st);
+    else launch_quest_score_mma<128, 2>(sc, Hkv, st);
+  } else {
+    if (G <= 4) launch_quest_score_mma<256, 1>(sc, Hkv, st);
+    else launch_quest_score_mma<256, 2>(sc, Hkv, st);
+  }
 
   QuestSelDev d;
-  d.keys = a.quest_keys; d.err = a.quest_err;
+  d.keys = a.quest_keys; d.err = a.quest_err; d.order = a.quest_order;
   d.sh = sh; d.kv = a.kv; d.r_permille = a.r_permille; d.Tmax = Tmax; d.S = S; d.splits = a.splits;
   d.split_len = attn_split_len(hd); d.Pstride = Tmax / 4; d.Prow = Tmax / S;
   d.q_rot = a.q_rot; d.page_mask = a.page_mask; d.list_idx = a.list_idx; d.list_row = a.kept_row;
   d.kept_cnt = a.kept_cnt; d.pages_out = a.quest_pages_out; d.cnt_out = a.quest_cnt_out;
   d.work_items = a.work_items; d.work_ctr = a.work_ctr; d.status = a.status;
-  d.heads_per_pass = 1;
   d.hmask = a.quest_hmask;
-  const int smem = QS_CAND_CAP * (8 + 4 + 1) + d.Prow * 4 + hd * 4 + 16;
+  const int smem = QS_CAND_CAP * (8 + 4 + 1) + d.Prow * (4 + 1) + hd * 4 + 16;
   ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_select_kernel), smem);
   SOL_LAUNCH("quest_select", quest_select_kernel, dim3(Hq, a.B), dim3(QS_THREADS), smem, st, d);
   ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_list_kernel), d.Prow * 8);

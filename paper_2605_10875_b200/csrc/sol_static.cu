@@ -104,6 +104,9 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
   a.quest_keys = nullptr;
   a.quest_err = nullptr;
   a.quest_hmask = nullptr;
+  a.quest_qsplit = nullptr;
+  a.quest_l1 = nullptr;
+  a.quest_order = nullptr;
   a.quest_pages_out = nullptr;
   a.quest_cnt_out = nullptr;
   a.status = reinterpret_cast<int*>(base);
