@@ -119,7 +119,8 @@ __device__ __forceinline__ unsigned long long quest_key(double s) {
   return k == ~0ull ? k - 1 : k;
 }
 
-// Exclusive prefix of v over the block (threads in index order) and the block total; `buf` holds one int per warp.
+// Exclusive prefix of v over a block of NTHR threads (in index order) and the block total; `buf` holds one int per warp.
+template <int NTHR = 256>
 __device__ __forceinline__ int quest_block_scan(int v, int& total, int* buf) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int incl = v;
@@ -133,7 +134,7 @@ __device__ __forceinline__ int quest_block_scan(int v, int& total, int* buf) {
   __syncthreads();
   int before = 0, tot = 0;
 #pragma unroll
-  for (int w = 0; w < QS_THREADS / 32; ++w) {
+  for (int w = 0; w < NTHR / 32; ++w) {
     const int x = buf[w];
     if (w < warp) before += x;
     tot += x;
@@ -142,7 +143,7 @@ __device__ __forceinline__ int quest_block_scan(int v, int& total, int* buf) {
   return before + incl - v;
 }
 
-constexpr int QS_CAND_CAP = 2048;  // pages per head whose bound is taken again in float64
+constexpr int QS_CAND_CAP = 1024;  // pages per head whose bound is taken again in float64
 
 // Monotone 32-bit key of a float; never the all-ones key (forced pages).
 __device__ __forceinline__ uint32_t quest_key32(float s) {
@@ -158,7 +159,7 @@ __device__ __forceinline__ float quest_key32_value(uint32_t k) {
 // first.  Leaves the key in *s_prefix and, in *s_remaining, how many keys EQUAL to it belong to the `need`
 // largest (keys above it all do).  The lanes of a warp with the same digit add to the histogram once: the
 // scores of a row share their upper bytes, so most keys of a pass fall into one or two bins.
-template <typename KeyT>
+template <typename KeyT, int NTHR>
 __device__ __forceinline__ void quest_radix_threshold(const KeyT* keys, int n, int need, int* hist,
                                                       unsigned long long* s_prefix, int* s_remaining) {
   const int tid = threadIdx.x;
@@ -167,16 +168,31 @@ __device__ __forceinline__ void quest_radix_threshold(const KeyT* keys, int n, i
     *s_remaining = need;
   }
   for (int pass = (int)sizeof(KeyT) - 1; pass >= 0; --pass) {
-    hist[tid] = 0;  // QS_THREADS == 256 bins
+    for (int i = tid; i < 256; i += NTHR) hist[i] = 0;
     __syncthreads();
     const unsigned long long prefix = *s_prefix;
     const int shift = 8 * pass;
     const bool top = pass == (int)sizeof(KeyT) - 1;
-    for (int base = 0; base < n; base += QS_THREADS) {
+    for (int base = 0; base < n; base += NTHR) {
       const int i = base + tid;
       const unsigned long long k = i < n ? (unsigned long long)keys[i] : 0ull;
       const bool in = i < n && (top || (k >> (shift + 8)) == (prefix >> (shift + 8)));
+      // Most keys share their upper bytes and few survive to the lower ones, so a warp's 32 keys are mostly all in
+      // one bin (one addition for the warp) or nearly all out (a handful of additions that cannot collide much);
+      // only a mixed warp pays for the match.
+      const unsigned act = __ballot_sync(0xffffffffu, in);
+      if (act == 0u) continue;
       const int dgt = in ? (int)((k >> shift) & 255ull) : 256 + (tid & 31);  // lanes without a key match nobody
+      if (__popc(act) <= 4) {
+        if (in) atomicAdd(&hist[dgt], 1);
+        continue;
+      }
+      const int lead = __ffs(act) - 1;
+      const int d0 = __shfl_sync(0xffffffffu, dgt, lead);
+      if (__ballot_sync(0xffffffffu, in && dgt == d0) == act) {
+        if ((tid & 31) == lead) atomicAdd(&hist[d0], __popc(act));
+        continue;
+      }
       const unsigned same = __match_any_sync(0xffffffffu, dgt);
       if (in && (tid & 31) == __ffs(same) - 1) atomicAdd(&hist[dgt], __popc(same));
     }
@@ -442,7 +458,10 @@ static void launch_quest_score_mma(const QuestScoreDev& d, int Hkv, cudaStream_t
 // at most w).  Only the pages in between are scored again in float64 (the widening of the extrema to float64
 // is the slow instruction: all pages in float64 took 400 us for a row of 2048 pages) and the missing ones are
 // taken from them by a second radix select on the 64-bit keys, ties to the lower page.
-__global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSelDev p) {
+constexpr int QSEL_THREADS = 128;   // a row of the median sequence has 256 pages: eight warps mostly waited for each other
+constexpr int QSEL_RANK_MAX = 256;  // candidates up to which ranking by counting beats a second radix select
+
+__global__ void __launch_bounds__(QSEL_THREADS) quest_select_kernel(const QuestSelDev p) {
   extern __shared__ __align__(16) unsigned char qsm[];
   const int tid = threadIdx.x, head = blockIdx.x;  // one query head per CTA
   const int Hkv = p.sh.n_kv_heads, Hq = p.sh.n_q_heads, G = Hq / Hkv, hd = p.sh.head_dim, S = p.S;
@@ -454,7 +473,7 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
   unsigned char* cand_sel = reinterpret_cast<unsigned char*>(cand_idx + QS_CAND_CAP);     // [QS_CAND_CAP]
   unsigned char* pflag = cand_sel + QS_CAND_CAP;                                          // [Prow] 1 = the head keeps the page
   __shared__ int hist[256];
-  __shared__ int scan_buf[QS_THREADS / 32];
+  __shared__ int scan_buf[QSEL_THREADS / 32];
   __shared__ unsigned long long s_prefix;
   __shared__ int s_remaining, s_ncand, s_cin;
   pdl_trigger();
@@ -479,10 +498,10 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
     return reinterpret_cast<const uint4*>(meta + quest_meta_offset(ok ? page : 0, kvh, (tok % PAGE) / S, Hkv, S, hd));
   };
 
-  for (int i = tid; i < hd; i += QS_THREADS) qf[i] = p.q_rot[((size_t)b * Hq + head) * hd + i];
+  for (int i = tid; i < hd; i += QSEL_THREADS) qf[i] = p.q_rot[((size_t)b * Hq + head) * hd + i];
   {  // the float32 keys of this head's bounds (quest_score)
     const uint32_t* src = p.keys + ((size_t)b * Hq + head) * p.Prow;
-    for (int pg = tid; pg < P; pg += QS_THREADS) keys[pg] = src[pg];
+    for (int pg = tid; pg < P; pg += QSEL_THREADS) keys[pg] = src[pg];
   }
   if (tid == 0) {
     s_ncand = 0;
@@ -493,7 +512,7 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
   uint32_t tau32 = 0u;
   int rem32 = 0;
   if (!all_pages && n_keep > 0) {
-    quest_radix_threshold<uint32_t>(keys, P, n_keep, hist, &s_prefix, &s_remaining);
+    quest_radix_threshold<uint32_t, QSEL_THREADS>(keys, P, n_keep, hist, &s_prefix, &s_remaining);
     tau32 = (uint32_t)s_prefix;
     rem32 = s_remaining;
   }
@@ -513,10 +532,10 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
   int n_cand = 0, c_in = 0;
   bool overflow = false;
   if (all_pages || only_forced) {
-    for (int pg = tid; pg < P; pg += QS_THREADS) pflag[pg] = (all_pages || keys[pg] == 0xffffffffu) ? 1 : 0;
+    for (int pg = tid; pg < P; pg += QSEL_THREADS) pflag[pg] = (all_pages || keys[pg] == 0xffffffffu) ? 1 : 0;
   } else {
     int my_in = 0;
-    for (int pg = tid; pg < P; pg += QS_THREADS) {
+    for (int pg = tid; pg < P; pg += QSEL_THREADS) {
       bool in, cand;
       classify(pg, in, cand);
       my_in += in ? 1 : 0;
@@ -534,16 +553,16 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
     c_in = s_cin;
     overflow = n_cand > QS_CAND_CAP;
     if (overflow && tid == 0) atomicAdd(p.status + ST_TOK_OVERFLOW, 1);
-    if (n_cand > QS_THREADS && !overflow) {
+    if (n_cand > QSEL_RANK_MAX && !overflow) {
       // a long list goes through the radix select below, whose tie rule (the lower page first) reads the list
       // in page order: listed again, by ordered scans
       int at = 0;
-      for (int base = 0; base < P; base += QS_THREADS) {
+      for (int base = 0; base < P; base += QSEL_THREADS) {
         const int pg = base + tid;
         bool in = false, cand = false;
         if (pg < P) classify(pg, in, cand);
         int tot;
-        const int pos = quest_block_scan(cand ? 1 : 0, tot, scan_buf);
+        const int pos = quest_block_scan<QSEL_THREADS>(cand ? 1 : 0, tot, scan_buf);
         if (cand) cand_idx[at + pos] = pg;
         at += tot;
       }
@@ -560,7 +579,7 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
       const bool minus = sub >= hd / 8;
       const int d0 = (minus ? sub - hd / 8 : sub) * 8;
       const float* q = qf + d0;
-      const int stride = (QS_THREADS / 32) * GPW;
+      const int stride = (QSEL_THREADS / 32) * GPW;
       for (int c0 = 0; c0 < n_cand; c0 += stride) {  // block-uniform trip count
         const int c = c0 + warp * GPW + grp;
         bool ok = true;
@@ -584,45 +603,47 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
     if (tid == 0) atomicAdd(p.status + ST_TOK_REFINED, n_cand);
     __syncthreads();
     const int need2 = min(max(n_keep - c_in, 0), n_cand);
-    if (n_cand <= QS_THREADS) {
+    if (n_cand <= QSEL_RANK_MAX) {
       // a short list: a candidate is kept when fewer than need2 others come before it (larger key, or the
       // same key and a lower page)
-      const unsigned long long mine = tid < n_cand ? cand_key[tid] : 0ull;
-      const int my_pg = tid < n_cand ? cand_idx[tid] : 0;
-      int rank = 0;
-      for (int x = 0; x < n_cand; ++x) {
-        const unsigned long long k = cand_key[x];
-        rank += (k > mine || (k == mine && cand_idx[x] < my_pg)) ? 1 : 0;
+      for (int c = tid; c < n_cand; c += QSEL_THREADS) {
+        const unsigned long long mine = cand_key[c];
+        const int my_pg = cand_idx[c];
+        int rank = 0;
+        for (int x = 0; x < n_cand; ++x) {
+          const unsigned long long k = cand_key[x];
+          rank += (k > mine || (k == mine && cand_idx[x] < my_pg)) ? 1 : 0;
+        }
+        if (rank < need2) pflag[my_pg] = 1;
       }
-      if (tid < n_cand && rank < need2) pflag[my_pg] = 1;
     } else {
       unsigned long long tau64 = ~0ull;  // need2 == 0: no candidate key reaches this
       int rem64 = 0;
       if (need2 > 0) {
-        quest_radix_threshold<unsigned long long>(cand_key, n_cand, need2, hist, &s_prefix, &s_remaining);
+        quest_radix_threshold<unsigned long long, QSEL_THREADS>(cand_key, n_cand, need2, hist, &s_prefix, &s_remaining);
         tau64 = s_prefix;
         rem64 = s_remaining;
       }
       // the candidates that are kept, ties in page order
       int seen = 0;
-      for (int base = 0; base < n_cand; base += QS_THREADS) {
+      for (int base = 0; base < n_cand; base += QSEL_THREADS) {
         const int c = base + tid;
         const unsigned long long k = c < n_cand ? cand_key[c] : 0ull;
         const bool eq = c < n_cand && k == tau64;
         int tot;
-        const int rank = quest_block_scan(eq ? 1 : 0, tot, scan_buf);
+        const int rank = quest_block_scan<QSEL_THREADS>(eq ? 1 : 0, tot, scan_buf);
         if (c < n_cand && (k > tau64 || (eq && seen + rank < rem64))) pflag[cand_idx[c]] = 1;
         seen += tot;
       }
     }
   } else if (overflow) {  // float32 order, ties to the lower page
     int seen_equal = 0;
-    for (int base = 0; base < P; base += QS_THREADS) {
+    for (int base = 0; base < P; base += QSEL_THREADS) {
       const int pg = base + tid;
       const uint32_t k = pg < P ? keys[pg] : 0u;
       const bool eq = pg < P && k == tau32;
       int tot;
-      const int rank = quest_block_scan(eq ? 1 : 0, tot, scan_buf);
+      const int rank = quest_block_scan<QSEL_THREADS>(eq ? 1 : 0, tot, scan_buf);
       if (pg < P) pflag[pg] = (k > tau32 || (eq && seen_equal + rank < rem32)) ? 1 : 0;
       seen_equal += tot;
     }
@@ -631,16 +652,16 @@ __global__ void __launch_bounds__(QS_THREADS) quest_select_kernel(const QuestSel
   // ---- the head's byte per page; its ascending page list where the caller asked for it ----
   unsigned char* hm = p.hmask + ((size_t)b * Hq + head) * p.Prow;
   if (p.pages_out == nullptr && p.cnt_out == nullptr) {
-    for (int pg = tid; pg < P; pg += QS_THREADS) hm[pg] = pflag[pg];
+    for (int pg = tid; pg < P; pg += QSEL_THREADS) hm[pg] = pflag[pg];
     return;
   }
   int written = 0;
   int32_t* out = p.pages_out ? p.pages_out + ((size_t)b * Hq + head) * p.Prow : nullptr;
-  for (int base = 0; base < P; base += QS_THREADS) {
+  for (int base = 0; base < P; base += QSEL_THREADS) {
     const int pg = base + tid;
     const bool sel = pg < P && pflag[pg] != 0;
     int tot_sel;
-    const int pos = quest_block_scan(sel ? 1 : 0, tot_sel, scan_buf);
+    const int pos = quest_block_scan<QSEL_THREADS>(sel ? 1 : 0, tot_sel, scan_buf);
     if (pg < P) hm[pg] = sel ? 1 : 0;
     if (sel && out) out[written + pos] = pg;
     written += tot_sel;
@@ -859,11 +880,15 @@ struct QuestLogitMmaDev {
 
 constexpr int QLM_WARPS = 4;
 
-template <int HD, int HG>
+// A warp takes NT runs of 16 list entries per unit and asks for all their rows at once (a lane per run reads the
+// run's list words and issues its copy): with one run per warp and unit, three dependent reads stood before
+// every 2 KB of keys, and the pass reached 3.1 TB/s where the scoring pass of the token selection, which finds
+// its rows without a list, reaches 5.
+template <int HD, int HG, int NT>
 __global__ void __launch_bounds__(QLM_WARPS * 32) quest_logits_mma_kernel(const QuestLogitMmaDev p) {
   extern __shared__ __align__(128) unsigned char qlsm[];
-  constexpr int TILE_BYTES = 16 * HD * 2;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(qlsm + QLM_WARPS * TILE_BYTES);
+  constexpr int TILE_BYTES = 16 * HD * 2, UNIT = 16 * NT * QLM_WARPS;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(qlsm + QLM_WARPS * NT * TILE_BYTES);
   __shared__ int s_cum[QLM_WARPS * 32 + 1], s_wsum[QLM_WARPS];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
   pdl_trigger();
@@ -877,7 +902,7 @@ __global__ void __launch_bounds__(QLM_WARPS * 32) quest_logits_mma_kernel(const 
   if (tid < p.B) {
     int mx = 0;
     for (int h = 0; h < p.Hkv; ++h) mx = max(mx, min(p.kept_cnt[tid * p.Hkv + h], p.Tmax));
-    my_incl = (mx + 16 * QLM_WARPS - 1) / (16 * QLM_WARPS);  // units of the sequence's longest list
+    my_incl = (mx + UNIT - 1) / UNIT;  // units of the sequence's longest list
   }
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -903,20 +928,33 @@ __global__ void __launch_bounds__(QLM_WARPS * 32) quest_logits_mma_kernel(const 
     const int kvh = rem / n_groups, grp = rem - kvh * n_groups;
     const int bk = b * p.Hkv + kvh;
     const int cnt = min(p.kept_cnt[bk], p.Tmax);
-    const int n0 = (grp * QLM_WARPS + warp) * 16;  // this warp's run of list entries
-    if (dead || n0 >= cnt) continue;
-    const int ntok = min(16, cnt - n0);
+    const int w0 = (grp * QLM_WARPS + warp) * NT * 16;  // this warp's NT runs of list entries
+    if (dead || w0 >= cnt) continue;
     const size_t row = (size_t)bk * p.Tmax;
-    const int j0 = p.list_idx[row + n0];
-    const uint32_t r0 = p.list_row[row + n0];
-    if (j0 < 0 || j0 + ntok > p.Tmax || r0 == 0xffffffffu || r0 + (uint32_t)ntok > p.n_rows) {  // checked, not trusted
-      if (lane == 0 && r0 != 0xffffffffu) atomicMax(p.status + 5, 3);
-      continue;
+    unsigned char* tiles = qlsm + warp * NT * TILE_BYTES;
+    // ---- lane i < NT: run i ----
+    int my_j0 = 0, my_ntok = 0;
+    unsigned my_m = 0u;
+    uint32_t my_r0 = 0u;
+    bool my_ok = false;
+    if (lane < NT && w0 + lane * 16 < cnt) {
+      const int n0 = w0 + lane * 16;
+      my_ntok = min(16, cnt - n0);
+      my_j0 = p.list_idx[row + n0];
+      my_r0 = p.list_row[row + n0];
+      my_ok = !(my_j0 < 0 || my_j0 + my_ntok > p.Tmax || my_r0 == 0xffffffffu || my_r0 + (uint32_t)my_ntok > p.n_rows);  // checked, not trusted
+      if (!my_ok && my_r0 != 0xffffffffu) atomicMax(p.status + 5, 3);
     }
-    unsigned char* tile = qlsm + warp * TILE_BYTES;
-    if (lane == 0) {
-      mbar_expect_tx(&bars[warp], ntok * HD * 2);
-      bulk_g2s(tile, static_cast<const uint16_t*>(p.kv.k_pool) + (size_t)r0 * HD, ntok * HD * 2, &bars[warp]);
+    const unsigned okmask = __ballot_sync(0xffffffffu, my_ok);
+    if (okmask == 0u) continue;
+    int bytes = my_ok ? my_ntok * HD * 2 : 0;
+#pragma unroll
+    for (int o = 1; o < NT; o <<= 1) bytes += __shfl_xor_sync(0xffffffffu, bytes, o);
+    if (lane == 0) mbar_expect_tx(&bars[warp], bytes);
+    __syncwarp();
+    if (my_ok) {
+      bulk_g2s(tiles + lane * TILE_BYTES, static_cast<const uint16_t*>(p.kv.k_pool) + (size_t)my_r0 * HD, my_ntok * HD * 2, &bars[warp]);
+      my_m = p.page_mask[(size_t)bk * p.Pstride + my_j0 / p.S];
     }
     uint4 qf[HG][KS][2];
 #pragma unroll
@@ -928,50 +966,57 @@ __global__ void __launch_bounds__(QLM_WARPS * 32) quest_logits_mma_kernel(const 
         qf[hg][sx][1] = *reinterpret_cast<const uint4*>(qb + (size_t)(8 + g) * HD + sx * 32 + t * 8);
       }
     }
-    const unsigned m = p.page_mask[(size_t)bk * p.Pstride + j0 / p.S];
     if (!mbar_wait(&bars[warp], phase, p.status)) {
       dead = true;
       continue;
     }
     phase ^= 1;
-    const uint32_t tb = smem_u32(tile);
-    uint4 ka[KS][2];
-#pragma unroll
-    for (int sx = 0; sx < KS; ++sx) {
-      ka[sx][0] = lds128(tb + g * (HD * 2) + (sx * 32 + t * 8) * 2);
-      ka[sx][1] = lds128(tb + (g + 8) * (HD * 2) + (sx * 32 + t * 8) * 2);
-    }
-#pragma unroll
-    for (int hg = 0; hg < HG; ++hg) {
-      float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+    for (int i = 0; i < NT; ++i) {
+      if (!((okmask >> i) & 1u)) continue;  // the same for the whole warp
+      const int j0 = __shfl_sync(0xffffffffu, my_j0, i), ntok = __shfl_sync(0xffffffffu, my_ntok, i);
+      const unsigned m = __shfl_sync(0xffffffffu, my_m, i);
+      const uint32_t tb = smem_u32(tiles + i * TILE_BYTES);
+      uint4 ka[KS][2];
 #pragma unroll
       for (int sx = 0; sx < KS; ++sx) {
-        mma_bf16(d0, ka[sx][0].x, ka[sx][1].x, ka[sx][0].y, ka[sx][1].y, qf[hg][sx][0].x, qf[hg][sx][0].y);
-        mma_bf16(d0, ka[sx][0].z, ka[sx][1].z, ka[sx][0].w, ka[sx][1].w, qf[hg][sx][0].z, qf[hg][sx][0].w);
-        mma_bf16(d1, ka[sx][0].x, ka[sx][1].x, ka[sx][0].y, ka[sx][1].y, qf[hg][sx][1].x, qf[hg][sx][1].y);
-        mma_bf16(d1, ka[sx][0].z, ka[sx][1].z, ka[sx][0].w, ka[sx][1].w, qf[hg][sx][1].z, qf[hg][sx][1].w);
+        ka[sx][0] = lds128(tb + g * (HD * 2) + (sx * 32 + t * 8) * 2);
+        ka[sx][1] = lds128(tb + (g + 8) * (HD * 2) + (sx * 32 + t * 8) * 2);
       }
-      // columns 2t, 2t+1 of the first n-tile are head t's high and middle parts; column 2t of the second its low part
-      const float s0 = d0[0] + (d0[1] + d1[0]);  // token g of the run
-      const float s1 = d0[2] + (d0[3] + d1[2]);  // token g + 8
-      const int head = hg * 4 + t;
-      if (head < p.G) {
-        const bool on = (m >> head) & 1u;
-        if (g < ntok) p.logits[(row + j0 + g) * p.G + head] = on ? s0 : -INFINITY;
-        if (g + 8 < ntok) p.logits[(row + j0 + g + 8) * p.G + head] = on ? s1 : -INFINITY;
+#pragma unroll
+      for (int hg = 0; hg < HG; ++hg) {
+        float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int sx = 0; sx < KS; ++sx) {
+          mma_bf16(d0, ka[sx][0].x, ka[sx][1].x, ka[sx][0].y, ka[sx][1].y, qf[hg][sx][0].x, qf[hg][sx][0].y);
+          mma_bf16(d0, ka[sx][0].z, ka[sx][1].z, ka[sx][0].w, ka[sx][1].w, qf[hg][sx][0].z, qf[hg][sx][0].w);
+          mma_bf16(d1, ka[sx][0].x, ka[sx][1].x, ka[sx][0].y, ka[sx][1].y, qf[hg][sx][1].x, qf[hg][sx][1].y);
+          mma_bf16(d1, ka[sx][0].z, ka[sx][1].z, ka[sx][0].w, ka[sx][1].w, qf[hg][sx][1].z, qf[hg][sx][1].w);
+        }
+        // columns 2t, 2t+1 of the first n-tile are head t's high and middle parts; column 2t of the second its low part
+        const float s0 = d0[0] + (d0[1] + d1[0]);  // token g of the run
+        const float s1 = d0[2] + (d0[3] + d1[2]);  // token g + 8
+        const int head = hg * 4 + t;
+        if (head < p.G) {
+          const bool on = (m >> head) & 1u;
+          if (g < ntok) p.logits[(row + j0 + g) * p.G + head] = on ? s0 : -INFINITY;
+          if (g + 8 < ntok) p.logits[(row + j0 + g + 8) * p.G + head] = on ? s1 : -INFINITY;
+        }
       }
     }
-    __syncwarp();  // the tile is rewritten by the next unit's copy
+    __syncwarp();  // the tiles are rewritten by the next unit's copies
   }
 }
 
 template <int HD, int HG>
 static void launch_quest_logits_mma(const QuestLogitMmaDev& d, cudaStream_t st) {
-  const int smem = QLM_WARPS * 16 * HD * 2 + QLM_WARPS * 8 + 32;
-  const long long upper = (long long)((d.Tmax + 16 * QLM_WARPS - 1) / (16 * QLM_WARPS)) * d.Hkv * d.B;
-  const dim3 grid((unsigned)(upper < 32768 ? upper : 32768));
-  ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_logits_mma_kernel<HD, HG>), smem);
-  SOL_LAUNCH("quest_logits", (quest_logits_mma_kernel<HD, HG>), grid, dim3(QLM_WARPS * 32), smem, st, d);
+  constexpr int NT = HD == 64 ? 4 : 2;  // 8 KB of keys per warp and unit
+  const int smem = QLM_WARPS * NT * 16 * HD * 2 + QLM_WARPS * 8 + 32;
+  const long long upper = (long long)((d.Tmax + 16 * NT * QLM_WARPS - 1) / (16 * NT * QLM_WARPS)) * d.Hkv * d.B;
+  const long long cap = (long long)sm_count() * 6 * 4;  // four rounds of the CTAs an SM holds: the CTAs' set-up is not free
+  const dim3 grid((unsigned)(upper < cap ? upper : cap));
+  ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_logits_mma_kernel<HD, HG, NT>), smem);
+  SOL_LAUNCH("quest_logits", (quest_logits_mma_kernel<HD, HG, NT>), grid, dim3(QLM_WARPS * 32), smem, st, d);
 }
 
 void launch_quest_selection(const AttnArgs& a, cudaStream_t st) {
@@ -1005,7 +1050,7 @@ void launch_quest_selection(const AttnArgs& a, cudaStream_t st) {
   d.hmask = a.quest_hmask;
   const int smem = QS_CAND_CAP * (8 + 4 + 1) + d.Prow * (4 + 1) + hd * 4 + 16;
   ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_select_kernel), smem);
-  SOL_LAUNCH("quest_select", quest_select_kernel, dim3(Hq, a.B), dim3(QS_THREADS), smem, st, d);
+  SOL_LAUNCH("quest_select", quest_select_kernel, dim3(Hq, a.B), dim3(QSEL_THREADS), smem, st, d);
   ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_list_kernel), d.Prow * 8);
   SOL_LAUNCH("quest_list", quest_list_kernel, dim3(Hkv, a.B), dim3(QS_THREADS), d.Prow * 8, st, d);
 
