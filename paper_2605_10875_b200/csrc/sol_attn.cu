@@ -1539,8 +1539,7 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   if (sh.token_select == SOL_SELECT_QUEST_PAGES) {
     // the paper's page selection per query head (sol_quest.cu) instead of pass 1 and the token selection; a
     // layer step has just appended a key, so the extrema of its block are taken again first
-    if (a.qkv_f32 != nullptr) launch_quest_meta(sh, a.kv, a.B, false, a.status, st);
-    launch_quest_selection(a, st);
+    launch_quest_selection(a, a.qkv_f32 != nullptr, st);
   } else {
     ScoreDev sd;
     sd.kv = a.kv; sd.Hkv = Hkv; sd.G = G; sd.HG = HG; sd.Tmax = Tmax;

@@ -267,7 +267,7 @@ struct AttnArgs {
 void launch_quest_meta(const sol_shape_t& sh, const sol_kv_t& kv, int B, bool all, int* status, cudaStream_t st);
 // Page scores and selection per query head, union token list + pass-2 work items per (sequence, kv-head), then the
 // logits of the listed tokens (minus infinity for the heads that did not pick the token's page).
-void launch_quest_selection(const AttnArgs& a, cudaStream_t st);
+void launch_quest_selection(const AttnArgs& a, bool update_meta, cudaStream_t st);
 
 // Offsets of the attention scratch inside a buffer, starting at `at` (a multiple of 256).
 struct AttnScratch {

@@ -40,13 +40,12 @@ struct QuestMetaDev {
 
 constexpr int QM_THREADS = 128;
 
-__global__ void __launch_bounds__(QM_THREADS) quest_meta_kernel(const QuestMetaDev p) {
-  const int b = blockIdx.z, kvh = blockIdx.y;
-  pdl_trigger();
-  pdl_wait();  // the newest key is written by the kernel before this one
+// The extrema of the blocks of one cache page of (sequence b, kv-head kvh): all its blocks, or only the one that
+// holds the newest token.  For a block of QM_THREADS threads.
+__device__ __forceinline__ void quest_meta_page(const QuestMetaDev& p, int b, int kvh, int lp_all) {
   const int T = min(max(p.kv.seq_lens[b], 0), p.kv.max_pages_per_seq * PAGE);
   if (T <= 0) return;
-  const int lp = p.all ? (int)blockIdx.x : (T - 1) / PAGE;  // logical cache page
+  const int lp = p.all ? lp_all : (T - 1) / PAGE;  // logical cache page
   if (lp * PAGE >= T) return;
   const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + lp];
   if (page < 0 || page >= p.kv.num_pages) {
@@ -77,6 +76,12 @@ __global__ void __launch_bounds__(QM_THREADS) quest_meta_kernel(const QuestMetaD
     meta[o + dp] = pack_bf16(mx0, mx1);
     meta[o + half + dp] = pack_bf16(-mn0, -mn1);
   }
+}
+
+__global__ void __launch_bounds__(QM_THREADS) quest_meta_kernel(const QuestMetaDev p) {
+  pdl_trigger();
+  pdl_wait();  // the newest key is written by the kernel before this one
+  quest_meta_page(p, blockIdx.z, blockIdx.y, blockIdx.x);
 }
 
 void launch_quest_meta(const sol_shape_t& sh, const sol_kv_t& kv, int B, bool all, int* status, cudaStream_t st) {
@@ -234,6 +239,7 @@ struct QuestScoreDev {
   uint16_t* qsplit;    // [B][Hkv][ceil(G / 4) * 16][2 hd] bf16: the sign-split queries as an operand
   float* l1;           // [B][Hq]: |q|_1
   int* order;          // [B]: the sequences, longest first
+  int update_meta;     // 1: quest_query_kernel first takes the extrema of the block with the step's new key
   int* status;
 };
 
@@ -267,6 +273,11 @@ __global__ void __launch_bounds__(QQ_THREADS) quest_query_kernel(const QuestScor
   if (tid < 8) s_l1[tid] = 0.f;
   __syncthreads();
   pdl_wait();  // the rotated queries come from the kernel before; the scratch below may still be read until then
+  if (p.update_meta) {  // the step's new key is in the cache: the extrema of its block
+    QuestMetaDev m;
+    m.kv = p.kv; m.Hkv = Hkv; m.hd = hd; m.S = p.S; m.all = 0; m.status = p.status;
+    quest_meta_page(m, b, kvh, 0);
+  }
   for (int i = tid; i < G * hd; i += QQ_THREADS) {
     const int gi = i / hd, d = i - gi * hd;
     const float q = p.q_rot[((size_t)b * Hq + kvh * G + gi) * hd + d];
@@ -672,13 +683,14 @@ __global__ void __launch_bounds__(QSEL_THREADS) quest_select_kernel(const QuestS
 // The union of the heads' pages of a (sequence, kv-head): the row's token list (every token of a page some head
 // keeps, ascending), a byte per page that says which heads keep it, and the row's pass-2 work items.
 __global__ void __launch_bounds__(QS_THREADS) quest_list_kernel(const QuestSelDev p) {
-  const int kvh = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int kvh = blockIdx.x, tid = threadIdx.x;
   const int Hkv = p.sh.n_kv_heads, Hq = p.sh.n_q_heads, G = Hq / Hkv, S = p.S;
-  const int bk = b * Hkv + kvh;
   __shared__ int scan_buf[QS_THREADS / 32];
   __shared__ int s_item0;
   pdl_trigger();
   pdl_wait();
+  const int b = p.order[blockIdx.y];  // longest sequences first
+  const int bk = b * Hkv + kvh;
   const int T = min(max(p.kv.seq_lens[b], 0), p.kv.max_pages_per_seq * PAGE);
   const int P = (T + S - 1) / S;
   const int32_t* table = p.kv.page_table + (size_t)b * p.kv.max_pages_per_seq;
@@ -690,33 +702,43 @@ __global__ void __launch_bounds__(QS_THREADS) quest_list_kernel(const QuestSelDe
   extern __shared__ __align__(16) unsigned char qlsm2[];
   int* sel_page = reinterpret_cast<int*>(qlsm2);                          // [Prow]
   uint32_t* sel_row0 = reinterpret_cast<uint32_t*>(sel_page + p.Prow);    // [Prow]
-  int n_sel = 0, n_list = 0;
+  int n_sel = 0;
+  bool last_kept = false;  // thread (P - 1) % QS_THREADS: the sequence's last page, the only one that may be short
   for (int base = 0; base < P; base += QS_THREADS) {
     const int pg = base + tid;
     unsigned char m = 0;
     if (pg < P)
       for (int h = 0; h < G; ++h) m |= (unsigned char)((p.hmask[((size_t)b * Hq + kvh * G + h) * p.Prow + pg] & 1u) << h);
     if (pg < P) p.page_mask[(size_t)bk * p.Pstride + pg] = m;
-    const int ntok = m ? min(S, T - pg * S) : 0;
-    int tot_sel, tot;
+    int tot_sel;
     const int pos = quest_block_scan(m ? 1 : 0, tot_sel, scan_buf);
-    (void)quest_block_scan(ntok, tot, scan_buf);
     if (m) {
+      if (pg == P - 1) last_kept = true;
       const int tok = pg * S, page = table[tok / PAGE];
       const bool ok = page >= 0 && page < p.kv.num_pages;
       sel_page[n_sel + pos] = pg;
       sel_row0[n_sel + pos] = ok ? (uint32_t)((page * Hkv + kvh) * PAGE + (tok % PAGE)) : 0xffffffffu;
     }
     n_sel += tot_sel;
-    n_list += tot;
   }
-  __syncthreads();
-  n_list = min(n_list, p.Tmax);
-  for (int n = tid; n < n_list; n += QS_THREADS) {
-    const int i = n / S, j = n - i * S;
+  // every kept page holds S tokens but the sequence's last, which holds the rest
+  const int n_list = min(n_sel * S - (__syncthreads_or(last_kept ? 1 : 0) ? P * S - T : 0), p.Tmax);
+  // four entries per store: S is a multiple of four, so they are tokens of one page
+  const int sh_s = 31 - __clz(S);  // S is a power of two
+  for (int n = tid * 4; n < n_list; n += QS_THREADS * 4) {
+    const int i = n >> sh_s, j = n & (S - 1);
     const uint32_t r0 = sel_row0[i];
-    p.list_idx[row + n] = sel_page[i] * S + j;
-    p.list_row[row + n] = r0 == 0xffffffffu ? r0 : r0 + j;
+    const int t0 = sel_page[i] * S + j;
+    const bool bad = r0 == 0xffffffffu;
+    if (n + 4 <= n_list) {
+      *reinterpret_cast<int4*>(p.list_idx + row + n) = make_int4(t0, t0 + 1, t0 + 2, t0 + 3);
+      *reinterpret_cast<uint4*>(p.list_row + row + n) = bad ? make_uint4(r0, r0, r0, r0) : make_uint4(r0 + j, r0 + j + 1, r0 + j + 2, r0 + j + 3);
+    } else {
+      for (int e = 0; n + e < n_list; ++e) {
+        p.list_idx[row + n + e] = t0 + e;
+        p.list_row[row + n + e] = bad ? r0 : r0 + j + e;
+      }
+    }
   }
   if (tid == 0) p.kept_cnt[bk] = n_list;
 
@@ -1019,7 +1041,7 @@ static void launch_quest_logits_mma(const QuestLogitMmaDev& d, cudaStream_t st) 
   SOL_LAUNCH("quest_logits", (quest_logits_mma_kernel<HD, HG, NT>), grid, dim3(QLM_WARPS * 32), smem, st, d);
 }
 
-void launch_quest_selection(const AttnArgs& a, cudaStream_t st) {
+void launch_quest_selection(const AttnArgs& a, bool update_meta, cudaStream_t st) {
   const sol_shape_t& sh = a.shape;
   const int Hq = sh.n_q_heads, Hkv = sh.n_kv_heads, hd = sh.head_dim, G = Hq / Hkv, S = sh.quest_page_size;
   const int Tmax = a.kv.max_pages_per_seq * PAGE;
@@ -1030,7 +1052,7 @@ void launch_quest_selection(const AttnArgs& a, cudaStream_t st) {
   sc.B = a.B;
   // the tensor-core kernel wants whole operand rows per cache page (S a power of two up to 64 gives that) and at
   // most 8 heads per kv-head, which the shape check has seen to
-  sc.qsplit = a.quest_qsplit; sc.l1 = a.quest_l1; sc.order = a.quest_order;
+  sc.qsplit = a.quest_qsplit; sc.l1 = a.quest_l1; sc.order = a.quest_order; sc.update_meta = update_meta ? 1 : 0;
   SOL_LAUNCH("quest_query", quest_query_kernel, dim3(Hkv, a.B), dim3(QQ_THREADS), ((G + 3) / 4) * 16 * 2 * hd * 2, st, sc);
   if (hd == 64) {
     if (G <= 4) launch_quest_score_mma<128, 1>(sc, Hkv, st);
