@@ -628,3 +628,37 @@ def decode_step(shape: Shape, layers: Sequence[LayerWeights], kvs: Sequence[Page
         h, tr = decode_layer(shape, w, kv, h, r_permille, p_permille, bits, placement, mlp_prune)
         traces.append(tr)
     return h, traces
+
+
+# ----------------------------------------------------------------------------
+# Periodic KV-cache refresh (Background, paragraph "Episodes and control
+# horizon"): after a horizon of decode steps a fully dense pass over the last
+# n_tokens already-known tokens rebuilds their cache entries; no token is
+# sampled.
+# ----------------------------------------------------------------------------
+
+
+def kv_refresh(shape: Shape, layers: Sequence[LayerWeights], kvs: Sequence[PagedKV], h_in_bf16: np.ndarray):
+    """Dense causal pass over the last n tokens of every sequence, layer by layer.
+
+    h_in_bf16 uint16 [B][n][d]: the layer-0 inputs of the span, oldest first.
+    kvs[l].seq_lens counts the span.  In layer l, span token i (position
+    T - n + i) is one dense decode_layer row whose context ends at its own
+    position: it appends its k, v there and attends to everything before, the
+    span tokens j < i of this layer included (they were rewritten just before),
+    so the stale entries of tokens j > i are never read.  Dense means keep-rate
+    1, prune rate 0, 16 bits.  kvs are modified in place; returns the last
+    layer's outputs, float64 [B][n][d]."""
+    B, n, d = h_in_bf16.shape
+    h = bf16_to_f64(h_in_bf16)
+    r, p, b = [1000] * B, [0] * B, [16] * B
+    for w, kv in zip(layers, kvs):
+        full = np.asarray(kv.seq_lens).copy()
+        assert np.all(full >= n), "a sequence is shorter than the refreshed span"
+        out = np.zeros_like(h)
+        for i in range(n):
+            kv.seq_lens = (full - n + 1 + i).astype(np.int32)
+            out[:, i], _ = decode_layer(shape, w, kv, h[:, i], r, p, b)
+        kv.seq_lens = full
+        h = out
+    return h

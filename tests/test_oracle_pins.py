@@ -781,3 +781,126 @@ def test_checker_near_tie_rule_and_output_bounds():
     assert not checker.outputs_ok(o, o + np.array([0, 0, 0.041, 0]))
     m, rel = checker.output_errors(np.ones(4), np.ones(4) * 1.02)
     assert abs(m - 0.02) < 1e-12 and abs(rel - 0.02) < 1e-12
+
+
+# ---------------------------------------------------------- KV refresh ------
+
+
+def _refresh_case(seed, n, L=2, theta=10000.0):
+    """L small layers, three paged sequences whose last n tokens are to be refreshed, and the span's inputs."""
+    rng = np.random.default_rng(seed)
+    shape, _, _, _ = _layer_case(seed, theta=theta)
+    d, hq, hkv, hd, ff = 32, 4, 2, 8, 48
+    w = lambda *s: synth.to_bf16((rng.standard_normal(s) * 0.2).astype(np.float32))
+    layers = [O.LayerWeights(w((hq + 2 * hkv) * hd, d), w(d, hq * hd), w(ff, d), w(ff, d), w(ff, d),
+                             synth.to_bf16((1 + 0.1 * rng.standard_normal(d)).astype(np.float32)),
+                             synth.to_bf16((1 + 0.1 * rng.standard_normal(d)).astype(np.float32))) for _ in range(L)]
+    lens = np.array([21, 17, n], np.int32)  # the last sequence is nothing but the span
+    n_pages = 6
+    table = rng.permutation(3 * n_pages).astype(np.int32).reshape(3, n_pages)
+    pools = [(synth.to_bf16(rng.standard_normal((3 * n_pages, hkv, 4, hd)).astype(np.float32)),
+              synth.to_bf16(rng.standard_normal((3 * n_pages, hkv, 4, hd)).astype(np.float32))) for _ in range(L)]
+    h_span = synth.to_bf16(rng.standard_normal((3, n, d)).astype(np.float32))
+    return shape, layers, pools, table, lens, h_span
+
+
+def _causal_prefill_layer_torch(shape, W, k_pool, v_pool, table, lens, h):
+    """Textbook causal prefill of one Llama layer over the last n tokens of each sequence, with torch library ops
+    in float64: all n keys and values are written first, then one masked attention call per sequence.
+    h float64 [B][n][d]; returns the outputs and the new pools."""
+    B, n, d = h.shape
+    Hq, Hkv, hd, P = shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.page_size
+    F = torch.nn.functional
+    carried = lambda x: x.to(torch.float32).to(torch.bfloat16).to(torch.float64)
+    as_u16 = lambda x: x.to(torch.float32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+    def rot(x, pos):  # x [n][heads][hd], pos [n]
+        if shape.rope_theta == 0:
+            return x
+        inv = shape.rope_theta ** (-torch.arange(0, hd, 2, dtype=torch.float64) / hd)
+        ang = torch.cat([pos[:, None] * inv, pos[:, None] * inv], dim=-1)[:, None, :]
+        x1, x2 = x[..., : hd // 2], x[..., hd // 2:]
+        return x * torch.cos(ang) + torch.cat([-x2, x1], dim=-1) * torch.sin(ang)
+
+    ht = torch.from_numpy(h)
+    x = carried(F.rms_norm(ht, (d,), t64(W.gamma1), shape.rms_eps))
+    qkv = F.linear(x, t64(W.w_qkv))  # [B][n][...]
+    k_pool, v_pool = k_pool.copy(), v_pool.copy()
+    attn = torch.zeros(B, n, Hq * hd, dtype=torch.float64)
+    for i in range(B):
+        T = int(lens[i])
+        pos = torch.arange(T - n, T, dtype=torch.float64)
+        q = rot(qkv[i, :, : Hq * hd].view(n, Hq, hd), pos)
+        k = rot(qkv[i, :, Hq * hd:(Hq + Hkv) * hd].view(n, Hkv, hd), pos)
+        v = qkv[i, :, (Hq + Hkv) * hd:].view(n, Hkv, hd)
+        for j in range(n):
+            t = T - n + j
+            k_pool[int(table[i, t // P]), :, t % P] = as_u16(k[j])
+            v_pool[int(table[i, t // P]), :, t % P] = as_u16(v[j])
+        pages = [int(table[i, p]) for p in range((T + P - 1) // P)]
+        Kc = t64(np.concatenate([k_pool[p] for p in pages], axis=1)[:, :T])  # [Hkv][T][hd]
+        Vc = t64(np.concatenate([v_pool[p] for p in pages], axis=1)[:, :T])
+        mask = torch.arange(T)[None, :] <= (T - n + torch.arange(n))[:, None]  # query j sees keys up to its own
+        o = F.scaled_dot_product_attention(q.transpose(0, 1)[None], Kc[None].repeat_interleave(Hq // Hkv, 1),
+                                           Vc[None].repeat_interleave(Hq // Hkv, 1), attn_mask=mask)
+        attn[i] = o[0].transpose(0, 1).reshape(n, Hq * hd)
+    h_mid = ht + F.linear(attn, t64(W.w_o))
+    x2 = carried(F.rms_norm(h_mid, (d,), t64(W.gamma2), shape.rms_eps))
+    mlp = (F.silu(F.linear(x2, t64(W.w_gate))) * F.linear(x2, t64(W.w_up))) @ t64(W.w_down_t)
+    return (h_mid + mlp).numpy(), k_pool, v_pool
+
+
+@pytest.mark.parametrize("n,theta", [(1, 10000.0), (5, 10000.0), (8, 0.0)])
+def test_kv_refresh_is_a_textbook_causal_prefill(n, theta):
+    shape, layers, pools, table, lens, h_span = _refresh_case(50 + n, n, theta=theta)
+    kvs = [O.PagedKV(k.copy(), v.copy(), table, lens.copy()) for k, v in pools]
+    out = O.kv_refresh(shape, layers, kvs, h_span)
+    h = O.bf16_to_f64(h_span)
+    for l, W in enumerate(layers):
+        h, k_ref, v_ref = _causal_prefill_layer_torch(shape, W, pools[l][0], pools[l][1], table, lens, h)
+        # cache entries agree up to the double rounding of the torch path (float64 -> float32 -> bf16)
+        assert np.max(np.abs(kvs[l].k_pool.astype(np.int64) - k_ref.astype(np.int64))) <= 1
+        assert np.max(np.abs(kvs[l].v_pool.astype(np.int64) - v_ref.astype(np.int64))) <= 1
+        assert np.mean(kvs[l].k_pool != k_ref) < 2e-3
+    assert np.allclose(out, h, rtol=1e-9, atol=1e-9)
+    assert all(np.array_equal(kv.seq_lens, lens) for kv in kvs)
+
+
+def test_kv_refresh_restores_the_dense_cache_after_polluted_steps():
+    """The paper's purpose of the refresh: n decode steps under aggressive actions leave cache entries that
+    differ from the dense ones; the refresh over the same n tokens rebuilds exactly what n dense steps write."""
+    n = 4
+    shape, layers, pools, table, lens, h_span = _refresh_case(60, n)
+    B = 3
+    dense_kvs = [O.PagedKV(k.copy(), v.copy(), table, lens.copy()) for k, v in pools]
+    dirty_kvs = [O.PagedKV(k.copy(), v.copy(), table, lens.copy()) for k, v in pools]
+    dense_out = np.zeros((B, n, 32))
+    for i in range(n):  # token-by-token decode, both ways
+        for kv in dense_kvs + dirty_kvs:
+            kv.seq_lens = (lens - n + 1 + i).astype(np.int32)
+        dense_out[:, i], _ = O.decode_step(shape, layers, dense_kvs, h_span[:, i], [1000] * B, [0] * B, [16] * B)
+        O.decode_step(shape, layers, dirty_kvs, h_span[:, i], [250] * B, [500] * B, [4] * B)
+    for kv in dense_kvs + dirty_kvs:
+        kv.seq_lens = lens.copy()
+    assert any(not np.array_equal(a.k_pool, b.k_pool) for a, b in zip(dense_kvs, dirty_kvs))
+    out = O.kv_refresh(shape, layers, dirty_kvs, h_span)
+    for a, b in zip(dense_kvs, dirty_kvs):
+        assert np.array_equal(a.k_pool, b.k_pool) and np.array_equal(a.v_pool, b.v_pool)
+    assert np.array_equal(out, dense_out)
+    # a second refresh changes nothing
+    before = [(kv.k_pool.copy(), kv.v_pool.copy()) for kv in dirty_kvs]
+    out2 = O.kv_refresh(shape, layers, dirty_kvs, h_span)
+    assert np.array_equal(out, out2)
+    assert all(np.array_equal(kv.k_pool, k) and np.array_equal(kv.v_pool, v) for kv, (k, v) in zip(dirty_kvs, before))
+
+
+def test_kv_refresh_touches_the_span_only():
+    n = 5
+    shape, layers, pools, table, lens, h_span = _refresh_case(61, n)
+    kvs = [O.PagedKV(k.copy(), v.copy(), table, lens.copy()) for k, v in pools]
+    O.kv_refresh(shape, layers, kvs, h_span)
+    want = sorted((int(table[i, t // 4]), t % 4) for i, T in enumerate(lens) for t in range(int(T) - n, int(T)))
+    for l, kv in enumerate(kvs):
+        for new, old in ((kv.k_pool, pools[l][0]), (kv.v_pool, pools[l][1])):
+            changed = sorted(set(map(tuple, np.argwhere((new != old).any(axis=(1, 3))).tolist())))
+            assert changed == want
