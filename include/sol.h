@@ -285,6 +285,23 @@ sol_status_t sol_decode_step_traced(const sol_shape_t *shape, int32_t n_layers, 
                                     const int32_t *bits, const sol_layer_trace_t *traces, void *ws, size_t ws_bytes,
                                     sol_stream_t stream);
 
+/* Periodic KV-cache refresh (Background, paragraph "Episodes and control horizon"): a fully dense pass
+ * (keep-rate 1, prune rate 0, 16 bits) over the last n_tokens already-known tokens of every
+ * sequence that rebuilds their keys and values in all layers; no token is sampled.  Token i of
+ * the span attends to the whole context before it and to tokens 0..i of the span (causal).
+ *   kvs[l].seq_lens  device [B]: lengths INCLUDING the span; each must be >= n_tokens (a shorter
+ *                    sequence raises the bad-action bit of the device status word and leaves
+ *                    that sequence's cache undefined)
+ *   h_in_bf16        device [B][n_tokens][d_model]: the layer-0 inputs of the span, oldest first
+ *   h_out_bf16       optional device [B][n_tokens][d_model]: the last layer's outputs
+ * 1 <= n_tokens <= 128.  The rows of floor(128 / n_tokens) sequences go through the layers
+ * together; the workspace must hold sol_workspace_bytes(shape, min(B, 128 / n_tokens) * n_tokens,
+ * max_pages_per_seq).  In the Quest mode the page extrema of the rewritten blocks are rebuilt.
+ * `layers`, `kvs`: HOST arrays of n_layers structs as in sol_decode_step. */
+sol_status_t sol_kv_refresh(const sol_shape_t *shape, int32_t n_layers, const sol_layer_weights_t *layers,
+                            const sol_kv_t *kvs, int32_t B, int32_t n_tokens, const void *h_in_bf16,
+                            void *h_out_bf16, void *ws, size_t ws_bytes, sol_stream_t stream);
+
 /* The same step for a caller whose per-step data lives on the HOST: h_in,
  * the three action arrays, seq_lens and h_out are host pointers (pinned
  * memory makes the copies of h_in and h_out asynchronous; the four int32

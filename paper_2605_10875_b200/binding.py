@@ -25,7 +25,7 @@ EXPORTS = [
     "sol_status_string", "sol_last_cuda_error", "sol_workspace_bytes", "sol_workspace_init", "sol_quant_act",
     "sol_packed_weight_bytes", "sol_pack_weights", "sol_quant_act_wide", "sol_quest_meta_bytes", "sol_quest_build_meta",
     "sol_sparse_decode_attn", "sol_sparse_decode_attn_static", "sol_pruned_swiglu_mlp", "sol_decode_layer", "sol_decode_step",
-    "sol_decode_step_traced", "sol_decode_step_host", "sol_read_device_status", "sol_selftest_wait_timeout", "sol_timing_enable", "sol_timing_collect",
+    "sol_decode_step_traced", "sol_kv_refresh", "sol_decode_step_host", "sol_read_device_status", "sol_selftest_wait_timeout", "sol_timing_enable", "sol_timing_collect",
     "sol_launch_count",
 ]
 
@@ -113,6 +113,9 @@ def lib() -> C.CDLL:
         L.sol_decode_step_traced.restype = I
         L.sol_decode_step_traced.argtypes = [C.POINTER(SolShape), I, C.POINTER(SolLayerWeights), C.POINTER(SolKV), I,
                                              P, P, P, P, P, P, C.POINTER(SolLayerTrace), P, S, P]
+        L.sol_kv_refresh.restype = I
+        L.sol_kv_refresh.argtypes = [C.POINTER(SolShape), I, C.POINTER(SolLayerWeights), C.POINTER(SolKV), I, I, P, P,
+                                     P, S, P]
         L.sol_selftest_wait_timeout.restype = I
         L.sol_selftest_wait_timeout.argtypes = [P, P]
         L.sol_decode_step_host.restype = I
@@ -306,6 +309,16 @@ def decode_step_traced(shape, layers, kvs, B: int, h_in_bf16, h_out_bf16, h_out_
                                      ws_bytes, _stream(stream))
     if check:
         _check(s, "sol_decode_step_traced")
+    return s
+
+
+def kv_refresh(shape, layers, kvs, B: int, n_tokens: int, h_in_bf16, h_out_bf16, ws, ws_bytes: int, stream=None,
+               check=True) -> int:
+    la, ka = _arrays(layers, kvs)
+    s = lib().sol_kv_refresh(C.byref(shape), len(layers), la, ka, B, n_tokens, _ptr(h_in_bf16), _ptr(h_out_bf16),
+                             _ptr(ws), ws_bytes, _stream(stream))
+    if check:
+        _check(s, "sol_kv_refresh")
     return s
 
 

@@ -94,7 +94,7 @@ void ensure_dynamic_smem(const void* kernel, int bytes) {
 // ---------------------------------------------------------------------------
 struct Layout {
   size_t status, zero_p, stage_h_in, stage_act, stage_h_out, a_op, scale, qkv, attn_hi, attn_lo, attn_f32, h_mid, o_part, g, u, t, t_hi, t_lo, kept_ch, kept_ch_cnt, live, ch_sel, ch_cand_val, ch_cand_idx, ch_keep, down_part,
-      h_a, h_b, total;
+      h_a, h_b, refresh_tab, refresh_act, total;
   AttnScratch attn;
   int chunks, Mpad, Tmax;
 };
@@ -170,6 +170,8 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   L.down_part = take((size_t)L.chunks * Mpad * d * 4);
   L.h_a = take(B * d * 4);
   L.h_b = take(B * d * 4);
+  L.refresh_tab = take((size_t)B * max_pages * 4);  // sol_kv_refresh: a page-table row per refreshed token
+  L.refresh_act = take(4 * (size_t)B * 4);           // ... its length and the dense action
   L.total = at;
   return L;
 }
@@ -648,6 +650,90 @@ sol_status_t sol_decode_step_traced(const sol_shape_t* shape, int32_t n_layers, 
   if (ws_bytes < L.total) return SOL_ERR_WORKSPACE_TOO_SMALL;
   return decode_step_impl(shape, n_layers, layers, kvs, nullptr, B, h_in_bf16, h_out_bf16, h_out_f32, r_permille,
                           p_permille, bits, ws, L, (cudaStream_t)stream, traces);
+}
+
+// ---------------------------------------------------------------------------
+// KV refresh: the last n_tokens tokens of every sequence go through the layers again as rows of one batch,
+// row (s, i) with the page table of sequence s and the length T_s - n_tokens + 1 + i, under the dense action.
+// Every row appends its key and value at its own position before any row's attention reads the cache (the
+// append is a kernel of its own, ahead of the scoring pass), so row i sees the refreshed entries of rows < i:
+// the causal pass the paper describes, on the kernels of the decode step.
+// ---------------------------------------------------------------------------
+__global__ void refresh_expand_kernel(const int32_t* __restrict__ table, const int32_t* __restrict__ seq_lens, int mp,
+                                      int n_tok, int rows, int32_t* __restrict__ out_table,
+                                      int32_t* __restrict__ out_act, int* __restrict__ status) {
+  const int row = blockIdx.x, s = row / n_tok, i = row - s * n_tok;
+  for (int j = threadIdx.x; j < mp; j += blockDim.x) out_table[(size_t)row * mp + j] = table[(size_t)s * mp + j];
+  if (threadIdx.x == 0) {
+    int len = seq_lens[s] - n_tok + 1 + i;
+    if (len < 1) {  // a sequence shorter than the refreshed span: reported, and the row kept inside the cache
+      atomicOr(status + ST_ERR, ERR_BAD_ACTION);
+      len = 1;
+    }
+    out_act[row] = 1000;             // keep-rate
+    out_act[rows + row] = 0;         // prune rate
+    out_act[2 * rows + row] = 16;    // bit-width
+    out_act[3 * rows + row] = len;   // length of the row's context, its own token included
+  }
+}
+
+sol_status_t sol_kv_refresh(const sol_shape_t* shape, int32_t n_layers, const sol_layer_weights_t* layers,
+                            const sol_kv_t* kvs, int32_t B, int32_t n_tokens, const void* h_in_bf16,
+                            void* h_out_bf16, void* ws, size_t ws_bytes, sol_stream_t stream) {
+  int mp = 0;
+  sol_status_t s = step_args_ok(shape, n_layers, layers, kvs, B, &mp);
+  if (s != SOL_OK) return s;
+  if (!h_in_bf16 || !ws || n_tokens < 1) return SOL_ERR_INVALID_ARG;
+  if (n_tokens > 128) return SOL_ERR_UNSUPPORTED;
+  if (B == 0) return SOL_OK;
+  sol_shape_t dense = *shape;
+  dense.token_select = SOL_SELECT_TOKENS;  // every token is kept: no page bounds are needed, and the rows of a
+  dense.quest_page_size = 0;               // sequence would race for the extrema of the block they share
+  const int per = 128 / n_tokens;          // sequences per pass
+  const int rows_max = (B < per ? B : per) * n_tokens;
+  if (ws_bytes < make_layout(dense, rows_max, mp).total) return SOL_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t row_bytes = (size_t)shape->d_model * 2;
+  for (int s0 = 0; s0 < B; s0 += per) {
+    const int ns = B - s0 < per ? B - s0 : per, rows = ns * n_tokens;
+    const Layout L = make_layout(dense, rows, mp);
+    int32_t* tab = at<int32_t>(ws, L.refresh_tab);
+    int32_t* act = at<int32_t>(ws, L.refresh_act);
+    const void* h = static_cast<const unsigned char*>(h_in_bf16) + (size_t)s0 * n_tokens * row_bytes;
+    void* out = h_out_bf16 ? static_cast<unsigned char*>(h_out_bf16) + (size_t)s0 * n_tokens * row_bytes : nullptr;
+    bool in_f32 = false;
+    const int32_t* prev_table = nullptr;
+    const int32_t* prev_lens = nullptr;
+    int prev_mp = 0;
+    for (int l = 0; l < n_layers; ++l) {
+      sol_kv_t kv = kvs[l];
+      if (kv.page_table != prev_table || kv.seq_lens != prev_lens || kv.max_pages_per_seq != prev_mp) {
+        // a plain launch: it starts after everything before it on the stream has ended, and the layer's first
+        // kernel after it
+        refresh_expand_kernel<<<rows, 128, 0, st>>>(kv.page_table + (size_t)s0 * kv.max_pages_per_seq, kv.seq_lens + s0,
+                                                    kv.max_pages_per_seq, n_tokens, rows, tab, act, at<int>(ws, L.status));
+        if (record_cuda_error(cudaGetLastError(), "refresh: page-table rows")) return finish();
+        prev_table = kv.page_table; prev_lens = kv.seq_lens; prev_mp = kv.max_pages_per_seq;
+      }
+      kv.page_table = tab;
+      kv.seq_lens = act + 3 * rows;
+      const bool last = l == n_layers - 1;
+      float* out32 = at<float>(ws, (l & 1) ? L.h_b : L.h_a);
+      run_layer(dense, L, ws, layers[l], kv, rows, h, in_f32, last ? out : nullptr, last && out ? nullptr : out32, act,
+                act + rows, act + 2 * rows, nullptr, st);
+      h = out32;
+      in_f32 = true;
+    }
+    if (shape->token_select == SOL_SELECT_QUEST_PAGES) {  // the extrema of the blocks that hold refreshed keys
+      for (int l = 0; l < n_layers; ++l) {
+        sol_kv_t kv = kvs[l];
+        kv.page_table += (size_t)s0 * kv.max_pages_per_seq;
+        kv.seq_lens += s0;
+        launch_quest_meta_tail(*shape, kv, ns, n_tokens, at<int>(ws, L.status), st);
+      }
+    }
+  }
+  return finish();
 }
 
 // The per-sequence actions and lengths of a step (at most 128 sequences) travel as kernel parameters:

@@ -265,6 +265,8 @@ struct AttnArgs {
 };
 // Quest page extrema of the cache (all pages of the B sequences, or only the block of each sequence's newest token).
 void launch_quest_meta(const sol_shape_t& sh, const sol_kv_t& kv, int B, bool all, int* status, cudaStream_t st);
+// ... the cache pages that hold the last n_tail tokens of each sequence.
+void launch_quest_meta_tail(const sol_shape_t& sh, const sol_kv_t& kv, int B, int n_tail, int* status, cudaStream_t st);
 // Page scores and selection per query head, union token list + pass-2 work items per (sequence, kv-head), then the
 // logits of the listed tokens (minus infinity for the heads that did not pick the token's page).
 void launch_quest_selection(const AttnArgs& a, bool update_meta, cudaStream_t st);

@@ -34,7 +34,8 @@ __host__ __device__ inline size_t quest_meta_offset(int page, int kvh, int qb, i
 // ============================================================================
 struct QuestMetaDev {
   sol_kv_t kv;
-  int Hkv, hd, S, all;
+  int Hkv, hd, S, all;  // all: 0 the block of the newest token, 1 every page, 2 the pages of the last n_tail tokens
+  int n_tail;
   int* status;
 };
 
@@ -45,8 +46,9 @@ constexpr int QM_THREADS = 128;
 __device__ __forceinline__ void quest_meta_page(const QuestMetaDev& p, int b, int kvh, int lp_all) {
   const int T = min(max(p.kv.seq_lens[b], 0), p.kv.max_pages_per_seq * PAGE);
   if (T <= 0) return;
-  const int lp = p.all ? lp_all : (T - 1) / PAGE;  // logical cache page
-  if (lp * PAGE >= T) return;
+  const int lp = p.all == 1 ? lp_all : (T - 1) / PAGE - (p.all == 2 ? lp_all : 0);  // logical cache page
+  if (lp < 0 || lp * PAGE >= T) return;
+  if (p.all == 2 && (lp + 1) * PAGE <= T - p.n_tail) return;  // wholly before the tail
   const int page = p.kv.page_table[(size_t)b * p.kv.max_pages_per_seq + lp];
   if (page < 0 || page >= p.kv.num_pages) {
     if (threadIdx.x == 0) atomicOr(p.status + ST_ERR, ERR_BAD_PAGE);
@@ -84,9 +86,16 @@ __global__ void __launch_bounds__(QM_THREADS) quest_meta_kernel(const QuestMetaD
   quest_meta_page(p, blockIdx.z, blockIdx.y, blockIdx.x);
 }
 
+void launch_quest_meta_tail(const sol_shape_t& sh, const sol_kv_t& kv, int B, int n_tail, int* status, cudaStream_t st) {
+  QuestMetaDev d;
+  d.kv = kv; d.Hkv = sh.n_kv_heads; d.hd = sh.head_dim; d.S = sh.quest_page_size; d.all = 2; d.n_tail = n_tail; d.status = status;
+  const dim3 grid((n_tail + PAGE - 1) / PAGE + 1, sh.n_kv_heads, B);  // n_tail tokens touch that many cache pages at most
+  SOL_LAUNCH("quest_meta", quest_meta_kernel, grid, dim3(QM_THREADS), 0, st, d);
+}
+
 void launch_quest_meta(const sol_shape_t& sh, const sol_kv_t& kv, int B, bool all, int* status, cudaStream_t st) {
   QuestMetaDev d;
-  d.kv = kv; d.Hkv = sh.n_kv_heads; d.hd = sh.head_dim; d.S = sh.quest_page_size; d.all = all ? 1 : 0; d.status = status;
+  d.kv = kv; d.Hkv = sh.n_kv_heads; d.hd = sh.head_dim; d.S = sh.quest_page_size; d.all = all ? 1 : 0; d.n_tail = 0; d.status = status;
   const dim3 grid(all ? kv.max_pages_per_seq : 1, sh.n_kv_heads, B);
   SOL_LAUNCH("quest_meta", quest_meta_kernel, grid, dim3(QM_THREADS), 0, st, d);
 }
@@ -275,7 +284,7 @@ __global__ void __launch_bounds__(QQ_THREADS) quest_query_kernel(const QuestScor
   pdl_wait();  // the rotated queries come from the kernel before; the scratch below may still be read until then
   if (p.update_meta) {  // the step's new key is in the cache: the extrema of its block
     QuestMetaDev m;
-    m.kv = p.kv; m.Hkv = Hkv; m.hd = hd; m.S = p.S; m.all = 0; m.status = p.status;
+    m.kv = p.kv; m.Hkv = Hkv; m.hd = hd; m.S = p.S; m.all = 0; m.n_tail = 0; m.status = p.status;
     quest_meta_page(m, b, kvh, 0);
   }
   for (int i = tid; i < G * hd; i += QQ_THREADS) {
