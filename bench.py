@@ -310,8 +310,24 @@ class Replica:
         n = max(1, len(step_indices))
         return tot / n, {k: v / n for k, v in per_kernel.items()}
 
+    def prepare_refresh(self, n_tokens):
+        """Buffers of the periodic KV-cache refresh over the last n_tokens tokens of every sequence."""
+        t, sol = self.torch, self.sol
+        self.refresh_n = n_tokens
+        rows = min(self.B, 128 // n_tokens) * n_tokens
+        self.refresh_ws_bytes = sol.workspace_bytes(self.shape, rows, self.max_pages)
+        self.refresh_ws = t.empty(self.refresh_ws_bytes, dtype=t.uint8, device=self.device)
+        sol.workspace_init(self.refresh_ws, self.refresh_ws_bytes)
+        span = synth.make_hidden(self.cfg, 7, self.B * n_tokens)
+        self.refresh_h = self._bf16(span).view(self.B, n_tokens, self.cfg["d_model"])
+
+    def refresh(self, i):
+        c, j = i % self.rotate, self.cycle - 1
+        self.sol.kv_refresh(self.shape, [w[c] for w in self.weights], [k[c][j] for k in self.kvs], self.B,
+                            self.refresh_n, self.refresh_h, None, self.refresh_ws, self.refresh_ws_bytes)
+
     def free(self):
-        self.weights = self.kvs = self._keep = self.ws = None
+        self.weights = self.kvs = self._keep = self.ws = self.refresh_ws = None
         self.torch.cuda.empty_cache()
 
 
@@ -564,6 +580,21 @@ def run_ours(args):
             rp.free()
             del rp
 
+    # --- the periodic KV-cache refresh: a dense pass over the last tokens of every sequence of the workload ---
+    refresh = None
+    if args.refresh:
+        rf = Replica(cfg, device, seed=0)
+        rf.prepare_refresh(args.refresh)
+        nr = 3
+        t_ms = max_over_ranks(timed_steps(rf, nr, 2, barrier, rf.refresh)) / nr
+        refresh = {"tokens": args.refresh, "ms_per_refresh": round(t_ms, 3),
+                   "decode_steps_of_the_horizon_ms": round(args.refresh * ms_per_step, 3),
+                   "share_of_horizon": round(t_ms / (t_ms + args.refresh * ms_per_step), 4),
+                   "tokens_per_s": round(world * 1e3 * rf.B * args.refresh / t_ms, 1),
+                   "device_status": sol.read_device_status(rf.refresh_ws)}
+        rf.free()
+        del rf
+
     # --- the same workload with the paper's own token sparsity (Quest pages per query head) ---
     quest = None
     if args.quest:
@@ -600,7 +631,7 @@ def run_ours(args):
             "roofline": roofline, "kernels": per_kernel, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks.summary(), "device_status": status,
             "budget_sweep": sweep, "per_workload": per_workload, "small_batch_prune_sweep": small_batch,
-            "quest_selection": quest,
+            "quest_selection": quest, "kv_refresh": refresh,
         }
         print(json.dumps(line, default=_plain), flush=True)
     ranks.close()
@@ -721,6 +752,8 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="override the workload's layer count (same purpose)")
     ap.add_argument("--quest", type=int, default=16, choices=[0, 4, 8, 16, 32, 64],
                     help="also time the workload with the paper's Quest page selection at this page size (0: skip)")
+    ap.add_argument("--refresh", type=int, default=16,
+                    help="tokens per sequence of the timed KV-cache refresh (the paper's horizon T = 16); 0: skip")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="skip the compact runs of the other workloads")

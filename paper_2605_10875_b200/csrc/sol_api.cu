@@ -200,11 +200,13 @@ static bool kv_ok(const sol_kv_t* kv) {
 static void run_attention(const sol_shape_t& s, const Layout& L, void* ws, const sol_kv_t& kv, int B,
                           const int32_t* r_permille, const float* qkv, int ldq, int qkv_ksplit, const float* qkv_scale,
                           const void* q_bf16, void* out_bf16,
-                          float* out_f32, bool want_split, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t st) {
+                          float* out_f32, bool want_split, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t st,
+                          int span_tokens = 0) {
   AttnArgs a;
   a.shape = s;
   a.kv = kv;
   a.B = B;
+  a.span_tokens = span_tokens;
   a.r_permille = r_permille;
   a.qkv_f32 = qkv;
   a.ldq = ldq;
@@ -324,7 +326,8 @@ static void run_mlp(const sol_shape_t& s, const Layout& L, void* ws, int B, cons
 static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol_layer_weights_t& w,
                       const sol_kv_t& kv, int B, const void* h_in, bool in_f32, void* h_out_bf16, float* h_out_f32,
                       const int32_t* r, const int32_t* p, const int32_t* bits, const sol_layer_trace_t* tr,
-                      cudaStream_t st, const LayerCarry* carry_in = nullptr, LayerCarry* carry_out = nullptr) {
+                      cudaStream_t st, const LayerCarry* carry_in = nullptr, LayerCarry* carry_out = nullptr,
+                      int span_tokens = 0) {
   int* status = at<int>(ws, L.status);
   const int d = s.d_model, Hq = s.n_q_heads, Hkv = s.n_kv_heads, hd = s.head_dim;
   const int Nqkv = (Hq + 2 * Hkv) * hd;
@@ -365,7 +368,8 @@ static void run_layer(const sol_shape_t& s, const Layout& L, void* ws, const sol
   launch_gemm_nk(q, EPI_PARTIAL, st);
 
   run_attention(s, L, ws, kv, B, r, at<float>(ws, L.qkv), Nqkv, nk_ksplit(Nqkv, d), scale, nullptr, nullptr,
-                tr ? tr->attn_out : nullptr, true, tr ? tr->kept_idx : nullptr, tr ? tr->kept_cnt : nullptr, st);
+                tr ? tr->attn_out : nullptr, true, tr ? tr->kept_idx : nullptr, tr ? tr->kept_cnt : nullptr, st,
+                span_tokens);
   if (tr && tr->q_rot)
     cudaMemcpyAsync(tr->q_rot, at<float>(ws, L.attn.q_rot), sizeof(float) * B * Hq * hd, cudaMemcpyDeviceToDevice, st);
 
@@ -656,8 +660,9 @@ sol_status_t sol_decode_step_traced(const sol_shape_t* shape, int32_t n_layers, 
 // KV refresh: the last n_tokens tokens of every sequence go through the layers again as rows of one batch,
 // row (s, i) with the page table of sequence s and the length T_s - n_tokens + 1 + i, under the dense action.
 // Every row appends its key and value at its own position before any row's attention reads the cache (the
-// append is a kernel of its own, ahead of the scoring pass), so row i sees the refreshed entries of rows < i:
-// the causal pass the paper describes, on the kernels of the decode step.
+// append is a kernel of its own, ahead of the attention), so row i sees the refreshed entries of rows < i: the
+// causal pass the paper describes.  The projections and the MLP are the decode step's kernels; the attention of
+// spans up to 16 tokens is the span kernel's (sol_span.cu).
 // ---------------------------------------------------------------------------
 __global__ void refresh_expand_kernel(const int32_t* __restrict__ table, const int32_t* __restrict__ seq_lens, int mp,
                                       int n_tok, int rows, int32_t* __restrict__ out_table,
@@ -719,8 +724,10 @@ sol_status_t sol_kv_refresh(const sol_shape_t* shape, int32_t n_layers, const so
       kv.seq_lens = act + 3 * rows;
       const bool last = l == n_layers - 1;
       float* out32 = at<float>(ws, (l & 1) ? L.h_b : L.h_a);
+      // up to 16 tokens per sequence are the rows of one tensor-core tile of the span attention, which reads a
+      // sequence's cache once for all of them; longer spans go through the decode step's attention row by row
       run_layer(dense, L, ws, layers[l], kv, rows, h, in_f32, last ? out : nullptr, last && out ? nullptr : out32, act,
-                act + rows, act + 2 * rows, nullptr, st);
+                act + rows, act + 2 * rows, nullptr, st, nullptr, nullptr, n_tokens <= 16 ? n_tokens : 0);
       h = out32;
       in_f32 = true;
     }

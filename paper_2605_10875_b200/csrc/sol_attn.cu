@@ -1536,6 +1536,10 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
   pd.max_item_chunks = 1024 / attn_split_len(hd);
   SOL_LAUNCH("attn_prep_rope_append", attn_prep_kernel, dim3(Hkv, a.B), dim3(PREP_THREADS), 0, st, pd);
 
+  if (a.span_tokens > 0) {  // KV refresh: the rows are spans of one sequence's tokens, every token before a row's own is kept
+    launch_span_attention(a, a.span_tokens, st);
+    return;
+  }
   if (sh.token_select == SOL_SELECT_QUEST_PAGES) {
     // the paper's page selection per query head (sol_quest.cu) instead of pass 1 and the token selection; a
     // layer step has just appended a key, so the extrema of its block are taken again first

@@ -215,6 +215,7 @@ struct AttnArgs {
   sol_shape_t shape;
   sol_kv_t kv;
   int B;
+  int span_tokens;  // 0, or: the rows are B / span_tokens spans of consecutive tokens (KV refresh): dense causal attention
   const int32_t* r_permille;
   // inputs of the query preparation: either the split-K partial sums of the QKV projection (layer
   // path: rotate q and k, append k and v) or bf16 q [B][Hq][hd] (stand-alone path: no rotation, no append)
@@ -270,6 +271,8 @@ void launch_quest_meta_tail(const sol_shape_t& sh, const sol_kv_t& kv, int B, in
 // Page scores and selection per query head, union token list + pass-2 work items per (sequence, kv-head), then the
 // logits of the listed tokens (minus infinity for the heads that did not pick the token's page).
 void launch_quest_selection(const AttnArgs& a, bool update_meta, cudaStream_t st);
+// Dense causal attention of spans of n_tok consecutive tokens per sequence, after the query preparation (sol_span.cu).
+void launch_span_attention(const AttnArgs& a, int n_tok, cudaStream_t st);
 
 // Offsets of the attention scratch inside a buffer, starting at `at` (a multiple of 256).
 struct AttnScratch {

@@ -88,6 +88,7 @@ extern "C" sol_status_t sol_sparse_decode_attn_static(const sol_shape_t* shape, 
   a.shape = *shape;
   a.kv = *kv;
   a.B = B;
+  a.span_tokens = 0;
   a.r_permille = r_permille;
   a.qkv_f32 = nullptr;
   a.ldq = 0;

@@ -78,9 +78,27 @@ def test_refresh_sixteen_tokens_two_layers_ragged():
     _check_against_oracle(TINY, 2, [300, 64, 16, 129], 16, seed=3)
 
 
-@pytest.mark.parametrize("n", [1, 4, 7])
+@pytest.mark.parametrize("n", [1, 4, 7, 20])
 def test_refresh_other_span_lengths(n):
+    """Up to 16 tokens the span kernel takes the attention; longer spans go row by row through the decode step's."""
     _check_against_oracle(TINY, 2, [200, 65, n], n, seed=10 + n)
+
+
+def test_refresh_long_ragged_contexts_split_over_ctas():
+    """Contexts of many pages (the span kernel splits them over CTAs), one ending right after a page boundary."""
+    _check_against_oracle(TINY, 1, [5000, 1025, 64 * 30 + 1, 17], 16, seed=71)
+
+
+@pytest.mark.parametrize("hq,hkv", [(4, 1), (2, 2), (8, 1)])
+def test_refresh_head_dim_128_and_other_group_sizes(hq, hkv):
+    """Two layers, so that the second layer's cache entries depend on the first layer's span attention."""
+    cfg = dict(TINY, head_dim=128, n_q_heads=hq, n_kv_heads=hkv)
+    _check_against_oracle(cfg, 2, [300, 70, 2049], 16, seed=81)
+
+
+def test_refresh_group_of_eight_heads_head_dim_64():
+    cfg = dict(TINY, n_q_heads=8, n_kv_heads=1)
+    _check_against_oracle(cfg, 2, [130, 64, 700], 9, seed=83)
 
 
 def test_refresh_more_rows_than_one_pass_takes():
