@@ -587,7 +587,13 @@ def run_ours(args):
         rf.prepare_refresh(args.refresh)
         nr = 3
         t_ms = max_over_ranks(timed_steps(rf, nr, 2, barrier, rf.refresh)) / nr
+        sol.timing_enable(True)
+        timed_steps(rf, 1, 1, barrier, rf.refresh)
+        rows_r = sol.timing_collect()
+        sol.timing_enable(False)
         refresh = {"tokens": args.refresh, "ms_per_refresh": round(t_ms, 3),
+                   "kernels_us_per_launch": {name: round(1e3 * tot / n, 2) for name, n, tot in rows_r},
+                   "kernel_launches_per_refresh": int(sum(n for _, n, _ in rows_r)),
                    "decode_steps_of_the_horizon_ms": round(args.refresh * ms_per_step, 3),
                    "share_of_horizon": round(t_ms / (t_ms + args.refresh * ms_per_step), 4),
                    "tokens_per_s": round(world * 1e3 * rf.B * args.refresh / t_ms, 1),

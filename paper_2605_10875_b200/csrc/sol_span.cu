@@ -28,7 +28,9 @@ namespace sol {
 
 struct SpanDev {
   sol_kv_t kv;  // page_table, seq_lens: one entry per ROW (the rows of a sequence share the table)
-  int Hq, Hkv, G, n_tok, n_seq, nsplit;
+  int Hq, Hkv, G, n_tok, n_seq;
+  int nsplit;  // splits of the longest context the table allows: the stride of `part`; a sequence uses the first ceil(pages / pps)
+  int pps;     // cache pages per split
   float scale_log2;     // log2(e) / sqrt(head_dim)
   const float* q_rot;   // [rows][Hq][hd]
   float* part;          // [rows][Hq][nsplit][hd + 2]: O, m (base-2 domain), l
@@ -50,10 +52,10 @@ __device__ __forceinline__ void span_wait() {
 }
 
 constexpr int SPAN_ROWS = 16;      // query tokens per sequence at most (the rows of one MMA tile)
-constexpr int SPAN_MAX_SPLITS = 16;
+constexpr int SPAN_PAGES = 8;      // cache pages per CTA
 
 template <int HD>
-__global__ void __launch_bounds__(256) span_attn_kernel(const SpanDev p) {
+__global__ void __launch_bounds__(256, HD == 64 ? 2 : 1) span_attn_kernel(const SpanDev p) {
   constexpr int PPR = HD / 8;             // 16-byte pieces per row
   constexpr int TILE = PAGE * HD * 2;     // bytes of a page's keys (or values) of one kv-head
   constexpr int QT = SPAN_ROWS * HD * 2;  // bytes of a head's query tile (one part)
@@ -70,8 +72,8 @@ __global__ void __launch_bounds__(256) span_attn_kernel(const SpanDev p) {
   pdl_wait();  // the rotated queries and the appended keys and values come from the kernel before
   const int T = min(max(p.kv.seq_lens[row0 + n - 1], 0), p.kv.max_pages_per_seq * PAGE);  // the last row sees it all
   const int NP = (T + PAGE - 1) / PAGE;
-  const int pps = (NP + p.nsplit - 1) / p.nsplit;
-  const int pg0 = split * pps, pg1 = min(NP, pg0 + pps);
+  const int pg0 = split * p.pps, pg1 = min(NP, pg0 + p.pps);
+  if (pg0 >= pg1) return;  // the sequence ends before this split (the combine step knows how many it has)
   const int32_t* table = p.kv.page_table + (size_t)row0 * p.kv.max_pages_per_seq;
 
   // a page's keys and values into stage st: piece c of token r sits at piece c ^ (r & 7) of its row
@@ -93,7 +95,7 @@ __global__ void __launch_bounds__(256) span_attn_kernel(const SpanDev p) {
       span_cp16(vd + off, vsrc + (size_t)r * HD + c * 8, valid);
     }
   };
-  if (pg0 < pg1) request(pg0, 0);
+  request(pg0, 0);
   span_commit();
 
   // ---- this warp's queries as bf16 high and low parts, rows beyond the span zero ----
@@ -256,10 +258,13 @@ __global__ void __launch_bounds__(HD / 2) span_combine_kernel(const SpanDev p) {
   pdl_trigger();
   pdl_wait();
   const float* src = p.part + ((size_t)row * p.Hq + head) * p.nsplit * (HD + 2);
+  const int s_last = (row / p.n_tok) * p.n_tok + p.n_tok - 1;  // the sequence's last row sees all of its context
+  const int T = min(max(p.kv.seq_lens[s_last], 0), p.kv.max_pages_per_seq * PAGE);
+  const int ns = min(p.nsplit, ((T + PAGE - 1) / PAGE + p.pps - 1) / p.pps);  // the splits that wrote a share
   float m = -INFINITY;
-  for (int sidx = 0; sidx < p.nsplit; ++sidx) m = fmaxf(m, src[sidx * (HD + 2) + HD]);
+  for (int sidx = 0; sidx < ns; ++sidx) m = fmaxf(m, src[sidx * (HD + 2) + HD]);
   float l = 0.f, o0 = 0.f, o1 = 0.f;
-  for (int sidx = 0; sidx < p.nsplit; ++sidx) {
+  for (int sidx = 0; sidx < ns; ++sidx) {
     const float ms = src[sidx * (HD + 2) + HD];
     if (ms == -INFINITY) continue;  // a split that saw no token of this row
     const float w = exp2f(ms - m);
@@ -297,12 +302,13 @@ void launch_span_attention(const AttnArgs& a, int n_tok, cudaStream_t st) {
   SpanDev d;
   d.kv = a.kv;
   d.Hq = sh.n_q_heads; d.Hkv = sh.n_kv_heads; d.G = d.Hq / d.Hkv; d.n_tok = n_tok; d.n_seq = a.B / n_tok;
-  // splits: about three CTAs per SM over the (sequence, kv-head) pairs; the shares fit the decode path's array of
-  // partial results ([B][Hkv][splits][G][hd + 2])
-  int ns = (3 * sm_count() + d.n_seq * d.Hkv - 1) / (d.n_seq * d.Hkv);
-  ns = ns < 1 ? 1 : ns;
-  ns = ns > SPAN_MAX_SPLITS ? SPAN_MAX_SPLITS : ns;
-  d.nsplit = ns > a.splits ? a.splits : ns;
+  // A CTA takes SPAN_PAGES cache pages of a (sequence, kv-head): contexts of very different lengths then give CTAs
+  // of the same length (a fixed number of splits per sequence left the longest sequence's CTAs running alone:
+  // 100 us per launch where this takes a third).  The shares go to the decode path's array of partial results
+  // ([B][Hkv][splits][G][hd + 2]), which bounds the number of splits.
+  d.pps = SPAN_PAGES;
+  while ((a.kv.max_pages_per_seq + d.pps - 1) / d.pps > a.splits) d.pps *= 2;
+  d.nsplit = (a.kv.max_pages_per_seq + d.pps - 1) / d.pps;
   d.scale_log2 = 1.4426950408889634f / sqrtf((float)sh.head_dim);
   d.q_rot = a.q_rot; d.part = a.part;
   d.out_f32 = a.out_f32; d.out_bf16 = static_cast<uint16_t*>(a.out_bf16); d.out_hi = static_cast<uint16_t*>(a.out_hi);
