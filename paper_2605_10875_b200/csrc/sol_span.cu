@@ -9,7 +9,7 @@
 //
 //   span_attn_kernel     grid (split, kv-head, sequence), a warp per query head of the group.  The CTA walks its
 //                        share of the sequence's cache pages; a page's keys and values (64 tokens) come by
-//                        cp.async into swizzled shared-memory tiles, two stages.  Per page and warp:
+//                        cp.async into swizzled shared-memory tiles, two stages, one barrier per page.  Per page and warp:
 //                        S = Q K^T on mma.sync m16n8k16 with Q as bf16 high + low parts (the oracle does not
 //                        round q), causal mask, online softmax in the base-2 domain, O += P V with P as bf16
 //                        high + low parts (V through ldmatrix.trans).  Leaves (O, m, l) per row, head and split.
@@ -136,10 +136,12 @@ __global__ void __launch_bounds__(256, HD == 64 ? 2 : 1) span_attn_kernel(const 
 #pragma unroll 1
   for (int pg = pg0; pg < pg1; ++pg) {
     const int st = (pg - pg0) & 1;
-    if (pg + 1 < pg1) request(pg + 1, st ^ 1);
-    span_commit();
-    span_wait<1>();  // everything but the newest group has landed: this page's tiles
-    __syncthreads();
+    span_wait<0>();   // this thread's pieces of the page have landed ...
+    __syncthreads();  // ... and everybody's; and every warp is done with the other stage (the page before)
+    if (pg + 1 < pg1) {
+      request(pg + 1, st ^ 1);  // travels while this page is worked on
+      span_commit();
+    }
     const uint32_t kb = smem_u32(kt + st * TILE), vb = smem_u32(vt + st * TILE);
 
     // ---- S = Q K^T for 64 tokens: 8 n-tiles, two k-steps (32 dims) per pass ----
@@ -228,9 +230,7 @@ __global__ void __launch_bounds__(256, HD == 64 ? 2 : 1) span_attn_kernel(const 
         mma_bf16(o[2 * j2 + 1], pl[0], pl[1], pl[2], pl[3], b[2], b[3]);
       }
     }
-    __syncthreads();  // the stage is rewritten by the request of the page after next
   }
-  span_wait<0>();
   l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
   l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
   l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
