@@ -187,3 +187,53 @@ def test_refresh_refuses_bad_arguments_and_reports_short_sequences():
     assert sol.kv_refresh(shape, *args, 4, h, None, ws.buf, ws.bytes, check=False) == 0
     torch.cuda.synchronize()
     assert ws.status()[0] & 4
+
+
+def test_horizon_of_decode_steps_then_refresh_then_decode():
+    """The paper's cycle at a small scale: a horizon of decode steps under sparse actions, the refresh over the
+    horizon's tokens, then the next decode step.  Each phase is compared with the oracle run on the cache the
+    GPU produced so far (a selection may legally differ after a one-ulp difference upstream)."""
+    n, L, B = 4, 2, 3
+    shape, oshape, ws_, pools, table, lens, dws, dkvs, h_span = _case(TINY, L, [300, 68, 129], n, 91)
+    lens_after = lens + 1
+    # room for one more token: a page table with a spare slot
+    table2, n_pages = synth.make_page_table(lens, True, 91, spare_tokens=1)
+    pools = [synth.make_kv_pool(TINY, n_pages, 91, l) for l in range(L)]
+    dkvs = [H.device_kv(k, v, table2, lens) for (k, v) in pools]
+    ow = [H.oracle_weights(w) for w in ws_]
+    ws = H.Workspace(shape, B, dkvs[0].max_pages)
+    out = torch.zeros((B, TINY["d_model"]), dtype=torch.bfloat16, device=H.DEV)
+    r, p, b = [250, 500, 125], [500, 250, 750], [4, 8, 4]
+    for i in range(n):  # the horizon
+        step_lens = lens - n + 1 + i
+        for k in dkvs:
+            k.seq_lens.copy_(H.dev_i32(step_lens))
+        host = [k.to_oracle() for k in dkvs]
+        sol.decode_step(shape, [w.struct() for w in dws], [k.struct() for k in dkvs], B, H.dev_bf16(h_span[:, i]), out,
+                        None, H.dev_i32(r), H.dev_i32(p), H.dev_i32(b), ws.buf, ws.bytes)
+        torch.cuda.synchronize()
+        okvs = [O.PagedKV(k.k_pool, k.v_pool, k.page_table, step_lens.astype(np.int32)) for k in host]
+        out_o, _ = O.decode_step(oshape, ow, okvs, h_span[:, i], r, p, b)
+        H.assert_outputs(out_o, synth.bf16_to_f32(H.host_u16(out)).astype(np.float64), f"horizon step {i}")
+    # the refresh over the horizon's tokens
+    for k in dkvs:
+        k.seq_lens.copy_(H.dev_i32(lens))
+    host = [k.to_oracle() for k in dkvs]
+    _refresh_gpu(shape, dws, dkvs, B, n, h_span, want_out=False)
+    okvs = [O.PagedKV(k.k_pool, k.v_pool, k.page_table, lens.copy()) for k in host]
+    O.kv_refresh(oshape, ow, okvs, h_span)
+    for l in range(L):
+        _assert_cache_close(H.host_u16(dkvs[l].k_pool), okvs[l].k_pool, f"keys of layer {l}")
+        _assert_cache_close(H.host_u16(dkvs[l].v_pool), okvs[l].v_pool, f"values of layer {l}")
+    # the next decode step reads the refreshed cache
+    for k in dkvs:
+        k.seq_lens.copy_(H.dev_i32(lens_after))
+    host = [k.to_oracle() for k in dkvs]
+    h_next = synth.make_hidden(TINY, 92, B)
+    sol.decode_step(shape, [w.struct() for w in dws], [k.struct() for k in dkvs], B, H.dev_bf16(h_next), out, None,
+                    H.dev_i32(r), H.dev_i32(p), H.dev_i32(b), ws.buf, ws.bytes)
+    torch.cuda.synchronize()
+    assert ws.status()[0] == 0
+    okvs = [O.PagedKV(k.k_pool, k.v_pool, k.page_table, lens_after.astype(np.int32)) for k in host]
+    out_o, _ = O.decode_step(oshape, ow, okvs, h_next, r, p, b)
+    H.assert_outputs(out_o, synth.bf16_to_f32(H.host_u16(out)).astype(np.float64), "step after the refresh")
