@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsol.so")
-SOURCES = ["sol_api.cu", "sol_quant.cu", "sol_gemm.cu", "sol_attn.cu", "sol_quest.cu", "sol_mlp.cu", "sol_static.cu", "sol_span.cu"]
+SOURCES = ["sol_api.cu", "sol_quant.cu", "sol_gemm.cu", "sol_attn.cu", "sol_quest.cu", "sol_mlp.cu", "sol_static.cu", "sol_span.cu", "sol_quest_attend.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 

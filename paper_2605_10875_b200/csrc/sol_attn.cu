@@ -1544,6 +1544,8 @@ void launch_attention(const AttnArgs& a, cudaStream_t st) {
     // the paper's page selection per query head (sol_quest.cu) instead of pass 1 and the token selection; a
     // layer step has just appended a key, so the extrema of its block are taken again first
     launch_quest_selection(a, a.qkv_f32 != nullptr, st);
+    launch_quest_attend(a, st);
+    return;
   } else {
     ScoreDev sd;
     sd.kv = a.kv; sd.Hkv = Hkv; sd.G = G; sd.HG = HG; sd.Tmax = Tmax;

@@ -271,6 +271,8 @@ void launch_quest_meta_tail(const sol_shape_t& sh, const sol_kv_t& kv, int B, in
 // Page scores and selection per query head, union token list + pass-2 work items per (sequence, kv-head), then the
 // logits of the listed tokens (minus infinity for the heads that did not pick the token's page).
 void launch_quest_selection(const AttnArgs& a, bool update_meta, cudaStream_t st);
+// Attention over the Quest selection's token lists in one pass (sol_quest_attend.cu), after launch_quest_selection.
+void launch_quest_attend(const AttnArgs& a, cudaStream_t st);
 // Dense causal attention of spans of n_tok consecutive tokens per sequence, after the query preparation (sol_span.cu).
 void launch_span_attention(const AttnArgs& a, int n_tok, cudaStream_t st);
 

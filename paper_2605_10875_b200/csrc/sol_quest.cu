@@ -1085,35 +1085,7 @@ void launch_quest_selection(const AttnArgs& a, bool update_meta, cudaStream_t st
   ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_list_kernel), d.Prow * 8);
   SOL_LAUNCH("quest_list", quest_list_kernel, dim3(Hkv, a.B), dim3(QS_THREADS), d.Prow * 8, st, d);
 
-  QuestLogitDev l;
-  l.kv = a.kv; l.Hq = Hq; l.Hkv = Hkv; l.G = G; l.hd = hd; l.Tmax = Tmax; l.S = S; l.Pstride = d.Pstride;
-  l.q_rot = a.q_rot; l.list_idx = a.list_idx; l.list_row = a.kept_row; l.kept_cnt = a.kept_cnt;
-  l.page_mask = a.page_mask; l.logits = a.logits;
-  l.n_rows = (uint32_t)a.kv.num_pages * Hkv * PAGE; l.status = a.status;
-  if (S % 16 == 0) {  // runs of 16 list entries are runs of 16 cache rows: tensor cores
-    QuestLogitMmaDev m;
-    m.kv = a.kv; m.B = a.B; m.Hq = Hq; m.Hkv = Hkv; m.G = G; m.Tmax = Tmax; m.S = S; m.Pstride = d.Pstride;
-    m.q_split = static_cast<const uint16_t*>(a.q_split); m.list_idx = a.list_idx; m.list_row = a.kept_row;
-    m.kept_cnt = a.kept_cnt; m.page_mask = a.page_mask; m.logits = a.logits;
-    m.n_rows = (uint32_t)a.kv.num_pages * Hkv * PAGE; m.status = a.status;
-    const int HG = (G + 3) / 4;
-    if (hd == 64) {
-      if (HG == 1) launch_quest_logits_mma<64, 1>(m, st);
-      else launch_quest_logits_mma<64, 2>(m, st);
-    } else {
-      if (HG == 1) launch_quest_logits_mma<128, 1>(m, st);
-      else launch_quest_logits_mma<128, 2>(m, st);
-    }
-    return;
-  }
-  const dim3 grid((Tmax + QL_CHUNK - 1) / QL_CHUNK, Hkv, a.B);
-  if (hd == 64) {
-    if (G <= 4) SOL_LAUNCH("quest_logits", (quest_logits_kernel<64, 4>), grid, dim3(QL_THREADS), 0, st, l);
-    else SOL_LAUNCH("quest_logits", (quest_logits_kernel<64, 8>), grid, dim3(QL_THREADS), 0, st, l);
-  } else {
-    if (G <= 4) SOL_LAUNCH("quest_logits", (quest_logits_kernel<128, 4>), grid, dim3(QL_THREADS), 0, st, l);
-    else SOL_LAUNCH("quest_logits", (quest_logits_kernel<128, 8>), grid, dim3(QL_THREADS), 0, st, l);
-  }
+  // the attention over the lists: launch_quest_attend
 }
 
 }  // namespace sol
