@@ -2,21 +2,19 @@
 // "Token sparsity via Quest": "Budgeted token selection", "Quest masking in LLaMA attention", "Granularity").
 //
 //   quest_meta    per block of S tokens of a cache page: the per-dimension maximum of its keys (m+) and the
-//                 negated minimum (m-), as bf16 (extrema of bf16 numbers are bf16 numbers).  Either for every
-//                 page of the sequences (after a prefill) or only for the block of each sequence's newest token
-//                 (after a decode step's append).
+//                 negated minimum (m-), as bf16 (extrema of bf16 numbers are bf16 numbers).  For every page of
+//                 the sequences (after a prefill) or for the pages of a refreshed span.
+//   quest_query   per (sequence, kv-head): the extrema of the block of the key a decode step appended, the G
+//                 heads' queries split by sign as a tensor-core operand, their 1-norms; the sequences by length.
 //   quest_score   the bound q_pos.m+ + q_neg.m- of every page for every query head, in float32, as sortable keys,
-//                 with a bound of its rounding error (a page costs 2/S of its keys' bytes).
+//                 with a bound of its rounding error (a page costs 2/S of its keys' bytes), on the tensor cores.
 //   quest_select  one CTA per (sequence, query head): an exact selection of the head's ceil(b_t / S) best pages: radix
 //                 select on the float32 keys, float64 bounds for the few pages within the error window of the
 //                 threshold (forced pages first, ties to the lower page); a byte per page: kept or not.
-//   quest_list    one CTA per (sequence, kv-head): the union of the group's heads' pages as the row's token list, its
-//                 pass-2 work items, and a byte per page that says which heads keep it.
-//   quest_logits  q.k of every listed token for the G heads (K rows are read only for pages in the union),
-//                 minus infinity for the heads that did not keep the token's page: pass 2 (attn_gather) then
-//                 weighs a token with zero for those heads, which is the paper's additive mask.  On the tensor
-//                 cores when the page size is a multiple of 16 (a run of 16 list entries is then 16 consecutive
-//                 cache rows), on the FMA pipes otherwise.
+//   quest_list    one CTA per (sequence, kv-head): the union of the group's heads' pages as the row's token list
+//                 and a byte per page that says which heads keep it.
+// The attention over the lists (keys and values read only for pages in the union, the paper's additive mask for
+// the heads that did not keep a page) is sol_quest_attend.cu.
 #include <math.h>
 
 #include "sol_common.cuh"
@@ -107,7 +105,7 @@ struct QuestSelDev {
   sol_shape_t sh;
   sol_kv_t kv;
   const int32_t* r_permille;
-  int Tmax, S, splits, split_len, Pstride, Prow;
+  int Tmax, S, Pstride, Prow;
   const float* q_rot;       // [B][Hq][hd]
   const uint32_t* keys;     // [B][Hq][Prow] float32 bounds as keys (quest_score)
   const uint32_t* err;      // [B][Hq] largest error bound of the row, float bits
@@ -119,8 +117,6 @@ struct QuestSelDev {
   int32_t* kept_cnt;        // [B][Hkv] tokens listed
   int32_t* pages_out;       // optional [B][Hq][Prow]
   int32_t* cnt_out;         // optional [B][Hq]
-  int32_t* work_items;
-  int32_t* work_ctr;
   int* status;
 };
 
@@ -690,12 +686,11 @@ __global__ void __launch_bounds__(QSEL_THREADS) quest_select_kernel(const QuestS
 }
 
 // The union of the heads' pages of a (sequence, kv-head): the row's token list (every token of a page some head
-// keeps, ascending), a byte per page that says which heads keep it, and the row's pass-2 work items.
+// keeps, ascending) and a byte per page that says which heads keep it.
 __global__ void __launch_bounds__(QS_THREADS) quest_list_kernel(const QuestSelDev p) {
   const int kvh = blockIdx.x, tid = threadIdx.x;
   const int Hkv = p.sh.n_kv_heads, Hq = p.sh.n_q_heads, G = Hq / Hkv, S = p.S;
   __shared__ int scan_buf[QS_THREADS / 32];
-  __shared__ int s_item0;
   pdl_trigger();
   pdl_wait();
   const int b = p.order[blockIdx.y];  // longest sequences first
@@ -750,304 +745,6 @@ __global__ void __launch_bounds__(QS_THREADS) quest_list_kernel(const QuestSelDe
     }
   }
   if (tid == 0) p.kept_cnt[bk] = n_list;
-
-  // Pass-2 work items of this (sequence, kv-head): runs of `cpi` chunks of split_len listed tokens (at least one
-  // item, so that the output is always written)
-  const int cpi = p.work_ctr[WC_CPI];
-  const int chunks = max(1, (n_list + p.split_len - 1) / p.split_len);
-  const int ns_items = (chunks + cpi - 1) / cpi;
-  __syncthreads();
-  if (tid == 0) s_item0 = atomicAdd(p.work_ctr + WC_ITEMS, ns_items);
-  __syncthreads();
-  const int item0 = s_item0;
-  for (int i = tid; i < ns_items; i += QS_THREADS) {
-    p.work_items[2 * (item0 + i)] = bk * p.splits + i * cpi;  // first chunk of the item
-    p.work_items[2 * (item0 + i) + 1] = n_list;
-  }
-}
-
-// ============================================================================
-// quest_logits
-// ============================================================================
-struct QuestLogitDev {
-  sol_kv_t kv;
-  int Hq, Hkv, G, hd, Tmax, S, Pstride;
-  const float* q_rot;
-  const int32_t* list_idx;
-  const uint32_t* list_row;
-  const int32_t* kept_cnt;
-  const unsigned char* page_mask;
-  float* logits;  // [B][Hkv][Tmax][G]
-  uint32_t n_rows;  // rows of the cache pool
-  int* status;
-};
-
-constexpr int QL_THREADS = 256;
-constexpr int QL_CHUNK = 1024;  // listed tokens per CTA
-
-template <int HD, int GMAX>
-__global__ void __launch_bounds__(QL_THREADS) quest_logits_kernel(const QuestLogitDev p) {
-  // lanes per token: each takes PCS 16-byte pieces of the key row (two when the group has up to four heads: half
-  // as many exchanges per token as with one piece; one for larger groups, whose queries fill the registers)
-  constexpr int PCS = GMAX <= 4 ? 2 : 1;
-  constexpr int LPT = HD / (8 * PCS);
-  constexpr int TPW = 32 / LPT;   // tokens per warp and pass
-  const int kvh = blockIdx.y, b = blockIdx.z, bk = b * p.Hkv + kvh;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, sub = lane % LPT;
-  pdl_trigger();
-  pdl_wait();
-  const int cnt = min(p.kept_cnt[bk], p.Tmax);
-  const int n0 = blockIdx.x * QL_CHUNK;
-  if (n0 >= cnt) return;
-  const int n1 = min(cnt, n0 + QL_CHUNK);
-  float q[GMAX][8 * PCS];  // this lane's dimensions: pieces sub, sub + LPT, ...
-#pragma unroll
-  for (int h = 0; h < GMAX; ++h) {
-#pragma unroll
-    for (int c = 0; c < PCS; ++c) {
-#pragma unroll
-      for (int e = 0; e < 8; ++e)
-        q[h][c * 8 + e] = h < p.G ? p.q_rot[((size_t)b * p.Hq + kvh * p.G + h) * HD + (sub + c * LPT) * 8 + e] : 0.f;
-    }
-  }
-  const size_t row = (size_t)bk * p.Tmax;
-  const uint16_t* kp = static_cast<const uint16_t*>(p.kv.k_pool);
-  // four tokens per lane group and pass; the list words of the next pass are fetched while the key pieces of
-  // this one are in flight, so a pass costs one memory round trip, not two
-  constexpr int UN = 4;
-  constexpr int STEP = (QL_THREADS / 32) * TPW * UN;
-  auto load_list = [&](int nb, int (&jj)[UN], uint32_t (&rr)[UN]) {
-#pragma unroll
-    for (int u = 0; u < UN; ++u) {
-      const int n = nb + u * TPW + lane / LPT;
-      jj[u] = -1;
-      rr[u] = 0xffffffffu;
-      if (n < n1) {
-        jj[u] = p.list_idx[row + n];
-        rr[u] = p.list_row[row + n];
-        if (jj[u] < 0 || jj[u] >= p.Tmax || (rr[u] != 0xffffffffu && rr[u] >= p.n_rows)) {  // checked, not trusted
-          atomicMax(p.status + 5, 2);
-          atomicMax(p.status + 6, jj[u]);
-          jj[u] = -1;
-          rr[u] = 0xffffffffu;
-        }
-      }
-    }
-  };
-  int j[UN], jn[UN];
-  uint32_t r[UN], rn[UN];
-  load_list(n0 + warp * TPW * UN, j, r);
-  for (int nb = n0 + warp * TPW * UN; nb < n1; nb += STEP) {
-    uint4 kv8[UN][PCS];
-#pragma unroll
-    for (int u = 0; u < UN; ++u) {
-#pragma unroll
-      for (int c = 0; c < PCS; ++c) {
-        kv8[u][c] = make_uint4(0u, 0u, 0u, 0u);
-        if (r[u] != 0xffffffffu) kv8[u][c] = *reinterpret_cast<const uint4*>(kp + (size_t)r[u] * HD + (sub + c * LPT) * 8);
-      }
-    }
-    load_list(nb + STEP, jn, rn);
-#pragma unroll
-    for (int u = 0; u < UN; ++u) {
-      float dot[GMAX];
-#pragma unroll
-      for (int h = 0; h < GMAX; ++h) dot[h] = 0.f;
-#pragma unroll
-      for (int c = 0; c < PCS; ++c) {
-        const uint32_t w[4] = {kv8[u][c].x, kv8[u][c].y, kv8[u][c].z, kv8[u][c].w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float k0 = bf16_lo(w[e]), k1 = bf16_hi(w[e]);
-#pragma unroll
-          for (int h = 0; h < GMAX; ++h) dot[h] = fmaf(q[h][c * 8 + 2 * e + 1], k1, fmaf(q[h][c * 8 + 2 * e], k0, dot[h]));
-        }
-      }
-#pragma unroll
-      for (int h = 0; h < GMAX; ++h) {
-#pragma unroll
-        for (int o = 1; o < LPT; o <<= 1) dot[h] += __shfl_xor_sync(0xffffffffu, dot[h], o);
-      }
-      if (j[u] >= 0 && sub == 0) {
-        const unsigned m = r[u] != 0xffffffffu ? p.page_mask[(size_t)bk * p.Pstride + j[u] / p.S] : 0u;
-        float* dst = p.logits + (row + j[u]) * p.G;
-        if (GMAX == 4 && p.G == 4) {
-          *reinterpret_cast<float4*>(dst) = make_float4((m & 1u) ? dot[0] : -INFINITY, (m & 2u) ? dot[1] : -INFINITY,
-                                                        (m & 4u) ? dot[2] : -INFINITY, (m & 8u) ? dot[3] : -INFINITY);
-        } else {
-#pragma unroll
-          for (int h = 0; h < GMAX; ++h)
-            if (h < p.G) dst[h] = ((m >> h) & 1u) ? dot[h] : -INFINITY;
-        }
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < UN; ++u) {
-      j[u] = jn[u];
-      r[u] = rn[u];
-    }
-  }
-}
-
-// ---- the same logits on the tensor cores, for page sizes that are multiples of 16 ----
-// The row's list holds the tokens of its kept pages in ascending order, so with pages of 16, 32 or 64 tokens every
-// run of 16 list entries is 16 consecutive cache rows of one page (only the sequence's last page can be short, and
-// it comes last).  A warp takes such a run: one bulk copy of its key rows, the rows as the M side of m16n8k16 and
-// the query (split into three bf16 parts per head, exact to 2^-24, as in the scoring pass) as the N side.  Units
-// of four runs are numbered along the batch as in the scoring pass: a thread per sequence takes the largest
-// unit count of its kv-heads, the CTA adds them up, and CTAs walk the numbered units.
-struct QuestLogitMmaDev {
-  sol_kv_t kv;
-  int B, Hq, Hkv, G, Tmax, S, Pstride;
-  const uint16_t* q_split;  // bf16 [B][Hkv][HG * 16][hd]
-  const int32_t* list_idx;
-  const uint32_t* list_row;
-  const int32_t* kept_cnt;
-  const unsigned char* page_mask;
-  float* logits;
-  uint32_t n_rows;
-  int* status;
-};
-
-constexpr int QLM_WARPS = 4;
-
-// A warp takes NT runs of 16 list entries per unit and asks for all their rows at once (a lane per run reads the
-// run's list words and issues its copy): with one run per warp and unit, three dependent reads stood before
-// every 2 KB of keys, and the pass reached 3.1 TB/s where the scoring pass of the token selection, which finds
-// its rows without a list, reaches 5.
-template <int HD, int HG, int NT>
-__global__ void __launch_bounds__(QLM_WARPS * 32) quest_logits_mma_kernel(const QuestLogitMmaDev p) {
-  extern __shared__ __align__(128) unsigned char qlsm[];
-  constexpr int TILE_BYTES = 16 * HD * 2, UNIT = 16 * NT * QLM_WARPS;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(qlsm + QLM_WARPS * NT * TILE_BYTES);
-  __shared__ int s_cum[QLM_WARPS * 32 + 1], s_wsum[QLM_WARPS];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
-  pdl_trigger();
-  if (tid == 0) {
-    for (int i = 0; i < QLM_WARPS; ++i) mbar_init(&bars[i], 1);
-    fence_mbar_init();
-    s_cum[0] = 0;
-  }
-  pdl_wait();  // the lists and their lengths come from the selection kernel
-  int my_incl = 0;
-  if (tid < p.B) {
-    int mx = 0;
-    for (int h = 0; h < p.Hkv; ++h) mx = max(mx, min(p.kept_cnt[tid * p.Hkv + h], p.Tmax));
-    my_incl = (mx + UNIT - 1) / UNIT;  // units of the sequence's longest list
-  }
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int x = __shfl_up_sync(0xffffffffu, my_incl, o);
-    if (lane >= o) my_incl += x;
-  }
-  if (lane == 31) s_wsum[warp] = my_incl;
-  __syncthreads();
-  for (int w = 0; w < warp; ++w) my_incl += s_wsum[w];
-  s_cum[tid + 1] = my_incl;
-  __syncthreads();
-  const int n_units = s_cum[p.B] * p.Hkv;
-  const int g = lane >> 2, t = lane & 3;
-  constexpr int KS = HD / 32;
-  uint32_t phase = 0;
-  bool dead = false;
-#pragma unroll 1
-  for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-    const int key = u / p.Hkv;
-    const int b = __syncthreads_count(tid < p.B && my_incl <= key);
-    const int first = s_cum[b], n_groups = s_cum[b + 1] - first;
-    const int rem = u - first * p.Hkv;
-    const int kvh = rem / n_groups, grp = rem - kvh * n_groups;
-    const int bk = b * p.Hkv + kvh;
-    const int cnt = min(p.kept_cnt[bk], p.Tmax);
-    const int w0 = (grp * QLM_WARPS + warp) * NT * 16;  // this warp's NT runs of list entries
-    if (dead || w0 >= cnt) continue;
-    const size_t row = (size_t)bk * p.Tmax;
-    unsigned char* tiles = qlsm + warp * NT * TILE_BYTES;
-    // ---- lane i < NT: run i ----
-    int my_j0 = 0, my_ntok = 0;
-    unsigned my_m = 0u;
-    uint32_t my_r0 = 0u;
-    bool my_ok = false;
-    if (lane < NT && w0 + lane * 16 < cnt) {
-      const int n0 = w0 + lane * 16;
-      my_ntok = min(16, cnt - n0);
-      my_j0 = p.list_idx[row + n0];
-      my_r0 = p.list_row[row + n0];
-      my_ok = !(my_j0 < 0 || my_j0 + my_ntok > p.Tmax || my_r0 == 0xffffffffu || my_r0 + (uint32_t)my_ntok > p.n_rows);  // checked, not trusted
-      if (!my_ok && my_r0 != 0xffffffffu) atomicMax(p.status + 5, 3);
-    }
-    const unsigned okmask = __ballot_sync(0xffffffffu, my_ok);
-    if (okmask == 0u) continue;
-    int bytes = my_ok ? my_ntok * HD * 2 : 0;
-#pragma unroll
-    for (int o = 1; o < NT; o <<= 1) bytes += __shfl_xor_sync(0xffffffffu, bytes, o);
-    if (lane == 0) mbar_expect_tx(&bars[warp], bytes);
-    __syncwarp();
-    if (my_ok) {
-      bulk_g2s(tiles + lane * TILE_BYTES, static_cast<const uint16_t*>(p.kv.k_pool) + (size_t)my_r0 * HD, my_ntok * HD * 2, &bars[warp]);
-      my_m = p.page_mask[(size_t)bk * p.Pstride + my_j0 / p.S];
-    }
-    uint4 qf[HG][KS][2];
-#pragma unroll
-    for (int hg = 0; hg < HG; ++hg) {
-      const uint16_t* qb = p.q_split + ((size_t)(bk * HG + hg) * 16) * HD;
-#pragma unroll
-      for (int sx = 0; sx < KS; ++sx) {
-        qf[hg][sx][0] = *reinterpret_cast<const uint4*>(qb + (size_t)g * HD + sx * 32 + t * 8);
-        qf[hg][sx][1] = *reinterpret_cast<const uint4*>(qb + (size_t)(8 + g) * HD + sx * 32 + t * 8);
-      }
-    }
-    if (!mbar_wait(&bars[warp], phase, p.status)) {
-      dead = true;
-      continue;
-    }
-    phase ^= 1;
-#pragma unroll 1
-    for (int i = 0; i < NT; ++i) {
-      if (!((okmask >> i) & 1u)) continue;  // the same for the whole warp
-      const int j0 = __shfl_sync(0xffffffffu, my_j0, i), ntok = __shfl_sync(0xffffffffu, my_ntok, i);
-      const unsigned m = __shfl_sync(0xffffffffu, my_m, i);
-      const uint32_t tb = smem_u32(tiles + i * TILE_BYTES);
-      uint4 ka[KS][2];
-#pragma unroll
-      for (int sx = 0; sx < KS; ++sx) {
-        ka[sx][0] = lds128(tb + g * (HD * 2) + (sx * 32 + t * 8) * 2);
-        ka[sx][1] = lds128(tb + (g + 8) * (HD * 2) + (sx * 32 + t * 8) * 2);
-      }
-#pragma unroll
-      for (int hg = 0; hg < HG; ++hg) {
-        float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int sx = 0; sx < KS; ++sx) {
-          mma_bf16(d0, ka[sx][0].x, ka[sx][1].x, ka[sx][0].y, ka[sx][1].y, qf[hg][sx][0].x, qf[hg][sx][0].y);
-          mma_bf16(d0, ka[sx][0].z, ka[sx][1].z, ka[sx][0].w, ka[sx][1].w, qf[hg][sx][0].z, qf[hg][sx][0].w);
-          mma_bf16(d1, ka[sx][0].x, ka[sx][1].x, ka[sx][0].y, ka[sx][1].y, qf[hg][sx][1].x, qf[hg][sx][1].y);
-          mma_bf16(d1, ka[sx][0].z, ka[sx][1].z, ka[sx][0].w, ka[sx][1].w, qf[hg][sx][1].z, qf[hg][sx][1].w);
-        }
-        // columns 2t, 2t+1 of the first n-tile are head t's high and middle parts; column 2t of the second its low part
-        const float s0 = d0[0] + (d0[1] + d1[0]);  // token g of the run
-        const float s1 = d0[2] + (d0[3] + d1[2]);  // token g + 8
-        const int head = hg * 4 + t;
-        if (head < p.G) {
-          const bool on = (m >> head) & 1u;
-          if (g < ntok) p.logits[(row + j0 + g) * p.G + head] = on ? s0 : -INFINITY;
-          if (g + 8 < ntok) p.logits[(row + j0 + g + 8) * p.G + head] = on ? s1 : -INFINITY;
-        }
-      }
-    }
-    __syncwarp();  // the tiles are rewritten by the next unit's copies
-  }
-}
-
-template <int HD, int HG>
-static void launch_quest_logits_mma(const QuestLogitMmaDev& d, cudaStream_t st) {
-  constexpr int NT = HD == 64 ? 4 : 2;  // 8 KB of keys per warp and unit
-  const int smem = QLM_WARPS * NT * 16 * HD * 2 + QLM_WARPS * 8 + 32;
-  const long long upper = (long long)((d.Tmax + 16 * NT * QLM_WARPS - 1) / (16 * NT * QLM_WARPS)) * d.Hkv * d.B;
-  const long long cap = (long long)sm_count() * 6 * 4;  // four rounds of the CTAs an SM holds: the CTAs' set-up is not free
-  const dim3 grid((unsigned)(upper < cap ? upper : cap));
-  ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_logits_mma_kernel<HD, HG, NT>), smem);
-  SOL_LAUNCH("quest_logits", (quest_logits_mma_kernel<HD, HG, NT>), grid, dim3(QLM_WARPS * 32), smem, st, d);
 }
 
 void launch_quest_selection(const AttnArgs& a, bool update_meta, cudaStream_t st) {
@@ -1073,11 +770,11 @@ void launch_quest_selection(const AttnArgs& a, bool update_meta, cudaStream_t st
 
   QuestSelDev d;
   d.keys = a.quest_keys; d.err = a.quest_err; d.order = a.quest_order;
-  d.sh = sh; d.kv = a.kv; d.r_permille = a.r_permille; d.Tmax = Tmax; d.S = S; d.splits = a.splits;
-  d.split_len = attn_split_len(hd); d.Pstride = Tmax / 4; d.Prow = Tmax / S;
+  d.sh = sh; d.kv = a.kv; d.r_permille = a.r_permille; d.Tmax = Tmax; d.S = S;
+  d.Pstride = Tmax / 4; d.Prow = Tmax / S;
   d.q_rot = a.q_rot; d.page_mask = a.page_mask; d.list_idx = a.list_idx; d.list_row = a.kept_row;
   d.kept_cnt = a.kept_cnt; d.pages_out = a.quest_pages_out; d.cnt_out = a.quest_cnt_out;
-  d.work_items = a.work_items; d.work_ctr = a.work_ctr; d.status = a.status;
+  d.status = a.status;
   d.hmask = a.quest_hmask;
   const int smem = QS_CAND_CAP * (8 + 4 + 1) + d.Prow * (4 + 1) + hd * 4 + 16;
   ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_select_kernel), smem);
