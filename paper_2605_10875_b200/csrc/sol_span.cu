@@ -251,27 +251,61 @@ __global__ void __launch_bounds__(256, HD == 64 ? 2 : 1) span_attn_kernel(const 
   }
 }
 
-// One (row, query head) per CTA, a thread per pair of dimensions: the splits' shares merged, the row written.
+// One (row, query head) per CTA of 128 threads: the splits' maxima and sums are read side by side (a thread per
+// split), then 128 / (HD / 2) groups of threads each add up every n-th split's share of the output (one thread
+// walking up to 64 splits with dependent reads took twice as long).
+constexpr int SC_THREADS = 128;
+constexpr int SC_MAX_SPLITS = MAX_PAGES_PER_SEQ / SPAN_PAGES;
+
 template <int HD>
-__global__ void __launch_bounds__(HD / 2) span_combine_kernel(const SpanDev p) {
-  const int head = blockIdx.x, row = blockIdx.y, e = threadIdx.x * 2;
+__global__ void __launch_bounds__(SC_THREADS) span_combine_kernel(const SpanDev p) {
+  constexpr int PAIRS = HD / 2, GROUPS = SC_THREADS / PAIRS;
+  __shared__ float s_w[SC_MAX_SPLITS];
+  __shared__ float s_red[SC_THREADS / 32], s_red2[SC_THREADS / 32];
+  __shared__ float2 s_o[GROUPS][PAIRS];
+  const int head = blockIdx.x, row = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   pdl_trigger();
   pdl_wait();
   const float* src = p.part + ((size_t)row * p.Hq + head) * p.nsplit * (HD + 2);
   const int s_last = (row / p.n_tok) * p.n_tok + p.n_tok - 1;  // the sequence's last row sees all of its context
   const int T = min(max(p.kv.seq_lens[s_last], 0), p.kv.max_pages_per_seq * PAGE);
-  const int ns = min(p.nsplit, ((T + PAGE - 1) / PAGE + p.pps - 1) / p.pps);  // the splits that wrote a share
+  const int ns = min(min(p.nsplit, SC_MAX_SPLITS), ((T + PAGE - 1) / PAGE + p.pps - 1) / p.pps);  // the splits that wrote a share
   float m = -INFINITY;
-  for (int sidx = 0; sidx < ns; ++sidx) m = fmaxf(m, src[sidx * (HD + 2) + HD]);
-  float l = 0.f, o0 = 0.f, o1 = 0.f;
-  for (int sidx = 0; sidx < ns; ++sidx) {
+  for (int sidx = tid; sidx < ns; sidx += SC_THREADS) {
     const float ms = src[sidx * (HD + 2) + HD];
-    if (ms == -INFINITY) continue;  // a split that saw no token of this row
-    const float w = exp2f(ms - m);
+    s_w[sidx] = ms;
+    m = fmaxf(m, ms);
+  }
+  m = warp_max(m);
+  if (lane == 0) s_red[warp] = m;
+  __syncthreads();
+  m = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+  float l = 0.f;
+  for (int sidx = tid; sidx < ns; sidx += SC_THREADS) {
+    const float ms = s_w[sidx];
+    const float w = ms == -INFINITY ? 0.f : exp2f(ms - m);  // -inf: a split that saw no token of this row
+    s_w[sidx] = w;
     l += w * src[sidx * (HD + 2) + HD + 1];
+  }
+  l = warp_sum(l);
+  if (lane == 0) s_red2[warp] = l;
+  __syncthreads();
+  l = (s_red2[0] + s_red2[1]) + (s_red2[2] + s_red2[3]);
+  const int gq = tid / PAIRS, e = (tid - gq * PAIRS) * 2;
+  float o0 = 0.f, o1 = 0.f;
+  for (int sidx = gq; sidx < ns; sidx += GROUPS) {
+    const float w = s_w[sidx];
     const float2 v = *reinterpret_cast<const float2*>(src + sidx * (HD + 2) + e);
     o0 += w * v.x;
     o1 += w * v.y;
+  }
+  s_o[gq][tid - gq * PAIRS] = make_float2(o0, o1);
+  __syncthreads();
+  if (gq != 0) return;
+#pragma unroll
+  for (int x = 1; x < GROUPS; ++x) {
+    o0 += s_o[x][tid].x;
+    o1 += s_o[x][tid].y;
   }
   const float inv = l > 0.f ? 1.0f / l : 0.f;
   o0 *= inv;
@@ -293,7 +327,7 @@ static void launch_span(const SpanDev& d, cudaStream_t st) {
   const int smem = 4 * PAGE * HD * 2 + d.G * 2 * SPAN_ROWS * HD * 2;
   ensure_dynamic_smem(reinterpret_cast<const void*>(&span_attn_kernel<HD>), smem);
   SOL_LAUNCH("span_attn", span_attn_kernel<HD>, dim3(d.nsplit, d.Hkv, d.n_seq), dim3(d.G * 32), smem, st, d);
-  SOL_LAUNCH("span_combine", span_combine_kernel<HD>, dim3(d.Hq, d.n_seq * d.n_tok), dim3(HD / 2), 0, st, d);
+  SOL_LAUNCH("span_combine", span_combine_kernel<HD>, dim3(d.Hq, d.n_seq * d.n_tok), dim3(SC_THREADS), 0, st, d);
 }
 
 // After the query preparation of a batch whose rows are n_seq spans of n_tok tokens (1 <= n_tok <= 16).
