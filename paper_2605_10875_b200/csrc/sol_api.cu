@@ -128,7 +128,7 @@ static Layout make_layout(const sol_shape_t& s, int B, int max_pages) {
   Layout L;
   memset(&L, 0, sizeof(L));
   const size_t d = s.d_model, Hq = s.n_q_heads, Hkv = s.n_kv_heads, hd = s.head_dim, ff = s.d_ff;
-  const size_t G = Hq / Hkv, HG = (G + 3) / 4, Nqkv = (Hq + 2 * Hkv) * hd;
+  const size_t Nqkv = (Hq + 2 * Hkv) * hd;
   const size_t Mpad = pad_rows(B), Tmax = (size_t)max_pages * s.page_size;
   L.Mpad = (int)Mpad;
   L.Tmax = (int)Tmax;

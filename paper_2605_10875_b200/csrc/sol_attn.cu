@@ -460,7 +460,6 @@ __global__ void __launch_bounds__(SC_WARPS * 32) attn_score_kernel(const ScoreDe
 // The row's list (token index and page-resolved cache row of every kept token) is what pass 2 reads: segment
 // by segment ascending, the settled candidates last; the order is the same on every run.
 constexpr int TS_THREADS = 256;
-constexpr int TS_MAX_SEGS = MAX_PAGES_PER_SEQ * PAGE / TS_SEG;     // 24
 constexpr float TS_FLT_MAX = 3.402823466e+38f;
 constexpr uint32_t TS_READY = 0x80000000u;
 
@@ -759,20 +758,16 @@ __global__ void __launch_bounds__(TS_THREADS) token_hist_kernel(const SelectDev 
 
 struct ScanSmem {
   SelectSmem sm;
-  double qsum[128];
-  int s_off, s_flag;
+  int s_off;
   int cum[PLAN_STRIDE];
 };
 
 // One (sequence, kv-head, 2048-token segment) of token_scan.
 __device__ __forceinline__ void token_scan_item(const SelectDev& p, ScanSmem& ss, int b, int kvh, int seg) {
   SelectSmem& sm = ss.sm;
-  double* qsum = ss.qsum;
   int& s_off = ss.s_off;
-  int& s_flag = ss.s_flag;
-  const int Hkv = p.sh.n_kv_heads, hd = p.sh.head_dim, G = p.sh.n_q_heads / Hkv;
+  const int Hkv = p.sh.n_kv_heads;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  constexpr int WARPS = TS_THREADS / 32;
   const int bk = b * Hkv + kvh;
   const RowPlan rp = row_plan(p.sh, p.kv, p.r_permille, b);
   const int T = rp.T;
