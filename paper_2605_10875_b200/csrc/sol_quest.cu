@@ -474,9 +474,11 @@ static void launch_quest_score_mma(const QuestScoreDev& d, int Hkv, cudaStream_t
 // at most w).  Only the pages in between are scored again in float64 (the widening of the extrema to float64
 // is the slow instruction: all pages in float64 took 400 us for a row of 2048 pages) and the missing ones are
 // taken from them by a second radix select on the 64-bit keys, ties to the lower page.
-constexpr int QSEL_THREADS = 128;   // a row of the median sequence has 256 pages: eight warps mostly waited for each other
+// QSEL_THREADS: 128 where a row has up to 4096 pages (a row of the median sequence has 256: eight warps mostly
+// waited for each other), 256 for longer rows (small page sizes).
 constexpr int QSEL_RANK_MAX = 256;  // candidates up to which ranking by counting beats a second radix select
 
+template <int QSEL_THREADS>
 __global__ void __launch_bounds__(QSEL_THREADS) quest_select_kernel(const QuestSelDev p) {
   extern __shared__ __align__(16) unsigned char qsm[];
   const int tid = threadIdx.x, head = blockIdx.x;  // one query head per CTA
@@ -777,8 +779,13 @@ void launch_quest_selection(const AttnArgs& a, bool update_meta, cudaStream_t st
   d.status = a.status;
   d.hmask = a.quest_hmask;
   const int smem = QS_CAND_CAP * (8 + 4 + 1) + d.Prow * (4 + 1) + hd * 4 + 16;
-  ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_select_kernel), smem);
-  SOL_LAUNCH("quest_select", quest_select_kernel, dim3(Hq, a.B), dim3(QSEL_THREADS), smem, st, d);
+  if (d.Prow <= 4096) {
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_select_kernel<128>), smem);
+    SOL_LAUNCH("quest_select", quest_select_kernel<128>, dim3(Hq, a.B), dim3(128), smem, st, d);
+  } else {
+    ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_select_kernel<256>), smem);
+    SOL_LAUNCH("quest_select", quest_select_kernel<256>, dim3(Hq, a.B), dim3(256), smem, st, d);
+  }
   ensure_dynamic_smem(reinterpret_cast<const void*>(&quest_list_kernel), d.Prow * 8);
   SOL_LAUNCH("quest_list", quest_list_kernel, dim3(Hkv, a.B), dim3(QS_THREADS), d.Prow * 8, st, d);
 
