@@ -710,22 +710,51 @@ __global__ void __launch_bounds__(QS_THREADS) quest_list_kernel(const QuestSelDe
   uint32_t* sel_row0 = reinterpret_cast<uint32_t*>(sel_page + p.Prow);    // [Prow]
   int n_sel = 0;
   bool last_kept = false;  // thread (P - 1) % QS_THREADS: the sequence's last page, the only one that may be short
-  for (int base = 0; base < P; base += QS_THREADS) {
-    const int pg = base + tid;
-    unsigned char m = 0;
-    if (pg < P)
-      for (int h = 0; h < G; ++h) m |= (unsigned char)((p.hmask[((size_t)b * Hq + kvh * G + h) * p.Prow + pg] & 1u) << h);
-    if (pg < P) p.page_mask[(size_t)bk * p.Pstride + pg] = m;
-    int tot_sel;
-    const int pos = quest_block_scan(m ? 1 : 0, tot_sel, scan_buf);
-    if (m) {
-      if (pg == P - 1) last_kept = true;
-      const int tok = pg * S, page = table[tok / PAGE];
-      const bool ok = page >= 0 && page < p.kv.num_pages;
-      sel_page[n_sel + pos] = pg;
-      sel_row0[n_sel + pos] = ok ? (uint32_t)((page * Hkv + kvh) * PAGE + (tok % PAGE)) : 0xffffffffu;
+  if ((p.Prow & 3) == 0) {
+    // four pages per thread: the heads' bytes come as 32-bit words, and a quarter of the scans
+    for (int base = 0; base < P; base += QS_THREADS * 4) {
+      const int pg0 = base + tid * 4;
+      uint32_t mm = 0;  // the four pages' head masks, a byte each
+      if (pg0 < P) {
+        for (int h = 0; h < G; ++h)
+          mm |= (*reinterpret_cast<const uint32_t*>(p.hmask + ((size_t)b * Hq + kvh * G + h) * p.Prow + pg0) & 0x01010101u) << h;
+        for (int e = 1; e < 4; ++e)
+          if (pg0 + e >= P) mm &= ~(0xffu << (8 * e));  // bytes beyond the sequence's pages are stale
+        *reinterpret_cast<uint32_t*>(p.page_mask + (size_t)bk * p.Pstride + pg0) = mm;
+      }
+      const int cnt = ((mm & 0xffu) ? 1 : 0) + ((mm & 0xff00u) ? 1 : 0) + ((mm & 0xff0000u) ? 1 : 0) + ((mm & 0xff000000u) ? 1 : 0);
+      int tot_sel;
+      int at = n_sel + quest_block_scan(cnt, tot_sel, scan_buf);
+      for (int e = 0; e < 4; ++e) {
+        if (!((mm >> (8 * e)) & 0xffu)) continue;
+        const int pg = pg0 + e;
+        if (pg == P - 1) last_kept = true;
+        const int tok = pg * S, page = table[tok / PAGE];
+        const bool ok = page >= 0 && page < p.kv.num_pages;
+        sel_page[at] = pg;
+        sel_row0[at] = ok ? (uint32_t)((page * Hkv + kvh) * PAGE + (tok % PAGE)) : 0xffffffffu;
+        ++at;
+      }
+      n_sel += tot_sel;
     }
-    n_sel += tot_sel;
+  } else {
+    for (int base = 0; base < P; base += QS_THREADS) {
+      const int pg = base + tid;
+      unsigned char m = 0;
+      if (pg < P)
+        for (int h = 0; h < G; ++h) m |= (unsigned char)((p.hmask[((size_t)b * Hq + kvh * G + h) * p.Prow + pg] & 1u) << h);
+      if (pg < P) p.page_mask[(size_t)bk * p.Pstride + pg] = m;
+      int tot_sel;
+      const int pos = quest_block_scan(m ? 1 : 0, tot_sel, scan_buf);
+      if (m) {
+        if (pg == P - 1) last_kept = true;
+        const int tok = pg * S, page = table[tok / PAGE];
+        const bool ok = page >= 0 && page < p.kv.num_pages;
+        sel_page[n_sel + pos] = pg;
+        sel_row0[n_sel + pos] = ok ? (uint32_t)((page * Hkv + kvh) * PAGE + (tok % PAGE)) : 0xffffffffu;
+      }
+      n_sel += tot_sel;
+    }
   }
   // every kept page holds S tokens but the sequence's last, which holds the rest
   const int n_list = min(n_sel * S - (__syncthreads_or(last_kept ? 1 : 0) ? P * S - T : 0), p.Tmax);
